@@ -1,0 +1,221 @@
+"""CPU oracle (fp64) for head-local weighted affine ridge mapping of KV caches.
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library never imports or calls it, and
+this package imports nothing from the CUDA package.
+
+The arithmetic lives in ``cb_oracle.c`` (plain C loops in fp64, one map per
+OpenMP thread); this file only marshals numpy arrays through ctypes.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "cb_oracle.c")
+_LIB = os.path.join(_HERE, "libcb_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no BLAS, no tuning flags beyond -O2)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.orc_work_list.restype = ctypes.c_int32
+        _lib.orc_ridge_solve.restype = ctypes.c_int32
+        _lib.orc_ridge_centered.restype = ctypes.c_int32
+    return _lib
+
+
+def n_threads() -> int:
+    """Threads the OpenMP loops will use (the cores this process may run on)."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        return int(env)
+    return len(os.sched_getaffinity(0))
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _i64(v) -> ctypes.c_int64:
+    return ctypes.c_int64(int(v))
+
+
+def _i32(v) -> ctypes.c_int32:
+    return ctypes.c_int32(int(v))
+
+
+# ----------------------------------------------------------------------------- bf16
+def bf16_decode(bits: np.ndarray) -> np.ndarray:
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    out = np.empty(bits.shape, dtype=np.float64)
+    _load().orc_bf16_decode(_p(bits), _p(out), _i64(bits.size))
+    return out
+
+
+def bf16_encode(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.empty(x.shape, dtype=np.uint16)
+    _load().orc_bf16_encode(_p(x), _p(out), _i64(x.size))
+    return out
+
+
+# ----------------------------------------------------------------------------- bookkeeping
+def head_map(Ls: int, Hs: int, Lt: int, Ht: int) -> Tuple[np.ndarray, np.ndarray]:
+    """(src_layer[Lt], src_head[Ht]) int32: nearest-depth layer, aligned head."""
+    sl = np.empty(Lt, dtype=np.int32)
+    sh = np.empty(Ht, dtype=np.int32)
+    _load().orc_head_map(_i32(Ls), _i32(Hs), _i32(Lt), _i32(Ht), _p(sl), _p(sh))
+    return sl, sh
+
+
+def work_list(Ls: int, Hs: int, Lt: int, Ht: int, src_layer: np.ndarray, src_head: np.ndarray):
+    """Static gather schedule: (item_comp, item_layer, item_head, item_begin, item_maps)."""
+    src_layer = np.ascontiguousarray(src_layer, dtype=np.int32)
+    src_head = np.ascontiguousarray(src_head, dtype=np.int32)
+    cap = 2 * Ls * Hs
+    ic = np.empty(cap, np.int32)
+    il = np.empty(cap, np.int32)
+    ih = np.empty(cap, np.int32)
+    ib = np.empty(cap + 1, np.int32)
+    im = np.empty(2 * Lt * Ht, np.int32)
+    n = _load().orc_work_list(_i32(Ls), _i32(Hs), _i32(Lt), _i32(Ht), _p(src_layer), _p(src_head),
+                              _p(ic), _p(il), _p(ih), _p(ib), _p(im))
+    return ic[:n].copy(), il[:n].copy(), ih[:n].copy(), ib[:n + 1].copy(), im[:ib[n]].copy()
+
+
+# ----------------------------------------------------------------------------- statistics
+def stats_f64(X: np.ndarray, Y: np.ndarray, w: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """G [p][p], C [p][d] of one map from fp64 rows X, Y [n][d] and weights w [n]."""
+    X = np.ascontiguousarray(X, dtype=np.float64)
+    Y = np.ascontiguousarray(Y, dtype=np.float64)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    n, d = X.shape
+    assert Y.shape == (n, d) and w.shape == (n,)
+    G = np.empty((d + 1, d + 1), np.float64)
+    C = np.empty((d + 1, d), np.float64)
+    _load().orc_stats_f64(_p(X), _p(Y), _p(w), _i64(n), _i32(d), _p(G), _p(C))
+    return G, C
+
+
+def _trace_strides(a: np.ndarray) -> Tuple[int, int, int]:
+    """Element strides (layer, token, head) of a [L][T][H][d] uint16 array with contiguous channels."""
+    assert a.dtype == np.uint16 and a.ndim == 4 and a.strides[3] == 2
+    return a.strides[0] // 2, a.strides[1] // 2, a.strides[2] // 2
+
+
+def stats_traces(src_k: np.ndarray, src_v: np.ndarray, tgt_k: np.ndarray, tgt_v: np.ndarray,
+                 w_k: np.ndarray, w_v: np.ndarray, src_layer: np.ndarray, src_head: np.ndarray,
+                 maps: Optional[Sequence[int]] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Statistics of the selected maps (all by default) from bf16-bit traces [L][T][H][d] (uint16)
+    and fp32 weights [Lt][Ht][T].  Returns fp64 G [n_sel][p][p], C [n_sel][p][d]."""
+    Lt, T, Ht, d = tgt_k.shape
+    assert src_v.shape == src_k.shape and tgt_v.shape == tgt_k.shape and src_k.shape[1] == T
+    assert w_k.dtype == np.float32 and w_v.dtype == np.float32
+    assert w_k.shape == (Lt, Ht, T) and w_v.shape == (Lt, Ht, T)
+    assert w_k.strides[2] == 4 and w_v.strides == w_k.strides
+    src_layer = np.ascontiguousarray(src_layer, dtype=np.int32)
+    src_head = np.ascontiguousarray(src_head, dtype=np.int32)
+    if maps is None:
+        maps = np.arange(2 * Lt * Ht, dtype=np.int32)
+    maps = np.ascontiguousarray(maps, dtype=np.int32)
+    s = _trace_strides(src_k)
+    assert _trace_strides(src_v) == s
+    t = _trace_strides(tgt_k)
+    assert _trace_strides(tgt_v) == t
+    p = d + 1
+    G = np.empty((len(maps), p, p), np.float64)
+    C = np.empty((len(maps), p, d), np.float64)
+    _load().orc_stats_traces(_p(src_k), _p(src_v), _i64(s[0]), _i64(s[1]), _i64(s[2]),
+                             _p(tgt_k), _p(tgt_v), _i64(t[0]), _i64(t[1]), _i64(t[2]),
+                             _p(w_k), _p(w_v), _i64(w_k.strides[0] // 4), _i64(w_k.strides[1] // 4),
+                             _i64(T), _i32(d), _i32(Lt), _i32(Ht), _p(src_layer), _p(src_head),
+                             _p(maps), _i32(len(maps)), _p(G), _p(C))
+    return G, C
+
+
+# ----------------------------------------------------------------------------- ridge
+def ridge_solve(G: np.ndarray, C: np.ndarray, n: int, lam: float, raw_lambda: bool = False):
+    """Theta = [W; b] ([..][p][d]) and info for one map or a batch of maps."""
+    G = np.ascontiguousarray(G, dtype=np.float64)
+    C = np.ascontiguousarray(C, dtype=np.float64)
+    single = G.ndim == 2
+    if single:
+        G, C = G[None], C[None]
+    n_maps, p, _ = G.shape
+    d = p - 1
+    assert C.shape == (n_maps, p, d)
+    Theta = np.empty((n_maps, p, d), np.float64)
+    info = np.empty(n_maps, np.int32)
+    _load().orc_ridge_solve_batch(_p(G), _p(C), _i32(n_maps), _i32(d), _i64(n), ctypes.c_double(lam),
+                                  _i32(1 if raw_lambda else 0), _p(Theta), _p(info))
+    if single:
+        return Theta[0], int(info[0])
+    return Theta, info
+
+
+def ridge_centered(X: np.ndarray, Y: np.ndarray, w: np.ndarray, lam: float):
+    """The centred two-pass estimator with mean-one weights, exactly as the paper writes it."""
+    X = np.ascontiguousarray(X, dtype=np.float64)
+    Y = np.ascontiguousarray(Y, dtype=np.float64)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    n, d = X.shape
+    Theta = np.empty((d + 1, d), np.float64)
+    info = _load().orc_ridge_centered(_p(X), _p(Y), _p(w), _i64(n), _i32(d), ctypes.c_double(lam), _p(Theta))
+    return Theta, int(info)
+
+
+# ----------------------------------------------------------------------------- apply
+def apply_maps(src_k: np.ndarray, src_v: np.ndarray, Theta: np.ndarray, Lt: int, Ht: int,
+               src_layer: np.ndarray, src_head: np.ndarray, maps: Optional[Sequence[int]] = None,
+               want_f64: bool = True, want_bf16: bool = True):
+    """Map a source cache [Ls][T][Hs][d] (bf16 bits) to a target cache [Lt][T][Ht][d].
+    Returns ((K, V) fp64 or None, (K, V) bf16 bits or None); entries of unselected maps are zero."""
+    Ls, T, Hs, d = src_k.shape
+    p = d + 1
+    Theta = np.ascontiguousarray(Theta, dtype=np.float64)
+    assert Theta.shape == (2 * Lt * Ht, p, d)
+    src_layer = np.ascontiguousarray(src_layer, dtype=np.int32)
+    src_head = np.ascontiguousarray(src_head, dtype=np.int32)
+    if maps is None:
+        maps = np.arange(2 * Lt * Ht, dtype=np.int32)
+    maps = np.ascontiguousarray(maps, dtype=np.int32)
+    s = _trace_strides(src_k)
+    assert _trace_strides(src_v) == s
+    shape = (Lt, T, Ht, d)
+    ok = np.zeros(shape, np.float64) if want_f64 else None
+    ov = np.zeros(shape, np.float64) if want_f64 else None
+    bk = np.zeros(shape, np.uint16) if want_bf16 else None
+    bv = np.zeros(shape, np.uint16) if want_bf16 else None
+    _load().orc_apply(_p(src_k), _p(src_v), _i64(s[0]), _i64(s[1]), _i64(s[2]), _i64(T), _i32(d),
+                      _i32(Lt), _i32(Ht), _p(src_layer), _p(src_head), _p(Theta), _p(maps), _i32(len(maps)),
+                      _p(ok), _p(ov), _p(bk), _p(bv), _i64(T * Ht * d), _i64(Ht * d), _i64(d))
+    return ((ok, ov) if want_f64 else None), ((bk, bv) if want_bf16 else None)
+
+
+# ----------------------------------------------------------------------------- artifact size
+def coefficient_counts(Lt: int, Ht: int, Hs: int, k: int, ds: int, dt: int):
+    """Non-bias coefficient counts over K and V (Section 3.2): (C_full, C_local, number of bias entries).
+    C_full = 2 L_t H_t (k H_s d_s) d_t,  C_local = 2 L_t H_t (k d_s) d_t."""
+    c_full = 2 * Lt * Ht * (k * Hs * ds) * dt
+    c_local = 2 * Lt * Ht * (k * ds) * dt
+    n_bias = 2 * Lt * Ht * dt
+    return c_full, c_local, n_bias

@@ -1,0 +1,366 @@
+/*
+ * CPU oracle for head-local weighted affine ridge mapping of KV caches.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition the CUDA
+ * library is checked against.  It shares no code, header, table or helper with
+ * the CUDA path and is never called by it.  Everything is fp64; bf16 inputs are
+ * widened exactly.  Loops are written in the order of the definitions they
+ * follow (no blocking, no fusion) so they can be read against the paper.
+ *
+ * Notation (paper, Section 2.1 and Section 3.1): source model has L_s layers,
+ * H_s KV heads of width d; target has L_t, H_t, d.  "comp" is 0 for keys, 1 for
+ * values.  A map is one (comp, target layer l, target head h); its id is
+ * m = (comp*L_t + l)*H_t + h.  Row-vector convention y_hat = x W + b.
+ *
+ * Pins (see tests/test_oracle_*.py): brute force on hand-checkable integers,
+ * closed forms of the bias row/column, additivity over token splits, weight
+ * scaling, equality with the centred two-pass estimator of Eq. "closedform",
+ * textbook least squares for constant weights, exact recovery of (A, b),
+ * identity recovery for X = Y, the effective-dimension bound, the coefficient
+ * counts of Section 3.2 and the storage figures of Section 4.4.
+ * Parity unpinned by the paper (defined by this build, not by the paper): the
+ * synthetic input laws, the nearest-depth single-layer match (k = 1), and the
+ * lambda_eff = lambda * s_w / n convention for weights that are not mean-one.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* bf16 -> fp64, exact: a bf16 is the upper half of an IEEE binary32. */
+static double orc_bf16(uint16_t v)
+{
+    uint32_t u = ((uint32_t)v) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* fp64 -> bf16, round to nearest even, via binary32 (double rounding avoided by
+ * rounding the fp64 value directly on the bf16 grid). */
+static uint16_t orc_to_bf16(double x)
+{
+    if (x != x) return 0x7fc0;
+    double ax = fabs(x);
+    uint16_t sign = (x < 0.0 || (x == 0.0 && 1.0 / x < 0.0)) ? 0x8000 : 0;
+    if (ax == 0.0) return sign;
+    if (isinf(ax)) return (uint16_t)(sign | 0x7f80);
+    int e;
+    double fr = frexp(ax, &e);        /* ax = fr * 2^e, fr in [0.5, 1) */
+    int E = e - 1;                    /* ax = (2 fr) * 2^E, 2 fr in [1, 2) */
+    if (E < -126) E = -126;           /* subnormal range of bf16 shares binary32's exponent floor */
+    double ulp = ldexp(1.0, E - 7);   /* 8 significant bits */
+    double q = ax / ulp;              /* exact scaling by a power of two */
+    double r = nearbyint(q);          /* default rounding mode: nearest even */
+    double y = r * ulp;
+    if (y >= ldexp(1.0, 128)) return (uint16_t)(sign | 0x7f80);
+    float f = (float)y;               /* exact: y has at most 8 significant bits */
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    (void)fr;
+    return (uint16_t)(sign | (uint16_t)((u >> 16) & 0x7fff));
+}
+
+void orc_bf16_decode(const uint16_t *in, double *out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_bf16(in[i]);
+}
+
+void orc_bf16_encode(const double *in, uint16_t *out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_to_bf16(in[i]);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Head match (Section 3.2: a(h) = h for aligned KV groups; one selected layer */
+/* per target layer, nearest relative depth).                                 */
+/* j(l) = round(l (L_s - 1) / (L_t - 1)) in integers, halves rounded up.       */
+/* ------------------------------------------------------------------------- */
+void orc_head_map(int32_t Ls, int32_t Hs, int32_t Lt, int32_t Ht,
+                  int32_t *src_layer /* [Lt] */, int32_t *src_head /* [Ht] */)
+{
+    for (int32_t l = 0; l < Lt; ++l) {
+        if (Lt == 1) { src_layer[l] = 0; continue; }
+        int64_t num = 2 * (int64_t)l * (Ls - 1) + (Lt - 1);
+        int64_t den = 2 * (int64_t)(Lt - 1);
+        src_layer[l] = (int32_t)(num / den);
+    }
+    for (int32_t h = 0; h < Ht; ++h)
+        src_head[h] = (int32_t)(((int64_t)h * Hs) / Ht);   /* identity when Hs == Ht */
+}
+
+/*
+ * Static gather schedule (Section 2.3): maps grouped by the source head they
+ * read, so the source block is fetched once per group.  Items are ordered by
+ * (comp, source layer, source head); the maps of an item are in ascending id.
+ * Only source heads with at least one map become items.
+ * Returns the number of items; arrays must hold 2*Ls*Hs (items) / 2*Lt*Ht (maps).
+ */
+int32_t orc_work_list(int32_t Ls, int32_t Hs, int32_t Lt, int32_t Ht,
+                      const int32_t *src_layer, const int32_t *src_head,
+                      int32_t *item_comp, int32_t *item_layer, int32_t *item_head,
+                      int32_t *item_begin /* [n_items+1] offsets into item_maps */,
+                      int32_t *item_maps)
+{
+    int32_t n_items = 0, n_listed = 0;
+    for (int32_t comp = 0; comp < 2; ++comp)
+        for (int32_t j = 0; j < Ls; ++j)
+            for (int32_t g = 0; g < Hs; ++g) {
+                int32_t first = n_listed;
+                for (int32_t l = 0; l < Lt; ++l)
+                    for (int32_t h = 0; h < Ht; ++h)
+                        if (src_layer[l] == j && src_head[h] == g)
+                            item_maps[n_listed++] = (comp * Lt + l) * Ht + h;
+                if (n_listed > first) {
+                    item_comp[n_items] = comp;
+                    item_layer[n_items] = j;
+                    item_head[n_items] = g;
+                    item_begin[n_items] = first;
+                    ++n_items;
+                }
+            }
+    item_begin[n_items] = n_listed;
+    return n_items;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Weighted sufficient statistics, augmented form (Section 3.4, Eq. fusedstats */
+/* before centring):                                                          */
+/*   G = sum_t w_t xt_t xt_t^T  (p x p),  C = sum_t w_t xt_t y_t^T  (p x d),   */
+/*   xt_t = [x_t, 1], p = d + 1, bias entry last.                              */
+/* One map, fp64 rows.                                                        */
+/* ------------------------------------------------------------------------- */
+void orc_stats_f64(const double *X /* [n][d] */, const double *Y /* [n][d] */,
+                   const double *w /* [n] */, int64_t n, int32_t d,
+                   double *G /* [p][p] */, double *C /* [p][d] */)
+{
+    const int32_t p = d + 1;
+    double *xt = (double *)malloc(sizeof(double) * (size_t)p);
+    memset(G, 0, sizeof(double) * (size_t)p * p);
+    memset(C, 0, sizeof(double) * (size_t)p * d);
+    for (int64_t t = 0; t < n; ++t) {
+        for (int32_t i = 0; i < d; ++i) xt[i] = X[t * d + i];
+        xt[d] = 1.0;
+        for (int32_t i = 0; i < p; ++i) {
+            const double wx = w[t] * xt[i];
+            for (int32_t j = 0; j < p; ++j) G[(size_t)i * p + j] += wx * xt[j];
+            for (int32_t j = 0; j < d; ++j) C[(size_t)i * d + j] += wx * Y[t * d + j];
+        }
+    }
+    free(xt);
+}
+
+/*
+ * The same statistics for a list of maps read straight from strided bf16 KV
+ * traces (element (layer, token, head, channel) at base + layer*sl + token*st +
+ * head*sh + channel, strides in elements) and fp32 weights
+ * w[comp][l][h][t] at w_comp + l*w_sl + h*w_sh + t.  Maps are independent, one
+ * per OpenMP thread.
+ */
+void orc_stats_traces(const uint16_t *src_k, const uint16_t *src_v,
+                      int64_t s_sl, int64_t s_st, int64_t s_sh,
+                      const uint16_t *tgt_k, const uint16_t *tgt_v,
+                      int64_t t_sl, int64_t t_st, int64_t t_sh,
+                      const float *w_k, const float *w_v, int64_t w_sl, int64_t w_sh,
+                      int64_t n_tokens, int32_t d, int32_t Lt, int32_t Ht,
+                      const int32_t *src_layer, const int32_t *src_head,
+                      const int32_t *maps, int32_t n_sel,
+                      double *G /* [n_sel][p][p] */, double *C /* [n_sel][p][d] */)
+{
+    const int32_t p = d + 1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t s = 0; s < n_sel; ++s) {
+        const int32_t m = maps[s];
+        const int32_t comp = m / (Lt * Ht);
+        const int32_t l = (m / Ht) % Lt;
+        const int32_t h = m % Ht;
+        const uint16_t *xs = (comp ? src_v : src_k) + (int64_t)src_layer[l] * s_sl + (int64_t)src_head[h] * s_sh;
+        const uint16_t *ys = (comp ? tgt_v : tgt_k) + (int64_t)l * t_sl + (int64_t)h * t_sh;
+        const float *ws = (comp ? w_v : w_k) + (int64_t)l * w_sl + (int64_t)h * w_sh;
+        double *Gm = G + (size_t)s * p * p;
+        double *Cm = C + (size_t)s * p * d;
+        double *xt = (double *)malloc(sizeof(double) * (size_t)p);
+        double *yt = (double *)malloc(sizeof(double) * (size_t)d);
+        memset(Gm, 0, sizeof(double) * (size_t)p * p);
+        memset(Cm, 0, sizeof(double) * (size_t)p * d);
+        for (int64_t t = 0; t < n_tokens; ++t) {
+            for (int32_t i = 0; i < d; ++i) xt[i] = orc_bf16(xs[t * s_st + i]);
+            xt[d] = 1.0;
+            for (int32_t i = 0; i < d; ++i) yt[i] = orc_bf16(ys[t * t_st + i]);
+            const double wt = (double)ws[t];
+            for (int32_t i = 0; i < p; ++i) {
+                const double wx = wt * xt[i];
+                double *gr = Gm + (size_t)i * p;
+                double *cr = Cm + (size_t)i * d;
+                for (int32_t j = 0; j < p; ++j) gr[j] += wx * xt[j];
+                for (int32_t j = 0; j < d; ++j) cr[j] += wx * yt[j];
+            }
+        }
+        free(xt);
+        free(yt);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Cholesky factorisation and solve, fp64, in place.  Returns 0, or r > 0 if   */
+/* pivot r (1-based) is not positive.                                         */
+/* ------------------------------------------------------------------------- */
+static int32_t orc_cholesky(double *A, int32_t p)
+{
+    for (int32_t j = 0; j < p; ++j) {
+        double s = A[(size_t)j * p + j];
+        for (int32_t k = 0; k < j; ++k) s -= A[(size_t)j * p + k] * A[(size_t)j * p + k];
+        if (!(s > 0.0)) return j + 1;
+        const double ljj = sqrt(s);
+        A[(size_t)j * p + j] = ljj;
+        for (int32_t i = j + 1; i < p; ++i) {
+            double v = A[(size_t)i * p + j];
+            for (int32_t k = 0; k < j; ++k) v -= A[(size_t)i * p + k] * A[(size_t)j * p + k];
+            A[(size_t)i * p + j] = v / ljj;
+        }
+    }
+    return 0;
+}
+
+static void orc_cholesky_solve(const double *L, int32_t p, double *B, int32_t nrhs)
+{
+    for (int32_t c = 0; c < nrhs; ++c) {
+        for (int32_t i = 0; i < p; ++i) {            /* L z = b */
+            double v = B[(size_t)i * nrhs + c];
+            for (int32_t k = 0; k < i; ++k) v -= L[(size_t)i * p + k] * B[(size_t)k * nrhs + c];
+            B[(size_t)i * nrhs + c] = v / L[(size_t)i * p + i];
+        }
+        for (int32_t i = p - 1; i >= 0; --i) {       /* L^T x = z */
+            double v = B[(size_t)i * nrhs + c];
+            for (int32_t k = i + 1; k < p; ++k) v -= L[(size_t)k * p + i] * B[(size_t)k * nrhs + c];
+            B[(size_t)i * nrhs + c] = v / L[(size_t)i * p + i];
+        }
+    }
+}
+
+/*
+ * Ridge solve on augmented statistics (Section 3.1, Eq. closedform, written
+ * for the bias-column form): (G + lambda_eff J) Theta = C, J = diag(1,..,1,0)
+ * (the bias is not penalised), Theta = [W; b].
+ * The paper states the objective for weights rescaled to mean one; rescaling w
+ * by n / s_w is the same as keeping w and using lambda_eff = lambda * s_w / n
+ * (s_w = G[d][d]).  raw_lambda != 0 uses lambda_eff = lambda instead.
+ * Degenerate systems: info = failing pivot, Theta zero-filled.
+ */
+int32_t orc_ridge_solve(const double *G, const double *C, int32_t d, int64_t n,
+                        double lambda, int32_t raw_lambda, double *Theta /* [p][d] */)
+{
+    const int32_t p = d + 1;
+    double *A = (double *)malloc(sizeof(double) * (size_t)p * p);
+    memcpy(A, G, sizeof(double) * (size_t)p * p);
+    const double s_w = G[(size_t)d * p + d];
+    const double lam = raw_lambda ? lambda : lambda * s_w / (double)n;
+    for (int32_t i = 0; i < d; ++i) A[(size_t)i * p + i] += lam;
+    int32_t info = orc_cholesky(A, p);
+    if (info != 0) {
+        memset(Theta, 0, sizeof(double) * (size_t)p * d);
+    } else {
+        memcpy(Theta, C, sizeof(double) * (size_t)p * d);
+        orc_cholesky_solve(A, p, Theta, d);
+    }
+    free(A);
+    return info;
+}
+
+void orc_ridge_solve_batch(const double *G, const double *C, int32_t n_maps, int32_t d, int64_t n,
+                           double lambda, int32_t raw_lambda, double *Theta, int32_t *info)
+{
+    const int32_t p = d + 1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t m = 0; m < n_maps; ++m)
+        info[m] = orc_ridge_solve(G + (size_t)m * p * p, C + (size_t)m * p * d, d, n, lambda, raw_lambda,
+                                  Theta + (size_t)m * p * d);
+}
+
+/*
+ * The paper's literal route (Section 3.1): rescale the weights to mean one,
+ * weighted means x_bar = n^-1 sum w_i x_i, y_bar likewise, centred rows,
+ * W = (Xc^T Dw Xc + lambda I)^-1 Xc^T Dw Yc, b = y_bar - x_bar W.
+ * Used to check that the bias-column form above is the same estimator.
+ */
+int32_t orc_ridge_centered(const double *X, const double *Y, const double *w, int64_t n, int32_t d,
+                           double lambda, double *Theta /* [d+1][d]: W then b */)
+{
+    double sw = 0.0;
+    for (int64_t t = 0; t < n; ++t) sw += w[t];
+    if (!(sw > 0.0)) { memset(Theta, 0, sizeof(double) * (size_t)(d + 1) * d); return 1; }
+    const double scale = (double)n / sw;                 /* mean-one rescale */
+    double *xb = (double *)calloc((size_t)d, sizeof(double));
+    double *yb = (double *)calloc((size_t)d, sizeof(double));
+    for (int64_t t = 0; t < n; ++t) {
+        const double wt = w[t] * scale;
+        for (int32_t i = 0; i < d; ++i) { xb[i] += wt * X[t * d + i]; yb[i] += wt * Y[t * d + i]; }
+    }
+    for (int32_t i = 0; i < d; ++i) { xb[i] /= (double)n; yb[i] /= (double)n; }
+    double *A = (double *)calloc((size_t)d * d, sizeof(double));
+    double *B = (double *)calloc((size_t)d * d, sizeof(double));
+    double *xc = (double *)malloc(sizeof(double) * (size_t)d);
+    double *yc = (double *)malloc(sizeof(double) * (size_t)d);
+    for (int64_t t = 0; t < n; ++t) {
+        const double wt = w[t] * scale;
+        for (int32_t i = 0; i < d; ++i) { xc[i] = X[t * d + i] - xb[i]; yc[i] = Y[t * d + i] - yb[i]; }
+        for (int32_t i = 0; i < d; ++i)
+            for (int32_t j = 0; j < d; ++j) {
+                A[(size_t)i * d + j] += wt * xc[i] * xc[j];
+                B[(size_t)i * d + j] += wt * xc[i] * yc[j];
+            }
+    }
+    for (int32_t i = 0; i < d; ++i) A[(size_t)i * d + i] += lambda;
+    int32_t info = orc_cholesky(A, d);
+    if (info == 0) {
+        orc_cholesky_solve(A, d, B, d);
+        memcpy(Theta, B, sizeof(double) * (size_t)d * d);
+        for (int32_t j = 0; j < d; ++j) {
+            double v = yb[j];
+            for (int32_t i = 0; i < d; ++i) v -= xb[i] * B[(size_t)i * d + j];
+            Theta[(size_t)d * d + j] = v;
+        }
+    } else {
+        memset(Theta, 0, sizeof(double) * (size_t)(d + 1) * d);
+    }
+    free(A); free(B); free(xc); free(yc); free(xb); free(yb);
+    return info;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Online affine apply (Section 3.2): y_hat_t = x_t W + b per map, written to  */
+/* a target cache.  Source rows come from strided bf16; output is fp64, and   */
+/* optionally also rounded to bf16 (nearest even) as a decode-ready cache.    */
+/* Output element (l, t, h, c) of component comp at                            */
+/*   out[comp] + l*o_sl + t*o_st + h*o_sh + c.                                 */
+/* ------------------------------------------------------------------------- */
+void orc_apply(const uint16_t *src_k, const uint16_t *src_v, int64_t s_sl, int64_t s_st, int64_t s_sh,
+               int64_t n_tokens, int32_t d, int32_t Lt, int32_t Ht,
+               const int32_t *src_layer, const int32_t *src_head,
+               const double *Theta /* [n_maps][p][d] */,
+               const int32_t *maps, int32_t n_sel,
+               double *out_k, double *out_v, uint16_t *out_k_bf16, uint16_t *out_v_bf16,
+               int64_t o_sl, int64_t o_st, int64_t o_sh)
+{
+    const int32_t p = d + 1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t s = 0; s < n_sel; ++s) {
+        const int32_t m = maps[s];
+        const int32_t comp = m / (Lt * Ht);
+        const int32_t l = (m / Ht) % Lt;
+        const int32_t h = m % Ht;
+        const uint16_t *xs = (comp ? src_v : src_k) + (int64_t)src_layer[l] * s_sl + (int64_t)src_head[h] * s_sh;
+        const double *W = Theta + (size_t)m * p * d;
+        double *o = (comp ? out_v : out_k);
+        uint16_t *ob = (comp ? out_v_bf16 : out_k_bf16);
+        for (int64_t t = 0; t < n_tokens; ++t) {
+            const int64_t base = (int64_t)l * o_sl + t * o_st + (int64_t)h * o_sh;
+            for (int32_t c = 0; c < d; ++c) {
+                double v = W[(size_t)d * d + c];                       /* b */
+                for (int32_t i = 0; i < d; ++i) v += orc_bf16(xs[t * s_st + i]) * W[(size_t)i * d + c];
+                if (o) o[base + c] = v;
+                if (ob) ob[base + c] = orc_to_bf16(v);
+            }
+        }
+    }
+}
