@@ -1,0 +1,188 @@
+/*
+ * cb.h - C ABI of the head-local KV-cache mapper construction and apply library (CUDA, sm_100a).
+ *
+ * The library builds, for every target (component, layer l, KV head h) matched to ONE source head
+ * (layer j(l), head a(h)), the attention-weighted sufficient statistics of an affine ridge map, solves the
+ * ridge systems in closed form, and applies the fitted maps to a source cache.
+ *
+ * Notation (paper, Section 2.1): source model L_s layers, H_s KV heads, head width d_s; target L_t, H_t, d_t.
+ * comp = 0 for keys, 1 for values.  Map id  m = (comp*L_t + l)*H_t + h,  n_maps = 2*L_t*H_t.
+ * d = d_s = d_t, p = d + 1.  Row-vector convention y_hat = x W + b (Section 3.1); the bias is the LAST row of
+ * Theta = [W; b] and the LAST row/column of G.
+ *
+ * All device pointers are plain CUDA device pointers owned by the caller.  The library allocates no device
+ * memory.  Every call enqueues its work on the given stream (a cudaStream_t passed as void*, NULL = default
+ * stream) and returns without synchronising unless stated.  Errors are returned as status codes; argument
+ * errors are detected on the host before anything is launched.  Preconditions that are NOT checked on the
+ * device: weights are finite and >= 0, traces are finite.
+ *
+ * There is no CPU implementation behind these calls: without a CUDA device they return CB_ERR_CUDA.
+ */
+#ifndef CB_H_
+#define CB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum cb_status {
+    CB_OK = 0,
+    CB_ERR_INVALID_ARG = 1,  /* null pointer, negative size, stride not usable, misaligned pointer        */
+    CB_ERR_UNSUPPORTED = 2,  /* head width not in {64, 128}, d_s != d_t, too many tokens in one call       */
+    CB_ERR_STATE = 3,        /* call order violated (e.g. reduce before any accumulate is fine, but a      */
+                             /* destroyed or foreign context is not)                                       */
+    CB_ERR_WORKSPACE = 4,    /* workspace smaller than cb_workspace_bytes() or not 256-byte aligned         */
+    CB_ERR_CUDA = 5,         /* a CUDA runtime/driver call failed (includes "no device")                    */
+    CB_ERR_NOT_PD = 6,       /* cb_check_info: at least one ridge system had a non-positive pivot           */
+    CB_ERR_TIMEOUT = 7       /* cb_device_status: a bounded device-side wait ran out                        */
+} cb_status;
+
+/* flags (cb_problem.flags and the flags argument of cb_ridge_solve) */
+#define CB_FLAG_COMPENSATED 1u /* accumulate: split the bf16 weighted operand into hi + lo (two MMAs per   */
+                               /* tile) so that folding the fp32 weight into a bf16 operand costs ~2^-17   */
+                               /* instead of ~2^-9 per element.  Meant for small token counts.             */
+#define CB_FLAG_RAW_LAMBDA  2u /* solve: penalise with lambda itself instead of lambda * s_w / n            */
+#define CB_FLAG_SIMT        4u /* accumulate/apply: use the plain fp32 CUDA-core kernels (no tensor cores) */
+
+#define CB_DTYPE_BF16 0
+#define CB_DTYPE_F32  1
+
+/*
+ * A strided bf16 view of one model's K and V traces (or caches) for n_tokens rows; device memory.
+ * Element (layer j, token t, head g, channel c) of K is at
+ *     (bf16*)k + j*stride_layer + t*stride_token + g*stride_head + c          (strides in elements)
+ * and likewise for V.  Channels are contiguous.  This covers the paper's index order K_{j,t,g} stored as
+ * [L][T][H][d] as well as [L][H][T][d].  k and v must be 16-byte aligned and every stride a multiple of 8.
+ */
+typedef struct cb_kv_view {
+    const void *k;
+    const void *v;
+    int32_t n_layers, n_heads, head_dim;
+    int64_t n_tokens;
+    int64_t stride_layer, stride_token, stride_head;
+} cb_kv_view;
+
+/*
+ * The mapping problem: model shapes and the static head match (Section 3.2, Eq. "localfeature" with one
+ * selected layer per target layer): target layer l reads source layer src_layer[l]; target head h reads
+ * source head src_head[h].  src_layer (length Lt) and src_head (length Ht) are HOST arrays, copied by
+ * cb_create / read by cb_apply during the call.
+ * n_splits: number of token splits (independent partial statistics per map, summed in fixed order by
+ * cb_stats_reduce); 0 selects a default.  Must be <= 64.
+ */
+typedef struct cb_problem {
+    int32_t Ls, Hs, ds;
+    int32_t Lt, Ht, dt;
+    const int32_t *src_layer;
+    const int32_t *src_head;
+    uint32_t flags;
+    int32_t n_splits;
+} cb_problem;
+
+typedef struct cb_ctx cb_ctx;
+
+const char *cb_status_string(cb_status s);
+
+/*
+ * Default head match.  Layer: nearest relative depth, j(l) = floor((2 l (Ls-1) + (Lt-1)) / (2 (Lt-1)))
+ * (0 if Lt == 1); head: a(h) = floor(h*Hs/Ht), the identity when both models expose the same number of KV
+ * groups (Section 3.2: "the natural assignment is a(h) = h").  Host arrays of length Lt and Ht.
+ */
+cb_status cb_head_map_nearest(int32_t Ls, int32_t Hs, int32_t Lt, int32_t Ht,
+                              int32_t *src_layer, int32_t *src_head);
+
+/*
+ * Static gather schedule (Section 2.3: support and head assignment are fixed before fitting, so the irregular
+ * gather is compiled once).  Maps are grouped by the source head they read.  Items are ordered by
+ * (comp, source layer, source head); only source heads read by at least one map become items; the maps of an
+ * item are listed in ascending id.  Host output arrays: item_comp/item_layer/item_head need 2*Ls*Hs entries,
+ * item_begin 2*Ls*Hs + 1 (offsets into item_maps), item_maps 2*Lt*Ht.  *n_items receives the item count.
+ */
+cb_status cb_work_list(const cb_problem *prob, int32_t *n_items, int32_t *item_comp, int32_t *item_layer,
+                       int32_t *item_head, int32_t *item_begin, int32_t *item_maps);
+
+/* Bytes of device workspace cb_create needs for this problem (partial statistics slots + small tables). */
+cb_status cb_workspace_bytes(const cb_problem *prob, size_t *bytes);
+
+/*
+ * Create a context on the current device.  workspace: device memory, 256-byte aligned, at least
+ * cb_workspace_bytes(); it stays owned by the caller and must outlive the context.  Copies the head match
+ * to the device (synchronous, small) and leaves the statistics in the reset state (zero) by enqueueing a
+ * clear on the default stream and synchronising it.
+ */
+cb_status cb_create(const cb_problem *prob, void *workspace, size_t workspace_bytes, cb_ctx **out);
+void cb_destroy(cb_ctx *ctx);
+
+/* Zero the partial statistics and the token count. */
+cb_status cb_stats_reset(cb_ctx *ctx, void *stream);
+
+/*
+ * Fused weighted-statistics accumulation (Section 3.4, Eq. "fusedstats", in the bias-column form): for every
+ * map m with matched source head, add over the n_tokens rows of this call
+ *     G_m += sum_t w_t [x_t,1]^T [x_t,1]      C_m += sum_t w_t [x_t,1]^T y_t
+ * reading x_t from src (layer src_layer[l], head src_head[h]), y_t from tgt (layer l, head h) and
+ * w_t from w_k (keys) or w_v (values) at  w + l*w_stride_layer + h*w_stride_head + t  (fp32, device,
+ * strides in elements, tokens contiguous).  w_v may equal w_k.  No concatenated observation matrix is built;
+ * head pairs are read straight from the strided views.  Statistics are additive over calls (token chunks of
+ * any size, including ragged batches packed back to back); src->n_tokens must equal tgt->n_tokens and be
+ * < 2^31.  n_tokens == 0 is a no-op.  Partial sums live in fp32 in the context's workspace: each (map, split)
+ * slot is owned by one thread block per call and calls are ordered by the stream, so results are bitwise
+ * reproducible for a fixed sequence of calls.
+ */
+cb_status cb_stats_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                              const float *w_k, const float *w_v,
+                              int64_t w_stride_layer, int64_t w_stride_head, void *stream);
+
+/*
+ * Deterministic reduction: sums the splits of every map in index order (fp64 inside), symmetrises
+ * G <- (G + G^T)/2 and writes fp32  G [n_maps][p][p]  and  C [n_maps][p][d]  (device).  n_tokens_out (host,
+ * may be NULL) receives the number of rows accumulated since the last reset; it is host bookkeeping and
+ * valid on return.  The partial statistics are left untouched, so accumulation can continue afterwards.
+ */
+cb_status cb_stats_reduce(cb_ctx *ctx, float *G, float *C, int64_t *n_tokens_out, void *stream);
+
+/*
+ * Batched closed-form ridge solve (Section 3.1, Eq. "closedform", written for the bias-column statistics):
+ * for every lambda and map,  (G_m + lambda_eff J) Theta = C_m,  J = diag(1,..,1,0) (bias not penalised),
+ * by Cholesky factorisation in fp64.  lambda_eff = lambda * s_w / n_tokens with s_w = G_m[d][d] (the paper
+ * states the objective for weights rescaled to mean one; this is that rescale), or lambda itself with
+ * CB_FLAG_RAW_LAMBDA.  G [n_maps][p][p], C [n_maps][p][d]: device fp32.  lambdas: HOST array of n_lambda
+ * (<= 16) values.  Wb: device fp32 [n_lambda][n_maps][p][d] (rows 0..d-1 = W, row d = b).  info: device int32
+ * [n_lambda][n_maps]: 0, or r > 0 if pivot r was not positive, in which case that map's Wb is zero-filled.
+ */
+cb_status cb_ridge_solve(const float *G, const float *C, int32_t n_maps, int32_t d, int64_t n_tokens,
+                         const float *lambdas, int32_t n_lambda, uint32_t flags,
+                         float *Wb, int32_t *info, void *stream);
+
+/* Synchronises the stream and returns CB_ERR_NOT_PD if any of the n info entries is non-zero
+ * (*first_bad, may be NULL, receives its index), CB_OK otherwise. */
+cb_status cb_check_info(const int32_t *info, int64_t n, void *stream, int64_t *first_bad);
+
+/*
+ * Online affine apply (Section 3.2; Section 1, online handoff): for every map m and token t of the source
+ * cache,  out[l][t][h][:] = x_t W_m + b_m  with x_t the matched source head's row.  Wb: device fp32
+ * [n_maps][p][d].  Outputs tgt_k / tgt_v: device, element (l, t, h, c) at
+ * l*t_stride_layer + t*t_stride_token + h*t_stride_head + c (elements of out_dtype: CB_DTYPE_BF16 rounds to
+ * nearest even, CB_DTYPE_F32 stores fp32), 16-byte aligned, strides multiples of 8.  Positional rotation is
+ * the caller's: the map acts in content coordinates.  prob->flags & CB_FLAG_SIMT selects the CUDA-core kernel.
+ */
+cb_status cb_apply(const cb_problem *prob, const float *Wb, const cb_kv_view *src_cache,
+                   void *tgt_k, void *tgt_v, int64_t t_stride_layer, int64_t t_stride_token,
+                   int64_t t_stride_head, int32_t out_dtype, void *stream);
+
+/*
+ * Synchronises the stream and reads the context's device status word: CB_OK, or CB_ERR_TIMEOUT if a bounded
+ * wait inside a kernel ran out (the statistics are then invalid; reset before reuse).
+ */
+cb_status cb_device_status(cb_ctx *ctx, void *stream);
+
+/* Number of kernels this library has launched in this process (all contexts); for accounting. */
+int64_t cb_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CB_H_ */

@@ -1,0 +1,242 @@
+"""ctypes binding of the C ABI declared in include/cb.h.
+
+Argument marshalling only: every step of the path runs in the CUDA library.  torch tensors are used as plain
+device buffers (data_ptr, strides) and torch streams as cudaStream_t.  There is no fallback: if the shared
+library has not been built, importing a function from here raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcb.so")
+
+CB_OK = 0
+CB_ERR_INVALID_ARG, CB_ERR_UNSUPPORTED, CB_ERR_STATE, CB_ERR_WORKSPACE = 1, 2, 3, 4
+CB_ERR_CUDA, CB_ERR_NOT_PD, CB_ERR_TIMEOUT = 5, 6, 7
+CB_FLAG_COMPENSATED, CB_FLAG_RAW_LAMBDA, CB_FLAG_SIMT = 1, 2, 4
+CB_DTYPE_BF16, CB_DTYPE_F32 = 0, 1
+
+EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_workspace_bytes", "cb_create",
+           "cb_destroy", "cb_stats_reset", "cb_stats_accumulate", "cb_stats_reduce", "cb_ridge_solve",
+           "cb_check_info", "cb_apply", "cb_device_status", "cb_launch_count")
+
+
+class CbError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+
+
+class _KvView(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+                ("n_layers", ctypes.c_int32), ("n_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("n_tokens", ctypes.c_int64),
+                ("stride_layer", ctypes.c_int64), ("stride_token", ctypes.c_int64), ("stride_head", ctypes.c_int64)]
+
+
+class _Problem(ctypes.Structure):
+    _fields_ = [("Ls", ctypes.c_int32), ("Hs", ctypes.c_int32), ("ds", ctypes.c_int32),
+                ("Lt", ctypes.c_int32), ("Ht", ctypes.c_int32), ("dt", ctypes.c_int32),
+                ("src_layer", ctypes.POINTER(ctypes.c_int32)), ("src_head", ctypes.POINTER(ctypes.c_int32)),
+                ("flags", ctypes.c_uint32), ("n_splits", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("CUDA library %s is missing: run `python -m paper_2609_00891_b200.build` "
+                               "(there is no CPU fallback)" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        L.cb_status_string.restype = ctypes.c_char_p
+        L.cb_status_string.argtypes = [ctypes.c_int]
+        L.cb_launch_count.restype = ctypes.c_int64
+        for name in EXPORTS:
+            if name not in ("cb_status_string", "cb_launch_count", "cb_destroy"):
+                getattr(L, name).restype = ctypes.c_int
+        L.cb_destroy.restype = None
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().cb_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != CB_OK:
+        raise CbError(status, where)
+
+
+def _stream_ptr(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+class Problem:
+    """Model shapes plus the static head match (host arrays), mirroring cb_problem."""
+
+    def __init__(self, Ls: int, Hs: int, ds: int, Lt: int, Ht: int, dt: int,
+                 src_layer: Sequence[int], src_head: Sequence[int], flags: int = 0, n_splits: int = 0):
+        self.src_layer = np.ascontiguousarray(src_layer, dtype=np.int32)
+        self.src_head = np.ascontiguousarray(src_head, dtype=np.int32)
+        assert self.src_layer.shape == (Lt,) and self.src_head.shape == (Ht,)
+        self.c = _Problem(Ls, Hs, ds, Lt, Ht, dt,
+                          self.src_layer.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                          self.src_head.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                          flags, n_splits)
+        self.Ls, self.Hs, self.ds, self.Lt, self.Ht, self.dt = Ls, Hs, ds, Lt, Ht, dt
+        self.flags, self.n_splits = flags, n_splits
+
+    @property
+    def n_maps(self) -> int:
+        return 2 * self.Lt * self.Ht
+
+    def with_flags(self, flags: int) -> "Problem":
+        return Problem(self.Ls, self.Hs, self.ds, self.Lt, self.Ht, self.dt, self.src_layer, self.src_head,
+                       flags, self.n_splits)
+
+
+def _kv_view(k: torch.Tensor, v: torch.Tensor) -> _KvView:
+    """View of K and V tensors indexed [layer][token][head][channel] (any strides, channels contiguous)."""
+    assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16 and k.dim() == 4
+    assert k.shape == v.shape and k.stride() == v.stride() and k.stride(3) == 1
+    L, T, H, d = k.shape
+    return _KvView(k.data_ptr(), v.data_ptr(), L, H, d, T, k.stride(0), k.stride(1), k.stride(2))
+
+
+# ---------------------------------------------------------------------------------------------- host-only calls
+def cb_head_map_nearest(Ls: int, Hs: int, Lt: int, Ht: int) -> Tuple[np.ndarray, np.ndarray]:
+    sl = np.empty(Lt, np.int32)
+    sh = np.empty(Ht, np.int32)
+    _check(lib().cb_head_map_nearest(Ls, Hs, Lt, Ht, sl.ctypes.data_as(ctypes.c_void_p),
+                                     sh.ctypes.data_as(ctypes.c_void_p)), "cb_head_map_nearest")
+    return sl, sh
+
+
+def cb_work_list(prob: Problem):
+    cap = 2 * prob.Ls * prob.Hs
+    n = ctypes.c_int32(0)
+    ic, il, ih = (np.empty(cap, np.int32) for _ in range(3))
+    ib = np.empty(cap + 1, np.int32)
+    im = np.empty(prob.n_maps, np.int32)
+    p = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    _check(lib().cb_work_list(ctypes.byref(prob.c), ctypes.byref(n), p(ic), p(il), p(ih), p(ib), p(im)), "cb_work_list")
+    k = n.value
+    return ic[:k].copy(), il[:k].copy(), ih[:k].copy(), ib[:k + 1].copy(), im.copy()
+
+
+def cb_workspace_bytes(prob: Problem) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().cb_workspace_bytes(ctypes.byref(prob.c), ctypes.byref(n)), "cb_workspace_bytes")
+    return n.value
+
+
+# ---------------------------------------------------------------------------------------------- device calls
+class Context:
+    """Owns a cb_ctx; the workspace tensor is kept alive with it."""
+
+    def __init__(self, prob: Problem, workspace: Optional[torch.Tensor] = None, device="cuda"):
+        self.prob = prob
+        if workspace is None:
+            workspace = torch.empty(cb_workspace_bytes(prob), dtype=torch.uint8, device=device)
+        self.workspace = workspace
+        h = ctypes.c_void_p()
+        _check(lib().cb_create(ctypes.byref(prob.c), ctypes.c_void_p(workspace.data_ptr()),
+                               ctypes.c_size_t(workspace.numel()), ctypes.byref(h)), "cb_create")
+        self.handle = h
+
+    def close(self):
+        if self.handle:
+            lib().cb_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def cb_create(prob: Problem, workspace: Optional[torch.Tensor] = None, device="cuda") -> Context:
+    return Context(prob, workspace, device)
+
+
+def cb_destroy(ctx: Context) -> None:
+    ctx.close()
+
+
+def cb_stats_reset(ctx: Context, stream=None) -> None:
+    _check(lib().cb_stats_reset(ctx.handle, _stream_ptr(stream)), "cb_stats_reset")
+
+
+def cb_stats_accumulate(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor, w_v: torch.Tensor, stream=None) -> None:
+    """Traces [L][T][H][d] bf16, weights [Lt][Ht][T] fp32 (tokens contiguous)."""
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    assert w_k.dtype == torch.float32 and w_v.dtype == torch.float32 and w_k.dim() == 3
+    assert w_k.stride() == w_v.stride() and (w_k.stride(2) == 1 or w_k.shape[2] <= 1)
+    _check(lib().cb_stats_accumulate(ctx.handle, ctypes.byref(sv), ctypes.byref(tv),
+                                     ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                     ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
+                                     _stream_ptr(stream)), "cb_stats_accumulate")
+
+
+def cb_stats_reduce(ctx: Context, G: torch.Tensor, C: torch.Tensor, stream=None) -> int:
+    p, d = ctx.prob.ds + 1, ctx.prob.ds
+    assert G.dtype == torch.float32 and C.dtype == torch.float32 and G.is_contiguous() and C.is_contiguous()
+    assert G.numel() == ctx.prob.n_maps * p * p and C.numel() == ctx.prob.n_maps * p * d
+    n = ctypes.c_int64(0)
+    _check(lib().cb_stats_reduce(ctx.handle, ctypes.c_void_p(G.data_ptr()), ctypes.c_void_p(C.data_ptr()),
+                                 ctypes.byref(n), _stream_ptr(stream)), "cb_stats_reduce")
+    return n.value
+
+
+def cb_ridge_solve(G: torch.Tensor, C: torch.Tensor, n_tokens: int, lambdas: Sequence[float], flags: int,
+                   Wb: torch.Tensor, info: torch.Tensor, stream=None) -> None:
+    n_maps, p, _ = G.shape
+    d = p - 1
+    lam = np.ascontiguousarray(lambdas, dtype=np.float32)
+    assert G.dtype == torch.float32 and C.dtype == torch.float32 and Wb.dtype == torch.float32 and info.dtype == torch.int32
+    assert G.is_contiguous() and C.is_contiguous() and Wb.is_contiguous() and info.is_contiguous()
+    assert Wb.numel() == len(lam) * n_maps * p * d and info.numel() == len(lam) * n_maps
+    _check(lib().cb_ridge_solve(ctypes.c_void_p(G.data_ptr()), ctypes.c_void_p(C.data_ptr()), n_maps, d,
+                                ctypes.c_int64(n_tokens), lam.ctypes.data_as(ctypes.c_void_p), len(lam),
+                                ctypes.c_uint32(flags), ctypes.c_void_p(Wb.data_ptr()),
+                                ctypes.c_void_p(info.data_ptr()), _stream_ptr(stream)), "cb_ridge_solve")
+
+
+def cb_check_info(info: torch.Tensor, stream=None) -> None:
+    bad = ctypes.c_int64(-1)
+    _check(lib().cb_check_info(ctypes.c_void_p(info.data_ptr()), ctypes.c_int64(info.numel()), _stream_ptr(stream),
+                               ctypes.byref(bad)), "cb_check_info (first bad index %d)" % bad.value)
+
+
+def cb_apply(prob: Problem, Wb: torch.Tensor, src_k: torch.Tensor, src_v: torch.Tensor,
+             tgt_k: torch.Tensor, tgt_v: torch.Tensor, stream=None) -> None:
+    """Wb fp32 [n_maps][p][d]; source cache [Ls][T][Hs][d] bf16; outputs [Lt][T][Ht][d] bf16 or fp32."""
+    sv = _kv_view(src_k, src_v)
+    assert Wb.dtype == torch.float32 and Wb.is_contiguous()
+    assert tgt_k.dtype == tgt_v.dtype and tgt_k.stride() == tgt_v.stride() and tgt_k.stride(3) == 1
+    dt = {torch.bfloat16: CB_DTYPE_BF16, torch.float32: CB_DTYPE_F32}[tgt_k.dtype]
+    _check(lib().cb_apply(ctypes.byref(prob.c), ctypes.c_void_p(Wb.data_ptr()), ctypes.byref(sv),
+                          ctypes.c_void_p(tgt_k.data_ptr()), ctypes.c_void_p(tgt_v.data_ptr()),
+                          ctypes.c_int64(tgt_k.stride(0)), ctypes.c_int64(tgt_k.stride(1)),
+                          ctypes.c_int64(tgt_k.stride(2)), dt, _stream_ptr(stream)), "cb_apply")
+
+
+def cb_device_status(ctx: Context, stream=None) -> None:
+    _check(lib().cb_device_status(ctx.handle, _stream_ptr(stream)), "cb_device_status")
+
+
+def cb_launch_count() -> int:
+    return int(lib().cb_launch_count())

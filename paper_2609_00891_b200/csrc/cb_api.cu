@@ -1,0 +1,339 @@
+// Host side of the C ABI: argument validation, the static gather schedule, workspace layout and launches.
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "cb_internal.cuh"
+
+namespace cb {
+
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static constexpr uint32_t CTX_MAGIC = 0xCB0C7A11u;
+static constexpr int DEFAULT_SPLITS = 4;
+static constexpr int MAX_SPLITS = 64;
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    size_t slots_off, slots_bytes, tab_off, status_off, total;
+};
+
+static Layout workspace_layout(int Lt, int Ht, int d, int n_splits)
+{
+    Layout L;
+    const size_t n_maps = 2 * (size_t)Lt * Ht;
+    L.slots_off = 0;
+    L.slots_bytes = (size_t)n_splits * n_maps * slot_floats(d) * sizeof(float);
+    L.tab_off = align_up(L.slots_bytes, 256);
+    L.status_off = align_up(L.tab_off + sizeof(int) * ((size_t)Lt + Ht), 256);
+    L.total = L.status_off + 256;
+    return L;
+}
+
+static cb_status check_problem(const cb_problem *p)
+{
+    if (!p || !p->src_layer || !p->src_head) return CB_ERR_INVALID_ARG;
+    if (p->Ls <= 0 || p->Hs <= 0 || p->Lt <= 0 || p->Ht <= 0 || p->ds <= 0 || p->dt <= 0) return CB_ERR_INVALID_ARG;
+    if (p->n_splits < 0 || p->n_splits > MAX_SPLITS) return CB_ERR_INVALID_ARG;
+    for (int l = 0; l < p->Lt; ++l)
+        if (p->src_layer[l] < 0 || p->src_layer[l] >= p->Ls) return CB_ERR_INVALID_ARG;
+    for (int h = 0; h < p->Ht; ++h)
+        if (p->src_head[h] < 0 || p->src_head[h] >= p->Hs) return CB_ERR_INVALID_ARG;
+    if (p->ds != p->dt || (p->ds != 64 && p->ds != 128)) return CB_ERR_UNSUPPORTED;
+    if ((long long)p->Lt * p->Ht > (1 << 20)) return CB_ERR_UNSUPPORTED;
+    return CB_OK;
+}
+
+static int splits_of(const cb_problem *p) { return p->n_splits > 0 ? p->n_splits : DEFAULT_SPLITS; }
+
+static cb_status check_view(const cb_kv_view *v, int L, int H, int d)
+{
+    if (!v) return CB_ERR_INVALID_ARG;
+    if (v->n_layers != L || v->n_heads != H || v->head_dim != d) return CB_ERR_INVALID_ARG;
+    if (v->n_tokens < 0) return CB_ERR_INVALID_ARG;
+    if (v->n_tokens >= (1ll << 31)) return CB_ERR_UNSUPPORTED;
+    if (v->n_tokens == 0) return CB_OK;
+    if (!v->k || !v->v) return CB_ERR_INVALID_ARG;
+    if (((uintptr_t)v->k | (uintptr_t)v->v) & 15) return CB_ERR_INVALID_ARG;
+    if (v->stride_layer < 0 || v->stride_token <= 0 || v->stride_head < 0) return CB_ERR_INVALID_ARG;
+    if ((v->stride_layer | v->stride_token | v->stride_head) & 7) return CB_ERR_INVALID_ARG;
+    return CB_OK;
+}
+
+}  // namespace cb
+
+using namespace cb;
+
+struct cb_ctx {
+    uint32_t magic;
+    cb_problem prob;
+    std::vector<int32_t> src_layer, src_head;
+    int d, n_maps, n_splits;
+    char *ws;
+    Layout lay;
+    long long n_tokens;
+};
+
+extern "C" {
+
+const char *cb_status_string(cb_status s)
+{
+    switch (s) {
+        case CB_OK: return "ok";
+        case CB_ERR_INVALID_ARG: return "invalid argument";
+        case CB_ERR_UNSUPPORTED: return "unsupported shape";
+        case CB_ERR_STATE: return "invalid context or call order";
+        case CB_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case CB_ERR_CUDA: return "CUDA call failed";
+        case CB_ERR_NOT_PD: return "ridge system not positive definite";
+        case CB_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int64_t cb_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+cb_status cb_head_map_nearest(int32_t Ls, int32_t Hs, int32_t Lt, int32_t Ht, int32_t *src_layer, int32_t *src_head)
+{
+    if (Ls <= 0 || Hs <= 0 || Lt <= 0 || Ht <= 0 || !src_layer || !src_head) return CB_ERR_INVALID_ARG;
+    for (int32_t l = 0; l < Lt; ++l) {
+        if (Lt == 1) { src_layer[l] = 0; continue; }
+        const int64_t num = (int64_t)2 * l * (Ls - 1) + (Lt - 1);
+        src_layer[l] = (int32_t)(num / ((int64_t)2 * (Lt - 1)));
+    }
+    for (int32_t h = 0; h < Ht; ++h) src_head[h] = (int32_t)(((int64_t)h * Hs) / Ht);
+    return CB_OK;
+}
+
+cb_status cb_work_list(const cb_problem *prob, int32_t *n_items, int32_t *item_comp, int32_t *item_layer,
+                       int32_t *item_head, int32_t *item_begin, int32_t *item_maps)
+{
+    cb_status s = check_problem(prob);
+    if (s != CB_OK && s != CB_ERR_UNSUPPORTED) return s;   // the schedule itself does not depend on d
+    if (!n_items || !item_comp || !item_layer || !item_head || !item_begin || !item_maps) return CB_ERR_INVALID_ARG;
+    const int Ls = prob->Ls, Hs = prob->Hs, Lt = prob->Lt, Ht = prob->Ht;
+    // bucket every map by its source head with a counting sort: key = (comp*Ls + j)*Hs + g
+    const int n_keys = 2 * Ls * Hs, n_maps = 2 * Lt * Ht;
+    std::vector<int32_t> count(n_keys + 1, 0);
+    auto key_of = [&](int m) {
+        const int comp = m / (Lt * Ht), l = (m / Ht) % Lt, h = m % Ht;
+        return (comp * Ls + prob->src_layer[l]) * Hs + prob->src_head[h];
+    };
+    for (int m = 0; m < n_maps; ++m) ++count[key_of(m) + 1];
+    for (int k = 0; k < n_keys; ++k) count[k + 1] += count[k];
+    std::vector<int32_t> fill(count.begin(), count.end() - 1);
+    for (int m = 0; m < n_maps; ++m) item_maps[fill[key_of(m)]++] = m;   // ascending m inside a bucket
+    int n = 0;
+    for (int k = 0; k < n_keys; ++k) {
+        if (count[k + 1] == count[k]) continue;
+        item_comp[n] = k / (Ls * Hs);
+        item_layer[n] = (k / Hs) % Ls;
+        item_head[n] = k % Hs;
+        item_begin[n] = count[k];
+        ++n;
+    }
+    item_begin[n] = n_maps;
+    *n_items = n;
+    return CB_OK;
+}
+
+cb_status cb_workspace_bytes(const cb_problem *prob, size_t *bytes)
+{
+    cb_status s = check_problem(prob);
+    if (s != CB_OK) return s;
+    if (!bytes) return CB_ERR_INVALID_ARG;
+    *bytes = workspace_layout(prob->Lt, prob->Ht, prob->ds, splits_of(prob)).total;
+    return CB_OK;
+}
+
+cb_status cb_create(const cb_problem *prob, void *workspace, size_t workspace_bytes, cb_ctx **out)
+{
+    if (!out) return CB_ERR_INVALID_ARG;
+    *out = nullptr;
+    cb_status s = check_problem(prob);
+    if (s != CB_OK) return s;
+    const int n_splits = splits_of(prob);
+    const Layout lay = workspace_layout(prob->Lt, prob->Ht, prob->ds, n_splits);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < lay.total) return CB_ERR_WORKSPACE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+
+    cb_ctx *c = new (std::nothrow) cb_ctx();
+    if (!c) return CB_ERR_INVALID_ARG;
+    c->magic = CTX_MAGIC;
+    c->prob = *prob;
+    c->src_layer.assign(prob->src_layer, prob->src_layer + prob->Lt);
+    c->src_head.assign(prob->src_head, prob->src_head + prob->Ht);
+    c->prob.src_layer = c->src_layer.data();
+    c->prob.src_head = c->src_head.data();
+    c->d = prob->ds;
+    c->n_maps = 2 * prob->Lt * prob->Ht;
+    c->n_splits = n_splits;
+    c->ws = static_cast<char *>(workspace);
+    c->lay = lay;
+    c->n_tokens = 0;
+
+    std::vector<int32_t> tab(c->src_layer);
+    tab.insert(tab.end(), c->src_head.begin(), c->src_head.end());
+    cudaError_t e = cudaMemcpy(c->ws + lay.tab_off, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + lay.slots_off, 0, lay.slots_bytes, 0);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + lay.status_off, 0, 256, 0);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return CB_ERR_CUDA;
+    }
+    *out = c;
+    return CB_OK;
+}
+
+void cb_destroy(cb_ctx *ctx)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return;
+    ctx->magic = 0;
+    delete ctx;
+}
+
+cb_status cb_stats_reset(cb_ctx *ctx, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.slots_off, 0, ctx->lay.slots_bytes, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + ctx->lay.status_off, 0, 256, st);
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    ctx->n_tokens = 0;
+    return CB_OK;
+}
+
+cb_status cb_stats_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                              const float *w_k, const float *w_v,
+                              int64_t w_stride_layer, int64_t w_stride_head, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    const cb_problem &P = ctx->prob;
+    cb_status s = check_view(src, P.Ls, P.Hs, P.ds);
+    if (s != CB_OK) return s;
+    s = check_view(tgt, P.Lt, P.Ht, P.dt);
+    if (s != CB_OK) return s;
+    if (src->n_tokens != tgt->n_tokens) return CB_ERR_INVALID_ARG;
+    if (src->n_tokens == 0) return CB_OK;
+    if (!w_k || !w_v || w_stride_layer < 0 || w_stride_head < 0) return CB_ERR_INVALID_ARG;
+    if (((uintptr_t)w_k | (uintptr_t)w_v) & 3) return CB_ERR_INVALID_ARG;
+
+    AccumArgs a;
+    a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src->k), static_cast<const __nv_bfloat16 *>(src->v),
+                  src->stride_layer, src->stride_token, src->stride_head};
+    a.tgt = KVPtr{static_cast<const __nv_bfloat16 *>(tgt->k), static_cast<const __nv_bfloat16 *>(tgt->v),
+                  tgt->stride_layer, tgt->stride_token, tgt->stride_head};
+    a.w_k = w_k; a.w_v = w_v; a.w_sl = w_stride_layer; a.w_sh = w_stride_head;
+    a.n_tokens = (int)src->n_tokens;
+    a.Lt = P.Lt; a.Ht = P.Ht; a.n_splits = ctx->n_splits;
+    a.src_layer = reinterpret_cast<const int *>(ctx->ws + ctx->lay.tab_off);
+    a.src_head = a.src_layer + P.Lt;
+    a.slots = reinterpret_cast<float *>(ctx->ws + ctx->lay.slots_off);
+    a.status = reinterpret_cast<int *>(ctx->ws + ctx->lay.status_off);
+    a.compensated = (P.flags & CB_FLAG_COMPENSATED) ? 1 : 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = (P.flags & CB_FLAG_SIMT) ? launch_accum_simt(a, ctx->d, st)
+                                             : launch_accum_tc(a, ctx->d, src, tgt, st);
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    ctx->n_tokens += src->n_tokens;
+    return CB_OK;
+}
+
+cb_status cb_stats_reduce(cb_ctx *ctx, float *G, float *C, int64_t *n_tokens_out, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (!G || !C) return CB_ERR_INVALID_ARG;
+    cudaError_t e = launch_reduce(reinterpret_cast<const float *>(ctx->ws + ctx->lay.slots_off), ctx->n_splits,
+                                  ctx->n_maps, ctx->d, G, C, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (n_tokens_out) *n_tokens_out = ctx->n_tokens;
+    return CB_OK;
+}
+
+cb_status cb_ridge_solve(const float *G, const float *C, int32_t n_maps, int32_t d, int64_t n_tokens,
+                         const float *lambdas, int32_t n_lambda, uint32_t flags,
+                         float *Wb, int32_t *info, void *stream)
+{
+    if (!G || !C || !lambdas || !Wb || !info) return CB_ERR_INVALID_ARG;
+    if (n_maps < 0 || n_lambda <= 0 || n_lambda > 16 || n_tokens < 0) return CB_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return CB_ERR_UNSUPPORTED;
+    if (n_maps > 65535 * 16) return CB_ERR_UNSUPPORTED;
+    for (int i = 0; i < n_lambda; ++i)
+        if (!(lambdas[i] >= 0.f)) return CB_ERR_INVALID_ARG;
+    if (n_maps == 0) return CB_OK;
+    cudaError_t e = launch_solve(G, C, n_maps, d, n_tokens, lambdas, n_lambda, flags, Wb, info,
+                                 static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+cb_status cb_check_info(const int32_t *info, int64_t n, void *stream, int64_t *first_bad)
+{
+    if (!info || n < 0) return CB_ERR_INVALID_ARG;
+    std::vector<int32_t> h((size_t)n);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(h.data(), info, sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    for (int64_t i = 0; i < n; ++i)
+        if (h[(size_t)i] != 0) {
+            if (first_bad) *first_bad = i;
+            return CB_ERR_NOT_PD;
+        }
+    return CB_OK;
+}
+
+cb_status cb_apply(const cb_problem *prob, const float *Wb, const cb_kv_view *src_cache,
+                   void *tgt_k, void *tgt_v, int64_t t_stride_layer, int64_t t_stride_token,
+                   int64_t t_stride_head, int32_t out_dtype, void *stream)
+{
+    cb_status s = check_problem(prob);
+    if (s != CB_OK) return s;
+    if (prob->Lt > 128 || prob->Ht > 64) return CB_ERR_UNSUPPORTED;
+    s = check_view(src_cache, prob->Ls, prob->Hs, prob->ds);
+    if (s != CB_OK) return s;
+    if (out_dtype != CB_DTYPE_BF16 && out_dtype != CB_DTYPE_F32) return CB_ERR_INVALID_ARG;
+    if (src_cache->n_tokens == 0) return CB_OK;
+    if (!Wb || !tgt_k || !tgt_v) return CB_ERR_INVALID_ARG;
+    if ((((uintptr_t)tgt_k | (uintptr_t)tgt_v | (uintptr_t)Wb) & 15)) return CB_ERR_INVALID_ARG;
+    if (t_stride_layer < 0 || t_stride_token <= 0 || t_stride_head < 0) return CB_ERR_INVALID_ARG;
+    if ((t_stride_layer | t_stride_token | t_stride_head) & 7) return CB_ERR_INVALID_ARG;
+
+    ApplyArgs a;
+    a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src_cache->k), static_cast<const __nv_bfloat16 *>(src_cache->v),
+                  src_cache->stride_layer, src_cache->stride_token, src_cache->stride_head};
+    a.Wb = Wb; a.out_k = tgt_k; a.out_v = tgt_v;
+    a.o_sl = t_stride_layer; a.o_st = t_stride_token; a.o_sh = t_stride_head;
+    a.out_dtype = out_dtype;
+    a.n_tokens = (int)src_cache->n_tokens;
+    a.Lt = prob->Lt; a.Ht = prob->Ht;
+    std::memset(a.src_layer, 0, sizeof a.src_layer);
+    std::memset(a.src_head, 0, sizeof a.src_head);
+    for (int l = 0; l < prob->Lt; ++l) a.src_layer[l] = prob->src_layer[l];
+    for (int h = 0; h < prob->Ht; ++h) a.src_head[h] = prob->src_head[h];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = (prob->flags & CB_FLAG_SIMT) ? launch_apply_simt(a, prob->ds, st)
+                                                 : launch_apply_tc(a, prob->ds, src_cache, st);
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+cb_status cb_device_status(cb_ctx *ctx, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    int h = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(&h, ctx->ws + ctx->lay.status_off, sizeof h, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return h == DEV_OK ? CB_OK : CB_ERR_TIMEOUT;
+}
+
+}  // extern "C"

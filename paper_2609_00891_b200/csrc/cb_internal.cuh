@@ -1,0 +1,67 @@
+// Internal declarations shared by the translation units of the library (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "cb.h"
+
+namespace cb {
+
+// ---- partial-statistics slot -------------------------------------------------------------------------
+// One slot holds the fp32 partial statistics of one (split, map):
+//   D   [d][2d]  D[i][j]     = sum_t w x_i x_j   (j <  d)      -> S_xx
+//                D[i][d + j] = sum_t w x_i y_j                 -> S_xy
+//   s_x [d], s_y [d], s_w, 3 floats of padding (keeps every slot 16-byte aligned)
+__host__ __device__ constexpr int slot_floats(int d) { return d * 2 * d + 2 * d + 4; }
+__host__ __device__ constexpr int slot_sx(int d) { return d * 2 * d; }
+__host__ __device__ constexpr int slot_sy(int d) { return d * 2 * d + d; }
+__host__ __device__ constexpr int slot_sw(int d) { return d * 2 * d + 2 * d; }
+
+// Device-side status word values.
+enum : int { DEV_OK = 0, DEV_TIMEOUT = 1 };
+
+// A resolved strided view of K and V (element strides).
+struct KVPtr {
+    const __nv_bfloat16 *k, *v;
+    long long sl, st, sh;
+};
+
+struct AccumArgs {
+    KVPtr src, tgt;
+    const float *w_k, *w_v;
+    long long w_sl, w_sh;
+    int n_tokens;
+    int Lt, Ht, n_splits;
+    const int *src_layer;  // device [Lt]
+    const int *src_head;   // device [Ht]
+    float *slots;          // device [n_splits][n_maps][slot_floats]
+    int *status;           // device status word
+    int compensated;
+};
+
+struct ApplyArgs {
+    KVPtr src;
+    const float *Wb;       // [n_maps][p][d]
+    void *out_k, *out_v;
+    long long o_sl, o_st, o_sh;
+    int out_dtype;
+    int n_tokens;
+    int Lt, Ht;
+    int src_layer[128];    // by value: cb_apply takes no context
+    int src_head[64];
+};
+
+// Launchers (each returns the cudaError_t of its launch and bumps the launch counter on success).
+cudaError_t launch_accum_simt(const AccumArgs &a, int d, cudaStream_t st);
+cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st);
+cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, float *G, float *C, cudaStream_t st);
+cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long long n_tokens,
+                         const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st);
+cudaError_t launch_apply_simt(const ApplyArgs &a, int d, cudaStream_t st);
+cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cudaStream_t st);
+
+void count_launch(int n = 1);
+
+}  // namespace cb

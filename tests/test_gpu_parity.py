@@ -1,0 +1,242 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle on the same seeded inputs.
+
+Tolerance: relative Frobenius error <= 1e-3 on G, C, the fitted maps and the mapped cache (the stated target);
+integer outputs (token count, info) bit-exact.  Errors are checked per map as well as pooled."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_00891_b200 import binding as cb
+from paper_2609_00891_b200 import synth
+from util import bits, rel_fro, max_rel_fro_per_map
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-3
+DEV = "cuda"
+
+
+def _chunks(wl, sl, sh):
+    law = synth.map_law(wl)
+    return [synth.make_chunk(wl, c, sl, sh, law=law) for c in range(wl.n_chunks)]
+
+
+def _oracle_stats(chunks, sl, sh, maps=None):
+    G = C = None
+    for ch in chunks:                                     # additivity over chunks is itself an oracle pin
+        g, c = oracle.stats_traces(bits(ch["src_k"]), bits(ch["src_v"]), bits(ch["tgt_k"]), bits(ch["tgt_v"]),
+                                   ch["w_k"].numpy(), ch["w_v"].numpy(), sl, sh, maps)
+        G, C = (g, c) if G is None else (G + g, C + c)
+    return G, C
+
+
+def _gpu_stats(wl, chunks, sl, sh, flags, n_splits=0, head_major=False):
+    prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, flags=flags, n_splits=n_splits)
+    ctx = cb.cb_create(prob, device=DEV)
+    for ch in chunks:
+        t = {k: v.to(DEV) for k, v in ch.items() if torch.is_tensor(v)}
+        if head_major:                                    # storage [L][H][T][d], indexed [L][T][H][d]
+            for k in ("src_k", "src_v", "tgt_k", "tgt_v"):
+                t[k] = t[k].permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        cb.cb_stats_accumulate(ctx, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], t["w_k"], t["w_v"])
+    p, d = wl.d + 1, wl.d
+    G = torch.full((wl.n_maps, p, p), float("nan"), device=DEV)
+    C = torch.full((wl.n_maps, p, d), float("nan"), device=DEV)
+    n = cb.cb_stats_reduce(ctx, G, C)
+    cb.cb_device_status(ctx)
+    return prob, ctx, G, C, n
+
+
+def _check_stats(G, C, Go, Co, tol=TOL):
+    Gc, Cc = G.cpu().numpy(), C.cpu().numpy()
+    assert np.isfinite(Gc).all() and np.isfinite(Cc).all()
+    assert np.array_equal(Gc, Gc.transpose(0, 2, 1))      # symmetrised exactly
+    assert rel_fro(Gc, Go) <= tol and rel_fro(Cc, Co) <= tol
+    assert max_rel_fro_per_map(Gc, Go) <= tol and max_rel_fro_per_map(Cc, Co) <= tol
+    return rel_fro(Gc, Go), rel_fro(Cc, Co)
+
+
+CASES = [
+    ("tiny", cb.CB_FLAG_SIMT, 0),
+    ("tiny", cb.CB_FLAG_COMPENSATED, 0),
+    ("tiny", 0, 3),
+    ("mini_scaled", cb.CB_FLAG_SIMT, 0),
+    ("mini_scaled", cb.CB_FLAG_COMPENSATED, 0),
+    ("mini_scaled", 0, 1),
+    ("mini_ragged", cb.CB_FLAG_COMPENSATED, 7),
+    ("mini_ragged", 0, 0),
+]
+
+
+@pytest.mark.parametrize("name,flags,n_splits", CASES)
+def test_statistics_match_oracle(name, flags, n_splits):
+    wl = synth.workload(name)
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    chunks = _chunks(wl, sl, sh)
+    Go, Co = _oracle_stats(chunks, sl, sh)
+    prob, ctx, G, C, n = _gpu_stats(wl, chunks, sl, sh, flags, n_splits)
+    assert n == wl.n_tokens
+    eg, ec = _check_stats(G, C, Go, Co)
+    print("%s flags=%d: rel err G %.2e C %.2e" % (name, flags, eg, ec))
+    if flags & (cb.CB_FLAG_SIMT | cb.CB_FLAG_COMPENSATED):
+        assert eg <= 2e-5 and ec <= 2e-5                  # fp32 fold / hi+lo fold: far below the bf16 fold's error
+
+
+def test_head_major_layout_gives_identical_statistics():
+    wl = synth.workload("mini_scaled")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    chunks = _chunks(wl, sl, sh)
+    _, _, G1, C1, _ = _gpu_stats(wl, chunks, sl, sh, 0)
+    _, _, G2, C2, _ = _gpu_stats(wl, chunks, sl, sh, 0, head_major=True)
+    assert torch.equal(G1, G2) and torch.equal(C1, C2)    # same tiles, same order: bitwise
+    _, _, G3, C3, _ = _gpu_stats(wl, chunks, sl, sh, 0)
+    assert torch.equal(G1, G3) and torch.equal(C1, C3)    # run-to-run reproducible
+
+
+def test_reset_and_continue():
+    wl = synth.workload("mini_ragged")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    chunks = _chunks(wl, sl, sh)
+    prob, ctx, G, C, n = _gpu_stats(wl, chunks[:1], sl, sh, cb.CB_FLAG_COMPENSATED)
+    Go, Co = _oracle_stats(chunks[:1], sl, sh)
+    _check_stats(G, C, Go, Co)
+    t = {k: v.to(DEV) for k, v in chunks[1].items() if torch.is_tensor(v)}
+    cb.cb_stats_accumulate(ctx, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], t["w_k"], t["w_v"])   # continue after a reduce
+    n2 = cb.cb_stats_reduce(ctx, G, C)
+    Go2, Co2 = _oracle_stats(chunks[:2], sl, sh)
+    assert n2 == wl.chunk_tokens(0) + wl.chunk_tokens(1)
+    _check_stats(G, C, Go2, Co2)
+    cb.cb_stats_reset(ctx)
+    assert cb.cb_stats_reduce(ctx, G, C) == 0
+    assert not G.any() and not C.any()
+    # empty call is a no-op
+    e = {k: v[:, :0] if k[:3] in ("src", "tgt") else v[:, :, :0] for k, v in t.items()}
+    cb.cb_stats_accumulate(ctx, e["src_k"], e["src_v"], e["tgt_k"], e["tgt_v"], e["w_k"], e["w_v"])
+    assert cb.cb_stats_reduce(ctx, G, C) == 0 and not G.any()
+
+
+@pytest.mark.parametrize("T", [1, 63, 64, 65, 200])
+def test_few_tokens(T):
+    wl = synth.workload("mini_scaled")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    ch = _chunks(wl, sl, sh)[0]
+    cut = {k: (v[:, :T].contiguous() if k[:3] in ("src", "tgt") else v[:, :, :T].contiguous()) for k, v in ch.items() if torch.is_tensor(v)}
+    Go, Co = _oracle_stats([cut], sl, sh)
+    for flags in (cb.CB_FLAG_SIMT, cb.CB_FLAG_COMPENSATED):
+        _, _, G, C, n = _gpu_stats(wl, [cut], sl, sh, flags)
+        assert n == T
+        _check_stats(G, C, Go, Co)
+
+
+@pytest.mark.parametrize("name,flags", [("tiny", cb.CB_FLAG_COMPENSATED), ("mini_ragged", cb.CB_FLAG_COMPENSATED),
+                                        ("mini_scaled", cb.CB_FLAG_SIMT)])
+def test_fit_and_mapped_cache_match_oracle(name, flags):
+    wl = synth.workload(name)
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    chunks = _chunks(wl, sl, sh)
+    Go, Co = _oracle_stats(chunks, sl, sh)
+    prob, ctx, G, C, n = _gpu_stats(wl, chunks, sl, sh, flags)
+    p, d, nl = wl.d + 1, wl.d, len(wl.lambdas)
+    Wb = torch.full((nl, wl.n_maps, p, d), float("nan"), device=DEV)
+    info = torch.full((nl, wl.n_maps), -1, dtype=torch.int32, device=DEV)
+    cb.cb_ridge_solve(G, C, n, wl.lambdas, 0, Wb, info)
+    cb.cb_check_info(info)
+    assert not info.any()
+    src = synth.make_source_cache(wl, wl.apply_tokens) if wl.apply_tokens else [chunks[0]["src_k"], chunks[0]["src_v"]]
+    for li, lam in enumerate(wl.lambdas):
+        To, io = oracle.ridge_solve(Go, Co, wl.n_tokens, lam)
+        assert not io.any()
+        Wg = Wb[li].cpu().numpy()
+        assert rel_fro(Wg, To) <= TOL and max_rel_fro_per_map(Wg, To) <= TOL
+    # mapped cache with the GPU's own maps (last lambda), fp32 and bf16 outputs
+    (ok, ov), (bk, bv) = oracle.apply_maps(bits(src[0]), bits(src[1]), To, wl.Lt, wl.Ht, sl, sh)
+    T = src[0].shape[1]
+    for dtype in (torch.float32, torch.bfloat16):
+        out_k = torch.zeros(wl.Lt, T, wl.Ht, d, dtype=dtype, device=DEV)
+        out_v = torch.zeros_like(out_k)
+        cb.cb_apply(prob, Wb[nl - 1], src[0].to(DEV), src[1].to(DEV), out_k, out_v)
+        torch.cuda.synchronize()
+        if dtype == torch.float32:
+            assert rel_fro(out_k.cpu().numpy(), ok) <= TOL and rel_fro(out_v.cpu().numpy(), ov) <= TOL
+        else:
+            # decode-ready cache: compare with the oracle rounded to bf16 the same way
+            ek = rel_fro(out_k.float().cpu().numpy(), oracle.bf16_decode(bk))
+            ev = rel_fro(out_v.float().cpu().numpy(), oracle.bf16_decode(bv))
+            print("bf16 mapped cache rel err K %.2e V %.2e" % (ek, ev))
+            assert ek <= 2e-3 and ev <= 2e-3            # made of 1-ulp flips of a 2^-9 grid
+            ulp_k = np.abs(bits(out_k).astype(np.int32) - bk.astype(np.int32))
+            assert ulp_k.max() <= 1
+
+
+def test_solve_alone_against_oracle_on_the_same_statistics():
+    wl = synth.workload("mini_ragged")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    Go, Co = _oracle_stats(_chunks(wl, sl, sh)[:1], sl, sh)
+    G32, C32 = Go.astype(np.float32), Co.astype(np.float32)
+    n = wl.chunk_tokens(0)
+    lams = [1e-3, 1e-2, 1e-1, 10.0]
+    G = torch.from_numpy(G32).to(DEV)
+    C = torch.from_numpy(C32).to(DEV)
+    p, d = wl.d + 1, wl.d
+    for flags in (0, cb.CB_FLAG_RAW_LAMBDA):
+        Wb = torch.empty(len(lams), wl.n_maps, p, d, device=DEV)
+        info = torch.empty(len(lams), wl.n_maps, dtype=torch.int32, device=DEV)
+        cb.cb_ridge_solve(G, C, n, lams, flags, Wb, info)
+        cb.cb_check_info(info)
+        for li, lam in enumerate(lams):
+            To, _ = oracle.ridge_solve(G32.astype(np.float64), C32.astype(np.float64), n, lam, raw_lambda=bool(flags))
+            assert max_rel_fro_per_map(Wb[li].cpu().numpy(), To) <= 1e-5      # same inputs, fp64 both sides, fp32 out
+
+
+def test_degenerate_map_is_reported_and_zero_filled():
+    wl = synth.workload("tiny")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    ch = _chunks(wl, sl, sh)[0]
+    ch["w_k"][1, 0] = 0.0                                  # map (K, layer 1, head 0) sees no weight at all
+    m_bad = (0 * wl.Lt + 1) * wl.Ht + 0
+    prob, ctx, G, C, n = _gpu_stats(wl, [ch], sl, sh, cb.CB_FLAG_COMPENSATED)
+    p, d = wl.d + 1, wl.d
+    Wb = torch.full((1, wl.n_maps, p, d), float("nan"), device=DEV)
+    info = torch.full((1, wl.n_maps), -1, dtype=torch.int32, device=DEV)
+    cb.cb_ridge_solve(G, C, n, [1e-2], 0, Wb, info)
+    with pytest.raises(cb.CbError) as e:
+        cb.cb_check_info(info)
+    assert e.value.status == cb.CB_ERR_NOT_PD
+    Go, Co = _oracle_stats([ch], sl, sh)
+    To, io = oracle.ridge_solve(Go, Co, n, 1e-2)
+    assert np.array_equal(info[0].cpu().numpy() != 0, io != 0) and io[m_bad] != 0
+    assert not Wb[0, m_bad].any() and torch.isfinite(Wb).all()
+
+
+def test_apply_alone_with_oracle_maps():
+    wl = synth.workload("mini_ragged")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    rng = np.random.default_rng(5)
+    p, d = wl.d + 1, wl.d
+    Th = (rng.standard_normal((wl.n_maps, p, d)) / np.sqrt(d)).astype(np.float32)
+    src = synth.make_source_cache(wl, 333)
+    (ok, ov), (bk, bv) = oracle.apply_maps(bits(src[0]), bits(src[1]), Th.astype(np.float64), wl.Lt, wl.Ht, sl, sh)
+    for flags in (0, cb.CB_FLAG_SIMT):
+        prob = cb.Problem(wl.Ls, wl.Hs, d, wl.Lt, wl.Ht, d, sl, sh, flags=flags)
+        out_k = torch.zeros(wl.Lt, 333, wl.Ht, d, dtype=torch.float32, device=DEV)
+        out_v = torch.zeros_like(out_k)
+        cb.cb_apply(prob, torch.from_numpy(Th).to(DEV), src[0].to(DEV), src[1].to(DEV), out_k, out_v)
+        assert rel_fro(out_k.cpu().numpy(), ok) <= 1e-5 and rel_fro(out_v.cpu().numpy(), ov) <= 1e-5
+        # identity map returns the source head bit for bit in bf16
+        I = np.zeros((wl.n_maps, p, d), np.float32)
+        I[:, :d] = np.eye(d)
+        ob_k = torch.zeros(wl.Lt, 333, wl.Ht, d, dtype=torch.bfloat16, device=DEV)
+        ob_v = torch.zeros_like(ob_k)
+        cb.cb_apply(prob, torch.from_numpy(I).to(DEV), src[0].to(DEV), src[1].to(DEV), ob_k, ob_v)
+        for l in range(wl.Lt):
+            for h in range(wl.Ht):
+                assert torch.equal(ob_k[l, :, h].cpu(), src[0][sl[l], :, sh[h]])
+                assert torch.equal(ob_v[l, :, h].cpu(), src[1][sl[l], :, sh[h]])
+
+
+def test_launch_counter_counts_kernels():
+    before = cb.cb_launch_count()
+    wl = synth.workload("tiny")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    _gpu_stats(wl, _chunks(wl, sl, sh), sl, sh, 0)
+    assert cb.cb_launch_count() == before + 2            # one accumulate, one reduce
