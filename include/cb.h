@@ -137,6 +137,20 @@ cb_status cb_stats_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_vi
                               int64_t w_stride_layer, int64_t w_stride_head, void *stream);
 
 /*
+ * The same accumulation for a chunk that lives in HOST memory (the end-to-end path of a streaming build whose
+ * traces do not fit on the device).  src/tgt are views of host memory and must be dense in the order
+ * [layer][token][head][channel] (stride_head = d, stride_token = H*d, stride_layer = n_tokens*H*d); w_k / w_v are
+ * host fp32 [Lt][Ht][n_tokens] dense.  staging is caller-owned DEVICE memory of at least
+ * cb_staging_bytes(prob, n_tokens) bytes, 256-byte aligned.  The call enqueues the host-to-device copies and then
+ * the accumulation on the stream; the host buffers (pinned memory gives asynchronous copies) and the staging
+ * buffer must stay untouched until that work has completed.
+ */
+cb_status cb_staging_bytes(const cb_problem *prob, int64_t n_tokens, size_t *bytes);
+cb_status cb_stats_accumulate_host(cb_ctx *ctx, const cb_kv_view *src_host, const cb_kv_view *tgt_host,
+                                   const float *w_k_host, const float *w_v_host,
+                                   void *staging, size_t staging_bytes, void *stream);
+
+/*
  * Deterministic reduction: sums the splits of every map in index order (fp64 inside), symmetrises
  * G <- (G + G^T)/2 and writes fp32  G [n_maps][p][p]  and  C [n_maps][p][d]  (device).  n_tokens_out (host,
  * may be NULL) receives the number of rows accumulated since the last reset; it is host bookkeeping and

@@ -23,7 +23,8 @@ CB_FLAG_COMPENSATED, CB_FLAG_RAW_LAMBDA, CB_FLAG_SIMT = 1, 2, 4
 CB_DTYPE_BF16, CB_DTYPE_F32 = 0, 1
 
 EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_workspace_bytes", "cb_create",
-           "cb_destroy", "cb_stats_reset", "cb_stats_accumulate", "cb_stats_reduce", "cb_ridge_solve",
+           "cb_destroy", "cb_stats_reset", "cb_stats_accumulate", "cb_staging_bytes", "cb_stats_accumulate_host",
+           "cb_stats_reduce", "cb_ridge_solve",
            "cb_check_info", "cb_apply", "cb_device_status", "cb_launch_count")
 
 
@@ -189,6 +190,25 @@ def cb_stats_accumulate(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k: torch.Ten
                                      ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
                                      ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
                                      _stream_ptr(stream)), "cb_stats_accumulate")
+
+
+def cb_staging_bytes(prob: Problem, n_tokens: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().cb_staging_bytes(ctypes.byref(prob.c), ctypes.c_int64(n_tokens), ctypes.byref(n)), "cb_staging_bytes")
+    return n.value
+
+
+def cb_stats_accumulate_host(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k, w_v, staging: torch.Tensor, stream=None) -> None:
+    """Host (CPU, ideally pinned) contiguous traces [L][T][H][d] bf16 and weights [Lt][Ht][T] fp32; `staging` is a
+    device uint8 tensor of at least cb_staging_bytes()."""
+    for t in (src_k, src_v, tgt_k, tgt_v, w_k, w_v):
+        assert t.device.type == "cpu" and t.is_contiguous()
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    assert staging.is_cuda and staging.dtype == torch.uint8
+    _check(lib().cb_stats_accumulate_host(ctx.handle, ctypes.byref(sv), ctypes.byref(tv),
+                                          ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                          ctypes.c_void_p(staging.data_ptr()), ctypes.c_size_t(staging.numel()),
+                                          _stream_ptr(stream)), "cb_stats_accumulate_host")
 
 
 def cb_stats_reduce(ctx: Context, G: torch.Tensor, C: torch.Tensor, stream=None) -> int:

@@ -246,6 +246,74 @@ cb_status cb_stats_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_vi
     return CB_OK;
 }
 
+static bool dense_view(const cb_kv_view *v)
+{
+    return v->stride_head == v->head_dim && v->stride_token == (int64_t)v->n_heads * v->head_dim &&
+           v->stride_layer == v->n_tokens * v->n_heads * v->head_dim;
+}
+
+struct StagingLayout { size_t src_k, src_v, tgt_k, tgt_v, w_k, w_v, total; };
+
+static StagingLayout staging_layout(const cb_problem *p, int64_t T)
+{
+    StagingLayout L;
+    const size_t sb = (size_t)p->Ls * T * p->Hs * p->ds * 2, tb = (size_t)p->Lt * T * p->Ht * p->dt * 2;
+    const size_t wb = (size_t)p->Lt * p->Ht * T * 4;
+    size_t o = 0;
+    L.src_k = o; o = align_up(o + sb, 256);
+    L.src_v = o; o = align_up(o + sb, 256);
+    L.tgt_k = o; o = align_up(o + tb, 256);
+    L.tgt_v = o; o = align_up(o + tb, 256);
+    L.w_k = o; o = align_up(o + wb, 256);
+    L.w_v = o; o = align_up(o + wb, 256);
+    L.total = o;
+    return L;
+}
+
+cb_status cb_staging_bytes(const cb_problem *prob, int64_t n_tokens, size_t *bytes)
+{
+    cb_status s = check_problem(prob);
+    if (s != CB_OK) return s;
+    if (!bytes || n_tokens < 0) return CB_ERR_INVALID_ARG;
+    *bytes = staging_layout(prob, n_tokens).total;
+    return CB_OK;
+}
+
+cb_status cb_stats_accumulate_host(cb_ctx *ctx, const cb_kv_view *src_host, const cb_kv_view *tgt_host,
+                                   const float *w_k_host, const float *w_v_host,
+                                   void *staging, size_t staging_bytes, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    const cb_problem &P = ctx->prob;
+    if (!src_host || !tgt_host) return CB_ERR_INVALID_ARG;
+    if (src_host->n_layers != P.Ls || src_host->n_heads != P.Hs || src_host->head_dim != P.ds) return CB_ERR_INVALID_ARG;
+    if (tgt_host->n_layers != P.Lt || tgt_host->n_heads != P.Ht || tgt_host->head_dim != P.dt) return CB_ERR_INVALID_ARG;
+    const int64_t T = src_host->n_tokens;
+    if (T < 0 || T != tgt_host->n_tokens) return CB_ERR_INVALID_ARG;
+    if (T == 0) return CB_OK;
+    if (!src_host->k || !src_host->v || !tgt_host->k || !tgt_host->v || !w_k_host || !w_v_host) return CB_ERR_INVALID_ARG;
+    if (!dense_view(src_host) || !dense_view(tgt_host)) return CB_ERR_INVALID_ARG;
+    const StagingLayout L = staging_layout(&P, T);
+    if (!staging || ((uintptr_t)staging & 255) || staging_bytes < L.total) return CB_ERR_WORKSPACE;
+    char *dv = static_cast<char *>(staging);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t sb = (size_t)P.Ls * T * P.Hs * P.ds * 2, tb = (size_t)P.Lt * T * P.Ht * P.dt * 2;
+    const size_t wb = (size_t)P.Lt * P.Ht * T * 4;
+    cudaError_t e = cudaMemcpyAsync(dv + L.src_k, src_host->k, sb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dv + L.src_v, src_host->v, sb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dv + L.tgt_k, tgt_host->k, tb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dv + L.tgt_v, tgt_host->v, tb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dv + L.w_k, w_k_host, wb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && w_v_host != w_k_host) e = cudaMemcpyAsync(dv + L.w_v, w_v_host, wb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    cb_kv_view s = *src_host, t = *tgt_host;
+    s.k = dv + L.src_k; s.v = dv + L.src_v;
+    t.k = dv + L.tgt_k; t.v = dv + L.tgt_v;
+    const float *wk = reinterpret_cast<const float *>(dv + L.w_k);
+    const float *wv = (w_v_host != w_k_host) ? reinterpret_cast<const float *>(dv + L.w_v) : wk;
+    return cb_stats_accumulate(ctx, &s, &t, wk, wv, (int64_t)P.Ht * T, T, stream);
+}
+
 cb_status cb_stats_reduce(cb_ctx *ctx, float *G, float *C, int64_t *n_tokens_out, void *stream)
 {
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
