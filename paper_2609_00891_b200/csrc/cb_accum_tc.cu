@@ -5,16 +5,27 @@
 // plus the bias sums s_x = sum w x, s_y = sum w y, s_w = sum w kept on the ALUs.
 //
 // Per thread block (one per SM, persistent over its units = (map, token split)):
-//   warp 0      TMA producer: tiles of TT tokens of X and Y go straight from the strided cache layout to shared
-//               memory (128-byte swizzle: one row = one token's 64 channels), NS stages deep.
-//   warps 2-9   fold: read the X tile, multiply each token row by its weight, round to bf16 (optionally hi+lo)
-//               into the A buffer in the same swizzled layout; accumulate the bias sums in registers.
+//   warp 0      TMA producer for X: tiles of TT tokens go straight from the strided cache layout to shared memory
+//               (128-byte swizzle: one row = one token's 64 channels), NS stages deep.  The last warp does the
+//               same for Y and copies the tile's token weights.
+//   fold warps  read the X tile, multiply each token row by its weight, round to bf16 (optionally hi+lo) into
+//               the A buffer in the same swizzled layout; accumulate the bias sums in registers.
 //   warp 1      MMA issuer: tcgen05.mma, A = weighted tile (M = 128 channels, MN-major), B = [X | Y]
 //               (N = 2d channels, MN-major), K = tokens, fp32 accumulator in tensor memory.
-//   warps 10-13 drain: when a unit's accumulator is complete, tensor memory -> registers -> read-modify-write of
+//   drain warps (4): when a unit's accumulator is complete, tensor memory -> registers -> read-modify-write of
 //               the unit's fp32 partial slot; two accumulators let the next unit start meanwhile.
 // Every wait is bounded: if one runs out the block sets the context's status word and tears down.
 #include <cudaTypedefs.h>
+
+#ifndef CB_NS
+#define CB_NS 5
+#endif
+#ifndef CB_NA
+#define CB_NA 2
+#endif
+#ifndef CB_FOLD_WARPS
+#define CB_FOLD_WARPS 16
+#endif
 
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
@@ -23,36 +34,71 @@ namespace cb {
 
 using namespace ptx;
 
-template <int D>
+template <int D, bool COMP>
 struct TcCfg {
     static constexpr int TT = 64;                     // tokens per tile
     static constexpr int NBX = D / 64;                // 64-channel blocks per head
     static constexpr int BLK = TT * 128;              // bytes of one block: TT rows of 128 bytes
     static constexpr int STAGE_BYTES = 2 * NBX * BLK; // X blocks, then Y blocks
     static constexpr int A_BYTES = 2 * BLK;           // M = 128 always: two blocks (second stays zero for d = 64)
-    static constexpr int NS = 4;                      // X/Y stages
-    static constexpr int NA = 2;                      // weighted-operand buffers (each hi + lo)
+    static constexpr int NS = COMP ? 4 : CB_NS;       // X/Y stages
+    static constexpr int NA = COMP ? 2 : CB_NA;                    // weighted-operand buffers (hi, and lo when compensated)
+    static constexpr int A_PARTS = COMP ? 2 : 1;
     static constexpr int N = 2 * D;                   // accumulator columns
     static constexpr int TMEM_COLS = 2 * N;           // two accumulators
-    static constexpr int FOLD_WARPS = 8, DRAIN_WARPS = 4;
+    static constexpr int FOLD_WARPS = CB_FOLD_WARPS, DRAIN_WARPS = 4;
+    static constexpr int YPROD_WARP = 2 + FOLD_WARPS + DRAIN_WARPS;   // second producer: target tiles + weights
     static constexpr int FOLD_THREADS = FOLD_WARPS * 32;
-    static constexpr int THREADS = (2 + FOLD_WARPS + DRAIN_WARPS) * 32;
+    static constexpr int THREADS = (3 + FOLD_WARPS + DRAIN_WARPS) * 32;
     static constexpr int CC = D / 8;                  // 16-byte chunk columns of a head row
     static constexpr int RG = FOLD_THREADS / CC;      // row groups
     static constexpr int RPT = TT / RG;               // rows per fold thread
     static constexpr int RED_STRIDE = 2 * D + 4;                 // per fold warp: s_x[D], s_y[D], s_w, pad
     static constexpr int RED_FLOATS = FOLD_WARPS * RED_STRIDE;      // cross-warp bias reduction buffer
-    static constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)NS * STAGE_BYTES + (size_t)NA * 2 * A_BYTES +
-                                         RED_FLOATS * 4 + 256 /*barriers*/;
+    static constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)NS * STAGE_BYTES + (size_t)NA * A_PARTS * A_BYTES +
+                                         RED_FLOATS * 4 + NS * TT * 4 /*weights*/ + 256 /*barriers*/;
     static_assert(TT % RG == 0 && RPT >= 1, "fold layout");
     static_assert(TMEM_COLS == 256 || TMEM_COLS == 512, "tensor memory columns must be a power of two");
 };
 
 struct TcParams {
-    CUtensorMap src_k, src_v, tgt_k, tgt_v;   // 4-D tiled maps, innermost dimension = channels
+    CUtensorMap src_k, src_v, tgt_k, tgt_v;   // 5-D tiled maps: (64 channels, token, channel block, head, layer)
     AccumArgs a;
-    int s_pos[3], t_pos[3];                   // coordinate slot (1..3) of head, token, layer in each map
     int drain_tiles;                          // tiles accumulated in tensor memory between drains
+};
+
+// Walks the tiles of this block's units in order: units u = blockIdx.x, += gridDim.x; unit -> (map, split)
+// -> tiles [tile0, tile1).  Empty units are skipped.
+struct TileIter {
+    int u, tile, tile1, m, split;
+    int comp, l, h, j, g;          // decoded once per unit: component, target layer/head, matched source layer/head
+    __device__ __forceinline__ void start(const AccumArgs &a, int n_units, int n_maps, int n_tiles)
+    {
+        u = (int)blockIdx.x - (int)gridDim.x;
+        tile = tile1 = 0;
+        next_unit(a, n_units, n_maps, n_tiles);
+    }
+    __device__ __forceinline__ bool valid(int n_units) const { return u < n_units; }
+    __device__ __forceinline__ void next_unit(const AccumArgs &a, int n_units, int n_maps, int n_tiles)
+    {
+        do {
+            u += gridDim.x;
+            if (u >= n_units) return;
+            m = u % n_maps;
+            split = u / n_maps;
+            tile = (int)(((long long)n_tiles * split) / a.n_splits);
+            tile1 = (int)(((long long)n_tiles * (split + 1)) / a.n_splits);
+        } while (tile >= tile1);
+        comp = m / (a.Lt * a.Ht);
+        l = (m / a.Ht) % a.Lt;
+        h = m % a.Ht;
+        j = a.src_layer[l];
+        g = a.src_head[h];
+    }
+    __device__ __forceinline__ void advance(const AccumArgs &a, int n_units, int n_maps, int n_tiles)
+    {
+        if (++tile >= tile1) next_unit(a, n_units, n_maps, n_tiles);
+    }
 };
 
 __device__ __forceinline__ void unpack_bf16x8(const uint4 &v, float *f)
@@ -71,19 +117,37 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
     return r;
 }
 
-template <int D>
-__global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_constant__ TcParams P)
+#ifdef CB_TRACE
+// Tuning aid: block 0 records clock64() of every role for tiles [CB_TRACE_T0, CB_TRACE_T0 + 64).
+#define CB_TRACE_T0 1000
+__device__ long long g_trace[64][40];
+#define CB_TR(itv, slot) do { if (blockIdx.x == 0 && lane == 0 && (itv) >= CB_TRACE_T0 && (itv) < CB_TRACE_T0 + 64) g_trace[(itv) - CB_TRACE_T0][slot] = clock64(); } while (0)
+extern "C" int cb_debug_trace(long long *host) { return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(g_trace)); }
+#else
+#define CB_TR(itv, slot) do {} while (0)
+#endif
+
+// Position in a ring of N buffers guarded by mbarriers: index and the parity of the current pass.
+template <int N>
+struct Ring {
+    uint32_t idx = 0, phase = 0;
+    __device__ __forceinline__ void next() { if (++idx == N) { idx = 0; phase ^= 1; } }
+};
+
+template <int D, bool COMP>
+__global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const __grid_constant__ TcParams P)
 {
-    using C = TcCfg<D>;
+    using C = TcCfg<D, COMP>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *xy = smem;                                       // [NS][STAGE_BYTES]
-    uint8_t *ab = xy + (size_t)C::NS * C::STAGE_BYTES;        // [NA][hi A_BYTES | lo A_BYTES]
-    float *red = reinterpret_cast<float *>(ab + (size_t)C::NA * 2 * C::A_BYTES);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(red + C::RED_FLOATS);
-    uint64_t *full = bars;                 // [NS] TMA landed
-    uint64_t *empty = full + C::NS;        // [NS] stage free: MMA done (1) + fold warps done (8)
-    uint64_t *afull = empty + C::NS;       // [NA] weighted operand written (8 fold warps)
+    uint8_t *ab = xy + (size_t)C::NS * C::STAGE_BYTES;        // [NA][hi A_BYTES (| lo A_BYTES)]
+    float *red = reinterpret_cast<float *>(ab + (size_t)C::NA * C::A_PARTS * C::A_BYTES);
+    float *wst = red + C::RED_FLOATS;                         // [NS][TT] token weights of the staged tile
+    uint64_t *bars = reinterpret_cast<uint64_t *>(wst + C::NS * C::TT);
+    uint64_t *full = bars;                 // [NS] tile landed: X bytes (1 arrival), Y bytes (1), weights (32 lanes)
+    uint64_t *empty = full + C::NS;        // [NS] stage free: MMA done (1) + every fold warp done
+    uint64_t *afull = empty + C::NS;       // [NA] weighted operand written (every fold warp)
     uint64_t *aempty = afull + C::NA;      // [NA] weighted operand consumed (MMA)
     uint64_t *accfull = aempty + C::NA;    // [2]  accumulator complete (MMA)
     uint64_t *accempty = accfull + 2;      // [2]  accumulator drained (4 drain warps)
@@ -99,7 +163,7 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
     const int n_tiles = (a.n_tokens + C::TT - 1) / C::TT;
 
     if (tid == 0) {
-        for (int i = 0; i < C::NS; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1 + C::FOLD_WARPS); }
+        for (int i = 0; i < C::NS; ++i) { mbar_init(&full[i], 2 + 32); mbar_init(&empty[i], 1 + C::FOLD_WARPS); }
         for (int i = 0; i < C::NA; ++i) { mbar_init(&afull[i], C::FOLD_WARPS); mbar_init(&aempty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&accfull[i], 1); mbar_init(&accempty[i], C::DRAIN_WARPS); }
         mbar_init(redfull, C::FOLD_WARPS);
@@ -113,7 +177,7 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
     if (D == 64 && warp >= 2 && warp < 2 + C::FOLD_WARPS) {
         // rows 64..127 of the M = 128 operand never get data: clear the second block of every A buffer once
         const int ft = tid - 64;
-        for (int i = ft; i < C::NA * 2 * (C::BLK / 16); i += C::FOLD_THREADS) {
+        for (int i = ft; i < C::NA * C::A_PARTS * (C::BLK / 16); i += C::FOLD_THREADS) {
             const int buf = i / (C::BLK / 16), off = i % (C::BLK / 16);
             *reinterpret_cast<uint4 *>(ab + (size_t)buf * C::A_BYTES + C::BLK + off * 16) = make_uint4(0, 0, 0, 0);
         }
@@ -124,73 +188,113 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // Every role walks the same sequence: units u = blockIdx.x, += gridDim.x; unit -> (map, split) -> tiles
-    // [tile0, tile1); sub-ranges of at most drain_tiles tiles share one accumulator.
+    // Every role walks the same tile sequence (TileIter).  The per-tile paths of the single-thread roles are kept
+    // to a handful of instructions: a lone thread issues one dependent instruction every several cycles, so every
+    // extra instruction there is paid once per tile by the whole pipeline.
     if (warp == 0) {
-        // ================================ TMA producer ================================
+        // ================================ X producer (one thread) ================================
         if (lane == 0) {
+            TileIter cur;
+            cur.start(a, n_units, n_maps, n_tiles);
+            Ring<C::NS> st;
             uint32_t it = 0;
-            for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-                const int m = u % n_maps, split = u / n_maps;
-                const int tile0 = (int)(((long long)n_tiles * split) / a.n_splits);
-                const int tile1 = (int)(((long long)n_tiles * (split + 1)) / a.n_splits);
-                const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
-                const int j = a.src_layer[l], g = a.src_head[h];
-                const CUtensorMap *ms = comp ? &P.src_v : &P.src_k;
-                const CUtensorMap *mt = comp ? &P.tgt_v : &P.tgt_k;
-                for (int tile = tile0; tile < tile1; ++tile, ++it) {
-                    const int s = it % C::NS;
-                    if (!mbar_wait(&empty[s], ((it / C::NS) & 1) ^ 1, abort_flag)) goto teardown;
-                    mbar_arrive_expect_tx(&full[s], C::STAGE_BYTES);
-                    uint8_t *dst = xy + (size_t)s * C::STAGE_BYTES;
-                    int cs[4], ct[4];
-                    cs[P.s_pos[0]] = g; cs[P.s_pos[1]] = tile * C::TT; cs[P.s_pos[2]] = j;
-                    ct[P.t_pos[0]] = h; ct[P.t_pos[1]] = tile * C::TT; ct[P.t_pos[2]] = l;
-#pragma unroll
-                    for (int b = 0; b < C::NBX; ++b) {
-                        tma_load_4d(dst + b * C::BLK, ms, &full[s], b * 64, cs[1], cs[2], cs[3]);
-                        tma_load_4d(dst + (C::NBX + b) * C::BLK, mt, &full[s], b * 64, ct[1], ct[2], ct[3]);
-                    }
-                }
+            while (cur.valid(n_units)) {
+                const CUtensorMap *map = cur.comp ? &P.src_v : &P.src_k;
+                const int g = cur.g, j = cur.j, u = cur.u;
+                do {   // tiles of one unit
+                    if (!mbar_wait(&empty[st.idx], st.phase ^ 1, abort_flag)) goto teardown;
+                    CB_TR(it, 0);
+                    mbar_arrive_expect_tx(&full[st.idx], C::STAGE_BYTES / 2);
+                    tma_load_5d(xy + st.idx * C::STAGE_BYTES, map, &full[st.idx], 0, cur.tile * C::TT, 0, g, j);
+                    CB_TR(it, 1);
+                    st.next();
+                    ++it;
+                    cur.advance(a, n_units, n_maps, n_tiles);
+                } while (cur.u == u);
             }
         }
+    } else if (warp == C::YPROD_WARP) {
+        // ================================ Y + weights producer ================================
+        // Lane 0 issues the Y tile copy; all 32 lanes copy the tile's token weights with 4-byte asynchronous copies
+        // (zero-filled past the last token, no alignment requirement) that arrive on the same barrier.
+        TileIter cur;
+        cur.start(a, n_units, n_maps, n_tiles);
+        Ring<C::NS> st;
+        uint32_t it = 0;
+        while (cur.valid(n_units)) {
+            const CUtensorMap *map = cur.comp ? &P.tgt_v : &P.tgt_k;
+            const int h = cur.h, l = cur.l, u = cur.u;
+            const float *w = (cur.comp ? a.w_v : a.w_k) + (long long)l * a.w_sl + (long long)h * a.w_sh;
+            do {
+                if (!mbar_wait_warp(&empty[st.idx], st.phase ^ 1, abort_flag, lane)) goto teardown;
+                CB_TR(it, 38);
+                const int tok0 = cur.tile * C::TT;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&full[st.idx], C::STAGE_BYTES / 2);
+                    tma_load_5d(xy + st.idx * C::STAGE_BYTES + C::NBX * C::BLK, map, &full[st.idx], 0, tok0, 0, h, l);
+                }
+#pragma unroll
+                for (int q = 0; q < C::TT / 32; ++q) {
+                    const int r = lane + 32 * q;
+                    const bool in = tok0 + r < a.n_tokens;
+                    cp_async_4(&wst[st.idx * C::TT + r], w + (in ? tok0 + r : 0), in ? 4u : 0u);
+                }
+                cp_async_arrive_noinc(&full[st.idx]);
+                CB_TR(it, 39);
+                st.next();
+                ++it;
+                cur.advance(a, n_units, n_maps, n_tiles);
+            } while (cur.u == u);
+        }
     } else if (warp == 1) {
-        // ================================ MMA issuer ================================
+        // ================================ MMA issuer (one thread) ================================
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, C::N, true, true);
+            // Operand descriptors differ only in their 14-bit start-address field: keep the constant upper word and
+            // the lower words of stage 0 / buffer 0, and step them with 32-bit adds.
+            const uint64_t proto = umma_smem_desc_sw128(0, C::BLK, 1024);
+            const uint32_t desc_hi = (uint32_t)(proto >> 32);
+            const uint32_t b_lo0 = (uint32_t)proto | ((smem_u32(xy) & 0x3FFFFu) >> 4);
+            const uint32_t a_lo0 = (uint32_t)proto | ((smem_u32(ab) & 0x3FFFFu) >> 4);
+            Ring<C::NS> st;
+            Ring<C::NA> ar;
             uint32_t it = 0, sr = 0;
-            for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-                const int split = u / n_maps;
-                const int tile0 = (int)(((long long)n_tiles * split) / a.n_splits);
-                const int tile1 = (int)(((long long)n_tiles * (split + 1)) / a.n_splits);
-                for (int sr0 = tile0; sr0 < tile1; sr0 += P.drain_tiles, ++sr) {
-                    const int sr1 = min(tile1, sr0 + P.drain_tiles);
-                    const int acc = sr & 1;
+            TileIter cur;
+            cur.start(a, n_units, n_maps, n_tiles);
+            while (cur.valid(n_units)) {
+                const int u = cur.u, tile1 = cur.tile1;
+                for (int sr0 = cur.tile; sr0 < tile1; sr0 += P.drain_tiles, ++sr) {
+                    const int n_sub = min(tile1 - sr0, P.drain_tiles);
+                    const uint32_t acc = sr & 1;
                     if (!mbar_wait(&accempty[acc], ((sr >> 1) & 1) ^ 1, abort_flag)) goto teardown;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * C::N;
-                    for (int tile = sr0; tile < sr1; ++tile, ++it) {
-                        const int s = it % C::NS, ai = it % C::NA;
-                        if (!mbar_wait(&full[s], (it / C::NS) & 1, abort_flag)) goto teardown;
-                        if (!mbar_wait(&afull[ai], (it / C::NA) & 1, abort_flag)) goto teardown;
+                    uint32_t accum = 0;
+                    for (int t = 0; t < n_sub; ++t) {
+                        if (!mbar_wait(&full[st.idx], st.phase, abort_flag)) goto teardown;
+                        CB_TR(it, 2);
+                        if (!mbar_wait(&afull[ar.idx], ar.phase, abort_flag)) goto teardown;
+                        CB_TR(it, 3);
                         tc_fence_after();
-                        const uint32_t b_addr = smem_u32(xy + (size_t)s * C::STAGE_BYTES);
-                        const uint32_t a_addr = smem_u32(ab + (size_t)ai * 2 * C::A_BYTES);
+                        const uint32_t bl = b_lo0 + st.idx * (C::STAGE_BYTES >> 4);
+                        const uint32_t al = a_lo0 + ar.idx * ((C::A_PARTS * C::A_BYTES) >> 4);
 #pragma unroll
                         for (int k = 0; k < C::TT / 16; ++k) {
-                            const uint64_t bd = umma_smem_desc_sw128(b_addr + k * 2048, C::BLK, 1024);
-                            const uint64_t ad = umma_smem_desc_sw128(a_addr + k * 2048, C::BLK, 1024);
-                            umma_bf16_ss(d_tmem, ad, bd, idesc, (tile > sr0 || k > 0) ? 1u : 0u);
-                            if (a.compensated) {
-                                const uint64_t ld = umma_smem_desc_sw128(a_addr + C::A_BYTES + k * 2048, C::BLK, 1024);
-                                umma_bf16_ss(d_tmem, ld, bd, idesc, 1u);
-                            }
+                            const uint64_t bd = ((uint64_t)desc_hi << 32) | (bl + k * 128);
+                            umma_bf16_ss(d_tmem, ((uint64_t)desc_hi << 32) | (al + k * 128), bd, idesc, k == 0 ? accum : 1u);
+                            if (COMP) umma_bf16_ss(d_tmem, ((uint64_t)desc_hi << 32) | (al + (C::A_BYTES >> 4) + k * 128), bd, idesc, 1u);
                         }
-                        umma_commit(&empty[s]);
-                        umma_commit(&aempty[ai]);
+                        accum = 1;
+                        umma_commit(&empty[st.idx]);
+                        umma_commit(&aempty[ar.idx]);
+                        CB_TR(it, 4);
+                        st.next();
+                        ar.next();
+                        ++it;
                     }
                     umma_commit(&accfull[acc]);
                 }
+                while (cur.valid(n_units) && cur.u == u) cur.next_unit(a, n_units, n_maps, n_tiles);
             }
         }
     } else if (warp < 2 + C::FOLD_WARPS) {
@@ -198,49 +302,32 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
         const int ft = tid - 64;
         const int cc = ft % C::CC, rg = ft / C::CC;
         const int blk = cc >> 3, lc = cc & 7;
+        static_assert(C::RG % 8 == 0, "row groups must preserve the swizzle phase");
+        // byte offset of this thread's first 16-byte chunk inside a block; its other rows are RG rows further down
+        const int off0 = blk * C::BLK + rg * 128 + ((lc ^ (rg & 7)) << 4);
         float sx[8], sy[8], sw = 0.f;
+        Ring<C::NS> st;
+        Ring<C::NA> ar;
         uint32_t it = 0, uc = 0;
-        for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-            const int m = u % n_maps, split = u / n_maps;
-            const int tile0 = (int)(((long long)n_tiles * split) / a.n_splits);
-            const int tile1 = (int)(((long long)n_tiles * (split + 1)) / a.n_splits);
-            if (tile0 >= tile1) continue;
-            const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
-            const float *w = (comp ? a.w_v : a.w_k) + (long long)l * a.w_sl + (long long)h * a.w_sh;
+        TileIter cur;
+        cur.start(a, n_units, n_maps, n_tiles);
+        while (cur.valid(n_units)) {
+            const int m = cur.m, split = cur.split, n_t = cur.tile1 - cur.tile;
 #pragma unroll
             for (int e = 0; e < 8; ++e) sx[e] = sy[e] = 0.f;
             sw = 0.f;
-            float wn[C::RPT];
-#pragma unroll
-            for (int i = 0; i < C::RPT; ++i) {
-                const int t = tile0 * C::TT + rg + i * C::RG;
-                wn[i] = (t < a.n_tokens) ? __ldg(w + t) : 0.f;
-            }
-            for (int tile = tile0; tile < tile1; ++tile, ++it) {
-                float wc[C::RPT];
-#pragma unroll
-                for (int i = 0; i < C::RPT; ++i) wc[i] = wn[i];
-                if (tile + 1 < tile1) {
-#pragma unroll
-                    for (int i = 0; i < C::RPT; ++i) {
-                        const int t = (tile + 1) * C::TT + rg + i * C::RG;
-                        wn[i] = (t < a.n_tokens) ? __ldg(w + t) : 0.f;
-                    }
-                }
-                const int s = it % C::NS, ai = it % C::NA;
-                {
-                    bool ok = mbar_wait(&full[s], (it / C::NS) & 1, abort_flag);
-                    ok = ok && mbar_wait(&aempty[ai], ((it / C::NA) & 1) ^ 1, abort_flag);
-                    if (!__all_sync(0xffffffffu, ok)) goto teardown;
-                }
-                const uint8_t *xs = xy + (size_t)s * C::STAGE_BYTES + blk * C::BLK;
+            for (int t = 0; t < n_t; ++t) {
+                if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
+                if (!mbar_wait_warp(&aempty[ar.idx], ar.phase ^ 1, abort_flag, lane)) goto teardown;
+                CB_TR(it, 5 + 2 * (warp - 2));
+                const float *wsm = wst + st.idx * C::TT + rg;
+                const uint8_t *xs = xy + st.idx * C::STAGE_BYTES + off0;
                 const uint8_t *ys = xs + C::NBX * C::BLK;
-                uint8_t *ah = ab + (size_t)ai * 2 * C::A_BYTES + blk * C::BLK;
+                uint8_t *ah = ab + ar.idx * (C::A_PARTS * C::A_BYTES) + off0;
 #pragma unroll
                 for (int i = 0; i < C::RPT; ++i) {
-                    const int r = rg + i * C::RG;
-                    const int off = r * 128 + ((lc ^ (r & 7)) << 4);
-                    const float wt = wc[i];
+                    const int off = i * C::RG * 128;
+                    const float wt = wsm[i * C::RG];
                     float f[8], pr[8];
                     unpack_bf16x8(*reinterpret_cast<const uint4 *>(xs + off), f);
 #pragma unroll
@@ -249,7 +336,7 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
                     hi.x = pack_bf16x2(pr[0], pr[1]); hi.y = pack_bf16x2(pr[2], pr[3]);
                     hi.z = pack_bf16x2(pr[4], pr[5]); hi.w = pack_bf16x2(pr[6], pr[7]);
                     *reinterpret_cast<uint4 *>(ah + off) = hi;
-                    if (a.compensated) {
+                    if (COMP) {
                         float hf[8];
                         unpack_bf16x8(hi, hf);
                         uint4 lo;
@@ -264,10 +351,14 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0) { mbar_arrive(&afull[ai]); mbar_arrive(&empty[s]); }
+                if (lane == 0) { mbar_arrive(&afull[ar.idx]); mbar_arrive(&empty[st.idx]); }
+                CB_TR(it, 6 + 2 * (warp - 2));
+                st.next();
+                ar.next();
+                ++it;
             }
-            // ---- bias sums of this unit: lanes pair up (two row groups per warp when CC = 16), then a fixed-order
-            //      sum over the warps, then read-modify-write of the slot ----
+            // ---- bias sums of this unit: lanes holding the same channels add up, then a fixed-order sum over the
+            //      warps, then read-modify-write of the slot ----
             if (C::CC == 16) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -288,7 +379,7 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
             }
             const int fw = warp - 2;
             // red[fw][v], v in [0, 2D): s_x channels then s_y channels; red[fw][2D] = s_w
-            if (!__all_sync(0xffffffffu, mbar_wait(reddone, (uc & 1) ^ 1, abort_flag))) goto teardown;
+            if (!mbar_wait_warp(reddone, (uc & 1) ^ 1, abort_flag, lane)) goto teardown;
             float *rw = red + fw * C::RED_STRIDE;
             if (lane < C::CC) {
 #pragma unroll
@@ -297,7 +388,7 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(redfull);
-            if (!__all_sync(0xffffffffu, mbar_wait(redfull, uc & 1, abort_flag))) goto teardown;
+            if (!mbar_wait_warp(redfull, uc & 1, abort_flag, lane)) goto teardown;
             float *slot = a.slots + ((size_t)split * n_maps + m) * slot_floats(D);
             for (int v = ft; v < 2 * D + 1; v += C::FOLD_THREADS) {
                 float sum = 0.f;
@@ -308,38 +399,38 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
             __syncwarp();
             if (lane == 0) mbar_arrive(reddone);
             ++uc;
+            cur.next_unit(a, n_units, n_maps, n_tiles);
         }
     } else {
         // ================================ drain warps ================================
         const int q = warp & 3;             // tensor-memory lane quarter this warp may access
         const int row = q * 32 + lane;      // row of D = channel of the weighted operand
         uint32_t sr = 0;
-        for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-            const int m = u % n_maps, split = u / n_maps;
-            const int tile0 = (int)(((long long)n_tiles * split) / a.n_splits);
-            const int tile1 = (int)(((long long)n_tiles * (split + 1)) / a.n_splits);
-            float *slot = a.slots + ((size_t)split * n_maps + m) * slot_floats(D);
-            for (int sr0 = tile0; sr0 < tile1; sr0 += P.drain_tiles, ++sr) {
+        TileIter cur;
+        cur.start(a, n_units, n_maps, n_tiles);
+        while (cur.valid(n_units)) {
+            float *slot = a.slots + ((size_t)cur.split * n_maps + cur.m) * slot_floats(D);
+            for (int sr0 = cur.tile; sr0 < cur.tile1; sr0 += P.drain_tiles, ++sr) {
                 const int acc = sr & 1;
-                if (!__all_sync(0xffffffffu, mbar_wait(&accfull[acc], (sr >> 1) & 1, abort_flag))) goto teardown;
+                if (!mbar_wait_warp(&accfull[acc], (sr >> 1) & 1, abort_flag, lane, true, 4, 512)) goto teardown;
                 tc_fence_after();
                 if (row < D) {
                     float *grow = slot + (size_t)row * C::N;
 #pragma unroll 1
-                    for (int c = 0; c < C::N / 32; ++c) {
-                        uint32_t r[32];
-                        float4 g[8];
+                    for (int c = 0; c < C::N / 16; ++c) {
+                        uint32_t r[16];
+                        float4 g[4];
 #pragma unroll
-                        for (int v = 0; v < 8; ++v) g[v] = *reinterpret_cast<const float4 *>(grow + c * 32 + v * 4);
-                        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * C::N + c * 32, r);
+                        for (int v = 0; v < 4; ++v) g[v] = *reinterpret_cast<const float4 *>(grow + c * 16 + v * 4);
+                        tmem_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + acc * C::N + c * 16, r);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int v = 0; v < 8; ++v) {
+                        for (int v = 0; v < 4; ++v) {
                             g[v].x += __uint_as_float(r[4 * v + 0]);
                             g[v].y += __uint_as_float(r[4 * v + 1]);
                             g[v].z += __uint_as_float(r[4 * v + 2]);
                             g[v].w += __uint_as_float(r[4 * v + 3]);
-                            *reinterpret_cast<float4 *>(grow + c * 32 + v * 4) = g[v];
+                            *reinterpret_cast<float4 *>(grow + c * 16 + v * 4) = g[v];
                         }
                     }
                 }
@@ -347,6 +438,7 @@ __global__ void __launch_bounds__(TcCfg<D>::THREADS, 1) k_accum_tc(const __grid_
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&accempty[acc]);
             }
+            cur.next_unit(a, n_units, n_maps, n_tiles);
         }
     }
 
@@ -381,34 +473,20 @@ static PFN_cuTensorMapEncodeTiled_v12000 encode_fn()
     return fn;
 }
 
-// 4-D map over (channels, and head/token/layer ordered by ascending stride); pos[0..2] receive the coordinate
-// slot of head, token and layer.  Box: 64 channels x box_tokens tokens of one head of one layer.
+// 5-D map over (64 channels, token, 64-channel block, head, layer).  One box = box_tokens tokens of one head of
+// one layer, laid out in shared memory as [channel block][token][64 channels] with the 128-byte swizzle.
 bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long long T, int L,
-                        long long sh, long long st, long long sl, int box_tokens, int pos[3])
+                        long long sh, long long st, long long sl, int box_tokens)
 {
     PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
     if (!enc) return false;
-    struct Dim { unsigned long long size, stride_bytes; int which; };
-    Dim dims[3] = {{(unsigned long long)H, (unsigned long long)sh * 2, 0},
-                   {(unsigned long long)T, (unsigned long long)st * 2, 1},
-                   {(unsigned long long)L, (unsigned long long)sl * 2, 2}};
-    for (int i = 0; i < 3; ++i)
-        if (dims[i].size == 1 || dims[i].stride_bytes == 0) dims[i].stride_bytes = 0;   // placed first, fixed below
-    // ascending stride (stable insertion sort)
-    for (int i = 1; i < 3; ++i)
-        for (int k = i; k > 0 && dims[k].stride_bytes < dims[k - 1].stride_bytes; --k) { Dim t = dims[k]; dims[k] = dims[k - 1]; dims[k - 1] = t; }
-    cuuint64_t gdim[4] = {(cuuint64_t)d, 1, 1, 1};
-    cuuint64_t gstr[3];
-    cuuint32_t box[4] = {64, 1, 1, 1}, estr[4] = {1, 1, 1, 1};
-    for (int i = 0; i < 3; ++i) {
-        gdim[i + 1] = dims[i].size;
-        unsigned long long sb = dims[i].stride_bytes;
-        if (sb == 0) sb = (unsigned long long)d * 2;   // size-1 dimension: any valid stride
-        gstr[i] = sb;
-        pos[dims[i].which] = i + 1;
-        if (dims[i].which == 1) box[i + 1] = (cuuint32_t)box_tokens;
-    }
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), gdim, gstr, box, estr,
+    auto stride = [&](long long elems, long long size) -> cuuint64_t {
+        return (size == 1 || elems == 0) ? (cuuint64_t)d * 2 : (cuuint64_t)elems * 2;   // size-1 dimension: any valid stride
+    };
+    cuuint64_t gdim[5] = {64, (cuuint64_t)T, (cuuint64_t)(d / 64), (cuuint64_t)H, (cuuint64_t)L};
+    cuuint64_t gstr[4] = {stride(st, T), 128, stride(sh, H), stride(sl, L)};
+    cuuint32_t box[5] = {64, (cuuint32_t)box_tokens, (cuuint32_t)(d / 64), 1, 1}, estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), gdim, gstr, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
@@ -426,19 +504,19 @@ static int sm_count()
     return n;
 }
 
-template <int D>
+template <int D, bool COMP>
 static cudaError_t launch_tc(const TcParams &P, cudaStream_t st)
 {
-    using C = TcCfg<D>;
+    using C = TcCfg<D, COMP>;
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D, COMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr = true;
     }
     const int n_units = 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
     const int grid = n_units < sm_count() ? n_units : sm_count();
-    k_accum_tc<D><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
+    k_accum_tc<D, COMP><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -448,16 +526,18 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     P.a = a;
     const int TT = 64;
     if (!make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
-                            src->stride_token, src->stride_layer, TT, P.s_pos) ||
+                            src->stride_token, src->stride_layer, TT) ||
         !make_kv_tensor_map(&P.src_v, src->v, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
-                            src->stride_token, src->stride_layer, TT, P.s_pos) ||
+                            src->stride_token, src->stride_layer, TT) ||
         !make_kv_tensor_map(&P.tgt_k, tgt->k, d, tgt->n_heads, tgt->n_tokens, tgt->n_layers, tgt->stride_head,
-                            tgt->stride_token, tgt->stride_layer, TT, P.t_pos) ||
+                            tgt->stride_token, tgt->stride_layer, TT) ||
         !make_kv_tensor_map(&P.tgt_v, tgt->v, d, tgt->n_heads, tgt->n_tokens, tgt->n_layers, tgt->stride_head,
-                            tgt->stride_token, tgt->stride_layer, TT, P.t_pos))
+                            tgt->stride_token, tgt->stride_layer, TT))
         return cudaErrorInvalidValue;
     P.drain_tiles = 16384 / TT;   // at most 16384 tokens are summed in tensor memory before a drain
-    cudaError_t e = (d == 128) ? launch_tc<128>(P, st) : launch_tc<64>(P, st);
+    cudaError_t e;
+    if (a.compensated) e = (d == 128) ? launch_tc<128, true>(P, st) : launch_tc<64, true>(P, st);
+    else e = (d == 128) ? launch_tc<128, false>(P, st) : launch_tc<64, false>(P, st);
     if (e == cudaSuccess) count_launch();
     return e;
 }

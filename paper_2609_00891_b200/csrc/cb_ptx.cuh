@@ -45,20 +45,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 }
 
 // Bounded wait.  Returns false if the limit ran out or another thread of the block already gave up
-// (*abort_flag != 0); the caller then leaves its loop and the block tears down.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+// (*abort_flag != 0); the caller then leaves its loop and the block tears down.  After `fast_polls` failed polls
+// the thread sleeps `sleep_ns` between polls: every poll is a shared-memory transaction, and a block full of
+// spinning threads slows down the shared-memory pipe for the threads that do the work.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          uint32_t fast_polls = 1u << 14, uint32_t sleep_ns = 64)
 {
-    constexpr uint32_t kSpinFast = 2048;
-    constexpr uint32_t kSpinMax = 1u << 22;
-    for (uint32_t i = 0; i < kSpinMax; ++i) {
+    constexpr uint32_t kPollMax = 1u << 22;
+    for (uint32_t i = 0; i < kPollMax; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (i >= kSpinFast) {
-            if (*abort_flag) return false;
-            __nanosleep(64);
+        if (i >= fast_polls) {
+            if ((i & 63) == 0 && *abort_flag) return false;
+            __nanosleep(sleep_ns);
         }
     }
     *abort_flag = 1;
     return false;
+}
+
+// Warp-wide wait with a warp-uniform outcome.  `one_lane`: only lane 0 polls (for long, uncritical waits: fewer
+// shared-memory transactions); otherwise every lane polls, which reacts fastest.  All 32 lanes must call it.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int lane,
+                                               bool one_lane = false, uint32_t fast_polls = 1u << 14, uint32_t sleep_ns = 64)
+{
+    if (one_lane) {
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, fast_polls, sleep_ns) ? 1 : 0;
+        return __shfl_sync(0xffffffffu, ok, 0) != 0;
+    }
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, fast_polls, sleep_ns)) != 0;
 }
 
 // Make this thread's generic-proxy writes to shared memory visible to the async proxy (TMA, tensor cores).
@@ -72,9 +87,36 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, u
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+// One copy brings [c_hi][tokens][64 channels] (dims: c_lo, token, c_hi, head, layer).
+__device__ __forceinline__ void tma_load_5d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2, int c3, int c4)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+// Pull a tile into L2 ahead of its copy (no completion tracking).
+__device__ __forceinline__ void tma_prefetch_l2_5d(const CUtensorMap *map, int c0, int c1, int c2, int c3, int c4)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global.tile [%0, {%1, %2, %3, %4, %5}];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+// ---- asynchronous 4-byte copies (any alignment, zero fill when src_bytes == 0) --------------------------
+__device__ __forceinline__ void cp_async_4(void *dst_smem, const void *src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst_smem)), "l"(src), "r"(src_bytes) : "memory");
+}
+// The barrier receives one arrival from this thread once all its earlier asynchronous copies have landed; the
+// arrival must be part of the barrier's expected count.
+__device__ __forceinline__ void cp_async_arrive_noinc(uint64_t *bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
 // ---- tcgen05 -----------------------------------------------------------------------------------------
@@ -119,6 +161,16 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
 }
