@@ -177,8 +177,7 @@ cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, f
 // ======================================================================================================
 // Batched ridge solve, fp64, one block per (map, lambda).
 //   A = G + lambda_eff * diag(1,..,1,0);  A = L L^T (packed lower triangle, rows padded to even length);
-//   L Z = C, L^T Theta = Z with each of the first d threads owning one right-hand-side column and keeping
-//   eight rows in registers at a time.
+//   L Z = C, L^T Theta = Z.
 // ======================================================================================================
 struct SolveArgs {
     const float *G, *C;
@@ -198,46 +197,157 @@ __host__ __device__ inline int tri_row_start(int i)
     return 2 * h * (h + 1) + ((i & 1) ? (i + 1) : 0);
 }
 
-__global__ void __launch_bounds__(256) k_ridge_solve(const SolveArgs a)
+// shuffle of a double between lane pairs
+__device__ __forceinline__ double shfl_xor_f64(double v, int mask)
 {
+    int lo = __double2loint(v), hi = __double2hiint(v);
+    lo = __shfl_xor_sync(0xffffffffu, lo, mask);
+    hi = __shfl_xor_sync(0xffffffffu, hi, mask);
+    return __hiloint2double(hi, lo);
+}
+
+// Cholesky by block columns of 8 (left-looking): thread i owns row i.  For a block column it pulls its 8
+// entries into registers, subtracts the contributions of all finished columns (its own row times the 8 rows of
+// the diagonal block, read as broadcasts), the 8 diagonal-block rows publish theirs, every thread factors that
+// 8x8 block redundantly in registers and solves its own row against it.  Two block barriers per block column.
+// The substitutions give every right-hand-side column to a pair of lanes that split the inner sums; eight rows
+// are kept in registers at a time, so each loaded L entry feeds one FMA and each loaded Z entry feeds eight.
+#ifdef CB_SOLVE_TIMING
+__device__ long long g_solve_t[8];
+extern "C" int cb_debug_solve_t(long long *h) { return (int)cudaMemcpyFromSymbol(h, g_solve_t, sizeof(g_solve_t)); }
+#define ST(i) do { if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) g_solve_t[i] = clock64(); } while (0)
+#else
+#define ST(i) do {} while (0)
+#endif
+__global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
+{
+    ST(0);
     extern __shared__ __align__(16) double sm[];
+    constexpr int NB = 8;
     const int d = a.d, p = d + 1;
     const int m = blockIdx.x, li = blockIdx.y;
-    double *Lp = sm;                                   // packed lower triangle
+    double *Lp = sm;                                   // packed lower triangle, rows padded to even length
     double *Z = sm + tri_row_start(p);                 // [p][d]
+    __shared__ double diag[NB][NB];
+    __shared__ double rdiag[136];                      // reciprocals of the diagonal of L
     __shared__ int s_fail;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const int tid = threadIdx.x;
 
     const float *Gm = a.G + (size_t)m * p * p;
     const float *Cm = a.C + (size_t)m * p * d;
     const double s_w = (double)Gm[(size_t)d * p + d];
     const double lam = (a.flags & CB_FLAG_RAW_LAMBDA) ? (double)a.lambdas[li] : (double)a.lambdas[li] * s_w * a.inv_n;
     if (tid == 0) s_fail = 0;
-    for (int e = tid; e < p * p; e += blockDim.x) {
-        const int i = e / p, k = e % p;
-        if (k <= i) Lp[tri_row_start(i) + k] = (double)Gm[e] + ((i == k && i < d) ? lam : 0.0);
+    {
+        const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+        // one warp per row (coalesced, no divisions); the global loads of a row are issued together before any
+        // shared-memory store so that they overlap
+        constexpr int MAXV = 5;                            // ceil(129 / 32)
+        for (int i = warp; i < p; i += nwarps) {
+            const int rsi = tri_row_start(i);
+            float gv[MAXV], cv[MAXV];
+#pragma unroll
+            for (int v = 0; v < MAXV; ++v) {
+                const int k = lane + 32 * v;
+                gv[v] = (k <= i) ? __ldg(Gm + (size_t)i * p + k) : 0.f;
+                cv[v] = (k < d) ? __ldg(Cm + (size_t)i * d + k) : 0.f;
+            }
+#pragma unroll
+            for (int v = 0; v < MAXV; ++v) {
+                const int k = lane + 32 * v;
+                if (k <= i) Lp[rsi + k] = (double)gv[v] + ((i == k && i < d) ? lam : 0.0);
+                if (k < d) Z[(size_t)i * d + k] = (double)cv[v];
+            }
+        }
     }
-    for (int e = tid; e < p * d; e += blockDim.x) Z[e] = (double)Cm[e];
     __syncthreads();
 
-    // ---- right-looking Cholesky ----
-    for (int j = 0; j < p; ++j) {
-        if (tid == 0) {
-            const double s = Lp[tri_row_start(j) + j];
-            if (!(s > 0.0)) s_fail = j + 1;
-            else Lp[tri_row_start(j) + j] = sqrt(s);
+    ST(1);
+    // ---------------- Cholesky ----------------
+    const int row = tid;
+    const int rs = tri_row_start(row < p ? row : 0);
+    for (int j0 = 0; j0 < p; j0 += NB) {
+        const int nb = min(NB, p - j0);
+        double acc[NB];
+        const bool active = row < p && row >= j0;
+        if (active) {
+#pragma unroll
+            for (int c = 0; c < NB; ++c) acc[c] = (c < nb && j0 + c <= row) ? Lp[rs + j0 + c] : 0.0;
+            int drs[NB];
+#pragma unroll
+            for (int c = 0; c < NB; ++c) drs[c] = tri_row_start(min(j0 + c, p - 1));
+            for (int k = 0; k < j0; k += 2) {          // j0 is a multiple of 8: aligned pairs
+                const double2 mine = *reinterpret_cast<const double2 *>(&Lp[rs + k]);
+#pragma unroll
+                for (int c = 0; c < NB; ++c) {
+                    const double2 o = *reinterpret_cast<const double2 *>(&Lp[drs[c] + k]);
+                    acc[c] -= mine.x * o.x;
+                    acc[c] -= mine.y * o.y;
+                }
+            }
+            if (row < j0 + nb) {
+#pragma unroll
+                for (int c = 0; c < NB; ++c) diag[row - j0][c] = acc[c];
+            }
+        }
+        __syncthreads();
+        if (row == j0) {
+            // one thread factors the nb x nb diagonal block (sqrt and reciprocal are long fp64 sequences: doing
+            // them once and broadcasting beats doing them in every thread); the block is held in registers
+            double Ld[NB][NB];
+#pragma unroll
+            for (int r = 0; r < NB; ++r)
+#pragma unroll
+                for (int c = 0; c < NB; ++c)
+                    if (c <= r) Ld[r][c] = (r < nb) ? diag[r][c] : (r == c ? 1.0 : 0.0);
+            int fail = 0;
+#pragma unroll
+            for (int c = 0; c < NB; ++c) {
+                double v = Ld[c][c];
+#pragma unroll
+                for (int q = 0; q < NB; ++q)
+                    if (q < c) v -= Ld[c][q] * Ld[c][q];
+                if (!(v > 0.0)) { if (!fail) fail = j0 + c + 1; v = 1.0; }
+                const double ri = rsqrt(v);
+                Ld[c][c] = v * ri;
+                if (c < nb) rdiag[j0 + c] = ri;
+#pragma unroll
+                for (int r = 0; r < NB; ++r)
+                    if (r > c) {
+                        double u = Ld[r][c];
+#pragma unroll
+                        for (int q = 0; q < NB; ++q)
+                            if (q < c) u -= Ld[r][q] * Ld[c][q];
+                        Ld[r][c] = u * ri;
+                    }
+            }
+            if (fail) s_fail = fail;
+#pragma unroll
+            for (int r = 0; r < NB; ++r)
+#pragma unroll
+                for (int c = 0; c < NB; ++c)
+                    if (c <= r) diag[r][c] = Ld[r][c];
+        }
+        __syncthreads();
+        if (active) {
+            if (row >= j0 + nb) {
+                // own row against the block: x_c = (acc_c - sum_{q<c} x_q L[c][q]) / L[c][c]
+#pragma unroll
+                for (int c = 0; c < NB; ++c)
+                    if (c < nb) {
+                        double v = acc[c];
+#pragma unroll
+                        for (int q = 0; q < NB; ++q)
+                            if (q < c) v -= acc[q] * diag[c][q];
+                        acc[c] = v * rdiag[j0 + c];
+                        Lp[rs + j0 + c] = acc[c];
+                    }
+            } else {
+                for (int c = 0; c <= row - j0; ++c) Lp[rs + j0 + c] = diag[row - j0][c];
+            }
         }
         __syncthreads();
         if (s_fail) break;
-        const double inv = 1.0 / Lp[tri_row_start(j) + j];
-        for (int i = j + 1 + tid; i < p; i += blockDim.x) Lp[tri_row_start(i) + j] *= inv;
-        __syncthreads();
-        for (int i = j + 1 + warp; i < p; i += nwarps) {
-            const int rs = tri_row_start(i);
-            const double lij = Lp[rs + j];
-            for (int k = j + 1 + lane; k <= i; k += 32) Lp[rs + k] -= lij * Lp[tri_row_start(k) + j];
-        }
-        __syncthreads();
     }
 
     float *Wm = a.Wb + ((size_t)li * a.n_maps + m) * p * d;
@@ -247,53 +357,63 @@ __global__ void __launch_bounds__(256) k_ridge_solve(const SolveArgs a)
         return;
     }
 
+    ST(2);
+    // ---------------- substitutions: column c = tid / 2, the two lanes of a pair split the inner sums ----------------
     constexpr int RB = 8;
-    if (tid < d) {
-        const int c = tid;
-        // ---- forward: L Z = C, row blocks top-down ----
+    if (tid < 2 * d) {
+        const int c = tid >> 1, half = tid & 1;
+        // forward: L Z = C, row blocks top-down
         for (int i0 = 0; i0 < p; i0 += RB) {
             double acc[RB];
+            int rsr[RB];
 #pragma unroll
-            for (int r = 0; r < RB; ++r) acc[r] = (i0 + r < p) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
-            for (int k = 0; k < i0; k += 2) {          // i0 is a multiple of 8: pairs are aligned
+            for (int r = 0; r < RB; ++r) {
+                rsr[r] = tri_row_start(min(i0 + r, p - 1));
+                acc[r] = (half == 0 && i0 + r < p) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
+            }
+            for (int k = 2 * half; k < i0; k += 4) {   // pairs (k, k+1), alternating between the two lanes
                 const double z0 = Z[(size_t)k * d + c], z1 = Z[(size_t)(k + 1) * d + c];
 #pragma unroll
-                for (int r = 0; r < RB; ++r)
-                    if (i0 + r < p) {
-                        const double2 lv = *reinterpret_cast<const double2 *>(&Lp[tri_row_start(i0 + r) + k]);
-                        acc[r] -= lv.x * z0;
-                        acc[r] -= lv.y * z1;
-                    }
+                for (int r = 0; r < RB; ++r) {
+                    const double2 lv = *reinterpret_cast<const double2 *>(&Lp[rsr[r] + k]);
+                    acc[r] -= lv.x * z0;
+                    acc[r] -= lv.y * z1;
+                }
             }
+#pragma unroll
+            for (int r = 0; r < RB; ++r) acc[r] += shfl_xor_f64(acc[r], 1);
 #pragma unroll
             for (int r = 0; r < RB; ++r)
                 if (i0 + r < p) {
-                    const int rs = tri_row_start(i0 + r);
                     double v = acc[r];
 #pragma unroll
                     for (int q = 0; q < RB; ++q)
-                        if (q < r) v -= Lp[rs + i0 + q] * acc[q];
-                    v /= Lp[rs + i0 + r];
+                        if (q < r) v -= Lp[rsr[r] + i0 + q] * acc[q];
+                    v *= rdiag[i0 + r];
                     acc[r] = v;
-                    Z[(size_t)(i0 + r) * d + c] = v;
+                    if (half == 0) Z[(size_t)(i0 + r) * d + c] = v;
                 }
+            __syncwarp();
         }
-        // ---- backward: L^T Theta = Z, row blocks bottom-up ----
+        ST(3);
+        // backward: L^T Theta = Z, row blocks bottom-up
         const int last = ((p - 1) / RB) * RB;
         for (int i0 = last; i0 >= 0; i0 -= RB) {
             double acc[RB];
 #pragma unroll
-            for (int r = 0; r < RB; ++r) acc[r] = (i0 + r < p) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
-            for (int k = i0 + RB; k < p; ++k) {
+            for (int r = 0; r < RB; ++r) acc[r] = (half == 0 && i0 + r < p) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
+            for (int k = i0 + RB + half; k < p; k += 2) {
                 const double xk = Z[(size_t)k * d + c];
-                const int rs = tri_row_start(k) + i0;   // even offset: aligned double2 loads
+                const int rsk = tri_row_start(k) + i0;   // even offset: aligned pairs
 #pragma unroll
                 for (int r = 0; r < RB; r += 2) {
-                    const double2 lv = *reinterpret_cast<const double2 *>(&Lp[rs + r]);
+                    const double2 lv = *reinterpret_cast<const double2 *>(&Lp[rsk + r]);
                     acc[r] -= lv.x * xk;
                     acc[r + 1] -= lv.y * xk;
                 }
             }
+#pragma unroll
+            for (int r = 0; r < RB; ++r) acc[r] += shfl_xor_f64(acc[r], 1);
 #pragma unroll
             for (int r = RB - 1; r >= 0; --r)
                 if (i0 + r < p) {
@@ -301,15 +421,18 @@ __global__ void __launch_bounds__(256) k_ridge_solve(const SolveArgs a)
 #pragma unroll
                     for (int q = RB - 1; q >= 0; --q)
                         if (q > r && i0 + q < p) v -= Lp[tri_row_start(i0 + q) + i0 + r] * acc[q];
-                    v /= Lp[tri_row_start(i0 + r) + i0 + r];
+                    v *= rdiag[i0 + r];
                     acc[r] = v;
-                    Z[(size_t)(i0 + r) * d + c] = v;
+                    if (half == 0) Z[(size_t)(i0 + r) * d + c] = v;
                 }
+            __syncwarp();
         }
     }
     __syncthreads();
+    ST(4);
     for (int e = tid; e < p * d; e += blockDim.x) Wm[e] = (float)Z[e];
     if (tid == 0) a.info[(size_t)li * a.n_maps + m] = 0;
+    ST(5);
 }
 
 cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long long n_tokens,
