@@ -99,7 +99,7 @@ def oracle_sample(n_tokens: int, seed_chunk: int = 0):
     from paper_2609_00891_b200 import synth
 
     full = synth.workload(WORKLOAD)
-    wl = synth.Workload("oracle_sample", full.index, 3, full.Hs, 4, full.Ht, full.d, (n_tokens,), 1,
+    wl = synth.Workload("oracle_sample", full.index, 3, full.Hs, 4, full.Ht, full.d, (n_tokens,) * (seed_chunk + 1), 1,
                         full.lambdas, full.kind, full.noise)
     sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     ch = synth.make_chunk(wl, seed_chunk, sl, sh, device="cpu")
@@ -300,9 +300,9 @@ def main():
     cpu = None
     if not args.no_cpu:
         import oracle
-        dt, token_maps, rate = oracle_sample(32768)
+        dt, token_maps, rate = oracle_sample(131072)
         cpu = {"value": rate, "unit": "tokens/s", "cores": oracle.n_threads(), "kind": "oracle",
-               "sample": "64 maps x 32768 tokens of the same trace law (statistics + 3 solves) in %.1f s; "
+               "sample": "64 maps x 131072 tokens of the same trace law (statistics + 3 solves) in %.1f s; "
                          "tokens/s = token-maps / 1024 maps / s" % dt}
     out = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
