@@ -293,7 +293,9 @@ def main():
     tpath = os.path.join(ROOT, "profiles", "traffic_k_accum_tc.json")
     if os.path.exists(tpath):
         with open(tpath) as f:
-            roof["traffic"] = json.load(f).get("dram_bytes_per_token", 0) * tok_launch
+            t = json.load(f)     # ncu capture of a smaller launch, scaled: per-token part x tokens + slot read-modify-write per split
+            n_splits = args.splits if args.splits > 0 else 4
+            roof["traffic"] = t["dram_bytes_per_token"] * tok_launch + t["dram_bytes_fixed_per_split"] * n_splits
     t_roof = max(ALG_BYTES_PER_TOKEN * tokens_per_step / (peaks["hbm_gbs"] * 1e9),
                  ALG_FLOPS_PER_TOKEN * tokens_per_step / (peaks["bf16_tflops"] * 1e12))
     ms_step = total_ms / args.steps
