@@ -37,7 +37,8 @@ typedef enum cb_status {
     CB_ERR_WORKSPACE = 4,    /* workspace smaller than cb_workspace_bytes() or not 256-byte aligned         */
     CB_ERR_CUDA = 5,         /* a CUDA runtime/driver call failed (includes "no device")                    */
     CB_ERR_NOT_PD = 6,       /* cb_check_info: at least one ridge system had a non-positive pivot           */
-    CB_ERR_TIMEOUT = 7       /* cb_device_status: a bounded device-side wait ran out                        */
+    CB_ERR_TIMEOUT = 7,      /* cb_device_status: a bounded device-side wait ran out                        */
+    CB_ERR_STATIC_LIMIT = 8  /* cb_stats_build_static: the problem needs more scratch than the built-in buffer  */
 } cb_status;
 
 /* flags (cb_problem.flags and the flags argument of cb_ridge_solve) */
@@ -192,6 +193,34 @@ cb_status cb_apply(const cb_problem *prob, const float *Wb, const cb_kv_view *sr
  * wait inside a kernel ran out (the statistics are then invalid; reset before reuse).
  */
 cb_status cb_device_status(cb_ctx *ctx, void *stream);
+
+/*
+ * Statistics of ONE batch of rows without any device allocation by anybody (the paper has no counterpart: this
+ * entry point exists for deployment, not for the method).  It is for callers that cannot obtain scratch memory:
+ * a serving process that gave all device memory to its own pool at start-up, an engine plug-in whose enqueue
+ * hook must not call cudaMalloc (it synchronises the whole device), or a process running under a hard memory
+ * cap.  Such callers cannot provide the workspace cb_create wants, so here the partial statistics live in a
+ * fixed buffer of CB_STATIC_SCRATCH_MAX_BYTES that is part of the library image (every GPU that loads the
+ * library holds it until the process exits).
+ *
+ * Computes the same G [n_maps][p][p] and C [n_maps][p][d] (device, fp32, caller-owned) that
+ * cb_create + cb_stats_accumulate + cb_stats_reduce give for this one call's rows; arguments as for
+ * cb_stats_accumulate, prob->n_splits == 0 means one split.  Work is enqueued on `stream`; the call itself
+ * calls no cudaMalloc, cudaFree or other allocating routine.
+ *   - Limit: n_splits * n_maps * (2 d^2 + 2 d + 4) * 4 bytes plus ~1 KB must fit in the buffer (e.g. 120 maps
+ *     of d = 128 with one split); larger problems return CB_ERR_STATIC_LIMIT and nothing is enqueued.
+ *   - The first call on each device looks up the buffer's device address (with that device current); make
+ *     that first call outside any stream capture.
+ *   - All calls on a device share the one buffer, which keeps the previous call's contents; each call clears
+ *     what it needs on its stream first.  Two calls whose work overlaps on the GPU (different streams, no
+ *     ordering between them) race on the buffer: order them.
+ *   - There is no context, so a device-side time-out cannot be reported through cb_device_status.
+ */
+#define CB_STATIC_SCRATCH_MAX_BYTES (16u << 20)
+cb_status cb_stats_build_static(const cb_problem *prob, const cb_kv_view *src, const cb_kv_view *tgt,
+                                const float *w_k, const float *w_v,
+                                int64_t w_stride_layer, int64_t w_stride_head,
+                                float *G, float *C, void *stream);
 
 /* Number of kernels this library has launched in this process (all contexts); for accounting. */
 int64_t cb_launch_count(void);

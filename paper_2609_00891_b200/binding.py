@@ -18,14 +18,14 @@ LIB_PATH = os.path.join(_HERE, "libcb.so")
 
 CB_OK = 0
 CB_ERR_INVALID_ARG, CB_ERR_UNSUPPORTED, CB_ERR_STATE, CB_ERR_WORKSPACE = 1, 2, 3, 4
-CB_ERR_CUDA, CB_ERR_NOT_PD, CB_ERR_TIMEOUT = 5, 6, 7
+CB_ERR_CUDA, CB_ERR_NOT_PD, CB_ERR_TIMEOUT, CB_ERR_STATIC_LIMIT = 5, 6, 7, 8
 CB_FLAG_COMPENSATED, CB_FLAG_RAW_LAMBDA, CB_FLAG_SIMT = 1, 2, 4
 CB_DTYPE_BF16, CB_DTYPE_F32 = 0, 1
 
 EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_workspace_bytes", "cb_create",
            "cb_destroy", "cb_stats_reset", "cb_stats_accumulate", "cb_staging_bytes", "cb_stats_accumulate_host",
            "cb_stats_reduce", "cb_ridge_solve",
-           "cb_check_info", "cb_apply", "cb_device_status", "cb_launch_count")
+           "cb_check_info", "cb_apply", "cb_device_status", "cb_stats_build_static", "cb_launch_count")
 
 
 class CbError(RuntimeError):
@@ -252,6 +252,23 @@ def cb_apply(prob: Problem, Wb: torch.Tensor, src_k: torch.Tensor, src_v: torch.
                           ctypes.c_void_p(tgt_k.data_ptr()), ctypes.c_void_p(tgt_v.data_ptr()),
                           ctypes.c_int64(tgt_k.stride(0)), ctypes.c_int64(tgt_k.stride(1)),
                           ctypes.c_int64(tgt_k.stride(2)), dt, _stream_ptr(stream)), "cb_apply")
+
+
+def cb_stats_build_static(prob: Problem, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor, w_v: torch.Tensor,
+                          G: torch.Tensor, C: torch.Tensor, stream=None) -> None:
+    """Statistics of one batch of rows into caller-owned G, C with the library's built-in scratch buffer: for
+    callers that cannot allocate device memory for a workspace (see include/cb.h).  Same argument layout as
+    cb_stats_accumulate; G [n_maps][p][p], C [n_maps][p][d] fp32 device tensors."""
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    p, d = prob.ds + 1, prob.ds
+    assert w_k.dtype == torch.float32 and w_v.dtype == torch.float32 and w_k.stride() == w_v.stride()
+    assert G.dtype == torch.float32 and C.dtype == torch.float32 and G.is_contiguous() and C.is_contiguous()
+    assert G.numel() == prob.n_maps * p * p and C.numel() == prob.n_maps * p * d
+    _check(lib().cb_stats_build_static(ctypes.byref(prob.c), ctypes.byref(sv), ctypes.byref(tv),
+                                       ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                       ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
+                                       ctypes.c_void_p(G.data_ptr()), ctypes.c_void_p(C.data_ptr()),
+                                       _stream_ptr(stream)), "cb_stats_build_static")
 
 
 def cb_device_status(ctx: Context, stream=None) -> None:

@@ -91,6 +91,7 @@ const char *cb_status_string(cb_status s)
         case CB_ERR_CUDA: return "CUDA call failed";
         case CB_ERR_NOT_PD: return "ridge system not positive definite";
         case CB_ERR_TIMEOUT: return "device-side wait timed out";
+        case CB_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch buffer of cb_stats_build_static";
     }
     return "unknown status";
 }
