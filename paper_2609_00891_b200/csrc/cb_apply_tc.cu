@@ -1,12 +1,384 @@
-// Affine apply on the tensor cores (placeholder translation unit until the tcgen05 kernel lands).
+// Online affine apply on the tensor cores (sm_100a):  out[t][:] = x_t W + b  for every map and token.
+//
+// Per thread block (persistent; units = (map, token range)):
+//   conversion warps  split the map's fp32 W into bf16 hi + lo and write both into shared memory in the layout the
+//                     tensor core reads (rows = input channel, 64 output channels per 128-byte row, swizzled);
+//                     the bias row goes to shared memory as fp32.
+//   producer thread   TMA: tiles of 128 tokens of the matched source head, [channel block][token][64 channels].
+//   MMA thread        tcgen05.mma  D[128 tokens][d] += X[128][16] * W[16][d], A K-major, B MN-major, twice per
+//                     K step (hi and lo part of W), fp32 accumulators in tensor memory (two, ping-pong).
+//   epilogue warps    tensor memory -> registers, + bias, -> bf16 into a shared-memory tile -> one TMA store
+//                     (coalesced 256-byte rows, rows past the end clipped); fp32 output is stored directly.
+// Every wait is bounded; a wait that runs out makes the block tear down (nothing else is reported: this call has
+// no context to carry a status word).
+#include <cudaTypedefs.h>
+
 #include "cb_internal.cuh"
+#include "cb_ptx.cuh"
 
 namespace cb {
 
+using namespace ptx;
+
+bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long long T, int L,
+                        long long sh, long long st, long long sl, int box_tokens);
+
+template <int D>
+struct ApCfg {
+    static constexpr int TT = 128;                      // tokens per tile = MMA M
+    static constexpr int NB = D / 64;                   // 64-channel blocks
+    static constexpr int XBLK = TT * 128;               // bytes of one X block
+    static constexpr int X_BYTES = NB * XBLK;           // one X stage
+    static constexpr int WBLK = D * 128;                // bytes of one W block: D rows (input channels) of 128 bytes
+    static constexpr int W_BYTES = NB * WBLK;           // hi (or lo) part of W
+    static constexpr int O_BYTES = NB * XBLK;           // bf16 output tile
+    static constexpr int NS = 3;
+    static constexpr int NACC = 2;
+    static constexpr int TMEM_COLS = (NACC * D < 32) ? 32 : NACC * D;
+    static constexpr int EPI_WARPS = 4, CONV_WARPS = 4;
+    static constexpr int THREADS = (2 + EPI_WARPS + CONV_WARPS) * 32;
+    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * X_BYTES + 2 * (size_t)W_BYTES + O_BYTES + D * 4 + 256;
+};
+
+struct ApParams {
+    CUtensorMap src_k, src_v, out_k, out_v;
+    ApplyArgs a;
+    int n_splits;
+};
+
+struct ApIter {   // units u = blockIdx.x, += gridDim.x; unit -> (map, split) -> tiles [tile, tile1)
+    int u, tile, tile1, m;
+    __device__ __forceinline__ void next_unit(int n_units, int n_maps, int n_tiles, int n_splits)
+    {
+        do {
+            u += gridDim.x;
+            if (u >= n_units) return;
+            m = u % n_maps;
+            const int split = u / n_maps;
+            tile = (int)(((long long)n_tiles * split) / n_splits);
+            tile1 = (int)(((long long)n_tiles * (split + 1)) / n_splits);
+        } while (tile >= tile1);
+    }
+    __device__ __forceinline__ void start(int n_units, int n_maps, int n_tiles, int n_splits)
+    {
+        u = (int)blockIdx.x - (int)gridDim.x;
+        tile = tile1 = 0;
+        next_unit(n_units, n_maps, n_tiles, n_splits);
+    }
+};
+
+template <int N>
+struct ApRing {
+    uint32_t idx = 0, phase = 0;
+    __device__ __forceinline__ void next() { if (++idx == N) { idx = 0; phase ^= 1; } }
+};
+
+__device__ __forceinline__ unsigned ap_pack_bf16x2(float lo, float hi)
+{
+    unsigned r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+template <int D>
+__global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_constant__ ApParams P)
+{
+    using C = ApCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *xs = smem;                                   // [NS][X_BYTES]
+    uint8_t *whi = xs + (size_t)C::NS * C::X_BYTES;       // [NB][D rows][128 B]
+    uint8_t *wlo = whi + C::W_BYTES;
+    uint8_t *os = wlo + C::W_BYTES;                       // [NB][TT rows][128 B] bf16 output tile
+    float *bias = reinterpret_cast<float *>(os + C::O_BYTES);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(bias + D);
+    uint64_t *xfull = bars;                  // [NS]
+    uint64_t *xempty = xfull + C::NS;        // [NS]   MMA done with the stage
+    uint64_t *accfull = xempty + C::NS;      // [NACC] accumulator complete
+    uint64_t *accempty = accfull + C::NACC;  // [NACC] accumulator read out (EPI_WARPS arrivals)
+    uint64_t *wready = accempty + C::NACC;   // [1]    W of the current unit converted (CONV_WARPS arrivals)
+    uint64_t *wfree = wready + 1;            // [1]    last MMA of the unit done: W may be overwritten
+    uint64_t *bfree = wfree + 1;             // [1]    bias of the unit no longer needed (EPI_WARPS arrivals)
+    uint64_t *owritten = bfree + 1;          // [1]    output tile written by all epilogue warps
+    uint64_t *ofree = owritten + 1;          // [1]    output tile read by the store
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ofree + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const ApplyArgs &a = P.a;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_maps = 2 * a.Lt * a.Ht;
+    const int n_units = n_maps * P.n_splits;
+    const int n_tiles = (a.n_tokens + C::TT - 1) / C::TT;
+    const bool out_bf16 = a.out_dtype == CB_DTYPE_BF16;
+
+    if (tid == 0) {
+        for (int i = 0; i < C::NS; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 1); }
+        for (int i = 0; i < C::NACC; ++i) { mbar_init(&accfull[i], 1); mbar_init(&accempty[i], C::EPI_WARPS); }
+        mbar_init(wready, C::CONV_WARPS);
+        mbar_init(wfree, 1);
+        mbar_init(bfree, C::EPI_WARPS);
+        mbar_init(owritten, C::EPI_WARPS);
+        mbar_init(ofree, 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
+        tma_prefetch_desc(&P.out_k); tma_prefetch_desc(&P.out_v);
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ================================ producer (one thread) ================================
+        if (lane == 0) {
+            ApIter cur;
+            cur.start(n_units, n_maps, n_tiles, P.n_splits);
+            ApRing<C::NS> st;
+            while (cur.u < n_units) {
+                const int m = cur.m;
+                const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
+                const CUtensorMap *map = comp ? &P.src_v : &P.src_k;
+                const int j = a.src_layer[l], g = a.src_head[h];
+                for (int tile = cur.tile; tile < cur.tile1; ++tile) {
+                    if (!mbar_wait(&xempty[st.idx], st.phase ^ 1, abort_flag)) goto teardown;
+                    mbar_arrive_expect_tx(&xfull[st.idx], C::X_BYTES);
+                    tma_load_5d(xs + st.idx * C::X_BYTES, map, &xfull[st.idx], 0, tile * C::TT, 0, g, j);
+                    st.next();
+                }
+                cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ MMA issuer (one thread) ================================
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(128, D, false, true);   // A K-major, B MN-major
+            // A (K-major, 128-byte swizzle): 8-row groups 1024 bytes apart; a K step of 16 channels is 32 bytes along
+            // the row, a block of 64 channels is XBLK further.  B (MN-major): K step = 16 rows = 2048 bytes,
+            // 64-output-channel blocks WBLK apart.
+            const uint64_t proto_a = umma_smem_desc_sw128(0, 16, 1024);
+            const uint64_t proto_b = umma_smem_desc_sw128(0, C::WBLK, 1024);
+            const uint32_t a_hi32 = (uint32_t)(proto_a >> 32), b_hi32 = (uint32_t)(proto_b >> 32);
+            const uint32_t a_lo0 = (uint32_t)proto_a | ((smem_u32(xs) & 0x3FFFFu) >> 4);
+            const uint32_t bh_lo0 = (uint32_t)proto_b | ((smem_u32(whi) & 0x3FFFFu) >> 4);
+            const uint32_t bl_lo0 = (uint32_t)proto_b | ((smem_u32(wlo) & 0x3FFFFu) >> 4);
+            ApIter cur;
+            cur.start(n_units, n_maps, n_tiles, P.n_splits);
+            ApRing<C::NS> st;
+            ApRing<C::NACC> ac;
+            uint32_t uc = 0;
+            while (cur.u < n_units) {
+                if (!mbar_wait(wready, uc & 1, abort_flag)) goto teardown;
+                for (int tile = cur.tile; tile < cur.tile1; ++tile) {
+                    if (!mbar_wait(&xfull[st.idx], st.phase, abort_flag)) goto teardown;
+                    if (!mbar_wait(&accempty[ac.idx], ac.phase ^ 1, abort_flag)) goto teardown;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + ac.idx * D;
+                    const uint32_t al = a_lo0 + st.idx * (C::X_BYTES >> 4);
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint32_t ak = al + (k >> 2) * (C::XBLK >> 4) + (k & 3) * 2;          // +32 bytes per K step
+                        const uint64_t ad = ((uint64_t)a_hi32 << 32) | ak;
+                        umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bh_lo0 + k * 128), idesc, k == 0 ? 0u : 1u);
+                        umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bl_lo0 + k * 128), idesc, 1u);
+                    }
+                    umma_commit(&xempty[st.idx]);
+                    umma_commit(&accfull[ac.idx]);
+                    st.next();
+                    ac.next();
+                }
+                umma_commit(wfree);
+                ++uc;
+                cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
+            }
+        }
+    } else if (warp < 2 + C::EPI_WARPS) {
+        // ================================ epilogue warps ================================
+        const int q = warp & 3;                 // tensor-memory lane quarter of this warp
+        const int row = q * 32 + lane;          // token row inside the tile
+        ApIter cur;
+        cur.start(n_units, n_maps, n_tiles, P.n_splits);
+        ApRing<C::NACC> ac;
+        uint32_t uc = 0, oc = 0;
+        const bool storer = (warp == 2 && lane == 0);
+        while (cur.u < n_units) {
+            const int m = cur.m;
+            const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
+            const CUtensorMap *omap = comp ? &P.out_v : &P.out_k;
+            if (!mbar_wait_warp(wready, uc & 1, abort_flag, lane)) goto teardown;      // bias is in shared memory
+            for (int tile = cur.tile; tile < cur.tile1; ++tile) {
+                if (!mbar_wait_warp(&accfull[ac.idx], ac.phase, abort_flag, lane)) goto teardown;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ac.idx * D;
+                const int tok = tile * C::TT + row;
+                if (out_bf16) {
+                    if (!mbar_wait_warp(ofree, (oc & 1) ^ 1, abort_flag, lane)) goto teardown;
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_32x32(taddr + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {           // 4 chunks of 8 channels
+                            const int n0 = c * 32 + v * 8;
+                            uint4 pk;
+                            pk.x = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 0]) + bias[n0 + 0], __uint_as_float(r[v * 8 + 1]) + bias[n0 + 1]);
+                            pk.y = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 2]) + bias[n0 + 2], __uint_as_float(r[v * 8 + 3]) + bias[n0 + 3]);
+                            pk.z = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 4]) + bias[n0 + 4], __uint_as_float(r[v * 8 + 5]) + bias[n0 + 5]);
+                            pk.w = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 6]) + bias[n0 + 6], __uint_as_float(r[v * 8 + 7]) + bias[n0 + 7]);
+                            const int blk = n0 >> 6, chunk = (n0 & 63) >> 3;
+                            *reinterpret_cast<uint4 *>(os + blk * C::XBLK + row * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
+                        }
+                    }
+                    tc_fence_before();
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) { mbar_arrive(&accempty[ac.idx]); mbar_arrive(owritten); }
+                    if (storer) {
+                        if (!mbar_wait(owritten, oc & 1, abort_flag)) goto teardown_store;
+                        tma_store_5d(omap, os, 0, tile * C::TT, 0, h, l);
+                        tma_store_commit();
+                        tma_store_wait_read();
+                        mbar_arrive(ofree);
+                    }
+                teardown_store:
+                    ++oc;
+                } else {
+                    float *orow = reinterpret_cast<float *>(comp ? a.out_v : a.out_k) +
+                                  (long long)l * a.o_sl + (long long)tok * a.o_st + (long long)h * a.o_sh;
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_32x32(taddr + c * 32, r);
+                        tmem_wait_ld();
+                        if (tok < a.n_tokens) {
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) {
+                                const int n0 = c * 32 + v * 4;
+                                *reinterpret_cast<float4 *>(orow + n0) =
+                                    make_float4(__uint_as_float(r[v * 4 + 0]) + bias[n0 + 0], __uint_as_float(r[v * 4 + 1]) + bias[n0 + 1],
+                                                __uint_as_float(r[v * 4 + 2]) + bias[n0 + 2], __uint_as_float(r[v * 4 + 3]) + bias[n0 + 3]);
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&accempty[ac.idx]);
+                }
+                ac.next();
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bfree);
+            ++uc;
+            cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
+        }
+        if (storer) tma_store_wait_all();
+    } else {
+        // ================================ W conversion warps ================================
+        const int ct = tid - (2 + C::EPI_WARPS) * 32;                 // 0 .. CONV_WARPS*32-1
+        constexpr int CT = C::CONV_WARPS * 32;
+        ApIter cur;
+        cur.start(n_units, n_maps, n_tiles, P.n_splits);
+        uint32_t uc = 0;
+        while (cur.u < n_units) {
+            const float *Wm = a.Wb + (size_t)cur.m * (D + 1) * D;
+            // the previous unit's last MMA has read W, and its epilogues have read the bias
+            if (!mbar_wait_warp(wfree, (uc & 1) ^ 1, abort_flag, lane)) goto teardown;
+            if (!mbar_wait_warp(bfree, (uc & 1) ^ 1, abort_flag, lane)) goto teardown;
+            for (int i = ct; i < D * (D / 8); i += CT) {              // (input channel k, chunk of 8 output channels)
+                const int k = i / (D / 8), n0 = (i % (D / 8)) * 8;
+                const float4 f0 = __ldg(reinterpret_cast<const float4 *>(Wm + (size_t)k * D + n0));
+                const float4 f1 = __ldg(reinterpret_cast<const float4 *>(Wm + (size_t)k * D + n0 + 4));
+                const float f[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+                unsigned hi[4], lo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    hi[e] = ap_pack_bf16x2(f[2 * e], f[2 * e + 1]);
+                    const float h0 = __uint_as_float(hi[e] << 16), h1 = __uint_as_float(hi[e] & 0xffff0000u);
+                    lo[e] = ap_pack_bf16x2(f[2 * e] - h0, f[2 * e + 1] - h1);
+                }
+                const int off = (n0 >> 6) * C::WBLK + k * 128 + ((((n0 & 63) >> 3) ^ (k & 7)) << 4);
+                *reinterpret_cast<uint4 *>(whi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4 *>(wlo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            }
+            for (int n = ct; n < D; n += CT) bias[n] = __ldg(Wm + (size_t)D * D + n);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(wready);
+            ++uc;
+            cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
+        }
+    }
+
+teardown:
+    __syncwarp();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+static int ap_sm_count()
+{
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <int D>
+static cudaError_t launch_ap(const ApParams &P, cudaStream_t st)
+{
+    using C = ApCfg<D>;
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(k_apply_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    const int n_units = 2 * P.a.Lt * P.a.Ht * P.n_splits;
+    const int grid = n_units < ap_sm_count() ? n_units : ap_sm_count();
+    k_apply_tc<D><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cudaStream_t st)
 {
-    (void)src;
-    return launch_apply_simt(a, d, st);
+    ApParams P;
+    P.a = a;
+    const int TT = 128;
+    const int n_maps = 2 * a.Lt * a.Ht;
+    const int n_tiles = (a.n_tokens + TT - 1) / TT;
+    int splits = (n_maps >= ap_sm_count()) ? 1 : (ap_sm_count() + n_maps - 1) / n_maps;
+    if (splits > n_tiles) splits = n_tiles;
+    if (splits < 1) splits = 1;
+    P.n_splits = splits;
+    if (!make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
+                            src->stride_token, src->stride_layer, TT) ||
+        !make_kv_tensor_map(&P.src_v, src->v, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
+                            src->stride_token, src->stride_layer, TT))
+        return cudaErrorInvalidValue;
+    if (a.out_dtype == CB_DTYPE_BF16) {
+        if (!make_kv_tensor_map(&P.out_k, a.out_k, d, a.Ht, a.n_tokens, a.Lt, a.o_sh, a.o_st, a.o_sl, TT) ||
+            !make_kv_tensor_map(&P.out_v, a.out_v, d, a.Ht, a.n_tokens, a.Lt, a.o_sh, a.o_st, a.o_sl, TT))
+            return cudaErrorInvalidValue;
+    } else {
+        P.out_k = P.src_k;   // unused for fp32 output
+        P.out_v = P.src_v;
+    }
+    cudaError_t e = (d == 128) ? launch_ap<128>(P, st) : launch_ap<64>(P, st);
+    if (e == cudaSuccess) count_launch();
+    return e;
 }
 
 }  // namespace cb
