@@ -189,6 +189,34 @@ cb_status cb_apply(const cb_problem *prob, const float *Wb, const cb_kv_view *sr
                    int64_t t_stride_head, int32_t out_dtype, void *stream);
 
 /*
+ * Full-head contrast (Section 3.1, Eq. "fullheadfeature"; the inherited baseline of Section 2.1): every target head
+ * of layer l is regressed from ALL H_s source KV heads of k selected source layers, feature order layer-major, then
+ * head, then channel, bias last: P_f = k*H_s*d + 1.  Statistics per (comp, l): one G (P_f x P_f) shared by the
+ * layer's heads and one C (P_f x d) per target head; the weights are per (comp, l, token).
+ *
+ * cb_fullhead_layer_sets: default selection, k consecutive source layers starting one below the nearest-depth layer
+ * j(l), shifted into [0, Ls-1] (host array [Lt][k]).
+ * cb_fullhead_stats_accumulate ADDS the statistics of this call's n_tokens rows to
+ *     G [2][Lt][P_f][P_f]   and   C [2][Lt][Ht][P_f][d]        (device fp32, caller-owned, zeroed by the caller
+ * before the first call).  G is filled on both triangles; its 128 x 128 diagonal blocks are not symmetrised.
+ * w_k / w_v: device fp32 [Lt][n_tokens] at w + l*w_stride_layer + t.  layer_sets: HOST [Lt][k], ascending layers in
+ * [0, Ls-1]; k*Hs must be even and <= 64.  workspace: device, 256-byte aligned, cb_fullhead_workspace_bytes() (small
+ * index tables, copied inside the call).  Same stream/ownership/error rules as cb_stats_accumulate; no context.
+ */
+typedef struct cb_fullhead_problem {
+    int32_t Ls, Hs, ds;
+    int32_t Lt, Ht, dt;
+    int32_t k;
+    const int32_t *layer_sets;
+    uint32_t flags;
+} cb_fullhead_problem;
+cb_status cb_fullhead_layer_sets(int32_t Ls, int32_t Lt, int32_t k, int32_t *layer_sets);
+cb_status cb_fullhead_workspace_bytes(const cb_fullhead_problem *prob, size_t *bytes);
+cb_status cb_fullhead_stats_accumulate(const cb_fullhead_problem *prob, const cb_kv_view *src, const cb_kv_view *tgt,
+                                       const float *w_k, const float *w_v, int64_t w_stride_layer,
+                                       float *G, float *C, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Synchronises the stream and reads the context's device status word: CB_OK, or CB_ERR_TIMEOUT if a bounded
  * wait inside a kernel ran out (the statistics are then invalid; reset before reuse).
  */

@@ -211,6 +211,30 @@ def apply_maps(src_k: np.ndarray, src_v: np.ndarray, Theta: np.ndarray, Lt: int,
     return ((ok, ov) if want_f64 else None), ((bk, bv) if want_bf16 else None)
 
 
+# ----------------------------------------------------------------------------- full-head contrast
+def fullhead_layer_sets(Ls: int, Lt: int, k: int = 4) -> np.ndarray:
+    """int32 [Lt][k]: k consecutive source layers around the nearest-depth layer, clipped into range."""
+    sets = np.empty((Lt, k), np.int32)
+    _load().orc_fullhead_layer_sets(_i32(Ls), _i32(Lt), _i32(k), _p(sets))
+    return sets
+
+
+def fullhead_stats(src: np.ndarray, tgt: np.ndarray, w: np.ndarray, l: int, layer_set: Sequence[int]):
+    """Full-head statistics of one (component, target layer l): src/tgt are that component's bf16-bit traces
+    [L][T][H][d], w fp32 [T].  Returns fp64 G [pf][pf] (pf = k*Hs*d + 1) and C [Ht][pf][d]."""
+    Ls, T, Hs, d = src.shape
+    Lt, T2, Ht, d2 = tgt.shape
+    assert T2 == T and d2 == d and w.dtype == np.float32 and w.shape == (T,) and w.strides[0] == 4
+    ls = np.ascontiguousarray(layer_set, dtype=np.int32)
+    pf = len(ls) * Hs * d + 1
+    G = np.empty((pf, pf), np.float64)
+    C = np.empty((Ht, pf, d), np.float64)
+    s, t = _trace_strides(src), _trace_strides(tgt)
+    _load().orc_fullhead_stats(_p(src), _i64(s[0]), _i64(s[1]), _i64(s[2]), _p(tgt), _i64(t[0]), _i64(t[1]), _i64(t[2]),
+                               _p(w), _i64(T), _i32(d), _i32(Hs), _i32(Ht), _i32(l), _p(ls), _i32(len(ls)), _p(G), _p(C))
+    return G, C
+
+
 # ----------------------------------------------------------------------------- artifact size
 def coefficient_counts(Lt: int, Ht: int, Hs: int, k: int, ds: int, dt: int):
     """Non-bias coefficient counts over K and V (Section 3.2): (C_full, C_local, number of bias entries).

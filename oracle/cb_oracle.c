@@ -23,6 +23,9 @@
  * lambda_eff = lambda * s_w / n convention for weights that are not mean-one.
  */
 #include <math.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
@@ -362,5 +365,73 @@ void orc_apply(const uint16_t *src_k, const uint16_t *src_v, int64_t s_sl, int64
                 if (ob) ob[base + c] = orc_to_bf16(v);
             }
         }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Full-head regressor (Section 3.1, Eq. "fullheadfeature"): the feature of a  */
+/* target layer l concatenates every source KV head of the k selected source  */
+/* layers S_l, layer-major then head then channel, bias last:                 */
+/*   x_full = concat_{j in S_l, g in [H_s]} Z_{j,t,g},  p_f = k H_s d + 1.     */
+/* One G (p_f x p_f) per (comp, l), shared by the layer's heads (weights are   */
+/* per (comp, l, token) here), and one C (p_f x d) per target head.           */
+/* Same definition of the statistics as above, written out for this feature.  */
+/* ------------------------------------------------------------------------- */
+void orc_fullhead_stats(const uint16_t *src /* one component: [Ls][T][Hs][d] */,
+                        int64_t s_sl, int64_t s_st, int64_t s_sh,
+                        const uint16_t *tgt /* one component */, int64_t t_sl, int64_t t_st, int64_t t_sh,
+                        const float *w /* [T] weights of this (comp, l) */,
+                        int64_t n_tokens, int32_t d, int32_t Hs, int32_t Ht, int32_t l,
+                        const int32_t *layer_set /* [k] */, int32_t k,
+                        double *G /* [pf][pf] */, double *C /* [Ht][pf][d] */)
+{
+    const int32_t nf = k * Hs * d, pf = nf + 1;
+    memset(G, 0, sizeof(double) * (size_t)pf * pf);
+    memset(C, 0, sizeof(double) * (size_t)Ht * pf * d);
+    int nthreads = 1;
+#ifdef _OPENMP
+    nthreads = omp_get_max_threads();
+#endif
+    /* rows of G are independent given the token's feature vector: parallel over row blocks, tokens in order */
+    double *xt_all = (double *)malloc(sizeof(double) * (size_t)pf);
+    double *yt_all = (double *)malloc(sizeof(double) * (size_t)Ht * d);
+    (void)nthreads;
+    for (int64_t t = 0; t < n_tokens; ++t) {
+        for (int32_t q = 0; q < k; ++q)
+            for (int32_t g = 0; g < Hs; ++g)
+                for (int32_t c = 0; c < d; ++c)
+                    xt_all[(q * Hs + g) * d + c] =
+                        orc_bf16(src[(int64_t)layer_set[q] * s_sl + t * s_st + (int64_t)g * s_sh + c]);
+        xt_all[nf] = 1.0;
+        for (int32_t h = 0; h < Ht; ++h)
+            for (int32_t c = 0; c < d; ++c)
+                yt_all[h * d + c] = orc_bf16(tgt[(int64_t)l * t_sl + t * t_st + (int64_t)h * t_sh + c]);
+        const double wt = (double)w[t];
+#pragma omp parallel for schedule(static)
+        for (int32_t i = 0; i < pf; ++i) {
+            const double wx = wt * xt_all[i];
+            double *gr = G + (size_t)i * pf;
+            for (int32_t j = 0; j < pf; ++j) gr[j] += wx * xt_all[j];
+            for (int32_t h = 0; h < Ht; ++h) {
+                double *cr = C + ((size_t)h * pf + i) * d;
+                for (int32_t c = 0; c < d; ++c) cr[c] += wx * yt_all[h * d + c];
+            }
+        }
+    }
+    free(xt_all);
+    free(yt_all);
+}
+
+/* Selected source layers of the full-head contrast: c = j(l) (nearest depth); S_l = {c-1, c, c+1, c+2}       */
+/* (k consecutive layers starting one below c), shifted into [0, L_s - 1], ascending.                        */
+void orc_fullhead_layer_sets(int32_t Ls, int32_t Lt, int32_t k, int32_t *sets /* [Lt][k] */)
+{
+    for (int32_t l = 0; l < Lt; ++l) {
+        int32_t c = 0;
+        if (Lt > 1) c = (int32_t)((2 * (int64_t)l * (Ls - 1) + (Lt - 1)) / (2 * (int64_t)(Lt - 1)));
+        int32_t lo = c - 1;
+        if (lo + k > Ls) lo = Ls - k;
+        if (lo < 0) lo = 0;
+        for (int32_t q = 0; q < k; ++q) sets[l * k + q] = lo + q;
     }
 }

@@ -25,7 +25,8 @@ CB_DTYPE_BF16, CB_DTYPE_F32 = 0, 1
 EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_workspace_bytes", "cb_create",
            "cb_destroy", "cb_stats_reset", "cb_stats_accumulate", "cb_staging_bytes", "cb_stats_accumulate_host",
            "cb_stats_reduce", "cb_ridge_solve",
-           "cb_check_info", "cb_apply", "cb_device_status", "cb_stats_build_static", "cb_launch_count")
+           "cb_check_info", "cb_apply", "cb_device_status", "cb_stats_build_static", "cb_fullhead_layer_sets",
+           "cb_fullhead_workspace_bytes", "cb_fullhead_stats_accumulate", "cb_launch_count")
 
 
 class CbError(RuntimeError):
@@ -269,6 +270,58 @@ def cb_stats_build_static(prob: Problem, src_k, src_v, tgt_k, tgt_v, w_k: torch.
                                        ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
                                        ctypes.c_void_p(G.data_ptr()), ctypes.c_void_p(C.data_ptr()),
                                        _stream_ptr(stream)), "cb_stats_build_static")
+
+
+class _FullHeadProblem(ctypes.Structure):
+    _fields_ = [("Ls", ctypes.c_int32), ("Hs", ctypes.c_int32), ("ds", ctypes.c_int32),
+                ("Lt", ctypes.c_int32), ("Ht", ctypes.c_int32), ("dt", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("layer_sets", ctypes.POINTER(ctypes.c_int32)), ("flags", ctypes.c_uint32)]
+
+
+class FullHeadProblem:
+    """Shapes plus the selected source layers [Lt][k] of the full-head contrast, mirroring cb_fullhead_problem."""
+
+    def __init__(self, Ls, Hs, ds, Lt, Ht, dt, layer_sets, flags: int = 0):
+        self.layer_sets = np.ascontiguousarray(layer_sets, dtype=np.int32)
+        assert self.layer_sets.ndim == 2 and self.layer_sets.shape[0] == Lt
+        self.k = int(self.layer_sets.shape[1])
+        self.c = _FullHeadProblem(Ls, Hs, ds, Lt, Ht, dt, self.k,
+                                  self.layer_sets.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), flags)
+        self.Ls, self.Hs, self.ds, self.Lt, self.Ht, self.dt = Ls, Hs, ds, Lt, Ht, dt
+
+    @property
+    def pf(self) -> int:
+        return self.k * self.Hs * self.ds + 1
+
+
+def cb_fullhead_layer_sets(Ls: int, Lt: int, k: int = 4) -> np.ndarray:
+    sets = np.empty((Lt, k), np.int32)
+    _check(lib().cb_fullhead_layer_sets(Ls, Lt, k, sets.ctypes.data_as(ctypes.c_void_p)), "cb_fullhead_layer_sets")
+    return sets
+
+
+def cb_fullhead_workspace_bytes(prob: FullHeadProblem) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().cb_fullhead_workspace_bytes(ctypes.byref(prob.c), ctypes.byref(n)), "cb_fullhead_workspace_bytes")
+    return n.value
+
+
+def cb_fullhead_stats_accumulate(prob: FullHeadProblem, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor, w_v: torch.Tensor,
+                                 G: torch.Tensor, C: torch.Tensor, workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Adds this batch's full-head statistics to G [2][Lt][pf][pf] and C [2][Lt][Ht][pf][d] (fp32, zeroed by the
+    caller before the first batch).  Weights [Lt][T] fp32."""
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    assert w_k.dtype == torch.float32 and w_v.dtype == torch.float32 and w_k.dim() == 2 and w_k.stride() == w_v.stride()
+    assert G.dtype == torch.float32 and C.dtype == torch.float32 and G.is_contiguous() and C.is_contiguous()
+    assert G.numel() == 2 * prob.Lt * prob.pf * prob.pf and C.numel() == 2 * prob.Lt * prob.Ht * prob.pf * prob.ds
+    if workspace is None:
+        workspace = torch.empty(cb_fullhead_workspace_bytes(prob), dtype=torch.uint8, device=G.device)
+    _check(lib().cb_fullhead_stats_accumulate(ctypes.byref(prob.c), ctypes.byref(sv), ctypes.byref(tv),
+                                              ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                              ctypes.c_int64(w_k.stride(0)), ctypes.c_void_p(G.data_ptr()),
+                                              ctypes.c_void_p(C.data_ptr()), ctypes.c_void_p(workspace.data_ptr()),
+                                              ctypes.c_size_t(workspace.numel()), _stream_ptr(stream)),
+           "cb_fullhead_stats_accumulate")
 
 
 def cb_device_status(ctx: Context, stream=None) -> None:

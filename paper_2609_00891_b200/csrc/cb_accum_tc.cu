@@ -34,14 +34,17 @@ namespace cb {
 
 using namespace ptx;
 
-template <int D, bool COMP>
+template <int D, bool COMP, bool FH = false>
 struct TcCfg {
     static constexpr int TT = 64;                     // tokens per tile
     static constexpr int NBX = D / 64;                // 64-channel blocks per head
     static constexpr int BLK = TT * 128;              // bytes of one block: TT rows of 128 bytes
-    static constexpr int STAGE_BYTES = 2 * NBX * BLK; // X blocks, then Y blocks
+    // A stage holds the second MMA operand [B1 | B2] (head-local: B1 = X, B2 = Y).  The rows to be weighted come
+    // from B1; the full-head variant (FH) weights a third head, staged behind B2.
+    static constexpr int STAGE_BYTES = (FH ? 3 : 2) * NBX * BLK;
+    static constexpr int AS_OFF = FH ? 2 * NBX * BLK : 0;   // where the rows to be weighted start inside a stage
     static constexpr int A_BYTES = 2 * BLK;           // M = 128 always: two blocks (second stays zero for d = 64)
-    static constexpr int NS = COMP ? 4 : CB_NS;       // X/Y stages
+    static constexpr int NS = FH ? 3 : (COMP ? 4 : CB_NS);   // stages
     static constexpr int NA = COMP ? 2 : CB_NA;                    // weighted-operand buffers (hi, and lo when compensated)
     static constexpr int A_PARTS = COMP ? 2 : 1;
     static constexpr int N = 2 * D;                   // accumulator columns
@@ -61,26 +64,71 @@ struct TcCfg {
     static_assert(TMEM_COLS == 256 || TMEM_COLS == 512, "tensor memory columns must be a power of two");
 };
 
+// Full-head contrast (FH): per (component, target layer l) the feature is every KV head of k selected source
+// layers: F = k*Hs feature heads.  Units per (comp, l): NG "G units" (i, q), 2q <= i: rows of feature head i against
+// feature heads 2q and 2q+1 (the lower triangle of G, mirrored on write), then F*Ht "C units" (i, h): feature head i
+// against target head h.  Results are added straight into G / C.
+struct FhDev {
+    float *G, *C;                 // [2][Lt][PF][PF], [2][Lt][Ht][PF][d]
+    const int *layer_sets;        // device [Lt][k]
+    const int *gi, *gq;           // device [NG]
+    int F, k, Hs, PF, NG, NC;
+};
+
 struct TcParams {
     CUtensorMap src_k, src_v, tgt_k, tgt_v;   // 5-D tiled maps: (64 channels, token, channel block, head, layer)
     AccumArgs a;
+    FhDev fh;
     int drain_tiles;                          // tiles accumulated in tensor memory between drains
 };
 
-// Walks the tiles of this block's units in order: units u = blockIdx.x, += gridDim.x; unit -> (map, split)
-// -> tiles [tile0, tile1).  Empty units are skipped.
-struct TileIter {
+// Walks the tiles of this block's units in order: units u = blockIdx.x, += gridDim.x.  Head-local: unit -> (map,
+// split) -> tiles [tile0, tile1); full-head: unit -> (comp, l, G or C unit), all tiles.  Empty units are skipped.
+// The operands of a unit are decoded once per unit.
+template <bool FH>
+struct TileIterT {
     int u, tile, tile1, m, split;
-    int comp, l, h, j, g;          // decoded once per unit: component, target layer/head, matched source layer/head
-    __device__ __forceinline__ void start(const AccumArgs &a, int n_units, int n_maps, int n_tiles)
+    int comp, l, h;                 // component, target layer, target head (C units / head-local)
+    int a_layer, a_head;            // source head whose rows are weighted
+    int b1_layer, b1_head;          // first half of the second operand (a source head)
+    int b2_layer, b2_head, b2_tgt;  // second half: target head (b2_tgt) or source head
+    int fi, fj;                     // full-head: feature head of the rows; first feature head of the columns, or -1
+    __device__ __forceinline__ void start(const TcParams &P, int n_units, int n_maps, int n_tiles)
     {
         u = (int)blockIdx.x - (int)gridDim.x;
         tile = tile1 = 0;
-        next_unit(a, n_units, n_maps, n_tiles);
+        next_unit(P, n_units, n_maps, n_tiles);
     }
     __device__ __forceinline__ bool valid(int n_units) const { return u < n_units; }
-    __device__ __forceinline__ void next_unit(const AccumArgs &a, int n_units, int n_maps, int n_tiles)
+    __device__ __forceinline__ void next_unit(const TcParams &P, int n_units, int n_maps, int n_tiles)
     {
+        const AccumArgs &a = P.a;
+        if (FH) {
+            u += gridDim.x;
+            if (u >= n_units) return;
+            const FhDev &f = P.fh;
+            const int per = f.NG + f.NC;
+            const int group = u / per, v = u % per;
+            comp = group / a.Lt;
+            l = group % a.Lt;
+            m = u; split = 0; tile = 0; tile1 = n_tiles;
+            if (v < f.NG) {
+                fi = f.gi[v];
+                fj = 2 * f.gq[v];
+                b1_layer = f.layer_sets[l * f.k + fj / f.Hs];          b1_head = fj % f.Hs;
+                b2_layer = f.layer_sets[l * f.k + (fj + 1) / f.Hs];    b2_head = (fj + 1) % f.Hs;
+                b2_tgt = 0; h = 0;
+            } else {
+                fi = (v - f.NG) / a.Ht;
+                h = (v - f.NG) % a.Ht;
+                fj = -1;
+                b1_layer = f.layer_sets[l * f.k + fi / f.Hs];          b1_head = fi % f.Hs;
+                b2_layer = l; b2_head = h; b2_tgt = 1;
+            }
+            a_layer = f.layer_sets[l * f.k + fi / f.Hs];
+            a_head = fi % f.Hs;
+            return;
+        }
         do {
             u += gridDim.x;
             if (u >= n_units) return;
@@ -92,12 +140,18 @@ struct TileIter {
         comp = m / (a.Lt * a.Ht);
         l = (m / a.Ht) % a.Lt;
         h = m % a.Ht;
-        j = a.src_layer[l];
-        g = a.src_head[h];
+        a_layer = b1_layer = a.src_layer[l];
+        a_head = b1_head = a.src_head[h];
+        b2_layer = l; b2_head = h; b2_tgt = 1;
+        fi = fj = 0;
     }
-    __device__ __forceinline__ void advance(const AccumArgs &a, int n_units, int n_maps, int n_tiles)
+    __device__ __forceinline__ void advance(const TcParams &P, int n_units, int n_maps, int n_tiles)
     {
-        if (++tile >= tile1) next_unit(a, n_units, n_maps, n_tiles);
+        if (++tile >= tile1) next_unit(P, n_units, n_maps, n_tiles);
+    }
+    __device__ __forceinline__ const float *weights(const AccumArgs &a) const
+    {
+        return (comp ? a.w_v : a.w_k) + (long long)l * a.w_sl + (FH ? 0ll : (long long)h * a.w_sh);
     }
 };
 
@@ -134,10 +188,11 @@ struct Ring {
     __device__ __forceinline__ void next() { if (++idx == N) { idx = 0; phase ^= 1; } }
 };
 
-template <int D, bool COMP>
-__global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const __grid_constant__ TcParams P)
+template <int D, bool COMP, bool FH>
+__global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(const __grid_constant__ TcParams P)
 {
-    using C = TcCfg<D, COMP>;
+    using C = TcCfg<D, COMP, FH>;
+    using TileIter = TileIterT<FH>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *xy = smem;                                       // [NS][STAGE_BYTES]
@@ -148,7 +203,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
     uint64_t *full = bars;                 // [NS] tile landed: X bytes (1 arrival), Y bytes (1), weights (32 lanes)
     uint64_t *empty = full + C::NS;        // [NS] stage free: MMA done (1) + every fold warp done
     uint64_t *afull = empty + C::NS;       // [NA] weighted operand written (every fold warp)
-    uint64_t *aempty = afull + C::NA;      // [NA] weighted operand consumed (MMA)
+    uint64_t *aempty = afull + C::NA;      // [NA] (unused)
     uint64_t *accfull = aempty + C::NA;    // [2]  accumulator complete (MMA)
     uint64_t *accempty = accfull + 2;      // [2]  accumulator drained (4 drain warps)
     uint64_t *redfull = accempty + 2;      // [1]  bias partials of all fold warps written
@@ -159,7 +214,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
     const AccumArgs &a = P.a;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_maps = 2 * a.Lt * a.Ht;
-    const int n_units = n_maps * a.n_splits;
+    const int n_units = FH ? 2 * a.Lt * (P.fh.NG + P.fh.NC) : n_maps * a.n_splits;
     const int n_tiles = (a.n_tokens + C::TT - 1) / C::TT;
 
     if (tid == 0) {
@@ -195,21 +250,22 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
         // ================================ X producer (one thread) ================================
         if (lane == 0) {
             TileIter cur;
-            cur.start(a, n_units, n_maps, n_tiles);
+            cur.start(P, n_units, n_maps, n_tiles);
             Ring<C::NS> st;
             uint32_t it = 0;
             while (cur.valid(n_units)) {
                 const CUtensorMap *map = cur.comp ? &P.src_v : &P.src_k;
-                const int g = cur.g, j = cur.j, u = cur.u;
+                const int g = cur.b1_head, j = cur.b1_layer, ag = cur.a_head, aj = cur.a_layer, u = cur.u;
                 do {   // tiles of one unit
                     if (!mbar_wait(&empty[st.idx], st.phase ^ 1, abort_flag)) goto teardown;
                     CB_TR(it, 0);
-                    mbar_arrive_expect_tx(&full[st.idx], C::STAGE_BYTES / 2);
+                    mbar_arrive_expect_tx(&full[st.idx], (FH ? 2 : 1) * C::NBX * C::BLK);
                     tma_load_5d(xy + st.idx * C::STAGE_BYTES, map, &full[st.idx], 0, cur.tile * C::TT, 0, g, j);
+                    if (FH) tma_load_5d(xy + st.idx * C::STAGE_BYTES + C::AS_OFF, map, &full[st.idx], 0, cur.tile * C::TT, 0, ag, aj);
                     CB_TR(it, 1);
                     st.next();
                     ++it;
-                    cur.advance(a, n_units, n_maps, n_tiles);
+                    cur.advance(P, n_units, n_maps, n_tiles);
                 } while (cur.u == u);
             }
         }
@@ -218,19 +274,19 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
         // Lane 0 issues the Y tile copy; all 32 lanes copy the tile's token weights with 4-byte asynchronous copies
         // (zero-filled past the last token, no alignment requirement) that arrive on the same barrier.
         TileIter cur;
-        cur.start(a, n_units, n_maps, n_tiles);
+        cur.start(P, n_units, n_maps, n_tiles);
         Ring<C::NS> st;
         uint32_t it = 0;
         while (cur.valid(n_units)) {
-            const CUtensorMap *map = cur.comp ? &P.tgt_v : &P.tgt_k;
-            const int h = cur.h, l = cur.l, u = cur.u;
-            const float *w = (cur.comp ? a.w_v : a.w_k) + (long long)l * a.w_sl + (long long)h * a.w_sh;
+            const CUtensorMap *map = cur.b2_tgt ? (cur.comp ? &P.tgt_v : &P.tgt_k) : (cur.comp ? &P.src_v : &P.src_k);
+            const int h = cur.b2_head, l = cur.b2_layer, u = cur.u;
+            const float *w = cur.weights(a);
             do {
                 if (!mbar_wait_warp(&empty[st.idx], st.phase ^ 1, abort_flag, lane)) goto teardown;
                 CB_TR(it, 38);
                 const int tok0 = cur.tile * C::TT;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&full[st.idx], C::STAGE_BYTES / 2);
+                    mbar_arrive_expect_tx(&full[st.idx], C::NBX * C::BLK);
                     tma_load_5d(xy + st.idx * C::STAGE_BYTES + C::NBX * C::BLK, map, &full[st.idx], 0, tok0, 0, h, l);
                 }
 #pragma unroll
@@ -243,7 +299,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
                 CB_TR(it, 39);
                 st.next();
                 ++it;
-                cur.advance(a, n_units, n_maps, n_tiles);
+                cur.advance(P, n_units, n_maps, n_tiles);
             } while (cur.u == u);
         }
     } else if (warp == 1) {
@@ -260,7 +316,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
             Ring<C::NA> ar;
             uint32_t it = 0, sr = 0;
             TileIter cur;
-            cur.start(a, n_units, n_maps, n_tiles);
+            cur.start(P, n_units, n_maps, n_tiles);
             while (cur.valid(n_units)) {
                 const int u = cur.u, tile1 = cur.tile1;
                 for (int sr0 = cur.tile; sr0 < tile1; sr0 += P.drain_tiles, ++sr) {
@@ -271,8 +327,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
                     const uint32_t d_tmem = tmem_base + acc * C::N;
                     uint32_t accum = 0;
                     for (int t = 0; t < n_sub; ++t) {
-                        if (!mbar_wait(&full[st.idx], st.phase, abort_flag)) goto teardown;
-                        CB_TR(it, 2);
+                        // afull implies full: every fold warp saw the tile land before it wrote the weighted operand
                         if (!mbar_wait(&afull[ar.idx], ar.phase, abort_flag)) goto teardown;
                         CB_TR(it, 3);
                         tc_fence_after();
@@ -285,8 +340,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
                             if (COMP) umma_bf16_ss(d_tmem, ((uint64_t)desc_hi << 32) | (al + (C::A_BYTES >> 4) + k * 128), bd, idesc, 1u);
                         }
                         accum = 1;
-                        umma_commit(&empty[st.idx]);
-                        umma_commit(&aempty[ar.idx]);
+                        umma_commit(&empty[st.idx]);     // frees the stage and (through it) the weighted-operand buffer
                         CB_TR(it, 4);
                         st.next();
                         ar.next();
@@ -294,7 +348,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
                     }
                     umma_commit(&accfull[acc]);
                 }
-                while (cur.valid(n_units) && cur.u == u) cur.next_unit(a, n_units, n_maps, n_tiles);
+                while (cur.valid(n_units) && cur.u == u) cur.next_unit(P, n_units, n_maps, n_tiles);
             }
         }
     } else if (warp < 2 + C::FOLD_WARPS) {
@@ -306,11 +360,11 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
         // byte offset of this thread's first 16-byte chunk inside a block; its other rows are RG rows further down
         const int off0 = blk * C::BLK + rg * 128 + ((lc ^ (rg & 7)) << 4);
         float sx[8], sy[8], sw = 0.f;
-        Ring<C::NS> st;
+        Ring<C::NS> st, old;       // `old` trails `st` by NA tiles
         Ring<C::NA> ar;
         uint32_t it = 0, uc = 0;
         TileIter cur;
-        cur.start(a, n_units, n_maps, n_tiles);
+        cur.start(P, n_units, n_maps, n_tiles);
         while (cur.valid(n_units)) {
             const int m = cur.m, split = cur.split, n_t = cur.tile1 - cur.tile;
 #pragma unroll
@@ -318,11 +372,15 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
             sw = 0.f;
             for (int t = 0; t < n_t; ++t) {
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
-                if (!mbar_wait_warp(&aempty[ar.idx], ar.phase ^ 1, abort_flag, lane)) goto teardown;
+                // the weighted-operand buffer was last used by tile it - NA; it is free once that tile's stage is free
+                if (it >= (uint32_t)C::NA) {
+                    if (!mbar_wait_warp(&empty[old.idx], old.phase, abort_flag, lane)) goto teardown;
+                    old.next();
+                }
                 CB_TR(it, 5 + 2 * (warp - 2));
                 const float *wsm = wst + st.idx * C::TT + rg;
-                const uint8_t *xs = xy + st.idx * C::STAGE_BYTES + off0;
-                const uint8_t *ys = xs + C::NBX * C::BLK;
+                const uint8_t *xs = xy + st.idx * C::STAGE_BYTES + C::AS_OFF + off0;          // rows to be weighted
+                const uint8_t *ys = xy + st.idx * C::STAGE_BYTES + C::NBX * C::BLK + off0;    // B2: summed with the weights
                 uint8_t *ah = ab + ar.idx * (C::A_PARTS * C::A_BYTES) + off0;
 #pragma unroll
                 for (int i = 0; i < C::RPT; ++i) {
@@ -389,17 +447,43 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
             __syncwarp();
             if (lane == 0) mbar_arrive(redfull);
             if (!mbar_wait_warp(redfull, uc & 1, abort_flag, lane)) goto teardown;
-            float *slot = a.slots + ((size_t)split * n_maps + m) * slot_floats(D);
-            for (int v = ft; v < 2 * D + 1; v += C::FOLD_THREADS) {
-                float sum = 0.f;
+            if (FH) {
+                // C units carry the bias entries: (i, h = 0) the column/row of feature head i, (i = 0, h) the bias row
+                // of target head h, (0, 0) the weight total.  G units carry none.
+                if (cur.fj < 0) {
+                    const FhDev &f = P.fh;
+                    const size_t PF = (size_t)f.PF;
+                    float *Gg = f.G + ((size_t)cur.comp * a.Lt + cur.l) * PF * PF;
+                    float *Cg = f.C + (((size_t)cur.comp * a.Lt + cur.l) * a.Ht + cur.h) * PF * D;
+                    for (int v = ft; v < 2 * D + 1; v += C::FOLD_THREADS) {
+                        float sum = 0.f;
 #pragma unroll
-                for (int q = 0; q < C::FOLD_WARPS; ++q) sum += red[q * C::RED_STRIDE + v];
-                slot[slot_sx(D) + v] += sum;    // s_x, s_y, s_w are adjacent in the slot
+                        for (int q = 0; q < C::FOLD_WARPS; ++q) sum += red[q * C::RED_STRIDE + v];
+                        if (v < D) {
+                            if (cur.h == 0) {
+                                Gg[((size_t)cur.fi * D + v) * PF + (PF - 1)] += sum;
+                                Gg[(PF - 1) * PF + (size_t)cur.fi * D + v] += sum;
+                            }
+                        } else if (v < 2 * D) {
+                            if (cur.fi == 0) Cg[(PF - 1) * D + (v - D)] += sum;
+                        } else if (cur.fi == 0 && cur.h == 0) {
+                            Gg[(PF - 1) * PF + (PF - 1)] += sum;
+                        }
+                    }
+                }
+            } else {
+                float *slot = a.slots + ((size_t)split * n_maps + m) * slot_floats(D);
+                for (int v = ft; v < 2 * D + 1; v += C::FOLD_THREADS) {
+                    float sum = 0.f;
+#pragma unroll
+                    for (int q = 0; q < C::FOLD_WARPS; ++q) sum += red[q * C::RED_STRIDE + v];
+                    slot[slot_sx(D) + v] += sum;    // s_x, s_y, s_w are adjacent in the slot
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(reddone);
             ++uc;
-            cur.next_unit(a, n_units, n_maps, n_tiles);
+            cur.next_unit(P, n_units, n_maps, n_tiles);
         }
     } else {
         // ================================ drain warps ================================
@@ -407,14 +491,45 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
         const int row = q * 32 + lane;      // row of D = channel of the weighted operand
         uint32_t sr = 0;
         TileIter cur;
-        cur.start(a, n_units, n_maps, n_tiles);
+        cur.start(P, n_units, n_maps, n_tiles);
         while (cur.valid(n_units)) {
-            float *slot = a.slots + ((size_t)cur.split * n_maps + cur.m) * slot_floats(D);
+            float *slot = FH ? nullptr : a.slots + ((size_t)cur.split * n_maps + cur.m) * slot_floats(D);
             for (int sr0 = cur.tile; sr0 < cur.tile1; sr0 += P.drain_tiles, ++sr) {
                 const int acc = sr & 1;
                 if (!mbar_wait_warp(&accfull[acc], (sr >> 1) & 1, abort_flag, lane, true, 4, 512)) goto teardown;
                 tc_fence_after();
-                if (row < D) {
+                if (FH) {
+                    if (row < D) {
+                        const FhDev &f = P.fh;
+                        const size_t PF = (size_t)f.PF;
+                        float *Gg = f.G + ((size_t)cur.comp * a.Lt + cur.l) * PF * PF;
+                        const size_t ri = (size_t)cur.fi * D + row;           // row of G / C this thread holds
+#pragma unroll 1
+                        for (int c = 0; c < C::N / 16; ++c) {
+                            uint32_t r[16];
+                            tmem_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + acc * C::N + c * 16, r);
+                            tmem_wait_ld();
+                            const int part = (c * 16) / D, c0 = (c * 16) % D;   // which half of [B1 | B2], first column
+                            if (cur.fj >= 0) {
+                                const int j = cur.fj + part;                    // feature head of these columns
+                                if (j <= cur.fi) {
+                                    float *dst = Gg + ri * PF + (size_t)j * D + c0;
+#pragma unroll
+                                    for (int e = 0; e < 16; ++e) dst[e] += __uint_as_float(r[e]);
+                                    if (j < cur.fi) {                           // mirror into the upper triangle
+                                        float *mir = Gg + ((size_t)j * D + c0) * PF + ri;
+#pragma unroll
+                                        for (int e = 0; e < 16; ++e) mir[(size_t)e * PF] += __uint_as_float(r[e]);
+                                    }
+                                }
+                            } else if (part == 1) {
+                                float *dst = f.C + ((((size_t)cur.comp * a.Lt + cur.l) * a.Ht + cur.h) * PF + ri) * D + c0;
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) dst[e] += __uint_as_float(r[e]);
+                            }
+                        }
+                    }
+                } else if (row < D) {
                     float *grow = slot + (size_t)row * C::N;
 #pragma unroll 1
                     for (int c = 0; c < C::N / 16; ++c) {
@@ -438,14 +553,14 @@ __global__ void __launch_bounds__(TcCfg<D, COMP>::THREADS, 1) k_accum_tc(const _
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&accempty[acc]);
             }
-            cur.next_unit(a, n_units, n_maps, n_tiles);
+            cur.next_unit(P, n_units, n_maps, n_tiles);
         }
     }
 
 teardown:
     __syncwarp();
     if (*abort_flag) {
-        if (tid == 0) atomicExch(a.status, DEV_TIMEOUT);
+        if (tid == 0 && a.status) atomicExch(a.status, DEV_TIMEOUT);
         // give copies that may still be in flight time to land before the block's shared memory is released
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
     }
@@ -504,40 +619,59 @@ static int sm_count()
     return n;
 }
 
-template <int D, bool COMP>
+template <int D, bool COMP, bool FH = false>
 static cudaError_t launch_tc(const TcParams &P, cudaStream_t st)
 {
-    using C = TcCfg<D, COMP>;
+    using C = TcCfg<D, COMP, FH>;
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D, COMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D, COMP, FH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr = true;
     }
-    const int n_units = 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
+    const int n_units = FH ? 2 * P.a.Lt * (P.fh.NG + P.fh.NC) : 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
     const int grid = n_units < sm_count() ? n_units : sm_count();
-    k_accum_tc<D, COMP><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
+    k_accum_tc<D, COMP, FH><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
+}
+
+static bool fill_maps(TcParams &P, int d, const cb_kv_view *src, const cb_kv_view *tgt, int TT)
+{
+    return make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
+                              src->stride_token, src->stride_layer, TT) &&
+           make_kv_tensor_map(&P.src_v, src->v, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
+                              src->stride_token, src->stride_layer, TT) &&
+           make_kv_tensor_map(&P.tgt_k, tgt->k, d, tgt->n_heads, tgt->n_tokens, tgt->n_layers, tgt->stride_head,
+                              tgt->stride_token, tgt->stride_layer, TT) &&
+           make_kv_tensor_map(&P.tgt_v, tgt->v, d, tgt->n_heads, tgt->n_tokens, tgt->n_layers, tgt->stride_head,
+                              tgt->stride_token, tgt->stride_layer, TT);
 }
 
 cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st)
 {
     TcParams P;
     P.a = a;
+    P.fh = FhDev{};
     const int TT = 64;
-    if (!make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
-                            src->stride_token, src->stride_layer, TT) ||
-        !make_kv_tensor_map(&P.src_v, src->v, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
-                            src->stride_token, src->stride_layer, TT) ||
-        !make_kv_tensor_map(&P.tgt_k, tgt->k, d, tgt->n_heads, tgt->n_tokens, tgt->n_layers, tgt->stride_head,
-                            tgt->stride_token, tgt->stride_layer, TT) ||
-        !make_kv_tensor_map(&P.tgt_v, tgt->v, d, tgt->n_heads, tgt->n_tokens, tgt->n_layers, tgt->stride_head,
-                            tgt->stride_token, tgt->stride_layer, TT))
-        return cudaErrorInvalidValue;
+    if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
     P.drain_tiles = 16384 / TT;   // at most 16384 tokens are summed in tensor memory before a drain
     cudaError_t e;
     if (a.compensated) e = (d == 128) ? launch_tc<128, true>(P, st) : launch_tc<64, true>(P, st);
     else e = (d == 128) ? launch_tc<128, false>(P, st) : launch_tc<64, false>(P, st);
+    if (e == cudaSuccess) count_launch();
+    return e;
+}
+
+cudaError_t launch_fullhead_tc(const AccumArgs &a, const FullHeadArgs &f, int d, const cb_kv_view *src, const cb_kv_view *tgt,
+                               cudaStream_t st)
+{
+    TcParams P;
+    P.a = a;
+    P.fh = FhDev{f.G, f.C, f.layer_sets, f.gi, f.gq, f.F, f.k, f.Hs, f.PF, f.NG, f.NC};
+    const int TT = 64;
+    if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
+    P.drain_tiles = 16384 / TT;
+    cudaError_t e = (d == 128) ? launch_tc<128, false, true>(P, st) : launch_tc<64, false, true>(P, st);
     if (e == cudaSuccess) count_launch();
     return e;
 }

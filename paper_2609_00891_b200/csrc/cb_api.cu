@@ -394,6 +394,92 @@ cb_status cb_apply(const cb_problem *prob, const float *Wb, const cb_kv_view *sr
     return CB_OK;
 }
 
+cb_status cb_fullhead_layer_sets(int32_t Ls, int32_t Lt, int32_t k, int32_t *layer_sets)
+{
+    if (Ls <= 0 || Lt <= 0 || k <= 0 || k > Ls || !layer_sets) return CB_ERR_INVALID_ARG;
+    for (int32_t l = 0; l < Lt; ++l) {
+        int32_t c = 0;
+        if (Lt > 1) c = (int32_t)(((int64_t)2 * l * (Ls - 1) + (Lt - 1)) / ((int64_t)2 * (Lt - 1)));
+        int32_t lo = c - 1;
+        if (lo + k > Ls) lo = Ls - k;
+        if (lo < 0) lo = 0;
+        for (int32_t q = 0; q < k; ++q) layer_sets[l * k + q] = lo + q;
+    }
+    return CB_OK;
+}
+
+static cb_status check_fullhead(const cb_fullhead_problem *p)
+{
+    if (!p || !p->layer_sets) return CB_ERR_INVALID_ARG;
+    if (p->Ls <= 0 || p->Hs <= 0 || p->Lt <= 0 || p->Ht <= 0 || p->k <= 0 || p->k > p->Ls) return CB_ERR_INVALID_ARG;
+    if (p->ds != p->dt || (p->ds != 64 && p->ds != 128)) return CB_ERR_UNSUPPORTED;
+    const int F = p->k * p->Hs;
+    if ((F & 1) || F > 64) return CB_ERR_UNSUPPORTED;
+    for (int i = 0; i < p->Lt * p->k; ++i)
+        if (p->layer_sets[i] < 0 || p->layer_sets[i] >= p->Ls) return CB_ERR_INVALID_ARG;
+    return CB_OK;
+}
+
+static int fullhead_ng(int F) { int n = 0; for (int i = 0; i < F; ++i) n += i / 2 + 1; return n; }
+
+cb_status cb_fullhead_workspace_bytes(const cb_fullhead_problem *prob, size_t *bytes)
+{
+    cb_status s = check_fullhead(prob);
+    if (s != CB_OK) return s;
+    if (!bytes) return CB_ERR_INVALID_ARG;
+    const int F = prob->k * prob->Hs;
+    *bytes = align_up(sizeof(int) * ((size_t)prob->Lt * prob->k + 2 * (size_t)fullhead_ng(F)), 256);
+    return CB_OK;
+}
+
+cb_status cb_fullhead_stats_accumulate(const cb_fullhead_problem *prob, const cb_kv_view *src, const cb_kv_view *tgt,
+                                       const float *w_k, const float *w_v, int64_t w_stride_layer,
+                                       float *G, float *C, void *workspace, size_t workspace_bytes, void *stream)
+{
+    cb_status s = check_fullhead(prob);
+    if (s != CB_OK) return s;
+    s = check_view(src, prob->Ls, prob->Hs, prob->ds);
+    if (s != CB_OK) return s;
+    s = check_view(tgt, prob->Lt, prob->Ht, prob->dt);
+    if (s != CB_OK) return s;
+    if (src->n_tokens != tgt->n_tokens) return CB_ERR_INVALID_ARG;
+    if (src->n_tokens == 0) return CB_OK;
+    if (!w_k || !w_v || w_stride_layer < 0 || !G || !C) return CB_ERR_INVALID_ARG;
+    const int F = prob->k * prob->Hs, NG = fullhead_ng(F);
+    size_t need = 0;
+    cb_fullhead_workspace_bytes(prob, &need);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return CB_ERR_WORKSPACE;
+
+    std::vector<int32_t> tab(prob->layer_sets, prob->layer_sets + (size_t)prob->Lt * prob->k);
+    std::vector<int32_t> gi, gq;
+    for (int i = 0; i < F; ++i)
+        for (int q = 0; 2 * q <= i; ++q) { gi.push_back(i); gq.push_back(q); }
+    tab.insert(tab.end(), gi.begin(), gi.end());
+    tab.insert(tab.end(), gq.begin(), gq.end());
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(workspace, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return CB_ERR_CUDA;
+    }
+    AccumArgs a;
+    a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src->k), static_cast<const __nv_bfloat16 *>(src->v),
+                  src->stride_layer, src->stride_token, src->stride_head};
+    a.tgt = KVPtr{static_cast<const __nv_bfloat16 *>(tgt->k), static_cast<const __nv_bfloat16 *>(tgt->v),
+                  tgt->stride_layer, tgt->stride_token, tgt->stride_head};
+    a.w_k = w_k; a.w_v = w_v; a.w_sl = w_stride_layer; a.w_sh = 0;
+    a.n_tokens = (int)src->n_tokens;
+    a.Lt = prob->Lt; a.Ht = prob->Ht; a.n_splits = 1;
+    a.src_layer = nullptr; a.src_head = nullptr; a.slots = nullptr; a.status = nullptr; a.compensated = 0;
+    FullHeadArgs f;
+    f.G = G; f.C = C;
+    f.layer_sets = static_cast<const int *>(workspace);
+    f.gi = f.layer_sets + (size_t)prob->Lt * prob->k;
+    f.gq = f.gi + NG;
+    f.F = F; f.k = prob->k; f.Hs = prob->Hs; f.PF = F * prob->ds + 1; f.NG = NG; f.NC = F * prob->Ht;
+    if (launch_fullhead_tc(a, f, prob->ds, src, tgt, st) != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
 cb_status cb_device_status(cb_ctx *ctx, void *stream)
 {
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;

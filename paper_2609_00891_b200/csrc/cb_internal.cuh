@@ -53,9 +53,18 @@ struct ApplyArgs {
     int src_head[64];
 };
 
+// Full-head contrast statistics: outputs and device tables (see cb_fullhead_stats_accumulate).
+struct FullHeadArgs {
+    float *G, *C;
+    const int *layer_sets, *gi, *gq;   // device
+    int F, k, Hs, PF, NG, NC;
+};
+
 // Launchers (each returns the cudaError_t of its launch and bumps the launch counter on success).
 cudaError_t launch_accum_simt(const AccumArgs &a, int d, cudaStream_t st);
 cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st);
+cudaError_t launch_fullhead_tc(const AccumArgs &a, const FullHeadArgs &f, int d, const cb_kv_view *src, const cb_kv_view *tgt,
+                               cudaStream_t st);
 cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, float *G, float *C, cudaStream_t st);
 cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long long n_tokens,
                          const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st);

@@ -1,0 +1,55 @@
+"""Full-head contrast statistics (all source heads of k selected layers) on the tensor-core kernel vs the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_00891_b200 import binding as cb
+from paper_2609_00891_b200 import synth
+from util import bits, rel_fro
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.mark.parametrize("name,k", [("mini_ragged", 2), ("mini_ragged", 4), ("mid_scaled", 2)])
+def test_fullhead_statistics_match_oracle(name, k):
+    wl = synth.workload(name)
+    sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    sets = cb.cb_fullhead_layer_sets(wl.Ls, wl.Lt, k)
+    assert np.array_equal(sets, oracle.fullhead_layer_sets(wl.Ls, wl.Lt, k))          # bookkeeping: bit-exact
+    law = synth.map_law(wl)
+    chunks = [synth.make_chunk(wl, c, sl, sh, law=law) for c in range(min(2, wl.n_chunks))]
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
+    pf, d = prob.pf, wl.d
+    G = torch.zeros(2, wl.Lt, pf, pf, device=DEV)
+    C = torch.zeros(2, wl.Lt, wl.Ht, pf, d, device=DEV)
+    for ch in chunks:                                                                  # two calls: additive
+        t = {k_: v.to(DEV) for k_, v in ch.items() if torch.is_tensor(v)}
+        wk, wv = t["w_k"][:, 0].contiguous(), t["w_v"][:, 0].contiguous()           # per (comp, layer, token)
+        cb.cb_fullhead_stats_accumulate(prob, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], wk, wv, G, C)
+    torch.cuda.synchronize()
+    Gc, Cc = G.cpu().numpy(), C.cpu().numpy()
+    assert np.isfinite(Gc).all() and np.isfinite(Cc).all()
+    n_tok = sum(ch["n_tokens"] for ch in chunks)
+    tol = 1e-3 if n_tok >= 4096 else 2e-3                                              # plain bf16 fold, see the design doc
+    for comp, l in [(0, 0), (1, wl.Lt - 1), (0, wl.Lt // 2)]:
+        Go = Co = None
+        for ch in chunks:
+            src = bits(ch["src_v" if comp else "src_k"])
+            tgt = bits(ch["tgt_v" if comp else "tgt_k"])
+            w = (ch["w_v"] if comp else ch["w_k"])[l, 0].contiguous().numpy()
+            g, c = oracle.fullhead_stats(src, tgt, w, l, sets[l])
+            Go, Co = (g, c) if Go is None else (Go + g, Co + c)
+        eg, ec = rel_fro(Gc[comp, l], Go), rel_fro(Cc[comp, l], Co)
+        print("full-head (comp %d, layer %d): rel err G %.2e C %.2e" % (comp, l, eg, ec))
+        assert eg <= tol and ec <= tol
+        # every 128 x 128 block separately (a wrong or missing block must not hide in the pooled norm)
+        F = k * wl.Hs
+        for i in range(F):
+            for j in range(F):
+                blk, ref = Gc[comp, l, i * d:(i + 1) * d, j * d:(j + 1) * d], Go[i * d:(i + 1) * d, j * d:(j + 1) * d]
+                assert np.linalg.norm(blk - ref) <= 3 * tol * np.sqrt(np.linalg.norm(Go[i*d:(i+1)*d, i*d:(i+1)*d]) * np.linalg.norm(Go[j*d:(j+1)*d, j*d:(j+1)*d]))
+        np.testing.assert_allclose(Gc[comp, l, pf - 1, :], Go[pf - 1, :], rtol=2e-4, atol=1e-3 * np.abs(Go[pf - 1]).max())
+        np.testing.assert_allclose(Gc[comp, l, :, pf - 1], Go[:, pf - 1], rtol=2e-4, atol=1e-3 * np.abs(Go[pf - 1]).max())
+        np.testing.assert_allclose(Cc[comp, l, :, pf - 1, :], Co[:, pf - 1, :], rtol=2e-4, atol=1e-3 * np.abs(Co[:, pf - 1]).max())
