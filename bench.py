@@ -155,6 +155,9 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--flags", type=int, default=0)
     ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--fullhead", type=int, default=0, metavar="CHUNKS",
+                    help="time the full-head contrast statistics (config 3 shapes: 4 source layers x 8 heads per target "
+                         "layer) on this many 50-sequence chunks and print its own JSON line")
     ap.add_argument("--profile-tokens", type=int, default=0,
                     help="profiling case: run only the accumulate kernel (3 launches) and the apply kernel on this many "
                          "tokens of the same shapes, print timings, no JSON line")
@@ -180,6 +183,9 @@ def main():
     sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     if args.profile_tokens > 0:
         profile_case(args, cb, synth, torch, wl, sl, sh, dev)
+        return
+    if args.fullhead > 0:
+        fullhead_case(args, cb, synth, torch, wl, sl, sh, dev)
         return
     prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, flags=args.flags, n_splits=args.splits)
     ctx = cb.cb_create(prob, device=dev)
@@ -321,6 +327,39 @@ def main():
            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "apply": apply_info,
            "gpu_launches": launches, "clocks": clocks}
     print(json.dumps(out))
+
+
+def fullhead_case(args, cb, synth, torch, wl, sl, sh, dev):
+    """Full-head contrast: statistics for the 4097-wide regressor on the same traces (compute-bound contrast)."""
+    sets = cb.cb_fullhead_layer_sets(wl.Ls, wl.Lt, 4)
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
+    pf, d = prob.pf, wl.d
+    G = torch.zeros(2, wl.Lt, pf, pf, device=dev)
+    C = torch.zeros(2, wl.Lt, wl.Ht, pf, d, device=dev)
+    law = synth.map_law(wl, dev)
+    ms = []
+    for c in range(args.fullhead):
+        ch = synth.make_chunk(wl, c, sl, sh, device=dev, law=law)
+        wk, wv = ch["w_k"][:, 0].contiguous(), ch["w_v"][:, 0].contiguous()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        cb.cb_fullhead_stats_accumulate(prob, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], wk, wv, G, C)
+        e1.record()
+        e1.synchronize()
+        ms.append(e0.elapsed_time(e1))
+        T = ch["n_tokens"]
+        del ch
+    peaks = measured_peaks()
+    F = 32
+    flops_dense = 2.0 * (2 * wl.Lt) * T * (pf * pf + wl.Ht * pf * d)              # definition: full G and every C
+    units = sum(i // 2 + 1 for i in range(F)) + F * wl.Ht
+    flops_issued = 2.0 * (2 * wl.Lt) * units * T * 128 * 256
+    t = min(ms) / 1e3
+    print(json.dumps({"workload": "full-head contrast, 14B->32B shapes, %d tokens per chunk" % T, "ms_per_chunk": ms,
+                      "tokens_per_s": T / t, "dense_tflops": flops_dense / t / 1e12,
+                      "issued_mma_tflops": flops_issued / t / 1e12,
+                      "frac_of_bf16_peak_dense": flops_dense / t / 1e12 / peaks["bf16_tflops"],
+                      "s_per_200_sequences": 4 * statistics.mean(ms) / 1e3}))
 
 
 def profile_case(args, cb, synth, torch, wl, sl, sh, dev):
