@@ -164,6 +164,36 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4 &v, float *f)
         f[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
     }
 }
+// Packed fp32 pairs (sm_100 executes add/mul/fma on two fp32 lanes per instruction): halves the number of
+// floating-point instructions of the fold, which is what the block runs out of (issue slots and power).
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+// bf16 pair (one 32-bit word: low half = first element) -> packed fp32 pair, exact
+__device__ __forceinline__ uint64_t f2_from_bf16x2(unsigned u) { return f2_pack(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)); }
+
 __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
 {
     unsigned r;
@@ -203,8 +233,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
     uint64_t *full = bars;                 // [NS] tile landed: X bytes (1 arrival), Y bytes (1), weights (32 lanes)
     uint64_t *empty = full + C::NS;        // [NS] stage free: MMA done (1) + every fold warp done
     uint64_t *afull = empty + C::NS;       // [NA] weighted operand written (every fold warp)
-    uint64_t *aempty = afull + C::NA;      // [NA] (unused)
-    uint64_t *accfull = aempty + C::NA;    // [2]  accumulator complete (MMA)
+    uint64_t *accfull = afull + C::NA;     // [2]  accumulator complete (MMA)
     uint64_t *accempty = accfull + 2;      // [2]  accumulator drained (4 drain warps)
     uint64_t *redfull = accempty + 2;      // [1]  bias partials of all fold warps written
     uint64_t *reddone = redfull + 1;       // [1]  bias partials consumed
@@ -219,7 +248,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
 
     if (tid == 0) {
         for (int i = 0; i < C::NS; ++i) { mbar_init(&full[i], 2 + 32); mbar_init(&empty[i], 1 + C::FOLD_WARPS); }
-        for (int i = 0; i < C::NA; ++i) { mbar_init(&afull[i], C::FOLD_WARPS); mbar_init(&aempty[i], 1); }
+        for (int i = 0; i < C::NA; ++i) mbar_init(&afull[i], C::FOLD_WARPS);
         for (int i = 0; i < 2; ++i) { mbar_init(&accfull[i], 1); mbar_init(&accempty[i], C::DRAIN_WARPS); }
         mbar_init(redfull, C::FOLD_WARPS);
         mbar_init(reddone, C::FOLD_WARPS);
@@ -367,8 +396,9 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
         cur.start(P, n_units, n_maps, n_tiles);
         while (cur.valid(n_units)) {
             const int m = cur.m, split = cur.split, n_t = cur.tile1 - cur.tile;
+            uint64_t sx2[4], sy2[4];        // packed fp32 pairs: channels (2e, 2e+1) of this thread's chunk
 #pragma unroll
-            for (int e = 0; e < 8; ++e) sx[e] = sy[e] = 0.f;
+            for (int e = 0; e < 4; ++e) sx2[e] = sy2[e] = 0ull;
             sw = 0.f;
             for (int t = 0; t < n_t; ++t) {
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
@@ -386,25 +416,25 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                 for (int i = 0; i < C::RPT; ++i) {
                     const int off = i * C::RG * 128;
                     const float wt = wsm[i * C::RG];
-                    float f[8], pr[8];
-                    unpack_bf16x8(*reinterpret_cast<const uint4 *>(xs + off), f);
+                    const uint64_t w2 = f2_pack(wt, wt);
+                    const uint4 xv = *reinterpret_cast<const uint4 *>(xs + off);
+                    const unsigned xu[4] = {xv.x, xv.y, xv.z, xv.w};
+                    unsigned hw[4], lw[4];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) { pr[e] = wt * f[e]; sx[e] += pr[e]; }
-                    uint4 hi;
-                    hi.x = pack_bf16x2(pr[0], pr[1]); hi.y = pack_bf16x2(pr[2], pr[3]);
-                    hi.z = pack_bf16x2(pr[4], pr[5]); hi.w = pack_bf16x2(pr[6], pr[7]);
-                    *reinterpret_cast<uint4 *>(ah + off) = hi;
-                    if (COMP) {
-                        float hf[8];
-                        unpack_bf16x8(hi, hf);
-                        uint4 lo;
-                        lo.x = pack_bf16x2(pr[0] - hf[0], pr[1] - hf[1]); lo.y = pack_bf16x2(pr[2] - hf[2], pr[3] - hf[3]);
-                        lo.z = pack_bf16x2(pr[4] - hf[4], pr[5] - hf[5]); lo.w = pack_bf16x2(pr[6] - hf[6], pr[7] - hf[7]);
-                        *reinterpret_cast<uint4 *>(ah + C::A_BYTES + off) = lo;
+                    for (int e = 0; e < 4; ++e) {
+                        const uint64_t pr = f2_mul(w2, f2_from_bf16x2(xu[e]));     // w * x for two channels
+                        sx2[e] = f2_add(sx2[e], pr);
+                        float p0, p1;
+                        f2_unpack(pr, p0, p1);
+                        hw[e] = pack_bf16x2(p0, p1);
+                        if (COMP) lw[e] = pack_bf16x2(p0 - __uint_as_float(hw[e] << 16), p1 - __uint_as_float(hw[e] & 0xffff0000u));
                     }
-                    unpack_bf16x8(*reinterpret_cast<const uint4 *>(ys + off), f);
+                    *reinterpret_cast<uint4 *>(ah + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                    if (COMP) *reinterpret_cast<uint4 *>(ah + C::A_BYTES + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                    const uint4 yv = *reinterpret_cast<const uint4 *>(ys + off);
+                    const unsigned yu[4] = {yv.x, yv.y, yv.z, yv.w};
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) sy[e] = fmaf(wt, f[e], sy[e]);
+                    for (int e = 0; e < 4; ++e) sy2[e] = f2_fma(w2, f2_from_bf16x2(yu[e]), sy2[e]);
                     if (cc == 0) sw += wt;
                 }
                 fence_async_smem();
@@ -415,6 +445,8 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                 ar.next();
                 ++it;
             }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { f2_unpack(sx2[e], sx[2 * e], sx[2 * e + 1]); f2_unpack(sy2[e], sy[2 * e], sy[2 * e + 1]); }
             // ---- bias sums of this unit: lanes holding the same channels add up, then a fixed-order sum over the
             //      warps, then read-modify-write of the slot ----
             if (C::CC == 16) {
