@@ -16,6 +16,16 @@
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
 
+#ifndef CB_AP_NS
+#define CB_AP_NS 3
+#endif
+#ifndef CB_AP_NO
+#define CB_AP_NO 2
+#endif
+#ifndef CB_AP_NACC
+#define CB_AP_NACC 4
+#endif
+
 namespace cb {
 
 using namespace ptx;
@@ -32,12 +42,13 @@ struct ApCfg {
     static constexpr int WBLK = D * 128;                // bytes of one W block: D rows (input channels) of 128 bytes
     static constexpr int W_BYTES = NB * WBLK;           // hi (or lo) part of W
     static constexpr int O_BYTES = NB * XBLK;           // bf16 output tile
-    static constexpr int NS = 3;
-    static constexpr int NACC = 2;
+    static constexpr int NS = CB_AP_NS;
+    static constexpr int NO = CB_AP_NO;                 // output tiles in shared memory
+    static constexpr int NACC = CB_AP_NACC;
     static constexpr int TMEM_COLS = (NACC * D < 32) ? 32 : NACC * D;
     static constexpr int EPI_WARPS = 4, CONV_WARPS = 4;
     static constexpr int THREADS = (2 + EPI_WARPS + CONV_WARPS) * 32;
-    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * X_BYTES + 2 * (size_t)W_BYTES + O_BYTES + D * 4 + 256;
+    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * X_BYTES + 2 * (size_t)W_BYTES + (size_t)NO * O_BYTES + D * 4 + 256;
 };
 
 struct ApParams {
@@ -90,7 +101,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
     uint8_t *whi = xs + (size_t)C::NS * C::X_BYTES;       // [NB][D rows][128 B]
     uint8_t *wlo = whi + C::W_BYTES;
     uint8_t *os = wlo + C::W_BYTES;                       // [NB][TT rows][128 B] bf16 output tile
-    float *bias = reinterpret_cast<float *>(os + C::O_BYTES);
+    float *bias = reinterpret_cast<float *>(os + (size_t)C::NO * C::O_BYTES);
     uint64_t *bars = reinterpret_cast<uint64_t *>(bias + D);
     uint64_t *xfull = bars;                  // [NS]
     uint64_t *xempty = xfull + C::NS;        // [NS]   MMA done with the stage
@@ -99,9 +110,9 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
     uint64_t *wready = accempty + C::NACC;   // [1]    W of the current unit converted (CONV_WARPS arrivals)
     uint64_t *wfree = wready + 1;            // [1]    last MMA of the unit done: W may be overwritten
     uint64_t *bfree = wfree + 1;             // [1]    bias of the unit no longer needed (EPI_WARPS arrivals)
-    uint64_t *owritten = bfree + 1;          // [1]    output tile written by all epilogue warps
-    uint64_t *ofree = owritten + 1;          // [1]    output tile read by the store
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ofree + 1);
+    uint64_t *owritten = bfree + 1;          // [NO]   output tile written by all epilogue warps
+    uint64_t *ofree = owritten + C::NO;      // [NO]   output tile read by its store
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ofree + C::NO);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const ApplyArgs &a = P.a;
@@ -117,8 +128,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         mbar_init(wready, C::CONV_WARPS);
         mbar_init(wfree, 1);
         mbar_init(bfree, C::EPI_WARPS);
-        mbar_init(owritten, C::EPI_WARPS);
-        mbar_init(ofree, 1);
+        for (int i = 0; i < C::NO; ++i) { mbar_init(&owritten[i], C::EPI_WARPS); mbar_init(&ofree[i], 1); }
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
@@ -200,8 +210,11 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         ApIter cur;
         cur.start(n_units, n_maps, n_tiles, P.n_splits);
         ApRing<C::NACC> ac;
-        uint32_t uc = 0, oc = 0;
+        ApRing<C::NO> ob;
+        uint32_t uc = 0;
         const bool storer = (warp == 2 && lane == 0);
+        ApRing<C::NO> oldest;          // storer only: oldest output tile whose store may still be reading
+        int pending = 0;
         while (cur.u < n_units) {
             const int m = cur.m;
             const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
@@ -213,7 +226,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ac.idx * D;
                 const int tok = tile * C::TT + row;
                 if (out_bf16) {
-                    if (!mbar_wait_warp(ofree, (oc & 1) ^ 1, abort_flag, lane)) goto teardown;
+                    uint8_t *ot = os + (size_t)ob.idx * C::O_BYTES;
+                    if (!mbar_wait_warp(&ofree[ob.idx], ob.phase ^ 1, abort_flag, lane)) goto teardown;
 #pragma unroll 1
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
@@ -228,22 +242,28 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                             pk.z = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 4]) + bias[n0 + 4], __uint_as_float(r[v * 8 + 5]) + bias[n0 + 5]);
                             pk.w = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 6]) + bias[n0 + 6], __uint_as_float(r[v * 8 + 7]) + bias[n0 + 7]);
                             const int blk = n0 >> 6, chunk = (n0 & 63) >> 3;
-                            *reinterpret_cast<uint4 *>(os + blk * C::XBLK + row * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
+                            *reinterpret_cast<uint4 *>(ot + blk * C::XBLK + row * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
                         }
                     }
                     tc_fence_before();
                     fence_async_smem();
                     __syncwarp();
-                    if (lane == 0) { mbar_arrive(&accempty[ac.idx]); mbar_arrive(owritten); }
+                    if (lane == 0) { mbar_arrive(&accempty[ac.idx]); mbar_arrive(&owritten[ob.idx]); }
                     if (storer) {
-                        if (!mbar_wait(owritten, oc & 1, abort_flag)) goto teardown_store;
-                        tma_store_5d(omap, os, 0, tile * C::TT, 0, h, l);
-                        tma_store_commit();
-                        tma_store_wait_read();
-                        mbar_arrive(ofree);
+                        // free the tile whose store was issued NO - 1 tiles ago, then issue this tile's store
+                        if (mbar_wait(&owritten[ob.idx], ob.phase, abort_flag)) {
+                            tma_store_5d(omap, ot, 0, tile * C::TT, 0, h, l);
+                            tma_store_commit();
+                            if (pending == C::NO - 1) {
+                                tma_store_wait_read_keep<C::NO - 1>();
+                                mbar_arrive(&ofree[oldest.idx]);
+                                oldest.next();
+                            } else {
+                                ++pending;
+                            }
+                        }
                     }
-                teardown_store:
-                    ++oc;
+                    ob.next();
                 } else {
                     float *orow = reinterpret_cast<float *>(comp ? a.out_v : a.out_k) +
                                   (long long)l * a.o_sl + (long long)tok * a.o_st + (long long)h * a.o_sh;
@@ -273,7 +293,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
             ++uc;
             cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
         }
-        if (storer) tma_store_wait_all();
+        if (storer) tma_store_wait_all();          // remaining tiles need no release: nobody waits for them
     } else {
         // ================================ W conversion warps ================================
         const int ct = tid - (2 + C::EPI_WARPS) * 32;                 // 0 .. CONV_WARPS*32-1

@@ -111,6 +111,9 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap *map, const void 
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // All of this thread's committed stores have finished READING shared memory (the buffer may be rewritten).
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// All but the N most recent committed store groups have finished reading shared memory.
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read_keep() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 // All of this thread's committed stores are complete.
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map)
