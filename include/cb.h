@@ -189,6 +189,19 @@ cb_status cb_apply(const cb_problem *prob, const float *Wb, const cb_kv_view *sr
                    int64_t t_stride_head, int32_t out_dtype, void *stream);
 
 /*
+ * Effective-sample-size floor on the calibration weights (Section 3.3): for each of the n_rows rows (one per layer,
+ * head and component) of raw sensitivities r_raw >= 0 over n_tokens rows of the calibration set,
+ *     r_i = r_raw_i / mean(r_raw),  CV^2 = mean (r_i - 1)^2,  tau = min(n, 2 p_width),
+ *     alpha* = 1 if CV^2 = 0 else min(1, sqrt((n / tau - 1) / CV^2)),      w_i = 1 + alpha* (r_i - 1),
+ * so that the Kish effective sample size n / (1 + alpha^2 CV^2) of the mean-one weights stays >= tau.
+ * r_raw, w: device fp32, row r at base + r*row_stride (elements), may not overlap; alpha_out: device fp32 [n_rows]
+ * or NULL.  p_width is the regressor's feature width (k * d_s).  A row without any sensitivity gives w = 1.
+ * The whole calibration set of a row must be passed in one call (the floor depends on n).
+ */
+cb_status cb_ess_weights(const float *r_raw, int32_t n_rows, int64_t n_tokens, int64_t r_row_stride,
+                         int64_t p_width, float *w, int64_t w_row_stride, float *alpha_out, void *stream);
+
+/*
  * Full-head contrast (Section 3.1, Eq. "fullheadfeature"; the inherited baseline of Section 2.1): every target head
  * of layer l is regressed from ALL H_s source KV heads of k selected source layers, feature order layer-major, then
  * head, then channel, bias last: P_f = k*H_s*d + 1.  Statistics per (comp, l): one G (P_f x P_f) shared by the

@@ -211,6 +211,28 @@ def apply_maps(src_k: np.ndarray, src_v: np.ndarray, Theta: np.ndarray, Lt: int,
     return ((ok, ov) if want_f64 else None), ((bk, bv) if want_bf16 else None)
 
 
+# ----------------------------------------------------------------------------- ESS floor on the weights
+def ess_weights(r_raw: np.ndarray, p_width: int):
+    """Shrink mean-normalised sensitivities toward uniform so that the Kish effective sample size stays at or above
+    min(n, 2 p).  r_raw: [n] or [maps][n].  Returns (w, alpha, cv2) with matching leading shape."""
+    r = np.ascontiguousarray(r_raw, dtype=np.float64)
+    single = r.ndim == 1
+    if single:
+        r = r[None]
+    w = np.empty_like(r)
+    alpha = np.empty(len(r))
+    cv2 = np.empty(len(r))
+    lib = _load()
+    lib.orc_ess_weights.restype = ctypes.c_double
+    for i in range(len(r)):
+        c = ctypes.c_double(0.0)
+        alpha[i] = lib.orc_ess_weights(_p(r[i]), _i64(r.shape[1]), _i64(p_width), _p(w[i]), ctypes.byref(c))
+        cv2[i] = c.value
+    if single:
+        return w[0], float(alpha[0]), float(cv2[0])
+    return w, alpha, cv2
+
+
 # ----------------------------------------------------------------------------- full-head contrast
 def fullhead_layer_sets(Ls: int, Lt: int, k: int = 4) -> np.ndarray:
     """int32 [Lt][k]: k consecutive source layers around the nearest-depth layer, clipped into range."""

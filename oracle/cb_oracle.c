@@ -435,3 +435,42 @@ void orc_fullhead_layer_sets(int32_t Ls, int32_t Lt, int32_t k, int32_t *sets /*
         for (int32_t q = 0; q < k; ++q) sets[l * k + q] = lo + q;
     }
 }
+
+/* ------------------------------------------------------------------------- */
+/* Effective-sample-size floor on the attention weights (Section 3.3).        */
+/* For one (layer, head, component): raw sensitivities r_raw >= 0 over n       */
+/* rows are mean-normalised (mean r = 1), CV^2 = mean (r_i - 1)^2, and the     */
+/* weights are shrunk toward uniform, w_i = 1 + alpha (r_i - 1), with the      */
+/* largest alpha in [0, 1] whose Kish effective sample size                    */
+/*   n_eff = (sum w)^2 / sum w^2 = n / (1 + alpha^2 CV^2)                      */
+/* stays at or above tau = min(n, 2 p) (p = feature width):                    */
+/*   alpha* = 1 if CV^2 = 0, else min(1, sqrt((n / tau - 1) / CV^2)).          */
+/* Returns alpha*; cv2_out (may be NULL) receives CV^2.  A row of zeros (no    */
+/* sensitivity at all) gives uniform weights.                                 */
+/* ------------------------------------------------------------------------- */
+double orc_ess_weights(const double *r_raw, int64_t n, int64_t p_width, double *w, double *cv2_out)
+{
+    double mean = 0.0;
+    for (int64_t i = 0; i < n; ++i) mean += r_raw[i];
+    mean /= (double)n;
+    if (!(mean > 0.0)) {
+        for (int64_t i = 0; i < n; ++i) w[i] = 1.0;
+        if (cv2_out) *cv2_out = 0.0;
+        return 1.0;
+    }
+    double cv2 = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        const double r = r_raw[i] / mean;
+        cv2 += (r - 1.0) * (r - 1.0);
+    }
+    cv2 /= (double)n;
+    const double tau = (double)((n < 2 * p_width) ? n : 2 * p_width);
+    double alpha = 1.0;
+    if (cv2 > 0.0) {
+        const double a = sqrt(((double)n / tau - 1.0) / cv2);
+        alpha = a < 1.0 ? a : 1.0;
+    }
+    for (int64_t i = 0; i < n; ++i) w[i] = 1.0 + alpha * (r_raw[i] / mean - 1.0);
+    if (cv2_out) *cv2_out = cv2;
+    return alpha;
+}

@@ -26,7 +26,7 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_destroy", "cb_stats_reset", "cb_stats_accumulate", "cb_staging_bytes", "cb_stats_accumulate_host",
            "cb_stats_reduce", "cb_ridge_solve",
            "cb_check_info", "cb_apply", "cb_device_status", "cb_stats_build_static", "cb_fullhead_layer_sets",
-           "cb_fullhead_workspace_bytes", "cb_fullhead_stats_accumulate", "cb_launch_count")
+           "cb_fullhead_workspace_bytes", "cb_fullhead_stats_accumulate", "cb_ess_weights", "cb_launch_count")
 
 
 class CbError(RuntimeError):
@@ -270,6 +270,20 @@ def cb_stats_build_static(prob: Problem, src_k, src_v, tgt_k, tgt_v, w_k: torch.
                                        ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
                                        ctypes.c_void_p(G.data_ptr()), ctypes.c_void_p(C.data_ptr()),
                                        _stream_ptr(stream)), "cb_stats_build_static")
+
+
+def cb_ess_weights(r_raw: torch.Tensor, p_width: int, w: torch.Tensor, alpha: Optional[torch.Tensor] = None, stream=None) -> None:
+    """r_raw, w: fp32 device tensors [..., n_tokens] (rows = everything but the last axis, dense); alpha: [rows] or None."""
+    assert r_raw.dtype == torch.float32 and w.dtype == torch.float32 and r_raw.is_contiguous() and w.is_contiguous()
+    assert r_raw.shape == w.shape
+    n = r_raw.shape[-1]
+    rows = r_raw.numel() // n
+    if alpha is not None:
+        assert alpha.dtype == torch.float32 and alpha.numel() == rows and alpha.is_contiguous()
+    _check(lib().cb_ess_weights(ctypes.c_void_p(r_raw.data_ptr()), rows, ctypes.c_int64(n), ctypes.c_int64(n),
+                                ctypes.c_int64(p_width), ctypes.c_void_p(w.data_ptr()), ctypes.c_int64(n),
+                                ctypes.c_void_p(alpha.data_ptr() if alpha is not None else 0), _stream_ptr(stream)),
+           "cb_ess_weights")
 
 
 class _FullHeadProblem(ctypes.Structure):
