@@ -172,6 +172,18 @@ cb_status cb_ridge_solve(const float *G, const float *C, int32_t n_maps, int32_t
                          const float *lambdas, int32_t n_lambda, uint32_t flags,
                          float *Wb, int32_t *info, void *stream);
 
+/*
+ * The same solve for wider regressors (head-local support over k > 1 selected layers, Section 3.2: P = k*d + 1, e.g.
+ * 1025 for k = 8), where a system does not fit in shared memory: blocked Cholesky and substitutions in fp64 on a
+ * padded copy of every system.  G [n_maps][P][P], C [n_maps][P][d], Wb [n_lambda][n_maps][P][d], info as above.
+ * workspace: device, 256-byte aligned, at least cb_ridge_solve_large_workspace_bytes(P, d, 1); systems are processed
+ * in batches of as many as fit (all n_lambda * n_maps at once if the workspace is large enough).
+ */
+cb_status cb_ridge_solve_large_workspace_bytes(int32_t P, int32_t d, int64_t n_systems, size_t *bytes);
+cb_status cb_ridge_solve_large(const float *G, const float *C, int32_t n_maps, int32_t P, int32_t d, int64_t n_tokens,
+                               const float *lambdas, int32_t n_lambda, uint32_t flags,
+                               float *Wb, int32_t *info, void *workspace, size_t workspace_bytes, void *stream);
+
 /* Synchronises the stream and returns CB_ERR_NOT_PD if any of the n info entries is non-zero
  * (*first_bad, may be NULL, receives its index), CB_OK otherwise. */
 cb_status cb_check_info(const int32_t *info, int64_t n, void *stream, int64_t *first_bad);
@@ -228,6 +240,21 @@ cb_status cb_fullhead_workspace_bytes(const cb_fullhead_problem *prob, size_t *b
 cb_status cb_fullhead_stats_accumulate(const cb_fullhead_problem *prob, const cb_kv_view *src, const cb_kv_view *tgt,
                                        const float *w_k, const float *w_v, int64_t w_stride_layer,
                                        float *G, float *C, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Head-local support over k > 1 selected source layers (Section 3.2, Eq. "localfeature": the paper's operating point,
+ * k = 8 for Qwen3): the feature of target (l, h) concatenates source head src_head[h] of the k layers
+ * prob->layer_sets[l][0..k-1] (layer-major, bias last), P = k*d + 1.  cb_multilayer_stats_accumulate ADDS this call's
+ * statistics to G [n_maps][P][P] and C [n_maps][P][d] (device fp32, caller-owned, zeroed by the caller first; map id
+ * m = (comp*Lt + l)*Ht + h; both triangles of G are filled).  Weights per (comp, l, h, token) as for
+ * cb_stats_accumulate.  prob->Hs, prob->Ht describe the models; src_head: HOST [Ht].  workspace: device, 256-byte
+ * aligned, cb_multilayer_workspace_bytes().  The systems are solved with cb_ridge_solve_large.
+ */
+cb_status cb_multilayer_workspace_bytes(const cb_fullhead_problem *prob, size_t *bytes);
+cb_status cb_multilayer_stats_accumulate(const cb_fullhead_problem *prob, const int32_t *src_head,
+                                         const cb_kv_view *src, const cb_kv_view *tgt,
+                                         const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                                         float *G, float *C, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Synchronises the stream and reads the context's device status word: CB_OK, or CB_ERR_TIMEOUT if a bounded

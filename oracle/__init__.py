@@ -257,6 +257,27 @@ def fullhead_stats(src: np.ndarray, tgt: np.ndarray, w: np.ndarray, l: int, laye
     return G, C
 
 
+def multilayer_stats(src: np.ndarray, tgt: np.ndarray, w: np.ndarray, l: int, h: int, g: int, layer_set: Sequence[int]):
+    """Head-local statistics over several selected layers for one map (component given by src/tgt): the feature
+    concatenates source head g of the layers in layer_set; target (l, h); w fp32 [T].  G [P][P], C [P][d], P = k*d + 1."""
+    G, C = fullhead_stats(src[:, :, g:g + 1, :], tgt[:, :, h:h + 1, :], w, l, layer_set)
+    return G, C[0]
+
+
+def ridge_solve_general(G: np.ndarray, C: np.ndarray, n: int, lam: float, raw_lambda: bool = False):
+    """Theta [p][dy] and info for one system of any width (bias entry last, not penalised)."""
+    G = np.ascontiguousarray(G, dtype=np.float64)
+    C = np.ascontiguousarray(C, dtype=np.float64)
+    p, dy = C.shape
+    assert G.shape == (p, p)
+    Theta = np.empty((p, dy), np.float64)
+    lib = _load()
+    lib.orc_ridge_solve_pd.restype = ctypes.c_int32
+    info = lib.orc_ridge_solve_pd(_p(G), _p(C), _i32(p), _i32(dy), _i64(n), ctypes.c_double(lam),
+                                  _i32(1 if raw_lambda else 0), _p(Theta))
+    return Theta, int(info)
+
+
 # ----------------------------------------------------------------------------- artifact size
 def coefficient_counts(Lt: int, Ht: int, Hs: int, k: int, ds: int, dt: int):
     """Non-bias coefficient counts over K and V (Section 3.2): (C_full, C_local, number of bias entries).

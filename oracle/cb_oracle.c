@@ -474,3 +474,24 @@ double orc_ess_weights(const double *r_raw, int64_t n, int64_t p_width, double *
     if (cv2_out) *cv2_out = cv2;
     return alpha;
 }
+
+/* The ridge solve for a regressor of any width (several selected layers): G [p][p], C [p][dy], bias entry last and not */
+/* penalised; same conventions as orc_ridge_solve.                                                                      */
+int32_t orc_ridge_solve_pd(const double *G, const double *C, int32_t p, int32_t dy, int64_t n,
+                           double lambda, int32_t raw_lambda, double *Theta /* [p][dy] */)
+{
+    double *A = (double *)malloc(sizeof(double) * (size_t)p * p);
+    memcpy(A, G, sizeof(double) * (size_t)p * p);
+    const double s_w = G[(size_t)(p - 1) * p + (p - 1)];
+    const double lam = raw_lambda ? lambda : lambda * s_w / (double)n;
+    for (int32_t i = 0; i < p - 1; ++i) A[(size_t)i * p + i] += lam;
+    int32_t info = orc_cholesky(A, p);
+    if (info != 0) {
+        memset(Theta, 0, sizeof(double) * (size_t)p * dy);
+    } else {
+        memcpy(Theta, C, sizeof(double) * (size_t)p * dy);
+        orc_cholesky_solve(A, p, Theta, dy);
+    }
+    free(A);
+    return info;
+}

@@ -26,7 +26,8 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_destroy", "cb_stats_reset", "cb_stats_accumulate", "cb_staging_bytes", "cb_stats_accumulate_host",
            "cb_stats_reduce", "cb_ridge_solve",
            "cb_check_info", "cb_apply", "cb_device_status", "cb_stats_build_static", "cb_fullhead_layer_sets",
-           "cb_fullhead_workspace_bytes", "cb_fullhead_stats_accumulate", "cb_ess_weights", "cb_launch_count")
+           "cb_fullhead_workspace_bytes", "cb_fullhead_stats_accumulate", "cb_ess_weights", "cb_ridge_solve_large_workspace_bytes", "cb_ridge_solve_large", "cb_multilayer_workspace_bytes",
+           "cb_multilayer_stats_accumulate", "cb_launch_count")
 
 
 class CbError(RuntimeError):
@@ -236,6 +237,29 @@ def cb_ridge_solve(G: torch.Tensor, C: torch.Tensor, n_tokens: int, lambdas: Seq
                                 ctypes.c_void_p(info.data_ptr()), _stream_ptr(stream)), "cb_ridge_solve")
 
 
+def cb_ridge_solve_large_workspace_bytes(P: int, d: int, n_systems: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().cb_ridge_solve_large_workspace_bytes(P, d, ctypes.c_int64(n_systems), ctypes.byref(n)),
+           "cb_ridge_solve_large_workspace_bytes")
+    return n.value
+
+
+def cb_ridge_solve_large(G: torch.Tensor, C: torch.Tensor, n_tokens: int, lambdas: Sequence[float], flags: int,
+                         Wb: torch.Tensor, info: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    """G [n_maps][P][P], C [n_maps][P][d] fp32; any P >= 2 (regressors over several source layers)."""
+    n_maps, P, _ = G.shape
+    d = C.shape[2]
+    lam = np.ascontiguousarray(lambdas, dtype=np.float32)
+    assert G.is_contiguous() and C.is_contiguous() and Wb.is_contiguous() and info.is_contiguous()
+    assert G.dtype == torch.float32 and C.dtype == torch.float32 and Wb.dtype == torch.float32 and info.dtype == torch.int32
+    assert C.shape == (n_maps, P, d) and Wb.numel() == len(lam) * n_maps * P * d and info.numel() == len(lam) * n_maps
+    _check(lib().cb_ridge_solve_large(ctypes.c_void_p(G.data_ptr()), ctypes.c_void_p(C.data_ptr()), n_maps, P, d,
+                                      ctypes.c_int64(n_tokens), lam.ctypes.data_as(ctypes.c_void_p), len(lam),
+                                      ctypes.c_uint32(flags), ctypes.c_void_p(Wb.data_ptr()), ctypes.c_void_p(info.data_ptr()),
+                                      ctypes.c_void_p(workspace.data_ptr()), ctypes.c_size_t(workspace.numel()),
+                                      _stream_ptr(stream)), "cb_ridge_solve_large")
+
+
 def cb_check_info(info: torch.Tensor, stream=None) -> None:
     bad = ctypes.c_int64(-1)
     _check(lib().cb_check_info(ctypes.c_void_p(info.data_ptr()), ctypes.c_int64(info.numel()), _stream_ptr(stream),
@@ -336,6 +360,28 @@ def cb_fullhead_stats_accumulate(prob: FullHeadProblem, src_k, src_v, tgt_k, tgt
                                               ctypes.c_void_p(C.data_ptr()), ctypes.c_void_p(workspace.data_ptr()),
                                               ctypes.c_size_t(workspace.numel()), _stream_ptr(stream)),
            "cb_fullhead_stats_accumulate")
+
+
+def cb_multilayer_stats_accumulate(prob: FullHeadProblem, src_head, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor,
+                                   w_v: torch.Tensor, G: torch.Tensor, C: torch.Tensor, stream=None) -> None:
+    """Head-local statistics over k selected layers: adds to G [n_maps][P][P], C [n_maps][P][d], P = k*d + 1.
+    Weights [Lt][Ht][T] fp32."""
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    sh = np.ascontiguousarray(src_head, dtype=np.int32)
+    P = prob.k * prob.ds + 1
+    n_maps = 2 * prob.Lt * prob.Ht
+    assert w_k.dtype == torch.float32 and w_v.dtype == torch.float32 and w_k.dim() == 3 and w_k.stride() == w_v.stride()
+    assert G.dtype == torch.float32 and C.dtype == torch.float32 and G.is_contiguous() and C.is_contiguous()
+    assert G.numel() == n_maps * P * P and C.numel() == n_maps * P * prob.ds
+    n = ctypes.c_size_t(0)
+    _check(lib().cb_multilayer_workspace_bytes(ctypes.byref(prob.c), ctypes.byref(n)), "cb_multilayer_workspace_bytes")
+    ws = torch.empty(n.value, dtype=torch.uint8, device=G.device)
+    _check(lib().cb_multilayer_stats_accumulate(ctypes.byref(prob.c), sh.ctypes.data_as(ctypes.c_void_p), ctypes.byref(sv),
+                                                ctypes.byref(tv), ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                                ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
+                                                ctypes.c_void_p(G.data_ptr()), ctypes.c_void_p(C.data_ptr()),
+                                                ctypes.c_void_p(ws.data_ptr()), ctypes.c_size_t(ws.numel()), _stream_ptr(stream)),
+           "cb_multilayer_stats_accumulate")
 
 
 def cb_device_status(ctx: Context, stream=None) -> None:

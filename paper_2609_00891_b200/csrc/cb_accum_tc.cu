@@ -68,11 +68,14 @@ struct TcCfg {
 // layers: F = k*Hs feature heads.  Units per (comp, l): NG "G units" (i, q), 2q <= i: rows of feature head i against
 // feature heads 2q and 2q+1 (the lower triangle of G, mirrored on write), then F*Ht "C units" (i, h): feature head i
 // against target head h.  Results are added straight into G / C.
+// per_head = 1 is the head-local support over k > 1 selected layers (Section 3.2): one group per map (comp, l, h),
+// F = k feature heads (layer S_l[f], source head a(h)), weights per (l, h), G [n_maps][PF][PF], C [n_maps][PF][d].
 struct FhDev {
-    float *G, *C;                 // [2][Lt][PF][PF], [2][Lt][Ht][PF][d]
+    float *G, *C;                 // full-head: [2][Lt][PF][PF], [2][Lt][Ht][PF][d]
     const int *layer_sets;        // device [Lt][k]
     const int *gi, *gq;           // device [NG]
-    int F, k, Hs, PF, NG, NC;
+    const int *src_head;          // device [Ht] (per_head only)
+    int F, k, Hs, PF, NG, NC, per_head;
 };
 
 struct TcParams {
@@ -93,6 +96,8 @@ struct TileIterT {
     int b1_layer, b1_head;          // first half of the second operand (a source head)
     int b2_layer, b2_head, b2_tgt;  // second half: target head (b2_tgt) or source head
     int fi, fj;                     // full-head: feature head of the rows; first feature head of the columns, or -1
+    int out_g, out_c;               // full-head: which G matrix / C block the unit adds to
+    int wr_sa, wr_sb, wr_sw;        // full-head C units: which bias entries this unit owns
     __device__ __forceinline__ void start(const TcParams &P, int n_units, int n_maps, int n_tiles)
     {
         u = (int)blockIdx.x - (int)gridDim.x;
@@ -109,24 +114,44 @@ struct TileIterT {
             const FhDev &f = P.fh;
             const int per = f.NG + f.NC;
             const int group = u / per, v = u % per;
-            comp = group / a.Lt;
-            l = group % a.Lt;
+            int src_h = 0;                                  // per_head: the one source head of this map
+            if (f.per_head) {
+                comp = group / (a.Lt * a.Ht);
+                l = (group / a.Ht) % a.Lt;
+                h = group % a.Ht;
+                src_h = f.src_head[h];
+            } else {
+                comp = group / a.Lt;
+                l = group % a.Lt;
+                h = 0;
+            }
             m = u; split = 0; tile = 0; tile1 = n_tiles;
+            // feature head f -> (source layer, source head)
+            auto feat_layer = [&](int ft) { return f.layer_sets[l * f.k + (f.per_head ? ft : ft / f.Hs)]; };
+            auto feat_head = [&](int ft) { return f.per_head ? src_h : ft % f.Hs; };
             if (v < f.NG) {
                 fi = f.gi[v];
                 fj = 2 * f.gq[v];
-                b1_layer = f.layer_sets[l * f.k + fj / f.Hs];          b1_head = fj % f.Hs;
-                b2_layer = f.layer_sets[l * f.k + (fj + 1) / f.Hs];    b2_head = (fj + 1) % f.Hs;
-                b2_tgt = 0; h = 0;
+                const int fj2 = (fj + 1 < f.F) ? fj + 1 : fj;    // odd F: the last pair repeats its first head (not stored)
+                b1_layer = feat_layer(fj);   b1_head = feat_head(fj);
+                b2_layer = feat_layer(fj2);  b2_head = feat_head(fj2);
+                b2_tgt = 0;
+                wr_sa = wr_sb = wr_sw = 0;
             } else {
-                fi = (v - f.NG) / a.Ht;
-                h = (v - f.NG) % a.Ht;
+                const int vc = v - f.NG;
                 fj = -1;
-                b1_layer = f.layer_sets[l * f.k + fi / f.Hs];          b1_head = fi % f.Hs;
+                if (f.per_head) { fi = vc; }
+                else { fi = vc / a.Ht; h = vc % a.Ht; }
+                b1_layer = feat_layer(fi);   b1_head = feat_head(fi);
                 b2_layer = l; b2_head = h; b2_tgt = 1;
+                wr_sa = f.per_head ? 1 : (h == 0);
+                wr_sb = (fi == 0);
+                wr_sw = (fi == 0) && (f.per_head || h == 0);
             }
-            a_layer = f.layer_sets[l * f.k + fi / f.Hs];
-            a_head = fi % f.Hs;
+            a_layer = feat_layer(fi);
+            a_head = feat_head(fi);
+            out_g = group;
+            out_c = f.per_head ? group : group * a.Ht + h;
             return;
         }
         do {
@@ -151,7 +176,7 @@ struct TileIterT {
     }
     __device__ __forceinline__ const float *weights(const AccumArgs &a) const
     {
-        return (comp ? a.w_v : a.w_k) + (long long)l * a.w_sl + (FH ? 0ll : (long long)h * a.w_sh);
+        return (comp ? a.w_v : a.w_k) + (long long)l * a.w_sl + (long long)h * a.w_sh;   // full-head passes w_sh = 0
     }
 };
 
@@ -243,7 +268,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
     const AccumArgs &a = P.a;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_maps = 2 * a.Lt * a.Ht;
-    const int n_units = FH ? 2 * a.Lt * (P.fh.NG + P.fh.NC) : n_maps * a.n_splits;
+    const int n_units = FH ? 2 * a.Lt * (P.fh.per_head ? a.Ht : 1) * (P.fh.NG + P.fh.NC) : n_maps * a.n_splits;
     const int n_tiles = (a.n_tokens + C::TT - 1) / C::TT;
 
     if (tid == 0) {
@@ -480,25 +505,24 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
             if (lane == 0) mbar_arrive(redfull);
             if (!mbar_wait_warp(redfull, uc & 1, abort_flag, lane)) goto teardown;
             if (FH) {
-                // C units carry the bias entries: (i, h = 0) the column/row of feature head i, (i = 0, h) the bias row
-                // of target head h, (0, 0) the weight total.  G units carry none.
+                // C units carry the bias entries (each entry has exactly one owner, see the unit decode).
                 if (cur.fj < 0) {
                     const FhDev &f = P.fh;
                     const size_t PF = (size_t)f.PF;
-                    float *Gg = f.G + ((size_t)cur.comp * a.Lt + cur.l) * PF * PF;
-                    float *Cg = f.C + (((size_t)cur.comp * a.Lt + cur.l) * a.Ht + cur.h) * PF * D;
+                    float *Gg = f.G + (size_t)cur.out_g * PF * PF;
+                    float *Cg = f.C + (size_t)cur.out_c * PF * D;
                     for (int v = ft; v < 2 * D + 1; v += C::FOLD_THREADS) {
                         float sum = 0.f;
 #pragma unroll
                         for (int q = 0; q < C::FOLD_WARPS; ++q) sum += red[q * C::RED_STRIDE + v];
                         if (v < D) {
-                            if (cur.h == 0) {
+                            if (cur.wr_sa) {
                                 Gg[((size_t)cur.fi * D + v) * PF + (PF - 1)] += sum;
                                 Gg[(PF - 1) * PF + (size_t)cur.fi * D + v] += sum;
                             }
                         } else if (v < 2 * D) {
-                            if (cur.fi == 0) Cg[(PF - 1) * D + (v - D)] += sum;
-                        } else if (cur.fi == 0 && cur.h == 0) {
+                            if (cur.wr_sb) Cg[(PF - 1) * D + (v - D)] += sum;
+                        } else if (cur.wr_sw) {
                             Gg[(PF - 1) * PF + (PF - 1)] += sum;
                         }
                     }
@@ -534,7 +558,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                     if (row < D) {
                         const FhDev &f = P.fh;
                         const size_t PF = (size_t)f.PF;
-                        float *Gg = f.G + ((size_t)cur.comp * a.Lt + cur.l) * PF * PF;
+                        float *Gg = f.G + (size_t)cur.out_g * PF * PF;
                         const size_t ri = (size_t)cur.fi * D + row;           // row of G / C this thread holds
 #pragma unroll 1
                         for (int c = 0; c < C::N / 16; ++c) {
@@ -544,7 +568,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                             const int part = (c * 16) / D, c0 = (c * 16) % D;   // which half of [B1 | B2], first column
                             if (cur.fj >= 0) {
                                 const int j = cur.fj + part;                    // feature head of these columns
-                                if (j <= cur.fi) {
+                                if (j <= cur.fi && j < f.F) {
                                     float *dst = Gg + ri * PF + (size_t)j * D + c0;
 #pragma unroll
                                     for (int e = 0; e < 16; ++e) dst[e] += __uint_as_float(r[e]);
@@ -555,7 +579,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                                     }
                                 }
                             } else if (part == 1) {
-                                float *dst = f.C + ((((size_t)cur.comp * a.Lt + cur.l) * a.Ht + cur.h) * PF + ri) * D + c0;
+                                float *dst = f.C + ((size_t)cur.out_c * PF + ri) * D + c0;
 #pragma unroll
                                 for (int e = 0; e < 16; ++e) dst[e] += __uint_as_float(r[e]);
                             }
@@ -661,7 +685,7 @@ static cudaError_t launch_tc(const TcParams &P, cudaStream_t st)
         if (e != cudaSuccess) return e;
         attr = true;
     }
-    const int n_units = FH ? 2 * P.a.Lt * (P.fh.NG + P.fh.NC) : 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
+    const int n_units = FH ? 2 * P.a.Lt * (P.fh.per_head ? P.a.Ht : 1) * (P.fh.NG + P.fh.NC) : 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
     const int grid = n_units < sm_count() ? n_units : sm_count();
     k_accum_tc<D, COMP, FH><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
@@ -699,7 +723,7 @@ cudaError_t launch_fullhead_tc(const AccumArgs &a, const FullHeadArgs &f, int d,
 {
     TcParams P;
     P.a = a;
-    P.fh = FhDev{f.G, f.C, f.layer_sets, f.gi, f.gq, f.F, f.k, f.Hs, f.PF, f.NG, f.NC};
+    P.fh = FhDev{f.G, f.C, f.layer_sets, f.gi, f.gq, f.src_head, f.F, f.k, f.Hs, f.PF, f.NG, f.NC, f.per_head};
     const int TT = 64;
     if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
     P.drain_tiles = 16384 / TT;

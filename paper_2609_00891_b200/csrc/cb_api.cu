@@ -343,6 +343,31 @@ cb_status cb_ridge_solve(const float *G, const float *C, int32_t n_maps, int32_t
     return CB_OK;
 }
 
+cb_status cb_ridge_solve_large_workspace_bytes(int32_t P, int32_t d, int64_t n_systems, size_t *bytes)
+{
+    if (P < 2 || (d != 64 && d != 128) || n_systems < 1 || !bytes) return CB_ERR_INVALID_ARG;
+    *bytes = solve_large_bytes_per_system(P, d) * (size_t)n_systems;
+    return CB_OK;
+}
+
+cb_status cb_ridge_solve_large(const float *G, const float *C, int32_t n_maps, int32_t P, int32_t d, int64_t n_tokens,
+                               const float *lambdas, int32_t n_lambda, uint32_t flags,
+                               float *Wb, int32_t *info, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!G || !C || !lambdas || !Wb || !info) return CB_ERR_INVALID_ARG;
+    if (n_maps < 0 || n_lambda <= 0 || n_lambda > 16 || n_tokens < 0 || P < 2) return CB_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return CB_ERR_UNSUPPORTED;
+    if (P > 8193) return CB_ERR_UNSUPPORTED;
+    for (int i = 0; i < n_lambda; ++i)
+        if (!(lambdas[i] >= 0.f)) return CB_ERR_INVALID_ARG;
+    if (n_maps == 0) return CB_OK;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < solve_large_bytes_per_system(P, d)) return CB_ERR_WORKSPACE;
+    cudaError_t e = launch_solve_large(G, C, n_maps, P, d, n_tokens, lambdas, n_lambda, flags, Wb, info, workspace,
+                                       workspace_bytes, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
 cb_status cb_check_info(const int32_t *info, int64_t n, void *stream, int64_t *first_bad)
 {
     if (!info || n < 0) return CB_ERR_INVALID_ARG;
@@ -475,7 +500,71 @@ cb_status cb_fullhead_stats_accumulate(const cb_fullhead_problem *prob, const cb
     f.layer_sets = static_cast<const int *>(workspace);
     f.gi = f.layer_sets + (size_t)prob->Lt * prob->k;
     f.gq = f.gi + NG;
+    f.src_head = nullptr; f.per_head = 0;
     f.F = F; f.k = prob->k; f.Hs = prob->Hs; f.PF = F * prob->ds + 1; f.NG = NG; f.NC = F * prob->Ht;
+    if (launch_fullhead_tc(a, f, prob->ds, src, tgt, st) != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+cb_status cb_multilayer_workspace_bytes(const cb_fullhead_problem *prob, size_t *bytes)
+{
+    if (!prob || !bytes || prob->k <= 0 || prob->k > 64 || prob->Lt <= 0 || prob->Ht <= 0) return CB_ERR_INVALID_ARG;
+    *bytes = align_up(sizeof(int) * ((size_t)prob->Lt * prob->k + 2 * (size_t)fullhead_ng(prob->k) + (size_t)prob->Ht), 256);
+    return CB_OK;
+}
+
+cb_status cb_multilayer_stats_accumulate(const cb_fullhead_problem *prob, const int32_t *src_head,
+                                         const cb_kv_view *src, const cb_kv_view *tgt,
+                                         const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                                         float *G, float *C, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!prob || !prob->layer_sets || !src_head) return CB_ERR_INVALID_ARG;
+    if (prob->Ls <= 0 || prob->Hs <= 0 || prob->Lt <= 0 || prob->Ht <= 0 || prob->k <= 0 || prob->k > prob->Ls || prob->k > 64)
+        return CB_ERR_INVALID_ARG;
+    if (prob->ds != prob->dt || (prob->ds != 64 && prob->ds != 128)) return CB_ERR_UNSUPPORTED;
+    for (int i = 0; i < prob->Lt * prob->k; ++i)
+        if (prob->layer_sets[i] < 0 || prob->layer_sets[i] >= prob->Ls) return CB_ERR_INVALID_ARG;
+    for (int h = 0; h < prob->Ht; ++h)
+        if (src_head[h] < 0 || src_head[h] >= prob->Hs) return CB_ERR_INVALID_ARG;
+    cb_status s = check_view(src, prob->Ls, prob->Hs, prob->ds);
+    if (s != CB_OK) return s;
+    s = check_view(tgt, prob->Lt, prob->Ht, prob->dt);
+    if (s != CB_OK) return s;
+    if (src->n_tokens != tgt->n_tokens) return CB_ERR_INVALID_ARG;
+    if (src->n_tokens == 0) return CB_OK;
+    if (!w_k || !w_v || w_stride_layer < 0 || w_stride_head < 0 || !G || !C) return CB_ERR_INVALID_ARG;
+    const int F = prob->k, NG = fullhead_ng(F);
+    size_t need = 0;
+    cb_multilayer_workspace_bytes(prob, &need);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return CB_ERR_WORKSPACE;
+    std::vector<int32_t> tab(prob->layer_sets, prob->layer_sets + (size_t)prob->Lt * prob->k);
+    for (int i = 0; i < F; ++i)
+        for (int q = 0; 2 * q <= i; ++q) tab.push_back(i);
+    for (int i = 0; i < F; ++i)
+        for (int q = 0; 2 * q <= i; ++q) tab.push_back(q);
+    tab.insert(tab.end(), src_head, src_head + prob->Ht);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(workspace, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return CB_ERR_CUDA;
+    }
+    AccumArgs a;
+    a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src->k), static_cast<const __nv_bfloat16 *>(src->v),
+                  src->stride_layer, src->stride_token, src->stride_head};
+    a.tgt = KVPtr{static_cast<const __nv_bfloat16 *>(tgt->k), static_cast<const __nv_bfloat16 *>(tgt->v),
+                  tgt->stride_layer, tgt->stride_token, tgt->stride_head};
+    a.w_k = w_k; a.w_v = w_v; a.w_sl = w_stride_layer; a.w_sh = w_stride_head;
+    a.n_tokens = (int)src->n_tokens;
+    a.Lt = prob->Lt; a.Ht = prob->Ht; a.n_splits = 1;
+    a.src_layer = nullptr; a.src_head = nullptr; a.slots = nullptr; a.status = nullptr; a.compensated = 0;
+    FullHeadArgs f;
+    f.G = G; f.C = C;
+    f.layer_sets = static_cast<const int *>(workspace);
+    f.gi = f.layer_sets + (size_t)prob->Lt * prob->k;
+    f.gq = f.gi + NG;
+    f.src_head = f.gq + NG;
+    f.per_head = 1;
+    f.F = F; f.k = prob->k; f.Hs = prob->Hs; f.PF = F * prob->ds + 1; f.NG = NG; f.NC = F;
     if (launch_fullhead_tc(a, f, prob->ds, src, tgt, st) != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     return CB_OK;
 }

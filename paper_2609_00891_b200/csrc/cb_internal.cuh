@@ -57,7 +57,8 @@ struct ApplyArgs {
 struct FullHeadArgs {
     float *G, *C;
     const int *layer_sets, *gi, *gq;   // device
-    int F, k, Hs, PF, NG, NC;
+    const int *src_head;               // device [Ht]; used when per_head
+    int F, k, Hs, PF, NG, NC, per_head;
 };
 
 // Launchers (each returns the cudaError_t of its launch and bumps the launch counter on success).
@@ -68,6 +69,10 @@ cudaError_t launch_fullhead_tc(const AccumArgs &a, const FullHeadArgs &f, int d,
 cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, float *G, float *C, cudaStream_t st);
 cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long long n_tokens,
                          const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st);
+size_t solve_large_bytes_per_system(int P, int d);
+cudaError_t launch_solve_large(const float *G, const float *C, int n_maps, int P, int d, long long n_tokens,
+                               const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info,
+                               void *workspace, size_t workspace_bytes, cudaStream_t st);
 cudaError_t launch_apply_simt(const ApplyArgs &a, int d, cudaStream_t st);
 cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cudaStream_t st);
 

@@ -1,0 +1,337 @@
+// Batched ridge solve for regressors wider than one head (head-local support over k > 1 selected layers, Section 3.2:
+// P = k*d + 1 up to a few thousand), where a system no longer fits in shared memory.  Blocked right-looking Cholesky
+// and blocked substitutions in fp64 on a padded copy of every system in a caller-provided workspace:
+//   per block column J (64 wide): factor the diagonal block and solve the panel below it (one block per system),
+//   then update the trailing matrix with 64 x 64 tile products (one block per tile and system);
+//   forward and backward substitution alternate a diagonal-block solve with tile updates of the remaining rows.
+// Padding rows/columns carry an identity block, so every block step has the same shape.
+#include "cb_internal.cuh"
+
+namespace cb {
+
+static constexpr int LNB = 64;                 // block size
+static constexpr int LPAD = LNB + 2;           // shared-memory row pitch (doubles) of transposed tiles
+
+struct LgArgs {
+    double *A;        // [nsys][Pp][Pp] row-major; lower triangle becomes L
+    double *Z;        // [nsys][Pp][d]
+    int *fail;        // [nsys] first non-positive pivot (1-based) or 0
+    int Pp, P, d, nsys;
+};
+
+// ---- copy in: A = G + lambda_eff J (fp32 -> fp64), identity on the padding; Z = C -----------------------------------
+struct LgLoadArgs {
+    const float *G, *C;
+    int n_maps, sys0;
+    double inv_n;
+    unsigned flags;
+    float lambdas[16];
+};
+
+__global__ void __launch_bounds__(256) k_lg_load(LgArgs a, LgLoadArgs la)
+{
+    const int s = blockIdx.y, i = blockIdx.x;                 // system in the batch, row
+    const int sys = la.sys0 + s, li = sys / la.n_maps, m = sys % la.n_maps;
+    const float *Gm = la.G + (size_t)m * a.P * a.P;
+    const float *Cm = la.C + (size_t)m * a.P * a.d;
+    const double s_w = (double)Gm[(size_t)(a.P - 1) * a.P + (a.P - 1)];
+    const double lam = (la.flags & CB_FLAG_RAW_LAMBDA) ? (double)la.lambdas[li] : (double)la.lambdas[li] * s_w * la.inv_n;
+    double *Ar = a.A + ((size_t)s * a.Pp + i) * a.Pp;
+    double *Zr = a.Z + ((size_t)s * a.Pp + i) * a.d;
+    for (int j = threadIdx.x; j < a.Pp; j += blockDim.x) {
+        double v;
+        if (i < a.P && j < a.P) v = (double)Gm[(size_t)i * a.P + j] + ((i == j && i < a.P - 1) ? lam : 0.0);
+        else v = (i == j) ? 1.0 : 0.0;
+        Ar[j] = v;
+    }
+    for (int c = threadIdx.x; c < a.d; c += blockDim.x) Zr[c] = (i < a.P) ? (double)Cm[(size_t)i * a.d + c] : 0.0;
+    if (i == 0 && threadIdx.x == 0) a.fail[s] = 0;
+}
+
+// ---- block column J: factor A_JJ, then L_IJ = A_IJ L_JJ^-T for every row below -----------------------------------
+__global__ void __launch_bounds__(256, 1) k_lg_panel(LgArgs a, int J)
+{
+    __shared__ double Ld[LNB][LNB + 1];
+    __shared__ double rinv[LNB];
+    __shared__ int s_fail;
+    const int s = blockIdx.x, tid = threadIdx.x;
+    double *A = a.A + (size_t)s * a.Pp * a.Pp;
+    const int j0 = J * LNB;
+    if (tid == 0) s_fail = 0;
+    for (int e = tid; e < LNB * LNB; e += 256) {
+        const int r = e / LNB, c = e % LNB;
+        Ld[r][c] = (c <= r) ? A[(size_t)(j0 + r) * a.Pp + j0 + c] : 0.0;
+    }
+    __syncthreads();
+    for (int j = 0; j < LNB; ++j) {                            // unblocked right-looking Cholesky of the 64 x 64 block
+        if (tid == 0) {
+            double v = Ld[j][j];
+            if (!(v > 0.0)) { if (!s_fail) s_fail = j0 + j + 1; v = 1.0; }
+            const double ri = rsqrt(v);
+            Ld[j][j] = v * ri;
+            rinv[j] = ri;
+        }
+        __syncthreads();
+        const double ri = rinv[j];
+        for (int i = j + 1 + tid; i < LNB; i += 256) Ld[i][j] *= ri;
+        __syncthreads();
+        for (int e = tid; e < (LNB - j - 1) * (LNB - j - 1); e += 256) {
+            const int i = j + 1 + e / (LNB - j - 1), k = j + 1 + e % (LNB - j - 1);
+            if (k <= i) Ld[i][k] -= Ld[i][j] * Ld[k][j];
+        }
+        __syncthreads();
+    }
+    for (int e = tid; e < LNB * LNB; e += 256) {
+        const int r = e / LNB, c = e % LNB;
+        if (c <= r) A[(size_t)(j0 + r) * a.Pp + j0 + c] = Ld[r][c];
+    }
+    if (tid == 0 && s_fail && a.fail[s] == 0) a.fail[s] = s_fail;
+    // rows below the block: x L_JJ^T = a, one row per thread, the row held in registers
+    for (int i0 = j0 + LNB; i0 < a.Pp; i0 += 256) {
+        const int i = i0 + tid;
+        if (i >= a.Pp) continue;
+        double *row = A + (size_t)i * a.Pp + j0;
+        double x[LNB];
+#pragma unroll
+        for (int c = 0; c < LNB; c += 2) {
+            const double2 v = *reinterpret_cast<const double2 *>(row + c);
+            x[c] = v.x;
+            x[c + 1] = v.y;
+        }
+#pragma unroll
+        for (int c = 0; c < LNB; ++c) {
+            double v = x[c];
+#pragma unroll
+            for (int q = 0; q < c; ++q) v -= x[q] * Ld[c][q];
+            x[c] = v * rinv[c];
+        }
+#pragma unroll
+        for (int c = 0; c < LNB; c += 2) *reinterpret_cast<double2 *>(row + c) = make_double2(x[c], x[c + 1]);
+    }
+}
+
+// ---- tile products: Ctile[64 x NT] -= At[64 x 64] * Bt[64 x NT] ---------------------------------------------------
+// MODE 0 (trailing update of step J): C = A[I][I'], At = L[I][J], Bt^T = L[I'][J]      (I >= I' > J, NT = 64)
+// MODE 1 (forward substitution):      C = Z[I],     At = L[I][J], Bt = Z[J]            (I > J,  NT = d)
+// MODE 2 (backward substitution):     C = Z[I],     At = L[J][I]^T, Bt = Z[J]          (I < J,  NT = d)
+template <int MODE, int NT>
+__global__ void __launch_bounds__(256) k_lg_tile(LgArgs a, int J)
+{
+    extern __shared__ __align__(16) double lg_sm[];
+    double (*Ats)[LPAD] = reinterpret_cast<double (*)[LPAD]>(lg_sm);                       // [k][row]
+    double (*Bts)[NT + 2] = reinterpret_cast<double (*)[NT + 2]>(lg_sm + LNB * LPAD);      // [k][col]
+    const int s = blockIdx.y, tid = threadIdx.x;
+    double *A = a.A + (size_t)s * a.Pp * a.Pp;
+    double *Z = a.Z + (size_t)s * a.Pp * a.d;
+    const int nblk = a.Pp / LNB;
+    int I, I2 = 0;
+    if (MODE == 0) {
+        // blockIdx.x enumerates pairs (bi >= bj) of blocks below J
+        int p = blockIdx.x, bi = 0;
+        while (p >= bi + 1) { p -= bi + 1; ++bi; }
+        I = J + 1 + bi;
+        I2 = J + 1 + p;
+    } else if (MODE == 1) {
+        I = J + 1 + blockIdx.x;
+    } else {
+        I = blockIdx.x;
+    }
+    (void)nblk;
+    // load At transposed: Ats[k][r]
+    for (int e = tid; e < LNB * LNB; e += 256) {
+        const int r = e / LNB, k = e % LNB;
+        double v;
+        if (MODE == 2) v = A[(size_t)(J * LNB + k) * a.Pp + I * LNB + r];      // L[J][I]^T
+        else v = A[(size_t)(I * LNB + r) * a.Pp + J * LNB + k];
+        Ats[k][r] = v;
+    }
+    for (int e = tid; e < LNB * NT; e += 256) {
+        if (MODE == 0) {
+            const int c = e / LNB, k = e % LNB;
+            Bts[k][c] = A[(size_t)(I2 * LNB + c) * a.Pp + J * LNB + k];
+        } else {
+            const int k = e / NT, c = e % NT;
+            Bts[k][c] = Z[(size_t)(J * LNB + k) * a.d + c];
+        }
+    }
+    __syncthreads();
+    constexpr int CT = NT / 16;               // columns per thread
+    const int ty = tid >> 4, tx = tid & 15;
+    double acc[4][CT];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < CT; ++j) acc[i][j] = 0.0;
+#pragma unroll 4
+    for (int k = 0; k < LNB; ++k) {
+        double av[4], bv[CT];
+#pragma unroll
+        for (int i = 0; i < 4; i += 2) {
+            const double2 v = *reinterpret_cast<const double2 *>(&Ats[k][ty * 4 + i]);
+            av[i] = v.x; av[i + 1] = v.y;
+        }
+#pragma unroll
+        for (int j = 0; j < CT; j += 2) {
+            const double2 v = *reinterpret_cast<const double2 *>(&Bts[k][tx * CT + j]);
+            bv[j] = v.x; bv[j + 1] = v.y;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < CT; ++j) acc[i][j] += av[i] * bv[j];
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = I * LNB + ty * 4 + i;
+        double *crow = (MODE == 0) ? A + (size_t)r * a.Pp + I2 * LNB + tx * CT : Z + (size_t)r * a.d + tx * CT;
+#pragma unroll
+        for (int j = 0; j < CT; ++j) {
+            if (MODE == 0 && I == I2 && tx * CT + j > ty * 4 + i) continue;      // keep the diagonal tile lower-triangular
+            crow[j] -= acc[i][j];
+        }
+    }
+}
+
+// ---- diagonal-block solves of the substitutions: Z_J <- L_JJ^-1 Z_J (FWD) or L_JJ^-T Z_J ---------------------------
+template <bool FWD>
+__global__ void __launch_bounds__(128) k_lg_diag(LgArgs a, int J)
+{
+    extern __shared__ __align__(16) double lg_zs[];          // [LNB][d]: the block of right-hand sides being solved
+    __shared__ double Ld[LNB][LNB + 1];
+    __shared__ double rinv[LNB];
+    const int s = blockIdx.x, tid = threadIdx.x;
+    const double *A = a.A + (size_t)s * a.Pp * a.Pp;
+    double *Z = a.Z + (size_t)s * a.Pp * a.d;
+    const int j0 = J * LNB, d = a.d;
+    for (int e = tid; e < LNB * LNB; e += 128) {
+        const int r = e / LNB, c = e % LNB;
+        Ld[r][c] = (c <= r) ? A[(size_t)(j0 + r) * a.Pp + j0 + c] : 0.0;
+    }
+    for (int e = tid; e < LNB * d; e += 128) lg_zs[e] = Z[(size_t)j0 * d + e];
+    __syncthreads();
+    if (tid < LNB) rinv[tid] = 1.0 / Ld[tid][tid];
+    __syncthreads();
+    for (int c = tid; c < d; c += 128) {                   // one column per thread; only its own column is touched
+        if (FWD) {
+            for (int r = 0; r < LNB; ++r) {
+                double v0 = lg_zs[r * d + c], v1 = 0.0;
+                int q = 0;
+                for (; q + 1 < r; q += 2) { v0 -= Ld[r][q] * lg_zs[q * d + c]; v1 -= Ld[r][q + 1] * lg_zs[(q + 1) * d + c]; }
+                if (q < r) v0 -= Ld[r][q] * lg_zs[q * d + c];
+                lg_zs[r * d + c] = (v0 + v1) * rinv[r];
+            }
+        } else {
+            for (int r = LNB - 1; r >= 0; --r) {
+                double v0 = lg_zs[r * d + c], v1 = 0.0;
+                int q = LNB - 1;
+                for (; q - 1 > r; q -= 2) { v0 -= Ld[q][r] * lg_zs[q * d + c]; v1 -= Ld[q - 1][r] * lg_zs[(q - 1) * d + c]; }
+                if (q > r) v0 -= Ld[q][r] * lg_zs[q * d + c];
+                lg_zs[r * d + c] = (v0 + v1) * rinv[r];
+            }
+        }
+    }
+    __syncthreads();
+    for (int e = tid; e < LNB * d; e += 128) Z[(size_t)j0 * d + e] = lg_zs[e];
+}
+
+// ---- copy out: Wb = Z (fp32), info; failed systems are zero-filled -------------------------------------------------
+__global__ void __launch_bounds__(256) k_lg_store(LgArgs a, float *Wb, int *info, int sys0)
+{
+    const int s = blockIdx.y, i = blockIdx.x;
+    const int sys = sys0 + s;
+    const int f = a.fail[s];
+    const double *Zr = a.Z + ((size_t)s * a.Pp + i) * a.d;
+    float *Wr = Wb + ((size_t)sys * a.P + i) * a.d;
+    for (int c = threadIdx.x; c < a.d; c += blockDim.x) Wr[c] = f ? 0.f : (float)Zr[c];
+    if (i == 0 && threadIdx.x == 0) info[sys] = f;
+}
+
+template <int MODE, int NT>
+static cudaError_t launch_tile(const LgArgs &a, int J, dim3 grid, cudaStream_t st)
+{
+    constexpr size_t smem = sizeof(double) * (LNB * LPAD + LNB * (NT + 2));
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(k_lg_tile<MODE, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    k_lg_tile<MODE, NT><<<grid, 256, smem, st>>>(a, J);
+    return cudaSuccess;
+}
+
+size_t solve_large_bytes_per_system(int P, int d)
+{
+    const size_t Pp = ((size_t)P + LNB - 1) / LNB * LNB;
+    return sizeof(double) * (Pp * Pp + Pp * (size_t)d) + 256;
+}
+
+template <bool FWD>
+static void launch_diag(const LgArgs &a, int J, cudaStream_t st)
+{
+    const size_t smem = sizeof(double) * LNB * (size_t)a.d;
+    static bool attr = false;
+    if (!attr) {
+        cudaFuncSetAttribute(k_lg_diag<FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(double) * LNB * 128));
+        attr = true;
+    }
+    k_lg_diag<FWD><<<a.nsys, 128, smem, st>>>(a, J);
+}
+
+template <int NT>
+static void launch_subst_tiles(const LgArgs &a, int nblk, cudaStream_t st)
+{
+    for (int J = 0; J < nblk; ++J) {
+        launch_diag<true>(a, J, st);
+        if (J + 1 < nblk) launch_tile<1, NT>(a, J, dim3(nblk - 1 - J, a.nsys), st);
+    }
+    for (int J = nblk - 1; J >= 0; --J) {
+        launch_diag<false>(a, J, st);
+        if (J > 0) launch_tile<2, NT>(a, J, dim3(J, a.nsys), st);
+    }
+}
+
+cudaError_t launch_solve_large(const float *G, const float *C, int n_maps, int P, int d, long long n_tokens,
+                               const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info,
+                               void *workspace, size_t workspace_bytes, cudaStream_t st)
+{
+    const int Pp = (P + LNB - 1) / LNB * LNB, nblk = Pp / LNB;
+    const size_t per = solve_large_bytes_per_system(P, d);
+    const long long total = (long long)n_maps * n_lambda;
+    long long batch = (long long)(workspace_bytes / per);
+    if (batch < 1) return cudaErrorInvalidValue;
+    if (batch > total) batch = total;
+    if (batch > 65535) batch = 65535;
+    LgLoadArgs la;
+    la.G = G; la.C = C; la.n_maps = n_maps;
+    la.inv_n = n_tokens > 0 ? 1.0 / (double)n_tokens : 0.0;
+    la.flags = flags;
+    for (int i = 0; i < 16; ++i) la.lambdas[i] = i < n_lambda ? lambdas[i] : 0.f;
+    char *ws = static_cast<char *>(workspace);
+    int launches = 0;
+    for (long long sys0 = 0; sys0 < total; sys0 += batch) {
+        LgArgs a;
+        a.nsys = (int)((total - sys0 < batch) ? total - sys0 : batch);
+        a.A = reinterpret_cast<double *>(ws);
+        a.Z = a.A + (size_t)batch * Pp * Pp;
+        a.fail = reinterpret_cast<int *>(a.Z + (size_t)batch * Pp * d);
+        a.Pp = Pp; a.P = P; a.d = d;
+        la.sys0 = (int)sys0;
+        k_lg_load<<<dim3(Pp, a.nsys), 256, 0, st>>>(a, la);
+        for (int J = 0; J < nblk; ++J) {
+            k_lg_panel<<<a.nsys, 256, 0, st>>>(a, J);
+            const int r = nblk - 1 - J;
+            if (r > 0) launch_tile<0, LNB>(a, J, dim3(r * (r + 1) / 2, a.nsys), st);
+        }
+        if (d == 128) launch_subst_tiles<128>(a, nblk, st);
+        else launch_subst_tiles<64>(a, nblk, st);
+        k_lg_store<<<dim3(P, a.nsys), 256, 0, st>>>(a, Wb, info, (int)sys0);
+        launches += 2 + 2 * nblk + 4 * nblk;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    count_launch(launches);
+    return cudaSuccess;
+}
+
+}  // namespace cb

@@ -1,0 +1,84 @@
+"""Head-local support over k > 1 selected layers: statistics (tensor-core kernel, per-map groups) and the blocked
+large-system ridge solve, against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_00891_b200 import binding as cb
+from paper_2609_00891_b200 import synth
+from util import bits, rel_fro
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.mark.parametrize("name,k", [("mini_ragged", 2), ("mini_ragged", 3), ("mid_scaled", 2), ("tiny", 2)])
+def test_multilayer_statistics_and_fit(name, k):
+    wl = synth.workload(name)
+    sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    sets = oracle.fullhead_layer_sets(wl.Ls, wl.Lt, k)
+    law = synth.map_law(wl)
+    chunks = [synth.make_chunk(wl, c, sl, sh, law=law) for c in range(min(2, wl.n_chunks))]
+    n_tok = sum(ch["n_tokens"] for ch in chunks)
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
+    d = wl.d
+    P = k * d + 1
+    G = torch.zeros(wl.n_maps, P, P, device=DEV)
+    C = torch.zeros(wl.n_maps, P, d, device=DEV)
+    for ch in chunks:
+        t = {k_: v.to(DEV) for k_, v in ch.items() if torch.is_tensor(v)}
+        cb.cb_multilayer_stats_accumulate(prob, sh, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], t["w_k"], t["w_v"], G, C)
+    torch.cuda.synchronize()
+    lam = 1e-2
+    ws = torch.empty(cb.cb_ridge_solve_large_workspace_bytes(P, d, 5), dtype=torch.uint8, device=DEV)   # forces several batches
+    Wb = torch.full((1, wl.n_maps, P, d), float("nan"), device=DEV)
+    info = torch.full((1, wl.n_maps), -1, dtype=torch.int32, device=DEV)
+    cb.cb_ridge_solve_large(G, C, n_tok, [lam], 0, Wb, info, ws)
+    cb.cb_check_info(info)
+    Gc, Cc, Wc = G.cpu().numpy(), C.cpu().numpy(), Wb[0].cpu().numpy()
+    assert np.isfinite(Gc).all() and np.isfinite(Wc).all()
+    tol = 1e-3 if n_tok >= 4096 else 2e-3
+    for m in (0, wl.n_maps // 2 + 1, wl.n_maps - 1):
+        comp, l, h = m // (wl.Lt * wl.Ht), (m // wl.Ht) % wl.Lt, m % wl.Ht
+        Go = Co = None
+        for ch in chunks:
+            g, c = oracle.multilayer_stats(bits(ch["src_v" if comp else "src_k"]), bits(ch["tgt_v" if comp else "tgt_k"]),
+                                           (ch["w_v"] if comp else ch["w_k"])[l, h].contiguous().numpy(), l, h, int(sh[h]), sets[l])
+            Go, Co = (g, c) if Go is None else (Go + g, Co + c)
+        eg, ec = rel_fro(Gc[m], Go), rel_fro(Cc[m], Co)
+        To, io = oracle.ridge_solve_general(Go, Co, n_tok, lam)
+        ew = rel_fro(Wc[m], To)
+        # the solver itself, on the GPU's own statistics
+        Ts, _ = oracle.ridge_solve_general(Gc[m].astype(np.float64), Cc[m].astype(np.float64), n_tok, lam)
+        es = rel_fro(Wc[m], Ts)
+        print("%s k=%d map %d: rel err G %.2e C %.2e fit %.2e (solver alone %.2e)" % (name, k, m, eg, ec, ew, es))
+        assert io == 0 and eg <= tol and ec <= tol and es <= 1e-5
+        assert ew <= 5 * tol            # wider regressors amplify the statistics' rounding in the fit
+
+
+def test_large_solver_agrees_with_the_single_head_solver():
+    g = torch.Generator(device=DEV).manual_seed(1)
+    n_maps, d = 7, 128
+    P = d + 1
+    X = torch.randn(n_maps, 600, P, device=DEV, generator=g)
+    G = (X.transpose(1, 2) @ X).contiguous()
+    G[:, P - 1, P - 1] = 600.0
+    C = torch.randn(n_maps, P, d, device=DEV, generator=g)
+    lams = [1e-3, 1.0]
+    W1 = torch.empty(2, n_maps, P, d, device=DEV)
+    i1 = torch.empty(2, n_maps, dtype=torch.int32, device=DEV)
+    cb.cb_ridge_solve(G, C, 600, lams, 0, W1, i1)
+    ws = torch.empty(cb.cb_ridge_solve_large_workspace_bytes(P, d, 3), dtype=torch.uint8, device=DEV)
+    W2 = torch.empty_like(W1)
+    i2 = torch.empty_like(i1)
+    cb.cb_ridge_solve_large(G, C, 600, lams, 0, W2, i2, ws)
+    torch.cuda.synchronize()
+    assert not i1.any() and not i2.any()
+    assert ((W1 - W2).norm() / W1.norm()).item() < 1e-5
+    # a system without weight is reported, zero-filled, and does not disturb its neighbours
+    G[3] = 0
+    cb.cb_ridge_solve_large(G, C, 600, lams, 0, W2, i2, ws)
+    torch.cuda.synchronize()
+    assert (i2[:, 3] != 0).all() and not W2[:, 3].any() and not i2[:, [0, 1, 2, 4, 5, 6]].any()
+    assert torch.isfinite(W2).all()
