@@ -158,6 +158,9 @@ def main():
     ap.add_argument("--fullhead", type=int, default=0, metavar="CHUNKS",
                     help="time the full-head contrast statistics (config 3 shapes: 4 source layers x 8 heads per target "
                          "layer) on this many 50-sequence chunks and print its own JSON line")
+    ap.add_argument("--multilayer", type=int, default=0, metavar="K",
+                    help="time the head-local build over K selected layers per target layer (the paper's operating point is "
+                         "K = 8) on one 50-sequence chunk plus the wide ridge solve, and print its own JSON line")
     ap.add_argument("--profile-tokens", type=int, default=0,
                     help="profiling case: run only the accumulate kernel (3 launches) and the apply kernel on this many "
                          "tokens of the same shapes, print timings, no JSON line")
@@ -186,6 +189,9 @@ def main():
         return
     if args.fullhead > 0:
         fullhead_case(args, cb, synth, torch, wl, sl, sh, dev)
+        return
+    if args.multilayer > 0:
+        multilayer_case(args, cb, synth, torch, wl, sl, sh, dev)
         return
     prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, flags=args.flags, n_splits=args.splits)
     ctx = cb.cb_create(prob, device=dev)
@@ -360,6 +366,50 @@ def fullhead_case(args, cb, synth, torch, wl, sl, sh, dev):
                       "issued_mma_tflops": flops_issued / t / 1e12,
                       "frac_of_bf16_peak_dense": flops_dense / t / 1e12 / peaks["bf16_tflops"],
                       "s_per_200_sequences": 4 * statistics.mean(ms) / 1e3}))
+
+
+def multilayer_case(args, cb, synth, torch, wl, sl, sh, dev):
+    """Head-local support over K selected layers (regressor width K*128 + 1): statistics of one chunk and the solve."""
+    k = args.multilayer
+    sets = cb.cb_fullhead_layer_sets(wl.Ls, wl.Lt, k)
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
+    d = wl.d
+    P = k * d + 1
+    G = torch.zeros(wl.n_maps, P, P, device=dev)
+    C = torch.zeros(wl.n_maps, P, d, device=dev)
+    ch = synth.make_chunk(wl, 0, sl, sh, device=dev)
+    T = ch["n_tokens"]
+    ms = []
+    for _ in range(2):
+        G.zero_(); C.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        cb.cb_multilayer_stats_accumulate(prob, sh, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"], G, C)
+        e1.record()
+        e1.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    del ch
+    lams = list(wl.lambdas)
+    nsys = len(lams) * wl.n_maps
+    ws = torch.empty(cb.cb_ridge_solve_large_workspace_bytes(P, d, min(nsys, 1024)), dtype=torch.uint8, device=dev)
+    Wb = torch.empty(len(lams), wl.n_maps, P, d, device=dev)
+    info = torch.empty(len(lams), wl.n_maps, dtype=torch.int32, device=dev)
+    ts = []
+    for _ in range(2):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        cb.cb_ridge_solve_large(G, C, T, lams, 0, Wb, info, ws)
+        e1.record()
+        e1.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    cb.cb_check_info(info)
+    units = sum(i // 2 + 1 for i in range(k)) + k
+    print(json.dumps({"workload": "head-local over k=%d layers, 14B->32B shapes, P=%d, %d tokens" % (k, P, T),
+                      "stats_ms_per_chunk": ms, "stats_tokens_per_s": T / (min(ms) / 1e3),
+                      "issued_mma_tflops": 2.0 * wl.n_maps * units * T * 128 * 256 / (min(ms) / 1e3) / 1e12,
+                      "solve_ms_%d_systems" % nsys: ts,
+                      "solve_fp64_tflops": nsys * (P ** 3 / 3.0 + 2.0 * P * P * d) * 2 / (min(ts) / 1e3) / 1e12,
+                      "s_per_128000_positions": 2.5 * min(ms) / 1e3 + min(ts) / 1e3}))
 
 
 def profile_case(args, cb, synth, torch, wl, sl, sh, dev):
