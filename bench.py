@@ -403,8 +403,26 @@ def multilayer_case(args, cb, synth, torch, wl, sl, sh, dev):
         e1.synchronize()
         ts.append(e0.elapsed_time(e1))
     cb.cb_check_info(info)
+    # online apply latency at the paper's prefix lengths (and a long cache)
+    apply_ms = {}
+    law = synth.map_law(wl, dev)
+    for Tp in (128, 512, 1024, 32768):
+        src = synth.make_source_cache(wl, Tp, dev, law)
+        out_k = torch.empty(wl.Lt, Tp, wl.Ht, d, dtype=torch.bfloat16, device=dev)
+        out_v = torch.empty_like(out_k)
+        tt = []
+        for i in range(6):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            cb.cb_apply_multilayer(prob, sh, Wb[1], src[0], src[1], out_k, out_v)
+            e1.record()
+            e1.synchronize()
+            if i >= 2:
+                tt.append(e0.elapsed_time(e1))
+        apply_ms[str(Tp)] = statistics.median(tt)
+        del src, out_k, out_v
     units = sum(i // 2 + 1 for i in range(k)) + k
-    print(json.dumps({"workload": "head-local over k=%d layers, 14B->32B shapes, P=%d, %d tokens" % (k, P, T),
+    print(json.dumps({"apply_ms_by_prefix_tokens": apply_ms, "workload": "head-local over k=%d layers, 14B->32B shapes, P=%d, %d tokens" % (k, P, T),
                       "stats_ms_per_chunk": ms, "stats_tokens_per_s": T / (min(ms) / 1e3),
                       "issued_mma_tflops": 2.0 * wl.n_maps * units * T * 128 * 256 / (min(ms) / 1e3) / 1e12,
                       "solve_ms_%d_systems" % nsys: ts,

@@ -257,6 +257,18 @@ cb_status cb_multilayer_stats_accumulate(const cb_fullhead_problem *prob, const 
                                          float *G, float *C, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Online apply for the same support:  out[l][t][h][:] = sum_f x_f W_f + b  with x_f the row of source head src_head[h]
+ * of layer layer_sets[l][f] and W_f the f-th d x d block of the map's Wb [n_maps][k*d + 1][d] (bias row last).
+ * Outputs and strides as for cb_apply.  workspace: device, 256-byte aligned, cb_apply_multilayer_workspace_bytes()
+ * (the bf16 hi/lo image of all maps, rebuilt by every call).
+ */
+cb_status cb_apply_multilayer_workspace_bytes(const cb_fullhead_problem *prob, size_t *bytes);
+cb_status cb_apply_multilayer(const cb_fullhead_problem *prob, const int32_t *src_head, const float *Wb,
+                              const cb_kv_view *src_cache, void *tgt_k, void *tgt_v,
+                              int64_t t_stride_layer, int64_t t_stride_token, int64_t t_stride_head, int32_t out_dtype,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Synchronises the stream and reads the context's device status word: CB_OK, or CB_ERR_TIMEOUT if a bounded
  * wait inside a kernel ran out (the statistics are then invalid; reset before reuse).
  */

@@ -264,6 +264,15 @@ def multilayer_stats(src: np.ndarray, tgt: np.ndarray, w: np.ndarray, l: int, h:
     return G, C[0]
 
 
+def apply_multilayer(src: np.ndarray, Theta: np.ndarray, layer_set: Sequence[int], g: int):
+    """Affine apply for one map over several source layers: rows x_t = concat_f src[layer_set[f]][t][g] (bf16 bits,
+    widened exactly), y_t = x_t W + b in fp64 (a plain fp64 matrix product).  Returns (fp64 [T][d], bf16 bits)."""
+    X = np.concatenate([bf16_decode(np.ascontiguousarray(src[j, :, g, :])) for j in layer_set], axis=1)
+    Theta = np.asarray(Theta, dtype=np.float64)
+    y = X @ Theta[:-1] + Theta[-1]
+    return y, bf16_encode(y)
+
+
 def ridge_solve_general(G: np.ndarray, C: np.ndarray, n: int, lam: float, raw_lambda: bool = False):
     """Theta [p][dy] and info for one system of any width (bias entry last, not penalised)."""
     G = np.ascontiguousarray(G, dtype=np.float64)

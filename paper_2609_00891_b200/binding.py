@@ -27,7 +27,8 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_stats_reduce", "cb_ridge_solve",
            "cb_check_info", "cb_apply", "cb_device_status", "cb_stats_build_static", "cb_fullhead_layer_sets",
            "cb_fullhead_workspace_bytes", "cb_fullhead_stats_accumulate", "cb_ess_weights", "cb_ridge_solve_large_workspace_bytes", "cb_ridge_solve_large", "cb_multilayer_workspace_bytes",
-           "cb_multilayer_stats_accumulate", "cb_launch_count")
+           "cb_multilayer_stats_accumulate", "cb_apply_multilayer_workspace_bytes", "cb_apply_multilayer",
+           "cb_launch_count")
 
 
 class CbError(RuntimeError):
@@ -382,6 +383,23 @@ def cb_multilayer_stats_accumulate(prob: FullHeadProblem, src_head, src_k, src_v
                                                 ctypes.c_void_p(G.data_ptr()), ctypes.c_void_p(C.data_ptr()),
                                                 ctypes.c_void_p(ws.data_ptr()), ctypes.c_size_t(ws.numel()), _stream_ptr(stream)),
            "cb_multilayer_stats_accumulate")
+
+
+def cb_apply_multilayer(prob: FullHeadProblem, src_head, Wb: torch.Tensor, src_k, src_v, tgt_k, tgt_v, stream=None) -> None:
+    """Wb fp32 [n_maps][k*d + 1][d]; source cache [Ls][T][Hs][d] bf16; outputs [Lt][T][Ht][d] bf16 or fp32."""
+    sv = _kv_view(src_k, src_v)
+    sh = np.ascontiguousarray(src_head, dtype=np.int32)
+    assert Wb.dtype == torch.float32 and Wb.is_contiguous()
+    assert tgt_k.dtype == tgt_v.dtype and tgt_k.stride() == tgt_v.stride() and tgt_k.stride(3) == 1
+    dt = {torch.bfloat16: CB_DTYPE_BF16, torch.float32: CB_DTYPE_F32}[tgt_k.dtype]
+    n = ctypes.c_size_t(0)
+    _check(lib().cb_apply_multilayer_workspace_bytes(ctypes.byref(prob.c), ctypes.byref(n)), "cb_apply_multilayer_workspace_bytes")
+    ws = torch.empty(n.value, dtype=torch.uint8, device=Wb.device)
+    _check(lib().cb_apply_multilayer(ctypes.byref(prob.c), sh.ctypes.data_as(ctypes.c_void_p), ctypes.c_void_p(Wb.data_ptr()),
+                                     ctypes.byref(sv), ctypes.c_void_p(tgt_k.data_ptr()), ctypes.c_void_p(tgt_v.data_ptr()),
+                                     ctypes.c_int64(tgt_k.stride(0)), ctypes.c_int64(tgt_k.stride(1)), ctypes.c_int64(tgt_k.stride(2)),
+                                     dt, ctypes.c_void_p(ws.data_ptr()), ctypes.c_size_t(ws.numel()), _stream_ptr(stream)),
+           "cb_apply_multilayer")
 
 
 def cb_device_status(ctx: Context, stream=None) -> None:

@@ -569,6 +569,55 @@ cb_status cb_multilayer_stats_accumulate(const cb_fullhead_problem *prob, const 
     return CB_OK;
 }
 
+cb_status cb_apply_multilayer_workspace_bytes(const cb_fullhead_problem *prob, size_t *bytes)
+{
+    if (!prob || !bytes || prob->k <= 0 || prob->Lt <= 0 || prob->Ht <= 0 || (prob->ds != 64 && prob->ds != 128)) return CB_ERR_INVALID_ARG;
+    *bytes = apply_ml_workspace_bytes(2 * prob->Lt * prob->Ht, prob->k, prob->ds, prob->Lt);
+    return CB_OK;
+}
+
+cb_status cb_apply_multilayer(const cb_fullhead_problem *prob, const int32_t *src_head, const float *Wb,
+                              const cb_kv_view *src_cache, void *tgt_k, void *tgt_v,
+                              int64_t t_stride_layer, int64_t t_stride_token, int64_t t_stride_head, int32_t out_dtype,
+                              void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!prob || !prob->layer_sets || !src_head) return CB_ERR_INVALID_ARG;
+    if (prob->Ls <= 0 || prob->Hs <= 0 || prob->Lt <= 0 || prob->Ht <= 0 || prob->k <= 0 || prob->k > prob->Ls) return CB_ERR_INVALID_ARG;
+    if (prob->ds != prob->dt || (prob->ds != 64 && prob->ds != 128)) return CB_ERR_UNSUPPORTED;
+    if (prob->Lt > 128 || prob->Ht > 64) return CB_ERR_UNSUPPORTED;
+    for (int i = 0; i < prob->Lt * prob->k; ++i)
+        if (prob->layer_sets[i] < 0 || prob->layer_sets[i] >= prob->Ls) return CB_ERR_INVALID_ARG;
+    for (int h = 0; h < prob->Ht; ++h)
+        if (src_head[h] < 0 || src_head[h] >= prob->Hs) return CB_ERR_INVALID_ARG;
+    cb_status s = check_view(src_cache, prob->Ls, prob->Hs, prob->ds);
+    if (s != CB_OK) return s;
+    if (out_dtype != CB_DTYPE_BF16 && out_dtype != CB_DTYPE_F32) return CB_ERR_INVALID_ARG;
+    if (src_cache->n_tokens == 0) return CB_OK;
+    if (!Wb || !tgt_k || !tgt_v) return CB_ERR_INVALID_ARG;
+    if ((((uintptr_t)tgt_k | (uintptr_t)tgt_v | (uintptr_t)Wb) & 15)) return CB_ERR_INVALID_ARG;
+    if (t_stride_layer < 0 || t_stride_token <= 0 || t_stride_head < 0) return CB_ERR_INVALID_ARG;
+    if ((t_stride_layer | t_stride_token | t_stride_head) & 7) return CB_ERR_INVALID_ARG;
+    size_t need = 0;
+    cb_apply_multilayer_workspace_bytes(prob, &need);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return CB_ERR_WORKSPACE;
+    ApplyArgs a;
+    a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src_cache->k), static_cast<const __nv_bfloat16 *>(src_cache->v),
+                  src_cache->stride_layer, src_cache->stride_token, src_cache->stride_head};
+    a.Wb = Wb; a.out_k = tgt_k; a.out_v = tgt_v;
+    a.o_sl = t_stride_layer; a.o_st = t_stride_token; a.o_sh = t_stride_head;
+    a.out_dtype = out_dtype;
+    a.n_tokens = (int)src_cache->n_tokens;
+    a.Lt = prob->Lt; a.Ht = prob->Ht;
+    std::memset(a.src_layer, 0, sizeof a.src_layer);
+    std::memset(a.src_head, 0, sizeof a.src_head);
+    for (int h = 0; h < prob->Ht; ++h) a.src_head[h] = src_head[h];
+    if (launch_apply_ml_tc(a, prob->ds, prob->k, prob->layer_sets, src_cache, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return CB_ERR_CUDA;
+    }
+    return CB_OK;
+}
+
 cb_status cb_device_status(cb_ctx *ctx, void *stream)
 {
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;

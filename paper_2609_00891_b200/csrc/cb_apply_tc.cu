@@ -401,4 +401,313 @@ cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cu
     return e;
 }
 
+// =====================================================================================================================
+// Apply for the head-local support over k > 1 selected layers:  out[t] = sum_f x_f[t] W_f + b, where x_f is source
+// head a(h) of layer S_l[f] and W_f the f-th d x d block of the map.  W is split into bf16 hi + lo and laid out for the
+// tensor core once by a preparation kernel (into the caller's workspace); the main kernel streams, per 128-token tile
+// and per f, the source tile (TMA) and the W block (one bulk copy) through a two-stage ring and accumulates all k
+// products in one tensor-memory accumulator before the epilogue.
+// =====================================================================================================================
+template <int D>
+struct MlCfg {
+    static constexpr int TT = 128;
+    static constexpr int NB = D / 64;
+    static constexpr int XBLK = TT * 128;
+    static constexpr int X_BYTES = NB * XBLK;
+    static constexpr int WBLK = D * 128;
+    static constexpr int W_BYTES = NB * WBLK;            // hi (or lo)
+    static constexpr int STAGE = X_BYTES + 2 * W_BYTES;  // source tile + W block (hi, lo)
+    static constexpr int O_BYTES = NB * XBLK;
+    static constexpr int NS = 2, NACC = 2;
+    static constexpr int TMEM_COLS = (NACC * D < 32) ? 32 : NACC * D;
+    static constexpr int EPI_WARPS = 4;
+    static constexpr int THREADS = (2 + EPI_WARPS) * 32;
+    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * STAGE + O_BYTES + 256;
+};
+
+struct MlParams {
+    CUtensorMap src_k, src_v, out_k, out_v;
+    ApplyArgs a;                 // src_layer / src_head arrays unused except src_head
+    const uint8_t *wsplit;       // [n_maps][k][hi | lo][W_BYTES]
+    const int *layer_sets;       // device [Lt][k]
+    int k, n_splits;
+};
+
+// One block per (map, f): split the f-th d x d block of W into bf16 hi + lo in the swizzled MN-major layout.
+template <int D>
+__global__ void __launch_bounds__(256) k_w_split(const float *__restrict__ Wb, uint8_t *__restrict__ wsplit, int k)
+{
+    using C = MlCfg<D>;
+    const int m = blockIdx.x / k, f = blockIdx.x % k;
+    const float *Wm = Wb + ((size_t)m * (k * D + 1) + (size_t)f * D) * D;
+    uint8_t *dst = wsplit + ((size_t)m * k + f) * 2 * C::W_BYTES;
+    for (int i = threadIdx.x; i < D * (D / 8); i += 256) {
+        const int kk = i / (D / 8), n0 = (i % (D / 8)) * 8;
+        const float4 f0 = __ldg(reinterpret_cast<const float4 *>(Wm + (size_t)kk * D + n0));
+        const float4 f1 = __ldg(reinterpret_cast<const float4 *>(Wm + (size_t)kk * D + n0 + 4));
+        const float v[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+        unsigned hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            hi[e] = ap_pack_bf16x2(v[2 * e], v[2 * e + 1]);
+            lo[e] = ap_pack_bf16x2(v[2 * e] - __uint_as_float(hi[e] << 16), v[2 * e + 1] - __uint_as_float(hi[e] & 0xffff0000u));
+        }
+        const int off = (n0 >> 6) * C::WBLK + kk * 128 + ((((n0 & 63) >> 3) ^ (kk & 7)) << 4);
+        *reinterpret_cast<uint4 *>(dst + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4 *>(dst + C::W_BYTES + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __grid_constant__ MlParams P)
+{
+    using C = MlCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *st_base = smem;                                // [NS][X | Whi | Wlo]
+    uint8_t *os = st_base + (size_t)C::NS * C::STAGE;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(os + C::O_BYTES);
+    uint64_t *sfull = bars, *sempty = sfull + C::NS;
+    uint64_t *accfull = sempty + C::NS, *accempty = accfull + C::NACC;
+    uint64_t *owritten = accempty + C::NACC, *ofree = owritten + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ofree + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const ApplyArgs &a = P.a;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_maps = 2 * a.Lt * a.Ht, k = P.k;
+    const int n_units = n_maps * P.n_splits;
+    const int n_tiles = (a.n_tokens + C::TT - 1) / C::TT;
+    const bool out_bf16 = a.out_dtype == CB_DTYPE_BF16;
+
+    if (tid == 0) {
+        for (int i = 0; i < C::NS; ++i) { mbar_init(&sfull[i], 1); mbar_init(&sempty[i], 1); }
+        for (int i = 0; i < C::NACC; ++i) { mbar_init(&accfull[i], 1); mbar_init(&accempty[i], C::EPI_WARPS); }
+        mbar_init(owritten, C::EPI_WARPS);
+        mbar_init(ofree, 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
+        tma_prefetch_desc(&P.out_k); tma_prefetch_desc(&P.out_v);
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {          // producer: source tile and W block of every (tile, f)
+            ApIter cur;
+            cur.start(n_units, n_maps, n_tiles, P.n_splits);
+            ApRing<C::NS> st;
+            while (cur.u < n_units) {
+                const int m = cur.m;
+                const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
+                const CUtensorMap *map = comp ? &P.src_v : &P.src_k;
+                const int g = a.src_head[h];
+                const uint8_t *wm = P.wsplit + (size_t)m * k * 2 * C::W_BYTES;
+                for (int tile = cur.tile; tile < cur.tile1; ++tile)
+                    for (int f = 0; f < k; ++f) {
+                        if (!mbar_wait(&sempty[st.idx], st.phase ^ 1, abort_flag)) goto ml_teardown;
+                        uint8_t *dst = st_base + (size_t)st.idx * C::STAGE;
+                        mbar_arrive_expect_tx(&sfull[st.idx], C::STAGE);
+                        tma_load_5d(dst, map, &sfull[st.idx], 0, tile * C::TT, 0, g, P.layer_sets[l * k + f]);
+                        bulk_load(dst + C::X_BYTES, wm + (size_t)f * 2 * C::W_BYTES, 2 * C::W_BYTES, &sfull[st.idx]);
+                        st.next();
+                    }
+                cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {          // MMA issuer
+            constexpr uint32_t idesc = umma_idesc_bf16(128, D, false, true);
+            const uint64_t proto_a = umma_smem_desc_sw128(0, 16, 1024);
+            const uint64_t proto_b = umma_smem_desc_sw128(0, C::WBLK, 1024);
+            const uint32_t a_hi32 = (uint32_t)(proto_a >> 32), b_hi32 = (uint32_t)(proto_b >> 32);
+            const uint32_t a_lo0 = (uint32_t)proto_a | ((smem_u32(st_base) & 0x3FFFFu) >> 4);
+            const uint32_t b_lo0 = (uint32_t)proto_b | ((smem_u32(st_base + C::X_BYTES) & 0x3FFFFu) >> 4);
+            ApIter cur;
+            cur.start(n_units, n_maps, n_tiles, P.n_splits);
+            ApRing<C::NS> st;
+            ApRing<C::NACC> ac;
+            while (cur.u < n_units) {
+                for (int tile = cur.tile; tile < cur.tile1; ++tile) {
+                    if (!mbar_wait(&accempty[ac.idx], ac.phase ^ 1, abort_flag)) goto ml_teardown;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + ac.idx * D;
+                    for (int f = 0; f < k; ++f) {
+                        if (!mbar_wait(&sfull[st.idx], st.phase, abort_flag)) goto ml_teardown;
+                        tc_fence_after();
+                        const uint32_t al = a_lo0 + st.idx * (C::STAGE >> 4);
+                        const uint32_t bl = b_lo0 + st.idx * (C::STAGE >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint64_t ad = ((uint64_t)a_hi32 << 32) | (al + (kk >> 2) * (C::XBLK >> 4) + (kk & 3) * 2);
+                            umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bl + kk * 128), idesc, (f == 0 && kk == 0) ? 0u : 1u);
+                            umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bl + (C::W_BYTES >> 4) + kk * 128), idesc, 1u);
+                        }
+                        umma_commit(&sempty[st.idx]);
+                        st.next();
+                    }
+                    umma_commit(&accfull[ac.idx]);
+                    ac.next();
+                }
+                cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
+            }
+        }
+    } else {
+        // epilogue warps: tensor memory -> + bias -> bf16 tile -> TMA store (or fp32 stored directly)
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        ApIter cur;
+        cur.start(n_units, n_maps, n_tiles, P.n_splits);
+        ApRing<C::NACC> ac;
+        uint32_t oc = 0;
+        const bool storer = (warp == 2 && lane == 0);
+        while (cur.u < n_units) {
+            const int m = cur.m;
+            const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
+            const CUtensorMap *omap = comp ? &P.out_v : &P.out_k;
+            const float *bias = a.Wb + ((size_t)m * (k * D + 1) + (size_t)k * D) * D;     // last row of the map
+            for (int tile = cur.tile; tile < cur.tile1; ++tile) {
+                if (!mbar_wait_warp(&accfull[ac.idx], ac.phase, abort_flag, lane)) goto ml_teardown;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ac.idx * D;
+                const int tok = tile * C::TT + row;
+                if (out_bf16) {
+                    if (!mbar_wait_warp(ofree, (oc & 1) ^ 1, abort_flag, lane)) goto ml_teardown;
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_32x32(taddr + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            const int n0 = c * 32 + v * 8;
+                            const float4 b0 = __ldg(reinterpret_cast<const float4 *>(bias + n0));
+                            const float4 b1 = __ldg(reinterpret_cast<const float4 *>(bias + n0 + 4));
+                            uint4 pk;
+                            pk.x = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 0]) + b0.x, __uint_as_float(r[v * 8 + 1]) + b0.y);
+                            pk.y = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 2]) + b0.z, __uint_as_float(r[v * 8 + 3]) + b0.w);
+                            pk.z = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 4]) + b1.x, __uint_as_float(r[v * 8 + 5]) + b1.y);
+                            pk.w = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 6]) + b1.z, __uint_as_float(r[v * 8 + 7]) + b1.w);
+                            const int blk = n0 >> 6, chunk = (n0 & 63) >> 3;
+                            *reinterpret_cast<uint4 *>(os + blk * C::XBLK + row * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
+                        }
+                    }
+                    tc_fence_before();
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) { mbar_arrive(&accempty[ac.idx]); mbar_arrive(owritten); }
+                    if (storer && mbar_wait(owritten, oc & 1, abort_flag)) {
+                        tma_store_5d(omap, os, 0, tile * C::TT, 0, h, l);
+                        tma_store_commit();
+                        tma_store_wait_read();
+                        mbar_arrive(ofree);
+                    }
+                    ++oc;
+                } else {
+                    float *orow = reinterpret_cast<float *>(comp ? a.out_v : a.out_k) +
+                                  (long long)l * a.o_sl + (long long)tok * a.o_st + (long long)h * a.o_sh;
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_32x32(taddr + c * 32, r);
+                        tmem_wait_ld();
+                        if (tok < a.n_tokens) {
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) {
+                                const int n0 = c * 32 + v * 4;
+                                const float4 b0 = __ldg(reinterpret_cast<const float4 *>(bias + n0));
+                                *reinterpret_cast<float4 *>(orow + n0) =
+                                    make_float4(__uint_as_float(r[v * 4 + 0]) + b0.x, __uint_as_float(r[v * 4 + 1]) + b0.y,
+                                                __uint_as_float(r[v * 4 + 2]) + b0.z, __uint_as_float(r[v * 4 + 3]) + b0.w);
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&accempty[ac.idx]);
+                }
+                ac.next();
+            }
+            cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
+        }
+        if (storer) tma_store_wait_all();
+    }
+
+ml_teardown:
+    __syncwarp();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+size_t apply_ml_workspace_bytes(int n_maps, int k, int d, int Lt)
+{
+    return (size_t)n_maps * k * 2 * (size_t)d * d * 2 + ((sizeof(int) * (size_t)Lt * k + 255) / 256) * 256;
+}
+
+template <int D>
+static cudaError_t launch_ml(const MlParams &P, const float *Wb, uint8_t *wsplit, cudaStream_t st)
+{
+    using C = MlCfg<D>;
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(k_apply_ml_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    const int n_maps = 2 * P.a.Lt * P.a.Ht;
+    k_w_split<D><<<n_maps * P.k, 256, 0, st>>>(Wb, wsplit, P.k);
+    const int n_units = n_maps * P.n_splits;
+    const int grid = n_units < ap_sm_count() ? n_units : ap_sm_count();
+    k_apply_ml_tc<D><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_apply_ml_tc(const ApplyArgs &a, int d, int k, const int *layer_sets_host, const cb_kv_view *src,
+                               void *workspace, cudaStream_t st)
+{
+    MlParams P;
+    P.a = a;
+    P.k = k;
+    const int TT = 128;
+    const int n_maps = 2 * a.Lt * a.Ht;
+    const int n_tiles = (a.n_tokens + TT - 1) / TT;
+    int splits = (n_maps >= ap_sm_count()) ? 1 : (ap_sm_count() + n_maps - 1) / n_maps;
+    if (splits > n_tiles) splits = n_tiles;
+    if (splits < 1) splits = 1;
+    P.n_splits = splits;
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    const size_t wbytes = (size_t)n_maps * k * 2 * (size_t)d * d * 2;
+    P.wsplit = ws;
+    P.layer_sets = reinterpret_cast<const int *>(ws + wbytes);
+    cudaError_t e = cudaMemcpyAsync(ws + wbytes, layer_sets_host, sizeof(int) * (size_t)a.Lt * k, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return e;
+    if (!make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
+                            src->stride_token, src->stride_layer, TT) ||
+        !make_kv_tensor_map(&P.src_v, src->v, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
+                            src->stride_token, src->stride_layer, TT))
+        return cudaErrorInvalidValue;
+    if (a.out_dtype == CB_DTYPE_BF16) {
+        if (!make_kv_tensor_map(&P.out_k, a.out_k, d, a.Ht, a.n_tokens, a.Lt, a.o_sh, a.o_st, a.o_sl, TT) ||
+            !make_kv_tensor_map(&P.out_v, a.out_v, d, a.Ht, a.n_tokens, a.Lt, a.o_sh, a.o_st, a.o_sl, TT))
+            return cudaErrorInvalidValue;
+    } else {
+        P.out_k = P.src_k;
+        P.out_v = P.src_v;
+    }
+    e = (d == 128) ? launch_ml<128>(P, a.Wb, ws, st) : launch_ml<64>(P, a.Wb, ws, st);
+    if (e == cudaSuccess) count_launch(2);
+    return e;
+}
+
 }  // namespace cb

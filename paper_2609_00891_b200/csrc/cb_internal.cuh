@@ -76,6 +76,10 @@ cudaError_t launch_solve_large(const float *G, const float *C, int n_maps, int P
 cudaError_t launch_apply_simt(const ApplyArgs &a, int d, cudaStream_t st);
 cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cudaStream_t st);
 
+size_t apply_ml_workspace_bytes(int n_maps, int k, int d, int Lt);
+cudaError_t launch_apply_ml_tc(const ApplyArgs &a, int d, int k, const int *layer_sets_host, const cb_kv_view *src,
+                               void *workspace, cudaStream_t st);
+
 void count_launch(int n = 1);
 
 }  // namespace cb

@@ -85,3 +85,39 @@ def test_large_solver_agrees_with_the_single_head_solver():
     torch.cuda.synchronize()
     assert (i2[:, 3] != 0).all() and not W2[:, 3].any() and not i2[:, [0, 1, 2, 4, 5, 6]].any()
     assert torch.isfinite(W2).all()
+
+
+@pytest.mark.parametrize("name,k,T", [("mini_ragged", 2, 333), ("deep_small", 8, 700), ("tiny", 2, 129)])
+def test_multilayer_apply(name, k, T):
+    wl = synth.workload(name)
+    sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    sets = oracle.fullhead_layer_sets(wl.Ls, wl.Lt, k)
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
+    d = wl.d
+    P = k * d + 1
+    rng = np.random.default_rng(7)
+    Th = (rng.standard_normal((wl.n_maps, P, d)) / np.sqrt(k * d)).astype(np.float32)
+    src = synth.make_source_cache(wl, T)
+    for dtype in (torch.float32, torch.bfloat16):
+        out_k = torch.zeros(wl.Lt, T, wl.Ht, d, dtype=dtype, device=DEV)
+        out_v = torch.zeros_like(out_k)
+        cb.cb_apply_multilayer(prob, sh, torch.from_numpy(Th).to(DEV), src[0].to(DEV), src[1].to(DEV), out_k, out_v)
+        torch.cuda.synchronize()
+        for m in (0, wl.n_maps // 2 + 1, wl.n_maps - 1):
+            comp, l, h = m // (wl.Lt * wl.Ht), (m // wl.Ht) % wl.Lt, m % wl.Ht
+            y, yb = oracle.apply_multilayer(bits(src[comp]), Th[m].astype(np.float64), sets[l], int(sh[h]))
+            got = (out_v if comp else out_k)[l, :, h].float().cpu().numpy()
+            if dtype == torch.float32:
+                assert rel_fro(got, y) <= 1e-5
+            else:
+                assert rel_fro(got, oracle.bf16_decode(yb)) <= 2e-3
+    # block-identity map (first layer's block = I, others 0) returns the first selected layer's head bit for bit
+    I = np.zeros((wl.n_maps, P, d), np.float32)
+    I[:, :d] = np.eye(d)
+    ob_k = torch.zeros(wl.Lt, T, wl.Ht, d, dtype=torch.bfloat16, device=DEV)
+    ob_v = torch.zeros_like(ob_k)
+    cb.cb_apply_multilayer(prob, sh, torch.from_numpy(I).to(DEV), src[0].to(DEV), src[1].to(DEV), ob_k, ob_v)
+    for l in range(wl.Lt):
+        for h in range(wl.Ht):
+            assert torch.equal(ob_k[l, :, h].cpu(), src[0][sets[l][0], :, sh[h]])
+            assert torch.equal(ob_v[l, :, h].cpu(), src[1][sets[l][0], :, sh[h]])
