@@ -17,7 +17,10 @@
  * scaling, equality with the centred two-pass estimator of Eq. "closedform",
  * textbook least squares for constant weights, exact recovery of (A, b),
  * identity recovery for X = Y, the effective-dimension bound, the coefficient
- * counts of Section 3.2 and the storage figures of Section 4.4.
+ * counts of Section 3.2 and the storage figures of Section 4.4; the full-head
+ * and multi-layer statistics against a library matrix product on gathered
+ * features; the general-width solve by exact recovery and its residual; the
+ * ESS floor by the Kish identity and the floors printed in Section 4.1.
  * Parity unpinned by the paper (defined by this build, not by the paper): the
  * synthetic input laws, the nearest-depth single-layer match (k = 1), and the
  * lambda_eff = lambda * s_w / n convention for weights that are not mean-one.

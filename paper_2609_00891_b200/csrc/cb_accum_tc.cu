@@ -387,12 +387,14 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                         tc_fence_after();
                         const uint32_t bl = b_lo0 + st.idx * (C::STAGE_BYTES >> 4);
                         const uint32_t al = a_lo0 + ar.idx * ((C::A_PARTS * C::A_BYTES) >> 4);
+#ifndef CB_ABLATE_MMA
 #pragma unroll
                         for (int k = 0; k < C::TT / 16; ++k) {
                             const uint64_t bd = ((uint64_t)desc_hi << 32) | (bl + k * 128);
                             umma_bf16_ss(d_tmem, ((uint64_t)desc_hi << 32) | (al + k * 128), bd, idesc, k == 0 ? accum : 1u);
                             if (COMP) umma_bf16_ss(d_tmem, ((uint64_t)desc_hi << 32) | (al + (C::A_BYTES >> 4) + k * 128), bd, idesc, 1u);
                         }
+#endif
                         accum = 1;
                         umma_commit(&empty[st.idx]);     // frees the stage and (through it) the weighted-operand buffer
                         CB_TR(it, 4);
@@ -437,6 +439,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                 const uint8_t *xs = xy + st.idx * C::STAGE_BYTES + C::AS_OFF + off0;          // rows to be weighted
                 const uint8_t *ys = xy + st.idx * C::STAGE_BYTES + C::NBX * C::BLK + off0;    // B2: summed with the weights
                 uint8_t *ah = ab + ar.idx * (C::A_PARTS * C::A_BYTES) + off0;
+#ifndef CB_ABLATE_FOLD
 #pragma unroll
                 for (int i = 0; i < C::RPT; ++i) {
                     const int off = i * C::RG * 128;
@@ -462,6 +465,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                     for (int e = 0; e < 4; ++e) sy2[e] = f2_fma(w2, f2_from_bf16x2(yu[e]), sy2[e]);
                     if (cc == 0) sw += wt;
                 }
+#endif
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&afull[ar.idx]); mbar_arrive(&empty[st.idx]); }
