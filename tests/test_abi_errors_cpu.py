@@ -1,0 +1,89 @@
+"""Error behaviour of the device entry points that can be checked without a GPU: argument errors are status codes
+found on the host before anything is launched, and without a CUDA device the calls fail loudly (no CPU fallback)."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_00891_b200 import binding as cb
+from paper_2609_00891_b200 import build as cb_build
+
+pytestmark = pytest.mark.skipif(torch.cuda.is_available(), reason="host-only behaviour; the GPU suite covers the rest")
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    cb_build.build()
+
+
+def _view(L, H, d, T, ptr=0x1000, st=None, sh=None, sl=None):
+    st = H * d if st is None else st
+    sh = d if sh is None else sh
+    sl = T * H * d if sl is None else sl
+    return cb._KvView(ptr, ptr, L, H, d, T, sl, st, sh)
+
+
+def _apply(prob, view, Wb=0x2000, out=0x3000, strides=None, dtype=cb.CB_DTYPE_BF16):
+    s = strides or (view.n_tokens * prob.Ht * prob.dt, prob.Ht * prob.dt, prob.dt)
+    return cb.lib().cb_apply(ctypes.byref(prob.c), ctypes.c_void_p(Wb), ctypes.byref(view), ctypes.c_void_p(out),
+                             ctypes.c_void_p(out), ctypes.c_int64(s[0]), ctypes.c_int64(s[1]), ctypes.c_int64(s[2]),
+                             dtype, ctypes.c_void_p(0))
+
+
+def test_apply_argument_errors_are_reported_before_any_launch():
+    sl, sh = cb.cb_head_map_nearest(4, 2, 6, 2)
+    prob = cb.Problem(4, 2, 128, 6, 2, 128, sl, sh)
+    before = cb.cb_launch_count()
+    assert _apply(prob, _view(4, 2, 128, 0)) == cb.CB_OK                              # empty cache: no-op
+    assert _apply(prob, _view(5, 2, 128, 64)) == cb.CB_ERR_INVALID_ARG               # wrong layer count
+    assert _apply(prob, _view(4, 2, 128, 64, ptr=0x1004)) == cb.CB_ERR_INVALID_ARG   # misaligned cache pointer
+    assert _apply(prob, _view(4, 2, 128, 64, st=2 * 128 + 4)) == cb.CB_ERR_INVALID_ARG   # stride not a multiple of 8
+    assert _apply(prob, _view(4, 2, 128, 64), Wb=0) == cb.CB_ERR_INVALID_ARG         # null maps
+    assert _apply(prob, _view(4, 2, 128, 64), out=0x3008) == cb.CB_ERR_INVALID_ARG   # misaligned output
+    assert _apply(prob, _view(4, 2, 128, 64), dtype=7) == cb.CB_ERR_INVALID_ARG      # unknown output type
+    assert _apply(prob, _view(4, 2, 128, 1 << 31)) == cb.CB_ERR_UNSUPPORTED          # too many rows for one call
+    assert cb.cb_launch_count() == before
+
+
+def test_solve_argument_errors():
+    lam = np.array([1e-2], np.float32)
+    call = lambda G, C, n_maps, d, n, nl, Wb, info: cb.lib().cb_ridge_solve(
+        ctypes.c_void_p(G), ctypes.c_void_p(C), n_maps, d, ctypes.c_int64(n), lam.ctypes.data_as(ctypes.c_void_p), nl,
+        ctypes.c_uint32(0), ctypes.c_void_p(Wb), ctypes.c_void_p(info), ctypes.c_void_p(0))
+    assert call(0, 0x10, 4, 128, 100, 1, 0x20, 0x30) == cb.CB_ERR_INVALID_ARG
+    assert call(0x10, 0x10, 4, 96, 100, 1, 0x20, 0x30) == cb.CB_ERR_UNSUPPORTED
+    assert call(0x10, 0x10, 4, 128, 100, 0, 0x20, 0x30) == cb.CB_ERR_INVALID_ARG
+    assert call(0x10, 0x10, 0, 128, 100, 1, 0x20, 0x30) == cb.CB_OK                   # no systems: nothing to do
+    bad = np.array([-1.0], np.float32)
+    assert cb.lib().cb_ridge_solve(ctypes.c_void_p(0x10), ctypes.c_void_p(0x10), 4, 128, ctypes.c_int64(10),
+                                   bad.ctypes.data_as(ctypes.c_void_p), 1, ctypes.c_uint32(0), ctypes.c_void_p(0x20),
+                                   ctypes.c_void_p(0x30), ctypes.c_void_p(0)) == cb.CB_ERR_INVALID_ARG
+
+
+def test_without_a_device_the_path_fails_loudly():
+    sl, sh = cb.cb_head_map_nearest(2, 2, 2, 2)
+    prob = cb.Problem(2, 2, 64, 2, 2, 64, sl, sh)
+    h = ctypes.c_void_p()
+    ws = np.zeros(cb.cb_workspace_bytes(prob) + 256, np.uint8)
+    addr = (ws.ctypes.data + 255) // 256 * 256
+    st = cb.lib().cb_create(ctypes.byref(prob.c), ctypes.c_void_p(addr), ctypes.c_size_t(cb.cb_workspace_bytes(prob)), ctypes.byref(h))
+    assert st == cb.CB_ERR_CUDA and not h                                            # no context, no fallback
+    assert _apply(prob, _view(2, 2, 64, 64)) == cb.CB_ERR_CUDA
+    assert "CUDA" in cb.status_string(cb.CB_ERR_CUDA)
+    with pytest.raises(cb.CbError):
+        cb.cb_create(prob, workspace=torch.zeros(16, dtype=torch.uint8))              # workspace too small
+
+
+def test_workspace_and_static_limits():
+    sl, sh = cb.cb_head_map_nearest(40, 8, 64, 8)
+    prob = cb.Problem(40, 8, 128, 64, 8, 128, sl, sh)
+    v_s, v_t = _view(40, 8, 128, 64), _view(64, 8, 128, 64)
+    st = cb.lib().cb_stats_build_static(ctypes.byref(prob.c), ctypes.byref(v_s), ctypes.byref(v_t), ctypes.c_void_p(0x100),
+                                        ctypes.c_void_p(0x100), ctypes.c_int64(8 * 64), ctypes.c_int64(64),
+                                        ctypes.c_void_p(0x200), ctypes.c_void_p(0x300), ctypes.c_void_p(0))
+    assert st == cb.CB_ERR_STATIC_LIMIT
+    n = ctypes.c_size_t(0)
+    assert cb.lib().cb_ridge_solve_large_workspace_bytes(1025, 128, ctypes.c_int64(1), ctypes.byref(n)) == cb.CB_OK
+    assert n.value >= 8 * (1088 * 1088 + 1088 * 128)
+    assert cb.lib().cb_ridge_solve_large_workspace_bytes(1025, 100, ctypes.c_int64(1), ctypes.byref(n)) == cb.CB_ERR_INVALID_ARG
