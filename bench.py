@@ -29,6 +29,14 @@ ALG_BYTES_PER_TOKEN = 2 * 40 * 8 * 128 * 2 + 2 * 64 * 8 * 128 * 2 + 2 * 64 * 8 *
 ALG_FLOPS_PER_TOKEN = 1024 * 2 * 129 * 257                                           # dense p x (2d+1) contraction per map
 
 
+def algorithmic_work(wl):
+    """(bytes, flops) per calibration token: every source element, target element and weight once; the dense
+    (d+1) x (2d+1) contraction per map."""
+    b = 2 * wl.Ls * wl.Hs * wl.d * 2 + 2 * wl.Lt * wl.Ht * wl.d * 2 + 2 * wl.Lt * wl.Ht * 4
+    f = wl.n_maps * 2 * (wl.d + 1) * (2 * wl.d + 1)
+    return b, f
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -155,6 +163,9 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--flags", type=int, default=0)
     ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--workload", default=WORKLOAD,
+                    help="synthetic workload (default: the 500-sequence 14B->32B build the metric is quoted on; "
+                         "qwen8b_14b and ragged_long are the other head-local configurations)")
     ap.add_argument("--fullhead", type=int, default=0, metavar="CHUNKS",
                     help="time the full-head contrast statistics (config 3 shapes: 4 source layers x 8 heads per target "
                          "layer) on this many 50-sequence chunks and print its own JSON line")
@@ -181,7 +192,8 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = synth.workload(WORKLOAD)
+    wl = synth.workload(args.workload)
+    alg_bytes, alg_flops = algorithmic_work(wl)
     n_chunks = args.chunks if args.chunks > 0 else wl.n_chunks
     sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     if args.profile_tokens > 0:
@@ -266,11 +278,11 @@ def main():
     # ---- online apply (reported beside the build, not part of the step) ----
     apply_info = None
     if rank == 0:
-        T = 32768
+        T = wl.apply_tokens or 32768
         src = synth.make_source_cache(wl, T, dev, law)
         out_k = torch.empty(wl.Lt, T, wl.Ht, d, dtype=torch.bfloat16, device=dev)
         out_v = torch.empty_like(out_k)
-        Wfull = full[1].contiguous()
+        Wfull = full[min(1, nl - 1)].contiguous()
         for _ in range(3):
             cb.cb_apply(prob, Wfull, src[0], src[1], out_k, out_v)
         ts = []
@@ -281,7 +293,7 @@ def main():
             e1.record()
             e1.synchronize()
             ts.append(e0.elapsed_time(e1))
-        abytes = 2 * (wl.Ls + wl.Lt) * T * wl.Hs * d * 2
+        abytes = 2 * (wl.Ls * wl.Hs + wl.Lt * wl.Ht) * T * d * 2
         apply_info = {"tokens": T, "ms": statistics.median(ts), "tokens_per_s": T / (statistics.median(ts) / 1e3),
                       "algorithmic_gb": abytes / 1e9, "gbs": abytes / 1e9 / (statistics.median(ts) / 1e3)}
         del src, out_k, out_v
@@ -296,20 +308,20 @@ def main():
     peaks = measured_peaks()
     acc_avg = statistics.mean(acc_ms)
     tok_launch = tokens_per_step / n_chunks
-    achieved = ALG_BYTES_PER_TOKEN * tok_launch / 1e9 / (acc_avg / 1e3)
+    achieved = alg_bytes * tok_launch / 1e9 / (acc_avg / 1e3)
     roof = {"bound": "hbm", "kernel": "k_accum_tc<128>", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
-            "ms_per_launch": acc_avg, "algorithmic_gb_per_launch": ALG_BYTES_PER_TOKEN * tok_launch / 1e9,
-            "tflops": ALG_FLOPS_PER_TOKEN * tok_launch / 1e12 / (acc_avg / 1e3),
-            "tensor_frac_of_burst": ALG_FLOPS_PER_TOKEN * tok_launch / 1e12 / (acc_avg / 1e3) / peaks["bf16_tflops"]}
+            "ms_per_launch": acc_avg, "algorithmic_gb_per_launch": alg_bytes * tok_launch / 1e9,
+            "tflops": alg_flops * tok_launch / 1e12 / (acc_avg / 1e3),
+            "tensor_frac_of_burst": alg_flops * tok_launch / 1e12 / (acc_avg / 1e3) / peaks["bf16_tflops"]}
     tpath = os.path.join(ROOT, "profiles", "traffic_k_accum_tc.json")
-    if os.path.exists(tpath):
+    if os.path.exists(tpath) and args.workload == WORKLOAD:
         with open(tpath) as f:
             t = json.load(f)     # ncu capture of a smaller launch, scaled: per-token part x tokens + slot read-modify-write per split
             n_splits = args.splits if args.splits > 0 else 4
             roof["traffic"] = t["dram_bytes_per_token"] * tok_launch + t["dram_bytes_fixed_per_split"] * n_splits
-    t_roof = max(ALG_BYTES_PER_TOKEN * tokens_per_step / (peaks["hbm_gbs"] * 1e9),
-                 ALG_FLOPS_PER_TOKEN * tokens_per_step / (peaks["bf16_tflops"] * 1e12))
+    t_roof = max(alg_bytes * tokens_per_step / (peaks["hbm_gbs"] * 1e9),
+                 alg_flops * tokens_per_step / (peaks["bf16_tflops"] * 1e12))
     ms_step = total_ms / args.steps
     cpu = None
     if not args.no_cpu:
@@ -321,12 +333,13 @@ def main():
     out = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-           "config": {"workload": WORKLOAD + (": 500 seq x 1024 tok, 40->64 layers x 8 KV heads x 128, 1024 maps, lambda in {1e-3,1e-2,1e-1}"
-                                              if n_chunks == wl.n_chunks else " PARTIAL (%d of %d chunks)" % (n_chunks, wl.n_chunks)),
+           "config": {"workload": args.workload + (": %d seq, %d tokens, %d->%d layers x %d KV heads x %d, %d maps, lambda in %s"
+                                                   % (len(wl.seq_lens), wl.n_tokens, wl.Ls, wl.Lt, wl.Ht, wl.d, wl.n_maps, list(wl.lambdas))
+                                                   if n_chunks == wl.n_chunks else " PARTIAL (%d of %d chunks)" % (n_chunks, wl.n_chunks)),
                       "chunks_per_step": n_chunks, "tokens_per_chunk": int(tok_launch), "flags": args.flags,
-                      "l2": "inputs larger than L2 (%.1f GB per launch)" % (ALG_BYTES_PER_TOKEN * tok_launch / 1e9),
+                      "l2": "inputs larger than L2 (%.1f GB per launch)" % (alg_bytes * tok_launch / 1e9),
                       "timed": "sum of CUDA-event regions: accumulate calls + reduce + exchange/solve; chunk generation untimed"},
-           "s_per_500seq_build": ms_step / 1e3 * (wl.n_chunks / n_chunks),
+           "s_per_500seq_build": ms_step / 1e3 * (wl.n_chunks / n_chunks) * (500.0 / len(wl.seq_lens)),
            "frac_of_roofline_whole_build": t_roof * 1e3 / ms_step,
            "breakdown_ms": {"accumulate": statistics.mean(acc_ms) * n_chunks, "reduce": statistics.mean(red_ms),
                             "solve_3_lambdas": statistics.mean(sol_ms)},

@@ -714,7 +714,11 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     P.fh = FhDev{};
     const int TT = 64;
     if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
+#ifdef CB_DRAIN_TOKENS
+    P.drain_tiles = CB_DRAIN_TOKENS / TT;
+#else
     P.drain_tiles = 16384 / TT;   // at most 16384 tokens are summed in tensor memory before a drain
+#endif
     cudaError_t e;
     if (a.compensated) e = (d == 128) ? launch_tc<128, true>(P, st) : launch_tc<64, true>(P, st);
     else e = (d == 128) ? launch_tc<128, false>(P, st) : launch_tc<64, false>(P, st);
