@@ -128,47 +128,61 @@ cudaError_t launch_accum_simt(const AccumArgs &a, int d, cudaStream_t st)
 
 // ======================================================================================================
 // Deterministic reduction of the splits: fixed index order, fp64 sums, symmetrised G.
-// Grid n_maps, 256 threads.
+// Grid n_maps, 1024 threads.  The splits are summed with coalesced reads into a shared-memory image of D
+// (fp32, padded rows); G and C are then written from that image, the transpose needed for the
+// symmetrisation being a shared-memory access.
 // ======================================================================================================
-__global__ void __launch_bounds__(256) k_reduce(const float *__restrict__ slots, int n_splits, int n_maps, int d,
+__global__ void __launch_bounds__(1024) k_reduce(const float *__restrict__ slots, int n_splits, int n_maps, int d,
                                                 float *__restrict__ G, float *__restrict__ C)
 {
-    const int m = blockIdx.x, p = d + 1;
+    extern __shared__ __align__(16) float rs[];       // [d][2d + 1] sums of D, then [2d + 1] sums of s_x, s_y, s_w
+    const int m = blockIdx.x, p = d + 1, n2 = 2 * d, pitch = 2 * d + 1;
     const int sf = slot_floats(d);
     const float *base = slots + (size_t)m * sf;
     const size_t sstride = (size_t)n_maps * sf;
+    // sum the splits four floats at a time (slots are 16-byte aligned and sf is a multiple of 4); the slot's last
+    // three floats are padding and land in unused tail entries
+    for (int e4 = threadIdx.x; e4 < sf / 4; e4 += blockDim.x) {
+        double v[4] = {0.0, 0.0, 0.0, 0.0};
+        for (int s = 0; s < n_splits; ++s) {
+            const float4 f = *reinterpret_cast<const float4 *>(base + s * sstride + 4 * e4);
+            v[0] += (double)f.x; v[1] += (double)f.y; v[2] += (double)f.z; v[3] += (double)f.w;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int e = 4 * e4 + q;
+            if (e < d * n2) rs[(e / n2) * pitch + (e % n2)] = (float)v[q];
+            else rs[d * pitch + (e - d * n2)] = (float)v[q];
+        }
+    }
+    __syncthreads();
+    const float *bs = rs + d * pitch;                               // s_x [d], s_y [d], s_w
     float *Gm = G + (size_t)m * p * p;
     float *Cm = C + (size_t)m * p * d;
     for (int e = threadIdx.x; e < p * p; e += blockDim.x) {
         const int i = e / p, j = e % p;
-        double v = 0.0;
-        if (i < d && j < d) {
-            for (int s = 0; s < n_splits; ++s)
-                v += (double)base[s * sstride + (size_t)i * 2 * d + j] + (double)base[s * sstride + (size_t)j * 2 * d + i];
-            v *= 0.5;
-        } else if (i == d && j == d) {
-            for (int s = 0; s < n_splits; ++s) v += (double)base[s * sstride + slot_sw(d)];
-        } else {
-            const int c = (i == d) ? j : i;
-            for (int s = 0; s < n_splits; ++s) v += (double)base[s * sstride + slot_sx(d) + c];
-        }
-        Gm[e] = (float)v;
+        float v;
+        if (i < d && j < d) v = 0.5f * (rs[i * pitch + j] + rs[j * pitch + i]);     // a + b == b + a: exactly symmetric
+        else if (i == d && j == d) v = bs[2 * d];
+        else v = bs[(i == d) ? j : i];
+        Gm[e] = v;
     }
     for (int e = threadIdx.x; e < p * d; e += blockDim.x) {
         const int i = e / d, j = e % d;
-        double v = 0.0;
-        if (i < d) {
-            for (int s = 0; s < n_splits; ++s) v += (double)base[s * sstride + (size_t)i * 2 * d + d + j];
-        } else {
-            for (int s = 0; s < n_splits; ++s) v += (double)base[s * sstride + slot_sy(d) + j];
-        }
-        Cm[e] = (float)v;
+        Cm[e] = (i < d) ? rs[i * pitch + d + j] : bs[d + j];
     }
 }
 
 cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, float *G, float *C, cudaStream_t st)
 {
-    k_reduce<<<n_maps, 256, 0, st>>>(slots, n_splits, n_maps, d, G, C);
+    const size_t smem = sizeof(float) * ((size_t)d * (2 * d + 1) + 2 * d + 4);
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(k_reduce, cudaFuncAttributeMaxDynamicSharedMemorySize, 140 * 1024);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    k_reduce<<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, d, G, C);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;
