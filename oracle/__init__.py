@@ -183,6 +183,76 @@ def ridge_centered(X: np.ndarray, Y: np.ndarray, w: np.ndarray, lam: float):
     return Theta, int(info)
 
 
+# ----------------------------------------------------------------------------- two-pass centred construction
+def _trace_args(src_k, src_v, tgt_k, tgt_v, w_k, w_v, src_layer, src_head, maps):
+    Lt, T, Ht, d = tgt_k.shape
+    assert src_v.shape == src_k.shape and tgt_v.shape == tgt_k.shape and src_k.shape[1] == T
+    assert w_k.dtype == np.float32 and w_v.dtype == np.float32
+    assert w_k.shape == (Lt, Ht, T) and w_v.shape == (Lt, Ht, T)
+    assert w_k.strides[2] == 4 and w_v.strides == w_k.strides
+    src_layer = np.ascontiguousarray(src_layer, dtype=np.int32)
+    src_head = np.ascontiguousarray(src_head, dtype=np.int32)
+    if maps is None:
+        maps = np.arange(2 * Lt * Ht, dtype=np.int32)
+    maps = np.ascontiguousarray(maps, dtype=np.int32)
+    s = _trace_strides(src_k)
+    assert _trace_strides(src_v) == s
+    t = _trace_strides(tgt_k)
+    assert _trace_strides(tgt_v) == t
+    keep = (src_layer, src_head, maps)
+    args = [_p(src_k), _p(src_v), _i64(s[0]), _i64(s[1]), _i64(s[2]),
+            _p(tgt_k), _p(tgt_v), _i64(t[0]), _i64(t[1]), _i64(t[2]),
+            _p(w_k), _p(w_v), _i64(w_k.strides[0] // 4), _i64(w_k.strides[1] // 4),
+            _i64(T), _i32(d), _i32(Lt), _i32(Ht), _p(src_layer), _p(src_head), _p(maps), _i32(len(maps))]
+    return args, keep, len(maps), d
+
+
+def weighted_sums_traces(src_k, src_v, tgt_k, tgt_v, w_k, w_v, src_layer, src_head, maps=None):
+    """First pass of the two-pass construction on one chunk: sum w x [n_sel][d], sum w y [n_sel][d], sum w [n_sel]
+    (fp64).  Sums of several chunks add; the means are sum / s_w."""
+    args, keep, n_sel, d = _trace_args(src_k, src_v, tgt_k, tgt_v, w_k, w_v, src_layer, src_head, maps)
+    sx = np.empty((n_sel, d), np.float64)
+    sy = np.empty((n_sel, d), np.float64)
+    sw = np.empty(n_sel, np.float64)
+    _load().orc_means_traces(*args, _p(sx), _p(sy), _p(sw))
+    return sx, sy, sw
+
+
+def centered_stats_traces(src_k, src_v, tgt_k, tgt_v, w_k, w_v, src_layer, src_head, mu_x, mu_y, maps=None):
+    """Second pass on one chunk: A = sum w (x - mu_x)(x - mu_x)^T, B = sum w (x - mu_x)(y - mu_y)^T, [n_sel][d][d]."""
+    args, keep, n_sel, d = _trace_args(src_k, src_v, tgt_k, tgt_v, w_k, w_v, src_layer, src_head, maps)
+    mu_x = np.ascontiguousarray(mu_x, dtype=np.float64)
+    mu_y = np.ascontiguousarray(mu_y, dtype=np.float64)
+    assert mu_x.shape == (n_sel, d) and mu_y.shape == (n_sel, d)
+    A = np.empty((n_sel, d, d), np.float64)
+    B = np.empty((n_sel, d, d), np.float64)
+    _load().orc_centered_stats_traces(*args, _p(mu_x), _p(mu_y), _p(A), _p(B))
+    return A, B
+
+
+def ridge_solve_centered(A, B, mu_x, mu_y, s_w, n: int, lam: float, raw_lambda: bool = False):
+    """Theta = [W; b] from centred statistics: W = (A + lambda_eff I)^-1 B, b = mu_y - mu_x W (one map or a batch)."""
+    A = np.ascontiguousarray(A, dtype=np.float64)
+    B = np.ascontiguousarray(B, dtype=np.float64)
+    mu_x = np.ascontiguousarray(mu_x, dtype=np.float64)
+    mu_y = np.ascontiguousarray(mu_y, dtype=np.float64)
+    single = A.ndim == 2
+    if single:
+        A, B, mu_x, mu_y, s_w = A[None], B[None], mu_x[None], mu_y[None], np.array([s_w], np.float64)
+    s_w = np.ascontiguousarray(s_w, dtype=np.float64)
+    n_maps, d, _ = A.shape
+    Theta = np.empty((n_maps, d + 1, d), np.float64)
+    info = np.empty(n_maps, np.int32)
+    lib = _load()
+    for m in range(n_maps):
+        info[m] = lib.orc_ridge_solve_centered(_p(A[m]), _p(B[m]), _p(mu_x[m]), _p(mu_y[m]), ctypes.c_double(s_w[m]),
+                                               _i32(d), _i64(n), ctypes.c_double(lam), _i32(1 if raw_lambda else 0),
+                                               _p(Theta[m]))
+    if single:
+        return Theta[0], int(info[0])
+    return Theta, info
+
+
 # ----------------------------------------------------------------------------- apply
 def apply_maps(src_k: np.ndarray, src_v: np.ndarray, Theta: np.ndarray, Lt: int, Ht: int,
                src_layer: np.ndarray, src_head: np.ndarray, maps: Optional[Sequence[int]] = None,

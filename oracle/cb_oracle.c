@@ -20,7 +20,10 @@
  * counts of Section 3.2 and the storage figures of Section 4.4; the full-head
  * and multi-layer statistics against a library matrix product on gathered
  * features; the general-width solve by exact recovery and its residual; the
- * ESS floor by the Kish identity and the floors printed in Section 4.1.
+ * ESS floor by the Kish identity and the floors printed in Section 4.1; the
+ * two-pass centred statistics against a library weighted covariance, a hand
+ * example, shift invariance and equality of the resulting map with both the
+ * bias-column solve and the literal centred route.
  * Parity unpinned by the paper (defined by this build, not by the paper): the
  * synthetic input laws, the nearest-depth single-layer match (k = 1), and the
  * lambda_eff = lambda * s_w / n convention for weights that are not mean-one.
@@ -330,6 +333,126 @@ int32_t orc_ridge_centered(const double *X, const double *Y, const double *w, in
         memset(Theta, 0, sizeof(double) * (size_t)(d + 1) * d);
     }
     free(A); free(B); free(xc); free(yc); free(xb); free(yb);
+    return info;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Two-pass centred construction (Section 3.4, Eq. fusedstats): first the      */
+/* weighted means of every map over ALL rows,                                  */
+/*   s_w = sum_t w_t,  mu_x = sum_t w_t x_t / s_w,  mu_y = sum_t w_t y_t / s_w, */
+/* then, in a second traversal,                                                */
+/*   A = sum_t w_t (x_t - mu_x)(x_t - mu_x)^T,                                 */
+/*   B = sum_t w_t (x_t - mu_x)(y_t - mu_y)^T.                                 */
+/* Same trace addressing and map numbering as orc_stats_traces.  The weights   */
+/* are used as given (not rescaled); a map whose weights sum to zero gets zero */
+/* means.                                                                      */
+/* ------------------------------------------------------------------------- */
+void orc_means_traces(const uint16_t *src_k, const uint16_t *src_v,
+                      int64_t s_sl, int64_t s_st, int64_t s_sh,
+                      const uint16_t *tgt_k, const uint16_t *tgt_v,
+                      int64_t t_sl, int64_t t_st, int64_t t_sh,
+                      const float *w_k, const float *w_v, int64_t w_sl, int64_t w_sh,
+                      int64_t n_tokens, int32_t d, int32_t Lt, int32_t Ht,
+                      const int32_t *src_layer, const int32_t *src_head,
+                      const int32_t *maps, int32_t n_sel,
+                      double *sum_x /* [n_sel][d]: sum w x */, double *sum_y /* [n_sel][d] */,
+                      double *s_w /* [n_sel] */)
+{
+    for (int32_t s = 0; s < n_sel; ++s) {
+        const int32_t m = maps[s];
+        const int32_t comp = m / (Lt * Ht);
+        const int32_t l = (m / Ht) % Lt;
+        const int32_t h = m % Ht;
+        const uint16_t *xs = (comp ? src_v : src_k) + (int64_t)src_layer[l] * s_sl + (int64_t)src_head[h] * s_sh;
+        const uint16_t *ys = (comp ? tgt_v : tgt_k) + (int64_t)l * t_sl + (int64_t)h * t_sh;
+        const float *ws = (comp ? w_v : w_k) + (int64_t)l * w_sl + (int64_t)h * w_sh;
+        double *ax = sum_x + (size_t)s * d, *ay = sum_y + (size_t)s * d;
+        for (int32_t i = 0; i < d; ++i) ax[i] = ay[i] = 0.0;
+        double sw = 0.0;
+        for (int64_t t = 0; t < n_tokens; ++t) {
+            const double wt = (double)ws[t];
+            sw += wt;
+            for (int32_t i = 0; i < d; ++i) {
+                ax[i] += wt * orc_bf16(xs[t * s_st + i]);
+                ay[i] += wt * orc_bf16(ys[t * t_st + i]);
+            }
+        }
+        s_w[s] = sw;
+    }
+}
+
+void orc_centered_stats_traces(const uint16_t *src_k, const uint16_t *src_v,
+                               int64_t s_sl, int64_t s_st, int64_t s_sh,
+                               const uint16_t *tgt_k, const uint16_t *tgt_v,
+                               int64_t t_sl, int64_t t_st, int64_t t_sh,
+                               const float *w_k, const float *w_v, int64_t w_sl, int64_t w_sh,
+                               int64_t n_tokens, int32_t d, int32_t Lt, int32_t Ht,
+                               const int32_t *src_layer, const int32_t *src_head,
+                               const int32_t *maps, int32_t n_sel,
+                               const double *mu_x /* [n_sel][d] */, const double *mu_y /* [n_sel][d] */,
+                               double *A /* [n_sel][d][d] */, double *B /* [n_sel][d][d] */)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t s = 0; s < n_sel; ++s) {
+        const int32_t m = maps[s];
+        const int32_t comp = m / (Lt * Ht);
+        const int32_t l = (m / Ht) % Lt;
+        const int32_t h = m % Ht;
+        const uint16_t *xs = (comp ? src_v : src_k) + (int64_t)src_layer[l] * s_sl + (int64_t)src_head[h] * s_sh;
+        const uint16_t *ys = (comp ? tgt_v : tgt_k) + (int64_t)l * t_sl + (int64_t)h * t_sh;
+        const float *ws = (comp ? w_v : w_k) + (int64_t)l * w_sl + (int64_t)h * w_sh;
+        const double *mx = mu_x + (size_t)s * d, *my = mu_y + (size_t)s * d;
+        double *Am = A + (size_t)s * d * d, *Bm = B + (size_t)s * d * d;
+        double *xc = (double *)malloc(sizeof(double) * (size_t)d);
+        double *yc = (double *)malloc(sizeof(double) * (size_t)d);
+        memset(Am, 0, sizeof(double) * (size_t)d * d);
+        memset(Bm, 0, sizeof(double) * (size_t)d * d);
+        for (int64_t t = 0; t < n_tokens; ++t) {
+            for (int32_t i = 0; i < d; ++i) {
+                xc[i] = orc_bf16(xs[t * s_st + i]) - mx[i];
+                yc[i] = orc_bf16(ys[t * t_st + i]) - my[i];
+            }
+            const double wt = (double)ws[t];
+            for (int32_t i = 0; i < d; ++i) {
+                const double wx = wt * xc[i];
+                for (int32_t j = 0; j < d; ++j) {
+                    Am[(size_t)i * d + j] += wx * xc[j];
+                    Bm[(size_t)i * d + j] += wx * yc[j];
+                }
+            }
+        }
+        free(xc);
+        free(yc);
+    }
+}
+
+/*
+ * The solve of the two-pass path (Section 3.4, last display; Section 3.1, Eq.
+ * closedform): W = (A + lambda_eff I)^-1 B, b = mu_y - mu_x W, with the same
+ * lambda_eff = lambda * s_w / n convention as orc_ridge_solve (weights not
+ * rescaled to mean one), or lambda itself when raw_lambda != 0.
+ */
+int32_t orc_ridge_solve_centered(const double *A, const double *B, const double *mu_x, const double *mu_y,
+                                 double s_w, int32_t d, int64_t n, double lambda, int32_t raw_lambda,
+                                 double *Theta /* [d+1][d]: W then b */)
+{
+    const double lam = raw_lambda ? lambda : (n > 0 ? lambda * s_w / (double)n : lambda);
+    double *M = (double *)malloc(sizeof(double) * (size_t)d * d);
+    memcpy(M, A, sizeof(double) * (size_t)d * d);
+    for (int32_t i = 0; i < d; ++i) M[(size_t)i * d + i] += lam;
+    int32_t info = orc_cholesky(M, d);
+    if (info == 0) {
+        memcpy(Theta, B, sizeof(double) * (size_t)d * d);
+        orc_cholesky_solve(M, d, Theta, d);
+        for (int32_t j = 0; j < d; ++j) {
+            double v = mu_y[j];
+            for (int32_t i = 0; i < d; ++i) v -= mu_x[i] * Theta[(size_t)i * d + j];
+            Theta[(size_t)d * d + j] = v;
+        }
+    } else {
+        memset(Theta, 0, sizeof(double) * (size_t)(d + 1) * d);
+    }
+    free(M);
     return info;
 }
 
