@@ -172,6 +172,9 @@ def main():
     ap.add_argument("--multilayer", type=int, default=0, metavar="K",
                     help="time the head-local build over K selected layers per target layer (the paper's operating point is "
                          "K = 8) on one 50-sequence chunk plus the wide ridge solve, and print its own JSON line")
+    ap.add_argument("--two-pass", action="store_true",
+                    help="time the two-pass centred construction (means pass, centred accumulation, reduce, centred solve) "
+                         "on the selected workload and print its own JSON line")
     ap.add_argument("--profile-tokens", type=int, default=0,
                     help="profiling case: run only the accumulate kernel (3 launches) and the apply kernel on this many "
                          "tokens of the same shapes, print timings, no JSON line")
@@ -204,6 +207,9 @@ def main():
         return
     if args.multilayer > 0:
         multilayer_case(args, cb, synth, torch, wl, sl, sh, dev)
+        return
+    if args.two_pass:
+        two_pass_case(args, cb, synth, torch, wl, sl, sh, dev)
         return
     prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, flags=args.flags, n_splits=args.splits)
     ctx = cb.cb_create(prob, device=dev)
@@ -346,6 +352,71 @@ def main():
            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "apply": apply_info,
            "gpu_launches": launches, "clocks": clocks}
     print(json.dumps(out))
+
+
+def two_pass_case(args, cb, synth, torch, wl, sl, sh, dev):
+    """Two-pass centred construction: every chunk is read twice (means, then centred statistics)."""
+    alg_bytes, alg_flops = algorithmic_work(wl)
+    n_chunks = args.chunks if args.chunks > 0 else wl.n_chunks
+    prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, flags=args.flags, n_splits=args.splits)
+    ctx = cb.cb_create(prob, device=dev)
+    law = synth.map_law(wl, dev)
+    d, nl = wl.d, len(wl.lambdas)
+    ws = torch.empty(cb.cb_means_workspace_bytes(prob), dtype=torch.uint8, device=dev)
+    mu = torch.empty(wl.n_maps, 2 * d + 1, device=dev)
+    A = torch.empty(wl.n_maps, d, d, device=dev)
+    B = torch.empty(wl.n_maps, d, d, device=dev)
+    Wb = torch.empty(nl, wl.n_maps, d + 1, d, device=dev)
+    info = torch.empty(nl, wl.n_maps, dtype=torch.int32, device=dev)
+
+    def timed(fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        r = fn()
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1), r
+
+    def one_step():
+        cb.cb_means_reset(ctx, ws)
+        cb.cb_stats_reset(ctx)
+        t = {"means": [], "accumulate": []}
+        for c in range(n_chunks):
+            ch = synth.make_chunk(wl, c, sl, sh, device=dev, law=law)
+            t["means"].append(timed(lambda: cb.cb_means_accumulate(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"],
+                                                                   ch["w_k"], ch["w_v"], ws))[0])
+            del ch
+        t["finalize"] = timed(lambda: cb.cb_means_finalize(ctx, ws, mu))[0]
+        for c in range(n_chunks):
+            ch = synth.make_chunk(wl, c, sl, sh, device=dev, law=law)
+            t["accumulate"].append(timed(lambda: cb.cb_stats_accumulate_centered(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"],
+                                                                                 ch["tgt_v"], ch["w_k"], ch["w_v"], mu))[0])
+            del ch
+        t["reduce"], n = timed(lambda: cb.cb_stats_reduce_centered(ctx, mu, A, B))
+        t["solve"] = timed(lambda: cb.cb_ridge_solve_centered(A, B, mu, n, wl.lambdas, 0, Wb, info))[0]
+        return t
+
+    for _ in range(args.warmup):
+        one_step()
+    runs = [one_step() for _ in range(args.steps)]
+    cb.cb_device_status(ctx)
+    cb.cb_check_info(info)
+    peaks = measured_peaks()
+    tok_launch = sum(wl.chunk_tokens(c) for c in range(n_chunks)) / n_chunks
+    means_ms = statistics.mean([x for r in runs for x in r["means"]])
+    acc_ms = statistics.mean([x for r in runs for x in r["accumulate"]])
+    step_ms = statistics.mean([sum(r["means"]) + r["finalize"] + sum(r["accumulate"]) + r["reduce"] + r["solve"] for r in runs])
+    gb = alg_bytes * tok_launch / 1e9
+    print(json.dumps({"workload": "two-pass centred construction, %s, %d chunks of %d tokens" % (args.workload, n_chunks, tok_launch),
+                      "ms_per_build": step_ms, "tokens_per_s": tok_launch * n_chunks / (step_ms / 1e3),
+                      "breakdown_ms": {"means_per_chunk": means_ms, "finalize": statistics.mean([r["finalize"] for r in runs]),
+                                       "accumulate_per_chunk": acc_ms, "reduce": statistics.mean([r["reduce"] for r in runs]),
+                                       "solve": statistics.mean([r["solve"] for r in runs])},
+                      "roofline_means": {"bound": "hbm", "kernel": "k_means", "achieved": gb / (means_ms / 1e3),
+                                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gb / (means_ms / 1e3) / peaks["hbm_gbs"]},
+                      "roofline_accumulate": {"bound": "hbm", "kernel": "k_accum_tc<128, centred>", "achieved": gb / (acc_ms / 1e3),
+                                              "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gb / (acc_ms / 1e3) / peaks["hbm_gbs"]},
+                      "frac_of_roofline_whole_build": 2 * alg_bytes * tok_launch * n_chunks / (peaks["hbm_gbs"] * 1e9) / (step_ms / 1e3)}))
 
 
 def fullhead_case(args, cb, synth, torch, wl, sl, sh, dev):

@@ -268,6 +268,49 @@ cb_status cb_apply_multilayer(const cb_fullhead_problem *prob, const int32_t *sr
                               int64_t t_stride_layer, int64_t t_stride_token, int64_t t_stride_head, int32_t out_dtype,
                               void *workspace, size_t workspace_bytes, void *stream);
 
+/* ------------------------------------------------------------------------------------------------------------------
+ * Two-pass centred construction (Section 3.4, Eq. "fusedstats" and the solve displayed below it).
+ *
+ * The paper's own construction: a first pass obtains the weighted means of every map by a fixed reduction tree,
+ * a second pass accumulates the centred statistics
+ *     A = sum_t w_t (x_t - mu_x)(x_t - mu_x)^T   [d][d],      B = sum_t w_t (x_t - mu_x)(y_t - mu_y)^T   [d][d],
+ * and the solve is  W = (A + lambda_eff I)^-1 B,  b = mu_y - mu_x W.  It is the same estimator as the one-pass
+ * bias-column path above; it costs a second read of the traces and is the robust choice when channel means dwarf
+ * the spread (the one-pass operand w x is rounded to bf16 BEFORE the mean cancels, the two-pass operand w (x - mu_x)
+ * after).  Both passes are additive over calls, so a streamed build runs pass 1 over all chunks, finalises, then
+ * pass 2 over all chunks.
+ *
+ * Call order:  cb_means_reset; cb_means_accumulate per chunk; cb_means_finalize -> mu;
+ *              cb_stats_reset; cb_stats_accumulate_centered per chunk (same chunks, same mu);
+ *              cb_stats_reduce_centered -> A, B;  cb_ridge_solve_centered -> Wb (same layout as cb_ridge_solve, so
+ *              cb_apply consumes it unchanged).
+ *
+ * means_ws: caller-owned device memory, 256-byte aligned, at least cb_means_workspace_bytes() bytes (fp64 partial
+ * sums, 8 token splits per map); it carries the first-pass state between calls.
+ * mu: device fp32 [n_maps][2 d + 1], per map  mu_x [d], mu_y [d], s_w  (a map whose weights sum to zero gets zero
+ * means).  Reduction order is fixed (per thread in token order, row groups in index order, splits in index order,
+ * chunks in call order), so results are bitwise reproducible for a fixed sequence of calls.
+ * The accumulate call takes the same arguments as cb_stats_accumulate plus mu; it uses the context's partial slots
+ * (do not mix one-pass and centred accumulation between two resets) and is not available with CB_FLAG_SIMT
+ * (CB_ERR_UNSUPPORTED).  cb_stats_reduce_centered writes fp32 A [n_maps][d][d] (exactly symmetric) and
+ * B [n_maps][d][d].  cb_ridge_solve_centered: arguments as cb_ridge_solve with (A, B, mu) in place of (G, C);
+ * lambda_eff = lambda * s_w / n_tokens unless CB_FLAG_RAW_LAMBDA.
+ * Errors: as for their one-pass counterparts; CB_ERR_WORKSPACE for a missing, misaligned or short means_ws.
+ */
+cb_status cb_means_workspace_bytes(const cb_problem *prob, size_t *bytes);
+cb_status cb_means_reset(cb_ctx *ctx, void *means_ws, size_t means_ws_bytes, void *stream);
+cb_status cb_means_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                              const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                              void *means_ws, size_t means_ws_bytes, void *stream);
+cb_status cb_means_finalize(cb_ctx *ctx, const void *means_ws, size_t means_ws_bytes, float *mu, void *stream);
+cb_status cb_stats_accumulate_centered(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                       const float *w_k, const float *w_v,
+                                       int64_t w_stride_layer, int64_t w_stride_head, const float *mu, void *stream);
+cb_status cb_stats_reduce_centered(cb_ctx *ctx, const float *mu, float *A, float *B, int64_t *n_tokens_out, void *stream);
+cb_status cb_ridge_solve_centered(const float *A, const float *B, const float *mu, int32_t n_maps, int32_t d,
+                                  int64_t n_tokens, const float *lambdas, int32_t n_lambda, uint32_t flags,
+                                  float *Wb, int32_t *info, void *stream);
+
 /*
  * Synchronises the stream and reads the context's device status word: CB_OK, or CB_ERR_TIMEOUT if a bounded
  * wait inside a kernel ran out (the statistics are then invalid; reset before reuse).

@@ -28,6 +28,8 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_check_info", "cb_apply", "cb_device_status", "cb_stats_build_static", "cb_fullhead_layer_sets",
            "cb_fullhead_workspace_bytes", "cb_fullhead_stats_accumulate", "cb_ess_weights", "cb_ridge_solve_large_workspace_bytes", "cb_ridge_solve_large", "cb_multilayer_workspace_bytes",
            "cb_multilayer_stats_accumulate", "cb_apply_multilayer_workspace_bytes", "cb_apply_multilayer",
+           "cb_means_workspace_bytes", "cb_means_reset", "cb_means_accumulate", "cb_means_finalize",
+           "cb_stats_accumulate_centered", "cb_stats_reduce_centered", "cb_ridge_solve_centered",
            "cb_launch_count")
 
 
@@ -236,6 +238,79 @@ def cb_ridge_solve(G: torch.Tensor, C: torch.Tensor, n_tokens: int, lambdas: Seq
                                 ctypes.c_int64(n_tokens), lam.ctypes.data_as(ctypes.c_void_p), len(lam),
                                 ctypes.c_uint32(flags), ctypes.c_void_p(Wb.data_ptr()),
                                 ctypes.c_void_p(info.data_ptr()), _stream_ptr(stream)), "cb_ridge_solve")
+
+
+# ----------------------------------------------------------------------------- two-pass centred construction
+def cb_means_workspace_bytes(prob: Problem) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().cb_means_workspace_bytes(ctypes.byref(prob.c), ctypes.byref(n)), "cb_means_workspace_bytes")
+    return n.value
+
+
+def cb_means_reset(ctx: Context, means_ws: torch.Tensor, stream=None) -> None:
+    _check(lib().cb_means_reset(ctx.handle, ctypes.c_void_p(means_ws.data_ptr()), ctypes.c_size_t(means_ws.numel()),
+                                _stream_ptr(stream)), "cb_means_reset")
+
+
+def cb_means_accumulate(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor, w_v: torch.Tensor,
+                        means_ws: torch.Tensor, stream=None) -> None:
+    """First pass over one chunk; arguments as cb_stats_accumulate plus the uint8 device tensor `means_ws`."""
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    assert w_k.dtype == torch.float32 and w_v.dtype == torch.float32 and w_k.dim() == 3
+    assert w_k.stride() == w_v.stride() and (w_k.stride(2) == 1 or w_k.shape[2] <= 1)
+    assert means_ws.is_cuda and means_ws.dtype == torch.uint8
+    _check(lib().cb_means_accumulate(ctx.handle, ctypes.byref(sv), ctypes.byref(tv),
+                                     ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                     ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
+                                     ctypes.c_void_p(means_ws.data_ptr()), ctypes.c_size_t(means_ws.numel()),
+                                     _stream_ptr(stream)), "cb_means_accumulate")
+
+
+def cb_means_finalize(ctx: Context, means_ws: torch.Tensor, mu: torch.Tensor, stream=None) -> None:
+    """mu: fp32 device [n_maps][2 d + 1] = mu_x, mu_y, s_w."""
+    assert mu.dtype == torch.float32 and mu.is_contiguous() and mu.numel() == ctx.prob.n_maps * (2 * ctx.prob.ds + 1)
+    _check(lib().cb_means_finalize(ctx.handle, ctypes.c_void_p(means_ws.data_ptr()), ctypes.c_size_t(means_ws.numel()),
+                                   ctypes.c_void_p(mu.data_ptr()), _stream_ptr(stream)), "cb_means_finalize")
+
+
+def cb_stats_accumulate_centered(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor, w_v: torch.Tensor,
+                                 mu: torch.Tensor, stream=None) -> None:
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    assert w_k.dtype == torch.float32 and w_v.dtype == torch.float32 and w_k.dim() == 3
+    assert w_k.stride() == w_v.stride() and (w_k.stride(2) == 1 or w_k.shape[2] <= 1)
+    assert mu.dtype == torch.float32 and mu.is_contiguous() and mu.numel() == ctx.prob.n_maps * (2 * ctx.prob.ds + 1)
+    _check(lib().cb_stats_accumulate_centered(ctx.handle, ctypes.byref(sv), ctypes.byref(tv),
+                                              ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                              ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
+                                              ctypes.c_void_p(mu.data_ptr()), _stream_ptr(stream)),
+           "cb_stats_accumulate_centered")
+
+
+def cb_stats_reduce_centered(ctx: Context, mu: torch.Tensor, A: torch.Tensor, B: torch.Tensor, stream=None) -> int:
+    d = ctx.prob.ds
+    assert A.dtype == torch.float32 and B.dtype == torch.float32 and A.is_contiguous() and B.is_contiguous()
+    assert A.numel() == ctx.prob.n_maps * d * d and B.numel() == ctx.prob.n_maps * d * d
+    n = ctypes.c_int64(0)
+    _check(lib().cb_stats_reduce_centered(ctx.handle, ctypes.c_void_p(mu.data_ptr()), ctypes.c_void_p(A.data_ptr()),
+                                          ctypes.c_void_p(B.data_ptr()), ctypes.byref(n), _stream_ptr(stream)),
+           "cb_stats_reduce_centered")
+    return n.value
+
+
+def cb_ridge_solve_centered(A: torch.Tensor, B: torch.Tensor, mu: torch.Tensor, n_tokens: int, lambdas: Sequence[float],
+                            flags: int, Wb: torch.Tensor, info: torch.Tensor, stream=None) -> None:
+    n_maps, d, _ = A.shape
+    lam = np.ascontiguousarray(lambdas, dtype=np.float32)
+    assert A.dtype == torch.float32 and B.dtype == torch.float32 and mu.dtype == torch.float32
+    assert Wb.dtype == torch.float32 and info.dtype == torch.int32
+    assert A.is_contiguous() and B.is_contiguous() and mu.is_contiguous() and Wb.is_contiguous() and info.is_contiguous()
+    assert B.shape == (n_maps, d, d) and mu.numel() == n_maps * (2 * d + 1)
+    assert Wb.numel() == len(lam) * n_maps * (d + 1) * d and info.numel() == len(lam) * n_maps
+    _check(lib().cb_ridge_solve_centered(ctypes.c_void_p(A.data_ptr()), ctypes.c_void_p(B.data_ptr()),
+                                         ctypes.c_void_p(mu.data_ptr()), n_maps, d, ctypes.c_int64(n_tokens),
+                                         lam.ctypes.data_as(ctypes.c_void_p), len(lam), ctypes.c_uint32(flags),
+                                         ctypes.c_void_p(Wb.data_ptr()), ctypes.c_void_p(info.data_ptr()),
+                                         _stream_ptr(stream)), "cb_ridge_solve_centered")
 
 
 def cb_ridge_solve_large_workspace_bytes(P: int, d: int, n_systems: int) -> int:

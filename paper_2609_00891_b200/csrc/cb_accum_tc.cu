@@ -243,7 +243,9 @@ struct Ring {
     __device__ __forceinline__ void next() { if (++idx == N) { idx = 0; phase ^= 1; } }
 };
 
-template <int D, bool COMP, bool FH>
+// CEN: two-pass centred construction: the weighted operand is w (x - mu_x) with the means of P.a.mu; the bias sums
+// become the column sums of the ROUNDED weighted operand (what the reduction needs for its exact correction).
+template <int D, bool COMP, bool FH, bool CEN>
 __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(const __grid_constant__ TcParams P)
 {
     using C = TcCfg<D, COMP, FH>;
@@ -424,8 +426,14 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
         while (cur.valid(n_units)) {
             const int m = cur.m, split = cur.split, n_t = cur.tile1 - cur.tile;
             uint64_t sx2[4], sy2[4];        // packed fp32 pairs: channels (2e, 2e+1) of this thread's chunk
+            uint64_t nmu2[4];               // centred: minus the means of those channels
 #pragma unroll
-            for (int e = 0; e < 4; ++e) sx2[e] = sy2[e] = 0ull;
+            for (int e = 0; e < 4; ++e) sx2[e] = sy2[e] = nmu2[e] = 0ull;
+            if (CEN) {
+                const float *mup = a.mu + (size_t)m * (2 * D + 1) + cc * 8;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) nmu2[e] = f2_pack(-__ldg(mup + 2 * e), -__ldg(mup + 2 * e + 1));
+            }
             sw = 0.f;
             for (int t = 0; t < n_t; ++t) {
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
@@ -450,19 +458,27 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                     unsigned hw[4], lw[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const uint64_t pr = f2_mul(w2, f2_from_bf16x2(xu[e]));     // w * x for two channels
-                        sx2[e] = f2_add(sx2[e], pr);
+                        uint64_t xf = f2_from_bf16x2(xu[e]);
+                        if (CEN) xf = f2_add(xf, nmu2[e]);                         // x - mu_x
+                        const uint64_t pr = f2_mul(w2, xf);                        // w * x for two channels
+                        if (!CEN) sx2[e] = f2_add(sx2[e], pr);
                         float p0, p1;
                         f2_unpack(pr, p0, p1);
                         hw[e] = pack_bf16x2(p0, p1);
                         if (COMP) lw[e] = pack_bf16x2(p0 - __uint_as_float(hw[e] << 16), p1 - __uint_as_float(hw[e] & 0xffff0000u));
+                        if (CEN) {                                                 // sum of what the tensor cores will see
+                            sx2[e] = f2_add(sx2[e], f2_from_bf16x2(hw[e]));
+                            if (COMP) sx2[e] = f2_add(sx2[e], f2_from_bf16x2(lw[e]));
+                        }
                     }
                     *reinterpret_cast<uint4 *>(ah + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
                     if (COMP) *reinterpret_cast<uint4 *>(ah + C::A_BYTES + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-                    const uint4 yv = *reinterpret_cast<const uint4 *>(ys + off);
-                    const unsigned yu[4] = {yv.x, yv.y, yv.z, yv.w};
+                    if (!CEN) {
+                        const uint4 yv = *reinterpret_cast<const uint4 *>(ys + off);
+                        const unsigned yu[4] = {yv.x, yv.y, yv.z, yv.w};
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) sy2[e] = f2_fma(w2, f2_from_bf16x2(yu[e]), sy2[e]);
+                        for (int e = 0; e < 4; ++e) sy2[e] = f2_fma(w2, f2_from_bf16x2(yu[e]), sy2[e]);
+                    }
                     if (cc == 0) sw += wt;
                 }
 #endif
@@ -679,19 +695,19 @@ static int sm_count()
     return n;
 }
 
-template <int D, bool COMP, bool FH = false>
+template <int D, bool COMP, bool FH = false, bool CEN = false>
 static cudaError_t launch_tc(const TcParams &P, cudaStream_t st)
 {
     using C = TcCfg<D, COMP, FH>;
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D, COMP, FH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D, COMP, FH, CEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr = true;
     }
     const int n_units = FH ? 2 * P.a.Lt * (P.fh.per_head ? P.a.Ht : 1) * (P.fh.NG + P.fh.NC) : 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
     const int grid = n_units < sm_count() ? n_units : sm_count();
-    k_accum_tc<D, COMP, FH><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
+    k_accum_tc<D, COMP, FH, CEN><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -720,7 +736,10 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     P.drain_tiles = 16384 / TT;   // at most 16384 tokens are summed in tensor memory before a drain
 #endif
     cudaError_t e;
-    if (a.compensated) e = (d == 128) ? launch_tc<128, true>(P, st) : launch_tc<64, true>(P, st);
+    if (a.mu) {
+        if (a.compensated) e = (d == 128) ? launch_tc<128, true, false, true>(P, st) : launch_tc<64, true, false, true>(P, st);
+        else e = (d == 128) ? launch_tc<128, false, false, true>(P, st) : launch_tc<64, false, false, true>(P, st);
+    } else if (a.compensated) e = (d == 128) ? launch_tc<128, true>(P, st) : launch_tc<64, true>(P, st);
     else e = (d == 128) ? launch_tc<128, false>(P, st) : launch_tc<64, false>(P, st);
     if (e == cudaSuccess) count_launch();
     return e;

@@ -211,11 +211,13 @@ cb_status cb_stats_reset(cb_ctx *ctx, void *stream)
     return CB_OK;
 }
 
-cb_status cb_stats_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
-                              const float *w_k, const float *w_v,
-                              int64_t w_stride_layer, int64_t w_stride_head, void *stream)
+static cb_status accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                 const float *w_k, const float *w_v,
+                                 int64_t w_stride_layer, int64_t w_stride_head, const float *mu, bool centred, void *stream)
 {
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (centred && !mu) return CB_ERR_INVALID_ARG;
+    if (centred && (ctx->prob.flags & CB_FLAG_SIMT)) return CB_ERR_UNSUPPORTED;
     const cb_problem &P = ctx->prob;
     cb_status s = check_view(src, P.Ls, P.Hs, P.ds);
     if (s != CB_OK) return s;
@@ -239,11 +241,122 @@ cb_status cb_stats_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_vi
     a.slots = reinterpret_cast<float *>(ctx->ws + ctx->lay.slots_off);
     a.status = reinterpret_cast<int *>(ctx->ws + ctx->lay.status_off);
     a.compensated = (P.flags & CB_FLAG_COMPENSATED) ? 1 : 0;
+    a.mu = centred ? mu : nullptr;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = (P.flags & CB_FLAG_SIMT) ? launch_accum_simt(a, ctx->d, st)
                                              : launch_accum_tc(a, ctx->d, src, tgt, st);
     if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     ctx->n_tokens += src->n_tokens;
+    return CB_OK;
+}
+
+cb_status cb_stats_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                              const float *w_k, const float *w_v,
+                              int64_t w_stride_layer, int64_t w_stride_head, void *stream)
+{
+    return accumulate_impl(ctx, src, tgt, w_k, w_v, w_stride_layer, w_stride_head, nullptr, false, stream);
+}
+
+// ---------------------------------------------------------------------------------------------------------------------
+// Two-pass centred construction
+// ---------------------------------------------------------------------------------------------------------------------
+static size_t means_bytes(const cb_ctx *ctx)
+{
+    return (size_t)MEANS_SPLITS * ctx->n_maps * means_stride(ctx->d) * sizeof(double);
+}
+
+cb_status cb_means_workspace_bytes(const cb_problem *prob, size_t *bytes)
+{
+    cb_status s = check_problem(prob);
+    if (s != CB_OK) return s;
+    if (!bytes) return CB_ERR_INVALID_ARG;
+    *bytes = (size_t)MEANS_SPLITS * 2 * prob->Lt * prob->Ht * means_stride(prob->ds) * sizeof(double);
+    return CB_OK;
+}
+
+cb_status cb_means_reset(cb_ctx *ctx, void *means_ws, size_t means_ws_bytes, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (!means_ws || ((uintptr_t)means_ws & 255) || means_ws_bytes < means_bytes(ctx)) return CB_ERR_WORKSPACE;
+    cudaError_t e = cudaMemsetAsync(means_ws, 0, means_bytes(ctx), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+cb_status cb_means_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                              const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                              void *means_ws, size_t means_ws_bytes, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    const cb_problem &P = ctx->prob;
+    cb_status s = check_view(src, P.Ls, P.Hs, P.ds);
+    if (s != CB_OK) return s;
+    s = check_view(tgt, P.Lt, P.Ht, P.dt);
+    if (s != CB_OK) return s;
+    if (src->n_tokens != tgt->n_tokens) return CB_ERR_INVALID_ARG;
+    if (!means_ws || ((uintptr_t)means_ws & 255) || means_ws_bytes < means_bytes(ctx)) return CB_ERR_WORKSPACE;
+    if (src->n_tokens == 0) return CB_OK;
+    if (!w_k || !w_v || w_stride_layer < 0 || w_stride_head < 0) return CB_ERR_INVALID_ARG;
+    if (((uintptr_t)w_k | (uintptr_t)w_v) & 3) return CB_ERR_INVALID_ARG;
+    MeansArgs a;
+    a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src->k), static_cast<const __nv_bfloat16 *>(src->v),
+                  src->stride_layer, src->stride_token, src->stride_head};
+    a.tgt = KVPtr{static_cast<const __nv_bfloat16 *>(tgt->k), static_cast<const __nv_bfloat16 *>(tgt->v),
+                  tgt->stride_layer, tgt->stride_token, tgt->stride_head};
+    a.w_k = w_k; a.w_v = w_v; a.w_sl = w_stride_layer; a.w_sh = w_stride_head;
+    a.n_tokens = (int)src->n_tokens;
+    a.Lt = P.Lt; a.Ht = P.Ht;
+    a.src_layer = reinterpret_cast<const int *>(ctx->ws + ctx->lay.tab_off);
+    a.src_head = a.src_layer + P.Lt;
+    a.msum = static_cast<double *>(means_ws);
+    cudaError_t e = launch_means(a, ctx->d, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+cb_status cb_means_finalize(cb_ctx *ctx, const void *means_ws, size_t means_ws_bytes, float *mu, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (!means_ws || ((uintptr_t)means_ws & 255) || means_ws_bytes < means_bytes(ctx)) return CB_ERR_WORKSPACE;
+    if (!mu) return CB_ERR_INVALID_ARG;
+    cudaError_t e = launch_means_finalize(static_cast<const double *>(means_ws), ctx->n_maps, ctx->d, mu,
+                                          static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+cb_status cb_stats_accumulate_centered(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                       const float *w_k, const float *w_v,
+                                       int64_t w_stride_layer, int64_t w_stride_head, const float *mu, void *stream)
+{
+    return accumulate_impl(ctx, src, tgt, w_k, w_v, w_stride_layer, w_stride_head, mu, true, stream);
+}
+
+cb_status cb_stats_reduce_centered(cb_ctx *ctx, const float *mu, float *A, float *B, int64_t *n_tokens_out, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (!mu || !A || !B) return CB_ERR_INVALID_ARG;
+    cudaError_t e = launch_reduce_centered(reinterpret_cast<const float *>(ctx->ws + ctx->lay.slots_off), ctx->n_splits,
+                                           ctx->n_maps, ctx->d, mu, A, B, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (n_tokens_out) *n_tokens_out = ctx->n_tokens;
+    return CB_OK;
+}
+
+cb_status cb_ridge_solve_centered(const float *A, const float *B, const float *mu, int32_t n_maps, int32_t d,
+                                  int64_t n_tokens, const float *lambdas, int32_t n_lambda, uint32_t flags,
+                                  float *Wb, int32_t *info, void *stream)
+{
+    if (!A || !B || !mu || !lambdas || !Wb || !info) return CB_ERR_INVALID_ARG;
+    if (n_maps < 0 || n_lambda <= 0 || n_lambda > 16 || n_tokens < 0) return CB_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return CB_ERR_UNSUPPORTED;
+    if (n_maps > 65535 * 16) return CB_ERR_UNSUPPORTED;
+    for (int i = 0; i < n_lambda; ++i)
+        if (!(lambdas[i] >= 0.f)) return CB_ERR_INVALID_ARG;
+    if (n_maps == 0) return CB_OK;
+    cudaError_t e = launch_solve_centered(A, B, mu, n_maps, d, n_tokens, lambdas, n_lambda, flags, Wb, info,
+                                          static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     return CB_OK;
 }
 

@@ -39,6 +39,24 @@ struct AccumArgs {
     float *slots;          // device [n_splits][n_maps][slot_floats]
     int *status;           // device status word
     int compensated;
+    // Two-pass centred construction: device [n_maps][2d + 1] = mu_x, mu_y, s_w per map; null for the one-pass path.
+    // When set, the weighted operand is w (x - mu_x) and the slot's s_x entries receive the sum of the ROUNDED
+    // weighted operand (the exact correction term of the reduction), s_y stays zero.
+    const float *mu = nullptr;
+};
+
+// First pass of the two-pass construction: fp64 partial sums [n_msplits][n_maps][means_stride(d)] = sum w x, sum w y, sum w.
+__host__ __device__ constexpr int means_stride(int d) { return 2 * d + 2; }
+constexpr int MEANS_SPLITS = 8;
+struct MeansArgs {
+    KVPtr src, tgt;
+    const float *w_k, *w_v;
+    long long w_sl, w_sh;
+    int n_tokens;
+    int Lt, Ht;
+    const int *src_layer;  // device [Lt]
+    const int *src_head;   // device [Ht]
+    double *msum;          // device [MEANS_SPLITS][n_maps][means_stride(d)]
 };
 
 struct ApplyArgs {
@@ -67,6 +85,12 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
 cudaError_t launch_fullhead_tc(const AccumArgs &a, const FullHeadArgs &f, int d, const cb_kv_view *src, const cb_kv_view *tgt,
                                cudaStream_t st);
 cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, float *G, float *C, cudaStream_t st);
+cudaError_t launch_means(const MeansArgs &a, int d, cudaStream_t st);
+cudaError_t launch_means_finalize(const double *msum, int n_maps, int d, float *mu, cudaStream_t st);
+cudaError_t launch_reduce_centered(const float *slots, int n_splits, int n_maps, int d, const float *mu, float *A, float *B,
+                                   cudaStream_t st);
+cudaError_t launch_solve_centered(const float *A, const float *B, const float *mu, int n_maps, int d, long long n_tokens,
+                                  const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st);
 cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long long n_tokens,
                          const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st);
 size_t solve_large_bytes_per_system(int P, int d);

@@ -1,0 +1,160 @@
+// Two-pass centred construction (Section 3.4): the pieces that the one-pass path does not have.
+//
+//   k_means            first pass: per map, sum w x, sum w y, sum w over a chunk, added to fp64 partial sums.
+//                      Pure streaming (every source/target element and weight is read once per map that uses it),
+//                      bound by HBM; the reduction order is fixed: a thread sums its rows in token order, the row
+//                      groups of a block are combined in index order, the block adds to its own (split, map) entry.
+//   k_means_finalize   sums the splits in index order (fp64) and divides by s_w.
+//   k_reduce_centered  second-pass reduction: the accumulate kernel multiplies the ROUNDED centred operand
+//                      a_t = bf16(w_t (x_t - mu_x)) with the uncentred [x_t | y_t]; with r = sum_t a_t (kept in the
+//                      slot's s_x entries) the centred statistics are exactly
+//                          A = sum_t a_t (x_t - mu_x)^T = D_xx - r mu_x^T,   B = D_xy - r mu_y^T.
+#include "cb_internal.cuh"
+
+namespace cb {
+
+template <int D>
+__global__ void __launch_bounds__(256) k_means(const MeansArgs a)
+{
+    constexpr int CC = D / 8;            // 16-byte chunks per head row
+    constexpr int RG = 256 / CC;         // row groups of the block
+    constexpr int UN = 4;                // rows in flight per thread
+    __shared__ float red[RG][2 * D + 1];
+    const int n_maps = 2 * a.Lt * a.Ht;
+    const int m = blockIdx.x, split = blockIdx.y;
+    const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
+    const int t0 = (int)(((long long)a.n_tokens * split) / gridDim.y);
+    const int t1 = (int)(((long long)a.n_tokens * (split + 1)) / gridDim.y);
+    const int cc = threadIdx.x % CC, rg = threadIdx.x / CC;
+    const __nv_bfloat16 *xs = (comp ? a.src.v : a.src.k) + (long long)a.src_layer[l] * a.src.sl + (long long)a.src_head[h] * a.src.sh + cc * 8;
+    const __nv_bfloat16 *ys = (comp ? a.tgt.v : a.tgt.k) + (long long)l * a.tgt.sl + (long long)h * a.tgt.sh + cc * 8;
+    const float *ws = (comp ? a.w_v : a.w_k) + (long long)l * a.w_sl + (long long)h * a.w_sh;
+
+    float sx[8], sy[8], sw = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) sx[e] = sy[e] = 0.f;
+    for (int r0 = t0 + rg; r0 < t1; r0 += UN * RG) {
+        uint4 xv[UN], yv[UN];
+        float wt[UN];
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const int r = r0 + u * RG;
+            const bool in = r < t1;
+            const int rr = in ? r : t0;
+            xv[u] = __ldg(reinterpret_cast<const uint4 *>(xs + (long long)rr * a.src.st));
+            yv[u] = __ldg(reinterpret_cast<const uint4 *>(ys + (long long)rr * a.tgt.st));
+            wt[u] = in ? __ldg(ws + rr) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const unsigned xu[4] = {xv[u].x, xv[u].y, xv[u].z, xv[u].w};
+            const unsigned yu[4] = {yv[u].x, yv[u].y, yv[u].z, yv[u].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                sx[2 * e] = fmaf(wt[u], __uint_as_float(xu[e] << 16), sx[2 * e]);
+                sx[2 * e + 1] = fmaf(wt[u], __uint_as_float(xu[e] & 0xffff0000u), sx[2 * e + 1]);
+                sy[2 * e] = fmaf(wt[u], __uint_as_float(yu[e] << 16), sy[2 * e]);
+                sy[2 * e + 1] = fmaf(wt[u], __uint_as_float(yu[e] & 0xffff0000u), sy[2 * e + 1]);
+            }
+            sw += wt[u];
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { red[rg][cc * 8 + e] = sx[e]; red[rg][D + cc * 8 + e] = sy[e]; }
+    if (cc == 0) red[rg][2 * D] = sw;
+    __syncthreads();
+    double *dst = a.msum + ((size_t)split * n_maps + m) * means_stride(D);
+    for (int v = threadIdx.x; v < 2 * D + 1; v += 256) {
+        double sum = 0.0;
+#pragma unroll 4
+        for (int g = 0; g < RG; ++g) sum += (double)red[g][v];
+        dst[v] += sum;
+    }
+}
+
+cudaError_t launch_means(const MeansArgs &a, int d, cudaStream_t st)
+{
+    dim3 grid(2 * a.Lt * a.Ht, MEANS_SPLITS);
+    if (d == 128) k_means<128><<<grid, 256, 0, st>>>(a);
+    else k_means<64><<<grid, 256, 0, st>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) count_launch();
+    return e;
+}
+
+// mu [n_maps][2d + 1]: mu_x, mu_y, s_w.  A map without weight gets zero means.
+__global__ void k_means_finalize(const double *__restrict__ msum, int n_maps, int d, float *__restrict__ mu)
+{
+    const int m = blockIdx.x, ms = means_stride(d);
+    double sw = 0.0;
+    for (int s = 0; s < MEANS_SPLITS; ++s) sw += msum[((size_t)s * n_maps + m) * ms + 2 * d];
+    for (int v = threadIdx.x; v < 2 * d + 1; v += blockDim.x) {
+        double sum = 0.0;
+        for (int s = 0; s < MEANS_SPLITS; ++s) sum += msum[((size_t)s * n_maps + m) * ms + v];
+        mu[(size_t)m * (2 * d + 1) + v] = (v == 2 * d) ? (float)sw : (sw > 0.0 ? (float)(sum / sw) : 0.f);
+    }
+}
+
+cudaError_t launch_means_finalize(const double *msum, int n_maps, int d, float *mu, cudaStream_t st)
+{
+    k_means_finalize<<<n_maps, 288, 0, st>>>(msum, n_maps, d, mu);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) count_launch();
+    return e;
+}
+
+// Same split summation as the one-pass reduction, then the rank-one corrections and the symmetrisation of A.
+__global__ void __launch_bounds__(1024) k_reduce_centered(const float *__restrict__ slots, int n_splits, int n_maps, int d,
+                                                         const float *__restrict__ mu, float *__restrict__ A,
+                                                         float *__restrict__ B)
+{
+    extern __shared__ __align__(16) float rs[];       // [d][2d + 1] sums of D, then [2d + 4] sums of r, -, s_w; then mu_x, mu_y
+    const int m = blockIdx.x, n2 = 2 * d, pitch = 2 * d + 1;
+    const int sf = slot_floats(d);
+    const float *base = slots + (size_t)m * sf;
+    const size_t sstride = (size_t)n_maps * sf;
+    float *mus = rs + (size_t)d * pitch + 2 * d + 4;
+    for (int v = threadIdx.x; v < 2 * d; v += blockDim.x) mus[v] = mu[(size_t)m * (2 * d + 1) + v];
+    for (int e4 = threadIdx.x; e4 < sf / 4; e4 += blockDim.x) {
+        double v[4] = {0.0, 0.0, 0.0, 0.0};
+        for (int s = 0; s < n_splits; ++s) {
+            const float4 f = *reinterpret_cast<const float4 *>(base + s * sstride + 4 * e4);
+            v[0] += (double)f.x; v[1] += (double)f.y; v[2] += (double)f.z; v[3] += (double)f.w;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int e = 4 * e4 + q;
+            if (e < d * n2) rs[(e / n2) * pitch + (e % n2)] = (float)v[q];
+            else rs[d * pitch + (e - d * n2)] = (float)v[q];
+        }
+    }
+    __syncthreads();
+    const float *r = rs + d * pitch;                                // sum of the rounded centred operand, per channel
+    float *Am = A + (size_t)m * d * d;
+    float *Bm = B + (size_t)m * d * d;
+    for (int e = threadIdx.x; e < d * d; e += blockDim.x) {
+        const int i = e / d, j = e % d;
+        const double aij = (double)rs[i * pitch + j] - (double)r[i] * (double)mus[j];
+        const double aji = (double)rs[j * pitch + i] - (double)r[j] * (double)mus[i];
+        Am[e] = (float)(0.5 * (aij + aji));                          // a + b == b + a: exactly symmetric
+        Bm[e] = (float)((double)rs[i * pitch + d + j] - (double)r[i] * (double)mus[d + j]);
+    }
+}
+
+cudaError_t launch_reduce_centered(const float *slots, int n_splits, int n_maps, int d, const float *mu, float *A, float *B,
+                                   cudaStream_t st)
+{
+    const size_t smem = sizeof(float) * ((size_t)d * (2 * d + 1) + 2 * d + 4 + 2 * d);
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(k_reduce_centered, cudaFuncAttributeMaxDynamicSharedMemorySize, 140 * 1024);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    k_reduce_centered<<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, d, mu, A, B);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) count_launch();
+    return e;
+}
+
+}  // namespace cb

@@ -194,7 +194,8 @@ cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, f
 //   L Z = C, L^T Theta = Z.
 // ======================================================================================================
 struct SolveArgs {
-    const float *G, *C;
+    const float *G, *C;    // augmented: G [p][p], C [p][d];  centred: A [d][d], B [d][d]
+    const float *mu;       // centred form only: [n_maps][2d + 1] = mu_x, mu_y, s_w; null for the augmented form
     float *Wb;
     int *info;
     int n_maps, d;
@@ -239,17 +240,19 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
     extern __shared__ __align__(16) double sm[];
     constexpr int NB = 8;
     const int d = a.d, p = d + 1;
+    const bool centred = a.mu != nullptr;
+    const int n = centred ? d : p;                     // order of the system: the centred form has no bias row
     const int m = blockIdx.x, li = blockIdx.y;
     double *Lp = sm;                                   // packed lower triangle, rows padded to even length
-    double *Z = sm + tri_row_start(p);                 // [p][d]
+    double *Z = sm + tri_row_start(n);                 // [n][d]
     __shared__ double diag[NB][NB];
     __shared__ double rdiag[136];                      // reciprocals of the diagonal of L
     __shared__ int s_fail;
     const int tid = threadIdx.x;
 
-    const float *Gm = a.G + (size_t)m * p * p;
-    const float *Cm = a.C + (size_t)m * p * d;
-    const double s_w = (double)Gm[(size_t)d * p + d];
+    const float *Gm = a.G + (size_t)m * n * n;
+    const float *Cm = a.C + (size_t)m * n * d;
+    const double s_w = centred ? (double)a.mu[(size_t)m * (2 * d + 1) + 2 * d] : (double)Gm[(size_t)d * p + d];
     const double lam = (a.flags & CB_FLAG_RAW_LAMBDA) ? (double)a.lambdas[li] : (double)a.lambdas[li] * s_w * a.inv_n;
     if (tid == 0) s_fail = 0;
     {
@@ -257,13 +260,13 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
         // one warp per row (coalesced, no divisions); the global loads of a row are issued together before any
         // shared-memory store so that they overlap
         constexpr int MAXV = 5;                            // ceil(129 / 32)
-        for (int i = warp; i < p; i += nwarps) {
+        for (int i = warp; i < n; i += nwarps) {
             const int rsi = tri_row_start(i);
             float gv[MAXV], cv[MAXV];
 #pragma unroll
             for (int v = 0; v < MAXV; ++v) {
                 const int k = lane + 32 * v;
-                gv[v] = (k <= i) ? __ldg(Gm + (size_t)i * p + k) : 0.f;
+                gv[v] = (k <= i) ? __ldg(Gm + (size_t)i * n + k) : 0.f;
                 cv[v] = (k < d) ? __ldg(Cm + (size_t)i * d + k) : 0.f;
             }
 #pragma unroll
@@ -279,17 +282,17 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
     ST(1);
     // ---------------- Cholesky ----------------
     const int row = tid;
-    const int rs = tri_row_start(row < p ? row : 0);
-    for (int j0 = 0; j0 < p; j0 += NB) {
-        const int nb = min(NB, p - j0);
+    const int rs = tri_row_start(row < n ? row : 0);
+    for (int j0 = 0; j0 < n; j0 += NB) {
+        const int nb = min(NB, n - j0);
         double acc[NB];
-        const bool active = row < p && row >= j0;
+        const bool active = row < n && row >= j0;
         if (active) {
 #pragma unroll
             for (int c = 0; c < NB; ++c) acc[c] = (c < nb && j0 + c <= row) ? Lp[rs + j0 + c] : 0.0;
             int drs[NB];
 #pragma unroll
-            for (int c = 0; c < NB; ++c) drs[c] = tri_row_start(min(j0 + c, p - 1));
+            for (int c = 0; c < NB; ++c) drs[c] = tri_row_start(min(j0 + c, n - 1));
             for (int k = 0; k < j0; k += 2) {          // j0 is a multiple of 8: aligned pairs
                 const double2 mine = *reinterpret_cast<const double2 *>(&Lp[rs + k]);
 #pragma unroll
@@ -377,13 +380,13 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
     if (tid < 2 * d) {
         const int c = tid >> 1, half = tid & 1;
         // forward: L Z = C, row blocks top-down
-        for (int i0 = 0; i0 < p; i0 += RB) {
+        for (int i0 = 0; i0 < n; i0 += RB) {
             double acc[RB];
             int rsr[RB];
 #pragma unroll
             for (int r = 0; r < RB; ++r) {
-                rsr[r] = tri_row_start(min(i0 + r, p - 1));
-                acc[r] = (half == 0 && i0 + r < p) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
+                rsr[r] = tri_row_start(min(i0 + r, n - 1));
+                acc[r] = (half == 0 && i0 + r < n) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
             }
             for (int k = 2 * half; k < i0; k += 4) {   // pairs (k, k+1), alternating between the two lanes
                 const double z0 = Z[(size_t)k * d + c], z1 = Z[(size_t)(k + 1) * d + c];
@@ -398,7 +401,7 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
             for (int r = 0; r < RB; ++r) acc[r] += shfl_xor_f64(acc[r], 1);
 #pragma unroll
             for (int r = 0; r < RB; ++r)
-                if (i0 + r < p) {
+                if (i0 + r < n) {
                     double v = acc[r];
 #pragma unroll
                     for (int q = 0; q < RB; ++q)
@@ -411,12 +414,12 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
         }
         ST(3);
         // backward: L^T Theta = Z, row blocks bottom-up
-        const int last = ((p - 1) / RB) * RB;
+        const int last = ((n - 1) / RB) * RB;
         for (int i0 = last; i0 >= 0; i0 -= RB) {
             double acc[RB];
 #pragma unroll
-            for (int r = 0; r < RB; ++r) acc[r] = (half == 0 && i0 + r < p) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
-            for (int k = i0 + RB + half; k < p; k += 2) {
+            for (int r = 0; r < RB; ++r) acc[r] = (half == 0 && i0 + r < n) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
+            for (int k = i0 + RB + half; k < n; k += 2) {
                 const double xk = Z[(size_t)k * d + c];
                 const int rsk = tri_row_start(k) + i0;   // even offset: aligned pairs
 #pragma unroll
@@ -430,11 +433,11 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
             for (int r = 0; r < RB; ++r) acc[r] += shfl_xor_f64(acc[r], 1);
 #pragma unroll
             for (int r = RB - 1; r >= 0; --r)
-                if (i0 + r < p) {
+                if (i0 + r < n) {
                     double v = acc[r];
 #pragma unroll
                     for (int q = RB - 1; q >= 0; --q)
-                        if (q > r && i0 + q < p) v -= Lp[tri_row_start(i0 + q) + i0 + r] * acc[q];
+                        if (q > r && i0 + q < n) v -= Lp[tri_row_start(i0 + q) + i0 + r] * acc[q];
                     v *= rdiag[i0 + r];
                     acc[r] = v;
                     if (half == 0) Z[(size_t)(i0 + r) * d + c] = v;
@@ -444,16 +447,23 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
     }
     __syncthreads();
     ST(4);
-    for (int e = tid; e < p * d; e += blockDim.x) Wm[e] = (float)Z[e];
+    for (int e = tid; e < n * d; e += blockDim.x) Wm[e] = (float)Z[e];
+    if (centred && tid < d) {
+        // b = mu_y - mu_x W (Section 3.4, last display)
+        const float *mup = a.mu + (size_t)m * (2 * d + 1);
+        double v = (double)mup[d + tid];
+        for (int i = 0; i < d; ++i) v -= (double)mup[i] * Z[(size_t)i * d + tid];
+        Wm[(size_t)d * d + tid] = (float)v;
+    }
     if (tid == 0) a.info[(size_t)li * a.n_maps + m] = 0;
     ST(5);
 }
 
-cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long long n_tokens,
-                         const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st)
+static cudaError_t launch_solve_any(const float *G, const float *C, const float *mu, int n_maps, int d, long long n_tokens,
+                                    const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st)
 {
     SolveArgs a;
-    a.G = G; a.C = C; a.Wb = Wb; a.info = info; a.n_maps = n_maps; a.d = d;
+    a.G = G; a.C = C; a.mu = mu; a.Wb = Wb; a.info = info; a.n_maps = n_maps; a.d = d;
     a.inv_n = n_tokens > 0 ? 1.0 / (double)n_tokens : 0.0;
     a.flags = flags; a.n_lambda = n_lambda;
     for (int i = 0; i < 16; ++i) a.lambdas[i] = i < n_lambda ? lambdas[i] : 0.f;
@@ -469,6 +479,18 @@ cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;
+}
+
+cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long long n_tokens,
+                         const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st)
+{
+    return launch_solve_any(G, C, nullptr, n_maps, d, n_tokens, lambdas, n_lambda, flags, Wb, info, st);
+}
+
+cudaError_t launch_solve_centered(const float *A, const float *B, const float *mu, int n_maps, int d, long long n_tokens,
+                                  const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st)
+{
+    return launch_solve_any(A, B, mu, n_maps, d, n_tokens, lambdas, n_lambda, flags, Wb, info, st);
 }
 
 // ======================================================================================================

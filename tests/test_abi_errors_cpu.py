@@ -87,3 +87,24 @@ def test_workspace_and_static_limits():
     assert cb.lib().cb_ridge_solve_large_workspace_bytes(1025, 128, ctypes.c_int64(1), ctypes.byref(n)) == cb.CB_OK
     assert n.value >= 8 * (1088 * 1088 + 1088 * 128)
     assert cb.lib().cb_ridge_solve_large_workspace_bytes(1025, 100, ctypes.c_int64(1), ctypes.byref(n)) == cb.CB_ERR_INVALID_ARG
+
+
+def test_two_pass_entry_points_reject_bad_arguments_on_the_host():
+    sl, sh = cb.cb_head_map_nearest(40, 8, 64, 8)
+    prob = cb.Problem(40, 8, 128, 64, 8, 128, sl, sh)
+    assert cb.cb_means_workspace_bytes(prob) == 8 * 1024 * (2 * 128 + 2) * 8          # fp64, 8 splits per map
+    null = ctypes.c_void_p(0)
+    L = cb.lib()
+    assert L.cb_means_reset(null, ctypes.c_void_p(0x1000), ctypes.c_size_t(1 << 30), null) == cb.CB_ERR_STATE
+    assert L.cb_means_finalize(null, ctypes.c_void_p(0x1000), ctypes.c_size_t(1 << 30), ctypes.c_void_p(0x10), null) == cb.CB_ERR_STATE
+    assert L.cb_stats_reduce_centered(null, ctypes.c_void_p(0x10), ctypes.c_void_p(0x10), ctypes.c_void_p(0x10), null, null) == cb.CB_ERR_STATE
+    lam = np.array([1e-2], np.float32)
+    call = lambda A, B, mu, n_maps, d, nl: L.cb_ridge_solve_centered(
+        ctypes.c_void_p(A), ctypes.c_void_p(B), ctypes.c_void_p(mu), n_maps, d, ctypes.c_int64(100),
+        lam.ctypes.data_as(ctypes.c_void_p), nl, ctypes.c_uint32(0), ctypes.c_void_p(0x20), ctypes.c_void_p(0x30), null)
+    before = cb.cb_launch_count()
+    assert call(0x10, 0x10, 0, 4, 128, 1) == cb.CB_ERR_INVALID_ARG                    # no means
+    assert call(0x10, 0x10, 0x10, 4, 100, 1) == cb.CB_ERR_UNSUPPORTED
+    assert call(0x10, 0x10, 0x10, 4, 128, 17) == cb.CB_ERR_INVALID_ARG
+    assert call(0x10, 0x10, 0x10, 0, 128, 1) == cb.CB_OK
+    assert cb.cb_launch_count() == before
