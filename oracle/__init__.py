@@ -253,6 +253,18 @@ def ridge_solve_centered(A, B, mu_x, mu_y, s_w, n: int, lam: float, raw_lambda: 
     return Theta, info
 
 
+# ----------------------------------------------------------------------------- rotary embedding at the boundary
+def rope_rotate(x: np.ndarray, pos: np.ndarray, base: float, inverse: bool = False) -> np.ndarray:
+    """Rotate-half RoPE of rows x [n][d] (fp64) at integer positions pos [n]; inverse removes the embedding."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    n, d = x.shape
+    assert pos.shape == (n,) and d % 2 == 0
+    out = np.empty_like(x)
+    _load().orc_rope_rotate(_p(x), _p(out), _i64(n), _i32(d), _p(pos), ctypes.c_double(base), _i32(1 if inverse else 0))
+    return out
+
+
 # ----------------------------------------------------------------------------- apply
 def apply_maps(src_k: np.ndarray, src_v: np.ndarray, Theta: np.ndarray, Lt: int, Ht: int,
                src_layer: np.ndarray, src_head: np.ndarray, maps: Optional[Sequence[int]] = None,

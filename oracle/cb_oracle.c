@@ -23,7 +23,9 @@
  * ESS floor by the Kish identity and the floors printed in Section 4.1; the
  * two-pass centred statistics against a library weighted covariance, a hand
  * example, shift invariance and equality of the resulting map with both the
- * bias-column solve and the literal centred route.
+ * bias-column solve and the literal centred route; the rotary embedding
+ * against a library implementation, the relative-position identity and a hand
+ * example.
  * Parity unpinned by the paper (defined by this build, not by the paper): the
  * synthetic input laws, the nearest-depth single-layer match (k = 1), and the
  * lambda_eff = lambda * s_w / n convention for weights that are not mean-one.
@@ -454,6 +456,31 @@ int32_t orc_ridge_solve_centered(const double *A, const double *B, const double 
     }
     free(M);
     return info;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Rotary position embedding at the boundary (Section 2.2 and Section 3.1:     */
+/* source RoPE is removed before fitting, target RoPE restored after mapping,  */
+/* so the map acts in content coordinates).  Keys only; values carry no RoPE.  */
+/* Convention (the paper does not print one; this is the rotate-half form of   */
+/* the RoFormer rotation used by the Llama / Qwen model families): channel i   */
+/* < d/2 pairs with channel i + d/2, angle phi_i = pos * base^(-2 i / d),       */
+/*   out_i       = x_i cos phi_i - x_{i+d/2} sin phi_i,                          */
+/*   out_{i+d/2} = x_i sin phi_i + x_{i+d/2} cos phi_i;                          */
+/* inverse != 0 rotates by -phi (removes the embedding).  Rows of width d.     */
+/* ------------------------------------------------------------------------- */
+void orc_rope_rotate(const double *in, double *out, int64_t n_rows, int32_t d,
+                     const int32_t *pos, double base, int32_t inverse)
+{
+    const int32_t half = d / 2;
+    for (int64_t t = 0; t < n_rows; ++t)
+        for (int32_t i = 0; i < half; ++i) {
+            const double phi = (double)pos[t] * pow(base, -2.0 * (double)i / (double)d);
+            const double c = cos(phi), s = inverse ? -sin(phi) : sin(phi);
+            const double a = in[t * d + i], b = in[t * d + i + half];
+            out[t * d + i] = a * c - b * s;
+            out[t * d + i + half] = a * s + b * c;
+        }
 }
 
 /* ------------------------------------------------------------------------- */
