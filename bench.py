@@ -172,6 +172,9 @@ def main():
     ap.add_argument("--multilayer", type=int, default=0, metavar="K",
                     help="time the head-local build over K selected layers per target layer (the paper's operating point is "
                          "K = 8) on one 50-sequence chunk plus the wide ridge solve, and print its own JSON line")
+    ap.add_argument("--rope", action="store_true",
+                    help="fit the key maps in content coordinates: rotary embedding (base 1e6, positions restart every "
+                         "1024 tokens) removed inside the accumulate kernel; the JSON line says so in config")
     ap.add_argument("--two-pass", action="store_true",
                     help="time the two-pass centred construction (means pass, centred accumulation, reduce, centred solve) "
                          "on the selected workload and print its own JSON line")
@@ -233,8 +236,13 @@ def main():
         for c in range(n_chunks):
             ch = synth.make_chunk(wl, c + 1000 * rank, sl, sh, device=dev, law=law)      # untimed: trace collection
             e0, e1 = ev(), ev()
+            pos = (torch.arange(ch["n_tokens"], dtype=torch.int32, device=dev) % 1024) if args.rope else None
             e0.record()
-            cb.cb_stats_accumulate(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"])
+            if args.rope:
+                cb.cb_stats_accumulate_rope(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"],
+                                            pos, 1e6, 1e6)
+            else:
+                cb.cb_stats_accumulate(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"])
             e1.record()
             acc_ev.append((e0, e1))
             e1.synchronize()
@@ -343,6 +351,7 @@ def main():
                                                    % (len(wl.seq_lens), wl.n_tokens, wl.Ls, wl.Lt, wl.Ht, wl.d, wl.n_maps, list(wl.lambdas))
                                                    if n_chunks == wl.n_chunks else " PARTIAL (%d of %d chunks)" % (n_chunks, wl.n_chunks)),
                       "chunks_per_step": n_chunks, "tokens_per_chunk": int(tok_launch), "flags": args.flags,
+                      "rope": bool(args.rope),
                       "l2": "inputs larger than L2 (%.1f GB per launch)" % (alg_bytes * tok_launch / 1e9),
                       "timed": "sum of CUDA-event regions: accumulate calls + reduce + exchange/solve; chunk generation untimed"},
            "s_per_500seq_build": ms_step / 1e3 * (wl.n_chunks / n_chunks) * (500.0 / len(wl.seq_lens)),

@@ -311,6 +311,33 @@ cb_status cb_ridge_solve_centered(const float *A, const float *B, const float *m
                                   int64_t n_tokens, const float *lambdas, int32_t n_lambda, uint32_t flags,
                                   float *Wb, int32_t *info, void *stream);
 
+/* ------------------------------------------------------------------------------------------------------------------
+ * Rotary position embedding at the boundary (Section 2.2; Section 3.1: source RoPE is inverted before fitting and
+ * target RoPE applied after mapping, so the affine map acts in content coordinates).  Keys only: values carry no
+ * rotary embedding and take the ordinary path.
+ *
+ * Convention (the paper prints none; this is the rotate-half form of the Llama / Qwen families): channel i < d/2
+ * pairs with channel i + d/2, angle phi_i = position * base^(-2 i / d); the embedding maps (x_i, x_{i+d/2}) to
+ * (x_i cos phi - x_{i+d/2} sin phi, x_i sin phi + x_{i+d/2} cos phi).  The whole head dimension rotates.
+ * positions: DEVICE int32 [n_tokens], the position of every row (ragged batches: each sequence restarts at its own
+ * origin), 4-byte aligned, 0 <= position < 2^20.  rope_base in (1, 1e12].
+ *
+ * cb_stats_accumulate_rope: as cb_stats_accumulate, but the key maps are fitted on source keys with the source
+ * model's embedding removed and target keys with the target model's removed; the rotation is applied to the staged
+ * tiles on chip (no extra pass over device memory).  The de-rotated rows are rounded to bf16 before they enter the
+ * tensor cores.  Not available with CB_FLAG_SIMT (CB_ERR_UNSUPPORTED).
+ *
+ * cb_rope_rotate: stand-alone rotation of a strided bf16 key tensor IN PLACE (inverse != 0 removes the embedding),
+ * element (layer, token, head, channel) at k + layer*stride_layer + token*stride_token + head*stride_head + channel,
+ * alignment rules as for cb_kv_view.
+ */
+cb_status cb_stats_accumulate_rope(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                   const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                                   const int32_t *positions, double rope_base_src, double rope_base_tgt, void *stream);
+cb_status cb_rope_rotate(void *k, int32_t n_layers, int32_t n_heads, int32_t head_dim, int64_t n_tokens,
+                         int64_t stride_layer, int64_t stride_token, int64_t stride_head,
+                         const int32_t *positions, double rope_base, int32_t inverse, void *stream);
+
 /*
  * Synchronises the stream and reads the context's device status word: CB_OK, or CB_ERR_TIMEOUT if a bounded
  * wait inside a kernel ran out (the statistics are then invalid; reset before reuse).

@@ -30,6 +30,7 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_multilayer_stats_accumulate", "cb_apply_multilayer_workspace_bytes", "cb_apply_multilayer",
            "cb_means_workspace_bytes", "cb_means_reset", "cb_means_accumulate", "cb_means_finalize",
            "cb_stats_accumulate_centered", "cb_stats_reduce_centered", "cb_ridge_solve_centered",
+           "cb_stats_accumulate_rope", "cb_rope_rotate",
            "cb_launch_count")
 
 
@@ -238,6 +239,33 @@ def cb_ridge_solve(G: torch.Tensor, C: torch.Tensor, n_tokens: int, lambdas: Seq
                                 ctypes.c_int64(n_tokens), lam.ctypes.data_as(ctypes.c_void_p), len(lam),
                                 ctypes.c_uint32(flags), ctypes.c_void_p(Wb.data_ptr()),
                                 ctypes.c_void_p(info.data_ptr()), _stream_ptr(stream)), "cb_ridge_solve")
+
+
+# ----------------------------------------------------------------------------- rotary embedding at the boundary
+def cb_stats_accumulate_rope(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor, w_v: torch.Tensor,
+                             positions: torch.Tensor, rope_base_src: float, rope_base_tgt: float, stream=None) -> None:
+    """As cb_stats_accumulate; `positions` is a device int32 tensor [T]."""
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    assert w_k.dtype == torch.float32 and w_v.dtype == torch.float32 and w_k.dim() == 3
+    assert w_k.stride() == w_v.stride() and (w_k.stride(2) == 1 or w_k.shape[2] <= 1)
+    assert positions.dtype == torch.int32 and positions.is_cuda and positions.is_contiguous()
+    assert positions.numel() == src_k.shape[1]
+    _check(lib().cb_stats_accumulate_rope(ctx.handle, ctypes.byref(sv), ctypes.byref(tv),
+                                          ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                          ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
+                                          ctypes.c_void_p(positions.data_ptr()), ctypes.c_double(rope_base_src),
+                                          ctypes.c_double(rope_base_tgt), _stream_ptr(stream)), "cb_stats_accumulate_rope")
+
+
+def cb_rope_rotate(k: torch.Tensor, positions: torch.Tensor, rope_base: float, inverse: bool, stream=None) -> None:
+    """In-place rotary embedding (or its removal) of a bf16 key tensor indexed [L][T][H][d]."""
+    assert k.dtype == torch.bfloat16 and k.dim() == 4 and k.stride(3) == 1
+    assert positions.dtype == torch.int32 and positions.is_contiguous() and positions.numel() == k.shape[1]
+    L, T, H, d = k.shape
+    _check(lib().cb_rope_rotate(ctypes.c_void_p(k.data_ptr()), L, H, d, ctypes.c_int64(T),
+                                ctypes.c_int64(k.stride(0)), ctypes.c_int64(k.stride(1)), ctypes.c_int64(k.stride(2)),
+                                ctypes.c_void_p(positions.data_ptr()), ctypes.c_double(rope_base),
+                                1 if inverse else 0, _stream_ptr(stream)), "cb_rope_rotate")
 
 
 # ----------------------------------------------------------------------------- two-pass centred construction

@@ -29,6 +29,7 @@
 
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
+#include "cb_rope.cuh"
 
 namespace cb {
 
@@ -59,7 +60,7 @@ struct TcCfg {
     static constexpr int RED_STRIDE = 2 * D + 4;                 // per fold warp: s_x[D], s_y[D], s_w, pad
     static constexpr int RED_FLOATS = FOLD_WARPS * RED_STRIDE;      // cross-warp bias reduction buffer
     static constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)NS * STAGE_BYTES + (size_t)NA * A_PARTS * A_BYTES +
-                                         RED_FLOATS * 4 + NS * TT * 4 /*weights*/ + 256 /*barriers*/;
+                                         RED_FLOATS * 4 + 2 * NS * TT * 4 /*weights, positions*/ + 256 /*barriers*/;
     static_assert(TT % RG == 0 && RPT >= 1, "fold layout");
     static_assert(TMEM_COLS == 256 || TMEM_COLS == 512, "tensor memory columns must be a power of two");
 };
@@ -83,6 +84,7 @@ struct TcParams {
     AccumArgs a;
     FhDev fh;
     int drain_tiles;                          // tiles accumulated in tensor memory between drains
+    RopeDev rope;                             // ROPE kernels only
 };
 
 // Walks the tiles of this block's units in order: units u = blockIdx.x, += gridDim.x.  Head-local: unit -> (map,
@@ -243,9 +245,12 @@ struct Ring {
     __device__ __forceinline__ void next() { if (++idx == N) { idx = 0; phase ^= 1; } }
 };
 
+// ROPE: key maps (comp = 0) are fitted in content coordinates (Section 3.1): the fold warps rotate every source and
+// target key row back by its position's angles IN PLACE in the staged tile (so the tensor cores read the de-rotated
+// rows as the second operand too) before weighting; value maps take the ordinary path.
 // CEN: two-pass centred construction: the weighted operand is w (x - mu_x) with the means of P.a.mu; the bias sums
 // become the column sums of the ROUNDED weighted operand (what the reduction needs for its exact correction).
-template <int D, bool COMP, bool FH, bool CEN>
+template <int D, bool COMP, bool FH, bool CEN, bool ROPE>
 __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(const __grid_constant__ TcParams P)
 {
     using C = TcCfg<D, COMP, FH>;
@@ -256,7 +261,8 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
     uint8_t *ab = xy + (size_t)C::NS * C::STAGE_BYTES;        // [NA][hi A_BYTES (| lo A_BYTES)]
     float *red = reinterpret_cast<float *>(ab + (size_t)C::NA * C::A_PARTS * C::A_BYTES);
     float *wst = red + C::RED_FLOATS;                         // [NS][TT] token weights of the staged tile
-    uint64_t *bars = reinterpret_cast<uint64_t *>(wst + C::NS * C::TT);
+    int *pst = reinterpret_cast<int *>(wst + C::NS * C::TT);  // [NS][TT] token positions (ROPE)
+    uint64_t *bars = reinterpret_cast<uint64_t *>(pst + C::NS * C::TT);
     uint64_t *full = bars;                 // [NS] tile landed: X bytes (1 arrival), Y bytes (1), weights (32 lanes)
     uint64_t *empty = full + C::NS;        // [NS] stage free: MMA done (1) + every fold warp done
     uint64_t *afull = empty + C::NS;       // [NA] weighted operand written (every fold warp)
@@ -350,6 +356,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                     const int r = lane + 32 * q;
                     const bool in = tok0 + r < a.n_tokens;
                     cp_async_4(&wst[st.idx * C::TT + r], w + (in ? tok0 + r : 0), in ? 4u : 0u);
+                    if (ROPE) cp_async_4(&pst[st.idx * C::TT + r], P.rope.pos + (in ? tok0 + r : 0), in ? 4u : 0u);
                 }
                 cp_async_arrive_noinc(&full[st.idx]);
                 CB_TR(it, 39);
@@ -418,6 +425,17 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
         // byte offset of this thread's first 16-byte chunk inside a block; its other rows are RG rows further down
         const int off0 = blk * C::BLK + rg * 128 + ((lc ^ (rg & 7)) << 4);
         float sx[8], sy[8], sw = 0.f;
+        // ROPE: this thread rotates half a chunk (4 frequencies) of rows rg, rg + RG, ..: channels 4 cc + e pair with
+        // channels D/2 + 4 cc + e.  Same (cc, rg) decomposition as the ordinary fold, other channels.
+        uint32_t fsrc[4] = {0, 0, 0, 0}, ftgt[4] = {0, 0, 0, 0};
+        int rp_lo = 0, rp_hi = 0;
+        if (ROPE) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { fsrc[e] = P.rope.f_src[cc * 4 + e]; ftgt[e] = P.rope.f_tgt[cc * 4 + e]; }
+            const int lcr = cc >> 1, hb = (cc & 1) * 8, swz = rg & 7;
+            rp_lo = rg * 128 + ((lcr ^ swz) << 4) + hb;
+            rp_hi = (D == 128) ? C::BLK + rp_lo : rg * 128 + (((lcr + 4) ^ swz) << 4) + hb;
+        }
         Ring<C::NS> st, old;       // `old` trails `st` by NA tiles
         Ring<C::NA> ar;
         uint32_t it = 0, uc = 0;
@@ -425,6 +443,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
         cur.start(P, n_units, n_maps, n_tiles);
         while (cur.valid(n_units)) {
             const int m = cur.m, split = cur.split, n_t = cur.tile1 - cur.tile;
+            const bool rope_unit = ROPE && cur.comp == 0;
             uint64_t sx2[4], sy2[4];        // packed fp32 pairs: channels (2e, 2e+1) of this thread's chunk
             uint64_t nmu2[4];               // centred: minus the means of those channels
 #pragma unroll
@@ -435,6 +454,10 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                 for (int e = 0; e < 4; ++e) nmu2[e] = f2_pack(-__ldg(mup + 2 * e), -__ldg(mup + 2 * e + 1));
             }
             sw = 0.f;
+            if (ROPE) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) sx[e] = sy[e] = 0.f;
+            }
             for (int t = 0; t < n_t; ++t) {
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
                 // the weighted-operand buffer was last used by tile it - NA; it is free once that tile's stage is free
@@ -448,6 +471,76 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                 const uint8_t *ys = xy + st.idx * C::STAGE_BYTES + C::NBX * C::BLK + off0;    // B2: summed with the weights
                 uint8_t *ah = ab + ar.idx * (C::A_PARTS * C::A_BYTES) + off0;
 #ifndef CB_ABLATE_FOLD
+                if (rope_unit) {
+                    uint8_t *xt = xy + st.idx * C::STAGE_BYTES;                       // X tile, rewritten in place
+                    uint8_t *yt = xt + C::NBX * C::BLK;                               // Y tile, rewritten in place
+                    uint8_t *at = ab + ar.idx * (C::A_PARTS * C::A_BYTES);
+                    const int *psm = pst + st.idx * C::TT + rg;
+#pragma unroll
+                    for (int i = 0; i < C::RPT; ++i) {
+                        const int off = i * C::RG * 128;
+                        const float wt = wsm[i * C::RG];
+                        const int pos = psm[i * C::RG];
+                        float cs[4], sn[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) rope_cs(fsrc[e], pos, cs[e], sn[e]);
+                        {
+                            const uint2 vl = *reinterpret_cast<const uint2 *>(xt + rp_lo + off);
+                            const uint2 vh = *reinterpret_cast<const uint2 *>(xt + rp_hi + off);
+                            const float lo[4] = {__uint_as_float(vl.x << 16), __uint_as_float(vl.x & 0xffff0000u),
+                                                 __uint_as_float(vl.y << 16), __uint_as_float(vl.y & 0xffff0000u)};
+                            const float hi[4] = {__uint_as_float(vh.x << 16), __uint_as_float(vh.x & 0xffff0000u),
+                                                 __uint_as_float(vh.y << 16), __uint_as_float(vh.y & 0xffff0000u)};
+                            float nl[4], nh[4], pl[4], ph[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {                              // rotation by -phi
+                                nl[e] = fmaf(lo[e], cs[e], hi[e] * sn[e]);
+                                nh[e] = fmaf(hi[e], cs[e], -lo[e] * sn[e]);
+                                pl[e] = wt * nl[e];
+                                ph[e] = wt * nh[e];
+                                sx[e] += pl[e];
+                                sx[4 + e] += ph[e];
+                            }
+                            *reinterpret_cast<uint2 *>(xt + rp_lo + off) = make_uint2(pack_bf16x2(nl[0], nl[1]), pack_bf16x2(nl[2], nl[3]));
+                            *reinterpret_cast<uint2 *>(xt + rp_hi + off) = make_uint2(pack_bf16x2(nh[0], nh[1]), pack_bf16x2(nh[2], nh[3]));
+                            const unsigned hl0 = pack_bf16x2(pl[0], pl[1]), hl1 = pack_bf16x2(pl[2], pl[3]);
+                            const unsigned hh0 = pack_bf16x2(ph[0], ph[1]), hh1 = pack_bf16x2(ph[2], ph[3]);
+                            *reinterpret_cast<uint2 *>(at + rp_lo + off) = make_uint2(hl0, hl1);
+                            *reinterpret_cast<uint2 *>(at + rp_hi + off) = make_uint2(hh0, hh1);
+                            if (COMP) {
+                                *reinterpret_cast<uint2 *>(at + C::A_BYTES + rp_lo + off) = make_uint2(
+                                    pack_bf16x2(pl[0] - __uint_as_float(hl0 << 16), pl[1] - __uint_as_float(hl0 & 0xffff0000u)),
+                                    pack_bf16x2(pl[2] - __uint_as_float(hl1 << 16), pl[3] - __uint_as_float(hl1 & 0xffff0000u)));
+                                *reinterpret_cast<uint2 *>(at + C::A_BYTES + rp_hi + off) = make_uint2(
+                                    pack_bf16x2(ph[0] - __uint_as_float(hh0 << 16), ph[1] - __uint_as_float(hh0 & 0xffff0000u)),
+                                    pack_bf16x2(ph[2] - __uint_as_float(hh1 << 16), ph[3] - __uint_as_float(hh1 & 0xffff0000u)));
+                            }
+                        }
+                        if (!P.rope.same) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) rope_cs(ftgt[e], pos, cs[e], sn[e]);
+                        }
+                        {
+                            const uint2 vl = *reinterpret_cast<const uint2 *>(yt + rp_lo + off);
+                            const uint2 vh = *reinterpret_cast<const uint2 *>(yt + rp_hi + off);
+                            const float lo[4] = {__uint_as_float(vl.x << 16), __uint_as_float(vl.x & 0xffff0000u),
+                                                 __uint_as_float(vl.y << 16), __uint_as_float(vl.y & 0xffff0000u)};
+                            const float hi[4] = {__uint_as_float(vh.x << 16), __uint_as_float(vh.x & 0xffff0000u),
+                                                 __uint_as_float(vh.y << 16), __uint_as_float(vh.y & 0xffff0000u)};
+                            float nl[4], nh[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                nl[e] = fmaf(lo[e], cs[e], hi[e] * sn[e]);
+                                nh[e] = fmaf(hi[e], cs[e], -lo[e] * sn[e]);
+                                sy[e] = fmaf(wt, nl[e], sy[e]);
+                                sy[4 + e] = fmaf(wt, nh[e], sy[4 + e]);
+                            }
+                            *reinterpret_cast<uint2 *>(yt + rp_lo + off) = make_uint2(pack_bf16x2(nl[0], nl[1]), pack_bf16x2(nl[2], nl[3]));
+                            *reinterpret_cast<uint2 *>(yt + rp_hi + off) = make_uint2(pack_bf16x2(nh[0], nh[1]), pack_bf16x2(nh[2], nh[3]));
+                        }
+                        if (cc == 0) sw += wt;
+                    }
+                } else {
 #pragma unroll
                 for (int i = 0; i < C::RPT; ++i) {
                     const int off = i * C::RG * 128;
@@ -481,6 +574,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                     }
                     if (cc == 0) sw += wt;
                 }
+                }
 #endif
                 fence_async_smem();
                 __syncwarp();
@@ -491,7 +585,8 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                 ++it;
             }
 #pragma unroll
-            for (int e = 0; e < 4; ++e) { f2_unpack(sx2[e], sx[2 * e], sx[2 * e + 1]); f2_unpack(sy2[e], sy[2 * e], sy[2 * e + 1]); }
+            for (int e = 0; e < 4; ++e)
+                if (!rope_unit) { f2_unpack(sx2[e], sx[2 * e], sx[2 * e + 1]); f2_unpack(sy2[e], sy[2 * e], sy[2 * e + 1]); }
             // ---- bias sums of this unit: lanes holding the same channels add up, then a fixed-order sum over the
             //      warps, then read-modify-write of the slot ----
             if (C::CC == 16) {
@@ -518,7 +613,12 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
             float *rw = red + fw * C::RED_STRIDE;
             if (lane < C::CC) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) { rw[cc * 8 + e] = sx[e]; rw[D + cc * 8 + e] = sy[e]; }
+                for (int e = 0; e < 8; ++e) {
+                    // ordinary fold: channels 8 cc + e; rotated key units: 4 cc + e and D/2 + 4 cc + (e - 4)
+                    const int ch = rope_unit ? ((e < 4) ? cc * 4 + e : D / 2 + cc * 4 + (e - 4)) : cc * 8 + e;
+                    rw[ch] = sx[e];
+                    rw[D + ch] = sy[e];
+                }
                 if (cc == 0) rw[2 * D] = sw;
             }
             __syncwarp();
@@ -695,19 +795,19 @@ static int sm_count()
     return n;
 }
 
-template <int D, bool COMP, bool FH = false, bool CEN = false>
+template <int D, bool COMP, bool FH = false, bool CEN = false, bool ROPE = false>
 static cudaError_t launch_tc(const TcParams &P, cudaStream_t st)
 {
     using C = TcCfg<D, COMP, FH>;
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D, COMP, FH, CEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D, COMP, FH, CEN, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr = true;
     }
     const int n_units = FH ? 2 * P.a.Lt * (P.fh.per_head ? P.a.Ht : 1) * (P.fh.NG + P.fh.NC) : 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
     const int grid = n_units < sm_count() ? n_units : sm_count();
-    k_accum_tc<D, COMP, FH, CEN><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
+    k_accum_tc<D, COMP, FH, CEN, ROPE><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -728,6 +828,13 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     TcParams P;
     P.a = a;
     P.fh = FhDev{};
+    P.rope = RopeDev{};
+    if (a.rope_pos) {
+        P.rope.pos = a.rope_pos;
+        rope_frequencies(a.rope_base_src, d, P.rope.f_src);
+        rope_frequencies(a.rope_base_tgt, d, P.rope.f_tgt);
+        P.rope.same = (a.rope_base_src == a.rope_base_tgt) ? 1 : 0;
+    }
     const int TT = 64;
     if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
 #ifdef CB_DRAIN_TOKENS
@@ -736,7 +843,10 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     P.drain_tiles = 16384 / TT;   // at most 16384 tokens are summed in tensor memory before a drain
 #endif
     cudaError_t e;
-    if (a.mu) {
+    if (a.rope_pos) {
+        if (a.compensated) e = (d == 128) ? launch_tc<128, true, false, false, true>(P, st) : launch_tc<64, true, false, false, true>(P, st);
+        else e = (d == 128) ? launch_tc<128, false, false, false, true>(P, st) : launch_tc<64, false, false, false, true>(P, st);
+    } else if (a.mu) {
         if (a.compensated) e = (d == 128) ? launch_tc<128, true, false, true>(P, st) : launch_tc<64, true, false, true>(P, st);
         else e = (d == 128) ? launch_tc<128, false, false, true>(P, st) : launch_tc<64, false, false, true>(P, st);
     } else if (a.compensated) e = (d == 128) ? launch_tc<128, true>(P, st) : launch_tc<64, true>(P, st);
@@ -751,6 +861,7 @@ cudaError_t launch_fullhead_tc(const AccumArgs &a, const FullHeadArgs &f, int d,
     TcParams P;
     P.a = a;
     P.fh = FhDev{f.G, f.C, f.layer_sets, f.gi, f.gq, f.src_head, f.F, f.k, f.Hs, f.PF, f.NG, f.NC, f.per_head};
+    P.rope = RopeDev{};
     const int TT = 64;
     if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
     P.drain_tiles = 16384 / TT;

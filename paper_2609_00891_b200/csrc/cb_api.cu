@@ -211,10 +211,21 @@ cb_status cb_stats_reset(cb_ctx *ctx, void *stream)
     return CB_OK;
 }
 
+struct RopeOpt { const int32_t *pos; double base_src, base_tgt; };
+
+static bool rope_base_ok(double b) { return b > 1.0 && b <= 1e12; }
+
 static cb_status accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
                                  const float *w_k, const float *w_v,
-                                 int64_t w_stride_layer, int64_t w_stride_head, const float *mu, bool centred, void *stream)
+                                 int64_t w_stride_layer, int64_t w_stride_head, const float *mu, bool centred, void *stream,
+                                 const RopeOpt *rope = nullptr)
 {
+    if (rope) {
+        if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+        if (!rope_base_ok(rope->base_src) || !rope_base_ok(rope->base_tgt)) return CB_ERR_INVALID_ARG;
+        if (ctx->prob.flags & CB_FLAG_SIMT) return CB_ERR_UNSUPPORTED;
+        if (src && src->n_tokens > 0 && (!rope->pos || ((uintptr_t)rope->pos & 3))) return CB_ERR_INVALID_ARG;
+    }
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
     if (centred && !mu) return CB_ERR_INVALID_ARG;
     if (centred && (ctx->prob.flags & CB_FLAG_SIMT)) return CB_ERR_UNSUPPORTED;
@@ -242,6 +253,7 @@ static cb_status accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const cb_kv
     a.status = reinterpret_cast<int *>(ctx->ws + ctx->lay.status_off);
     a.compensated = (P.flags & CB_FLAG_COMPENSATED) ? 1 : 0;
     a.mu = centred ? mu : nullptr;
+    if (rope) { a.rope_pos = rope->pos; a.rope_base_src = rope->base_src; a.rope_base_tgt = rope->base_tgt; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = (P.flags & CB_FLAG_SIMT) ? launch_accum_simt(a, ctx->d, st)
                                              : launch_accum_tc(a, ctx->d, src, tgt, st);
@@ -255,6 +267,35 @@ cb_status cb_stats_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_vi
                               int64_t w_stride_layer, int64_t w_stride_head, void *stream)
 {
     return accumulate_impl(ctx, src, tgt, w_k, w_v, w_stride_layer, w_stride_head, nullptr, false, stream);
+}
+
+// ---------------------------------------------------------------------------------------------------------------------
+// Rotary embedding at the boundary
+// ---------------------------------------------------------------------------------------------------------------------
+cb_status cb_stats_accumulate_rope(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                   const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                                   const int32_t *positions, double rope_base_src, double rope_base_tgt, void *stream)
+{
+    const RopeOpt r{positions, rope_base_src, rope_base_tgt};
+    return accumulate_impl(ctx, src, tgt, w_k, w_v, w_stride_layer, w_stride_head, nullptr, false, stream, &r);
+}
+
+cb_status cb_rope_rotate(void *k, int32_t n_layers, int32_t n_heads, int32_t head_dim, int64_t n_tokens,
+                         int64_t stride_layer, int64_t stride_token, int64_t stride_head,
+                         const int32_t *positions, double rope_base, int32_t inverse, void *stream)
+{
+    if (n_layers <= 0 || n_heads <= 0 || n_tokens < 0) return CB_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return CB_ERR_UNSUPPORTED;
+    if (n_tokens >= (1ll << 31) || (long long)n_layers * n_heads > 65535) return CB_ERR_UNSUPPORTED;
+    if (!rope_base_ok(rope_base)) return CB_ERR_INVALID_ARG;
+    if (n_tokens == 0) return CB_OK;
+    if (!k || ((uintptr_t)k & 15) || !positions || ((uintptr_t)positions & 3)) return CB_ERR_INVALID_ARG;
+    if (stride_layer < 0 || stride_token <= 0 || stride_head < 0) return CB_ERR_INVALID_ARG;
+    if ((stride_layer | stride_token | stride_head) & 7) return CB_ERR_INVALID_ARG;
+    cudaError_t e = launch_rope_rotate(k, n_layers, n_heads, head_dim, n_tokens, stride_layer, stride_token, stride_head,
+                                       positions, rope_base, inverse ? 1 : 0, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
 }
 
 // ---------------------------------------------------------------------------------------------------------------------

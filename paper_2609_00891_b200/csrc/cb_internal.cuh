@@ -43,6 +43,10 @@ struct AccumArgs {
     // When set, the weighted operand is w (x - mu_x) and the slot's s_x entries receive the sum of the ROUNDED
     // weighted operand (the exact correction term of the reduction), s_y stays zero.
     const float *mu = nullptr;
+    // Rotary embedding at the boundary: device [n_tokens] positions (null: keys are taken as stored) and the rotary
+    // bases of the two models.  Key maps are then fitted on de-rotated source and target keys.
+    const int *rope_pos = nullptr;
+    double rope_base_src = 0.0, rope_base_tgt = 0.0;
 };
 
 // First pass of the two-pass construction: fp64 partial sums [n_msplits][n_maps][means_stride(d)] = sum w x, sum w y, sum w.
@@ -103,6 +107,9 @@ cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cu
 size_t apply_ml_workspace_bytes(int n_maps, int k, int d, int Lt);
 cudaError_t launch_apply_ml_tc(const ApplyArgs &a, int d, int k, const int *layer_sets_host, const cb_kv_view *src,
                                void *workspace, cudaStream_t st);
+
+cudaError_t launch_rope_rotate(void *k, int L, int H, int d, long long T, long long sl, long long st, long long sh,
+                               const int *pos, double base, int inverse, cudaStream_t stream);
 
 void count_launch(int n = 1);
 
