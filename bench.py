@@ -297,13 +297,21 @@ def main():
         out_k = torch.empty(wl.Lt, T, wl.Ht, d, dtype=torch.bfloat16, device=dev)
         out_v = torch.empty_like(out_k)
         Wfull = full[min(1, nl - 1)].contiguous()
+        apos = torch.arange(T, dtype=torch.int32, device=dev)
+
+        def do_apply():
+            if args.rope:
+                cb.cb_apply_rope(prob, Wfull, src[0], src[1], out_k, out_v, apos, 1e6, 1e6)
+            else:
+                cb.cb_apply(prob, Wfull, src[0], src[1], out_k, out_v)
+
         for _ in range(3):
-            cb.cb_apply(prob, Wfull, src[0], src[1], out_k, out_v)
+            do_apply()
         ts = []
         for _ in range(5):
             e0, e1 = ev(), ev()
             e0.record()
-            cb.cb_apply(prob, Wfull, src[0], src[1], out_k, out_v)
+            do_apply()
             e1.record()
             e1.synchronize()
             ts.append(e0.elapsed_time(e1))

@@ -337,6 +337,17 @@ cb_status cb_stats_accumulate_rope(cb_ctx *ctx, const cb_kv_view *src, const cb_
 cb_status cb_rope_rotate(void *k, int32_t n_layers, int32_t n_heads, int32_t head_dim, int64_t n_tokens,
                          int64_t stride_layer, int64_t stride_token, int64_t stride_head,
                          const int32_t *positions, double rope_base, int32_t inverse, void *stream);
+/*
+ * cb_apply_rope: as cb_apply, for a source cache whose keys carry the source model's rotary embedding and a target
+ * cache that must carry the target model's:  K_out[l][t][h] = R_tgt(pos_t) ( R_src(-pos_t) x_t W + b ),  values as in
+ * cb_apply.  Both rotations run inside the apply kernel (the staged source tile is rotated on chip, the mapped rows in
+ * the epilogue).  The de-rotated keys enter the tensor cores as fp16 (11 significant bits; magnitudes above 65504
+ * are clamped) with W split into fp16 hi + lo.  Not available with CB_FLAG_SIMT.
+ */
+cb_status cb_apply_rope(const cb_problem *prob, const float *Wb, const cb_kv_view *src_cache,
+                        void *tgt_k, void *tgt_v, int64_t t_stride_layer, int64_t t_stride_token,
+                        int64_t t_stride_head, int32_t out_dtype,
+                        const int32_t *positions, double rope_base_src, double rope_base_tgt, void *stream);
 
 /*
  * Synchronises the stream and reads the context's device status word: CB_OK, or CB_ERR_TIMEOUT if a bounded

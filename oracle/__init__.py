@@ -265,6 +265,17 @@ def rope_rotate(x: np.ndarray, pos: np.ndarray, base: float, inverse: bool = Fal
     return out
 
 
+def apply_rope_rows(x_bits: np.ndarray, Theta: np.ndarray, pos: np.ndarray, base_src: float, base_tgt: float) -> np.ndarray:
+    """Key rows through a map in content coordinates (Section 3.1): remove the source model's rotary embedding, apply
+    y = x W + b, restore the target model's.  x_bits [n][d] bf16 bit patterns, Theta [d+1][d] (W then b); fp64 out."""
+    x = bf16_decode(np.ascontiguousarray(x_bits)).reshape(x_bits.shape)
+    d = x.shape[1]
+    Theta = np.asarray(Theta, dtype=np.float64)
+    content = rope_rotate(x, pos, base_src, inverse=True)
+    mapped = content @ Theta[:d] + Theta[d]
+    return rope_rotate(mapped, pos, base_tgt, inverse=False)
+
+
 # ----------------------------------------------------------------------------- apply
 def apply_maps(src_k: np.ndarray, src_v: np.ndarray, Theta: np.ndarray, Lt: int, Ht: int,
                src_layer: np.ndarray, src_head: np.ndarray, maps: Optional[Sequence[int]] = None,

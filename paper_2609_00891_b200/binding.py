@@ -30,7 +30,7 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_multilayer_stats_accumulate", "cb_apply_multilayer_workspace_bytes", "cb_apply_multilayer",
            "cb_means_workspace_bytes", "cb_means_reset", "cb_means_accumulate", "cb_means_finalize",
            "cb_stats_accumulate_centered", "cb_stats_reduce_centered", "cb_ridge_solve_centered",
-           "cb_stats_accumulate_rope", "cb_rope_rotate",
+           "cb_stats_accumulate_rope", "cb_rope_rotate", "cb_apply_rope",
            "cb_launch_count")
 
 
@@ -381,6 +381,24 @@ def cb_apply(prob: Problem, Wb: torch.Tensor, src_k: torch.Tensor, src_v: torch.
                           ctypes.c_void_p(tgt_k.data_ptr()), ctypes.c_void_p(tgt_v.data_ptr()),
                           ctypes.c_int64(tgt_k.stride(0)), ctypes.c_int64(tgt_k.stride(1)),
                           ctypes.c_int64(tgt_k.stride(2)), dt, _stream_ptr(stream)), "cb_apply")
+
+
+def cb_apply_rope(prob: Problem, Wb: torch.Tensor, src_k: torch.Tensor, src_v: torch.Tensor,
+                  tgt_k: torch.Tensor, tgt_v: torch.Tensor, positions: torch.Tensor,
+                  rope_base_src: float, rope_base_tgt: float, stream=None) -> None:
+    """As cb_apply for caches whose keys carry rotary embeddings; `positions` is a device int32 tensor [T]."""
+    sv = _kv_view(src_k, src_v)
+    assert Wb.dtype == torch.float32 and Wb.is_contiguous()
+    assert tgt_k.dtype == tgt_v.dtype and tgt_k.stride() == tgt_v.stride() and tgt_k.stride(3) == 1
+    assert positions.dtype == torch.int32 and positions.is_cuda and positions.is_contiguous()
+    assert positions.numel() == src_k.shape[1]
+    dt = {torch.bfloat16: CB_DTYPE_BF16, torch.float32: CB_DTYPE_F32}[tgt_k.dtype]
+    _check(lib().cb_apply_rope(ctypes.byref(prob.c), ctypes.c_void_p(Wb.data_ptr()), ctypes.byref(sv),
+                               ctypes.c_void_p(tgt_k.data_ptr()), ctypes.c_void_p(tgt_v.data_ptr()),
+                               ctypes.c_int64(tgt_k.stride(0)), ctypes.c_int64(tgt_k.stride(1)),
+                               ctypes.c_int64(tgt_k.stride(2)), dt, ctypes.c_void_p(positions.data_ptr()),
+                               ctypes.c_double(rope_base_src), ctypes.c_double(rope_base_tgt), _stream_ptr(stream)),
+           "cb_apply_rope")
 
 
 def cb_stats_build_static(prob: Problem, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor, w_v: torch.Tensor,

@@ -538,13 +538,18 @@ cb_status cb_check_info(const int32_t *info, int64_t n, void *stream, int64_t *f
     return CB_OK;
 }
 
-cb_status cb_apply(const cb_problem *prob, const float *Wb, const cb_kv_view *src_cache,
-                   void *tgt_k, void *tgt_v, int64_t t_stride_layer, int64_t t_stride_token,
-                   int64_t t_stride_head, int32_t out_dtype, void *stream)
+static cb_status apply_impl(const cb_problem *prob, const float *Wb, const cb_kv_view *src_cache,
+                            void *tgt_k, void *tgt_v, int64_t t_stride_layer, int64_t t_stride_token,
+                            int64_t t_stride_head, int32_t out_dtype, void *stream, const RopeOpt *rope)
 {
     cb_status s = check_problem(prob);
     if (s != CB_OK) return s;
     if (prob->Lt > 128 || prob->Ht > 64) return CB_ERR_UNSUPPORTED;
+    if (rope) {
+        if (!rope_base_ok(rope->base_src) || !rope_base_ok(rope->base_tgt)) return CB_ERR_INVALID_ARG;
+        if (prob->flags & CB_FLAG_SIMT) return CB_ERR_UNSUPPORTED;
+        if (src_cache && src_cache->n_tokens > 0 && (!rope->pos || ((uintptr_t)rope->pos & 3))) return CB_ERR_INVALID_ARG;
+    }
     s = check_view(src_cache, prob->Ls, prob->Hs, prob->ds);
     if (s != CB_OK) return s;
     if (out_dtype != CB_DTYPE_BF16 && out_dtype != CB_DTYPE_F32) return CB_ERR_INVALID_ARG;
@@ -566,11 +571,29 @@ cb_status cb_apply(const cb_problem *prob, const float *Wb, const cb_kv_view *sr
     std::memset(a.src_head, 0, sizeof a.src_head);
     for (int l = 0; l < prob->Lt; ++l) a.src_layer[l] = prob->src_layer[l];
     for (int h = 0; h < prob->Ht; ++h) a.src_head[h] = prob->src_head[h];
+    if (rope) { a.rope_pos = rope->pos; a.rope_base_src = rope->base_src; a.rope_base_tgt = rope->base_tgt; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = (prob->flags & CB_FLAG_SIMT) ? launch_apply_simt(a, prob->ds, st)
                                                  : launch_apply_tc(a, prob->ds, src_cache, st);
     if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     return CB_OK;
+}
+
+cb_status cb_apply(const cb_problem *prob, const float *Wb, const cb_kv_view *src_cache,
+                   void *tgt_k, void *tgt_v, int64_t t_stride_layer, int64_t t_stride_token,
+                   int64_t t_stride_head, int32_t out_dtype, void *stream)
+{
+    return apply_impl(prob, Wb, src_cache, tgt_k, tgt_v, t_stride_layer, t_stride_token, t_stride_head, out_dtype, stream,
+                      nullptr);
+}
+
+cb_status cb_apply_rope(const cb_problem *prob, const float *Wb, const cb_kv_view *src_cache,
+                        void *tgt_k, void *tgt_v, int64_t t_stride_layer, int64_t t_stride_token,
+                        int64_t t_stride_head, int32_t out_dtype,
+                        const int32_t *positions, double rope_base_src, double rope_base_tgt, void *stream)
+{
+    const RopeOpt r{positions, rope_base_src, rope_base_tgt};
+    return apply_impl(prob, Wb, src_cache, tgt_k, tgt_v, t_stride_layer, t_stride_token, t_stride_head, out_dtype, stream, &r);
 }
 
 cb_status cb_fullhead_layer_sets(int32_t Ls, int32_t Lt, int32_t k, int32_t *layer_sets)

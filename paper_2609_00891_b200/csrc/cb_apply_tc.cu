@@ -13,8 +13,11 @@
 // no context to carry a status word).
 #include <cudaTypedefs.h>
 
+#include <cuda_fp16.h>
+
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
+#include "cb_rope.cuh"
 
 #ifndef CB_AP_NS
 #define CB_AP_NS 3
@@ -55,6 +58,7 @@ struct ApParams {
     CUtensorMap src_k, src_v, out_k, out_v;
     ApplyArgs a;
     int n_splits;
+    RopeDev rope;        // ROPE kernels only
 };
 
 struct ApIter {   // units u = blockIdx.x, += gridDim.x; unit -> (map, split) -> tiles [tile, tile1)
@@ -91,7 +95,21 @@ __device__ __forceinline__ unsigned ap_pack_bf16x2(float lo, float hi)
     return r;
 }
 
-template <int D>
+// fp16 pair (low half = first element), clamped to the finite fp16 range
+__device__ __forceinline__ unsigned ap_pack_f16x2(float lo, float hi)
+{
+    lo = fminf(fmaxf(lo, -65504.f), 65504.f);
+    hi = fminf(fmaxf(hi, -65504.f), 65504.f);
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const unsigned *>(&h);
+}
+
+// ROPE (Section 3.1: source RoPE removed before the map, target RoPE restored after it): for key maps (comp = 0) the
+// conversion warps rotate every staged source tile back by its rows' angles in place, writing fp16 (the rotated
+// values are no longer bf16 numbers: fp16 keeps 11 significant bits, and W is split into fp16 hi + lo to match), the
+// tensor cores run with fp16 operands, and the epilogue rotates the mapped rows forward by the target model's angles.
+// Value maps take the ordinary bf16 path through the same barriers.
+template <int D, bool ROPE>
 __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_constant__ ApParams P)
 {
     using C = ApCfg<D>;
@@ -112,7 +130,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
     uint64_t *bfree = wfree + 1;             // [1]    bias of the unit no longer needed (EPI_WARPS arrivals)
     uint64_t *owritten = bfree + 1;          // [NO]   output tile written by all epilogue warps
     uint64_t *ofree = owritten + C::NO;      // [NO]   output tile read by its store
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ofree + C::NO);
+    uint64_t *xrot = ofree + C::NO;          // [NS]   ROPE: source tile ready for the tensor cores (CONV_WARPS arrivals)
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(xrot + C::NS);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const ApplyArgs &a = P.a;
@@ -123,7 +142,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
     const bool out_bf16 = a.out_dtype == CB_DTYPE_BF16;
 
     if (tid == 0) {
-        for (int i = 0; i < C::NS; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 1); }
+        for (int i = 0; i < C::NS; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 1); mbar_init(&xrot[i], C::CONV_WARPS); }
         for (int i = 0; i < C::NACC; ++i) { mbar_init(&accfull[i], 1); mbar_init(&accempty[i], C::EPI_WARPS); }
         mbar_init(wready, C::CONV_WARPS);
         mbar_init(wfree, 1);
@@ -163,7 +182,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
     } else if (warp == 1) {
         // ================================ MMA issuer (one thread) ================================
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(128, D, false, true);   // A K-major, B MN-major
+            constexpr uint32_t idesc_bf = umma_idesc_bf16(128, D, false, true);   // A K-major, B MN-major
+            constexpr uint32_t idesc_hf = umma_idesc_f16(128, D, false, true);
             // A (K-major, 128-byte swizzle): 8-row groups 1024 bytes apart; a K step of 16 channels is 32 bytes along
             // the row, a block of 64 channels is XBLK further.  B (MN-major): K step = 16 rows = 2048 bytes,
             // 64-output-channel blocks WBLK apart.
@@ -180,8 +200,10 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
             uint32_t uc = 0;
             while (cur.u < n_units) {
                 if (!mbar_wait(wready, uc & 1, abort_flag)) goto teardown;
+                const uint32_t idesc = (ROPE && cur.m < a.Lt * a.Ht) ? idesc_hf : idesc_bf;   // key maps of a ROPE launch: fp16
                 for (int tile = cur.tile; tile < cur.tile1; ++tile) {
-                    if (!mbar_wait(&xfull[st.idx], st.phase, abort_flag)) goto teardown;
+                    // ROPE launches: every tile passes through the conversion warps (which rotate key tiles)
+                    if (!mbar_wait(ROPE ? &xrot[st.idx] : &xfull[st.idx], st.phase, abort_flag)) goto teardown;
                     if (!mbar_wait(&accempty[ac.idx], ac.phase ^ 1, abort_flag)) goto teardown;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + ac.idx * D;
@@ -225,7 +247,69 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ac.idx * D;
                 const int tok = tile * C::TT + row;
-                if (out_bf16) {
+                const bool rope_unit = ROPE && comp == 0;
+                if (rope_unit) {
+                    // forward rotation by the target model's angles: columns i and i + D/2 are a pair
+                    const int pos = (tok < a.n_tokens) ? __ldg(P.rope.pos + tok) : 0;
+                    uint8_t *ot = os + (size_t)ob.idx * C::O_BYTES;
+                    float *orow = reinterpret_cast<float *>(a.out_k) + (long long)l * a.o_sl + (long long)tok * a.o_st + (long long)h * a.o_sh;
+                    if (out_bf16 && !mbar_wait_warp(&ofree[ob.idx], ob.phase ^ 1, abort_flag, lane)) goto teardown;
+#pragma unroll 1
+                    for (int c = 0; c < D / 64; ++c) {
+                        uint32_t rl[32], rh[32];
+                        tmem_ld_32x32(taddr + c * 32, rl);
+                        tmem_ld_32x32(taddr + D / 2 + c * 32, rh);
+                        tmem_wait_ld();
+                        float ol[32], oh[32];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int i = c * 32 + j;
+                            float cs, sn;
+                            rope_cs(P.rope.f_tgt[i], pos, cs, sn);
+                            const float vl = __uint_as_float(rl[j]) + bias[i], vh = __uint_as_float(rh[j]) + bias[D / 2 + i];
+                            ol[j] = fmaf(vl, cs, -vh * sn);
+                            oh[j] = fmaf(vl, sn, vh * cs);
+                        }
+                        if (out_bf16) {
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                const int nl = c * 32 + v * 8, nh = D / 2 + nl;
+                                const uint4 pl = make_uint4(ap_pack_bf16x2(ol[v * 8 + 0], ol[v * 8 + 1]), ap_pack_bf16x2(ol[v * 8 + 2], ol[v * 8 + 3]),
+                                                            ap_pack_bf16x2(ol[v * 8 + 4], ol[v * 8 + 5]), ap_pack_bf16x2(ol[v * 8 + 6], ol[v * 8 + 7]));
+                                const uint4 ph = make_uint4(ap_pack_bf16x2(oh[v * 8 + 0], oh[v * 8 + 1]), ap_pack_bf16x2(oh[v * 8 + 2], oh[v * 8 + 3]),
+                                                            ap_pack_bf16x2(oh[v * 8 + 4], oh[v * 8 + 5]), ap_pack_bf16x2(oh[v * 8 + 6], oh[v * 8 + 7]));
+                                *reinterpret_cast<uint4 *>(ot + (nl >> 6) * C::XBLK + row * 128 + ((((nl & 63) >> 3) ^ (row & 7)) << 4)) = pl;
+                                *reinterpret_cast<uint4 *>(ot + (nh >> 6) * C::XBLK + row * 128 + ((((nh & 63) >> 3) ^ (row & 7)) << 4)) = ph;
+                            }
+                        } else if (tok < a.n_tokens) {
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) {
+                                *reinterpret_cast<float4 *>(orow + c * 32 + v * 4) = make_float4(ol[v * 4], ol[v * 4 + 1], ol[v * 4 + 2], ol[v * 4 + 3]);
+                                *reinterpret_cast<float4 *>(orow + D / 2 + c * 32 + v * 4) = make_float4(oh[v * 4], oh[v * 4 + 1], oh[v * 4 + 2], oh[v * 4 + 3]);
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    if (out_bf16) fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) { mbar_arrive(&accempty[ac.idx]); if (out_bf16) mbar_arrive(&owritten[ob.idx]); }
+                    if (out_bf16) {
+                        if (storer) {
+                            if (mbar_wait(&owritten[ob.idx], ob.phase, abort_flag)) {
+                                tma_store_5d(omap, ot, 0, tile * C::TT, 0, h, l);
+                                tma_store_commit();
+                                if (pending == C::NO - 1) {
+                                    tma_store_wait_read_keep<C::NO - 1>();
+                                    mbar_arrive(&ofree[oldest.idx]);
+                                    oldest.next();
+                                } else {
+                                    ++pending;
+                                }
+                            }
+                        }
+                        ob.next();
+                    }
+                } else if (out_bf16) {
                     uint8_t *ot = os + (size_t)ob.idx * C::O_BYTES;
                     if (!mbar_wait_warp(&ofree[ob.idx], ob.phase ^ 1, abort_flag, lane)) goto teardown;
 #pragma unroll 1
@@ -301,8 +385,18 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         ApIter cur;
         cur.start(n_units, n_maps, n_tiles, P.n_splits);
         uint32_t uc = 0;
+        ApRing<C::NS> st;                                             // ROPE: follows the producer's ring
+        // ROPE: this thread rotates the pair of 16-byte chunks (lc, lc + half a row) of rows r0, r0 + RP, ..
+        constexpr int HC = D / 16, RP = CT / HC;
+        const int lc = ct % HC, r0 = ct / HC;
+        uint32_t fsrc[8];
+        if (ROPE) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) fsrc[e] = P.rope.f_src[lc * 8 + e];
+        }
         while (cur.u < n_units) {
             const float *Wm = a.Wb + (size_t)cur.m * (D + 1) * D;
+            const bool rope_unit = ROPE && cur.m < a.Lt * a.Ht;
             // the previous unit's last MMA has read W, and its epilogues have read the bias
             if (!mbar_wait_warp(wfree, (uc & 1) ^ 1, abort_flag, lane)) goto teardown;
             if (!mbar_wait_warp(bfree, (uc & 1) ^ 1, abort_flag, lane)) goto teardown;
@@ -314,6 +408,12 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                 unsigned hi[4], lo[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
+                    if (rope_unit) {                                  // fp16 hi + lo
+                        hi[e] = ap_pack_f16x2(f[2 * e], f[2 * e + 1]);
+                        const float2 hf = __half22float2(*reinterpret_cast<const __half2 *>(&hi[e]));
+                        lo[e] = ap_pack_f16x2(f[2 * e] - hf.x, f[2 * e + 1] - hf.y);
+                        continue;
+                    }
                     hi[e] = ap_pack_bf16x2(f[2 * e], f[2 * e + 1]);
                     const float h0 = __uint_as_float(hi[e] << 16), h1 = __uint_as_float(hi[e] & 0xffff0000u);
                     lo[e] = ap_pack_bf16x2(f[2 * e] - h0, f[2 * e + 1] - h1);
@@ -327,6 +427,42 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
             __syncwarp();
             if (lane == 0) mbar_arrive(wready);
             ++uc;
+            if (ROPE) {
+                for (int tile = cur.tile; tile < cur.tile1; ++tile) {
+                    if (!mbar_wait_warp(&xfull[st.idx], st.phase, abort_flag, lane)) goto teardown;
+                    if (rope_unit) {
+                        uint8_t *xt = xs + st.idx * C::X_BYTES;
+#pragma unroll 2
+                        for (int r = r0; r < C::TT; r += RP) {
+                            const int tok = tile * C::TT + r;
+                            const int pos = (tok < a.n_tokens) ? __ldg(P.rope.pos + tok) : 0;
+                            const int olo = r * 128 + ((lc ^ (r & 7)) << 4);
+                            const int ohi = (D == 128) ? C::XBLK + olo : r * 128 + (((lc + 4) ^ (r & 7)) << 4);
+                            const uint4 vl = *reinterpret_cast<const uint4 *>(xt + olo);
+                            const uint4 vh = *reinterpret_cast<const uint4 *>(xt + ohi);
+                            const unsigned ul[4] = {vl.x, vl.y, vl.z, vl.w}, uh[4] = {vh.x, vh.y, vh.z, vh.w};
+                            unsigned wl[4], wh[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                float c0, s0, c1, s1;
+                                rope_cs(fsrc[2 * e], pos, c0, s0);
+                                rope_cs(fsrc[2 * e + 1], pos, c1, s1);
+                                const float l0 = __uint_as_float(ul[e] << 16), l1 = __uint_as_float(ul[e] & 0xffff0000u);
+                                const float h0 = __uint_as_float(uh[e] << 16), h1 = __uint_as_float(uh[e] & 0xffff0000u);
+                                // rotation by -phi
+                                wl[e] = ap_pack_f16x2(fmaf(l0, c0, h0 * s0), fmaf(l1, c1, h1 * s1));
+                                wh[e] = ap_pack_f16x2(fmaf(h0, c0, -l0 * s0), fmaf(h1, c1, -l1 * s1));
+                            }
+                            *reinterpret_cast<uint4 *>(xt + olo) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                            *reinterpret_cast<uint4 *>(xt + ohi) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                        }
+                        fence_async_smem();
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&xrot[st.idx]);
+                    st.next();
+                }
+            }
             cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
         }
     }
@@ -356,19 +492,19 @@ static int ap_sm_count()
     return n;
 }
 
-template <int D>
+template <int D, bool ROPE>
 static cudaError_t launch_ap(const ApParams &P, cudaStream_t st)
 {
     using C = ApCfg<D>;
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_apply_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(k_apply_tc<D, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr = true;
     }
     const int n_units = 2 * P.a.Lt * P.a.Ht * P.n_splits;
     const int grid = n_units < ap_sm_count() ? n_units : ap_sm_count();
-    k_apply_tc<D><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
+    k_apply_tc<D, ROPE><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -396,7 +532,17 @@ cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cu
         P.out_k = P.src_k;   // unused for fp32 output
         P.out_v = P.src_v;
     }
-    cudaError_t e = (d == 128) ? launch_ap<128>(P, st) : launch_ap<64>(P, st);
+    P.rope = RopeDev{};
+    cudaError_t e;
+    if (a.rope_pos) {
+        P.rope.pos = a.rope_pos;
+        rope_frequencies(a.rope_base_src, d, P.rope.f_src);
+        rope_frequencies(a.rope_base_tgt, d, P.rope.f_tgt);
+        P.rope.same = (a.rope_base_src == a.rope_base_tgt) ? 1 : 0;
+        e = (d == 128) ? launch_ap<128, true>(P, st) : launch_ap<64, true>(P, st);
+    } else {
+        e = (d == 128) ? launch_ap<128, false>(P, st) : launch_ap<64, false>(P, st);
+    }
     if (e == cudaSuccess) count_launch();
     return e;
 }

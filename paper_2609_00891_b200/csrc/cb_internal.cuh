@@ -73,6 +73,9 @@ struct ApplyArgs {
     int Lt, Ht;
     int src_layer[128];    // by value: cb_apply takes no context
     int src_head[64];
+    // Rotary embedding at the boundary (key maps): device [n_tokens] positions, or null for the ordinary apply.
+    const int *rope_pos = nullptr;
+    double rope_base_src = 0.0, rope_base_tgt = 0.0;
 };
 
 // Full-head contrast statistics: outputs and device tables (see cb_fullhead_stats_accumulate).

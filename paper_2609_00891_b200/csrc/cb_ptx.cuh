@@ -224,5 +224,15 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, bool a_mn_m
            | ((uint32_t)(M >> 4) << 24);
 }
 
+// The same with fp16 operands (format code 0 for A and B).
+__host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N, bool a_mn_major, bool b_mn_major)
+{
+    return (1u << 4)                         // accumulator format: fp32
+           | ((a_mn_major ? 1u : 0u) << 15)  // A major
+           | ((b_mn_major ? 1u : 0u) << 16)  // B major
+           | ((uint32_t)(N >> 3) << 17)
+           | ((uint32_t)(M >> 4) << 24);
+}
+
 }  // namespace ptx
 }  // namespace cb

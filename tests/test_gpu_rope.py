@@ -159,3 +159,66 @@ def test_argument_errors():
     with pytest.raises(cb.CbError) as e:
         cb.cb_stats_accumulate_rope(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"], pos, 0.5, 1e6)
     assert e.value.status == cb.CB_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("name,T,bases,out_dtype", [("mini_scaled", 300, (1e6, 1e6), torch.float32),
+                                                     ("mini_scaled", 300, (1e6, 1e4), torch.bfloat16),
+                                                     ("tiny", 129, (1e4, 5e5), torch.float32),
+                                                     ("mini_scaled", 1, (1e6, 1e6), torch.bfloat16)])
+def test_apply_in_content_coordinates(name, T, bases, out_dtype):
+    wl = synth.workload(name)
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    d, p = wl.d, wl.d + 1
+    g = torch.Generator().manual_seed(5)
+    src_k = torch.randn(wl.Ls, T, wl.Hs, d, generator=g).to(torch.bfloat16)
+    src_v = torch.randn(wl.Ls, T, wl.Hs, d, generator=g).to(torch.bfloat16)
+    Wb = (torch.randn(wl.n_maps, p, d, generator=g) / np.sqrt(d)).float()
+    pos = torch.randint(0, 32768, (T,), generator=g, dtype=torch.int32)
+    prob = cb.Problem(wl.Ls, wl.Hs, d, wl.Lt, wl.Ht, d, sl, sh)
+    out_k = torch.full((wl.Lt, T, wl.Ht, d), float("nan"), dtype=out_dtype, device=DEV)
+    out_v = torch.full_like(out_k, float("nan"))
+    cb.cb_apply_rope(prob, Wb.to(DEV), src_k.to(DEV), src_v.to(DEV), out_k, out_v, pos.to(DEV), bases[0], bases[1])
+    torch.cuda.synchronize()
+    # values: identical to the ordinary apply
+    ref_k = torch.empty_like(out_k)
+    ref_v = torch.empty_like(out_v)
+    cb.cb_apply(prob, Wb.to(DEV), src_k.to(DEV), src_v.to(DEV), ref_k, ref_v)
+    assert torch.equal(out_v, ref_v)
+    got = out_k.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    Th = Wb.numpy().astype(np.float64)
+    worst = 0.0
+    for l in range(wl.Lt):
+        for h in range(wl.Ht):
+            m = l * wl.Ht + h                                    # key maps come first
+            want = oracle.apply_rope_rows(bits(src_k[sl[l], :, sh[h], :].contiguous()), Th[m], pos.numpy(), *bases)
+            if out_dtype == torch.bfloat16:
+                ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 2.0 ** -120))) - 7)
+                assert (np.abs(got[l, :, h, :] - want) <= 0.5 * ulp + 2e-3 * np.abs(want).max()).all()
+                worst = max(worst, rel_fro(got[l, :, h, :], want))
+            else:
+                worst = max(worst, rel_fro(got[l, :, h, :], want))
+    print("apply with rope %s T=%d %s: worst map rel err %.2e" % (name, T, out_dtype, worst))
+    # fp16 operands (11 significant bits) and the 2.4e-5 rad angle grid: well inside the 1e-3 target; bf16 output adds
+    # its own rounding (~1.6e-3 rms per element)
+    assert worst <= (1e-3 if out_dtype == torch.float32 else 3e-3)
+
+
+def test_apply_identity_map_turns_source_embedding_into_target_embedding():
+    """W = I, b = 0: the output keys are the source keys re-embedded with the target base (and exactly the source
+    keys when the bases agree, up to the fp16 / bf16 roundings on the way)."""
+    wl = synth.workload("mini_scaled")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    d, p, T = wl.d, wl.d + 1, 200
+    g = torch.Generator().manual_seed(6)
+    src_k = torch.randn(wl.Ls, T, wl.Hs, d, generator=g).to(torch.bfloat16)
+    Wb = torch.zeros(wl.n_maps, p, d)
+    Wb[:, :d, :] = torch.eye(d)
+    pos = torch.arange(T, dtype=torch.int32) * 7
+    prob = cb.Problem(wl.Ls, wl.Hs, d, wl.Lt, wl.Ht, d, sl, sh)
+    out_k = torch.empty(wl.Lt, T, wl.Ht, d, dtype=torch.float32, device=DEV)
+    out_v = torch.empty_like(out_k)
+    cb.cb_apply_rope(prob, Wb.to(DEV), src_k.to(DEV), src_k.to(DEV), out_k, out_v, pos.to(DEV), 1e6, 1e6)
+    for l in range(wl.Lt):
+        for h in range(wl.Ht):
+            assert rel_fro(out_k[l, :, h, :].cpu().numpy(), src_k[sl[l], :, sh[h], :].float().numpy()) < 5e-4
