@@ -341,8 +341,9 @@ cb_status cb_rope_rotate(void *k, int32_t n_layers, int32_t n_heads, int32_t hea
  * cb_apply_rope: as cb_apply, for a source cache whose keys carry the source model's rotary embedding and a target
  * cache that must carry the target model's:  K_out[l][t][h] = R_tgt(pos_t) ( R_src(-pos_t) x_t W + b ),  values as in
  * cb_apply.  Both rotations run inside the apply kernel (the staged source tile is rotated on chip, the mapped rows in
- * the epilogue).  The de-rotated keys enter the tensor cores as fp16 (11 significant bits; magnitudes above 65504
- * are clamped) with W split into fp16 hi + lo.  Not available with CB_FLAG_SIMT.
+ * the epilogue).  The de-rotated keys enter the tensor cores as fp16 (11 significant bits; key magnitudes must stay
+ * below 65504, the fp16 range, which bf16 caches of normalised keys do by orders of magnitude) with W split into fp16
+ * hi + lo.  Not available with CB_FLAG_SIMT.
  */
 cb_status cb_apply_rope(const cb_problem *prob, const float *Wb, const cb_kv_view *src_cache,
                         void *tgt_k, void *tgt_v, int64_t t_stride_layer, int64_t t_stride_token,

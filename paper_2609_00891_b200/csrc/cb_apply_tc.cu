@@ -95,11 +95,9 @@ __device__ __forceinline__ unsigned ap_pack_bf16x2(float lo, float hi)
     return r;
 }
 
-// fp16 pair (low half = first element), clamped to the finite fp16 range
+// fp16 pair (low half = first element)
 __device__ __forceinline__ unsigned ap_pack_f16x2(float lo, float hi)
 {
-    lo = fminf(fmaxf(lo, -65504.f), 65504.f);
-    hi = fminf(fmaxf(hi, -65504.f), 65504.f);
     const __half2 h = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<const unsigned *>(&h);
 }
@@ -386,13 +384,20 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         cur.start(n_units, n_maps, n_tiles, P.n_splits);
         uint32_t uc = 0;
         ApRing<C::NS> st;                                             // ROPE: follows the producer's ring
-        // ROPE: this thread rotates the pair of 16-byte chunks (lc, lc + half a row) of rows r0, r0 + RP, ..
-        constexpr int HC = D / 16, RP = CT / HC;
-        const int lc = ct % HC, r0 = ct / HC;
+        // ROPE: this thread rotates the pair of 16-byte chunks (lc, lc + half a row) of RB consecutive rows.  Along
+        // consecutive positions the angle of a frequency advances by a fixed step, so (cos, sin) of the next row follow
+        // from the current ones by one rotation with the thread's constants (cos, sin)(theta_i); the special-function
+        // unit is only needed at the first row and where the positions do not advance by one.
+        constexpr int HC = D / 16, RB = C::TT / (CT / HC);
+        const int lc = ct % HC, r0 = (ct / HC) * RB;
         uint32_t fsrc[8];
+        float stc[8], sts[8];
         if (ROPE) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) fsrc[e] = P.rope.f_src[lc * 8 + e];
+            for (int e = 0; e < 8; ++e) {
+                fsrc[e] = P.rope.f_src[lc * 8 + e];
+                rope_cs(fsrc[e], 1, stc[e], sts[e]);
+            }
         }
         while (cur.u < n_units) {
             const float *Wm = a.Wb + (size_t)cur.m * (D + 1) * D;
@@ -432,10 +437,25 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                     if (!mbar_wait_warp(&xfull[st.idx], st.phase, abort_flag, lane)) goto teardown;
                     if (rope_unit) {
                         uint8_t *xt = xs + st.idx * C::X_BYTES;
-#pragma unroll 2
-                        for (int r = r0; r < C::TT; r += RP) {
+                        float cs[8], sn[8];
+                        int prev = 0;
+#pragma unroll 1
+                        for (int i = 0; i < RB; ++i) {
+                            const int r = r0 + i;
                             const int tok = tile * C::TT + r;
                             const int pos = (tok < a.n_tokens) ? __ldg(P.rope.pos + tok) : 0;
+                            if (i == 0 || pos != prev + 1) {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) rope_cs(fsrc[e], pos, cs[e], sn[e]);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    const float c1 = fmaf(cs[e], stc[e], -sn[e] * sts[e]);
+                                    sn[e] = fmaf(sn[e], stc[e], cs[e] * sts[e]);
+                                    cs[e] = c1;
+                                }
+                            }
+                            prev = pos;
                             const int olo = r * 128 + ((lc ^ (r & 7)) << 4);
                             const int ohi = (D == 128) ? C::XBLK + olo : r * 128 + (((lc + 4) ^ (r & 7)) << 4);
                             const uint4 vl = *reinterpret_cast<const uint4 *>(xt + olo);
@@ -444,14 +464,11 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                             unsigned wl[4], wh[4];
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                float c0, s0, c1, s1;
-                                rope_cs(fsrc[2 * e], pos, c0, s0);
-                                rope_cs(fsrc[2 * e + 1], pos, c1, s1);
                                 const float l0 = __uint_as_float(ul[e] << 16), l1 = __uint_as_float(ul[e] & 0xffff0000u);
                                 const float h0 = __uint_as_float(uh[e] << 16), h1 = __uint_as_float(uh[e] & 0xffff0000u);
                                 // rotation by -phi
-                                wl[e] = ap_pack_f16x2(fmaf(l0, c0, h0 * s0), fmaf(l1, c1, h1 * s1));
-                                wh[e] = ap_pack_f16x2(fmaf(h0, c0, -l0 * s0), fmaf(h1, c1, -l1 * s1));
+                                wl[e] = ap_pack_f16x2(fmaf(l0, cs[2 * e], h0 * sn[2 * e]), fmaf(l1, cs[2 * e + 1], h1 * sn[2 * e + 1]));
+                                wh[e] = ap_pack_f16x2(fmaf(h0, cs[2 * e], -l0 * sn[2 * e]), fmaf(h1, cs[2 * e + 1], -l1 * sn[2 * e + 1]));
                             }
                             *reinterpret_cast<uint4 *>(xt + olo) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
                             *reinterpret_cast<uint4 *>(xt + ohi) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
