@@ -35,7 +35,7 @@ namespace cb {
 
 using namespace ptx;
 
-template <int D, bool COMP, bool FH = false>
+template <int D, bool COMP, bool FH = false, bool ROPE = false>
 struct TcCfg {
     static constexpr int TT = 64;                     // tokens per tile
     static constexpr int NBX = D / 64;                // 64-channel blocks per head
@@ -50,7 +50,9 @@ struct TcCfg {
     static constexpr int A_PARTS = COMP ? 2 : 1;
     static constexpr int N = 2 * D;                   // accumulator columns
     static constexpr int TMEM_COLS = 2 * N;           // two accumulators
-    static constexpr int FOLD_WARPS = CB_FOLD_WARPS, DRAIN_WARPS = 4;
+    // ROPE: half as many fold warps, so that each fold thread may hold the rotation state of its rows in registers
+    // (the block's register file divided by its threads caps a thread at 80 registers with 16 fold warps)
+    static constexpr int FOLD_WARPS = ROPE ? 8 : CB_FOLD_WARPS, DRAIN_WARPS = 4;
     static constexpr int YPROD_WARP = 2 + FOLD_WARPS + DRAIN_WARPS;   // second producer: target tiles + weights
     static constexpr int FOLD_THREADS = FOLD_WARPS * 32;
     static constexpr int THREADS = (3 + FOLD_WARPS + DRAIN_WARPS) * 32;
@@ -251,9 +253,9 @@ struct Ring {
 // CEN: two-pass centred construction: the weighted operand is w (x - mu_x) with the means of P.a.mu; the bias sums
 // become the column sums of the ROUNDED weighted operand (what the reduction needs for its exact correction).
 template <int D, bool COMP, bool FH, bool CEN, bool ROPE>
-__global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(const __grid_constant__ TcParams P)
+__global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_tc(const __grid_constant__ TcParams P)
 {
-    using C = TcCfg<D, COMP, FH>;
+    using C = TcCfg<D, COMP, FH, ROPE>;
     using TileIter = TileIterT<FH>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -427,11 +429,23 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
         float sx[8], sy[8], sw = 0.f;
         // ROPE: this thread rotates half a chunk (4 frequencies) of rows rg, rg + RG, ..: channels 4 cc + e pair with
         // channels D/2 + 4 cc + e.  Same (cc, rg) decomposition as the ordinary fold, other channels.
-        uint32_t fsrc[4] = {0, 0, 0, 0}, ftgt[4] = {0, 0, 0, 0};
+        // Between consecutive tiles of a sequence every position advances by TT, so (cos, sin) of a (row, frequency)
+        // follow from the previous tile's by one rotation with the thread's constants (cos, sin)(TT theta_i); the
+        // special-function unit (slow: it is shared by the whole scheduler) is only used at the first tile of a unit,
+        // where the positions do not advance by TT, and every 16th tile to bound the drift of the recurrence.
+        float stc[4] = {1.f, 1.f, 1.f, 1.f}, sts[4] = {0.f, 0.f, 0.f, 0.f};
+        float rcs[C::RPT][4], rsn[C::RPT][4];
+        int rprev[C::RPT];
         int rp_lo = 0, rp_hi = 0;
         if (ROPE) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) { fsrc[e] = P.rope.f_src[cc * 4 + e]; ftgt[e] = P.rope.f_tgt[cc * 4 + e]; }
+            for (int e = 0; e < 4; ++e) rope_cs(P.rope.f_src[cc * 4 + e], C::TT, stc[e], sts[e]);
+#pragma unroll
+            for (int i = 0; i < C::RPT; ++i) {
+                rprev[i] = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { rcs[i][e] = 1.f; rsn[i][e] = 0.f; }
+            }
             const int lcr = cc >> 1, hb = (cc & 1) * 8, swz = rg & 7;
             rp_lo = rg * 128 + ((lcr ^ swz) << 4) + hb;
             rp_hi = (D == 128) ? C::BLK + rp_lo : rg * 128 + (((lcr + 4) ^ swz) << 4) + hb;
@@ -482,8 +496,19 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                         const float wt = wsm[i * C::RG];
                         const int pos = psm[i * C::RG];
                         float cs[4], sn[4];
+                        if (t == 0 || pos != rprev[i] + C::TT || (t & 15) == 0) {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) rope_cs(fsrc[e], pos, cs[e], sn[e]);
+                            for (int e = 0; e < 4; ++e) rope_cs(P.rope.f_src[cc * 4 + e], pos, cs[e], sn[e]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                cs[e] = fmaf(rcs[i][e], stc[e], -rsn[i][e] * sts[e]);
+                                sn[e] = fmaf(rsn[i][e], stc[e], rcs[i][e] * sts[e]);
+                            }
+                        }
+                        rprev[i] = pos;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) { rcs[i][e] = cs[e]; rsn[i][e] = sn[e]; }
                         {
                             const uint2 vl = *reinterpret_cast<const uint2 *>(xt + rp_lo + off);
                             const uint2 vh = *reinterpret_cast<const uint2 *>(xt + rp_hi + off);
@@ -518,7 +543,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH>::THREADS, 1) k_accum_tc(con
                         }
                         if (!P.rope.same) {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) rope_cs(ftgt[e], pos, cs[e], sn[e]);
+                            for (int e = 0; e < 4; ++e) rope_cs(P.rope.f_tgt[cc * 4 + e], pos, cs[e], sn[e]);
                         }
                         {
                             const uint2 vl = *reinterpret_cast<const uint2 *>(yt + rp_lo + off);
@@ -798,7 +823,7 @@ static int sm_count()
 template <int D, bool COMP, bool FH = false, bool CEN = false, bool ROPE = false>
 static cudaError_t launch_tc(const TcParams &P, cudaStream_t st)
 {
-    using C = TcCfg<D, COMP, FH>;
+    using C = TcCfg<D, COMP, FH, ROPE>;
     static bool attr = false;
     if (!attr) {
         cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D, COMP, FH, CEN, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);

@@ -140,7 +140,8 @@ def test_fused_equals_rotate_then_accumulate():
         out.append((G.cpu().numpy(), C.cpu().numpy()))
     (G1, C1), (G2, C2) = out
     half = wl.n_maps // 2
-    assert np.array_equal(G1[half:], G2[half:]) and np.array_equal(C1[half:], C2[half:])     # value maps: untouched path
+    # value maps take the ordinary arithmetic (the launch only sums the bias entries over fewer fold warps)
+    assert max_rel_fro_per_map(G1[half:], G2[half:]) < 1e-6 and max_rel_fro_per_map(C1[half:], C2[half:]) < 1e-6
     # key maps: the fused path weights the unrounded de-rotated row, the two-step path the stored bf16 one; they
     # differ by that rounding (see the tolerance note above: ~5e-4 at ~1000 tokens per map), not more
     assert max_rel_fro_per_map(G1[:half], G2[:half]) < 1e-3 and max_rel_fro_per_map(C1[:half], C2[:half]) < 2e-3
