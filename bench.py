@@ -211,7 +211,7 @@ def main():
     if args.multilayer > 0:
         multilayer_case(args, cb, synth, torch, wl, sl, sh, dev)
         return
-    if args.two_pass:
+    if args.two_pass and args.profile_tokens <= 0:
         two_pass_case(args, cb, synth, torch, wl, sl, sh, dev)
         return
     prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, flags=args.flags, n_splits=args.splits)
@@ -549,6 +549,38 @@ def profile_case(args, cb, synth, torch, wl, sl, sh, dev):
         ts.append(e0.elapsed_time(e1))
     cb.cb_device_status(ctx)
     p, d = wl.d + 1, wl.d
+    if args.two_pass or args.rope:
+        # the other accumulate variants on the same small case (two launches each), for ncu -k
+        ws = torch.empty(cb.cb_means_workspace_bytes(prob), dtype=torch.uint8, device=dev)
+        mu = torch.empty(wl.n_maps, 2 * d + 1, device=dev)
+        pos = torch.arange(T, dtype=torch.int32, device=dev) % 1024
+        tm, tc, tr = [], [], []
+        cb.cb_means_reset(ctx, ws)
+        for _ in range(2):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            cb.cb_means_accumulate(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"], ws)
+            e1.record()
+            e1.synchronize()
+            tm.append(e0.elapsed_time(e1))
+        cb.cb_means_finalize(ctx, ws, mu)
+        for fn, acc in ((lambda: cb.cb_stats_accumulate_centered(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"],
+                                                                 ch["w_k"], ch["w_v"], mu), tc),
+                        (lambda: cb.cb_stats_accumulate_rope(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"],
+                                                             ch["w_k"], ch["w_v"], pos, 1e6, 1e6), tr)):
+            cb.cb_stats_reset(ctx)
+            for _ in range(2):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                e1.synchronize()
+                acc.append(e0.elapsed_time(e1))
+        cb.cb_device_status(ctx)
+        print("profile case: %d tokens, means ms %s, centred accumulate ms %s, rope accumulate ms %s" % (
+            T, ["%.3f" % t for t in tm], ["%.3f" % t for t in tc], ["%.3f" % t for t in tr]))
+        cb.cb_stats_reset(ctx)
+        cb.cb_stats_accumulate(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"])
     G = torch.empty(wl.n_maps, p, p, device=dev)
     C = torch.empty(wl.n_maps, p, d, device=dev)
     n = cb.cb_stats_reduce(ctx, G, C)
