@@ -47,6 +47,9 @@ typedef enum cb_status {
                                /* instead of ~2^-9 per element.  Meant for small token counts.             */
 #define CB_FLAG_RAW_LAMBDA  2u /* solve: penalise with lambda itself instead of lambda * s_w / n            */
 #define CB_FLAG_SIMT        4u /* accumulate/apply: use the plain fp32 CUDA-core kernels (no tensor cores) */
+#define CB_FLAG_ONE_ROW_HEAD 8u /* cb_fullhead_problem only: statistics by the kernel that weights one feature head  */
+                               /* per unit (three staged tiles for two products) instead of the default 2 x 2 blocked */
+                               /* kernel (four tiles for four products); kept as a cross-check                        */
 
 #define CB_DTYPE_BF16 0
 #define CB_DTYPE_F32  1

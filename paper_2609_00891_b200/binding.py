@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libcb.so")
 CB_OK = 0
 CB_ERR_INVALID_ARG, CB_ERR_UNSUPPORTED, CB_ERR_STATE, CB_ERR_WORKSPACE = 1, 2, 3, 4
 CB_ERR_CUDA, CB_ERR_NOT_PD, CB_ERR_TIMEOUT, CB_ERR_STATIC_LIMIT = 5, 6, 7, 8
-CB_FLAG_COMPENSATED, CB_FLAG_RAW_LAMBDA, CB_FLAG_SIMT = 1, 2, 4
+CB_FLAG_COMPENSATED, CB_FLAG_RAW_LAMBDA, CB_FLAG_SIMT, CB_FLAG_ONE_ROW_HEAD = 1, 2, 4, 8
 CB_DTYPE_BF16, CB_DTYPE_F32 = 0, 1
 
 EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_workspace_bytes", "cb_create",

@@ -91,6 +91,8 @@ cudaError_t launch_accum_simt(const AccumArgs &a, int d, cudaStream_t st);
 cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st);
 cudaError_t launch_fullhead_tc(const AccumArgs &a, const FullHeadArgs &f, int d, const cb_kv_view *src, const cb_kv_view *tgt,
                                cudaStream_t st);
+cudaError_t launch_gram2_tc(const AccumArgs &a, const FullHeadArgs &f, int d, const cb_kv_view *src, const cb_kv_view *tgt,
+                            cudaStream_t st);
 cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, float *G, float *C, cudaStream_t st);
 cudaError_t launch_means(const MeansArgs &a, int d, cudaStream_t st);
 cudaError_t launch_means_finalize(const double *msum, int n_maps, int d, float *mu, cudaStream_t st);

@@ -12,15 +12,16 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-@pytest.mark.parametrize("name,k", [("mini_ragged", 2), ("mini_ragged", 4), ("mid_scaled", 2)])
-def test_fullhead_statistics_match_oracle(name, k):
+@pytest.mark.parametrize("name,k,flags", [("mini_ragged", 2, 0), ("mini_ragged", 4, 0), ("mid_scaled", 2, 0), ("tiny", 1, 0),
+                                          ("mini_ragged", 2, cb.CB_FLAG_ONE_ROW_HEAD), ("mid_scaled", 2, cb.CB_FLAG_ONE_ROW_HEAD)])
+def test_fullhead_statistics_match_oracle(name, k, flags):
     wl = synth.workload(name)
     sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     sets = cb.cb_fullhead_layer_sets(wl.Ls, wl.Lt, k)
     assert np.array_equal(sets, oracle.fullhead_layer_sets(wl.Ls, wl.Lt, k))          # bookkeeping: bit-exact
     law = synth.map_law(wl)
     chunks = [synth.make_chunk(wl, c, sl, sh, law=law) for c in range(min(2, wl.n_chunks))]
-    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets, flags=flags)
     pf, d = prob.pf, wl.d
     G = torch.zeros(2, wl.Lt, pf, pf, device=DEV)
     C = torch.zeros(2, wl.Lt, wl.Ht, pf, d, device=DEV)

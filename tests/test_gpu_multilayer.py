@@ -13,15 +13,17 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-@pytest.mark.parametrize("name,k", [("mini_ragged", 2), ("mini_ragged", 3), ("mid_scaled", 2), ("tiny", 2), ("deep_small", 8)])
-def test_multilayer_statistics_and_fit(name, k):
+@pytest.mark.parametrize("name,k,flags", [("mini_ragged", 2, 0), ("mini_ragged", 3, 0), ("mid_scaled", 2, 0), ("tiny", 2, 0),
+                                          ("tiny", 1, 0), ("deep_small", 8, 0), ("deep_small", 5, 0),
+                                          ("mini_ragged", 3, cb.CB_FLAG_ONE_ROW_HEAD), ("deep_small", 8, cb.CB_FLAG_ONE_ROW_HEAD)])
+def test_multilayer_statistics_and_fit(name, k, flags):
     wl = synth.workload(name)
     sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     sets = oracle.fullhead_layer_sets(wl.Ls, wl.Lt, k)
     law = synth.map_law(wl)
     chunks = [synth.make_chunk(wl, c, sl, sh, law=law) for c in range(min(2, wl.n_chunks))]
     n_tok = sum(ch["n_tokens"] for ch in chunks)
-    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets, flags=flags)
     d = wl.d
     P = k * d + 1
     G = torch.zeros(wl.n_maps, P, P, device=DEV)
