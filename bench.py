@@ -202,7 +202,11 @@ def main():
     alg_bytes, alg_flops = algorithmic_work(wl)
     n_chunks = args.chunks if args.chunks > 0 else wl.n_chunks
     sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
-    if args.profile_tokens > 0:
+    if args.profile_tokens > 0 and (args.fullhead > 0 or args.multilayer > 0):
+        import dataclasses                      # small case of the wide-regressor kernels for ncu
+        T = args.profile_tokens
+        wl = dataclasses.replace(wl, seq_lens=(1024,) * (T // 1024) + ((T % 1024,) if T % 1024 else ()), seqs_per_chunk=10 ** 6)
+    elif args.profile_tokens > 0:
         profile_case(args, cb, synth, torch, wl, sl, sh, dev)
         return
     if args.fullhead > 0:
@@ -459,8 +463,9 @@ def fullhead_case(args, cb, synth, torch, wl, sl, sh, dev):
     peaks = measured_peaks()
     F = 32
     flops_dense = 2.0 * (2 * wl.Lt) * T * (pf * pf + wl.Ht * pf * d)              # definition: full G and every C
-    units = sum(i // 2 + 1 for i in range(F)) + F * wl.Ht
-    flops_issued = 2.0 * (2 * wl.Lt) * units * T * 128 * 256
+    fp, hpn = (F + 1) // 2, (wl.Ht + 1) // 2                                          # 2 x 2 blocked units: four products each
+    units = fp * (fp + 1) // 2 + fp * hpn
+    flops_issued = 2.0 * (2 * wl.Lt) * units * T * 4 * 128 * 128
     t = min(ms) / 1e3
     print(json.dumps({"workload": "full-head contrast, 14B->32B shapes, %d tokens per chunk" % T, "ms_per_chunk": ms,
                       "tokens_per_s": T / t, "dense_tflops": flops_dense / t / 1e12,
@@ -522,10 +527,14 @@ def multilayer_case(args, cb, synth, torch, wl, sl, sh, dev):
                 tt.append(e0.elapsed_time(e1))
         apply_ms[str(Tp)] = statistics.median(tt)
         del src, out_k, out_v
-    units = sum(i // 2 + 1 for i in range(k)) + k
+    fp = (k + 1) // 2                       # 2 x 2 blocked G units (four products) and C units (two rows x one target head)
+    products = 4 * (fp * (fp + 1) // 2) + 2 * fp
+    dense = 2.0 * wl.n_maps * T * (P * P + P * d)
     print(json.dumps({"apply_ms_by_prefix_tokens": apply_ms, "workload": "head-local over k=%d layers, 14B->32B shapes, P=%d, %d tokens" % (k, P, T),
                       "stats_ms_per_chunk": ms, "stats_tokens_per_s": T / (min(ms) / 1e3),
-                      "issued_mma_tflops": 2.0 * wl.n_maps * units * T * 128 * 256 / (min(ms) / 1e3) / 1e12,
+                      "issued_mma_tflops": 2.0 * wl.n_maps * products * T * 128 * 128 / (min(ms) / 1e3) / 1e12,
+                      "dense_tflops": dense / (min(ms) / 1e3) / 1e12,
+                      "frac_of_bf16_peak_dense": dense / (min(ms) / 1e3) / 1e12 / measured_peaks()["bf16_tflops"],
                       "solve_ms_%d_systems" % nsys: ts,
                       "solve_fp64_tflops": nsys * (P ** 3 / 3.0 + 2.0 * P * P * d) * 2 / (min(ts) / 1e3) / 1e12,
                       "s_per_128000_positions": 2.5 * min(ms) / 1e3 + min(ts) / 1e3}))

@@ -679,7 +679,7 @@ cb_status cb_fullhead_stats_accumulate(const cb_fullhead_problem *prob, const cb
     f.gq = f.gi + NG;
     f.src_head = nullptr; f.per_head = 0;
     f.F = F; f.k = prob->k; f.Hs = prob->Hs; f.PF = F * prob->ds + 1; f.NG = NG; f.NC = F * prob->Ht;
-    const cudaError_t e = (prob->flags & CB_FLAG_ONE_ROW_HEAD) ? launch_fullhead_tc(a, f, prob->ds, src, tgt, st)
+    const cudaError_t e = ((prob->flags & CB_FLAG_ONE_ROW_HEAD) || prob->ds != 128) ? launch_fullhead_tc(a, f, prob->ds, src, tgt, st)
                                                                : launch_gram2_tc(a, f, prob->ds, src, tgt, st);
     if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     return CB_OK;
@@ -744,7 +744,7 @@ cb_status cb_multilayer_stats_accumulate(const cb_fullhead_problem *prob, const 
     f.src_head = f.gq + NG;
     f.per_head = 1;
     f.F = F; f.k = prob->k; f.Hs = prob->Hs; f.PF = F * prob->ds + 1; f.NG = NG; f.NC = F;
-    const cudaError_t e = (prob->flags & CB_FLAG_ONE_ROW_HEAD) ? launch_fullhead_tc(a, f, prob->ds, src, tgt, st)
+    const cudaError_t e = ((prob->flags & CB_FLAG_ONE_ROW_HEAD) || prob->ds != 128) ? launch_fullhead_tc(a, f, prob->ds, src, tgt, st)
                                                                : launch_gram2_tc(a, f, prob->ds, src, tgt, st);
     if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     return CB_OK;

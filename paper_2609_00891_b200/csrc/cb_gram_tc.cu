@@ -13,10 +13,14 @@
 // wasted diagonal product.
 //
 // Roles per block (persistent over units): warp 0 stages the two row heads (TMA); the last warp stages the two column
-// heads and the token weights; 16 fold warps (8 per row head) write w .* rows as bf16 into the A buffers and keep the
-// bias sums; warp 1 issues tcgen05.mma into two tensor-memory accumulators (all 512 columns at d = 128); 4 drain warps
-// add a finished accumulator to G / C with fire-and-forget reductions (each output block has exactly one owner unit,
+// heads and the token weights; 16 fold warps (8 per row head) replace the staged row heads by w .* rows IN PLACE (bf16)
+// and keep the bias sums; warp 1 issues tcgen05.mma into two tensor-memory accumulators (all 512 columns at d = 128); 4 drain warps
+// add a finished accumulator to G / C with fire-and-forget reductions (lower block triangle only; a mirror kernel
+// fills the rest) (each output block has exactly one owner unit,
 // and a thread's reductions to one address are performed in program order, so results are reproducible).
+// Weighting in place leaves room for three stages of four 16 KB head tiles.  (Measured: the kernel is bound by the
+// feed of those tiles into shared memory, ~7.6 TB/s over all SMs, plus ~640 cycles of synchronisation per tile: six
+// stages of 32-token tiles were slower.)
 // Every wait is bounded: if one runs out the block sets a flag, tears down and frees its tensor memory.
 #include <cudaTypedefs.h>
 
@@ -32,14 +36,13 @@ bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long l
 
 template <int D>
 struct GrCfg {
+    static_assert(D == 128, "two 64-channel blocks per head make the M = 128 operand");
     static constexpr int TT = 64;
     static constexpr int NBX = D / 64;
     static constexpr int BLK = TT * 128;
-    static constexpr int HEAD = NBX * BLK;                    // bytes of one staged head tile
+    static constexpr int HEAD = NBX * BLK;                    // bytes of one staged head tile (16 KB)
     static constexpr int STAGE_BYTES = 4 * HEAD;              // [column head 0 | column head 1 | row head 0 | row head 1]
-    static constexpr int NS = 2;
-    static constexpr int A_BYTES = 2 * BLK;                   // M = 128 always
-    static constexpr int NA = 2;                              // sets of (two) weighted operands
+    static constexpr int NS = 3;
     static constexpr int N = 2 * D;                           // accumulator columns per row head
     static constexpr int TMEM_COLS = 2 * N;
     static constexpr int FOLD_WARPS = 16, GROUP_WARPS = 8, DRAIN_WARPS = 4;
@@ -49,8 +52,7 @@ struct GrCfg {
     static constexpr int RG = GROUP_WARPS * 32 / CC;          // row groups of one fold group
     static constexpr int RPT = TT / RG;
     static constexpr int RED_STRIDE = 2 * D + 4;              // per fold warp: row-head sums [D], column-head sums [D], s_w
-    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * STAGE_BYTES + (size_t)NA * 2 * A_BYTES +
-                                         FOLD_WARPS * RED_STRIDE * 4 + NS * TT * 4 + 256;
+    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * STAGE_BYTES + FOLD_WARPS * RED_STRIDE * 4 + NS * TT * 4 + 256;
     static_assert(RG % 8 == 0 && TT % RG == 0, "fold layout");
 };
 
@@ -58,8 +60,8 @@ struct GrParams {
     CUtensorMap src_k, src_v, tgt_k, tgt_v;
     AccumArgs a;
     FullHeadArgs f;
-    int drain_tiles;
-    int FP, HPn, NGU, NCU;        // head pairs of the feature, target-head pairs, G and C units per group
+    int sub_tiles;                // token tiles summed in tensor memory between two drains
+    int FP, HPn, NGU, NCU;        // head pairs of the feature, target-head pairs, G and C blocks per group
 };
 
 // One unit, decoded once per unit by every role.
@@ -79,16 +81,21 @@ struct GrUnit {
         u = unit;
         const AccumArgs &a = P.a;
         const FullHeadArgs &f = P.f;
+        // Unit order: block fastest, then group.  The blocks of a group read the same few heads and thread blocks
+        // take consecutive units at about the same pace, so most tiles are served from L2.  Head-local groups are
+        // ordered target layer fastest: neighbouring layers select almost the same source layers.
         const int per = P.NGU + P.NCU;
-        group = u / per;
         const int v = u % per;
+        const int gidx = u / per;
         int src_h = 0;
         if (f.per_head) {
-            comp = group / (a.Lt * a.Ht);
-            l = (group / a.Ht) % a.Lt;
-            h = group % a.Ht;
+            comp = gidx / (a.Lt * a.Ht);
+            h = (gidx / a.Lt) % a.Ht;
+            l = gidx % a.Lt;
+            group = (comp * a.Lt + l) * a.Ht + h;
             src_h = f.src_head[h];
         } else {
+            group = gidx;
             comp = group / a.Lt;
             l = group % a.Lt;
             h = 0;
@@ -188,14 +195,13 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *stg = smem;                                          // [NS][STAGE_BYTES]
-    uint8_t *ab = stg + (size_t)C::NS * C::STAGE_BYTES;           // [NA][2 row heads][A_BYTES]
-    float *red = reinterpret_cast<float *>(ab + (size_t)C::NA * 2 * C::A_BYTES);
+    float *red = reinterpret_cast<float *>(stg + (size_t)C::NS * C::STAGE_BYTES);
     float *wst = red + C::FOLD_WARPS * C::RED_STRIDE;             // [NS][TT]
     uint64_t *bars = reinterpret_cast<uint64_t *>(wst + C::NS * C::TT);
     uint64_t *full = bars;                  // [NS] row heads (1 arrival + bytes), column heads (1 + bytes), weights (32 lanes)
-    uint64_t *empty = full + C::NS;         // [NS] MMA done (1) + every fold warp done
-    uint64_t *afull = empty + C::NS;        // [NA] weighted operands written (every fold warp)
-    uint64_t *accfull = afull + C::NA;      // [1]
+    uint64_t *empty = full + C::NS;         // [NS] MMA done with the stage
+    uint64_t *afull = empty + C::NS;        // [NS] row heads weighted in place (every fold warp)
+    uint64_t *accfull = afull + C::NS;      // [1]
     uint64_t *accempty = accfull + 1;       // [1]  (4 drain warps)
     uint64_t *redfull = accempty + 1;       // [1]
     uint64_t *reddone = redfull + 1;        // [1]
@@ -211,8 +217,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
     const size_t PF = (size_t)f.PF;
 
     if (tid == 0) {
-        for (int i = 0; i < C::NS; ++i) { mbar_init(&full[i], 2 + 32); mbar_init(&empty[i], 1 + C::FOLD_WARPS); }
-        for (int i = 0; i < C::NA; ++i) mbar_init(&afull[i], C::FOLD_WARPS);
+        for (int i = 0; i < C::NS; ++i) { mbar_init(&full[i], 2 + 32); mbar_init(&empty[i], 1); mbar_init(&afull[i], C::FOLD_WARPS); }
         mbar_init(accfull, 1);
         mbar_init(accempty, C::DRAIN_WARPS);
         mbar_init(redfull, C::FOLD_WARPS);
@@ -223,15 +228,6 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
         tma_prefetch_desc(&P.tgt_k); tma_prefetch_desc(&P.tgt_v);
     }
     if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
-    if (D == 64 && warp >= 2 && warp < 2 + C::FOLD_WARPS) {
-        // rows 64..127 of the M = 128 operands never get data: clear the second block of every A buffer once
-        const int ft = tid - 64;
-        for (int i = ft; i < C::NA * 2 * (C::BLK / 16); i += C::FOLD_WARPS * 32) {
-            const int buf = i / (C::BLK / 16), off = i % (C::BLK / 16);
-            *reinterpret_cast<uint4 *>(ab + (size_t)buf * C::A_BYTES + C::BLK + off * 16) = make_uint4(0, 0, 0, 0);
-        }
-        fence_async_smem();
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -292,9 +288,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
             const uint64_t proto = umma_smem_desc_sw128(0, C::BLK, 1024);
             const uint32_t desc_hi = (uint32_t)(proto >> 32);
             const uint32_t b_lo0 = (uint32_t)proto | ((smem_u32(stg) & 0x3FFFFu) >> 4);
-            const uint32_t a_lo0 = (uint32_t)proto | ((smem_u32(ab) & 0x3FFFFu) >> 4);
             GrRing<C::NS> st;
-            GrRing<C::NA> ar;
             uint32_t sr = 0;
             GrUnit un;
             for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
@@ -302,28 +296,27 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                 // a missing second column head (odd count) leaves stale bytes in its half of the stage: use N = D then
                 const uint32_t idesc = (un.nb == 2 && un.vb[1]) ? idesc2 : idesc1;
                 const int two_rows = un.va[1];
-                for (int sr0 = 0; sr0 < n_tiles; sr0 += P.drain_tiles, ++sr) {
-                    const int n_sub = min(n_tiles - sr0, P.drain_tiles);
+                for (int sr0 = 0; sr0 < n_tiles; sr0 += P.sub_tiles, ++sr) {
+                    const int n_sub = min(n_tiles - sr0, P.sub_tiles);
                     if (!mbar_wait(accempty, (sr & 1) ^ 1, abort_flag)) goto teardown;
                     tc_fence_after();
                     uint32_t accum = 0;
                     for (int t = 0; t < n_sub; ++t) {
-                        if (!mbar_wait(&afull[ar.idx], ar.phase, abort_flag)) goto teardown;
+                        if (!mbar_wait(&afull[st.idx], st.phase, abort_flag)) goto teardown;
                         tc_fence_after();
                         const uint32_t bl = b_lo0 + st.idx * (C::STAGE_BYTES >> 4);
-                        const uint32_t al = a_lo0 + ar.idx * ((2 * C::A_BYTES) >> 4);
+                        const uint32_t al = bl + ((2 * C::HEAD) >> 4);                 // weighted row heads
 #pragma unroll
                         for (int k = 0; k < C::TT / 16; ++k) {
                             const uint64_t bd = ((uint64_t)desc_hi << 32) | (bl + k * 128);
                             const uint32_t acc_flag = (k == 0) ? accum : 1u;
                             umma_bf16_ss(tmem_base, ((uint64_t)desc_hi << 32) | (al + k * 128), bd, idesc, acc_flag);
                             if (two_rows)
-                                umma_bf16_ss(tmem_base + C::N, ((uint64_t)desc_hi << 32) | (al + (C::A_BYTES >> 4) + k * 128), bd, idesc, acc_flag);
+                                umma_bf16_ss(tmem_base + C::N, ((uint64_t)desc_hi << 32) | (al + (C::HEAD >> 4) + k * 128), bd, idesc, acc_flag);
                         }
                         accum = 1;
                         umma_commit(&empty[st.idx]);
                         st.next();
-                        ar.next();
                     }
                     umma_commit(accfull);
                 }
@@ -337,9 +330,8 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
         const int cc = gt % C::CC, rg = gt / C::CC;
         const int blk = cc >> 3, lc = cc & 7;
         const int off0 = blk * C::BLK + rg * 128 + ((lc ^ (rg & 7)) << 4);
-        GrRing<C::NS> st, old;
-        GrRing<C::NA> ar;
-        uint32_t it = 0, uc = 0;
+        GrRing<C::NS> st;
+        uint32_t uc = 0;
         GrUnit un;
         for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++uc) {
             un.decode(P, u);
@@ -352,14 +344,10 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
             float sw = 0.f;
             for (int t = 0; t < n_tiles; ++t) {
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
-                if (it >= (uint32_t)C::NA) {
-                    if (!mbar_wait_warp(&empty[old.idx], old.phase, abort_flag, lane)) goto teardown;
-                    old.next();
-                }
                 const float *wsm = wst + st.idx * C::TT + rg;
-                const uint8_t *rs = stg + st.idx * C::STAGE_BYTES + (2 + g) * C::HEAD + off0;     // row head g
+                uint8_t *rs = stg + st.idx * C::STAGE_BYTES + (2 + g) * C::HEAD + off0;           // row head g, weighted in place
                 const uint8_t *cs = stg + st.idx * C::STAGE_BYTES + g * C::HEAD + off0;           // column head g
-                uint8_t *ah = ab + ar.idx * (2 * C::A_BYTES) + g * C::A_BYTES + off0;
+                uint8_t *ah = rs;
                 if (active) {
 #pragma unroll
                     for (int i = 0; i < C::RPT; ++i) {
@@ -400,10 +388,8 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0) { mbar_arrive(&afull[ar.idx]); mbar_arrive(&empty[st.idx]); }
+                if (lane == 0) mbar_arrive(&afull[st.idx]);
                 st.next();
-                ar.next();
-                ++it;
             }
             // ---- bias entries (C units only): lanes holding the same channels add up, fixed-order sum over the
             //      group's warps, then one owner thread per entry adds to G / C ----
@@ -447,16 +433,15 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                     for (int q = 0; q < C::GROUP_WARPS; ++q) sum += red[(g * C::GROUP_WARPS + q) * C::RED_STRIDE + v];
                     if (v < D) {
                         if (un.own_sa && active) {
-                            Gg[((size_t)un.fa[g] * D + v) * PF + (PF - 1)] += sum;
-                            Gg[(PF - 1) * PF + (size_t)un.fa[g] * D + v] += sum;
+                            atomicAdd(&Gg[(PF - 1) * PF + (size_t)un.fa[g] * D + v], sum);     // bias row; the column is mirrored
                         }
                     } else if (v < 2 * D) {
                         if (un.own_sy && (g == 0 || (un.nb == 2 && un.vb[1]))) {
                             const size_t oc = f.per_head ? (size_t)un.group : (size_t)un.group * a.Ht + un.fb[g];
-                            f.C[(oc * PF + (PF - 1)) * D + (v - D)] += sum;
+                            atomicAdd(&f.C[(oc * PF + (PF - 1)) * D + (v - D)], sum);
                         }
                     } else if (un.own_sw && g == 0) {
-                        Gg[(PF - 1) * PF + (PF - 1)] += sum;
+                        atomicAdd(&Gg[(PF - 1) * PF + (PF - 1)], sum);
                     }
                 }
                 __syncwarp();
@@ -479,7 +464,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
             un.decode(P, u);
             float *Gg = f.G + (size_t)un.group * PF * PF;
             const int ncolh = (un.nb == 2 && un.vb[1]) ? 2 : 1;
-            for (int sr0 = 0; sr0 < n_tiles; sr0 += P.drain_tiles, ++sr) {
+            for (int sr0 = 0; sr0 < n_tiles; sr0 += P.sub_tiles, ++sr) {
                 if (!mbar_wait_warp(accfull, sr & 1, abort_flag, lane, true, 4, 512)) goto teardown;
                 tc_fence_after();
                 if (row < D) {
@@ -493,15 +478,10 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                             const int part = (c * 16) / D, c0 = (c * 16) % D;
                             if (!un.is_c) {
                                 const int j = un.fb[part], i = un.fa[ra];
-                                if (j <= i) {
+                                if (j <= i) {                      // block row i, block column j <= i; the mirror kernel fills the rest
                                     float *dst = Gg + ri * PF + (size_t)j * D + c0;
 #pragma unroll
                                     for (int e = 0; e < 16; ++e) atomicAdd(dst + e, __uint_as_float(r[e]));
-                                    if (j < i) {
-                                        float *mir = Gg + ((size_t)j * D + c0) * PF + ri;
-#pragma unroll
-                                        for (int e = 0; e < 16; ++e) atomicAdd(mir + (size_t)e * PF, __uint_as_float(r[e]));
-                                    }
                                 }
                             } else {
                                 const size_t oc = f.per_head ? (size_t)un.group : (size_t)un.group * a.Ht + un.fb[part];
@@ -530,6 +510,24 @@ teardown:
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+// G[c][r] = G[r][c] for r > c, per group; 32 x 32 tiles through shared memory so that both sides are coalesced.
+__global__ void k_mirror_lower(float *__restrict__ G, int pf)
+{
+    if (blockIdx.y > blockIdx.x) return;                    // tile (row block x, column block y) with x >= y
+    __shared__ float t[32][33];
+    float *Gg = G + (size_t)blockIdx.z * pf * pf;
+    const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    for (int i = threadIdx.y; i < 32; i += 8) {
+        const int r = r0 + i, c = c0 + threadIdx.x;
+        t[i][threadIdx.x] = (r < pf && c < pf) ? Gg[(size_t)r * pf + c] : 0.f;
+    }
+    __syncthreads();
+    for (int i = threadIdx.y; i < 32; i += 8) {
+        const int c = c0 + i, r = r0 + threadIdx.x;         // writes G[c][r], r fastest
+        if (r < pf && c < pf && r > c) Gg[(size_t)c * pf + r] = t[threadIdx.x][i];
     }
 }
 
@@ -576,7 +574,18 @@ cudaError_t launch_gram2_tc(const AccumArgs &a, const FullHeadArgs &f, int d, co
         !make_kv_tensor_map(&P.tgt_v, tgt->v, d, tgt->n_heads, tgt->n_tokens, tgt->n_layers, tgt->stride_head,
                             tgt->stride_token, tgt->stride_layer, TT))
         return cudaErrorInvalidValue;
-    P.drain_tiles = 16384 / TT;
+    // The tensor-core accumulator truncates: at most 32,768 tokens are summed in tensor memory between drains (mean
+    // relative drift of an all-positive sum ~2e-4 there), in equal parts.  A drain stalls the MMA thread here (both
+    // accumulators belong to the unit), so fewer, longer parts than in the head-local k = 1 kernel.
+    const int n_tiles = (a.n_tokens + TT - 1) / TT;
+#ifdef CB_GRAM_SUB_TILES
+    const int cap = CB_GRAM_SUB_TILES;
+#else
+    const int cap = 32768 / TT;
+#endif
+    const int parts = (n_tiles + cap - 1) / cap;
+    P.sub_tiles = (n_tiles + parts - 1) / (parts > 0 ? parts : 1);
+    if (P.sub_tiles < 1) P.sub_tiles = 1;
     P.FP = (f.F + 1) / 2;
     const int NH = f.per_head ? 1 : a.Ht;
     P.HPn = (NH + 1) / 2;
@@ -584,7 +593,15 @@ cudaError_t launch_gram2_tc(const AccumArgs &a, const FullHeadArgs &f, int d, co
     P.NCU = P.FP * P.HPn;
     const int n_groups = 2 * a.Lt * (f.per_head ? a.Ht : 1);
     const int n_units = n_groups * (P.NGU + P.NCU);
-    cudaError_t e = (d == 128) ? launch_gr<128>(P, n_units, st) : launch_gr<64>(P, n_units, st);
+    if (d != 128) return cudaErrorInvalidValue;          // the caller routes other widths to the one-row-head kernel
+    cudaError_t e = launch_gr<128>(P, n_units, st);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    // upper triangle <- lower triangle (the units only add to block rows >= block columns and to the bias row)
+    const int pf = f.PF;
+    dim3 grid((pf + 31) / 32, (pf + 31) / 32, n_groups);
+    k_mirror_lower<<<grid, dim3(32, 8), 0, st>>>(f.G, pf);
+    e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;
 }
