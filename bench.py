@@ -606,6 +606,17 @@ def profile_case(args, cb, synth, torch, wl, sl, sh, dev):
         e1.record()
         e1.synchronize()
         ta.append(e0.elapsed_time(e1))
+    if args.rope:
+        pos = torch.arange(T, dtype=torch.int32, device=dev) % 4096
+        tr = []
+        for _ in range(2):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            cb.cb_apply_rope(prob, Wb[0], ch["src_k"], ch["src_v"], out_k, out_v, pos, 1e6, 1e6)
+            e1.record()
+            e1.synchronize()
+            tr.append(e0.elapsed_time(e1))
+        print("profile case: rope apply ms %s" % ["%.3f" % t for t in tr])
     torch.cuda.synchronize()
     print("profile case: %d tokens, accumulate ms %s (%.0f GB/s algorithmic), apply ms %s" % (
         T, ["%.3f" % t for t in ts], ALG_BYTES_PER_TOKEN * T / 1e9 / (min(ts) / 1e3), ["%.3f" % t for t in ta]))

@@ -439,7 +439,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
         int rp_lo = 0, rp_hi = 0;
         if (ROPE) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) rope_cs(P.rope.f_src[cc * 4 + e], C::TT, stc[e], sts[e]);
+            for (int e = 0; e < 4; ++e) rope_cs_poly(P.rope.f_src[cc * 4 + e], C::TT, stc[e], sts[e]);
 #pragma unroll
             for (int i = 0; i < C::RPT; ++i) {
                 rprev[i] = 0;
@@ -498,7 +498,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                         float cs[4], sn[4];
                         if (t == 0 || pos != rprev[i] + C::TT || (t & 15) == 0) {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) rope_cs(P.rope.f_src[cc * 4 + e], pos, cs[e], sn[e]);
+                            for (int e = 0; e < 4; ++e) rope_cs_poly(P.rope.f_src[cc * 4 + e], pos, cs[e], sn[e]);
                         } else {
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
@@ -543,7 +543,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                         }
                         if (!P.rope.same) {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) rope_cs(P.rope.f_tgt[cc * 4 + e], pos, cs[e], sn[e]);
+                            for (int e = 0; e < 4; ++e) rope_cs_poly(P.rope.f_tgt[cc * 4 + e], pos, cs[e], sn[e]);
                         }
                         {
                             const uint2 vl = *reinterpret_cast<const uint2 *>(yt + rp_lo + off);

@@ -38,7 +38,7 @@ __global__ void __launch_bounds__(256) k_rope_rotate(const RopeArgs a)
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             float c, s;
-            rope_cs(a.f[lc * 8 + 2 * e + q], pos, c, s);
+            rope_cs_poly(a.f[lc * 8 + 2 * e + q], pos, c, s);
             if (a.inverse) s = -s;
             nl[q] = lo[q] * c - hi[q] * s;
             nh[q] = lo[q] * s + hi[q] * c;

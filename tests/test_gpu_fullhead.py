@@ -54,3 +54,21 @@ def test_fullhead_statistics_match_oracle(name, k, flags):
         np.testing.assert_allclose(Gc[comp, l, pf - 1, :], Go[pf - 1, :], rtol=2e-4, atol=1e-3 * np.abs(Go[pf - 1]).max())
         np.testing.assert_allclose(Gc[comp, l, :, pf - 1], Go[:, pf - 1], rtol=2e-4, atol=1e-3 * np.abs(Go[pf - 1]).max())
         np.testing.assert_allclose(Cc[comp, l, :, pf - 1, :], Co[:, pf - 1, :], rtol=2e-4, atol=1e-3 * np.abs(Co[:, pf - 1]).max())
+
+
+def test_wide_statistics_are_bitwise_reproducible():
+    wl = synth.workload("mini_ragged")
+    sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    sets = cb.cb_fullhead_layer_sets(wl.Ls, wl.Lt, 2)
+    ch = synth.make_chunk(wl, 0, sl, sh, law=synth.map_law(wl))
+    t = {k_: v.to(DEV) for k_, v in ch.items() if torch.is_tensor(v)}
+    wk, wv = t["w_k"][:, 0].contiguous(), t["w_v"][:, 0].contiguous()
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
+    out = []
+    for _ in range(2):
+        G = torch.zeros(2, wl.Lt, prob.pf, prob.pf, device=DEV)
+        C = torch.zeros(2, wl.Lt, wl.Ht, prob.pf, wl.d, device=DEV)
+        cb.cb_fullhead_stats_accumulate(prob, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], wk, wv, G, C)
+        out.append((G, C))
+    assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1])
+    assert torch.equal(out[0][0], out[0][0].transpose(2, 3))          # exactly symmetric
