@@ -48,8 +48,9 @@ __global__ void __launch_bounds__(256) k_lg_load(LgArgs a, LgLoadArgs la)
     if (i == 0 && threadIdx.x == 0) a.fail[s] = 0;
 }
 
-// ---- block column J: factor A_JJ, then L_IJ = A_IJ L_JJ^-T for every row below -----------------------------------
-__global__ void __launch_bounds__(256, 1) k_lg_panel(LgArgs a, int J)
+// ---- block column J, part 1: factor the 64 x 64 diagonal block A_JJ in place ---------------------------------------
+// A chain of 64 dependent pivots: latency-bound, so the block is small (128 threads, 33 KB) and many systems share an SM.
+__global__ void __launch_bounds__(128) k_lg_factor(LgArgs a, int J)
 {
     __shared__ double Ld[LNB][LNB + 1];
     __shared__ double rinv[LNB];
@@ -58,7 +59,7 @@ __global__ void __launch_bounds__(256, 1) k_lg_panel(LgArgs a, int J)
     double *A = a.A + (size_t)s * a.Pp * a.Pp;
     const int j0 = J * LNB;
     if (tid == 0) s_fail = 0;
-    for (int e = tid; e < LNB * LNB; e += 256) {
+    for (int e = tid; e < LNB * LNB; e += 128) {
         const int r = e / LNB, c = e % LNB;
         Ld[r][c] = (c <= r) ? A[(size_t)(j0 + r) * a.Pp + j0 + c] : 0.0;
     }
@@ -73,41 +74,56 @@ __global__ void __launch_bounds__(256, 1) k_lg_panel(LgArgs a, int J)
         }
         __syncthreads();
         const double ri = rinv[j];
-        for (int i = j + 1 + tid; i < LNB; i += 256) Ld[i][j] *= ri;
+        for (int i = j + 1 + tid; i < LNB; i += 128) Ld[i][j] *= ri;
         __syncthreads();
-        for (int e = tid; e < (LNB - j - 1) * (LNB - j - 1); e += 256) {
+        for (int e = tid; e < (LNB - j - 1) * (LNB - j - 1); e += 128) {
             const int i = j + 1 + e / (LNB - j - 1), k = j + 1 + e % (LNB - j - 1);
             if (k <= i) Ld[i][k] -= Ld[i][j] * Ld[k][j];
         }
         __syncthreads();
     }
-    for (int e = tid; e < LNB * LNB; e += 256) {
+    for (int e = tid; e < LNB * LNB; e += 128) {
         const int r = e / LNB, c = e % LNB;
         if (c <= r) A[(size_t)(j0 + r) * a.Pp + j0 + c] = Ld[r][c];
     }
     if (tid == 0 && s_fail && a.fail[s] == 0) a.fail[s] = s_fail;
-    // rows below the block: x L_JJ^T = a, one row per thread, the row held in registers
-    for (int i0 = j0 + LNB; i0 < a.Pp; i0 += 256) {
-        const int i = i0 + tid;
-        if (i >= a.Pp) continue;
-        double *row = A + (size_t)i * a.Pp + j0;
-        double x[LNB];
-#pragma unroll
-        for (int c = 0; c < LNB; c += 2) {
-            const double2 v = *reinterpret_cast<const double2 *>(row + c);
-            x[c] = v.x;
-            x[c + 1] = v.y;
-        }
-#pragma unroll
-        for (int c = 0; c < LNB; ++c) {
-            double v = x[c];
-#pragma unroll
-            for (int q = 0; q < c; ++q) v -= x[q] * Ld[c][q];
-            x[c] = v * rinv[c];
-        }
-#pragma unroll
-        for (int c = 0; c < LNB; c += 2) *reinterpret_cast<double2 *>(row + c) = make_double2(x[c], x[c + 1]);
+}
+
+// ---- block column J, part 2: L_IJ = A_IJ L_JJ^-T for the rows below; grid (row chunks of 128, systems) -------------
+__global__ void __launch_bounds__(128) k_lg_panel(LgArgs a, int J)
+{
+    __shared__ double Ld[LNB][LNB + 1];
+    __shared__ double rinv[LNB];
+    const int s = blockIdx.y, tid = threadIdx.x;
+    double *A = a.A + (size_t)s * a.Pp * a.Pp;
+    const int j0 = J * LNB;
+    for (int e = tid; e < LNB * LNB; e += 128) {
+        const int r = e / LNB, c = e % LNB;
+        Ld[r][c] = (c <= r) ? A[(size_t)(j0 + r) * a.Pp + j0 + c] : 0.0;
     }
+    __syncthreads();
+    if (tid < LNB) rinv[tid] = 1.0 / Ld[tid][tid];
+    __syncthreads();
+    // x L_JJ^T = a, one row per thread, the row held in registers
+    const int i = j0 + LNB + blockIdx.x * 128 + tid;
+    if (i >= a.Pp) return;
+    double *row = A + (size_t)i * a.Pp + j0;
+    double x[LNB];
+#pragma unroll
+    for (int c = 0; c < LNB; c += 2) {
+        const double2 v = *reinterpret_cast<const double2 *>(row + c);
+        x[c] = v.x;
+        x[c + 1] = v.y;
+    }
+#pragma unroll
+    for (int c = 0; c < LNB; ++c) {
+        double v = x[c];
+#pragma unroll
+        for (int q = 0; q < c; ++q) v -= x[q] * Ld[c][q];
+        x[c] = v * rinv[c];
+    }
+#pragma unroll
+    for (int c = 0; c < LNB; c += 2) *reinterpret_cast<double2 *>(row + c) = make_double2(x[c], x[c + 1]);
 }
 
 // ---- tile products: Ctile[64 x NT] -= At[64 x 64] * Bt[64 x NT] ---------------------------------------------------
@@ -155,39 +171,46 @@ __global__ void __launch_bounds__(256) k_lg_tile(LgArgs a, int J)
         }
     }
     __syncthreads();
-    constexpr int CT = NT / 16;               // columns per thread
+    // Thread (ty, tx) owns rows ty*4 .. ty*4+3 and the column pairs {32 jj + 2 tx, 32 jj + 2 tx + 1}, jj < NT/32: the 16
+    // threads of a row group read 16 consecutive 16-byte pairs of Bts per access (no bank conflicts; a thread owning
+    // NT/16 consecutive columns would put all 16 on two bank groups) and write 256 contiguous bytes per output row.
+    constexpr int CJ = NT / 32;               // column pairs per thread
     const int ty = tid >> 4, tx = tid & 15;
-    double acc[4][CT];
+    double acc[4][2 * CJ];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < CT; ++j) acc[i][j] = 0.0;
+        for (int j = 0; j < 2 * CJ; ++j) acc[i][j] = 0.0;
 #pragma unroll 4
     for (int k = 0; k < LNB; ++k) {
-        double av[4], bv[CT];
+        double av[4], bv[2 * CJ];
 #pragma unroll
         for (int i = 0; i < 4; i += 2) {
             const double2 v = *reinterpret_cast<const double2 *>(&Ats[k][ty * 4 + i]);
             av[i] = v.x; av[i + 1] = v.y;
         }
 #pragma unroll
-        for (int j = 0; j < CT; j += 2) {
-            const double2 v = *reinterpret_cast<const double2 *>(&Bts[k][tx * CT + j]);
-            bv[j] = v.x; bv[j + 1] = v.y;
+        for (int jj = 0; jj < CJ; ++jj) {
+            const double2 v = *reinterpret_cast<const double2 *>(&Bts[k][jj * 32 + tx * 2]);
+            bv[2 * jj] = v.x; bv[2 * jj + 1] = v.y;
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
-            for (int j = 0; j < CT; ++j) acc[i][j] += av[i] * bv[j];
+            for (int j = 0; j < 2 * CJ; ++j) acc[i][j] += av[i] * bv[j];
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int r = I * LNB + ty * 4 + i;
-        double *crow = (MODE == 0) ? A + (size_t)r * a.Pp + I2 * LNB + tx * CT : Z + (size_t)r * a.d + tx * CT;
+        double *crow = (MODE == 0) ? A + (size_t)r * a.Pp + I2 * LNB : Z + (size_t)r * a.d;
 #pragma unroll
-        for (int j = 0; j < CT; ++j) {
-            if (MODE == 0 && I == I2 && tx * CT + j > ty * 4 + i) continue;      // keep the diagonal tile lower-triangular
-            crow[j] -= acc[i][j];
+        for (int jj = 0; jj < CJ; ++jj) {
+            const int c = jj * 32 + tx * 2;
+            double2 v = *reinterpret_cast<double2 *>(crow + c);
+            // MODE 0, diagonal tile: keep it lower-triangular
+            if (!(MODE == 0 && I == I2 && c > ty * 4 + i)) v.x -= acc[i][2 * jj];
+            if (!(MODE == 0 && I == I2 && c + 1 > ty * 4 + i)) v.y -= acc[i][2 * jj + 1];
+            *reinterpret_cast<double2 *>(crow + c) = v;
         }
     }
 }
@@ -319,14 +342,15 @@ cudaError_t launch_solve_large(const float *G, const float *C, int n_maps, int P
         la.sys0 = (int)sys0;
         k_lg_load<<<dim3(Pp, a.nsys), 256, 0, st>>>(a, la);
         for (int J = 0; J < nblk; ++J) {
-            k_lg_panel<<<a.nsys, 256, 0, st>>>(a, J);
+            k_lg_factor<<<a.nsys, 128, 0, st>>>(a, J);
             const int r = nblk - 1 - J;
+            if (r > 0) k_lg_panel<<<dim3((r * LNB + 127) / 128, a.nsys), 128, 0, st>>>(a, J);
             if (r > 0) launch_tile<0, LNB>(a, J, dim3(r * (r + 1) / 2, a.nsys), st);
         }
         if (d == 128) launch_subst_tiles<128>(a, nblk, st);
         else launch_subst_tiles<64>(a, nblk, st);
         k_lg_store<<<dim3(P, a.nsys), 256, 0, st>>>(a, Wb, info, (int)sys0);
-        launches += 2 + 2 * nblk + 4 * nblk;
+        launches += 2 + 3 * nblk + 4 * nblk - 4;
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
