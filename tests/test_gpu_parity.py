@@ -261,3 +261,28 @@ def test_launch_counter_counts_kernels():
     sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     _gpu_stats(wl, _chunks(wl, sl, sh), sl, sh, 0)
     assert cb.cb_launch_count() == before + 2            # one accumulate, one reduce
+
+
+def test_token_subsampling_through_the_token_stride():
+    """Every 4th calibration row (the paper subsamples positions): the caller passes views with 4 x the token stride;
+    nothing is copied."""
+    wl = synth.workload("mid_scaled")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    ch = _chunks(wl, sl, sh)[0]
+    sub = {k: (v[:, ::4] if k[:3] in ("src", "tgt") else v[:, :, ::4].contiguous()) for k, v in ch.items() if torch.is_tensor(v)}
+    dense = {k: v.contiguous() for k, v in sub.items()}
+    Go, Co = _oracle_stats([dense], sl, sh)
+    prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, flags=cb.CB_FLAG_COMPENSATED)
+    ctx = cb.cb_create(prob, device=DEV)
+    t = {k: v.to(DEV) for k, v in ch.items() if torch.is_tensor(v)}
+    views = {k: t[k][:, ::4] for k in ("src_k", "src_v", "tgt_k", "tgt_v")}
+    assert not views["src_k"].is_contiguous()
+    cb.cb_stats_accumulate(ctx, views["src_k"], views["src_v"], views["tgt_k"], views["tgt_v"],
+                           t["w_k"][:, :, ::4].contiguous(), t["w_v"][:, :, ::4].contiguous())
+    p, d = wl.d + 1, wl.d
+    G = torch.empty((wl.n_maps, p, p), device=DEV)
+    C = torch.empty((wl.n_maps, p, d), device=DEV)
+    n = cb.cb_stats_reduce(ctx, G, C)
+    cb.cb_device_status(ctx)
+    assert n == dense["src_k"].shape[1]
+    _check_stats(G, C, Go, Co)
