@@ -398,14 +398,12 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                         tc_fence_after();
                         const uint32_t bl = b_lo0 + st.idx * (C::STAGE_BYTES >> 4);
                         const uint32_t al = a_lo0 + ar.idx * ((C::A_PARTS * C::A_BYTES) >> 4);
-#ifndef CB_ABLATE_MMA
 #pragma unroll
                         for (int k = 0; k < C::TT / 16; ++k) {
                             const uint64_t bd = ((uint64_t)desc_hi << 32) | (bl + k * 128);
                             umma_bf16_ss(d_tmem, ((uint64_t)desc_hi << 32) | (al + k * 128), bd, idesc, k == 0 ? accum : 1u);
                             if (COMP) umma_bf16_ss(d_tmem, ((uint64_t)desc_hi << 32) | (al + (C::A_BYTES >> 4) + k * 128), bd, idesc, 1u);
                         }
-#endif
                         accum = 1;
                         umma_commit(&empty[st.idx]);     // frees the stage and (through it) the weighted-operand buffer
                         CB_TR(it, 4);
@@ -484,7 +482,6 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                 const uint8_t *xs = xy + st.idx * C::STAGE_BYTES + C::AS_OFF + off0;          // rows to be weighted
                 const uint8_t *ys = xy + st.idx * C::STAGE_BYTES + C::NBX * C::BLK + off0;    // B2: summed with the weights
                 uint8_t *ah = ab + ar.idx * (C::A_PARTS * C::A_BYTES) + off0;
-#ifndef CB_ABLATE_FOLD
                 if (rope_unit) {
                     uint8_t *xt = xy + st.idx * C::STAGE_BYTES;                       // X tile, rewritten in place
                     uint8_t *yt = xt + C::NBX * C::BLK;                               // Y tile, rewritten in place
@@ -600,7 +597,6 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                     if (cc == 0) sw += wt;
                 }
                 }
-#endif
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&afull[ar.idx]); mbar_arrive(&empty[st.idx]); }
@@ -862,11 +858,7 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     }
     const int TT = 64;
     if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
-#ifdef CB_DRAIN_TOKENS
-    P.drain_tiles = CB_DRAIN_TOKENS / TT;
-#else
     P.drain_tiles = 16384 / TT;   // at most 16384 tokens are summed in tensor memory before a drain
-#endif
     cudaError_t e;
     if (a.rope_pos) {
         if (a.compensated) e = (d == 128) ? launch_tc<128, true, false, false, true>(P, st) : launch_tc<64, true, false, false, true>(P, st);

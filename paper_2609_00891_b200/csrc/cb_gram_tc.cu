@@ -578,11 +578,7 @@ cudaError_t launch_gram2_tc(const AccumArgs &a, const FullHeadArgs &f, int d, co
     // relative drift of an all-positive sum ~2e-4 there), in equal parts.  A drain stalls the MMA thread here (both
     // accumulators belong to the unit), so fewer, longer parts than in the head-local k = 1 kernel.
     const int n_tiles = (a.n_tokens + TT - 1) / TT;
-#ifdef CB_GRAM_SUB_TILES
-    const int cap = CB_GRAM_SUB_TILES;
-#else
     const int cap = 32768 / TT;
-#endif
     const int parts = (n_tiles + cap - 1) / cap;
     P.sub_tiles = (n_tiles + parts - 1) / (parts > 0 ? parts : 1);
     if (P.sub_tiles < 1) P.sub_tiles = 1;

@@ -35,18 +35,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     asm volatile(
         "{\n\t"
         ".reg .pred p;\n\t"
-#ifdef CB_WAIT_HINT_NS
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-#else
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-#endif
         "selp.u32 %0, 1, 0, p;\n\t"
         "}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
-#ifdef CB_WAIT_HINT_NS
-          , "r"((uint32_t)CB_WAIT_HINT_NS)
-#endif
         : "memory");
     return ok != 0;
 }
