@@ -139,7 +139,7 @@ def test_config3_fullhead_sampled_group():
     Go, Co = oracle.fullhead_stats(bits(ch["src_v"].cpu()), bits(ch["tgt_v"].cpu()), wv[l].cpu().numpy(), l, sets[l])
     eg, ec = rel_fro(G[comp, l].cpu().numpy(), Go), rel_fro(C[comp, l].cpu().numpy(), Co)
     print("config 3, (V, layer 17), 2048 tokens: rel err G %.2e C %.2e" % (eg, ec))
-    assert eg <= 2e-3 and ec <= 2e-3                                   # 2,048 tokens per entry: plain-fold bound, see the design doc
+    assert eg <= 2e-3 and ec <= 2e-3                                   # 2,048 tokens per entry: the plain bf16 fold averages out like 1/sqrt(tokens)
     assert torch.isfinite(G).all() and torch.isfinite(C).all()
     # every other group must have been filled too (property check): the weight totals
     sw = torch.stack([wk.double().sum(-1), wv.double().sum(-1)]).cpu().numpy()
