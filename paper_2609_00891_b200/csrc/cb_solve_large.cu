@@ -1,8 +1,9 @@
 // Batched ridge solve for regressors wider than one head (head-local support over k > 1 selected layers, Section 3.2:
-// P = k*d + 1 up to a few thousand), where a system no longer fits in shared memory.  Blocked right-looking Cholesky
+// P = k*d + 1 up to a few thousand), where a system no longer fits in shared memory.  Blocked left-looking Cholesky
 // and blocked substitutions in fp64 on a padded copy of every system in a caller-provided workspace:
-//   per block column J (64 wide): factor the diagonal block and solve the panel below it (one block per system),
-//   then update the trailing matrix with 64 x 64 tile products (one block per tile and system);
+//   per block column J (64 wide): subtract the products of the finished block columns from column J (one block per
+//   64 x 64 tile and system, the tile held in registers over all products), factor the diagonal block, solve the
+//   panel below it;
 //   forward and backward substitution alternate a diagonal-block solve with tile updates of the remaining rows.
 // Padding rows/columns carry an identity block, so every block step has the same shape.
 #include "cb_internal.cuh"
@@ -28,24 +29,30 @@ struct LgLoadArgs {
     float lambdas[16];
 };
 
+constexpr int LG_LOAD_ROWS = 8;               // rows per block of the copy-in
+
 __global__ void __launch_bounds__(256) k_lg_load(LgArgs a, LgLoadArgs la)
 {
-    const int s = blockIdx.y, i = blockIdx.x;                 // system in the batch, row
+    const int s = blockIdx.y;                                 // system in the batch
     const int sys = la.sys0 + s, li = sys / la.n_maps, m = sys % la.n_maps;
     const float *Gm = la.G + (size_t)m * a.P * a.P;
     const float *Cm = la.C + (size_t)m * a.P * a.d;
     const double s_w = (double)Gm[(size_t)(a.P - 1) * a.P + (a.P - 1)];
     const double lam = (la.flags & CB_FLAG_RAW_LAMBDA) ? (double)la.lambdas[li] : (double)la.lambdas[li] * s_w * la.inv_n;
-    double *Ar = a.A + ((size_t)s * a.Pp + i) * a.Pp;
-    double *Zr = a.Z + ((size_t)s * a.Pp + i) * a.d;
-    for (int j = threadIdx.x; j < a.Pp; j += blockDim.x) {
-        double v;
-        if (i < a.P && j < a.P) v = (double)Gm[(size_t)i * a.P + j] + ((i == j && i < a.P - 1) ? lam : 0.0);
-        else v = (i == j) ? 1.0 : 0.0;
-        Ar[j] = v;
+    for (int q = 0; q < LG_LOAD_ROWS; ++q) {
+        const int i = blockIdx.x * LG_LOAD_ROWS + q;          // row
+        if (i >= a.Pp) break;
+        double *Ar = a.A + ((size_t)s * a.Pp + i) * a.Pp;
+        double *Zr = a.Z + ((size_t)s * a.Pp + i) * a.d;
+        for (int j = threadIdx.x; j < a.Pp; j += blockDim.x) {
+            double v;
+            if (i < a.P && j < a.P) v = (double)__ldg(Gm + (size_t)i * a.P + j) + ((i == j && i < a.P - 1) ? lam : 0.0);
+            else v = (i == j) ? 1.0 : 0.0;
+            Ar[j] = v;
+        }
+        for (int c = threadIdx.x; c < a.d; c += blockDim.x) Zr[c] = (i < a.P) ? (double)__ldg(Cm + (size_t)i * a.d + c) : 0.0;
     }
-    for (int c = threadIdx.x; c < a.d; c += blockDim.x) Zr[c] = (i < a.P) ? (double)Cm[(size_t)i * a.d + c] : 0.0;
-    if (i == 0 && threadIdx.x == 0) a.fail[s] = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) a.fail[s] = 0;
 }
 
 // ---- block column J, part 1: factor the 64 x 64 diagonal block A_JJ in place ---------------------------------------
@@ -126,12 +133,15 @@ __global__ void __launch_bounds__(128) k_lg_panel(LgArgs a, int J)
     for (int c = 0; c < LNB; c += 2) *reinterpret_cast<double2 *>(row + c) = make_double2(x[c], x[c + 1]);
 }
 
-// ---- tile products: Ctile[64 x NT] -= At[64 x 64] * Bt[64 x NT] ---------------------------------------------------
-// MODE 0 (trailing update of step J): C = A[I][I'], At = L[I][J], Bt^T = L[I'][J]      (I >= I' > J, NT = 64)
-// MODE 1 (forward substitution):      C = Z[I],     At = L[I][J], Bt = Z[J]            (I > J,  NT = d)
-// MODE 2 (backward substitution):     C = Z[I],     At = L[J][I]^T, Bt = Z[J]          (I < J,  NT = d)
+// ---- tile products: Ctile[64 x NT] -= sum_K At_K[64 x 64] * Bt_K[64 x NT] --------------------------------------------
+// MODE 0 (left-looking update of block column J before it is factored):
+//                                     C = A[I][J],  At_K = L[I][K], Bt_K^T = L[J][K], K = 0 .. J-1   (I >= J, NT = 64)
+// MODE 1 (forward substitution):      C = Z[I],     At = L[I][J],   Bt = Z[J]                        (I > J,  NT = d)
+// MODE 2 (backward substitution):     C = Z[I],     At = L[J][I]^T, Bt = Z[J]                        (I < J,  NT = d)
+// The left-looking form keeps the output tile in registers over all K: every tile of A is read and written once
+// (the right-looking form re-read and re-wrote the whole trailing matrix at every step).
 template <int MODE, int NT>
-__global__ void __launch_bounds__(256) k_lg_tile(LgArgs a, int J)
+__global__ void __launch_bounds__(256, 2) k_lg_tile(LgArgs a, int J)
 {
     extern __shared__ __align__(16) double lg_sm[];
     double (*Ats)[LPAD] = reinterpret_cast<double (*)[LPAD]>(lg_sm);                       // [k][row]
@@ -139,38 +149,11 @@ __global__ void __launch_bounds__(256) k_lg_tile(LgArgs a, int J)
     const int s = blockIdx.y, tid = threadIdx.x;
     double *A = a.A + (size_t)s * a.Pp * a.Pp;
     double *Z = a.Z + (size_t)s * a.Pp * a.d;
-    const int nblk = a.Pp / LNB;
-    int I, I2 = 0;
-    if (MODE == 0) {
-        // blockIdx.x enumerates pairs (bi >= bj) of blocks below J
-        int p = blockIdx.x, bi = 0;
-        while (p >= bi + 1) { p -= bi + 1; ++bi; }
-        I = J + 1 + bi;
-        I2 = J + 1 + p;
-    } else if (MODE == 1) {
-        I = J + 1 + blockIdx.x;
-    } else {
-        I = blockIdx.x;
-    }
-    (void)nblk;
-    // load At transposed: Ats[k][r]
-    for (int e = tid; e < LNB * LNB; e += 256) {
-        const int r = e / LNB, k = e % LNB;
-        double v;
-        if (MODE == 2) v = A[(size_t)(J * LNB + k) * a.Pp + I * LNB + r];      // L[J][I]^T
-        else v = A[(size_t)(I * LNB + r) * a.Pp + J * LNB + k];
-        Ats[k][r] = v;
-    }
-    for (int e = tid; e < LNB * NT; e += 256) {
-        if (MODE == 0) {
-            const int c = e / LNB, k = e % LNB;
-            Bts[k][c] = A[(size_t)(I2 * LNB + c) * a.Pp + J * LNB + k];
-        } else {
-            const int k = e / NT, c = e % NT;
-            Bts[k][c] = Z[(size_t)(J * LNB + k) * a.d + c];
-        }
-    }
-    __syncthreads();
+    int I;
+    if (MODE == 0) I = J + blockIdx.x;
+    else if (MODE == 1) I = J + 1 + blockIdx.x;
+    else I = blockIdx.x;
+    const int Kb = (MODE == 0) ? 0 : J, Ke = (MODE == 0) ? J : J + 1;
     // Thread (ty, tx) owns rows ty*4 .. ty*4+3 and the column pairs {32 jj + 2 tx, 32 jj + 2 tx + 1}, jj < NT/32: the 16
     // threads of a row group read 16 consecutive 16-byte pairs of Bts per access (no bank conflicts; a thread owning
     // NT/16 consecutive columns would put all 16 on two bank groups) and write 256 contiguous bytes per output row.
@@ -181,35 +164,89 @@ __global__ void __launch_bounds__(256) k_lg_tile(LgArgs a, int J)
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 2 * CJ; ++j) acc[i][j] = 0.0;
+    for (int K = Kb; K < Ke; ++K) {
+        if (K > Kb) __syncthreads();                              // the previous product has been read
+        // All global loads of the iteration are issued before the first shared-memory store (16-byte loads, fixed
+        // trip counts), so their latencies overlap instead of adding up.
+        {
+            // At transposed into Ats[k][r]: thread -> (row r, column pair k2) of a 64 x 64 tile, 8 pairs per thread
+            double2 va[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int e = tid + q * 256, r = e / (LNB / 2), k = (e % (LNB / 2)) * 2;
+                if (MODE == 2) {                                   // L[K][I]^T: rows k, k+1 of block (K, I), column r
+                    va[q].x = A[(size_t)(K * LNB + k) * a.Pp + I * LNB + r];
+                    va[q].y = A[(size_t)(K * LNB + k + 1) * a.Pp + I * LNB + r];
+                } else {
+                    va[q] = *reinterpret_cast<const double2 *>(&A[(size_t)(I * LNB + r) * a.Pp + K * LNB + k]);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int e = tid + q * 256, r = e / (LNB / 2), k = (e % (LNB / 2)) * 2;
+                Ats[k][r] = va[q].x;
+                Ats[k + 1][r] = va[q].y;
+            }
+            constexpr int NB2 = LNB * NT / 2 / 256;                // column pairs of Bt per thread, in batches of 8
+#pragma unroll
+            for (int q0 = 0; q0 < NB2; q0 += 8) {
+                double2 vb[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int e = tid + (q0 + q) * 256;
+                    if (MODE == 0) {
+                        const int c = e / (LNB / 2), k = (e % (LNB / 2)) * 2;
+                        vb[q] = *reinterpret_cast<const double2 *>(&A[(size_t)(J * LNB + c) * a.Pp + K * LNB + k]);
+                    } else {
+                        const int k = e / (NT / 2), c = (e % (NT / 2)) * 2;
+                        vb[q] = *reinterpret_cast<const double2 *>(&Z[(size_t)(K * LNB + k) * a.d + c]);
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int e = tid + (q0 + q) * 256;
+                    if (MODE == 0) {
+                        const int c = e / (LNB / 2), k = (e % (LNB / 2)) * 2;
+                        Bts[k][c] = vb[q].x;
+                        Bts[k + 1][c] = vb[q].y;
+                    } else {
+                        const int k = e / (NT / 2), c = (e % (NT / 2)) * 2;
+                        *reinterpret_cast<double2 *>(&Bts[k][c]) = vb[q];
+                    }
+                }
+            }
+        }
+        __syncthreads();
 #pragma unroll 4
-    for (int k = 0; k < LNB; ++k) {
-        double av[4], bv[2 * CJ];
+        for (int k = 0; k < LNB; ++k) {
+            double av[4], bv[2 * CJ];
 #pragma unroll
-        for (int i = 0; i < 4; i += 2) {
-            const double2 v = *reinterpret_cast<const double2 *>(&Ats[k][ty * 4 + i]);
-            av[i] = v.x; av[i + 1] = v.y;
+            for (int i = 0; i < 4; i += 2) {
+                const double2 v = *reinterpret_cast<const double2 *>(&Ats[k][ty * 4 + i]);
+                av[i] = v.x; av[i + 1] = v.y;
+            }
+#pragma unroll
+            for (int jj = 0; jj < CJ; ++jj) {
+                const double2 v = *reinterpret_cast<const double2 *>(&Bts[k][jj * 32 + tx * 2]);
+                bv[2 * jj] = v.x; bv[2 * jj + 1] = v.y;
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 2 * CJ; ++j) acc[i][j] += av[i] * bv[j];
         }
-#pragma unroll
-        for (int jj = 0; jj < CJ; ++jj) {
-            const double2 v = *reinterpret_cast<const double2 *>(&Bts[k][jj * 32 + tx * 2]);
-            bv[2 * jj] = v.x; bv[2 * jj + 1] = v.y;
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 2 * CJ; ++j) acc[i][j] += av[i] * bv[j];
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int r = I * LNB + ty * 4 + i;
-        double *crow = (MODE == 0) ? A + (size_t)r * a.Pp + I2 * LNB : Z + (size_t)r * a.d;
+        double *crow = (MODE == 0) ? A + (size_t)r * a.Pp + J * LNB : Z + (size_t)r * a.d;
 #pragma unroll
         for (int jj = 0; jj < CJ; ++jj) {
             const int c = jj * 32 + tx * 2;
             double2 v = *reinterpret_cast<double2 *>(crow + c);
             // MODE 0, diagonal tile: keep it lower-triangular
-            if (!(MODE == 0 && I == I2 && c > ty * 4 + i)) v.x -= acc[i][2 * jj];
-            if (!(MODE == 0 && I == I2 && c + 1 > ty * 4 + i)) v.y -= acc[i][2 * jj + 1];
+            if (!(MODE == 0 && I == J && c > ty * 4 + i)) v.x -= acc[i][2 * jj];
+            if (!(MODE == 0 && I == J && c + 1 > ty * 4 + i)) v.y -= acc[i][2 * jj + 1];
             *reinterpret_cast<double2 *>(crow + c) = v;
         }
     }
@@ -340,12 +377,12 @@ cudaError_t launch_solve_large(const float *G, const float *C, int n_maps, int P
         a.fail = reinterpret_cast<int *>(a.Z + (size_t)batch * Pp * d);
         a.Pp = Pp; a.P = P; a.d = d;
         la.sys0 = (int)sys0;
-        k_lg_load<<<dim3(Pp, a.nsys), 256, 0, st>>>(a, la);
+        k_lg_load<<<dim3((Pp + LG_LOAD_ROWS - 1) / LG_LOAD_ROWS, a.nsys), 256, 0, st>>>(a, la);
         for (int J = 0; J < nblk; ++J) {
+            if (J > 0) launch_tile<0, LNB>(a, J, dim3(nblk - J, a.nsys), st);      // column J -= L[:, <J] L[J, <J]^T
             k_lg_factor<<<a.nsys, 128, 0, st>>>(a, J);
             const int r = nblk - 1 - J;
             if (r > 0) k_lg_panel<<<dim3((r * LNB + 127) / 128, a.nsys), 128, 0, st>>>(a, J);
-            if (r > 0) launch_tile<0, LNB>(a, J, dim3(r * (r + 1) / 2, a.nsys), st);
         }
         if (d == 128) launch_subst_tiles<128>(a, nblk, st);
         else launch_subst_tiles<64>(a, nblk, st);
