@@ -152,6 +152,10 @@ def run_reference(args):
     print(json.dumps(out))
 
 
+TRAFFIC_DRAM_BYTES_PER_TOKEN = 435500        # dram__bytes_read + dram__bytes_write per token, k_accum_tc<128>, 14B->32B shapes
+TRAFFIC_DRAM_BYTES_PER_SPLIT = 270600000     # partial-slot read-modify-write per token split (1,024 maps)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -340,12 +344,12 @@ def main():
             "ms_per_launch": acc_avg, "algorithmic_gb_per_launch": alg_bytes * tok_launch / 1e9,
             "tflops": alg_flops * tok_launch / 1e12 / (acc_avg / 1e3),
             "tensor_frac_of_burst": alg_flops * tok_launch / 1e12 / (acc_avg / 1e3) / peaks["bf16_tflops"]}
-    tpath = os.path.join(ROOT, "profiles", "traffic_k_accum_tc.json")
-    if os.path.exists(tpath) and args.workload == WORKLOAD:
-        with open(tpath) as f:
-            t = json.load(f)     # ncu capture of a smaller launch, scaled: per-token part x tokens + slot read-modify-write per split
-            n_splits = args.splits if args.splits > 0 else 4
-            roof["traffic"] = t["dram_bytes_per_token"] * tok_launch + t["dram_bytes_fixed_per_split"] * n_splits
+    if args.workload == WORKLOAD:
+        # DRAM traffic of one launch from the ncu capture of an 8,192-token launch of the same shapes (summary:
+        # profiles/k_accum_tc_qwen14b_32b_8192tok.md), scaled: the per-token part x tokens + the read-modify-write of
+        # the partial slots per split, which does not grow with tokens
+        n_splits = args.splits if args.splits > 0 else 4
+        roof["traffic"] = TRAFFIC_DRAM_BYTES_PER_TOKEN * tok_launch + TRAFFIC_DRAM_BYTES_PER_SPLIT * n_splits
     t_roof = max(alg_bytes * tokens_per_step / (peaks["hbm_gbs"] * 1e9),
                  alg_flops * tokens_per_step / (peaks["bf16_tflops"] * 1e12))
     ms_step = total_ms / args.steps
