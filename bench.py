@@ -501,7 +501,7 @@ def multilayer_case(args, cb, synth, torch, wl, sl, sh, dev):
     del ch
     lams = list(wl.lambdas)
     nsys = len(lams) * wl.n_maps
-    ws = torch.empty(cb.cb_ridge_solve_large_workspace_bytes(P, d, min(nsys, 1024)), dtype=torch.uint8, device=dev)
+    ws = torch.empty(cb.cb_ridge_solve_large_workspace_bytes(P, d, min(nsys, 3072)), dtype=torch.uint8, device=dev)
     Wb = torch.empty(len(lams), wl.n_maps, P, d, device=dev)
     info = torch.empty(len(lams), wl.n_maps, dtype=torch.int32, device=dev)
     ts = []

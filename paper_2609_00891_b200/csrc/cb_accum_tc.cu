@@ -431,18 +431,26 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
         // follow from the previous tile's by one rotation with the thread's constants (cos, sin)(TT theta_i); the
         // special-function unit (slow: it is shared by the whole scheduler) is only used at the first tile of a unit,
         // where the positions do not advance by TT, and every 16th tile to bound the drift of the recurrence.
-        float stc[4] = {1.f, 1.f, 1.f, 1.f}, sts[4] = {0.f, 0.f, 0.f, 0.f};
-        float rcs[C::RPT][4], rsn[C::RPT][4];
+        // Packed fp32 pairs throughout: frequencies (4 cc, 4 cc + 1) and (4 cc + 2, 4 cc + 3).
+        uint64_t stc2[2] = {0ull, 0ull}, sts2[2] = {0ull, 0ull}, nsts2[2] = {0ull, 0ull};
+        uint64_t rc2[C::RPT][2], rs2[C::RPT][2];
         int rprev[C::RPT];
         int rp_lo = 0, rp_hi = 0;
         if (ROPE) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) rope_cs_poly(P.rope.f_src[cc * 4 + e], C::TT, stc[e], sts[e]);
+            for (int p = 0; p < 2; ++p) {
+                float c0, s0, c1, s1;
+                rope_cs_poly(P.rope.f_src[cc * 4 + 2 * p], C::TT, c0, s0);
+                rope_cs_poly(P.rope.f_src[cc * 4 + 2 * p + 1], C::TT, c1, s1);
+                stc2[p] = f2_pack(c0, c1);
+                sts2[p] = f2_pack(s0, s1);
+                nsts2[p] = f2_pack(-s0, -s1);
+            }
 #pragma unroll
             for (int i = 0; i < C::RPT; ++i) {
                 rprev[i] = 0;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) { rcs[i][e] = 1.f; rsn[i][e] = 0.f; }
+                for (int p = 0; p < 2; ++p) { rc2[i][p] = f2_pack(1.f, 1.f); rs2[i][p] = 0ull; }
             }
             const int lcr = cc >> 1, hb = (cc & 1) * 8, swz = rg & 7;
             rp_lo = rg * 128 + ((lcr ^ swz) << 4) + hb;
@@ -466,10 +474,6 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                 for (int e = 0; e < 4; ++e) nmu2[e] = f2_pack(-__ldg(mup + 2 * e), -__ldg(mup + 2 * e + 1));
             }
             sw = 0.f;
-            if (ROPE) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) sx[e] = sy[e] = 0.f;
-            }
             for (int t = 0; t < n_t; ++t) {
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
                 // the weighted-operand buffer was last used by tile it - NA; it is free once that tile's stage is free
@@ -491,74 +495,92 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                     for (int i = 0; i < C::RPT; ++i) {
                         const int off = i * C::RG * 128;
                         const float wt = wsm[i * C::RG];
+                        const uint64_t w2 = f2_pack(wt, wt);
                         const int pos = psm[i * C::RG];
-                        float cs[4], sn[4];
+                        uint64_t cs2[2], sn2[2];
                         if (t == 0 || pos != rprev[i] + C::TT || (t & 15) == 0) {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) rope_cs_poly(P.rope.f_src[cc * 4 + e], pos, cs[e], sn[e]);
+                            for (int p = 0; p < 2; ++p) {
+                                float c0, s0, c1, s1;
+                                rope_cs_poly(P.rope.f_src[cc * 4 + 2 * p], pos, c0, s0);
+                                rope_cs_poly(P.rope.f_src[cc * 4 + 2 * p + 1], pos, c1, s1);
+                                cs2[p] = f2_pack(c0, c1);
+                                sn2[p] = f2_pack(s0, s1);
+                            }
                         } else {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                cs[e] = fmaf(rcs[i][e], stc[e], -rsn[i][e] * sts[e]);
-                                sn[e] = fmaf(rsn[i][e], stc[e], rcs[i][e] * sts[e]);
+                            for (int p = 0; p < 2; ++p) {                              // angle += TT theta
+                                cs2[p] = f2_fma(rc2[i][p], stc2[p], f2_mul(rs2[i][p], nsts2[p]));
+                                sn2[p] = f2_fma(rs2[i][p], stc2[p], f2_mul(rc2[i][p], sts2[p]));
                             }
                         }
                         rprev[i] = pos;
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) { rcs[i][e] = cs[e]; rsn[i][e] = sn[e]; }
+                        for (int p = 0; p < 2; ++p) { rc2[i][p] = cs2[p]; rs2[i][p] = sn2[p]; }
+                        const uint64_t neg1 = f2_pack(-1.f, -1.f);
+                        uint64_t nsn2[2] = {f2_mul(sn2[0], neg1), f2_mul(sn2[1], neg1)};
                         {
                             const uint2 vl = *reinterpret_cast<const uint2 *>(xt + rp_lo + off);
                             const uint2 vh = *reinterpret_cast<const uint2 *>(xt + rp_hi + off);
-                            const float lo[4] = {__uint_as_float(vl.x << 16), __uint_as_float(vl.x & 0xffff0000u),
-                                                 __uint_as_float(vl.y << 16), __uint_as_float(vl.y & 0xffff0000u)};
-                            const float hi[4] = {__uint_as_float(vh.x << 16), __uint_as_float(vh.x & 0xffff0000u),
-                                                 __uint_as_float(vh.y << 16), __uint_as_float(vh.y & 0xffff0000u)};
-                            float nl[4], nh[4], pl[4], ph[4];
+                            const unsigned ul[2] = {vl.x, vl.y}, uh[2] = {vh.x, vh.y};
+                            unsigned xl[2], xh[2], al[2], ah2[2], bl[2], bh[2];
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {                              // rotation by -phi
-                                nl[e] = fmaf(lo[e], cs[e], hi[e] * sn[e]);
-                                nh[e] = fmaf(hi[e], cs[e], -lo[e] * sn[e]);
-                                pl[e] = wt * nl[e];
-                                ph[e] = wt * nh[e];
-                                sx[e] += pl[e];
-                                sx[4 + e] += ph[e];
+                            for (int p = 0; p < 2; ++p) {                              // rotation by -phi
+                                const uint64_t lo2 = f2_from_bf16x2(ul[p]), hi2 = f2_from_bf16x2(uh[p]);
+                                const uint64_t nl2 = f2_fma(lo2, cs2[p], f2_mul(hi2, sn2[p]));
+                                const uint64_t nh2 = f2_fma(hi2, cs2[p], f2_mul(lo2, nsn2[p]));
+                                const uint64_t pl2 = f2_mul(w2, nl2), ph2 = f2_mul(w2, nh2);
+                                sx2[p] = f2_add(sx2[p], pl2);
+                                sx2[2 + p] = f2_add(sx2[2 + p], ph2);
+                                float a0, a1;
+                                f2_unpack(nl2, a0, a1); xl[p] = pack_bf16x2(a0, a1);
+                                f2_unpack(nh2, a0, a1); xh[p] = pack_bf16x2(a0, a1);
+                                float q0, q1, r0, r1;
+                                f2_unpack(pl2, q0, q1); al[p] = pack_bf16x2(q0, q1);
+                                f2_unpack(ph2, r0, r1); ah2[p] = pack_bf16x2(r0, r1);
+                                if (COMP) {
+                                    bl[p] = pack_bf16x2(q0 - __uint_as_float(al[p] << 16), q1 - __uint_as_float(al[p] & 0xffff0000u));
+                                    bh[p] = pack_bf16x2(r0 - __uint_as_float(ah2[p] << 16), r1 - __uint_as_float(ah2[p] & 0xffff0000u));
+                                }
                             }
-                            *reinterpret_cast<uint2 *>(xt + rp_lo + off) = make_uint2(pack_bf16x2(nl[0], nl[1]), pack_bf16x2(nl[2], nl[3]));
-                            *reinterpret_cast<uint2 *>(xt + rp_hi + off) = make_uint2(pack_bf16x2(nh[0], nh[1]), pack_bf16x2(nh[2], nh[3]));
-                            const unsigned hl0 = pack_bf16x2(pl[0], pl[1]), hl1 = pack_bf16x2(pl[2], pl[3]);
-                            const unsigned hh0 = pack_bf16x2(ph[0], ph[1]), hh1 = pack_bf16x2(ph[2], ph[3]);
-                            *reinterpret_cast<uint2 *>(at + rp_lo + off) = make_uint2(hl0, hl1);
-                            *reinterpret_cast<uint2 *>(at + rp_hi + off) = make_uint2(hh0, hh1);
+                            *reinterpret_cast<uint2 *>(xt + rp_lo + off) = make_uint2(xl[0], xl[1]);
+                            *reinterpret_cast<uint2 *>(xt + rp_hi + off) = make_uint2(xh[0], xh[1]);
+                            *reinterpret_cast<uint2 *>(at + rp_lo + off) = make_uint2(al[0], al[1]);
+                            *reinterpret_cast<uint2 *>(at + rp_hi + off) = make_uint2(ah2[0], ah2[1]);
                             if (COMP) {
-                                *reinterpret_cast<uint2 *>(at + C::A_BYTES + rp_lo + off) = make_uint2(
-                                    pack_bf16x2(pl[0] - __uint_as_float(hl0 << 16), pl[1] - __uint_as_float(hl0 & 0xffff0000u)),
-                                    pack_bf16x2(pl[2] - __uint_as_float(hl1 << 16), pl[3] - __uint_as_float(hl1 & 0xffff0000u)));
-                                *reinterpret_cast<uint2 *>(at + C::A_BYTES + rp_hi + off) = make_uint2(
-                                    pack_bf16x2(ph[0] - __uint_as_float(hh0 << 16), ph[1] - __uint_as_float(hh0 & 0xffff0000u)),
-                                    pack_bf16x2(ph[2] - __uint_as_float(hh1 << 16), ph[3] - __uint_as_float(hh1 & 0xffff0000u)));
+                                *reinterpret_cast<uint2 *>(at + C::A_BYTES + rp_lo + off) = make_uint2(bl[0], bl[1]);
+                                *reinterpret_cast<uint2 *>(at + C::A_BYTES + rp_hi + off) = make_uint2(bh[0], bh[1]);
                             }
                         }
                         if (!P.rope.same) {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) rope_cs_poly(P.rope.f_tgt[cc * 4 + e], pos, cs[e], sn[e]);
+                            for (int p = 0; p < 2; ++p) {
+                                float c0, s0, c1, s1;
+                                rope_cs_poly(P.rope.f_tgt[cc * 4 + 2 * p], pos, c0, s0);
+                                rope_cs_poly(P.rope.f_tgt[cc * 4 + 2 * p + 1], pos, c1, s1);
+                                cs2[p] = f2_pack(c0, c1);
+                                sn2[p] = f2_pack(s0, s1);
+                                nsn2[p] = f2_pack(-s0, -s1);
+                            }
                         }
                         {
                             const uint2 vl = *reinterpret_cast<const uint2 *>(yt + rp_lo + off);
                             const uint2 vh = *reinterpret_cast<const uint2 *>(yt + rp_hi + off);
-                            const float lo[4] = {__uint_as_float(vl.x << 16), __uint_as_float(vl.x & 0xffff0000u),
-                                                 __uint_as_float(vl.y << 16), __uint_as_float(vl.y & 0xffff0000u)};
-                            const float hi[4] = {__uint_as_float(vh.x << 16), __uint_as_float(vh.x & 0xffff0000u),
-                                                 __uint_as_float(vh.y << 16), __uint_as_float(vh.y & 0xffff0000u)};
-                            float nl[4], nh[4];
+                            const unsigned ul[2] = {vl.x, vl.y}, uh[2] = {vh.x, vh.y};
+                            unsigned yl[2], yh[2];
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                nl[e] = fmaf(lo[e], cs[e], hi[e] * sn[e]);
-                                nh[e] = fmaf(hi[e], cs[e], -lo[e] * sn[e]);
-                                sy[e] = fmaf(wt, nl[e], sy[e]);
-                                sy[4 + e] = fmaf(wt, nh[e], sy[4 + e]);
+                            for (int p = 0; p < 2; ++p) {
+                                const uint64_t lo2 = f2_from_bf16x2(ul[p]), hi2 = f2_from_bf16x2(uh[p]);
+                                const uint64_t nl2 = f2_fma(lo2, cs2[p], f2_mul(hi2, sn2[p]));
+                                const uint64_t nh2 = f2_fma(hi2, cs2[p], f2_mul(lo2, nsn2[p]));
+                                sy2[p] = f2_fma(w2, nl2, sy2[p]);
+                                sy2[2 + p] = f2_fma(w2, nh2, sy2[2 + p]);
+                                float a0, a1;
+                                f2_unpack(nl2, a0, a1); yl[p] = pack_bf16x2(a0, a1);
+                                f2_unpack(nh2, a0, a1); yh[p] = pack_bf16x2(a0, a1);
                             }
-                            *reinterpret_cast<uint2 *>(yt + rp_lo + off) = make_uint2(pack_bf16x2(nl[0], nl[1]), pack_bf16x2(nl[2], nl[3]));
-                            *reinterpret_cast<uint2 *>(yt + rp_hi + off) = make_uint2(pack_bf16x2(nh[0], nh[1]), pack_bf16x2(nh[2], nh[3]));
+                            *reinterpret_cast<uint2 *>(yt + rp_lo + off) = make_uint2(yl[0], yl[1]);
+                            *reinterpret_cast<uint2 *>(yt + rp_hi + off) = make_uint2(yh[0], yh[1]);
                         }
                         if (cc == 0) sw += wt;
                     }
@@ -606,8 +628,7 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                 ++it;
             }
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (!rope_unit) { f2_unpack(sx2[e], sx[2 * e], sx[2 * e + 1]); f2_unpack(sy2[e], sy[2 * e], sy[2 * e + 1]); }
+            for (int e = 0; e < 4; ++e) { f2_unpack(sx2[e], sx[2 * e], sx[2 * e + 1]); f2_unpack(sy2[e], sy[2 * e], sy[2 * e + 1]); }
             // ---- bias sums of this unit: lanes holding the same channels add up, then a fixed-order sum over the
             //      warps, then read-modify-write of the slot ----
             if (C::CC == 16) {
