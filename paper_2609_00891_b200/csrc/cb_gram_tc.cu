@@ -70,6 +70,7 @@ struct GrUnit {
     int comp, l, h;               // h: target head of the map (head-local) or 0
     int group;
     int is_c;                     // C unit
+    int diag;                     // G unit with I == J: the row heads are the column heads, staged once
     int I;
     int fa[2], va[2];             // row heads (feature index) and whether the second exists
     int fb[2], vb[2];             // column heads: feature index (G units) or target head (C units)
@@ -126,6 +127,7 @@ struct GrUnit {
             vb[1] = (2 * J + 1 < f.F) ? 1 : 0;
             fb[1] = vb[1] ? 2 * J + 1 : 2 * J;
             nb = 2;
+            diag = (I == J);
 #pragma unroll
             for (int q = 0; q < 2; ++q) { lb[q] = feat_layer(fb[q]); hb[q] = feat_head(fb[q]); }
             own_sa = own_sy = own_sw = 0;
@@ -136,6 +138,7 @@ struct GrUnit {
             vb[1] = (!f.per_head && 2 * hp + 1 < NH) ? 1 : 0;
             fb[1] = vb[1] ? 2 * hp + 1 : fb[0];
             nb = f.per_head ? 1 : 2;
+            diag = 0;
 #pragma unroll
             for (int q = 0; q < 2; ++q) { lb[q] = l; hb[q] = fb[q]; }
             own_sa = (hp == 0);
@@ -245,9 +248,13 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                 for (int tile = 0; tile < n_tiles; ++tile) {
                     if (!mbar_wait(&empty[st.idx], st.phase ^ 1, abort_flag)) goto teardown;
                     uint8_t *dst = stg + st.idx * C::STAGE_BYTES + 2 * C::HEAD;
-                    mbar_arrive_expect_tx(&full[st.idx], nrow * C::HEAD);
-                    tma_load_5d(dst, map, &full[st.idx], 0, tile * C::TT, 0, un.ha[0], un.la[0]);
-                    if (un.va[1]) tma_load_5d(dst + C::HEAD, map, &full[st.idx], 0, tile * C::TT, 0, un.ha[1], un.la[1]);
+                    if (un.diag) {
+                        mbar_arrive(&full[st.idx]);              // the fold warps weight the column heads' tiles
+                    } else {
+                        mbar_arrive_expect_tx(&full[st.idx], nrow * C::HEAD);
+                        tma_load_5d(dst, map, &full[st.idx], 0, tile * C::TT, 0, un.ha[0], un.la[0]);
+                        if (un.va[1]) tma_load_5d(dst + C::HEAD, map, &full[st.idx], 0, tile * C::TT, 0, un.ha[1], un.la[1]);
+                    }
                     st.next();
                 }
             }
@@ -345,9 +352,9 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
             for (int t = 0; t < n_tiles; ++t) {
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
                 const float *wsm = wst + st.idx * C::TT + rg;
-                uint8_t *rs = stg + st.idx * C::STAGE_BYTES + (2 + g) * C::HEAD + off0;           // row head g, weighted in place
+                uint8_t *ah = stg + st.idx * C::STAGE_BYTES + (2 + g) * C::HEAD + off0;           // weighted row head g
                 const uint8_t *cs = stg + st.idx * C::STAGE_BYTES + g * C::HEAD + off0;           // column head g
-                uint8_t *ah = rs;
+                const uint8_t *rs = un.diag ? cs : ah;      // rows to weight: staged in place, or the column head itself
                 if (active) {
 #pragma unroll
                     for (int i = 0; i < C::RPT; ++i) {
