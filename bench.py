@@ -356,9 +356,9 @@ def main():
     cpu = None
     if not args.no_cpu:
         import oracle
-        dt, token_maps, rate = oracle_sample(131072)
+        dt, token_maps, rate = oracle_sample(262144)
         cpu = {"value": rate, "unit": "tokens/s", "cores": oracle.n_threads(), "kind": "oracle",
-               "sample": "64 maps x 131072 tokens of the same trace law (statistics + 3 solves) in %.1f s; "
+               "sample": "64 maps x 262144 tokens of the same trace law (statistics + 3 solves) in %.1f s; "
                          "tokens/s = token-maps / 1024 maps / s" % dt}
     out = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
