@@ -223,3 +223,58 @@ def test_apply_identity_map_turns_source_embedding_into_target_embedding():
     for l in range(wl.Lt):
         for h in range(wl.Ht):
             assert rel_fro(out_k[l, :, h, :].cpu().numpy(), src_k[sl[l], :, sh[h], :].float().numpy()) < 5e-4
+
+
+def test_rotary_boundary_for_k_selected_layers_by_composition():
+    """The paper's operating point (k > 1 selected layers, RoPE-aware interface) with the stand-alone rotation around
+    the wide-regressor calls: keys de-rotated in place, statistics over k layers, apply, target embedding restored."""
+    wl = synth.workload("mini_ragged")
+    k, base_s, base_t = 2, 1e6, 1e4
+    sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    sets = oracle.fullhead_layer_sets(wl.Ls, wl.Lt, k)
+    ch = synth.make_chunk(wl, 0, sl, sh, law=synth.map_law(wl))
+    T, d = ch["n_tokens"], wl.d
+    pos = (np.arange(T) % 700 + 11).astype(np.int32)
+    ch = dict(ch)
+    ch["src_k"] = _embed(ch["src_k"], pos, base_s)                 # stored keys carry their models' embeddings
+    ch["tgt_k"] = _embed(ch["tgt_k"], pos, base_t)
+    t = {k_: v.to(DEV) for k_, v in ch.items() if torch.is_tensor(v)}
+    posd = torch.from_numpy(pos).to(DEV)
+    sk, tk = t["src_k"].clone(), t["tgt_k"].clone()
+    cb.cb_rope_rotate(sk, posd, base_s, True)
+    cb.cb_rope_rotate(tk, posd, base_t, True)
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, d, wl.Lt, wl.Ht, d, sets)
+    P = k * d + 1
+    G = torch.zeros(wl.n_maps, P, P, device=DEV)
+    C = torch.zeros(wl.n_maps, P, d, device=DEV)
+    cb.cb_multilayer_stats_accumulate(prob, sh, sk, t["src_v"], tk, t["tgt_v"], t["w_k"], t["w_v"], G, C)
+    torch.cuda.synchronize()
+    # oracle: de-rotate in fp64, round to bf16 (the boundary stores bf16), statistics of the k-layer feature
+    def derot(x, base):
+        L, T_, H, d_ = x.shape
+        v = oracle.bf16_decode(bits(x)).reshape(L, T_, H, d_)
+        out = np.empty_like(v)
+        for l in range(L):
+            for h in range(H):
+                out[l, :, h, :] = oracle.rope_rotate(v[l, :, h, :], pos, base, inverse=True)
+        return oracle.bf16_encode(out).reshape(L, T_, H, d_)
+    src_c, tgt_c = derot(ch["src_k"], base_s), derot(ch["tgt_k"], base_t)
+    for m in (0, wl.Lt * wl.Ht - 1):                              # key maps
+        l, h = (m // wl.Ht) % wl.Lt, m % wl.Ht
+        Go, Co = oracle.multilayer_stats(src_c, tgt_c, ch["w_k"][l, h].contiguous().numpy(), l, h, int(sh[h]), sets[l])
+        eg, ec = rel_fro(G[m].cpu().numpy(), Go), rel_fro(C[m].cpu().numpy(), Co)
+        print("k=%d with rope, map %d: G %.2e C %.2e" % (k, m, eg, ec))
+        assert eg <= 2.5e-3 and ec <= 2.5e-3                      # ~1,000 tokens per map: plain bf16 fold
+    # apply: de-rotate the source cache, map, restore the target embedding
+    rng = np.random.default_rng(3)
+    Th = (rng.standard_normal((wl.n_maps, P, d)) / np.sqrt(k * d)).astype(np.float32)
+    out_k = torch.zeros(wl.Lt, T, wl.Ht, d, dtype=torch.bfloat16, device=DEV)
+    out_v = torch.zeros_like(out_k)
+    cb.cb_apply_multilayer(prob, sh, torch.from_numpy(Th).to(DEV), sk, t["src_v"], out_k, out_v)
+    cb.cb_rope_rotate(out_k, posd, base_t, False)
+    m = 1
+    l, h = (m // wl.Ht) % wl.Lt, m % wl.Ht
+    y, _ = oracle.apply_multilayer(src_c, Th[m].astype(np.float64), sets[l], int(sh[h]))
+    want = oracle.rope_rotate(oracle.bf16_decode(oracle.bf16_encode(y)).reshape(y.shape), pos, base_t)
+    got = out_k[l, :, h].float().cpu().numpy()
+    assert rel_fro(got, want) <= 4e-3                              # two bf16 roundings on the way (mapped, then rotated)
