@@ -276,6 +276,49 @@ def apply_rope_rows(x_bits: np.ndarray, Theta: np.ndarray, pos: np.ndarray, base
     return rope_rotate(mapped, pos, base_tgt, inverse=False)
 
 
+# ----------------------------------------------------------------------------- layer selector
+def probe_r2(X: np.ndarray, Y: np.ndarray, w: np.ndarray, lambda_rel: float = 0.0):
+    """Held-in R^2 (pooled over channels) of the centred weighted least-squares probe y ~ x W + b."""
+    X = np.ascontiguousarray(X, dtype=np.float64)
+    Y = np.ascontiguousarray(Y, dtype=np.float64)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    n, d = X.shape
+    r2 = ctypes.c_double(0.0)
+    lib = _load()
+    lib.orc_probe_r2.restype = ctypes.c_int32
+    info = lib.orc_probe_r2(_p(X), _p(Y), _p(w), _i64(n), _i32(d), ctypes.c_double(lambda_rel), ctypes.byref(r2))
+    return r2.value, int(info)
+
+
+def layer_scores(src_k, src_v, tgt_k, tgt_v, w_k, w_v, src_head, lambda_rel: float = 0.0, layers=None) -> np.ndarray:
+    """scores [Lt][Ls]: mean over KV heads and K/V of the probe R^2 of (source layer j, head a(h)) -> (target layer l,
+    head h).  Inputs as bf16 bit patterns [L][T][H][d] and fp32 weights [Lt][Ht][T]; `layers` restricts the target
+    layers (others stay NaN)."""
+    Ls, T, Hs, d = src_k.shape
+    Lt, _, Ht, _ = tgt_k.shape
+    dec = [bf16_decode(np.ascontiguousarray(a)).reshape(a.shape) for a in (src_k, src_v, tgt_k, tgt_v)]
+    scores = np.full((Lt, Ls), np.nan)
+    for l in (range(Lt) if layers is None else layers):
+        for j in range(Ls):
+            acc = 0.0
+            for comp in range(2):
+                for h in range(Ht):
+                    X = dec[comp][j, :, src_head[h], :]
+                    Y = dec[2 + comp][l, :, h, :]
+                    r2, _ = probe_r2(X, Y, (w_v if comp else w_k)[l, h].astype(np.float64), lambda_rel)
+                    acc += r2
+            scores[l, j] = acc / (2 * Ht)
+    return scores
+
+
+def rank_layers(scores: np.ndarray, k: int) -> np.ndarray:
+    scores = np.ascontiguousarray(scores, dtype=np.float64)
+    Lt, Ls = scores.shape
+    sets = np.empty((Lt, k), np.int32)
+    _load().orc_rank_layers(_p(scores), _i32(Lt), _i32(Ls), _i32(k), _p(sets))
+    return sets
+
+
 # ----------------------------------------------------------------------------- apply
 def apply_maps(src_k: np.ndarray, src_v: np.ndarray, Theta: np.ndarray, Lt: int, Ht: int,
                src_layer: np.ndarray, src_head: np.ndarray, maps: Optional[Sequence[int]] = None,

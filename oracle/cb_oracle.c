@@ -25,7 +25,9 @@
  * example, shift invariance and equality of the resulting map with both the
  * bias-column solve and the literal centred route; the rotary embedding
  * against a library implementation, the relative-position identity and a hand
- * example.
+ * example; the selector's probe R^2 against a library regression score and
+ * closed cases (exact linear target: 1, independent target: ~0), the ranking
+ * by brute force.
  * Parity unpinned by the paper (defined by this build, not by the paper): the
  * synthetic input laws, the nearest-depth single-layer match (k = 1), and the
  * lambda_eff = lambda * s_w / n convention for weights that are not mean-one.
@@ -481,6 +483,81 @@ void orc_rope_rotate(const double *in, double *out, int64_t n_rows, int32_t d,
             out[t * d + i] = a * c - b * s;
             out[t * d + i + half] = a * s + b * c;
         }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Layer selector (Section 3.1, first paragraph): for a target layer, every    */
+/* candidate source layer gets centred single-source-layer OLS probes under    */
+/* the same head assignment; the held-in R^2 of a probe is                     */
+/*   R^2 = 1 - sum_t w_t ||yc_t - xc_t W||^2 / sum_t w_t ||yc_t||^2            */
+/* (xc, yc centred at the weighted means, W the least-squares solution,        */
+/* residuals pooled over the d target channels: the paper does not say how the */
+/* channels are combined; this is the variance-weighted multi-output R^2).     */
+/* The layer's score is the mean over KV heads and K/V; the first k layers in  */
+/* descending score (ties: lower index) are the selected set, returned in      */
+/* ascending order.  lambda_rel > 0 adds lambda_rel * tr(A)/d to the diagonal  */
+/* (0 = plain OLS).  Returns 0, or the failing pivot of the factorisation.     */
+/* ------------------------------------------------------------------------- */
+int32_t orc_probe_r2(const double *X, const double *Y, const double *w, int64_t n, int32_t d,
+                     double lambda_rel, double *r2_out)
+{
+    double sw = 0.0;
+    double *xb = (double *)calloc((size_t)d, sizeof(double));
+    double *yb = (double *)calloc((size_t)d, sizeof(double));
+    for (int64_t t = 0; t < n; ++t) {
+        sw += w[t];
+        for (int32_t i = 0; i < d; ++i) { xb[i] += w[t] * X[t * d + i]; yb[i] += w[t] * Y[t * d + i]; }
+    }
+    if (!(sw > 0.0)) { free(xb); free(yb); *r2_out = 0.0; return 1; }
+    for (int32_t i = 0; i < d; ++i) { xb[i] /= sw; yb[i] /= sw; }
+    double *A = (double *)calloc((size_t)d * d, sizeof(double));
+    double *B = (double *)calloc((size_t)d * d, sizeof(double));
+    for (int64_t t = 0; t < n; ++t)
+        for (int32_t i = 0; i < d; ++i) {
+            const double wx = w[t] * (X[t * d + i] - xb[i]);
+            for (int32_t j = 0; j < d; ++j) {
+                A[(size_t)i * d + j] += wx * (X[t * d + j] - xb[j]);
+                B[(size_t)i * d + j] += wx * (Y[t * d + j] - yb[j]);
+            }
+        }
+    double tr = 0.0;
+    for (int32_t i = 0; i < d; ++i) tr += A[(size_t)i * d + i];
+    for (int32_t i = 0; i < d; ++i) A[(size_t)i * d + i] += lambda_rel * tr / (double)d;
+    int32_t info = orc_cholesky(A, d);
+    if (info == 0) {
+        orc_cholesky_solve(A, d, B, d);            /* B now holds W */
+        double sse = 0.0, sst = 0.0;
+        for (int64_t t = 0; t < n; ++t)
+            for (int32_t j = 0; j < d; ++j) {
+                double pred = 0.0;
+                for (int32_t i = 0; i < d; ++i) pred += (X[t * d + i] - xb[i]) * B[(size_t)i * d + j];
+                const double yc = Y[t * d + j] - yb[j];
+                sse += w[t] * (yc - pred) * (yc - pred);
+                sst += w[t] * yc * yc;
+            }
+        *r2_out = sst > 0.0 ? 1.0 - sse / sst : 0.0;
+    } else {
+        *r2_out = 0.0;
+    }
+    free(A); free(B); free(xb); free(yb);
+    return info;
+}
+
+void orc_rank_layers(const double *scores /* [Lt][Ls] */, int32_t Lt, int32_t Ls, int32_t k, int32_t *sets /* [Lt][k] */)
+{
+    for (int32_t l = 0; l < Lt; ++l) {
+        char *taken = (char *)calloc((size_t)Ls, 1);
+        for (int32_t q = 0; q < k; ++q) {
+            int32_t best = -1;
+            for (int32_t j = 0; j < Ls; ++j)
+                if (!taken[j] && (best < 0 || scores[(size_t)l * Ls + j] > scores[(size_t)l * Ls + best])) best = j;
+            taken[best] = 1;
+        }
+        int32_t q = 0;
+        for (int32_t j = 0; j < Ls; ++j)
+            if (taken[j]) sets[(size_t)l * k + q++] = j;   /* ascending */
+        free(taken);
+    }
 }
 
 /* ------------------------------------------------------------------------- */
