@@ -290,7 +290,7 @@ cb_status cb_apply_multilayer(const cb_fullhead_problem *prob, const int32_t *sr
  *              cb_apply consumes it unchanged).
  *
  * means_ws: caller-owned device memory, 256-byte aligned, at least cb_means_workspace_bytes() bytes (fp64 partial
- * sums, 8 token splits per map); it carries the first-pass state between calls.
+ * sums of w x, w y, w and w y^2, 8 token splits per map); it carries the first-pass state between calls.
  * mu: device fp32 [n_maps][2 d + 1], per map  mu_x [d], mu_y [d], s_w  (a map whose weights sum to zero gets zero
  * means).  Reduction order is fixed (per thread in token order, row groups in index order, splits in index order,
  * chunks in call order), so results are bitwise reproducible for a fixed sequence of calls.
@@ -353,6 +353,31 @@ cb_status cb_apply_rope(const cb_problem *prob, const float *Wb, const cb_kv_vie
                         void *tgt_k, void *tgt_v, int64_t t_stride_layer, int64_t t_stride_token,
                         int64_t t_stride_head, int32_t out_dtype,
                         const int32_t *positions, double rope_base_src, double rope_base_tgt, void *stream);
+
+/* ------------------------------------------------------------------------------------------------------------------
+ * Layer selector (Section 3.1, first paragraph): for each target layer, centred single-source-layer least-squares
+ * probes under the same head assignment, held-in R^2 averaged over KV heads and K/V, source layers ranked, the first k
+ * taken.  Everything comes from statistics the path produces anyway:
+ *   - a probe set = one cb_problem whose src_layer[] pairs every target layer with one candidate source layer; its
+ *     statistics (cb_stats_accumulate .. cb_stats_reduce) and its fit (cb_ridge_solve with ONE lambda, 0 for the
+ *     paper's OLS probe) are the ordinary ones; Ls probe sets with rotated src_layer[] cover every (l, j) pair;
+ *   - the target's total sum of squares comes from the first pass of the two-pass path: cb_means_energy returns
+ *     syy [n_maps][d] = sum w y^2 (device fp32) from a means workspace filled by cb_means_accumulate (the source side
+ *     of that pass does not matter);
+ *   - cb_probe_r2:  r2[m] = (tr(B^T W) + lambda_eff ||W||_F^2) / SST  with the centred B and SST formed from G, C, syy
+ *     (= 1 - SSE/SST of the fitted probe, residuals pooled over the d channels: a reading, the paper does not say how
+ *     channels are combined); G, C, Wb [n_maps][p][d] as produced for that lambda; r2 device fp32 [n_maps];
+ *   - cb_probe_scores ADDS, for every target layer l, the mean of r2 over (K/V, head) to scores[l][src_layer[l]]
+ *     (device fp32 [Lt][Ls], zeroed by the caller); src_layer is the HOST array of the probe set; Lt <= 128;
+ *   - cb_rank_layers (host arrays): the k best source layers per target layer by descending score, ties to the lower
+ *     index, written in ascending order as layer_sets [Lt][k] (the layout cb_fullhead_problem wants).
+ */
+cb_status cb_means_energy(cb_ctx *ctx, const void *means_ws, size_t means_ws_bytes, float *syy, void *stream);
+cb_status cb_probe_r2(const float *G, const float *C, const float *Wb, const float *syy, int32_t n_maps, int32_t d,
+                      int64_t n_tokens, float lambda, uint32_t flags, float *r2, void *stream);
+cb_status cb_probe_scores(const float *r2, int32_t Lt, int32_t Ht, const int32_t *src_layer, int32_t Ls, float *scores,
+                          void *stream);
+cb_status cb_rank_layers(const float *scores, int32_t Lt, int32_t Ls, int32_t k, int32_t *layer_sets);
 
 /*
  * Synchronises the stream and reads the context's device status word: CB_OK, or CB_ERR_TIMEOUT if a bounded

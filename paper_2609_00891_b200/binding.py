@@ -31,6 +31,7 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_means_workspace_bytes", "cb_means_reset", "cb_means_accumulate", "cb_means_finalize",
            "cb_stats_accumulate_centered", "cb_stats_reduce_centered", "cb_ridge_solve_centered",
            "cb_stats_accumulate_rope", "cb_rope_rotate", "cb_apply_rope",
+           "cb_means_energy", "cb_probe_r2", "cb_probe_scores", "cb_rank_layers",
            "cb_launch_count")
 
 
@@ -239,6 +240,43 @@ def cb_ridge_solve(G: torch.Tensor, C: torch.Tensor, n_tokens: int, lambdas: Seq
                                 ctypes.c_int64(n_tokens), lam.ctypes.data_as(ctypes.c_void_p), len(lam),
                                 ctypes.c_uint32(flags), ctypes.c_void_p(Wb.data_ptr()),
                                 ctypes.c_void_p(info.data_ptr()), _stream_ptr(stream)), "cb_ridge_solve")
+
+
+# ----------------------------------------------------------------------------- layer selector
+def cb_means_energy(ctx: Context, means_ws: torch.Tensor, syy: torch.Tensor, stream=None) -> None:
+    """syy: fp32 device [n_maps][d] = sum w y^2 from a means workspace filled by cb_means_accumulate."""
+    assert syy.dtype == torch.float32 and syy.is_contiguous() and syy.numel() == ctx.prob.n_maps * ctx.prob.ds
+    _check(lib().cb_means_energy(ctx.handle, ctypes.c_void_p(means_ws.data_ptr()), ctypes.c_size_t(means_ws.numel()),
+                                 ctypes.c_void_p(syy.data_ptr()), _stream_ptr(stream)), "cb_means_energy")
+
+
+def cb_probe_r2(G: torch.Tensor, C: torch.Tensor, Wb: torch.Tensor, syy: torch.Tensor, n_tokens: int, lam: float,
+                flags: int, r2: torch.Tensor, stream=None) -> None:
+    n_maps, p, _ = G.shape
+    d = p - 1
+    for t in (G, C, Wb, syy, r2):
+        assert t.dtype == torch.float32 and t.is_contiguous()
+    assert Wb.numel() == n_maps * p * d and syy.numel() == n_maps * d and r2.numel() == n_maps
+    _check(lib().cb_probe_r2(ctypes.c_void_p(G.data_ptr()), ctypes.c_void_p(C.data_ptr()), ctypes.c_void_p(Wb.data_ptr()),
+                             ctypes.c_void_p(syy.data_ptr()), n_maps, d, ctypes.c_int64(n_tokens), ctypes.c_float(lam),
+                             ctypes.c_uint32(flags), ctypes.c_void_p(r2.data_ptr()), _stream_ptr(stream)), "cb_probe_r2")
+
+
+def cb_probe_scores(r2: torch.Tensor, Lt: int, Ht: int, src_layer, Ls: int, scores: torch.Tensor, stream=None) -> None:
+    sl = np.ascontiguousarray(src_layer, dtype=np.int32)
+    assert r2.dtype == torch.float32 and scores.dtype == torch.float32 and scores.is_contiguous()
+    assert r2.numel() == 2 * Lt * Ht and scores.numel() == Lt * Ls and sl.shape == (Lt,)
+    _check(lib().cb_probe_scores(ctypes.c_void_p(r2.data_ptr()), Lt, Ht, sl.ctypes.data_as(ctypes.c_void_p), Ls,
+                                 ctypes.c_void_p(scores.data_ptr()), _stream_ptr(stream)), "cb_probe_scores")
+
+
+def cb_rank_layers(scores: np.ndarray, k: int) -> np.ndarray:
+    scores = np.ascontiguousarray(scores, dtype=np.float32)
+    Lt, Ls = scores.shape
+    sets = np.empty((Lt, k), np.int32)
+    _check(lib().cb_rank_layers(scores.ctypes.data_as(ctypes.c_void_p), Lt, Ls, k, sets.ctypes.data_as(ctypes.c_void_p)),
+           "cb_rank_layers")
+    return sets
 
 
 # ----------------------------------------------------------------------------- rotary embedding at the boundary

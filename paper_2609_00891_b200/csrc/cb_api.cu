@@ -1,4 +1,5 @@
 // Host side of the C ABI: argument validation, the static gather schedule, workspace layout and launches.
+#include <algorithm>
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
@@ -363,6 +364,64 @@ cb_status cb_means_finalize(cb_ctx *ctx, const void *means_ws, size_t means_ws_b
     cudaError_t e = launch_means_finalize(static_cast<const double *>(means_ws), ctx->n_maps, ctx->d, mu,
                                           static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+cb_status cb_means_energy(cb_ctx *ctx, const void *means_ws, size_t means_ws_bytes, float *syy, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (!means_ws || ((uintptr_t)means_ws & 255) || means_ws_bytes < means_bytes(ctx)) return CB_ERR_WORKSPACE;
+    if (!syy) return CB_ERR_INVALID_ARG;
+    cudaError_t e = launch_means_energy(static_cast<const double *>(means_ws), ctx->n_maps, ctx->d, syy,
+                                        static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------------------
+// Layer selector
+// ---------------------------------------------------------------------------------------------------------------------
+cb_status cb_probe_r2(const float *G, const float *C, const float *Wb, const float *syy, int32_t n_maps, int32_t d,
+                      int64_t n_tokens, float lambda, uint32_t flags, float *r2, void *stream)
+{
+    if (!G || !C || !Wb || !syy || !r2) return CB_ERR_INVALID_ARG;
+    if (n_maps < 0 || n_tokens < 0 || !(lambda >= 0.f)) return CB_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return CB_ERR_UNSUPPORTED;
+    if (n_maps == 0) return CB_OK;
+    cudaError_t e = launch_probe_r2(G, C, Wb, syy, n_maps, d, (double)lambda, n_tokens > 0 ? 1.0 / (double)n_tokens : 0.0,
+                                    (flags & CB_FLAG_RAW_LAMBDA) ? 1 : 0, r2, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+cb_status cb_probe_scores(const float *r2, int32_t Lt, int32_t Ht, const int32_t *src_layer, int32_t Ls, float *scores,
+                          void *stream)
+{
+    if (!r2 || !src_layer || !scores || Lt <= 0 || Ht <= 0 || Ls <= 0) return CB_ERR_INVALID_ARG;
+    if (Lt > 128) return CB_ERR_UNSUPPORTED;
+    for (int l = 0; l < Lt; ++l)
+        if (src_layer[l] < 0 || src_layer[l] >= Ls) return CB_ERR_INVALID_ARG;
+    cudaError_t e = launch_probe_scores(r2, Lt, Ht, src_layer, Ls, scores, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    return CB_OK;
+}
+
+cb_status cb_rank_layers(const float *scores, int32_t Lt, int32_t Ls, int32_t k, int32_t *layer_sets)
+{
+    if (!scores || !layer_sets || Lt <= 0 || Ls <= 0 || k <= 0 || k > Ls) return CB_ERR_INVALID_ARG;
+    std::vector<char> taken((size_t)Ls);
+    for (int l = 0; l < Lt; ++l) {
+        std::fill(taken.begin(), taken.end(), 0);
+        for (int q = 0; q < k; ++q) {
+            int best = -1;
+            for (int j = 0; j < Ls; ++j)
+                if (!taken[j] && (best < 0 || scores[(size_t)l * Ls + j] > scores[(size_t)l * Ls + best])) best = j;
+            taken[best] = 1;
+        }
+        int q = 0;
+        for (int j = 0; j < Ls; ++j)
+            if (taken[j]) layer_sets[(size_t)l * k + q++] = j;
+    }
     return CB_OK;
 }
 

@@ -49,8 +49,9 @@ struct AccumArgs {
     double rope_base_src = 0.0, rope_base_tgt = 0.0;
 };
 
-// First pass of the two-pass construction: fp64 partial sums [n_msplits][n_maps][means_stride(d)] = sum w x, sum w y, sum w.
-__host__ __device__ constexpr int means_stride(int d) { return 2 * d + 2; }
+// First pass of the two-pass construction: fp64 partial sums [n_msplits][n_maps][means_stride(d)] =
+// sum w x [d], sum w y [d], sum w, sum w y^2 [d] (the last for the layer selector's total sum of squares), padding.
+__host__ __device__ constexpr int means_stride(int d) { return 3 * d + 2; }
 constexpr int MEANS_SPLITS = 8;
 struct MeansArgs {
     KVPtr src, tgt;
@@ -96,6 +97,10 @@ cudaError_t launch_gram2_tc(const AccumArgs &a, const FullHeadArgs &f, int d, co
 cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, float *G, float *C, cudaStream_t st);
 cudaError_t launch_means(const MeansArgs &a, int d, cudaStream_t st);
 cudaError_t launch_means_finalize(const double *msum, int n_maps, int d, float *mu, cudaStream_t st);
+cudaError_t launch_means_energy(const double *msum, int n_maps, int d, float *syy, cudaStream_t st);
+cudaError_t launch_probe_r2(const float *G, const float *C, const float *Wb, const float *syy, int n_maps, int d,
+                            double lambda, double inv_n, int raw_lambda, float *r2, cudaStream_t st);
+cudaError_t launch_probe_scores(const float *r2, int Lt, int Ht, const int *src_layer_host, int Ls, float *scores, cudaStream_t st);
 cudaError_t launch_reduce_centered(const float *slots, int n_splits, int n_maps, int d, const float *mu, float *A, float *B,
                                    cudaStream_t st);
 cudaError_t launch_solve_centered(const float *A, const float *B, const float *mu, int n_maps, int d, long long n_tokens,

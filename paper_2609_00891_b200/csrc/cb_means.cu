@@ -1,6 +1,7 @@
 // Two-pass centred construction (Section 3.4): the pieces that the one-pass path does not have.
 //
-//   k_means            first pass: per map, sum w x, sum w y, sum w over a chunk, added to fp64 partial sums.
+//   k_means            first pass: per map, sum w x, sum w y, sum w (and sum w y^2, which the layer selector needs)
+//                      over a chunk, added to fp64 partial sums.
 //                      Pure streaming (every source/target element and weight is read once per map that uses it),
 //                      bound by HBM; the reduction order is fixed: a thread sums its rows in token order, the row
 //                      groups of a block are combined in index order, the block adds to its own (split, map) entry.
@@ -19,7 +20,7 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a)
     constexpr int CC = D / 8;            // 16-byte chunks per head row
     constexpr int RG = 256 / CC;         // row groups of the block
     constexpr int UN = 4;                // rows in flight per thread
-    __shared__ float red[RG][2 * D + 1];
+    __shared__ float red[RG][3 * D + 1];
     const int n_maps = 2 * a.Lt * a.Ht;
     const int m = blockIdx.x, split = blockIdx.y;
     const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
@@ -30,9 +31,9 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a)
     const __nv_bfloat16 *ys = (comp ? a.tgt.v : a.tgt.k) + (long long)l * a.tgt.sl + (long long)h * a.tgt.sh + cc * 8;
     const float *ws = (comp ? a.w_v : a.w_k) + (long long)l * a.w_sl + (long long)h * a.w_sh;
 
-    float sx[8], sy[8], sw = 0.f;
+    float sx[8], sy[8], sq[8], sw = 0.f;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) sx[e] = sy[e] = 0.f;
+    for (int e = 0; e < 8; ++e) sx[e] = sy[e] = sq[e] = 0.f;
     for (int r0 = t0 + rg; r0 < t1; r0 += UN * RG) {
         uint4 xv[UN], yv[UN];
         float wt[UN];
@@ -53,18 +54,22 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a)
             for (int e = 0; e < 4; ++e) {
                 sx[2 * e] = fmaf(wt[u], __uint_as_float(xu[e] << 16), sx[2 * e]);
                 sx[2 * e + 1] = fmaf(wt[u], __uint_as_float(xu[e] & 0xffff0000u), sx[2 * e + 1]);
-                sy[2 * e] = fmaf(wt[u], __uint_as_float(yu[e] << 16), sy[2 * e]);
-                sy[2 * e + 1] = fmaf(wt[u], __uint_as_float(yu[e] & 0xffff0000u), sy[2 * e + 1]);
+                const float y0 = __uint_as_float(yu[e] << 16), y1 = __uint_as_float(yu[e] & 0xffff0000u);
+                const float wy0 = wt[u] * y0, wy1 = wt[u] * y1;
+                sy[2 * e] += wy0;
+                sy[2 * e + 1] += wy1;
+                sq[2 * e] = fmaf(wy0, y0, sq[2 * e]);
+                sq[2 * e + 1] = fmaf(wy1, y1, sq[2 * e + 1]);
             }
             sw += wt[u];
         }
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) { red[rg][cc * 8 + e] = sx[e]; red[rg][D + cc * 8 + e] = sy[e]; }
+    for (int e = 0; e < 8; ++e) { red[rg][cc * 8 + e] = sx[e]; red[rg][D + cc * 8 + e] = sy[e]; red[rg][2 * D + 1 + cc * 8 + e] = sq[e]; }
     if (cc == 0) red[rg][2 * D] = sw;
     __syncthreads();
     double *dst = a.msum + ((size_t)split * n_maps + m) * means_stride(D);
-    for (int v = threadIdx.x; v < 2 * D + 1; v += 256) {
+    for (int v = threadIdx.x; v < 3 * D + 1; v += 256) {
         double sum = 0.0;
 #pragma unroll 4
         for (int g = 0; g < RG; ++g) sum += (double)red[g][v];
@@ -93,6 +98,25 @@ __global__ void k_means_finalize(const double *__restrict__ msum, int n_maps, in
         for (int s = 0; s < MEANS_SPLITS; ++s) sum += msum[((size_t)s * n_maps + m) * ms + v];
         mu[(size_t)m * (2 * d + 1) + v] = (v == 2 * d) ? (float)sw : (sw > 0.0 ? (float)(sum / sw) : 0.f);
     }
+}
+
+// syy [n_maps][d] = sum over the calibration rows of w y^2 per target channel (splits summed in index order)
+__global__ void k_means_energy(const double *__restrict__ msum, int n_maps, int d, float *__restrict__ syy)
+{
+    const int m = blockIdx.x, ms = means_stride(d);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        double sum = 0.0;
+        for (int s = 0; s < MEANS_SPLITS; ++s) sum += msum[((size_t)s * n_maps + m) * ms + 2 * d + 1 + c];
+        syy[(size_t)m * d + c] = (float)sum;
+    }
+}
+
+cudaError_t launch_means_energy(const double *msum, int n_maps, int d, float *syy, cudaStream_t st)
+{
+    k_means_energy<<<n_maps, 128, 0, st>>>(msum, n_maps, d, syy);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) count_launch();
+    return e;
 }
 
 cudaError_t launch_means_finalize(const double *msum, int n_maps, int d, float *mu, cudaStream_t st)

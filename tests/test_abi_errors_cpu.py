@@ -92,7 +92,7 @@ def test_workspace_and_static_limits():
 def test_two_pass_entry_points_reject_bad_arguments_on_the_host():
     sl, sh = cb.cb_head_map_nearest(40, 8, 64, 8)
     prob = cb.Problem(40, 8, 128, 64, 8, 128, sl, sh)
-    assert cb.cb_means_workspace_bytes(prob) == 8 * 1024 * (2 * 128 + 2) * 8          # fp64, 8 splits per map
+    assert cb.cb_means_workspace_bytes(prob) == 8 * 1024 * (3 * 128 + 2) * 8          # fp64, 8 splits per map
     null = ctypes.c_void_p(0)
     L = cb.lib()
     assert L.cb_means_reset(null, ctypes.c_void_p(0x1000), ctypes.c_size_t(1 << 30), null) == cb.CB_ERR_STATE
@@ -108,3 +108,19 @@ def test_two_pass_entry_points_reject_bad_arguments_on_the_host():
     assert call(0x10, 0x10, 0x10, 4, 128, 17) == cb.CB_ERR_INVALID_ARG
     assert call(0x10, 0x10, 0x10, 0, 128, 1) == cb.CB_OK
     assert cb.cb_launch_count() == before
+
+
+def test_selector_host_logic_and_argument_errors():
+    scores = np.array([[0.1, 0.9, 0.9, 0.3], [0.5, 0.2, 0.7, 0.6]], np.float32)
+    assert cb.cb_rank_layers(scores, 1).tolist() == [[1], [2]]                          # tie -> lower index
+    assert cb.cb_rank_layers(scores, 2).tolist() == [[1, 2], [2, 3]]
+    assert cb.cb_rank_layers(scores, 4).tolist() == [[0, 1, 2, 3], [0, 1, 2, 3]]
+    L = cb.lib()
+    null = ctypes.c_void_p(0)
+    assert L.cb_rank_layers(scores.ctypes.data_as(ctypes.c_void_p), 2, 4, 5, ctypes.c_void_p(0x10)) == cb.CB_ERR_INVALID_ARG
+    assert L.cb_probe_r2(null, null, null, null, 4, 128, ctypes.c_int64(10), ctypes.c_float(0), 0, null, null) == cb.CB_ERR_INVALID_ARG
+    p = ctypes.c_void_p(0x10)
+    assert L.cb_probe_r2(p, p, p, p, 4, 96, ctypes.c_int64(10), ctypes.c_float(0), 0, p, null) == cb.CB_ERR_UNSUPPORTED
+    assert L.cb_probe_r2(p, p, p, p, 0, 128, ctypes.c_int64(10), ctypes.c_float(0), 0, p, null) == cb.CB_OK
+    bad = np.array([0, 7], np.int32)
+    assert L.cb_probe_scores(p, 2, 2, bad.ctypes.data_as(ctypes.c_void_p), 4, p, null) == cb.CB_ERR_INVALID_ARG

@@ -20,7 +20,7 @@ def _built():
 
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "cb.h")).read()
-    declared = set(re.findall(r"\b(cb_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(cb_[a-z0-9_]+)\s*\(", header))
     assert declared == set(cb.EXPORTS)
     L = cb.lib()
     for name in declared:
