@@ -179,6 +179,9 @@ def main():
     ap.add_argument("--rope", action="store_true",
                     help="fit the key maps in content coordinates: rotary embedding (base 1e6, positions restart every "
                          "1024 tokens) removed inside the accumulate kernel; the JSON line says so in config")
+    ap.add_argument("--selector", type=int, default=0, metavar="SETS",
+                    help="time this many probe sets of the layer selector (one candidate source layer per target layer "
+                         "each) on one 50-sequence chunk and print its own JSON line")
     ap.add_argument("--two-pass", action="store_true",
                     help="time the two-pass centred construction (means pass, centred accumulation, reduce, centred solve) "
                          "on the selected workload and print its own JSON line")
@@ -218,6 +221,9 @@ def main():
         return
     if args.multilayer > 0:
         multilayer_case(args, cb, synth, torch, wl, sl, sh, dev)
+        return
+    if args.selector > 0:
+        selector_case(args, cb, synth, torch, wl, dev)
         return
     if args.two_pass and args.profile_tokens <= 0:
         two_pass_case(args, cb, synth, torch, wl, sl, sh, dev)
@@ -377,6 +383,62 @@ def main():
            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "apply": apply_info,
            "gpu_launches": launches, "clocks": clocks}
     print(json.dumps(out))
+
+
+def selector_case(args, cb, synth, torch, wl, dev):
+    """Layer selector: probe sets with rotated layer pairing on one chunk (statistics, OLS fit, R^2, scores)."""
+    import numpy as np
+    sl0, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    ch = synth.make_chunk(wl, 0, sl0, sh, device=dev)
+    T, d, p = ch["n_tokens"], wl.d, wl.d + 1
+    scores = torch.zeros(wl.Lt, wl.Ls, device=dev)
+    G = torch.empty(wl.n_maps, p, p, device=dev)
+    C = torch.empty(wl.n_maps, p, d, device=dev)
+    Wb = torch.empty(1, wl.n_maps, p, d, device=dev)
+    info = torch.empty(1, wl.n_maps, dtype=torch.int32, device=dev)
+    r2 = torch.empty(wl.n_maps, device=dev)
+    syy = torch.empty(wl.n_maps, d, device=dev)
+    times = {"energy": None, "accumulate": [], "reduce_solve_r2": []}
+
+    def timed(fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1)
+
+    for r in range(args.selector):
+        sl = np.array([(int(sl0[l]) + r) % wl.Ls for l in range(wl.Lt)], np.int32)
+        prob = cb.Problem(wl.Ls, wl.Hs, d, wl.Lt, wl.Ht, d, sl, sh)
+        ctx = cb.cb_create(prob, device=dev)
+        if r == 0:
+            ws = torch.empty(cb.cb_means_workspace_bytes(prob), dtype=torch.uint8, device=dev)
+            cb.cb_means_reset(ctx, ws)
+
+            def energy():
+                cb.cb_means_accumulate(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"], ws)
+                cb.cb_means_energy(ctx, ws, syy)
+            times["energy"] = timed(energy)
+        times["accumulate"].append(timed(lambda: cb.cb_stats_accumulate(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"],
+                                                                        ch["w_k"], ch["w_v"])))
+
+        def rest():
+            n = cb.cb_stats_reduce(ctx, G, C)
+            cb.cb_ridge_solve(G, C, n, [0.0], 0, Wb, info)
+            cb.cb_probe_r2(G, C, Wb[0], syy, n, 0.0, 0, r2)
+            cb.cb_probe_scores(r2, wl.Lt, wl.Ht, sl, wl.Ls, scores)
+        times["reduce_solve_r2"].append(timed(rest))
+        cb.cb_device_status(ctx)
+        del ctx
+    cb.cb_check_info(info)
+    sets = cb.cb_rank_layers(scores.cpu().numpy(), 1)
+    acc, rest_ms = statistics.mean(times["accumulate"][1:] or times["accumulate"]), statistics.mean(times["reduce_solve_r2"])
+    print(json.dumps({"workload": "layer selector, %s shapes, %d probe sets on one chunk of %d tokens" % (args.workload, args.selector, T),
+                      "ms": {"target_energy_pass": times["energy"], "accumulate_per_set": acc, "reduce_solve_r2_per_set": rest_ms},
+                      "s_all_layer_pairs_per_chunk": (times["energy"] + wl.Ls * (acc + rest_ms)) / 1e3,
+                      "nearest_depth_ranked_first_for_layers": int(sum(int(sets[l][0]) == int(sl0[l]) for l in range(wl.Lt))),
+                      "n_target_layers": wl.Lt}))
 
 
 def two_pass_case(args, cb, synth, torch, wl, sl, sh, dev):
