@@ -29,8 +29,11 @@
  * closed cases (exact linear target: 1, independent target: ~0), the ranking
  * by brute force.
  * Parity unpinned by the paper (defined by this build, not by the paper): the
- * synthetic input laws, the nearest-depth single-layer match (k = 1), and the
- * lambda_eff = lambda * s_w / n convention for weights that are not mean-one.
+ * synthetic input laws, the nearest-depth single-layer match (k = 1), the
+ * lambda_eff = lambda * s_w / n convention for weights that are not mean-one,
+ * the rotate-half pairing of the rotary embedding, and the pooling of the
+ * selector's R^2 over target channels (each is pinned as an implementation of
+ * the stated convention; the convention itself is this build's reading).
  */
 #include <math.h>
 #ifdef _OPENMP
