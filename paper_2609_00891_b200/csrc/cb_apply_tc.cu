@@ -5,8 +5,11 @@
 //                     tensor core reads (rows = input channel, 64 output channels per 128-byte row, swizzled);
 //                     the bias row goes to shared memory as fp32.
 //   producer thread   TMA: tiles of 128 tokens of the matched source head, [channel block][token][64 channels].
-//   MMA thread        tcgen05.mma  D[128 tokens][d] += X[128][16] * W[16][d], A K-major, B MN-major, twice per
-//                     K step (hi and lo part of W), fp32 accumulators in tensor memory (two, ping-pong).
+//   MMA thread        tcgen05.mma  D[128 tokens][2d] += X[128][16] * [W_hi | W_lo][16][2d], A K-major, B MN-major: the hi
+//                     and lo parts of W sit side by side as one N = 2d operand, so the X tile is read from shared
+//                     memory once per K step (two MMAs of N = d read it twice: shared-memory bandwidth is what this
+//                     kernel runs out of next to HBM); fp32 accumulators in tensor memory (two, ping-pong); the
+//                     epilogue adds the two halves.
 //   epilogue warps    tensor memory -> registers, + bias, -> bf16 into a shared-memory tile -> one TMA store
 //                     (coalesced 256-byte rows, rows past the end clipped); fp32 output is stored directly.
 // Every wait is bounded; a wait that runs out makes the block tear down (nothing else is reported: this call has
@@ -26,7 +29,7 @@
 #define CB_AP_NO 2
 #endif
 #ifndef CB_AP_NACC
-#define CB_AP_NACC 4
+#define CB_AP_NACC 2
 #endif
 
 namespace cb {
@@ -48,7 +51,8 @@ struct ApCfg {
     static constexpr int NS = CB_AP_NS;
     static constexpr int NO = CB_AP_NO;                 // output tiles in shared memory
     static constexpr int NACC = CB_AP_NACC;
-    static constexpr int TMEM_COLS = (NACC * D < 32) ? 32 : NACC * D;
+    static constexpr int AW = 2 * D;                    // accumulator columns per tile: X W_hi | X W_lo
+    static constexpr int TMEM_COLS = (NACC * AW < 32) ? 32 : NACC * AW;
     static constexpr int EPI_WARPS = 4, CONV_WARPS = 4;
     static constexpr int THREADS = (2 + EPI_WARPS + CONV_WARPS) * 32;
     static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * X_BYTES + 2 * (size_t)W_BYTES + (size_t)NO * O_BYTES + D * 4 + 256;
@@ -180,8 +184,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
     } else if (warp == 1) {
         // ================================ MMA issuer (one thread) ================================
         if (lane == 0) {
-            constexpr uint32_t idesc_bf = umma_idesc_bf16(128, D, false, true);   // A K-major, B MN-major
-            constexpr uint32_t idesc_hf = umma_idesc_f16(128, D, false, true);
+            constexpr uint32_t idesc_bf = umma_idesc_bf16(128, 2 * D, false, true);   // A K-major, B MN-major, N = hi | lo
+            constexpr uint32_t idesc_hf = umma_idesc_f16(128, 2 * D, false, true);
             // A (K-major, 128-byte swizzle): 8-row groups 1024 bytes apart; a K step of 16 channels is 32 bytes along
             // the row, a block of 64 channels is XBLK further.  B (MN-major): K step = 16 rows = 2048 bytes,
             // 64-output-channel blocks WBLK apart.
@@ -190,7 +194,6 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
             const uint32_t a_hi32 = (uint32_t)(proto_a >> 32), b_hi32 = (uint32_t)(proto_b >> 32);
             const uint32_t a_lo0 = (uint32_t)proto_a | ((smem_u32(xs) & 0x3FFFFu) >> 4);
             const uint32_t bh_lo0 = (uint32_t)proto_b | ((smem_u32(whi) & 0x3FFFFu) >> 4);
-            const uint32_t bl_lo0 = (uint32_t)proto_b | ((smem_u32(wlo) & 0x3FFFFu) >> 4);
             ApIter cur;
             cur.start(n_units, n_maps, n_tiles, P.n_splits);
             ApRing<C::NS> st;
@@ -204,14 +207,14 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                     if (!mbar_wait(ROPE ? &xrot[st.idx] : &xfull[st.idx], st.phase, abort_flag)) goto teardown;
                     if (!mbar_wait(&accempty[ac.idx], ac.phase ^ 1, abort_flag)) goto teardown;
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + ac.idx * D;
+                    const uint32_t d_tmem = tmem_base + ac.idx * C::AW;
                     const uint32_t al = a_lo0 + st.idx * (C::X_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k) {
                         const uint32_t ak = al + (k >> 2) * (C::XBLK >> 4) + (k & 3) * 2;          // +32 bytes per K step
                         const uint64_t ad = ((uint64_t)a_hi32 << 32) | ak;
+                        // the lo image follows the hi image in shared memory: 2 d / 64 column blocks, WBLK apart
                         umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bh_lo0 + k * 128), idesc, k == 0 ? 0u : 1u);
-                        umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bl_lo0 + k * 128), idesc, 1u);
                     }
                     umma_commit(&xempty[st.idx]);
                     umma_commit(&accfull[ac.idx]);
@@ -243,7 +246,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
             for (int tile = cur.tile; tile < cur.tile1; ++tile) {
                 if (!mbar_wait_warp(&accfull[ac.idx], ac.phase, abort_flag, lane)) goto teardown;
                 tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ac.idx * D;
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ac.idx * C::AW;
                 const int tok = tile * C::TT + row;
                 const bool rope_unit = ROPE && comp == 0;
                 if (rope_unit) {
@@ -255,9 +258,19 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
 #pragma unroll 1
                     for (int c = 0; c < D / 64; ++c) {
                         uint32_t rl[32], rh[32];
-                        tmem_ld_32x32(taddr + c * 32, rl);
-                        tmem_ld_32x32(taddr + D / 2 + c * 32, rh);
-                        tmem_wait_ld();
+                        {
+                            uint32_t tl[32], th[32];
+                            tmem_ld_32x32(taddr + c * 32, rl);
+                            tmem_ld_32x32(taddr + D + c * 32, tl);               // lo-part products
+                            tmem_ld_32x32(taddr + D / 2 + c * 32, rh);
+                            tmem_ld_32x32(taddr + D + D / 2 + c * 32, th);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                rl[j] = __float_as_uint(__uint_as_float(rl[j]) + __uint_as_float(tl[j]));
+                                rh[j] = __float_as_uint(__uint_as_float(rh[j]) + __uint_as_float(th[j]));
+                            }
+                        }
                         float ol[32], oh[32];
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
@@ -313,8 +326,14 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
 #pragma unroll 1
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
-                        tmem_ld_32x32(taddr + c * 32, r);
-                        tmem_wait_ld();
+                        {
+                            uint32_t t2[32];
+                            tmem_ld_32x32(taddr + c * 32, r);
+                            tmem_ld_32x32(taddr + D + c * 32, t2);               // lo-part products
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(t2[j]));
+                        }
 #pragma unroll
                         for (int v = 0; v < 4; ++v) {           // 4 chunks of 8 channels
                             const int n0 = c * 32 + v * 8;
@@ -352,8 +371,14 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
 #pragma unroll 1
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
-                        tmem_ld_32x32(taddr + c * 32, r);
-                        tmem_wait_ld();
+                        {
+                            uint32_t t2[32];
+                            tmem_ld_32x32(taddr + c * 32, r);
+                            tmem_ld_32x32(taddr + D + c * 32, t2);               // lo-part products
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(t2[j]));
+                        }
                         if (tok < a.n_tokens) {
 #pragma unroll
                             for (int v = 0; v < 8; ++v) {
