@@ -44,7 +44,8 @@ typedef enum cb_status {
 /* flags (cb_problem.flags and the flags argument of cb_ridge_solve) */
 #define CB_FLAG_COMPENSATED 1u /* accumulate: split the bf16 weighted operand into hi + lo (two MMAs per   */
                                /* tile) so that folding the fp32 weight into a bf16 operand costs ~2^-17   */
-                               /* instead of ~2^-9 per element.  Meant for small token counts.             */
+                               /* instead of ~2^-9 per element.  Meant for small token counts; calls of     */
+                               /* fewer than 4,096 rows use it in any case.                                 */
 #define CB_FLAG_RAW_LAMBDA  2u /* solve: penalise with lambda itself instead of lambda * s_w / n            */
 #define CB_FLAG_SIMT        4u /* accumulate/apply: use the plain fp32 CUDA-core kernels (no tensor cores) */
 #define CB_FLAG_ONE_ROW_HEAD 8u /* cb_fullhead_problem only: statistics by the kernel that weights one feature head  */

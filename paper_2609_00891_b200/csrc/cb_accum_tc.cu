@@ -881,13 +881,16 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
     P.drain_tiles = 16384 / TT;   // at most 16384 tokens are summed in tensor memory before a drain
     cudaError_t e;
+    // Calls of fewer than 4,096 rows take the hi + lo weighted operand regardless of the flag: the single bf16
+    // rounding averages out only like 1/sqrt(rows), such calls are bound by launch latency, not by the second MMA.
+    const bool comp = a.compensated || a.n_tokens < 4096;
     if (a.rope_pos) {
-        if (a.compensated) e = (d == 128) ? launch_tc<128, true, false, false, true>(P, st) : launch_tc<64, true, false, false, true>(P, st);
+        if (comp) e = (d == 128) ? launch_tc<128, true, false, false, true>(P, st) : launch_tc<64, true, false, false, true>(P, st);
         else e = (d == 128) ? launch_tc<128, false, false, false, true>(P, st) : launch_tc<64, false, false, false, true>(P, st);
     } else if (a.mu) {
-        if (a.compensated) e = (d == 128) ? launch_tc<128, true, false, true>(P, st) : launch_tc<64, true, false, true>(P, st);
+        if (comp) e = (d == 128) ? launch_tc<128, true, false, true>(P, st) : launch_tc<64, true, false, true>(P, st);
         else e = (d == 128) ? launch_tc<128, false, false, true>(P, st) : launch_tc<64, false, false, true>(P, st);
-    } else if (a.compensated) e = (d == 128) ? launch_tc<128, true>(P, st) : launch_tc<64, true>(P, st);
+    } else if (comp) e = (d == 128) ? launch_tc<128, true>(P, st) : launch_tc<64, true>(P, st);
     else e = (d == 128) ? launch_tc<128, false>(P, st) : launch_tc<64, false>(P, st);
     if (e == cudaSuccess) count_launch();
     return e;

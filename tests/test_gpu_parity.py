@@ -73,13 +73,11 @@ CASES = [
 
 
 def _tol(wl, flags):
-    """1e-3 is the stated target.  The plain (single bf16) weight fold rounds every w*x to 8 significant bits;
-    these roundings are independent across tokens, so the relative error of a sum over n tokens falls like
-    1/sqrt(n): measured 1.1e-3 on C at n = 797, 5e-4 expected by n = 4096.  Below 4096 tokens per map the plain
-    fold is only held to 2e-3 here (the compensated fold is the documented choice for such sizes)."""
-    if flags & (cb.CB_FLAG_SIMT | cb.CB_FLAG_COMPENSATED) or wl.n_tokens >= 4096:
-        return TOL
-    return 2e-3
+    """1e-3 is the stated target.  The plain (single bf16) weight fold rounds every w*x to 8 significant bits; these
+    roundings are independent across tokens, so the relative error of a sum over n tokens falls like 1/sqrt(n)
+    (measured 1.1e-3 on C at n = 797).  The library therefore takes the hi + lo fold for every call of fewer than
+    4,096 rows, and the target holds at every size."""
+    return TOL
 
 
 

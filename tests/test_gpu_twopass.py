@@ -1,7 +1,6 @@
 """Parity of the two-pass centred construction (Section 3.4) against the fp64 oracle, through the C ABI.
 
-Tolerance: relative Frobenius error <= 1e-3 on the centred statistics A, B and on the maps (2e-3 below 4096 tokens
-per map for the single-bf16 weighted operand, as for the one-pass path); means to fp32 accuracy."""
+Tolerance: relative Frobenius error <= 1e-3 on the centred statistics A, B and on the maps; means to fp32 accuracy."""
 import numpy as np
 import pytest
 import torch
@@ -95,7 +94,7 @@ def test_two_pass_matches_oracle(name, flags, n_splits):
     scale = np.abs(np.concatenate([mu_x, mu_y], axis=1)).max() + 1.0
     assert np.abs(muc[:, :d] - mu_x).max() <= 2e-6 * scale and np.abs(muc[:, d:2 * d] - mu_y).max() <= 2e-6 * scale
     assert np.allclose(muc[:, 2 * d], sw, rtol=1e-6)
-    tol = 1e-3 if (flags & cb.CB_FLAG_COMPENSATED or wl.n_tokens >= 4096) else 2e-3
+    tol = 1e-3                      # calls of fewer than 4,096 rows take the hi + lo fold by themselves
     print("%s flags=%d: A %.2e (max map %.2e)  B %.2e (max map %.2e)" % (
         name, flags, rel_fro(Ac, Ao), max_rel_fro_per_map(Ac, Ao), rel_fro(Bc, Bo), max_rel_fro_per_map(Bc, Bo)))
     assert np.isfinite(Ac).all() and np.isfinite(Bc).all()
