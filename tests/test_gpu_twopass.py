@@ -205,3 +205,25 @@ def test_argument_errors():
     with pytest.raises(cb.CbError) as e:
         cb.cb_stats_accumulate_centered(ctx2, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"], mu)
     assert e.value.status == cb.CB_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("T", [1, 65, 200])
+def test_two_pass_few_rows(T):
+    wl = synth.workload("mini_scaled")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    ch = _chunks(wl, sl, sh)[0]
+    cut = {k: (v[:, :T].contiguous() if k[:3] in ("src", "tgt") else v[:, :, :T].contiguous()) for k, v in ch.items() if torch.is_tensor(v)}
+    mu_x, mu_y, sw, Ao, Bo = _oracle_twopass([cut], sl, sh)
+    import dataclasses
+    small = dataclasses.replace(wl, seq_lens=(T,), seqs_per_chunk=1)
+    prob, ctx, mu, A, B, n = _gpu_twopass(small, [cut], sl, sh)
+    assert n == T
+    d = wl.d
+    muc = mu.cpu().numpy().astype(np.float64)
+    assert np.allclose(muc[:, :d], mu_x, atol=1e-5) and np.allclose(muc[:, d:2 * d], mu_y, atol=1e-5)
+    Ac, Bc = A.cpu().numpy(), B.cpu().numpy()
+    assert np.isfinite(Ac).all() and np.isfinite(Bc).all()
+    if T == 1:
+        assert np.abs(Ac).max() <= 1e-3 and np.abs(Bc).max() <= 1e-3          # one row: centred statistics vanish
+    else:
+        assert max_rel_fro_per_map(Ac, Ao) <= 1e-3 and max_rel_fro_per_map(Bc, Bo) <= 1e-3
