@@ -152,7 +152,7 @@ def run_reference(args):
     print(json.dumps(out))
 
 
-TRAFFIC_DRAM_BYTES_PER_TOKEN = 435500        # dram__bytes_read + dram__bytes_write per token, k_accum_tc<128>, 14B->32B shapes
+TRAFFIC_DRAM_BYTES_PER_TOKEN = 440400        # dram__bytes_read + dram__bytes_write per token, k_accum_ts, 14B->32B shapes
 TRAFFIC_DRAM_BYTES_PER_SPLIT = 270600000     # partial-slot read-modify-write per token split (1,024 maps)
 
 
@@ -345,14 +345,14 @@ def main():
     acc_avg = statistics.mean(acc_ms)
     tok_launch = tokens_per_step / n_chunks
     achieved = alg_bytes * tok_launch / 1e9 / (acc_avg / 1e3)
-    roof = {"bound": "hbm", "kernel": "k_accum_tc<128>", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+    roof = {"bound": "hbm", "kernel": "k_accum_ts<plain>", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
             "ms_per_launch": acc_avg, "algorithmic_gb_per_launch": alg_bytes * tok_launch / 1e9,
             "tflops": alg_flops * tok_launch / 1e12 / (acc_avg / 1e3),
             "tensor_frac_of_burst": alg_flops * tok_launch / 1e12 / (acc_avg / 1e3) / peaks["bf16_tflops"]}
     if args.workload == WORKLOAD:
         # DRAM traffic of one launch from the ncu capture of an 8,192-token launch of the same shapes (summary:
-        # profiles/k_accum_tc_qwen14b_32b_8192tok.md), scaled: the per-token part x tokens + the read-modify-write of
+        # profiles/k_accum_ts_qwen14b_32b_8192tok.md), scaled: the per-token part x tokens + the read-modify-write of
         # the partial slots per split, which does not grow with tokens
         n_splits = args.splits if args.splits > 0 else 4
         roof["traffic"] = TRAFFIC_DRAM_BYTES_PER_TOKEN * tok_launch + TRAFFIC_DRAM_BYTES_PER_SPLIT * n_splits
@@ -501,7 +501,7 @@ def two_pass_case(args, cb, synth, torch, wl, sl, sh, dev):
                                        "solve": statistics.mean([r["solve"] for r in runs])},
                       "roofline_means": {"bound": "hbm", "kernel": "k_means", "achieved": gb / (means_ms / 1e3),
                                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gb / (means_ms / 1e3) / peaks["hbm_gbs"]},
-                      "roofline_accumulate": {"bound": "hbm", "kernel": "k_accum_tc<128, centred>", "achieved": gb / (acc_ms / 1e3),
+                      "roofline_accumulate": {"bound": "hbm", "kernel": "k_accum_ts<centred>", "achieved": gb / (acc_ms / 1e3),
                                               "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gb / (acc_ms / 1e3) / peaks["hbm_gbs"]},
                       "frac_of_roofline_whole_build": 2 * alg_bytes * tok_launch * n_chunks / (peaks["hbm_gbs"] * 1e9) / (step_ms / 1e3)}))
 

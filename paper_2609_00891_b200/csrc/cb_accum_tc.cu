@@ -879,11 +879,17 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     }
     const int TT = 64;
     if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
-    P.drain_tiles = 16384 / TT;   // at most 16384 tokens are summed in tensor memory before a drain
     cudaError_t e;
     // Calls of fewer than 4,096 rows take the hi + lo weighted operand regardless of the flag: the single bf16
     // rounding averages out only like 1/sqrt(rows), such calls are bound by launch latency, not by the second MMA.
     const bool comp = a.compensated || a.n_tokens < 4096;
+    // Tokens summed in tensor memory before a drain (the fp32 accumulation of the tensor cores loses about 1e-4 over
+    // 16,384 tokens; the compensated fold drains eight times as often).
+    P.drain_tiles = (comp ? 2048 : 16384) / TT;
+#ifndef CB_NO_TS
+    // d = 128 without the rotary fold: the kernel that keeps the weighted operand in tensor memory
+    if (d == 128 && !a.rope_pos) return launch_accum_ts(a, comp, src, tgt, st);
+#endif
     if (a.rope_pos) {
         if (comp) e = (d == 128) ? launch_tc<128, true, false, false, true>(P, st) : launch_tc<64, true, false, false, true>(P, st);
         else e = (d == 128) ? launch_tc<128, false, false, false, true>(P, st) : launch_tc<64, false, false, false, true>(P, st);

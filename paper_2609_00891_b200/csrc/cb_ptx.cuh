@@ -157,6 +157,19 @@ __device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, u
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// D[tmem] (+)= A[tmem] * B[smem]: the first operand is read from tensor memory (lane = row of A, two bf16 of
+// consecutive K per 32-bit column: K = 16 takes 8 columns), K-major by construction.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // Arrive on an mbarrier once all tcgen05 operations issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint64_t *bar)
 {
@@ -188,6 +201,29 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16])
         : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Store 16 lanes x 16 columns: thread i holds, for n = 0..3, register 2n = (lane i/4, column 4n + i%4) and register
+// 2n+1 = (lane i/4 + 8, column 4n + i%4): the register layout that ldmatrix (8x8, 16-bit, transposed) produces.
+__device__ __forceinline__ void tmem_st_16x128_x4(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.16x128b.x4.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Four 8x8 matrices of 16-bit elements, transposed: thread i supplies the address of row i%8 of matrix i/8 and
+// receives in register j the elements (row 2(i%4), column i/4) [low half] and (row 2(i%4)+1, column i/4) of matrix j.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t smem_addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_addr) : "memory");
+}
+
+// Four fp32 added to 16-byte aligned global memory, no value returned.
+__device__ __forceinline__ void red_add_f32x4(float *dst, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
 
 // ---- descriptors -------------------------------------------------------------------------------------
 // Shared-memory operand descriptor, 128-byte swizzle.  For an MN-major operand (the contraction index is the

@@ -86,6 +86,8 @@ def workload(name: str) -> Workload:
         return Workload("mini_scaled", 11, 3, 2, 5, 2, 128, (301, 77, 419), 2, (1e-2,), "scaled", 0.1)
     if name == "mid_scaled":      # enough tokens per map (8709) for the plain bf16 weight fold to meet 1e-3
         return Workload("mid_scaled", 12, 2, 2, 3, 2, 128, (1024,) * 8 + (517,), 5, (1e-2,), "scaled", 0.1)
+    if name == "long_unit":       # one chunk whose tokens exceed what a unit sums in tensor memory between drains
+        return Workload("long_unit", 16, 2, 2, 3, 2, 128, (16384, 4099), 2, (1e-2,), "scaled", 0.1)
     if name == "deep_small":      # enough source layers for the paper's k = 8 selected layers (regressor width 1025)
         return Workload("deep_small", 15, 10, 2, 3, 2, 128, (1100, 1000), 2, (1e-2,), "scaled", 0.1)
     if name == "mini_ragged":     # several chunks of unequal size

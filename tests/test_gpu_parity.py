@@ -69,6 +69,9 @@ CASES = [
     ("mini_ragged", 0, 0),
     ("mid_scaled", 0, 0),
     ("mid_scaled", 0, 5),
+    ("long_unit", 0, 1),                       # 20,483 tokens in one unit: the accumulator is drained mid-unit
+    ("long_unit", cb.CB_FLAG_COMPENSATED, 1),
+    ("long_unit", 0, 3),
 ]
 
 

@@ -78,7 +78,7 @@ def _solve(A, B, mu, n, lams, flags=0):
 
 
 CASES = [("tiny", cb.CB_FLAG_COMPENSATED, 0), ("tiny", 0, 3), ("mini_scaled", 0, 0), ("mini_ragged", cb.CB_FLAG_COMPENSATED, 7),
-         ("mini_ragged", 0, 0), ("mid_scaled", 0, 0)]
+         ("mini_ragged", 0, 0), ("mid_scaled", 0, 0), ("long_unit", 0, 1), ("long_unit", cb.CB_FLAG_COMPENSATED, 1)]
 
 
 @pytest.mark.parametrize("name,flags,n_splits", CASES)
