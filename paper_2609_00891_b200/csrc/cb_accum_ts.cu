@@ -24,17 +24,20 @@
 // Every wait is bounded: if one runs out the block sets the context's status word and tears down.
 #include <cudaTypedefs.h>
 
+#ifndef CB_TS_TT
+#define CB_TS_TT 128
+#endif
 #ifndef CB_TS_NS
-#define CB_TS_NS 5
+#define CB_TS_NS (CB_TS_TT == 128 ? 3 : 5)
 #endif
 #ifndef CB_TS_NA
-#define CB_TS_NA 4
+#define CB_TS_NA (CB_TS_TT == 128 ? 3 : 4)
 #endif
 #ifndef CB_TS_GSPLIT
 #define CB_TS_GSPLIT 1
 #endif
 #ifndef CB_TS_YW
-#define CB_TS_YW 4
+#define CB_TS_YW 8
 #endif
 
 #include "cb_internal.cuh"
@@ -52,13 +55,14 @@ namespace {
 template <bool COMP>
 struct TsCfg {
     static constexpr int D = 128;
-    static constexpr int TT = 64;                     // tokens per tile
+    static constexpr int TT = CB_TS_TT;               // tokens per tile
     static constexpr int BLK = TT * 128;              // one 64-channel block of a tile: TT rows of 128 bytes
     static constexpr int STAGE_BYTES = 4 * BLK;       // [X blocks 0, 1 | Y blocks 0, 1]
     static constexpr int NS = CB_TS_NS;
     static constexpr int A_PARTS = COMP ? 2 : 1;
-    static constexpr int A_COLS = 32 * A_PARTS;       // columns of one weighted operand (64 tokens x bf16 = 32 columns)
-    static constexpr int NA = COMP ? (CB_TS_NA > 2 ? CB_TS_NA / 2 : 1) : CB_TS_NA;
+    static constexpr int A_PART_COLS = TT / 2;        // columns of one image of the weighted operand (two tokens per column)
+    static constexpr int A_COLS = A_PART_COLS * A_PARTS;
+    static constexpr int NA = (CB_TS_NA * A_COLS > 256) ? 256 / A_COLS : CB_TS_NA;
     static constexpr int N = 2 * D;                   // accumulator columns
     static constexpr int A_COL0 = N;
     static constexpr int TMEM_COLS = 512;
@@ -276,7 +280,7 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                         for (int k = 0; k < C::TT / 16; ++k) {
                             const uint64_t bd = ((uint64_t)desc_hi << 32) | (bl + k * 128);
                             umma_bf16_ts(tmem_base, at + k * 8, bd, idesc, k == 0 ? accum : 1u);
-                            if (COMP) umma_bf16_ts(tmem_base, at + 32 + k * 8, bd, idesc, 1u);
+                            if (COMP) umma_bf16_ts(tmem_base, at + C::A_PART_COLS + k * 8, bd, idesc, 1u);
                         }
                         accum = 1;
                         umma_commit(&empty[st.idx]);     // frees the stage and (through it) the weighted-operand buffer
@@ -297,12 +301,12 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
         const int g0 = (C::GSPLIT == 2) ? (fw >> 3) : 0;
         // ldmatrix row address of this lane: matrix j = lane / 8 is (8-channel chunk j & 1, token group j / 2), row
         // lane % 8 is a token; the 128-byte swizzle XORs the chunk index with the token's low three bits.
-        const int lm_row = hf * 32 + 8 * (lane >> 4) + (lane & 7);
+        const int lm_row = hf * (C::TT / 2) + 8 * (lane >> 4) + (lane & 7);
         uint32_t lm_off[GN];
 #pragma unroll
         for (int g = 0; g < GN; ++g)
             lm_off[g] = (q >> 1) * C::BLK + lm_row * 128 + (((4 * (q & 1) + 2 * (g0 + g) + ((lane >> 3) & 1)) ^ (lane & 7)) << 4);
-        const uint32_t a_lane = tmem_base + ((uint32_t)(q * 32) << 16) + C::A_COL0 + hf * 16;
+        const uint32_t a_lane = tmem_base + ((uint32_t)(q * 32) << 16) + C::A_COL0 + hf * (C::TT / 4);
         Ring<C::NS> st, old;       // `old` trails `st` by NA tiles
         Ring<C::NA> ar;
         uint32_t it = 0, uc = 0;
@@ -333,17 +337,18 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                 }
                 const uint32_t stage_u32 = smem_u32(xy + st.idx * C::STAGE_BYTES);
                 const float *wt = wst + st.idx * C::TT;
-                // token pairs of this lane: tokens hf*32 + 8 j + 2 (lane % 4) + {0, 1}, j = 0..3
+                // 32 tokens of this warp's half at a time; token pairs of this lane: + 8 j + 2 (lane % 4) + {0, 1}
+#pragma unroll
+                for (int sub = 0; sub < C::TT / 64; ++sub) {
                 uint64_t w2[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) w2[j] = *reinterpret_cast<const uint64_t *>(wt + hf * 32 + 8 * j + 2 * (lane & 3));
+                for (int j = 0; j < 4; ++j)
+                    w2[j] = *reinterpret_cast<const uint64_t *>(wt + hf * (C::TT / 2) + sub * 32 + 8 * j + 2 * (lane & 3));
                 uint32_t r[GN][2][4];
 #pragma unroll
                 for (int g = 0; g < GN; ++g)
 #pragma unroll
-                    for (int tp = 0; tp < 2; ++tp) {
-                        ldmatrix_x4_trans(stage_u32 + lm_off[g] + tp * (16 * 128), r[g][tp]);
-                    }
+                    for (int tp = 0; tp < 2; ++tp) ldmatrix_x4_trans(stage_u32 + lm_off[g] + (sub * 32 + tp * 16) * 128, r[g][tp]);
 #pragma unroll
                 for (int g = 0; g < GN; ++g) {
                     uint32_t oh[8], ol[8];
@@ -367,9 +372,10 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                             }
                         }
                     }
-                    const uint32_t ta = a_lane + ((uint32_t)(16 * (g0 + g)) << 16) + ar.idx * C::A_COLS;
+                    const uint32_t ta = a_lane + ((uint32_t)(16 * (g0 + g)) << 16) + ar.idx * C::A_COLS + sub * 16;
                     tmem_st_16x128_x4(ta, oh);
-                    if (COMP) tmem_st_16x128_x4(ta + 32, ol);
+                    if (COMP) tmem_st_16x128_x4(ta + C::A_PART_COLS, ol);
+                }
                 }
                 tmem_wait_st();
                 tc_fence_before();
@@ -403,7 +409,7 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
         const int yt = tid - C::YSUM_WARP0 * 32, yw = warp - C::YSUM_WARP0;
         const int cc = yt & 15, rg = yt >> 4;
         constexpr int YRG = C::YSUM_THREADS / 16, YR = C::TT / YRG;   // row groups, rows per thread
-        static_assert(YRG % 8 == 0, "row groups must preserve the swizzle phase");
+        static_assert(YRG % 8 == 0 && YR % 4 == 0, "row groups must preserve the swizzle phase; rows go in batches of four");
         const int y_off = 2 * C::BLK + (cc >> 3) * C::BLK + rg * 128 + (((cc & 7) ^ (rg & 7)) << 4);
         Ring<C::NS> st;
         uint32_t uc = 0;
@@ -419,24 +425,24 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
                 const uint8_t *stage = xy + st.idx * C::STAGE_BYTES;
                 const float *wt = wst + st.idx * C::TT;
-                float wr[YR];
 #pragma unroll
-                for (int i = 0; i < YR; ++i) wr[i] = wt[rg + YRG * i];
-                if (!CEN) {
-                    uint4 yv[YR];
+                for (int i0 = 0; i0 < YR; i0 += 4) {
+                    float wr[4];
 #pragma unroll
-                    for (int i = 0; i < YR; ++i) yv[i] = *reinterpret_cast<const uint4 *>(stage + y_off + i * (YRG * 128));
+                    for (int i = 0; i < 4; ++i) wr[i] = wt[rg + YRG * (i0 + i)];
+                    if (!CEN) {
+                        uint4 yv[4];
 #pragma unroll
-                    for (int i = 0; i < YR; ++i) {
-                        const uint64_t wr2 = f2_pack(wr[i], wr[i]);
-                        const unsigned yu[4] = {yv[i].x, yv[i].y, yv[i].z, yv[i].w};
+                        for (int i = 0; i < 4; ++i) yv[i] = *reinterpret_cast<const uint4 *>(stage + y_off + (i0 + i) * (YRG * 128));
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) sy2[e] = f2_fma(wr2, f2_from_bf16x2(yu[e]), sy2[e]);
+                        for (int i = 0; i < 4; ++i) {
+                            const uint64_t wr2 = f2_pack(wr[i], wr[i]);
+                            const unsigned yu[4] = {yv[i].x, yv[i].y, yv[i].z, yv[i].w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) sy2[e] = f2_fma(wr2, f2_from_bf16x2(yu[e]), sy2[e]);
+                        }
                     }
-                }
-                if (cc == 0) {
-#pragma unroll
-                    for (int i = 0; i < YR; ++i) sw += wr[i];
+                    if (cc == 0) sw += (wr[0] + wr[1]) + (wr[2] + wr[3]);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[st.idx]);
@@ -559,7 +565,7 @@ cudaError_t launch_accum_ts(const AccumArgs &a, bool comp, const cb_kv_view *src
 {
     TsParams P;
     P.a = a;
-    const int d = 128, TT = 64;
+    const int d = 128, TT = CB_TS_TT;
     if (!make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
                             src->stride_token, src->stride_layer, TT) ||
         !make_kv_tensor_map(&P.src_v, src->v, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
