@@ -152,7 +152,7 @@ def run_reference(args):
     print(json.dumps(out))
 
 
-TRAFFIC_DRAM_BYTES_PER_TOKEN = 440400        # dram__bytes_read + dram__bytes_write per token, k_accum_ts, 14B->32B shapes
+TRAFFIC_DRAM_BYTES_PER_TOKEN = 437400        # dram__bytes_read + dram__bytes_write per token, k_accum_ts, 14B->32B shapes
 TRAFFIC_DRAM_BYTES_PER_SPLIT = 270600000     # partial-slot read-modify-write per token split (1,024 maps)
 
 
