@@ -1,43 +1,39 @@
-// Head-local weighted statistics (d = 128) with the weighted operand in TENSOR MEMORY.
+// Head-local weighted statistics (d = 128) with the weighted operand in TENSOR MEMORY and the bias sum s_y on the
+// tensor cores.
 //
 // Same contraction as the shared-memory kernel (D[d][2d] = (w .* X)^T [X | Y] over tokens plus the bias sums), same
 // units, slots and summation order of the splits.  What differs is where the first MMA operand lives: the fold warps
 // write A = bf16(w x) straight into tensor memory (lane = channel, two tokens per 32-bit column) and the MMA reads it
-// from there.  Per 64-token tile that saves the 16 KB shared-memory write of the weighted tile and its 16 KB read by
-// the tensor cores (96 KB of shared-memory traffic instead of 128 KB) and the shared-memory space of the operand
-// buffers.  On full launches the board runs into its power limit (the SM clock measured inside the kernel falls to
-// about 1.43 GHz, while each part of the kernel alone runs at 1.8 - 1.96 GHz): what counts is the energy per tile.
+// from there.  Per 64 tokens that saves the 16 KB shared-memory write of the weighted tile and its 16 KB read by
+// the tensor cores and the shared-memory space of the operand buffers.  On full launches the board runs into its
+// power limit (the SM clock measured inside the kernel falls to about 1.43 GHz, while each part of the kernel alone
+// runs at 1.8 - 1.96 GHz): what counts is the energy per token, and most of what is left to save is instructions.
 //
-//   warp 0       X tile producer (TMA); last warp: Y tile + token weights producer
+//   warp 0       X tile producer (TMA); warp 14: Y tile + token weights producer
 //   warps 2..9   fold: a warp owns the channel quarter (warp % 4) that its tensor-memory lanes cover and one half of
 //                the tile's tokens.  ldmatrix (8x8, transposed) delivers for thread i the pair (token 2j, 2j+1) of
 //                channel i/4, which is exactly the register layout of the 16-lane x 128-bit tensor-memory store; the
-//                swizzled tile is read without bank conflicts.
-//   warp 1       MMA issuer: A from tensor memory, B = [X | Y] from shared memory (N = 256, MN-major)
+//                swizzled tile is read without a transposition in registers.  s_x = sum w x falls out of the fold
+//                (one packed add per two elements).  Each warp also writes the bf16 images w_hi, w_lo of 1/8 of the
+//                tile's weights into a small K-major operand "wb" (16 rows per 64 tokens: w_hi, w_lo, zeros).
+//   warp 1       MMA issuer, per 16 tokens:  D    += A [X | Y]   (A from tensor memory, N = 256)
+//                                            D_sy += Y^T wb      (Y tile as the MN-major first operand, N = 16: the
+//                                                                 w_hi and w_lo columns give s_y = sum_t w_t y_t
+//                                                                 to 2^-17; products of bf16 are exact in fp32)
+//                The small MMA replaces eight warps that summed w y on the ALUs (~600 warp instructions per 64
+//                tokens, 0.4 ms of a 4.4 ms launch) at a cost of 0.15 ms.  Measured alternatives: s_x from a second
+//                small MMA (A from tensor memory times a ones column) costs 0.08 ms alone but 0.25 ms beside the
+//                s_y one (the tensor pipe is then 80 % busy at the capped clock); the packed add in the fold costs
+//                0.07 ms.
 //   warps 10..13 drain: tensor memory -> registers -> vector reductions onto the unit's slot (one writer per slot
 //                and launch: the result does not depend on timing)
-//   warps 14..   bias sums s_y = sum w y, s_w = sum w on the ALUs, in warps of their own: the MMA of a tile waits for
-//                the weighted operand only.  Measured: 4 such warps 1 % faster than 8; 16 fold warps (16 channels
-//                each) 4 % slower than 8.
-// Tensor memory: columns 0..255 the accumulator, from 256 the ring of weighted operands (32 columns each; hi and lo
-// images when compensated).  One accumulator: the MMA waits while a unit's result is read out (about 1 % of a unit).
+// Tensor memory: columns 0..255 the accumulator, 256..447 a ring of three weighted operands, 448..463 D_sy.
+// One accumulator: the MMA waits while a unit's result is read out (about 1 % of a unit).
 // Every wait is bounded: if one runs out the block sets the context's status word and tears down.
 #include <cudaTypedefs.h>
 
 #ifndef CB_TS_TT
 #define CB_TS_TT 128
-#endif
-#ifndef CB_TS_NS
-#define CB_TS_NS (CB_TS_TT == 128 ? 3 : 5)
-#endif
-#ifndef CB_TS_NA
-#define CB_TS_NA (CB_TS_TT == 128 ? 3 : 4)
-#endif
-#ifndef CB_TS_GSPLIT
-#define CB_TS_GSPLIT 1
-#endif
-#ifndef CB_TS_YW
-#define CB_TS_YW 8
 #endif
 
 #include "cb_internal.cuh"
@@ -55,27 +51,26 @@ namespace {
 template <bool COMP>
 struct TsCfg {
     static constexpr int D = 128;
-    static constexpr int TT = CB_TS_TT;               // tokens per tile
+    static constexpr int TT = COMP ? 64 : CB_TS_TT;   // tokens per tile (compensated: two operand images per tile)
     static constexpr int BLK = TT * 128;              // one 64-channel block of a tile: TT rows of 128 bytes
     static constexpr int STAGE_BYTES = 4 * BLK;       // [X blocks 0, 1 | Y blocks 0, 1]
-    static constexpr int NS = CB_TS_NS;
+    static constexpr int WB_BYTES = (TT / 64) * 2048; // per 64 tokens: 16 rows of 128 bytes (K-major, 128-byte swizzle)
+    static constexpr int NS = TT == 128 ? 3 : 5;
     static constexpr int A_PARTS = COMP ? 2 : 1;
     static constexpr int A_PART_COLS = TT / 2;        // columns of one image of the weighted operand (two tokens per column)
     static constexpr int A_COLS = A_PART_COLS * A_PARTS;
-    static constexpr int NA = (CB_TS_NA * A_COLS > 256) ? 256 / A_COLS : CB_TS_NA;
+    static constexpr int NA = 3;
     static constexpr int N = 2 * D;                   // accumulator columns
     static constexpr int A_COL0 = N;
+    static constexpr int BIAS_COL = A_COL0 + NA * A_COLS;   // 16 columns of D_sy
     static constexpr int TMEM_COLS = 512;
-    static constexpr int GSPLIT = CB_TS_GSPLIT;       // 2: a fold warp takes 16 of its quarter's 32 channels
-    static constexpr int FOLD_WARPS = 8 * GSPLIT, DRAIN_WARPS = 4, YSUM_WARPS = CB_TS_YW;
-    static constexpr int YSUM_WARP0 = 2 + FOLD_WARPS + DRAIN_WARPS;
-    static constexpr int YPROD_WARP = YSUM_WARP0 + YSUM_WARPS;
-    static constexpr int YSUM_THREADS = YSUM_WARPS * 32;
+    static constexpr int FOLD_WARPS = 8, DRAIN_WARPS = 4;
+    static constexpr int YPROD_WARP = 2 + FOLD_WARPS + DRAIN_WARPS;
     static constexpr int THREADS = (YPROD_WARP + 1) * 32;
-    static constexpr int RED_STRIDE = D + 4;          // per bias warp: s_y[D], s_w, pad
-    static constexpr int RED_FLOATS = YSUM_WARPS * RED_STRIDE + 2 * D;   // ... then s_x of the two token halves
-    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * STAGE_BYTES + RED_FLOATS * 4 + NS * TT * 4 + 256;
-    static_assert(N + NA * A_COLS <= TMEM_COLS, "tensor memory columns");
+    static constexpr int TW = TT / FOLD_WARPS;        // tokens whose weights a fold warp converts
+    static constexpr int RED_FLOATS = 2 * D + 16;     // s_x of the two token halves, partial s_w of the fold warps
+    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * (STAGE_BYTES + WB_BYTES) + RED_FLOATS * 4 + NS * TT * 4 + 256;
+    static_assert(BIAS_COL + 16 <= TMEM_COLS, "tensor memory columns");
     static_assert(NA <= NS, "an operand buffer is released through its tile's stage barrier");
 };
 
@@ -144,12 +139,6 @@ __device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
-__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
 __device__ __forceinline__ uint64_t f2_from_bf16x2(unsigned u) { return f2_pack(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)); }
 __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
 {
@@ -158,8 +147,9 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
     return r;
 }
 
-// CEN: two-pass centred construction: the weighted operand is w (x - mu_x) with the means of P.a.mu; the slot's s_x
-// entries become the column sums of the ROUNDED weighted operand (what the reduction needs for its exact correction).
+// CEN: two-pass centred construction: the weighted operand is w (x - mu_x) with the means of P.a.mu; s_y is not
+// formed (the slot's entries stay zero); the slot's s_x entries become the column sums of the ROUNDED weighted
+// operand (what the centred reduction needs for its exact correction).
 template <bool COMP, bool CEN>
 __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __grid_constant__ TsParams P)
 {
@@ -168,17 +158,18 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *xy = smem;                                       // [NS][STAGE_BYTES]
-    float *red = reinterpret_cast<float *>(xy + (size_t)C::NS * C::STAGE_BYTES);
-    float *redx = red + C::YSUM_WARPS * C::RED_STRIDE;        // [2 token halves][D]
-    float *wst = red + C::RED_FLOATS;                         // [NS][TT] token weights of the staged tile
+    uint8_t *wb = xy + (size_t)C::NS * C::STAGE_BYTES;        // [NS][WB_BYTES] rows 0, 1, 2 = w_hi, w_lo, ones
+    float *redx = reinterpret_cast<float *>(wb + (size_t)C::NS * C::WB_BYTES);   // [2 token halves][D] partial s_x
+    float *red = redx + 2 * D;                                // [FOLD_WARPS] partial s_w
+    float *wst = red + 16;                                    // [NS][TT] token weights of the staged tile
     uint64_t *bars = reinterpret_cast<uint64_t *>(wst + C::NS * C::TT);
     uint64_t *full = bars;                 // [NS] tile landed: X bytes (1 arrival), Y bytes (1), weights (32 lanes)
-    uint64_t *empty = full + C::NS;        // [NS] stage free: MMA done (1) + every fold and bias warp done
+    uint64_t *empty = full + C::NS;        // [NS] stage free: MMA done (1) + every fold warp done
     uint64_t *afull = empty + C::NS;       // [NA] weighted operand written to tensor memory (every fold warp)
-    uint64_t *accfull = afull + C::NA;     // [1]  accumulator complete (MMA)
-    uint64_t *accempty = accfull + 1;      // [1]  accumulator read out (4 drain warps)
-    uint64_t *redfull = accempty + 1;      // [1]  bias partials of all fold and bias warps written
-    uint64_t *reddone = redfull + 1;       // [1]  bias partials consumed
+    uint64_t *accfull = afull + C::NA;     // [1]  accumulators complete (MMA)
+    uint64_t *accempty = accfull + 1;      // [1]  accumulators read out (4 drain warps)
+    uint64_t *redfull = accempty + 1;      // [1]  partial s_x, s_w of all fold warps written
+    uint64_t *reddone = redfull + 1;       // [1]  partials consumed (fold warps 0..3)
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(reddone + 1);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
@@ -189,18 +180,22 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
     const int n_tiles = (a.n_tokens + C::TT - 1) / C::TT;
 
     if (tid == 0) {
-        for (int i = 0; i < C::NS; ++i) { mbar_init(&full[i], 2 + 32); mbar_init(&empty[i], 1 + C::FOLD_WARPS + C::YSUM_WARPS); }
+        for (int i = 0; i < C::NS; ++i) { mbar_init(&full[i], 2 + 32); mbar_init(&empty[i], 1 + C::FOLD_WARPS); }
         for (int i = 0; i < C::NA; ++i) mbar_init(&afull[i], C::FOLD_WARPS);
         mbar_init(accfull, 1);
         mbar_init(accempty, C::DRAIN_WARPS);
-        mbar_init(redfull, C::FOLD_WARPS + C::YSUM_WARPS);
-        mbar_init(reddone, C::YSUM_WARPS);
+        mbar_init(redfull, C::FOLD_WARPS);
+        mbar_init(reddone, 4);
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
         tma_prefetch_desc(&P.tgt_k); tma_prefetch_desc(&P.tgt_v);
     }
     if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
+    // wb: rows 2..15 of every 16-row block stay zero; rows 0 and 1 are rewritten for every tile
+    for (int i = tid; i < C::NS * C::WB_BYTES / 16; i += C::THREADS)
+        *reinterpret_cast<uint4 *>(wb + (size_t)i * 16) = make_uint4(0u, 0u, 0u, 0u);
+    fence_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -254,10 +249,14 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
     } else if (warp == 1) {
         // ================================ MMA issuer (one thread) ================================
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(128, C::N, false, true);
+            constexpr uint32_t idesc = umma_idesc_bf16(128, C::N, false, true);     // A: tensor memory, B: MN-major
+            constexpr uint32_t idesc_sy = umma_idesc_bf16(128, 16, true, false);    // A = Y tile: MN-major, B = wb
             const uint64_t proto = umma_smem_desc_sw128(0, C::BLK, 1024);
-            const uint32_t desc_hi = (uint32_t)(proto >> 32);
+            const uint64_t proto_w = umma_smem_desc_sw128(0, 16, 1024);
+            const uint32_t desc_hi = (uint32_t)(proto >> 32), w_hi32 = (uint32_t)(proto_w >> 32);
             const uint32_t b_lo0 = (uint32_t)proto | ((smem_u32(xy) & 0x3FFFFu) >> 4);
+            const uint32_t w_lo0 = (uint32_t)proto_w | ((smem_u32(wb) & 0x3FFFFu) >> 4);
+            const uint32_t d_sy = tmem_base + C::BIAS_COL;
             Ring<C::NS> st;
             Ring<C::NA> ar;
             uint32_t sr = 0;
@@ -275,12 +274,17 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                         if (!mbar_wait(&afull[ar.idx], ar.phase, abort_flag)) goto teardown;
                         tc_fence_after();
                         const uint32_t bl = b_lo0 + st.idx * (C::STAGE_BYTES >> 4);
+                        const uint32_t wl = w_lo0 + st.idx * (C::WB_BYTES >> 4);
                         const uint32_t at = tmem_base + C::A_COL0 + ar.idx * C::A_COLS;
 #pragma unroll
                         for (int k = 0; k < C::TT / 16; ++k) {
-                            const uint64_t bd = ((uint64_t)desc_hi << 32) | (bl + k * 128);
-                            umma_bf16_ts(tmem_base, at + k * 8, bd, idesc, k == 0 ? accum : 1u);
+                            const uint32_t acc_k = (k == 0) ? accum : 1u;
+                            const uint64_t bd = ((uint64_t)desc_hi << 32) | (bl + k * 128);   // 16 tokens = 2048 bytes
+                            // wb: 64 tokens per 2048-byte block, 16 tokens = 32 bytes along the row
+                            const uint64_t wd = ((uint64_t)w_hi32 << 32) | (wl + (k >> 2) * 128 + (k & 3) * 2);
+                            umma_bf16_ts(tmem_base, at + k * 8, bd, idesc, acc_k);
                             if (COMP) umma_bf16_ts(tmem_base, at + C::A_PART_COLS + k * 8, bd, idesc, 1u);
+                            if (!CEN) umma_bf16_ss(d_sy, ((uint64_t)desc_hi << 32) | (bl + ((2 * C::BLK) >> 4) + k * 128), wd, idesc_sy, acc_k);
                         }
                         accum = 1;
                         umma_commit(&empty[st.idx]);     // frees the stage and (through it) the weighted-operand buffer
@@ -296,34 +300,38 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
         // ================================ fold warps ================================
         const int fw = warp - 2;
         const int q = warp & 3;             // tensor-memory lane quarter = channels 32 q .. 32 q + 31
-        const int hf = (fw >> 2) & 1;       // token half of the tile
-        constexpr int GN = 2 / C::GSPLIT;   // 16-channel groups per warp
-        const int g0 = (C::GSPLIT == 2) ? (fw >> 3) : 0;
+        const int hf = fw >> 2;             // token half of the tile
         // ldmatrix row address of this lane: matrix j = lane / 8 is (8-channel chunk j & 1, token group j / 2), row
         // lane % 8 is a token; the 128-byte swizzle XORs the chunk index with the token's low three bits.
         const int lm_row = hf * (C::TT / 2) + 8 * (lane >> 4) + (lane & 7);
-        uint32_t lm_off[GN];
+        uint32_t lm_off[2];
 #pragma unroll
-        for (int g = 0; g < GN; ++g)
-            lm_off[g] = (q >> 1) * C::BLK + lm_row * 128 + (((4 * (q & 1) + 2 * (g0 + g) + ((lane >> 3) & 1)) ^ (lane & 7)) << 4);
+        for (int g = 0; g < 2; ++g)
+            lm_off[g] = (q >> 1) * C::BLK + lm_row * 128 + (((4 * (q & 1) + 2 * g + ((lane >> 3) & 1)) ^ (lane & 7)) << 4);
         const uint32_t a_lane = tmem_base + ((uint32_t)(q * 32) << 16) + C::A_COL0 + hf * (C::TT / 4);
+        // this lane's weight token (lanes below TW) and where its bf16 images go in wb (rows 0 and 1 of the block)
+        const int wtok = fw * C::TW + (lane < C::TW ? lane : 0);
+        // (64-token block, row n, 16-byte chunk (token / 8) XOR n, token % 8): rows 0 and 1
+        const int wb_off0 = (wtok >> 6) * 2048 + (((wtok & 63) >> 3) << 4) + (wtok & 7) * 2;
+        const int wb_off1 = (wtok >> 6) * 2048 + 128 + ((((wtok & 63) >> 3) ^ 1) << 4) + (wtok & 7) * 2;
         Ring<C::NS> st, old;       // `old` trails `st` by NA tiles
         Ring<C::NA> ar;
         uint32_t it = 0, uc = 0;
         UnitIter cur;
         cur.start(a, n_units, n_maps, n_tiles);
         while (cur.valid(n_units)) {
-            const int m = cur.m, n_t = cur.tile1 - cur.tile;
-            uint64_t sx2[GN][2];           // [16-channel group][chunk]: sums over this thread's token pairs
-            uint64_t nmu2[GN][2];
+            const int m = cur.m, split = cur.split, n_t = cur.tile1 - cur.tile;
+            uint64_t sx2[2][2];            // [16-channel group][chunk]: sums over this thread's token pairs
+            uint64_t nmu2[2][2];
+            float sw = 0.f;
 #pragma unroll
-            for (int g = 0; g < GN; ++g)
+            for (int g = 0; g < 2; ++g)
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     sx2[g][c] = 0ull;
                     nmu2[g][c] = 0ull;
                     if (CEN) {
-                        const float mu = __ldg(a.mu + (size_t)m * (2 * D + 1) + q * 32 + 16 * (g0 + g) + 8 * c + (lane >> 2));
+                        const float mu = __ldg(a.mu + (size_t)m * (2 * D + 1) + q * 32 + 16 * g + 8 * c + (lane >> 2));
                         nmu2[g][c] = f2_pack(-mu, -mu);
                     }
                 }
@@ -337,47 +345,56 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                 }
                 const uint32_t stage_u32 = smem_u32(xy + st.idx * C::STAGE_BYTES);
                 const float *wt = wst + st.idx * C::TT;
+                if (lane < C::TW) {
+                    const float wv = wt[wtok];
+                    const __nv_bfloat16 h = __float2bfloat16_rn(wv);
+                    const __nv_bfloat16 l = __float2bfloat16_rn(wv - __bfloat162float(h));
+                    uint8_t *dst = wb + st.idx * C::WB_BYTES;
+                    *reinterpret_cast<__nv_bfloat16 *>(dst + wb_off0) = h;
+                    *reinterpret_cast<__nv_bfloat16 *>(dst + wb_off1) = l;
+                    sw += wv;
+                }
                 // 32 tokens of this warp's half at a time; token pairs of this lane: + 8 j + 2 (lane % 4) + {0, 1}
 #pragma unroll
                 for (int sub = 0; sub < C::TT / 64; ++sub) {
-                uint64_t w2[4];
+                    uint64_t w2[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    w2[j] = *reinterpret_cast<const uint64_t *>(wt + hf * (C::TT / 2) + sub * 32 + 8 * j + 2 * (lane & 3));
-                uint32_t r[GN][2][4];
+                    for (int j = 0; j < 4; ++j)
+                        w2[j] = *reinterpret_cast<const uint64_t *>(wt + hf * (C::TT / 2) + sub * 32 + 8 * j + 2 * (lane & 3));
+                    uint32_t r[2][2][4];
 #pragma unroll
-                for (int g = 0; g < GN; ++g)
+                    for (int g = 0; g < 2; ++g)
 #pragma unroll
-                    for (int tp = 0; tp < 2; ++tp) ldmatrix_x4_trans(stage_u32 + lm_off[g] + (sub * 32 + tp * 16) * 128, r[g][tp]);
+                        for (int tp = 0; tp < 2; ++tp) ldmatrix_x4_trans(stage_u32 + lm_off[g] + (sub * 32 + tp * 16) * 128, r[g][tp]);
 #pragma unroll
-                for (int g = 0; g < GN; ++g) {
-                    uint32_t oh[8], ol[8];
+                    for (int g = 0; g < 2; ++g) {
+                        uint32_t oh[8], ol[8];
 #pragma unroll
-                    for (int tp = 0; tp < 2; ++tp) {
+                        for (int tp = 0; tp < 2; ++tp) {
 #pragma unroll
-                        for (int mi = 0; mi < 4; ++mi) {
-                            const int c = mi & 1;
-                            uint64_t xf = f2_from_bf16x2(r[g][tp][mi]);
-                            if (CEN) xf = f2_add(xf, nmu2[g][c]);                       // x - mu_x
-                            const uint64_t pr = f2_mul(w2[2 * tp + (mi >> 1)], xf);      // w x for two tokens
-                            if (!CEN) sx2[g][c] = f2_add(sx2[g][c], pr);
-                            float p0, p1;
-                            f2_unpack(pr, p0, p1);
-                            const unsigned hw = pack_bf16x2(p0, p1);
-                            oh[4 * tp + mi] = hw;
-                            if (COMP) ol[4 * tp + mi] = pack_bf16x2(p0 - __uint_as_float(hw << 16), p1 - __uint_as_float(hw & 0xffff0000u));
-                            if (CEN) {                                                  // sum of what the tensor cores will see
-                                sx2[g][c] = f2_add(sx2[g][c], f2_from_bf16x2(hw));
-                                if (COMP) sx2[g][c] = f2_add(sx2[g][c], f2_from_bf16x2(ol[4 * tp + mi]));
+                            for (int mi = 0; mi < 4; ++mi) {
+                                uint64_t xf = f2_from_bf16x2(r[g][tp][mi]);
+                                if (CEN) xf = f2_add(xf, nmu2[g][mi & 1]);                  // x - mu_x
+                                const uint64_t pr = f2_mul(w2[2 * tp + (mi >> 1)], xf);      // w x for two tokens
+                                if (!CEN) sx2[g][mi & 1] = f2_add(sx2[g][mi & 1], pr);
+                                float p0, p1;
+                                f2_unpack(pr, p0, p1);
+                                const unsigned hw = pack_bf16x2(p0, p1);
+                                oh[4 * tp + mi] = hw;
+                                if (COMP) ol[4 * tp + mi] = pack_bf16x2(p0 - __uint_as_float(hw << 16), p1 - __uint_as_float(hw & 0xffff0000u));
+                                if (CEN) {                                                  // sum of what the tensor cores will see
+                                    sx2[g][mi & 1] = f2_add(sx2[g][mi & 1], f2_from_bf16x2(hw));
+                                    if (COMP) sx2[g][mi & 1] = f2_add(sx2[g][mi & 1], f2_from_bf16x2(ol[4 * tp + mi]));
+                                }
                             }
                         }
+                        const uint32_t ta = a_lane + ((uint32_t)(16 * g) << 16) + ar.idx * C::A_COLS + sub * 16;
+                        tmem_st_16x128_x4(ta, oh);
+                        if (COMP) tmem_st_16x128_x4(ta + C::A_PART_COLS, ol);
                     }
-                    const uint32_t ta = a_lane + ((uint32_t)(16 * (g0 + g)) << 16) + ar.idx * C::A_COLS + sub * 16;
-                    tmem_st_16x128_x4(ta, oh);
-                    if (COMP) tmem_st_16x128_x4(ta + C::A_PART_COLS, ol);
-                }
                 }
                 tmem_wait_st();
+                fence_async_smem();          // the wb rows written above are read by the tensor cores
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&afull[ar.idx]); mbar_arrive(&empty[st.idx]); }
@@ -385,10 +402,12 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                 ar.next();
                 ++it;
             }
-            // ---- s_x of this unit: the four lanes that hold a channel add up; the bias warps write the slot ----
-            if (!mbar_wait_warp(reddone, (uc & 1) ^ 1, abort_flag, lane, true)) goto teardown;
+            // ---- s_x and s_w of this unit: partial sums through shared memory, added in a fixed order ----
 #pragma unroll
-            for (int g = 0; g < GN; ++g)
+            for (int o = 16; o >= 1; o >>= 1) sw += __shfl_xor_sync(0xffffffffu, sw, o);
+            if (!mbar_wait_warp(reddone, (uc & 1) ^ 1, abort_flag, lane)) goto teardown;
+#pragma unroll
+            for (int g = 0; g < 2; ++g)
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     float lo, hi;
@@ -396,109 +415,48 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                     float v = lo + hi;
                     v += __shfl_xor_sync(0xffffffffu, v, 1);
                     v += __shfl_xor_sync(0xffffffffu, v, 2);
-                    if ((lane & 3) == 0) redx[hf * D + q * 32 + 16 * (g0 + g) + 8 * c + (lane >> 2)] = v;
+                    if ((lane & 3) == 0) redx[hf * D + q * 32 + 16 * g + 8 * c + (lane >> 2)] = v;
                 }
+            if (lane == 0) red[fw] = sw;
             __syncwarp();
             if (lane == 0) mbar_arrive(redfull);
-            ++uc;
-            cur.next_unit(a, n_units, n_maps, n_tiles);
-        }
-    } else if (warp >= C::YSUM_WARP0 && warp < C::YPROD_WARP) {
-        // ================================ bias warps: s_y = sum w y, s_w = sum w ================================
-        // thread = (16-byte chunk cc of the target row, row group rg), rows rg + 16 i.  Off the MMA's critical path.
-        const int yt = tid - C::YSUM_WARP0 * 32, yw = warp - C::YSUM_WARP0;
-        const int cc = yt & 15, rg = yt >> 4;
-        constexpr int YRG = C::YSUM_THREADS / 16, YR = C::TT / YRG;   // row groups, rows per thread
-        static_assert(YRG % 8 == 0 && YR % 4 == 0, "row groups must preserve the swizzle phase; rows go in batches of four");
-        const int y_off = 2 * C::BLK + (cc >> 3) * C::BLK + rg * 128 + (((cc & 7) ^ (rg & 7)) << 4);
-        Ring<C::NS> st;
-        uint32_t uc = 0;
-        UnitIter cur;
-        cur.start(a, n_units, n_maps, n_tiles);
-        while (cur.valid(n_units)) {
-            const int m = cur.m, split = cur.split, n_t = cur.tile1 - cur.tile;
-            uint64_t sy2[4];
-            float sw = 0.f;
+            if (fw < 4) {
+                if (!mbar_wait_warp(redfull, uc & 1, abort_flag, lane)) goto teardown;
+                float *slot = a.slots + ((size_t)split * n_maps + m) * slot_floats(D);
+                const int v = fw * 32 + lane;
+                slot[slot_sx(D) + v] += redx[v] + redx[D + v];
+                if (v == 0) {
+                    float sum = 0.f;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) sy2[e] = 0ull;
-            for (int t = 0; t < n_t; ++t) {
-                if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
-                const uint8_t *stage = xy + st.idx * C::STAGE_BYTES;
-                const float *wt = wst + st.idx * C::TT;
-#pragma unroll
-                for (int i0 = 0; i0 < YR; i0 += 4) {
-                    float wr[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) wr[i] = wt[rg + YRG * (i0 + i)];
-                    if (!CEN) {
-                        uint4 yv[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) yv[i] = *reinterpret_cast<const uint4 *>(stage + y_off + (i0 + i) * (YRG * 128));
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint64_t wr2 = f2_pack(wr[i], wr[i]);
-                            const unsigned yu[4] = {yv[i].x, yv[i].y, yv[i].z, yv[i].w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) sy2[e] = f2_fma(wr2, f2_from_bf16x2(yu[e]), sy2[e]);
-                        }
-                    }
-                    if (cc == 0) sw += (wr[0] + wr[1]) + (wr[2] + wr[3]);
+                    for (int k = 0; k < C::FOLD_WARPS; ++k) sum += red[k];
+                    slot[slot_sw(D)] += sum;
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[st.idx]);
-                st.next();
+                if (lane == 0) mbar_arrive(reddone);
             }
-            if (!mbar_wait_warp(reddone, (uc & 1) ^ 1, abort_flag, lane)) goto teardown;
-            {
-                float sy[8];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) f2_unpack(sy2[e], sy[2 * e], sy[2 * e + 1]);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) sy[e] += __shfl_xor_sync(0xffffffffu, sy[e], 16);
-                sw += __shfl_xor_sync(0xffffffffu, sw, 16);
-                float *rw = red + yw * C::RED_STRIDE;
-                if (lane < 16) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) rw[cc * 8 + e] = sy[e];
-                    if (cc == 0) rw[D] = sw;
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(redfull);
-            if (!mbar_wait_warp(redfull, uc & 1, abort_flag, lane)) goto teardown;
-            {
-                float *slot = a.slots + ((size_t)split * n_maps + m) * slot_floats(D);
-                for (int v = yt; v < 2 * D + 1; v += C::YSUM_THREADS) {
-                    float sum = 0.f;
-                    if (v < D) sum = redx[v] + redx[D + v];
-                    else {
-#pragma unroll
-                        for (int k = 0; k < C::YSUM_WARPS; ++k) sum += red[k * C::RED_STRIDE + (v - D)];
-                    }
-                    slot[slot_sx(D) + v] += sum;    // s_x, s_y, s_w are adjacent in the slot
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(reddone);
             ++uc;
             cur.next_unit(a, n_units, n_maps, n_tiles);
         }
     } else {
         // ================================ drain warps ================================
         const int q = warp & 3;             // tensor-memory lane quarter this warp may access
-        const int row = q * 32 + lane;      // row of D = channel of the weighted operand
+        const int row = q * 32 + lane;      // row of D = channel of the weighted operand (D_sy: target channel)
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
         uint32_t sr = 0;
         UnitIter cur;
         cur.start(a, n_units, n_maps, n_tiles);
         while (cur.valid(n_units)) {
-            float *grow = a.slots + ((size_t)cur.split * n_maps + cur.m) * slot_floats(D) + (size_t)row * C::N;
+            float *slot = a.slots + ((size_t)cur.split * n_maps + cur.m) * slot_floats(D);
+            float *grow = slot + (size_t)row * C::N;
             for (int sr0 = cur.tile; sr0 < cur.tile1; sr0 += P.drain_tiles, ++sr) {
                 if (!mbar_wait_warp(accfull, sr & 1, abort_flag, lane)) goto teardown;
                 tc_fence_after();
+                uint32_t b[16];
+                tmem_ld_32x16(lane_base + C::BIAS_COL, b);
 #pragma unroll 1
                 for (int c = 0; c < C::N / 32; ++c) {
                     uint32_t r[32];
-                    tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + c * 32, r);
+                    tmem_ld_32x32(lane_base + c * 32, r);
                     tmem_wait_ld();
                     if (c == C::N / 32 - 1) {       // everything is in registers: the next accumulation may start
                         tc_fence_before();
@@ -510,6 +468,8 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                         red_add_f32x4(grow + c * 32 + v * 4, __uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
                                       __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
                 }
+                // D_sy columns 0 and 1: the w_hi and w_lo columns of wb
+                if (!CEN) atomicAdd(slot + slot_sy(D) + row, __uint_as_float(b[0]) + __uint_as_float(b[1]));
             }
             cur.next_unit(a, n_units, n_maps, n_tiles);
         }
@@ -565,7 +525,7 @@ cudaError_t launch_accum_ts(const AccumArgs &a, bool comp, const cb_kv_view *src
 {
     TsParams P;
     P.a = a;
-    const int d = 128, TT = CB_TS_TT;
+    const int d = 128, TT = comp ? TsCfg<true>::TT : TsCfg<false>::TT;
     if (!make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
                             src->stride_token, src->stride_layer, TT) ||
         !make_kv_tensor_map(&P.src_v, src->v, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
