@@ -1,4 +1,6 @@
-// Fused weighted-statistics accumulation on the 5th-generation tensor cores (sm_100a).
+// Fused weighted-statistics accumulation on the 5th-generation tensor cores (sm_100a), both MMA operands in shared
+// memory.  This kernel serves d = 64, the rotary fold and the one-row-head full-head variant; head-local calls with
+// d = 128 go to the kernel that keeps the weighted operand in tensor memory (cb_accum_ts.cu).
 //
 // For one map (matched source head X, target head Y, token weights w) the statistics are the dense contraction
 //     D[d][2d] = (w .* X)^T [X | Y]          over tokens,
@@ -867,6 +869,11 @@ static bool fill_maps(TcParams &P, int d, const cb_kv_view *src, const cb_kv_vie
 
 cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st)
 {
+    // Calls of fewer than 4,096 rows take the hi + lo weighted operand regardless of the flag: the single bf16
+    // rounding averages out only like 1/sqrt(rows), such calls are bound by launch latency, not by the second MMA.
+    const bool comp = a.compensated || a.n_tokens < 4096;
+    // d = 128 without the rotary fold: the kernel that keeps the weighted operand in tensor memory
+    if (d == 128 && !a.rope_pos) return launch_accum_ts(a, comp, src, tgt, st);
     TcParams P;
     P.a = a;
     P.fh = FhDev{};
@@ -880,24 +887,14 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     const int TT = 64;
     if (!fill_maps(P, d, src, tgt, TT)) return cudaErrorInvalidValue;
     cudaError_t e;
-    // Calls of fewer than 4,096 rows take the hi + lo weighted operand regardless of the flag: the single bf16
-    // rounding averages out only like 1/sqrt(rows), such calls are bound by launch latency, not by the second MMA.
-    const bool comp = a.compensated || a.n_tokens < 4096;
     // Tokens summed in tensor memory before a drain (the fp32 accumulation of the tensor cores loses about 1e-4 over
     // 16,384 tokens; the compensated fold drains eight times as often).
     P.drain_tiles = (comp ? 2048 : 16384) / TT;
-#ifndef CB_NO_TS
-    // d = 128 without the rotary fold: the kernel that keeps the weighted operand in tensor memory
-    if (d == 128 && !a.rope_pos) return launch_accum_ts(a, comp, src, tgt, st);
-#endif
     if (a.rope_pos) {
         if (comp) e = (d == 128) ? launch_tc<128, true, false, false, true>(P, st) : launch_tc<64, true, false, false, true>(P, st);
         else e = (d == 128) ? launch_tc<128, false, false, false, true>(P, st) : launch_tc<64, false, false, false, true>(P, st);
-    } else if (a.mu) {
-        if (comp) e = (d == 128) ? launch_tc<128, true, false, true>(P, st) : launch_tc<64, true, false, true>(P, st);
-        else e = (d == 128) ? launch_tc<128, false, false, true>(P, st) : launch_tc<64, false, false, true>(P, st);
-    } else if (comp) e = (d == 128) ? launch_tc<128, true>(P, st) : launch_tc<64, true>(P, st);
-    else e = (d == 128) ? launch_tc<128, false>(P, st) : launch_tc<64, false>(P, st);
+    } else if (a.mu) e = comp ? launch_tc<64, true, false, true>(P, st) : launch_tc<64, false, false, true>(P, st);
+    else e = comp ? launch_tc<64, true>(P, st) : launch_tc<64, false>(P, st);
     if (e == cudaSuccess) count_launch();
     return e;
 }
