@@ -88,6 +88,8 @@ def workload(name: str) -> Workload:
         return Workload("mid_scaled", 12, 2, 2, 3, 2, 128, (1024,) * 8 + (517,), 5, (1e-2,), "scaled", 0.1)
     if name == "long_unit":       # one chunk whose tokens exceed what a unit sums in tensor memory between drains
         return Workload("long_unit", 16, 2, 2, 3, 2, 128, (16384, 4099), 2, (1e-2,), "scaled", 0.1)
+    if name == "very_long_unit":  # one map pair, 200,003 tokens in one call: many drains inside a unit, long rings
+        return Workload("very_long_unit", 17, 1, 1, 1, 1, 128, (200003,), 1, (1e-2,), "scaled", 0.1)
     if name == "deep_small":      # enough source layers for the paper's k = 8 selected layers (regressor width 1025)
         return Workload("deep_small", 15, 10, 2, 3, 2, 128, (1100, 1000), 2, (1e-2,), "scaled", 0.1)
     if name == "mini_ragged":     # several chunks of unequal size

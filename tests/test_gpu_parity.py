@@ -72,6 +72,8 @@ CASES = [
     ("long_unit", 0, 1),                       # 20,483 tokens in one unit: the accumulator is drained mid-unit
     ("long_unit", cb.CB_FLAG_COMPENSATED, 1),
     ("long_unit", 0, 3),
+    ("very_long_unit", 0, 1),                  # 200,003 tokens in one unit: thirteen drains, 1,563 tiles
+    ("very_long_unit", 0, 0),
 ]
 
 
