@@ -354,7 +354,7 @@ def main():
         # DRAM traffic of one launch from the ncu capture of an 8,192-token launch of the same shapes (summary:
         # profiles/k_accum_ts_qwen14b_32b_8192tok.md), scaled: the per-token part x tokens + the read-modify-write of
         # the partial slots per split, which does not grow with tokens
-        n_splits = args.splits if args.splits > 0 else 4
+        n_splits = cb.cb_token_splits(prob)
         roof["traffic"] = TRAFFIC_DRAM_BYTES_PER_TOKEN * tok_launch + TRAFFIC_DRAM_BYTES_PER_SPLIT * n_splits
     t_roof = max(alg_bytes * tokens_per_step / (peaks["hbm_gbs"] * 1e9),
                  alg_flops * tokens_per_step / (peaks["bf16_tflops"] * 1e12))

@@ -76,7 +76,8 @@ typedef struct cb_kv_view {
  * source head src_head[h].  src_layer (length Lt) and src_head (length Ht) are HOST arrays, copied by
  * cb_create / read by cb_apply during the call.
  * n_splits: number of token splits (independent partial statistics per map, summed in fixed order by
- * cb_stats_reduce); 0 selects a default.  Must be <= 64.
+ * cb_stats_reduce); 0 lets the library choose (cb_token_splits reports the choice, which depends on the
+ * problem's shapes only).  Must be <= 64.
  */
 typedef struct cb_problem {
     int32_t Ls, Hs, ds;
@@ -111,6 +112,14 @@ cb_status cb_work_list(const cb_problem *prob, int32_t *n_items, int32_t *item_c
 
 /* Bytes of device workspace cb_create needs for this problem (partial statistics slots + small tables). */
 cb_status cb_workspace_bytes(const cb_problem *prob, size_t *bytes);
+
+/*
+ * The number of token splits the statistics calls will use for this problem (Section 3.4: partial statistics
+ * per bounded block of observations, then a fixed reduction): prob->n_splits if it is positive, else the count in
+ * 1..8 that balances the persistent blocks' units (map, split) over the SMs against the cost of one more set
+ * of partial slots per split.  Host only; *n_splits receives the count.
+ */
+cb_status cb_token_splits(const cb_problem *prob, int32_t *n_splits);
 
 /*
  * Create a context on the current device.  workspace: device memory, 256-byte aligned, at least

@@ -22,7 +22,7 @@ CB_ERR_CUDA, CB_ERR_NOT_PD, CB_ERR_TIMEOUT, CB_ERR_STATIC_LIMIT = 5, 6, 7, 8
 CB_FLAG_COMPENSATED, CB_FLAG_RAW_LAMBDA, CB_FLAG_SIMT, CB_FLAG_ONE_ROW_HEAD = 1, 2, 4, 8
 CB_DTYPE_BF16, CB_DTYPE_F32 = 0, 1
 
-EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_workspace_bytes", "cb_create",
+EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_workspace_bytes", "cb_token_splits", "cb_create",
            "cb_destroy", "cb_stats_reset", "cb_stats_accumulate", "cb_staging_bytes", "cb_stats_accumulate_host",
            "cb_stats_reduce", "cb_ridge_solve",
            "cb_check_info", "cb_apply", "cb_device_status", "cb_stats_build_static", "cb_fullhead_layer_sets",
@@ -142,6 +142,12 @@ def cb_work_list(prob: Problem):
     _check(lib().cb_work_list(ctypes.byref(prob.c), ctypes.byref(n), p(ic), p(il), p(ih), p(ib), p(im)), "cb_work_list")
     k = n.value
     return ic[:k].copy(), il[:k].copy(), ih[:k].copy(), ib[:k + 1].copy(), im.copy()
+
+
+def cb_token_splits(prob: Problem) -> int:
+    n = ctypes.c_int32(0)
+    _check(lib().cb_token_splits(ctypes.byref(prob.c), ctypes.byref(n)), "cb_token_splits")
+    return int(n.value)
 
 
 def cb_workspace_bytes(prob: Problem) -> int:

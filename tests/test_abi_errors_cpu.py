@@ -124,3 +124,11 @@ def test_selector_host_logic_and_argument_errors():
     assert L.cb_probe_r2(p, p, p, p, 0, 128, ctypes.c_int64(10), ctypes.c_float(0), 0, p, null) == cb.CB_OK
     bad = np.array([0, 7], np.int32)
     assert L.cb_probe_scores(p, 2, 2, bad.ctypes.data_as(ctypes.c_void_p), 4, p, null) == cb.CB_ERR_INVALID_ARG
+
+
+def test_token_splits_choice():
+    """Left open (0), the split count balances units over 148 SMs against one more slot set per split."""
+    for (Ls, Lt, H, want) in [(40, 64, 8, 1), (36, 40, 8, 3), (2, 2, 2, 8)]:
+        sl, sh = cb.cb_head_map_nearest(Ls, H, Lt, H)
+        assert cb.cb_token_splits(cb.Problem(Ls, H, 128, Lt, H, 128, sl, sh)) == want
+        assert cb.cb_token_splits(cb.Problem(Ls, H, 128, Lt, H, 128, sl, sh, n_splits=5)) == 5
