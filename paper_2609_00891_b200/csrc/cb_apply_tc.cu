@@ -5,11 +5,12 @@
 //                     tensor core reads (rows = input channel, 64 output channels per 128-byte row, swizzled);
 //                     the bias row goes to shared memory as fp32.
 //   producer thread   TMA: tiles of 128 tokens of the matched source head, [channel block][token][64 channels].
-//   MMA thread        tcgen05.mma  D[128 tokens][2d] += X[128][16] * [W_hi | W_lo][16][2d], A K-major, B MN-major: the hi
-//                     and lo parts of W sit side by side as one N = 2d operand, so the X tile is read from shared
-//                     memory once per K step (two MMAs of N = d read it twice: shared-memory bandwidth is what this
-//                     kernel runs out of next to HBM); fp32 accumulators in tensor memory (two, ping-pong); the
-//                     epilogue adds the two halves.
+//   MMA thread        tcgen05.mma  D[128 tokens][d] += X[128][16] * W_hi[16][d], then the same with W_lo, A K-major,
+//                     B MN-major: both products accumulate into the same tensor-memory columns, so the epilogue has
+//                     no halves to add (one N = 2d operand with the halves added in registers measured 1.5 % slower:
+//                     like the statistics kernel, this one is limited by the board's power, and 128 fp32 adds per
+//                     row cost more than a second read of the X tile by the tensor cores); four fp32 accumulators
+//                     in tensor memory.
 //   epilogue warps    tensor memory -> registers, + bias, -> bf16 into a shared-memory tile -> one TMA store
 //                     (coalesced 256-byte rows, rows past the end clipped); fp32 output is stored directly.
 // Every wait is bounded; a wait that runs out makes the block tear down (nothing else is reported: this call has
@@ -29,7 +30,7 @@
 #define CB_AP_NO 2
 #endif
 #ifndef CB_AP_NACC
-#define CB_AP_NACC 2
+#define CB_AP_NACC 4
 #endif
 
 namespace cb {
@@ -51,7 +52,7 @@ struct ApCfg {
     static constexpr int NS = CB_AP_NS;
     static constexpr int NO = CB_AP_NO;                 // output tiles in shared memory
     static constexpr int NACC = CB_AP_NACC;
-    static constexpr int AW = 2 * D;                    // accumulator columns per tile: X W_hi | X W_lo
+    static constexpr int AW = D;                        // accumulator columns per tile: X W_hi + X W_lo
     static constexpr int TMEM_COLS = (NACC * AW < 32) ? 32 : NACC * AW;
     static constexpr int EPI_WARPS = 4, CONV_WARPS = 4;
     static constexpr int THREADS = (2 + EPI_WARPS + CONV_WARPS) * 32;
@@ -184,8 +185,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
     } else if (warp == 1) {
         // ================================ MMA issuer (one thread) ================================
         if (lane == 0) {
-            constexpr uint32_t idesc_bf = umma_idesc_bf16(128, 2 * D, false, true);   // A K-major, B MN-major, N = hi | lo
-            constexpr uint32_t idesc_hf = umma_idesc_f16(128, 2 * D, false, true);
+            constexpr uint32_t idesc_bf = umma_idesc_bf16(128, C::AW, false, true);   // A K-major, B MN-major
+            constexpr uint32_t idesc_hf = umma_idesc_f16(128, C::AW, false, true);
             // A (K-major, 128-byte swizzle): 8-row groups 1024 bytes apart; a K step of 16 channels is 32 bytes along
             // the row, a block of 64 channels is XBLK further.  B (MN-major): K step = 16 rows = 2048 bytes,
             // 64-output-channel blocks WBLK apart.
@@ -215,6 +216,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                         const uint64_t ad = ((uint64_t)a_hi32 << 32) | ak;
                         // the lo image follows the hi image in shared memory: 2 d / 64 column blocks, WBLK apart
                         umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bh_lo0 + k * 128), idesc, k == 0 ? 0u : 1u);
+                        umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bh_lo0 + ((D / 64) * (C::WBLK >> 4)) + k * 128), idesc, 1u);
                     }
                     umma_commit(&xempty[st.idx]);
                     umma_commit(&accfull[ac.idx]);
@@ -259,17 +261,9 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                     for (int c = 0; c < D / 64; ++c) {
                         uint32_t rl[32], rh[32];
                         {
-                            uint32_t tl[32], th[32];
                             tmem_ld_32x32(taddr + c * 32, rl);
-                            tmem_ld_32x32(taddr + D + c * 32, tl);               // lo-part products
                             tmem_ld_32x32(taddr + D / 2 + c * 32, rh);
-                            tmem_ld_32x32(taddr + D + D / 2 + c * 32, th);
                             tmem_wait_ld();
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                rl[j] = __float_as_uint(__uint_as_float(rl[j]) + __uint_as_float(tl[j]));
-                                rh[j] = __float_as_uint(__uint_as_float(rh[j]) + __uint_as_float(th[j]));
-                            }
                         }
                         float ol[32], oh[32];
 #pragma unroll
@@ -327,12 +321,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
                         {
-                            uint32_t t2[32];
                             tmem_ld_32x32(taddr + c * 32, r);
-                            tmem_ld_32x32(taddr + D + c * 32, t2);               // lo-part products
                             tmem_wait_ld();
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(t2[j]));
                         }
 #pragma unroll
                         for (int v = 0; v < 4; ++v) {           // 4 chunks of 8 channels
@@ -372,12 +362,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
                         {
-                            uint32_t t2[32];
                             tmem_ld_32x32(taddr + c * 32, r);
-                            tmem_ld_32x32(taddr + D + c * 32, t2);               // lo-part products
                             tmem_wait_ld();
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(t2[j]));
                         }
                         if (tok < a.n_tokens) {
 #pragma unroll
