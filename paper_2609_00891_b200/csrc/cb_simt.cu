@@ -230,7 +230,7 @@ __device__ __forceinline__ double shfl_xor_f64(double v, int mask)
 #ifdef CB_SOLVE_TIMING
 __device__ long long g_solve_t[8];
 extern "C" int cb_debug_solve_t(long long *h) { return (int)cudaMemcpyFromSymbol(h, g_solve_t, sizeof(g_solve_t)); }
-#define ST(i) do { if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) g_solve_t[i] = clock64(); } while (0)
+#define ST(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_solve_t[i] = clock64(); } while (0)
 #else
 #define ST(i) do {} while (0)
 #endif
@@ -242,7 +242,8 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
     const int d = a.d, p = d + 1;
     const bool centred = a.mu != nullptr;
     const int n = centred ? d : p;                     // order of the system: the centred form has no bias row
-    const int m = blockIdx.x, li = blockIdx.y;
+    // blocks of one map's lambdas are neighbours in launch order: the second and third read G and C from L2
+    const int m = blockIdx.x / a.n_lambda, li = blockIdx.x % a.n_lambda;
     double *Lp = sm;                                   // packed lower triangle, rows padded to even length
     double *Z = sm + tri_row_start(n);                 // [n][d]
     __shared__ double diag[NB][NB];
@@ -475,7 +476,7 @@ static cudaError_t launch_solve_any(const float *G, const float *C, const float 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    k_ridge_solve<<<dim3(n_maps, n_lambda), 256, smem, st>>>(a);
+    k_ridge_solve<<<n_maps * n_lambda, 256, smem, st>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;
