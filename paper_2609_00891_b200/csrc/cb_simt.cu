@@ -234,6 +234,9 @@ extern "C" int cb_debug_solve_t(long long *h) { return (int)cudaMemcpyFromSymbol
 #else
 #define ST(i) do {} while (0)
 #endif
+#ifndef CB_SOLVE_AHEAD
+#define CB_SOLVE_AHEAD 148
+#endif
 __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
 {
     ST(0);
@@ -256,6 +259,18 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
     const double s_w = centred ? (double)a.mu[(size_t)m * (2 * d + 1) + 2 * d] : (double)Gm[(size_t)d * p + d];
     const double lam = (a.flags & CB_FLAG_RAW_LAMBDA) ? (double)a.lambdas[li] : (double)a.lambdas[li] * s_w * a.inv_n;
     if (tid == 0) s_fail = 0;
+    {
+        // The block that will follow this one on the SM is, to a good guess, gridDim-resident blocks further on (one
+        // block per SM): ask L2 for its statistics now, so that its load phase does not wait for DRAM.
+        const int nb = blockIdx.x + CB_SOLVE_AHEAD;
+        if (nb < (int)gridDim.x && nb / a.n_lambda != m) {
+            const int m2 = nb / a.n_lambda;
+            const char *g2 = reinterpret_cast<const char *>(a.G + (size_t)m2 * n * n);
+            const char *c2 = reinterpret_cast<const char *>(a.C + (size_t)m2 * n * d);
+            for (int o = tid * 128; o < n * n * 4; o += blockDim.x * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(g2 + o));
+            for (int o = tid * 128; o < n * d * 4; o += blockDim.x * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(c2 + o));
+        }
+    }
     {
         const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
         // one warp per row (coalesced, no divisions); the global loads of a row are issued together before any
