@@ -234,10 +234,11 @@ extern "C" int cb_debug_solve_t(long long *h) { return (int)cudaMemcpyFromSymbol
 #else
 #define ST(i) do {} while (0)
 #endif
+constexpr int SOLVE_THREADS = 288;     // 129 rows of L + 128 right-hand-side columns, rounded up to warps
 #ifndef CB_SOLVE_AHEAD
 #define CB_SOLVE_AHEAD 148
 #endif
-__global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
+__global__ void __launch_bounds__(SOLVE_THREADS, 1) k_ridge_solve(const SolveArgs a)
 {
     ST(0);
     extern __shared__ __align__(16) double sm[];
@@ -296,21 +297,35 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
     __syncthreads();
 
     ST(1);
-    // ---------------- Cholesky ----------------
+    // ---------------- Cholesky, with the forward substitution riding along ----------------
+    // Z^T = (L^-1 C)^T obeys the same recurrence as the rows of L below the diagonal block:
+    //     Z[j][c] = (C[j][c] - sum_{k<j} Z[k][c] L[j][k]) / L[j][j],
+    // so thread n + c treats right-hand-side column c as one more row of the matrix being factored (it never
+    // contributes to a diagonal block).  All 257 threads work through the block columns together and no separate
+    // forward pass is needed.
     const int row = tid;
+    const bool is_rhs = tid >= n && tid < n + d;
+    const int col = tid - n;                           // right-hand-side column of an extra row
     const int rs = tri_row_start(row < n ? row : 0);
     for (int j0 = 0; j0 < n; j0 += NB) {
         const int nb = min(NB, n - j0);
         double acc[NB];
-        const bool active = row < n && row >= j0;
+        const bool active = (row < n && row >= j0) || is_rhs;
         if (active) {
+            if (is_rhs) {
 #pragma unroll
-            for (int c = 0; c < NB; ++c) acc[c] = (c < nb && j0 + c <= row) ? Lp[rs + j0 + c] : 0.0;
+                for (int c = 0; c < NB; ++c) acc[c] = (c < nb) ? Z[(size_t)(j0 + c) * d + col] : 0.0;
+            } else {
+#pragma unroll
+                for (int c = 0; c < NB; ++c) acc[c] = (c < nb && j0 + c <= row) ? Lp[rs + j0 + c] : 0.0;
+            }
             int drs[NB];
 #pragma unroll
             for (int c = 0; c < NB; ++c) drs[c] = tri_row_start(min(j0 + c, n - 1));
             for (int k = 0; k < j0; k += 2) {          // j0 is a multiple of 8: aligned pairs
-                const double2 mine = *reinterpret_cast<const double2 *>(&Lp[rs + k]);
+                double2 mine;
+                if (is_rhs) mine = make_double2(Z[(size_t)k * d + col], Z[(size_t)(k + 1) * d + col]);
+                else mine = *reinterpret_cast<const double2 *>(&Lp[rs + k]);
 #pragma unroll
                 for (int c = 0; c < NB; ++c) {
                     const double2 o = *reinterpret_cast<const double2 *>(&Lp[drs[c] + k]);
@@ -318,7 +333,7 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
                     acc[c] -= mine.y * o.y;
                 }
             }
-            if (row < j0 + nb) {
+            if (!is_rhs && row < j0 + nb) {
 #pragma unroll
                 for (int c = 0; c < NB; ++c) diag[row - j0][c] = acc[c];
             }
@@ -363,7 +378,7 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
         }
         __syncthreads();
         if (active) {
-            if (row >= j0 + nb) {
+            if (is_rhs || row >= j0 + nb) {
                 // own row against the block: x_c = (acc_c - sum_{q<c} x_q L[c][q]) / L[c][c]
 #pragma unroll
                 for (int c = 0; c < NB; ++c)
@@ -373,7 +388,8 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
                         for (int q = 0; q < NB; ++q)
                             if (q < c) v -= acc[q] * diag[c][q];
                         acc[c] = v * rdiag[j0 + c];
-                        Lp[rs + j0 + c] = acc[c];
+                        if (is_rhs) Z[(size_t)(j0 + c) * d + col] = acc[c];
+                        else Lp[rs + j0 + c] = acc[c];
                     }
             } else {
                 for (int c = 0; c <= row - j0; ++c) Lp[rs + j0 + c] = diag[row - j0][c];
@@ -391,43 +407,10 @@ __global__ void __launch_bounds__(256, 1) k_ridge_solve(const SolveArgs a)
     }
 
     ST(2);
-    // ---------------- substitutions: column c = tid / 2, the two lanes of a pair split the inner sums ----------------
+    // ---------------- backward substitution: column c = tid / 2, the two lanes of a pair split the inner sums ----------------
     constexpr int RB = 8;
     if (tid < 2 * d) {
         const int c = tid >> 1, half = tid & 1;
-        // forward: L Z = C, row blocks top-down
-        for (int i0 = 0; i0 < n; i0 += RB) {
-            double acc[RB];
-            int rsr[RB];
-#pragma unroll
-            for (int r = 0; r < RB; ++r) {
-                rsr[r] = tri_row_start(min(i0 + r, n - 1));
-                acc[r] = (half == 0 && i0 + r < n) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
-            }
-            for (int k = 2 * half; k < i0; k += 4) {   // pairs (k, k+1), alternating between the two lanes
-                const double z0 = Z[(size_t)k * d + c], z1 = Z[(size_t)(k + 1) * d + c];
-#pragma unroll
-                for (int r = 0; r < RB; ++r) {
-                    const double2 lv = *reinterpret_cast<const double2 *>(&Lp[rsr[r] + k]);
-                    acc[r] -= lv.x * z0;
-                    acc[r] -= lv.y * z1;
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < RB; ++r) acc[r] += shfl_xor_f64(acc[r], 1);
-#pragma unroll
-            for (int r = 0; r < RB; ++r)
-                if (i0 + r < n) {
-                    double v = acc[r];
-#pragma unroll
-                    for (int q = 0; q < RB; ++q)
-                        if (q < r) v -= Lp[rsr[r] + i0 + q] * acc[q];
-                    v *= rdiag[i0 + r];
-                    acc[r] = v;
-                    if (half == 0) Z[(size_t)(i0 + r) * d + c] = v;
-                }
-            __syncwarp();
-        }
         ST(3);
         // backward: L^T Theta = Z, row blocks bottom-up
         const int last = ((n - 1) / RB) * RB;
@@ -491,7 +474,7 @@ static cudaError_t launch_solve_any(const float *G, const float *C, const float 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    k_ridge_solve<<<n_maps * n_lambda, 256, smem, st>>>(a);
+    k_ridge_solve<<<n_maps * n_lambda, SOLVE_THREADS, smem, st>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;
