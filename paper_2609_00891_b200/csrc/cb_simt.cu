@@ -221,12 +221,14 @@ __device__ __forceinline__ double shfl_xor_f64(double v, int mask)
     return __hiloint2double(hi, lo);
 }
 
-// Cholesky by block columns of 8 (left-looking): thread i owns row i.  For a block column it pulls its 8
-// entries into registers, subtracts the contributions of all finished columns (its own row times the 8 rows of
-// the diagonal block, read as broadcasts), the 8 diagonal-block rows publish theirs, every thread factors that
-// 8x8 block redundantly in registers and solves its own row against it.  Two block barriers per block column.
-// The substitutions give every right-hand-side column to a pair of lanes that split the inner sums; eight rows
-// are kept in registers at a time, so each loaded L entry feeds one FMA and each loaded Z entry feeds eight.
+// Cholesky by block columns of 8 (left-looking): thread i owns row i of L; thread n + c owns right-hand-side column c,
+// whose forward substitution obeys the same recurrence as a row of L below the diagonal block and rides along.  For
+// a block column a thread pulls its 8 entries into registers, subtracts the contributions of all finished columns
+// (its own row times the 8 rows of the diagonal block, read as broadcasts), the 8 diagonal-block rows publish theirs,
+// one otherwise idle thread factors that 8 x 8 block in registers while the others already work on the next block
+// column, and every thread solves its own row against the block.  Three block barriers per block column.
+// The backward substitution gives every right-hand-side column to a pair of lanes that split the inner sums; eight
+// rows are kept in registers at a time, so each loaded L entry feeds one FMA and each loaded Z entry feeds eight.
 #ifdef CB_SOLVE_TIMING
 __device__ long long g_solve_t[8];
 extern "C" int cb_debug_solve_t(long long *h) { return (int)cudaMemcpyFromSymbol(h, g_solve_t, sizeof(g_solve_t)); }
@@ -234,7 +236,8 @@ extern "C" int cb_debug_solve_t(long long *h) { return (int)cudaMemcpyFromSymbol
 #else
 #define ST(i) do {} while (0)
 #endif
-constexpr int SOLVE_THREADS = 288;     // 129 rows of L + 128 right-hand-side columns, rounded up to warps
+constexpr int SOLVE_THREADS = 320;     // 129 rows of L + 128 right-hand-side columns, and a warp for the thread that
+constexpr int SOLVE_FACTOR_THREAD = 288;   // factors the diagonal blocks
 #ifndef CB_SOLVE_AHEAD
 #define CB_SOLVE_AHEAD 148
 #endif
@@ -303,43 +306,60 @@ __global__ void __launch_bounds__(SOLVE_THREADS, 1) k_ridge_solve(const SolveArg
     // so thread n + c treats right-hand-side column c as one more row of the matrix being factored (it never
     // contributes to a diagonal block).  All 257 threads work through the block columns together and no separate
     // forward pass is needed.
+    // While one otherwise idle thread factors the 8 x 8 diagonal block of block column j0 (a serial chain of eight
+    // reciprocal square roots), the row threads already subtract the finished columns k < j0 from their entries of
+    // block column j0 + 8; the eight columns of block j0 itself are subtracted at the top of the next iteration.
     const int row = tid;
     const bool is_rhs = tid >= n && tid < n + d;
     const int col = tid - n;                           // right-hand-side column of an extra row
     const int rs = tri_row_start(row < n ? row : 0);
+    // entries of block column jb owned by this thread, before any subtraction
+    auto init_block = [&](double (&ac)[NB], int jb) {
+        const int nbb = min(NB, n - jb);
+        if (is_rhs) {
+#pragma unroll
+            for (int c = 0; c < NB; ++c) ac[c] = (c < nbb) ? Z[(size_t)(jb + c) * d + col] : 0.0;
+        } else {
+#pragma unroll
+            for (int c = 0; c < NB; ++c) ac[c] = (c < nbb && jb + c <= row) ? Lp[rs + jb + c] : 0.0;
+        }
+    };
+    // ac[c] -= sum_{k0 <= k < k1} (own row)[k] * L[jb + c][k]; k0, k1 multiples of 8: aligned pairs
+    auto subtract_columns = [&](double (&ac)[NB], int jb, int k0, int k1) {
+        int drs[NB];
+#pragma unroll
+        for (int c = 0; c < NB; ++c) drs[c] = tri_row_start(min(jb + c, n - 1));
+        for (int k = k0; k < k1; k += 2) {
+            double2 mine;
+            if (is_rhs) mine = make_double2(Z[(size_t)k * d + col], Z[(size_t)(k + 1) * d + col]);
+            else mine = *reinterpret_cast<const double2 *>(&Lp[rs + k]);
+#pragma unroll
+            for (int c = 0; c < NB; ++c) {
+                const double2 o = *reinterpret_cast<const double2 *>(&Lp[drs[c] + k]);
+                ac[c] -= mine.x * o.x;
+                ac[c] -= mine.y * o.y;
+            }
+        }
+    };
+    double acc[NB];
+#pragma unroll
+    for (int c = 0; c < NB; ++c) acc[c] = 0.0;
+    if (row < n || is_rhs) init_block(acc, 0);
     for (int j0 = 0; j0 < n; j0 += NB) {
         const int nb = min(NB, n - j0);
-        double acc[NB];
         const bool active = (row < n && row >= j0) || is_rhs;
         if (active) {
-            if (is_rhs) {
-#pragma unroll
-                for (int c = 0; c < NB; ++c) acc[c] = (c < nb) ? Z[(size_t)(j0 + c) * d + col] : 0.0;
-            } else {
-#pragma unroll
-                for (int c = 0; c < NB; ++c) acc[c] = (c < nb && j0 + c <= row) ? Lp[rs + j0 + c] : 0.0;
-            }
-            int drs[NB];
-#pragma unroll
-            for (int c = 0; c < NB; ++c) drs[c] = tri_row_start(min(j0 + c, n - 1));
-            for (int k = 0; k < j0; k += 2) {          // j0 is a multiple of 8: aligned pairs
-                double2 mine;
-                if (is_rhs) mine = make_double2(Z[(size_t)k * d + col], Z[(size_t)(k + 1) * d + col]);
-                else mine = *reinterpret_cast<const double2 *>(&Lp[rs + k]);
-#pragma unroll
-                for (int c = 0; c < NB; ++c) {
-                    const double2 o = *reinterpret_cast<const double2 *>(&Lp[drs[c] + k]);
-                    acc[c] -= mine.x * o.x;
-                    acc[c] -= mine.y * o.y;
-                }
-            }
+            if (j0 > 0) subtract_columns(acc, j0, j0 - NB, j0);
             if (!is_rhs && row < j0 + nb) {
 #pragma unroll
                 for (int c = 0; c < NB; ++c) diag[row - j0][c] = acc[c];
             }
         }
         __syncthreads();
-        if (row == j0) {
+        double accn[NB];
+#pragma unroll
+        for (int c = 0; c < NB; ++c) accn[c] = 0.0;
+        if (tid == SOLVE_FACTOR_THREAD) {
             // one thread factors the nb x nb diagonal block (sqrt and reciprocal are long fp64 sequences: doing
             // them once and broadcasting beats doing them in every thread); the block is held in registers
             double Ld[NB][NB];
@@ -375,6 +395,9 @@ __global__ void __launch_bounds__(SOLVE_THREADS, 1) k_ridge_solve(const SolveArg
 #pragma unroll
                 for (int c = 0; c < NB; ++c)
                     if (c <= r) diag[r][c] = Ld[r][c];
+        } else if (j0 + NB < n && ((row < n && row >= j0 + NB) || is_rhs)) {
+            init_block(accn, j0 + NB);
+            subtract_columns(accn, j0 + NB, 0, j0);
         }
         __syncthreads();
         if (active) {
@@ -397,6 +420,8 @@ __global__ void __launch_bounds__(SOLVE_THREADS, 1) k_ridge_solve(const SolveArg
         }
         __syncthreads();
         if (s_fail) break;
+#pragma unroll
+        for (int c = 0; c < NB; ++c) acc[c] = accn[c];
     }
 
     float *Wm = a.Wb + ((size_t)li * a.n_maps + m) * p * d;
