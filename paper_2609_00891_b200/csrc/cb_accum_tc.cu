@@ -31,6 +31,7 @@
 
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
+#include "cb_math.cuh"
 #include "cb_rope.cuh"
 
 namespace cb {
@@ -186,52 +187,6 @@ struct TileIterT {
     }
 };
 
-__device__ __forceinline__ void unpack_bf16x8(const uint4 &v, float *f)
-{
-    const unsigned u[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        f[2 * i] = __uint_as_float(u[i] << 16);
-        f[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
-    }
-}
-// Packed fp32 pairs (sm_100 executes add/mul/fma on two fp32 lanes per instruction): halves the number of
-// floating-point instructions of the fold, which is what the block runs out of (issue slots and power).
-__device__ __forceinline__ uint64_t f2_pack(float lo, float hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void f2_unpack(uint64_t v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-// bf16 pair (one 32-bit word: low half = first element) -> packed fp32 pair, exact
-__device__ __forceinline__ uint64_t f2_from_bf16x2(unsigned u) { return f2_pack(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)); }
-
-__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
-{
-    unsigned r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
 #ifdef CB_TRACE
 // Tuning aid: block 0 records clock64() of every role for tiles [CB_TRACE_T0, CB_TRACE_T0 + 64).
 #define CB_TRACE_T0 1000
@@ -241,13 +196,6 @@ extern "C" int cb_debug_trace(long long *host) { return (int)cudaMemcpyFromSymbo
 #else
 #define CB_TR(itv, slot) do {} while (0)
 #endif
-
-// Position in a ring of N buffers guarded by mbarriers: index and the parity of the current pass.
-template <int N>
-struct Ring {
-    uint32_t idx = 0, phase = 0;
-    __device__ __forceinline__ void next() { if (++idx == N) { idx = 0; phase ^= 1; } }
-};
 
 // ROPE: key maps (comp = 0) are fitted in content coordinates (Section 3.1): the fold warps rotate every source and
 // target key row back by its position's angles IN PLACE in the staged tile (so the tensor cores read the de-rotated

@@ -38,6 +38,7 @@
 
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
+#include "cb_math.cuh"
 
 namespace cb {
 
@@ -112,40 +113,6 @@ struct UnitIter {
         if (++tile >= tile1) next_unit(a, n_units, n_maps, n_tiles);
     }
 };
-
-template <int N>
-struct Ring {
-    uint32_t idx = 0, phase = 0;
-    __device__ __forceinline__ void next() { if (++idx == N) { idx = 0; phase ^= 1; } }
-};
-
-// Packed fp32 pairs (two fp32 lanes per instruction).
-__device__ __forceinline__ uint64_t f2_pack(float lo, float hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void f2_unpack(uint64_t v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t f2_from_bf16x2(unsigned u) { return f2_pack(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)); }
-__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
-{
-    unsigned r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
 
 // CEN: two-pass centred construction: the weighted operand is w (x - mu_x) with the means of P.a.mu; s_y is not
 // formed (the slot's entries stay zero); the slot's s_x entries become the column sums of the ROUNDED weighted

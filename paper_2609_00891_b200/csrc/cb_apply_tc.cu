@@ -21,6 +21,7 @@
 
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
+#include "cb_math.cuh"
 #include "cb_rope.cuh"
 
 #ifndef CB_AP_NS
@@ -86,19 +87,6 @@ struct ApIter {   // units u = blockIdx.x, += gridDim.x; unit -> (map, split) ->
         next_unit(n_units, n_maps, n_tiles, n_splits);
     }
 };
-
-template <int N>
-struct ApRing {
-    uint32_t idx = 0, phase = 0;
-    __device__ __forceinline__ void next() { if (++idx == N) { idx = 0; phase ^= 1; } }
-};
-
-__device__ __forceinline__ unsigned ap_pack_bf16x2(float lo, float hi)
-{
-    unsigned r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
 
 // fp16 pair (low half = first element)
 __device__ __forceinline__ unsigned ap_pack_f16x2(float lo, float hi)
@@ -167,7 +155,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         if (lane == 0) {
             ApIter cur;
             cur.start(n_units, n_maps, n_tiles, P.n_splits);
-            ApRing<C::NS> st;
+            Ring<C::NS> st;
             while (cur.u < n_units) {
                 const int m = cur.m;
                 const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
@@ -197,8 +185,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
             const uint32_t bh_lo0 = (uint32_t)proto_b | ((smem_u32(whi) & 0x3FFFFu) >> 4);
             ApIter cur;
             cur.start(n_units, n_maps, n_tiles, P.n_splits);
-            ApRing<C::NS> st;
-            ApRing<C::NACC> ac;
+            Ring<C::NS> st;
+            Ring<C::NACC> ac;
             uint32_t uc = 0;
             while (cur.u < n_units) {
                 if (!mbar_wait(wready, uc & 1, abort_flag)) goto teardown;
@@ -234,11 +222,11 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         const int row = q * 32 + lane;          // token row inside the tile
         ApIter cur;
         cur.start(n_units, n_maps, n_tiles, P.n_splits);
-        ApRing<C::NACC> ac;
-        ApRing<C::NO> ob;
+        Ring<C::NACC> ac;
+        Ring<C::NO> ob;
         uint32_t uc = 0;
         const bool storer = (warp == 2 && lane == 0);
-        ApRing<C::NO> oldest;          // storer only: oldest output tile whose store may still be reading
+        Ring<C::NO> oldest;          // storer only: oldest output tile whose store may still be reading
         int pending = 0;
         while (cur.u < n_units) {
             const int m = cur.m;
@@ -279,10 +267,10 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
 #pragma unroll
                             for (int v = 0; v < 4; ++v) {
                                 const int nl = c * 32 + v * 8, nh = D / 2 + nl;
-                                const uint4 pl = make_uint4(ap_pack_bf16x2(ol[v * 8 + 0], ol[v * 8 + 1]), ap_pack_bf16x2(ol[v * 8 + 2], ol[v * 8 + 3]),
-                                                            ap_pack_bf16x2(ol[v * 8 + 4], ol[v * 8 + 5]), ap_pack_bf16x2(ol[v * 8 + 6], ol[v * 8 + 7]));
-                                const uint4 ph = make_uint4(ap_pack_bf16x2(oh[v * 8 + 0], oh[v * 8 + 1]), ap_pack_bf16x2(oh[v * 8 + 2], oh[v * 8 + 3]),
-                                                            ap_pack_bf16x2(oh[v * 8 + 4], oh[v * 8 + 5]), ap_pack_bf16x2(oh[v * 8 + 6], oh[v * 8 + 7]));
+                                const uint4 pl = make_uint4(pack_bf16x2(ol[v * 8 + 0], ol[v * 8 + 1]), pack_bf16x2(ol[v * 8 + 2], ol[v * 8 + 3]),
+                                                            pack_bf16x2(ol[v * 8 + 4], ol[v * 8 + 5]), pack_bf16x2(ol[v * 8 + 6], ol[v * 8 + 7]));
+                                const uint4 ph = make_uint4(pack_bf16x2(oh[v * 8 + 0], oh[v * 8 + 1]), pack_bf16x2(oh[v * 8 + 2], oh[v * 8 + 3]),
+                                                            pack_bf16x2(oh[v * 8 + 4], oh[v * 8 + 5]), pack_bf16x2(oh[v * 8 + 6], oh[v * 8 + 7]));
                                 *reinterpret_cast<uint4 *>(ot + (nl >> 6) * C::XBLK + row * 128 + ((((nl & 63) >> 3) ^ (row & 7)) << 4)) = pl;
                                 *reinterpret_cast<uint4 *>(ot + (nh >> 6) * C::XBLK + row * 128 + ((((nh & 63) >> 3) ^ (row & 7)) << 4)) = ph;
                             }
@@ -328,10 +316,10 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                         for (int v = 0; v < 4; ++v) {           // 4 chunks of 8 channels
                             const int n0 = c * 32 + v * 8;
                             uint4 pk;
-                            pk.x = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 0]) + bias[n0 + 0], __uint_as_float(r[v * 8 + 1]) + bias[n0 + 1]);
-                            pk.y = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 2]) + bias[n0 + 2], __uint_as_float(r[v * 8 + 3]) + bias[n0 + 3]);
-                            pk.z = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 4]) + bias[n0 + 4], __uint_as_float(r[v * 8 + 5]) + bias[n0 + 5]);
-                            pk.w = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 6]) + bias[n0 + 6], __uint_as_float(r[v * 8 + 7]) + bias[n0 + 7]);
+                            pk.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]) + bias[n0 + 0], __uint_as_float(r[v * 8 + 1]) + bias[n0 + 1]);
+                            pk.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]) + bias[n0 + 2], __uint_as_float(r[v * 8 + 3]) + bias[n0 + 3]);
+                            pk.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]) + bias[n0 + 4], __uint_as_float(r[v * 8 + 5]) + bias[n0 + 5]);
+                            pk.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]) + bias[n0 + 6], __uint_as_float(r[v * 8 + 7]) + bias[n0 + 7]);
                             const int blk = n0 >> 6, chunk = (n0 & 63) >> 3;
                             *reinterpret_cast<uint4 *>(ot + blk * C::XBLK + row * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
                         }
@@ -394,7 +382,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         ApIter cur;
         cur.start(n_units, n_maps, n_tiles, P.n_splits);
         uint32_t uc = 0;
-        ApRing<C::NS> st;                                             // ROPE: follows the producer's ring
+        Ring<C::NS> st;                                             // ROPE: follows the producer's ring
         // ROPE: this thread rotates the pair of 16-byte chunks (lc, lc + half a row) of RB consecutive rows.  Along
         // consecutive positions the angle of a frequency advances by a fixed step, so (cos, sin) of the next row follow
         // from the current ones by one rotation with the thread's constants (cos, sin)(theta_i); the special-function
@@ -430,9 +418,9 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                         lo[e] = ap_pack_f16x2(f[2 * e] - hf.x, f[2 * e + 1] - hf.y);
                         continue;
                     }
-                    hi[e] = ap_pack_bf16x2(f[2 * e], f[2 * e + 1]);
+                    hi[e] = pack_bf16x2(f[2 * e], f[2 * e + 1]);
                     const float h0 = __uint_as_float(hi[e] << 16), h1 = __uint_as_float(hi[e] & 0xffff0000u);
-                    lo[e] = ap_pack_bf16x2(f[2 * e] - h0, f[2 * e + 1] - h1);
+                    lo[e] = pack_bf16x2(f[2 * e] - h0, f[2 * e + 1] - h1);
                 }
                 const int off = (n0 >> 6) * C::WBLK + k * 128 + ((((n0 & 63) >> 3) ^ (k & 7)) << 4);
                 *reinterpret_cast<uint4 *>(whi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -623,8 +611,8 @@ __global__ void __launch_bounds__(256) k_w_split(const float *__restrict__ Wb, u
         unsigned hi[4], lo[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            hi[e] = ap_pack_bf16x2(v[2 * e], v[2 * e + 1]);
-            lo[e] = ap_pack_bf16x2(v[2 * e] - __uint_as_float(hi[e] << 16), v[2 * e + 1] - __uint_as_float(hi[e] & 0xffff0000u));
+            hi[e] = pack_bf16x2(v[2 * e], v[2 * e + 1]);
+            lo[e] = pack_bf16x2(v[2 * e] - __uint_as_float(hi[e] << 16), v[2 * e + 1] - __uint_as_float(hi[e] & 0xffff0000u));
         }
         const int off = (n0 >> 6) * C::WBLK + kk * 128 + ((((n0 & 63) >> 3) ^ (kk & 7)) << 4);
         *reinterpret_cast<uint4 *>(dst + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -674,7 +662,7 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
         if (lane == 0) {          // producer: source tile and W block of every (tile, f)
             ApIter cur;
             cur.start(n_units, n_maps, n_tiles, P.n_splits);
-            ApRing<C::NS> st;
+            Ring<C::NS> st;
             while (cur.u < n_units) {
                 const int m = cur.m;
                 const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
@@ -703,8 +691,8 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
             const uint32_t b_lo0 = (uint32_t)proto_b | ((smem_u32(st_base + C::X_BYTES) & 0x3FFFFu) >> 4);
             ApIter cur;
             cur.start(n_units, n_maps, n_tiles, P.n_splits);
-            ApRing<C::NS> st;
-            ApRing<C::NACC> ac;
+            Ring<C::NS> st;
+            Ring<C::NACC> ac;
             while (cur.u < n_units) {
                 for (int tile = cur.tile; tile < cur.tile1; ++tile) {
                     if (!mbar_wait(&accempty[ac.idx], ac.phase ^ 1, abort_flag)) goto ml_teardown;
@@ -736,7 +724,7 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
         const int row = q * 32 + lane;
         ApIter cur;
         cur.start(n_units, n_maps, n_tiles, P.n_splits);
-        ApRing<C::NACC> ac;
+        Ring<C::NACC> ac;
         uint32_t oc = 0;
         const bool storer = (warp == 2 && lane == 0);
         while (cur.u < n_units) {
@@ -762,10 +750,10 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
                             const float4 b0 = __ldg(reinterpret_cast<const float4 *>(bias + n0));
                             const float4 b1 = __ldg(reinterpret_cast<const float4 *>(bias + n0 + 4));
                             uint4 pk;
-                            pk.x = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 0]) + b0.x, __uint_as_float(r[v * 8 + 1]) + b0.y);
-                            pk.y = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 2]) + b0.z, __uint_as_float(r[v * 8 + 3]) + b0.w);
-                            pk.z = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 4]) + b1.x, __uint_as_float(r[v * 8 + 5]) + b1.y);
-                            pk.w = ap_pack_bf16x2(__uint_as_float(r[v * 8 + 6]) + b1.z, __uint_as_float(r[v * 8 + 7]) + b1.w);
+                            pk.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]) + b0.x, __uint_as_float(r[v * 8 + 1]) + b0.y);
+                            pk.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]) + b0.z, __uint_as_float(r[v * 8 + 3]) + b0.w);
+                            pk.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]) + b1.x, __uint_as_float(r[v * 8 + 5]) + b1.y);
+                            pk.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]) + b1.z, __uint_as_float(r[v * 8 + 7]) + b1.w);
                             const int blk = n0 >> 6, chunk = (n0 & 63) >> 3;
                             *reinterpret_cast<uint4 *>(os + blk * C::XBLK + row * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
                         }

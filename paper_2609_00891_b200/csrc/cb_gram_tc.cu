@@ -26,6 +26,7 @@
 
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
+#include "cb_math.cuh"
 
 namespace cb {
 
@@ -152,45 +153,6 @@ struct GrUnit {
     }
 };
 
-__device__ __forceinline__ uint64_t g2_pack(float lo, float hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void g2_unpack(uint64_t v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ uint64_t g2_mul(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t g2_add(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t g2_fma(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ uint64_t g2_from_bf16x2(unsigned u) { return g2_pack(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)); }
-__device__ __forceinline__ unsigned g2_to_bf16x2(float lo, float hi)
-{
-    unsigned r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
-template <int N>
-struct GrRing {
-    uint32_t idx = 0, phase = 0;
-    __device__ __forceinline__ void next() { if (++idx == N) { idx = 0; phase ^= 1; } }
-};
-
 #ifdef CB_GTRACE
 // Tuning aid: block 0 records clock64() of its roles for its tiles [CB_GTRACE_T0, CB_GTRACE_T0 + 64).
 #define CB_GTRACE_T0 2000
@@ -249,7 +211,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
     if (warp == 0) {
         // ================================ row-head producer (one thread) ================================
         if (lane == 0) {
-            GrRing<C::NS> st;
+            Ring<C::NS> st;
             GrUnit un;
             int itc = 0;
             for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
@@ -274,7 +236,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
         }
     } else if (warp == C::CPROD_WARP) {
         // ================================ column-head + weights producer ================================
-        GrRing<C::NS> st;
+        Ring<C::NS> st;
         GrUnit un;
         for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
             un.decode(P, u);
@@ -308,7 +270,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
             const uint64_t proto = umma_smem_desc_sw128(0, C::BLK, 1024);
             const uint32_t desc_hi = (uint32_t)(proto >> 32);
             const uint32_t b_lo0 = (uint32_t)proto | ((smem_u32(stg) & 0x3FFFFu) >> 4);
-            GrRing<C::NS> st;
+            Ring<C::NS> st;
             uint32_t sr = 0;
             int itm = 0;
             GrUnit un;
@@ -354,7 +316,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
         const int cc = gt % C::CC, rg = gt / C::CC;
         const int blk = cc >> 3, lc = cc & 7;
         const int off0 = blk * C::BLK + rg * 128 + ((lc ^ (rg & 7)) << 4);
-        GrRing<C::NS> st;
+        Ring<C::NS> st;
         uint32_t uc = 0;
         int itf = 0;
         GrUnit un;
@@ -380,24 +342,24 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                     for (int i = 0; i < C::RPT; ++i) {
                         const int off = i * C::RG * 128;
                         const float wt = wsm[i * C::RG];
-                        const uint64_t w2 = g2_pack(wt, wt);
+                        const uint64_t w2 = f2_pack(wt, wt);
                         const uint4 xv = *reinterpret_cast<const uint4 *>(rs + off);
                         const unsigned xu[4] = {xv.x, xv.y, xv.z, xv.w};
                         unsigned hw[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const uint64_t pr = g2_mul(w2, g2_from_bf16x2(xu[e]));
-                            if (sum_rows) sa2[e] = g2_add(sa2[e], pr);
+                            const uint64_t pr = f2_mul(w2, f2_from_bf16x2(xu[e]));
+                            if (sum_rows) sa2[e] = f2_add(sa2[e], pr);
                             float p0, p1;
-                            g2_unpack(pr, p0, p1);
-                            hw[e] = g2_to_bf16x2(p0, p1);
+                            f2_unpack(pr, p0, p1);
+                            hw[e] = pack_bf16x2(p0, p1);
                         }
                         *reinterpret_cast<uint4 *>(ah + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
                         if (sum_cols) {
                             const uint4 yv = *reinterpret_cast<const uint4 *>(cs + off);
                             const unsigned yu[4] = {yv.x, yv.y, yv.z, yv.w};
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) sb2[e] = g2_fma(w2, g2_from_bf16x2(yu[e]), sb2[e]);
+                            for (int e = 0; e < 4; ++e) sb2[e] = f2_fma(w2, f2_from_bf16x2(yu[e]), sb2[e]);
                         }
                         if (cc == 0 && g == 0) sw += wt;
                     }
@@ -406,11 +368,11 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                     for (int i = 0; i < C::RPT; ++i) {
                         const int off = i * C::RG * 128;
                         const float wt = wsm[i * C::RG];
-                        const uint64_t w2 = g2_pack(wt, wt);
+                        const uint64_t w2 = f2_pack(wt, wt);
                         const uint4 yv = *reinterpret_cast<const uint4 *>(cs + off);
                         const unsigned yu[4] = {yv.x, yv.y, yv.z, yv.w};
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) sb2[e] = g2_fma(w2, g2_from_bf16x2(yu[e]), sb2[e]);
+                        for (int e = 0; e < 4; ++e) sb2[e] = f2_fma(w2, f2_from_bf16x2(yu[e]), sb2[e]);
                     }
                 }
                 if (lane == 0 && fw == 0) GTR(itf, 11);
@@ -426,7 +388,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
             if (un.is_c) {
                 float sa[8], sb[8];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) { g2_unpack(sa2[e], sa[2 * e], sa[2 * e + 1]); g2_unpack(sb2[e], sb[2 * e], sb[2 * e + 1]); }
+                for (int e = 0; e < 4; ++e) { f2_unpack(sa2[e], sa[2 * e], sa[2 * e + 1]); f2_unpack(sb2[e], sb[2 * e], sb[2 * e + 1]); }
                 if (C::CC == 16) {
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
