@@ -1,6 +1,6 @@
 // Fused weighted-statistics accumulation on the 5th-generation tensor cores (sm_100a), both MMA operands in shared
-// memory.  This kernel serves d = 64, the rotary fold and the one-row-head full-head variant; head-local calls with
-// d = 128 go to the kernel that keeps the weighted operand in tensor memory (cb_accum_ts.cu).
+// memory.  This kernel serves d = 64 and the one-row-head full-head variant; head-local calls with d = 128 go to
+// the kernel that keeps the weighted operand in tensor memory (cb_accum_ts.cu).
 //
 // For one map (matched source head X, target head Y, token weights w) the statistics are the dense contraction
 //     D[d][2d] = (w .* X)^T [X | Y]          over tokens,
@@ -820,8 +820,8 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     // Calls of fewer than 4,096 rows take the hi + lo weighted operand regardless of the flag: the single bf16
     // rounding averages out only like 1/sqrt(rows), such calls are bound by launch latency, not by the second MMA.
     const bool comp = a.compensated || a.n_tokens < 4096;
-    // d = 128 without the rotary fold: the kernel that keeps the weighted operand in tensor memory
-    if (d == 128 && !a.rope_pos) return launch_accum_ts(a, comp, src, tgt, st);
+    // d = 128: the kernel that keeps the weighted operand in tensor memory
+    if (d == 128) return launch_accum_ts(a, comp, src, tgt, st);
     TcParams P;
     P.a = a;
     P.fh = FhDev{};
@@ -838,10 +838,8 @@ cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, co
     // Tokens summed in tensor memory before a drain (the fp32 accumulation of the tensor cores loses about 1e-4 over
     // 16,384 tokens; the compensated fold drains eight times as often).
     P.drain_tiles = (comp ? 2048 : 16384) / TT;
-    if (a.rope_pos) {
-        if (comp) e = (d == 128) ? launch_tc<128, true, false, false, true>(P, st) : launch_tc<64, true, false, false, true>(P, st);
-        else e = (d == 128) ? launch_tc<128, false, false, false, true>(P, st) : launch_tc<64, false, false, false, true>(P, st);
-    } else if (a.mu) e = comp ? launch_tc<64, true, false, true>(P, st) : launch_tc<64, false, false, true>(P, st);
+    if (a.rope_pos) e = comp ? launch_tc<64, true, false, false, true>(P, st) : launch_tc<64, false, false, false, true>(P, st);
+    else if (a.mu) e = comp ? launch_tc<64, true, false, true>(P, st) : launch_tc<64, false, false, true>(P, st);
     else e = comp ? launch_tc<64, true>(P, st) : launch_tc<64, false>(P, st);
     if (e == cudaSuccess) count_launch();
     return e;

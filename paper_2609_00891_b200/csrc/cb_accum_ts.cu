@@ -1,5 +1,5 @@
 // Head-local weighted statistics (d = 128) with the weighted operand in TENSOR MEMORY and the bias sum s_y on the
-// tensor cores.
+// tensor cores; plain, compensated, centred (two-pass) and rotary-boundary variants.
 //
 // Same contraction as the shared-memory kernel (D[d][2d] = (w .* X)^T [X | Y] over tokens plus the bias sums), same
 // units, slots and summation order of the splits.  What differs is where the first MMA operand lives: the fold warps
@@ -39,6 +39,7 @@
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
 #include "cb_math.cuh"
+#include "cb_rope.cuh"
 
 namespace cb {
 
@@ -70,7 +71,7 @@ struct TsCfg {
     static constexpr int THREADS = (YPROD_WARP + 1) * 32;
     static constexpr int TW = TT / FOLD_WARPS;        // tokens whose weights a fold warp converts
     static constexpr int RED_FLOATS = 2 * D + 16;     // s_x of the two token halves, partial s_w of the fold warps
-    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * (STAGE_BYTES + WB_BYTES) + RED_FLOATS * 4 + NS * TT * 4 + 256;
+    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * (STAGE_BYTES + WB_BYTES) + RED_FLOATS * 4 + 2 * NS * TT * 4 + 256;
     static_assert(BIAS_COL + 16 <= TMEM_COLS, "tensor memory columns");
     static_assert(NA <= NS, "an operand buffer is released through its tile's stage barrier");
 };
@@ -79,6 +80,7 @@ struct TsParams {
     CUtensorMap src_k, src_v, tgt_k, tgt_v;   // 5-D tiled maps: (64 channels, token, channel block, head, layer)
     AccumArgs a;
     int drain_tiles;                          // tiles accumulated in tensor memory between drains
+    RopeDev rope;                             // ROPE kernels only
 };
 
 // Walks the tiles of this block's units in order: units u = blockIdx.x, += gridDim.x; unit -> (map, split) -> tiles
@@ -117,7 +119,10 @@ struct UnitIter {
 // CEN: two-pass centred construction: the weighted operand is w (x - mu_x) with the means of P.a.mu; s_y is not
 // formed (the slot's entries stay zero); the slot's s_x entries become the column sums of the ROUNDED weighted
 // operand (what the centred reduction needs for its exact correction).
-template <bool COMP, bool CEN>
+// ROPE: key maps (comp = 0) are fitted in content coordinates (Section 3.1): before the fold proper, the fold warps
+// rotate every source and target key row of the staged tile back by its position's angles IN PLACE (the tensor cores
+// read the de-rotated rows as the second operand and for s_y); value maps take the ordinary path.
+template <bool COMP, bool CEN, bool ROPE>
 __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __grid_constant__ TsParams P)
 {
     using C = TsCfg<COMP>;
@@ -129,7 +134,8 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
     float *redx = reinterpret_cast<float *>(wb + (size_t)C::NS * C::WB_BYTES);   // [2 token halves][D] partial s_x
     float *red = redx + 2 * D;                                // [FOLD_WARPS] partial s_w
     float *wst = red + 16;                                    // [NS][TT] token weights of the staged tile
-    uint64_t *bars = reinterpret_cast<uint64_t *>(wst + C::NS * C::TT);
+    int *pst = reinterpret_cast<int *>(wst + C::NS * C::TT);  // [NS][TT] token positions (ROPE)
+    uint64_t *bars = reinterpret_cast<uint64_t *>(pst + C::NS * C::TT);
     uint64_t *full = bars;                 // [NS] tile landed: X bytes (1 arrival), Y bytes (1), weights (32 lanes)
     uint64_t *empty = full + C::NS;        // [NS] stage free: MMA done (1) + every fold warp done
     uint64_t *afull = empty + C::NS;       // [NA] weighted operand written to tensor memory (every fold warp)
@@ -207,6 +213,7 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                     const int r = lane + 32 * q;
                     const bool in = tok0 + r < a.n_tokens;
                     cp_async_4(&wst[st.idx * C::TT + r], w + (in ? tok0 + r : 0), in ? 4u : 0u);
+                    if (ROPE) cp_async_4(&pst[st.idx * C::TT + r], P.rope.pos + (in ? tok0 + r : 0), in ? 4u : 0u);
                 }
                 cp_async_arrive_noinc(&full[st.idx]);
                 st.next();
@@ -281,6 +288,28 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
         // (64-token block, row n, 16-byte chunk (token / 8) XOR n, token % 8): rows 0 and 1
         const int wb_off0 = (wtok >> 6) * 2048 + (((wtok & 63) >> 3) << 4) + (wtok & 7) * 2;
         const int wb_off1 = (wtok >> 6) * 2048 + 128 + ((((wtok & 63) >> 3) ^ 1) << 4) + (wtok & 7) * 2;
+        // ROPE: thread (rc, rr) rotates the frequencies 4 rc .. 4 rc + 3 (channels i and i + 64: the same place in the
+        // two 64-channel blocks of a tile) of rows rr, rr + 16, ..  Along its rows the positions advance by 16 and from
+        // tile to tile by TT, so (cos, sin) follow from the previous ones by one rotation with the thread's constants;
+        // the polynomial is needed at the first tile of a unit, where positions break, and every 16th tile (drift).
+        // Packed fp32 pairs: frequencies (4 rc, 4 rc + 1) and (4 rc + 2, 4 rc + 3).
+        const int rc = (tid - 64) & 15, rr = (tid - 64) >> 4;
+        const int rp_off = rr * 128 + (((rc >> 1) ^ (rr & 7)) << 4) + (rc & 1) * 8;
+        uint64_t rs16c[2] = {0ull, 0ull}, rs16s[2] = {0ull, 0ull}, rsTc[2] = {0ull, 0ull}, rsTs[2] = {0ull, 0ull};   // cos, sin of 16 theta, TT theta
+        uint64_t seedc[2] = {0ull, 0ull}, seeds[2] = {0ull, 0ull};
+        int seedpos = 0;
+        if (ROPE) {
+#pragma unroll
+            for (int pp = 0; pp < 2; ++pp) {
+                float c0, s0, c1, s1;
+                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp], 16, c0, s0);
+                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp + 1], 16, c1, s1);
+                rs16c[pp] = f2_pack(c0, c1); rs16s[pp] = f2_pack(s0, s1);
+                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp], C::TT, c0, s0);
+                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp + 1], C::TT, c1, s1);
+                rsTc[pp] = f2_pack(c0, c1); rsTs[pp] = f2_pack(s0, s1);
+            }
+        }
         Ring<C::NS> st, old;       // `old` trails `st` by NA tiles
         Ring<C::NA> ar;
         uint32_t it = 0, uc = 0;
@@ -288,6 +317,7 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
         cur.start(a, n_units, n_maps, n_tiles);
         while (cur.valid(n_units)) {
             const int m = cur.m, split = cur.split, n_t = cur.tile1 - cur.tile;
+            const bool rope_unit = ROPE && cur.comp == 0;
             uint64_t sx2[2][2];            // [16-channel group][chunk]: sums over this thread's token pairs
             uint64_t nmu2[2][2];
             float sw = 0.f;
@@ -312,6 +342,70 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                 }
                 const uint32_t stage_u32 = smem_u32(xy + st.idx * C::STAGE_BYTES);
                 const float *wt = wst + st.idx * C::TT;
+                if (rope_unit) {
+                    uint8_t *xt = xy + st.idx * C::STAGE_BYTES + rp_off;      // this thread's place in row rr of block 0
+                    const int *pt = pst + st.idx * C::TT + rr;
+                    const uint64_t neg1 = f2_pack(-1.f, -1.f);
+                    uint64_t cc2[2], ss2[2];
+                    int curpos = 0;
+#pragma unroll
+                    for (int i = 0; i < C::TT / 16; ++i) {
+                        const int pos = pt[16 * i];
+                        bool fresh;
+                        if (i == 0) fresh = (t == 0) || (pos != seedpos + C::TT) || ((t & 15) == 0);
+                        else fresh = (pos != curpos + 16);
+                        if (fresh) {
+#pragma unroll
+                            for (int pp = 0; pp < 2; ++pp) {
+                                float c0, s0, c1, s1;
+                                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp], pos, c0, s0);
+                                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp + 1], pos, c1, s1);
+                                cc2[pp] = f2_pack(c0, c1); ss2[pp] = f2_pack(s0, s1);
+                            }
+                        } else {
+#pragma unroll
+                            for (int pp = 0; pp < 2; ++pp) {        // angle += (TT or 16) theta
+                                const uint64_t pc = (i == 0) ? seedc[pp] : cc2[pp], ps = (i == 0) ? seeds[pp] : ss2[pp];
+                                const uint64_t kc = (i == 0) ? rsTc[pp] : rs16c[pp], ks = (i == 0) ? rsTs[pp] : rs16s[pp];
+                                cc2[pp] = f2_fma(pc, kc, f2_mul(f2_mul(ps, ks), neg1));
+                                ss2[pp] = f2_fma(ps, kc, f2_mul(pc, ks));
+                            }
+                        }
+                        if (i == 0) { seedc[0] = cc2[0]; seedc[1] = cc2[1]; seeds[0] = ss2[0]; seeds[1] = ss2[1]; seedpos = pos; }
+                        curpos = pos;
+                        uint64_t yc2[2] = {cc2[0], cc2[1]}, ys2[2] = {ss2[0], ss2[1]};
+                        if (!P.rope.same) {
+#pragma unroll
+                            for (int pp = 0; pp < 2; ++pp) {
+                                float c0, s0, c1, s1;
+                                rope_cs_poly(P.rope.f_tgt[rc * 4 + 2 * pp], pos, c0, s0);
+                                rope_cs_poly(P.rope.f_tgt[rc * 4 + 2 * pp + 1], pos, c1, s1);
+                                yc2[pp] = f2_pack(c0, c1); ys2[pp] = f2_pack(s0, s1);
+                            }
+                        }
+#pragma unroll
+                        for (int xyi = 0; xyi < 2; ++xyi) {           // source tile, then target tile
+                            uint8_t *lo = xt + xyi * 2 * C::BLK + i * (16 * 128), *hi = lo + C::BLK;
+                            const uint2 vl = *reinterpret_cast<const uint2 *>(lo), vh = *reinterpret_cast<const uint2 *>(hi);
+                            const unsigned ul[2] = {vl.x, vl.y}, uh[2] = {vh.x, vh.y};
+                            unsigned ol[2], oh[2];
+#pragma unroll
+                            for (int pp = 0; pp < 2; ++pp) {          // rotation by -phi
+                                const uint64_t c2 = xyi ? yc2[pp] : cc2[pp], s2 = xyi ? ys2[pp] : ss2[pp];
+                                const uint64_t l2 = f2_from_bf16x2(ul[pp]), h2 = f2_from_bf16x2(uh[pp]);
+                                const uint64_t nl = f2_fma(l2, c2, f2_mul(h2, s2));
+                                const uint64_t nh = f2_fma(h2, c2, f2_mul(f2_mul(l2, s2), neg1));
+                                float a0, a1;
+                                f2_unpack(nl, a0, a1); ol[pp] = pack_bf16x2(a0, a1);
+                                f2_unpack(nh, a0, a1); oh[pp] = pack_bf16x2(a0, a1);
+                            }
+                            *reinterpret_cast<uint2 *>(lo) = make_uint2(ol[0], ol[1]);
+                            *reinterpret_cast<uint2 *>(hi) = make_uint2(oh[0], oh[1]);
+                        }
+                    }
+                    // every fold warp reads rows that other fold warps have just rewritten
+                    asm volatile("bar.sync 1, %0;" ::"n"(C::FOLD_WARPS * 32) : "memory");
+                }
                 if (lane < C::TW) {
                     const float wv = wt[wtok];
                     const __nv_bfloat16 h = __float2bfloat16_rn(wv);
@@ -361,7 +455,7 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                     }
                 }
                 tmem_wait_st();
-                fence_async_smem();          // the wb rows written above are read by the tensor cores
+                fence_async_smem();          // the wb rows (and rotated tiles) written above are read by the tensor cores
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&afull[ar.idx]); mbar_arrive(&empty[st.idx]); }
@@ -469,25 +563,25 @@ int ts_sm_count()
     return n;
 }
 
-template <bool COMP, bool CEN>
+template <bool COMP, bool CEN, bool ROPE = false>
 cudaError_t launch_ts(const TsParams &P, cudaStream_t st)
 {
     using C = TsCfg<COMP>;
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_accum_ts<COMP, CEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(k_accum_ts<COMP, CEN, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr = true;
     }
     const int n_units = 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
     const int grid = n_units < ts_sm_count() ? n_units : ts_sm_count();
-    k_accum_ts<COMP, CEN><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
+    k_accum_ts<COMP, CEN, ROPE><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-// d = 128, keys taken as stored (no rotary fold).  `comp`: hi + lo weighted operand.
+// d = 128.  `comp`: hi + lo weighted operand.
 cudaError_t launch_accum_ts(const AccumArgs &a, bool comp, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st)
 {
     TsParams P;
@@ -507,7 +601,14 @@ cudaError_t launch_accum_ts(const AccumArgs &a, bool comp, const cb_kv_view *src
     // its result stays an order of magnitude below the single-bf16 fold's error.
     P.drain_tiles = (comp ? 2048 : 16384) / TT;
     cudaError_t e;
-    if (a.mu) e = comp ? launch_ts<true, true>(P, st) : launch_ts<false, true>(P, st);
+    P.rope = RopeDev{};
+    if (a.rope_pos) {
+        P.rope.pos = a.rope_pos;
+        rope_frequencies(a.rope_base_src, d, P.rope.f_src);
+        rope_frequencies(a.rope_base_tgt, d, P.rope.f_tgt);
+        P.rope.same = (a.rope_base_src == a.rope_base_tgt) ? 1 : 0;
+        e = comp ? launch_ts<true, false, true>(P, st) : launch_ts<false, false, true>(P, st);
+    } else if (a.mu) e = comp ? launch_ts<true, true>(P, st) : launch_ts<false, true>(P, st);
     else e = comp ? launch_ts<true, false>(P, st) : launch_ts<false, false>(P, st);
     if (e == cudaSuccess) count_launch();
     return e;
