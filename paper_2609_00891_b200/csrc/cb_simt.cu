@@ -280,6 +280,8 @@ __global__ void __launch_bounds__(SOLVE_THREADS, 1) k_ridge_solve(const SolveArg
         // one warp per row (coalesced, no divisions); the global loads of a row are issued together before any
         // shared-memory store so that they overlap
         constexpr int MAXV = 5;                            // ceil(129 / 32)
+        // four rows in flight per warp (36 loads per lane): the phase is bound by load latency, L2 or DRAM
+#pragma unroll 4
         for (int i = warp; i < n; i += nwarps) {
             const int rsi = tri_row_start(i);
             float gv[MAXV], cv[MAXV];
