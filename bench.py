@@ -351,8 +351,8 @@ def main():
             "tflops": alg_flops * tok_launch / 1e12 / (acc_avg / 1e3),
             "tensor_frac_of_burst": alg_flops * tok_launch / 1e12 / (acc_avg / 1e3) / peaks["bf16_tflops"]}
     if args.workload == WORKLOAD:
-        # DRAM traffic of one launch from the ncu capture of an 8,192-token launch of the same shapes (summary:
-        # profiles/k_accum_ts_qwen14b_32b_8192tok.md), scaled: the per-token part x tokens + the read-modify-write of
+        # DRAM traffic of one launch from the ncu capture of an 8,192-token launch of the same shapes (summarised
+        # under profiles/), scaled: the per-token part x tokens + the read-modify-write of
         # the partial slots per split, which does not grow with tokens
         n_splits = cb.cb_token_splits(prob)
         roof["traffic"] = TRAFFIC_DRAM_BYTES_PER_TOKEN * tok_launch + TRAFFIC_DRAM_BYTES_PER_SPLIT * n_splits
