@@ -39,7 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         subprocess.check_call(cmd)
         objs.append(obj)
     tmp = LIB + ".tmp.%d" % os.getpid()
-    subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs + ["-cudart", "static"])
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs + ["-cudart", "static"])
     os.replace(tmp, LIB)
     return LIB
 
