@@ -37,7 +37,7 @@ typedef enum cb_status {
     CB_ERR_WORKSPACE = 4,    /* workspace smaller than cb_workspace_bytes() or not 256-byte aligned         */
     CB_ERR_CUDA = 5,         /* a CUDA runtime/driver call failed (includes "no device")                    */
     CB_ERR_NOT_PD = 6,       /* cb_check_info: at least one ridge system had a non-positive pivot           */
-    CB_ERR_TIMEOUT = 7,      /* cb_device_status: a bounded device-side wait ran out                        */
+    CB_ERR_TIMEOUT = 7,      /* cb_device_status / cb_last_device_status: a bounded device-side wait ran out */
     CB_ERR_STATIC_LIMIT = 8  /* cb_stats_build_static: the problem needs more scratch than the built-in buffer  */
 } cb_status;
 
@@ -61,6 +61,8 @@ typedef enum cb_status {
  *     (bf16*)k + j*stride_layer + t*stride_token + g*stride_head + c          (strides in elements)
  * and likewise for V.  Channels are contiguous.  This covers the paper's index order K_{j,t,g} stored as
  * [L][T][H][d] as well as [L][H][T][d].  k and v must be 16-byte aligned and every stride a multiple of 8.
+ * A stride of 0 (a broadcast view, e.g. one head expanded to several) is accepted only on a dimension of size 1;
+ * otherwise the call returns CB_ERR_UNSUPPORTED.  The same holds for the output strides of the apply calls.
  */
 typedef struct cb_kv_view {
     const void *k;
@@ -95,7 +97,7 @@ const char *cb_status_string(cb_status s);
 /*
  * Default head match.  Layer: nearest relative depth, j(l) = floor((2 l (Ls-1) + (Lt-1)) / (2 (Lt-1)))
  * (0 if Lt == 1); head: a(h) = floor(h*Hs/Ht), the identity when both models expose the same number of KV
- * groups (Section 3.2: "the natural assignment is a(h) = h").  Host arrays of length Lt and Ht.
+ * groups (Section 3.2).  Host arrays of length Lt and Ht.
  */
 cb_status cb_head_map_nearest(int32_t Ls, int32_t Hs, int32_t Lt, int32_t Ht,
                               int32_t *src_layer, int32_t *src_head);
@@ -116,8 +118,8 @@ cb_status cb_workspace_bytes(const cb_problem *prob, size_t *bytes);
 /*
  * The number of token splits the statistics calls will use for this problem (Section 3.4: partial statistics
  * per bounded block of observations, then a fixed reduction): prob->n_splits if it is positive, else the count in
- * 1..8 that balances the persistent blocks' units (map, split) over the SMs against the cost of one more set
- * of partial slots per split.  Host only; *n_splits receives the count.
+ * 1..8 that balances the persistent blocks' units (map, split) over the current device's SMs (148 if there is no
+ * device to ask) against the cost of one more set of partial slots per split.  Host only; *n_splits receives the count.
  */
 cb_status cb_token_splits(const cb_problem *prob, int32_t *n_splits);
 
@@ -396,6 +398,24 @@ cb_status cb_rank_layers(const float *scores, int32_t Lt, int32_t Ls, int32_t k,
 cb_status cb_device_status(cb_ctx *ctx, void *stream);
 
 /*
+ * The same for the entry points that take no context (cb_apply, cb_apply_rope, cb_apply_multilayer,
+ * cb_fullhead_stats_accumulate, cb_multilayer_stats_accumulate, cb_stats_build_static): their kernels record a
+ * time-out in a status word that belongs to the library (one per device).  Synchronises the stream, returns
+ * CB_ERR_TIMEOUT if any such kernel on the current device gave up since the last call (the outputs of that call are
+ * then incomplete) and clears the word; CB_OK otherwise.  The paper has no counterpart: error reporting only.
+ */
+cb_status cb_last_device_status(void *stream);
+
+/*
+ * TEST HOOK, not for production use (the paper has no counterpart).  Affects every later launch of this process:
+ * poll_limit > 0 shortens the number of polls after which a bounded device-side wait gives up (0 restores the
+ * default of 2^22); starve_producer != 0 makes the source-tile producer of the statistics kernel (d = 128) and of
+ * the apply kernel issue no copies at all, so that every consumer's bounded wait runs out, the blocks tear down by
+ * themselves and the status word reads CB_ERR_TIMEOUT.  Nothing faults, traps or spins without a limit.
+ */
+cb_status cb_test_hooks(uint32_t poll_limit, int32_t starve_producer);
+
+/*
  * Statistics of ONE batch of rows without any device allocation by anybody (the paper has no counterpart: this
  * entry point exists for deployment, not for the method).  It is for callers that cannot obtain scratch memory:
  * a serving process that gave all device memory to its own pool at start-up, an engine plug-in whose enqueue
@@ -411,11 +431,12 @@ cb_status cb_device_status(cb_ctx *ctx, void *stream);
  *   - Limit: n_splits * n_maps * (2 d^2 + 2 d + 4) * 4 bytes plus ~1 KB must fit in the buffer (e.g. 120 maps
  *     of d = 128 with one split); larger problems return CB_ERR_STATIC_LIMIT and nothing is enqueued.
  *   - The first call on each device looks up the buffer's device address (with that device current); make
- *     that first call outside any stream capture.
+ *     that first call outside any stream capture.  Every call also copies the two head tables of `prob` from
+ *     host memory to the device on `stream`.
  *   - All calls on a device share the one buffer, which keeps the previous call's contents; each call clears
  *     what it needs on its stream first.  Two calls whose work overlaps on the GPU (different streams, no
  *     ordering between them) race on the buffer: order them.
- *   - There is no context, so a device-side time-out cannot be reported through cb_device_status.
+ *   - There is no context: a device-side time-out shows in cb_last_device_status.
  */
 #define CB_STATIC_SCRATCH_MAX_BYTES (16u << 20)
 cb_status cb_stats_build_static(const cb_problem *prob, const cb_kv_view *src, const cb_kv_view *tgt,

@@ -32,6 +32,7 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_stats_accumulate_centered", "cb_stats_reduce_centered", "cb_ridge_solve_centered",
            "cb_stats_accumulate_rope", "cb_rope_rotate", "cb_apply_rope",
            "cb_means_energy", "cb_probe_r2", "cb_probe_scores", "cb_rank_layers",
+           "cb_last_device_status", "cb_test_hooks",
            "cb_launch_count")
 
 
@@ -569,6 +570,14 @@ def cb_apply_multilayer(prob: FullHeadProblem, src_head, Wb: torch.Tensor, src_k
 
 def cb_device_status(ctx: Context, stream=None) -> None:
     _check(lib().cb_device_status(ctx.handle, _stream_ptr(stream)), "cb_device_status")
+
+
+def cb_last_device_status(stream=None) -> None:
+    _check(lib().cb_last_device_status(_stream_ptr(stream)), "cb_last_device_status")
+
+
+def cb_test_hooks(poll_limit: int = 0, starve_producer: bool = False) -> None:
+    _check(lib().cb_test_hooks(ctypes.c_uint32(poll_limit), ctypes.c_int32(1 if starve_producer else 0)), "cb_test_hooks")
 
 
 def cb_launch_count() -> int:

@@ -2,6 +2,7 @@
 from __future__ import annotations
 
 import glob
+from concurrent.futures import ThreadPoolExecutor
 import os
 import subprocess
 import sys
@@ -28,7 +29,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    objs = []
+    objs, cmds = [], []
     for src in sources():
         obj = os.path.join(CSRC, os.path.basename(src)[:-3] + ".o")
         cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -36,8 +37,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
-        subprocess.check_call(cmd)
+        cmds.append(cmd)
         objs.append(obj)
+    # one nvcc per translation unit, side by side (the files are independent)
+    with ThreadPoolExecutor(max_workers=min(len(cmds), os.cpu_count() or 1)) as pool:
+        list(pool.map(subprocess.check_call, cmds))
     tmp = LIB + ".tmp.%d" % os.getpid()
     subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs + ["-cudart", "static"])
     os.replace(tmp, LIB)

@@ -237,7 +237,8 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
         for (int i = 0; i < 2; ++i) { mbar_init(&accfull[i], 1); mbar_init(&accempty[i], C::DRAIN_WARPS); }
         mbar_init(redfull, C::FOLD_WARPS);
         mbar_init(reddone, C::FOLD_WARPS);
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = (int)P.a.poll_limit;
         mbar_fence_init();
         tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
         tma_prefetch_desc(&P.tgt_k); tma_prefetch_desc(&P.tgt_v);
@@ -775,30 +776,17 @@ bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long l
     return r == CUDA_SUCCESS;
 }
 
-static int sm_count()
-{
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
-}
-
 template <int D, bool COMP, bool FH = false, bool CEN = false, bool ROPE = false>
 static cudaError_t launch_tc(const TcParams &P, cudaStream_t st)
 {
     using C = TcCfg<D, COMP, FH, ROPE>;
-    static bool attr = false;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_accum_tc<D, COMP, FH, CEN, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+    static bool attr[MAX_DEVICES] = {};
+    {
+        cudaError_t e = opt_in_smem(k_accum_tc<D, COMP, FH, CEN, ROPE>, (size_t)((int)C::SMEM_BYTES), attr);
         if (e != cudaSuccess) return e;
-        attr = true;
     }
     const int n_units = FH ? 2 * P.a.Lt * (P.fh.per_head ? P.a.Ht : 1) * (P.fh.NG + P.fh.NC) : 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
-    const int grid = n_units < sm_count() ? n_units : sm_count();
+    const int grid = n_units < device_sm_count() ? n_units : device_sm_count();
     k_accum_tc<D, COMP, FH, CEN, ROPE><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }

@@ -159,7 +159,8 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
         mbar_init(accempty, C::DRAIN_WARPS);
         mbar_init(redfull, C::FOLD_WARPS);
         mbar_init(reddone, 4);
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = (int)P.a.poll_limit;
         mbar_fence_init();
         tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
         tma_prefetch_desc(&P.tgt_k); tma_prefetch_desc(&P.tgt_v);
@@ -176,7 +177,7 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
 
     if (warp == 0) {
         // ================================ X producer (one thread) ================================
-        if (lane == 0) {
+        if (lane == 0 && !a.starve) {       // starve (test hook): no source tile is ever requested
             UnitIter cur;
             cur.start(a, n_units, n_maps, n_tiles);
             Ring<C::NS> st;
@@ -551,30 +552,17 @@ teardown:
     }
 }
 
-int ts_sm_count()
-{
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
-}
-
 template <bool COMP, bool CEN, bool ROPE = false>
 cudaError_t launch_ts(const TsParams &P, cudaStream_t st)
 {
     using C = TsCfg<COMP>;
-    static bool attr = false;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_accum_ts<COMP, CEN, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+    static bool attr[MAX_DEVICES] = {};
+    {
+        cudaError_t e = opt_in_smem(k_accum_ts<COMP, CEN, ROPE>, (size_t)((int)C::SMEM_BYTES), attr);
         if (e != cudaSuccess) return e;
-        attr = true;
     }
     const int n_units = 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
-    const int grid = n_units < ts_sm_count() ? n_units : ts_sm_count();
+    const int grid = n_units < device_sm_count() ? n_units : device_sm_count();
     k_accum_ts<COMP, CEN, ROPE><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }

@@ -34,7 +34,7 @@ static Layout workspace_layout(int Lt, int Ht, int d, int n_splits)
     return L;
 }
 
-static cb_status check_problem(const cb_problem *p)
+cb_status check_problem(const cb_problem *p)
 {
     if (!p || !p->src_layer || !p->src_head) return CB_ERR_INVALID_ARG;
     if (p->Ls <= 0 || p->Hs <= 0 || p->Lt <= 0 || p->Ht <= 0 || p->ds <= 0 || p->dt <= 0) return CB_ERR_INVALID_ARG;
@@ -56,7 +56,7 @@ static cb_status check_problem(const cb_problem *p)
 static int splits_of(const cb_problem *p)
 {
     if (p->n_splits > 0) return p->n_splits;
-    const long long n_maps = 2ll * p->Lt * p->Ht, sms = 148;
+    const long long n_maps = 2ll * p->Lt * p->Ht, sms = device_sm_count();
     int best = 1;
     double best_cost = 0.0;
     for (int s = 1; s <= 8; ++s) {
@@ -67,7 +67,7 @@ static int splits_of(const cb_problem *p)
     return best;
 }
 
-static cb_status check_view(const cb_kv_view *v, int L, int H, int d)
+cb_status check_view(const cb_kv_view *v, int L, int H, int d)
 {
     if (!v) return CB_ERR_INVALID_ARG;
     if (v->n_layers != L || v->n_heads != H || v->head_dim != d) return CB_ERR_INVALID_ARG;
@@ -78,7 +78,28 @@ static cb_status check_view(const cb_kv_view *v, int L, int H, int d)
     if (((uintptr_t)v->k | (uintptr_t)v->v) & 15) return CB_ERR_INVALID_ARG;
     if (v->stride_layer < 0 || v->stride_token <= 0 || v->stride_head < 0) return CB_ERR_INVALID_ARG;
     if ((v->stride_layer | v->stride_token | v->stride_head) & 7) return CB_ERR_INVALID_ARG;
+    // a broadcast (stride 0) over more than one layer or head cannot be described to the tile copies
+    if ((L > 1 && v->stride_layer == 0) || (H > 1 && v->stride_head == 0)) return CB_ERR_UNSUPPORTED;
     return CB_OK;
+}
+
+// Output strides of the apply calls: same rules as a view's.
+cb_status check_out_strides(int Lt, int Ht, int64_t sl, int64_t st, int64_t sh)
+{
+    if (sl < 0 || st <= 0 || sh < 0) return CB_ERR_INVALID_ARG;
+    if ((sl | st | sh) & 7) return CB_ERR_INVALID_ARG;
+    if ((Lt > 1 && sl == 0) || (Ht > 1 && sh == 0)) return CB_ERR_UNSUPPORTED;
+    return CB_OK;
+}
+
+// Status word, poll limit and test hooks of a launch.
+template <class Args>
+static void fill_launch_state(Args &a)
+{
+    if (!a.status) a.status = library_status_word();
+    const TestHooks h = test_hooks();
+    a.poll_limit = h.poll_limit;
+    a.starve = h.starve;
 }
 
 }  // namespace cb
@@ -280,6 +301,7 @@ static cb_status accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const cb_kv
     a.compensated = (P.flags & CB_FLAG_COMPENSATED) ? 1 : 0;
     a.mu = centred ? mu : nullptr;
     if (rope) { a.rope_pos = rope->pos; a.rope_base_src = rope->base_src; a.rope_base_tgt = rope->base_tgt; }
+    fill_launch_state(a);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = (P.flags & CB_FLAG_SIMT) ? launch_accum_simt(a, ctx->d, st)
                                              : launch_accum_tc(a, ctx->d, src, tgt, st);
@@ -640,8 +662,8 @@ static cb_status apply_impl(const cb_problem *prob, const float *Wb, const cb_kv
     if (src_cache->n_tokens == 0) return CB_OK;
     if (!Wb || !tgt_k || !tgt_v) return CB_ERR_INVALID_ARG;
     if ((((uintptr_t)tgt_k | (uintptr_t)tgt_v | (uintptr_t)Wb) & 15)) return CB_ERR_INVALID_ARG;
-    if (t_stride_layer < 0 || t_stride_token <= 0 || t_stride_head < 0) return CB_ERR_INVALID_ARG;
-    if ((t_stride_layer | t_stride_token | t_stride_head) & 7) return CB_ERR_INVALID_ARG;
+    s = check_out_strides(prob->Lt, prob->Ht, t_stride_layer, t_stride_token, t_stride_head);
+    if (s != CB_OK) return s;
 
     ApplyArgs a;
     a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src_cache->k), static_cast<const __nv_bfloat16 *>(src_cache->v),
@@ -656,6 +678,7 @@ static cb_status apply_impl(const cb_problem *prob, const float *Wb, const cb_kv
     for (int l = 0; l < prob->Lt; ++l) a.src_layer[l] = prob->src_layer[l];
     for (int h = 0; h < prob->Ht; ++h) a.src_head[h] = prob->src_head[h];
     if (rope) { a.rope_pos = rope->pos; a.rope_base_src = rope->base_src; a.rope_base_tgt = rope->base_tgt; }
+    fill_launch_state(a);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = (prob->flags & CB_FLAG_SIMT) ? launch_apply_simt(a, prob->ds, st)
                                                  : launch_apply_tc(a, prob->ds, src_cache, st);
@@ -756,6 +779,7 @@ cb_status cb_fullhead_stats_accumulate(const cb_fullhead_problem *prob, const cb
     a.n_tokens = (int)src->n_tokens;
     a.Lt = prob->Lt; a.Ht = prob->Ht; a.n_splits = 1;
     a.src_layer = nullptr; a.src_head = nullptr; a.slots = nullptr; a.status = nullptr; a.compensated = 0;
+    fill_launch_state(a);
     FullHeadArgs f;
     f.G = G; f.C = C;
     f.layer_sets = static_cast<const int *>(workspace);
@@ -820,6 +844,7 @@ cb_status cb_multilayer_stats_accumulate(const cb_fullhead_problem *prob, const 
     a.n_tokens = (int)src->n_tokens;
     a.Lt = prob->Lt; a.Ht = prob->Ht; a.n_splits = 1;
     a.src_layer = nullptr; a.src_head = nullptr; a.slots = nullptr; a.status = nullptr; a.compensated = 0;
+    fill_launch_state(a);
     FullHeadArgs f;
     f.G = G; f.C = C;
     f.layer_sets = static_cast<const int *>(workspace);
@@ -860,8 +885,8 @@ cb_status cb_apply_multilayer(const cb_fullhead_problem *prob, const int32_t *sr
     if (src_cache->n_tokens == 0) return CB_OK;
     if (!Wb || !tgt_k || !tgt_v) return CB_ERR_INVALID_ARG;
     if ((((uintptr_t)tgt_k | (uintptr_t)tgt_v | (uintptr_t)Wb) & 15)) return CB_ERR_INVALID_ARG;
-    if (t_stride_layer < 0 || t_stride_token <= 0 || t_stride_head < 0) return CB_ERR_INVALID_ARG;
-    if ((t_stride_layer | t_stride_token | t_stride_head) & 7) return CB_ERR_INVALID_ARG;
+    s = check_out_strides(prob->Lt, prob->Ht, t_stride_layer, t_stride_token, t_stride_head);
+    if (s != CB_OK) return s;
     size_t need = 0;
     cb_apply_multilayer_workspace_bytes(prob, &need);
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return CB_ERR_WORKSPACE;
@@ -876,6 +901,7 @@ cb_status cb_apply_multilayer(const cb_fullhead_problem *prob, const int32_t *sr
     std::memset(a.src_layer, 0, sizeof a.src_layer);
     std::memset(a.src_head, 0, sizeof a.src_head);
     for (int h = 0; h < prob->Ht; ++h) a.src_head[h] = src_head[h];
+    fill_launch_state(a);
     if (launch_apply_ml_tc(a, prob->ds, prob->k, prob->layer_sets, src_cache, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         cudaGetLastError();
         return CB_ERR_CUDA;

@@ -13,8 +13,8 @@
 //                     in tensor memory.
 //   epilogue warps    tensor memory -> registers, + bias, -> bf16 into a shared-memory tile -> one TMA store
 //                     (coalesced 256-byte rows, rows past the end clipped); fp32 output is stored directly.
-// Every wait is bounded; a wait that runs out makes the block tear down (nothing else is reported: this call has
-// no context to carry a status word).
+// Every wait is bounded; a wait that runs out makes the block set the library's status word (cb_last_device_status)
+// and tear down.
 #include <cudaTypedefs.h>
 
 #include <cuda_fp16.h>
@@ -139,7 +139,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         mbar_init(wfree, 1);
         mbar_init(bfree, C::EPI_WARPS);
         for (int i = 0; i < C::NO; ++i) { mbar_init(&owritten[i], C::EPI_WARPS); mbar_init(&ofree[i], 1); }
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = (int)P.a.poll_limit;
         mbar_fence_init();
         tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
         tma_prefetch_desc(&P.out_k); tma_prefetch_desc(&P.out_v);
@@ -152,7 +153,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
 
     if (warp == 0) {
         // ================================ producer (one thread) ================================
-        if (lane == 0) {
+        if (lane == 0 && !a.starve) {       // starve (test hook): no source tile is ever requested
             ApIter cur;
             cur.start(n_units, n_maps, n_tiles, P.n_splits);
             Ring<C::NS> st;
@@ -486,6 +487,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
 teardown:
     __syncwarp();
     if (*abort_flag) {
+        if (tid == 0 && a.status) atomicExch(a.status, DEV_TIMEOUT);
+        // give copies that may still be in flight time to land before the block's shared memory is released
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
     }
     tc_fence_before();
@@ -496,30 +499,17 @@ teardown:
     }
 }
 
-static int ap_sm_count()
-{
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
-}
-
 template <int D, bool ROPE>
 static cudaError_t launch_ap(const ApParams &P, cudaStream_t st)
 {
     using C = ApCfg<D>;
-    static bool attr = false;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_apply_tc<D, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+    static bool attr[MAX_DEVICES] = {};
+    {
+        cudaError_t e = opt_in_smem(k_apply_tc<D, ROPE>, (size_t)((int)C::SMEM_BYTES), attr);
         if (e != cudaSuccess) return e;
-        attr = true;
     }
     const int n_units = 2 * P.a.Lt * P.a.Ht * P.n_splits;
-    const int grid = n_units < ap_sm_count() ? n_units : ap_sm_count();
+    const int grid = n_units < device_sm_count() ? n_units : device_sm_count();
     k_apply_tc<D, ROPE><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }
@@ -531,7 +521,7 @@ cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cu
     const int TT = 128;
     const int n_maps = 2 * a.Lt * a.Ht;
     const int n_tiles = (a.n_tokens + TT - 1) / TT;
-    int splits = (n_maps >= ap_sm_count()) ? 1 : (ap_sm_count() + n_maps - 1) / n_maps;
+    int splits = (n_maps >= device_sm_count()) ? 1 : (device_sm_count() + n_maps - 1) / n_maps;
     if (splits > n_tiles) splits = n_tiles;
     if (splits < 1) splits = 1;
     P.n_splits = splits;
@@ -647,7 +637,8 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
         for (int i = 0; i < C::NACC; ++i) { mbar_init(&accfull[i], 1); mbar_init(&accempty[i], C::EPI_WARPS); }
         mbar_init(owritten, C::EPI_WARPS);
         mbar_init(ofree, 1);
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = (int)P.a.poll_limit;
         mbar_fence_init();
         tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
         tma_prefetch_desc(&P.out_k); tma_prefetch_desc(&P.out_v);
@@ -802,6 +793,8 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
 ml_teardown:
     __syncwarp();
     if (*abort_flag) {
+        if (tid == 0 && a.status) atomicExch(a.status, DEV_TIMEOUT);
+        // give copies that may still be in flight time to land before the block's shared memory is released
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
     }
     tc_fence_before();
@@ -821,16 +814,15 @@ template <int D>
 static cudaError_t launch_ml(const MlParams &P, const float *Wb, uint8_t *wsplit, cudaStream_t st)
 {
     using C = MlCfg<D>;
-    static bool attr = false;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_apply_ml_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+    static bool attr[MAX_DEVICES] = {};
+    {
+        cudaError_t e = opt_in_smem(k_apply_ml_tc<D>, (size_t)((int)C::SMEM_BYTES), attr);
         if (e != cudaSuccess) return e;
-        attr = true;
     }
     const int n_maps = 2 * P.a.Lt * P.a.Ht;
     k_w_split<D><<<n_maps * P.k, 256, 0, st>>>(Wb, wsplit, P.k);
     const int n_units = n_maps * P.n_splits;
-    const int grid = n_units < ap_sm_count() ? n_units : ap_sm_count();
+    const int grid = n_units < device_sm_count() ? n_units : device_sm_count();
     k_apply_ml_tc<D><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }
@@ -844,7 +836,7 @@ cudaError_t launch_apply_ml_tc(const ApplyArgs &a, int d, int k, const int *laye
     const int TT = 128;
     const int n_maps = 2 * a.Lt * a.Ht;
     const int n_tiles = (a.n_tokens + TT - 1) / TT;
-    int splits = (n_maps >= ap_sm_count()) ? 1 : (ap_sm_count() + n_maps - 1) / n_maps;
+    int splits = (n_maps >= device_sm_count()) ? 1 : (device_sm_count() + n_maps - 1) / n_maps;
     if (splits > n_tiles) splits = n_tiles;
     if (splits < 1) splits = 1;
     P.n_splits = splits;

@@ -197,7 +197,8 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
         mbar_init(accempty, C::DRAIN_WARPS);
         mbar_init(redfull, C::FOLD_WARPS);
         mbar_init(reddone, C::FOLD_WARPS);
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = (int)P.a.poll_limit;
         mbar_fence_init();
         tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
         tma_prefetch_desc(&P.tgt_k); tma_prefetch_desc(&P.tgt_v);
@@ -523,29 +524,16 @@ __global__ void k_mirror_lower(float *__restrict__ G, int pf)
     }
 }
 
-static int gr_sm_count()
-{
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
-}
-
 template <int D>
 static cudaError_t launch_gr(const GrParams &P, int n_units, cudaStream_t st)
 {
     using C = GrCfg<D>;
-    static bool attr = false;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_gram2_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+    static bool attr[MAX_DEVICES] = {};
+    {
+        cudaError_t e = opt_in_smem(k_gram2_tc<D>, (size_t)((int)C::SMEM_BYTES), attr);
         if (e != cudaSuccess) return e;
-        attr = true;
     }
-    const int grid = n_units < gr_sm_count() ? n_units : gr_sm_count();
+    const int grid = n_units < device_sm_count() ? n_units : device_sm_count();
     k_gram2_tc<D><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }

@@ -37,8 +37,10 @@ struct AccumArgs {
     const int *src_layer;  // device [Lt]
     const int *src_head;   // device [Ht]
     float *slots;          // device [n_splits][n_maps][slot_floats]
-    int *status;           // device status word
+    int *status;           // device status word (the context's, else the library's own: library_status_word())
     int compensated;
+    unsigned poll_limit = 1u << 22;   // polls after which a bounded device-side wait gives up
+    int starve = 0;                   // test hook: the source-tile producer issues nothing, so the waits run out
     // Two-pass centred construction: device [n_maps][2d + 1] = mu_x, mu_y, s_w per map; null for the one-pass path.
     // When set, the weighted operand is w (x - mu_x) and the slot's s_x entries receive the sum of the ROUNDED
     // weighted operand (the exact correction term of the reduction), s_y stays zero.
@@ -77,6 +79,9 @@ struct ApplyArgs {
     // Rotary embedding at the boundary (key maps): device [n_tokens] positions, or null for the ordinary apply.
     const int *rope_pos = nullptr;
     double rope_base_src = 0.0, rope_base_tgt = 0.0;
+    int *status = nullptr;            // device status word (the library's own: library_status_word())
+    unsigned poll_limit = 1u << 22;   // as in AccumArgs
+    int starve = 0;
 };
 
 // Full-head contrast statistics: outputs and device tables (see cb_fullhead_stats_accumulate).
@@ -123,5 +128,35 @@ cudaError_t launch_rope_rotate(void *k, int L, int H, int d, long long T, long l
                                const int *pos, double base, int inverse, cudaStream_t stream);
 
 void count_launch(int n = 1);
+
+// Host-side argument checks shared by the entry points (status codes of the C ABI).
+cb_status check_problem(const cb_problem *p);
+cb_status check_view(const cb_kv_view *v, int L, int H, int d);
+
+// ---- per-device host state ---------------------------------------------------------------------------
+constexpr int MAX_DEVICES = 64;
+// SM count of the current device (asked once per device; 148 if there is no device to ask).
+int device_sm_count();
+// Device address, on the current device, of the library's own status word: kernels launched without a context
+// record a device-side time-out there and cb_last_device_status reads it.  Null if the lookup failed.
+int *library_status_word();
+// Test hooks (cb_test_hooks): poll limit of the bounded waits and the starved-producer switch for later launches.
+struct TestHooks { unsigned poll_limit; int starve; };
+TestHooks test_hooks();
+// Opt a kernel in to more than 48 KB of dynamic shared memory, once per device.
+template <class K>
+inline cudaError_t opt_in_smem(K kernel, size_t bytes, bool (&done)[MAX_DEVICES])
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    if (!done[dev]) {
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+        if (e != cudaSuccess) return e;
+        done[dev] = true;
+    }
+    return cudaSuccess;
+}
 
 }  // namespace cb

@@ -169,11 +169,10 @@ cudaError_t launch_reduce_centered(const float *slots, int n_splits, int n_maps,
                                    cudaStream_t st)
 {
     const size_t smem = sizeof(float) * ((size_t)d * (2 * d + 1) + 2 * d + 4 + 2 * d);
-    static bool attr = false;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_reduce_centered, cudaFuncAttributeMaxDynamicSharedMemorySize, 140 * 1024);
+    static bool attr[MAX_DEVICES] = {};
+    {
+        cudaError_t e = opt_in_smem(k_reduce_centered, (size_t)(140 * 1024), attr);
         if (e != cudaSuccess) return e;
-        attr = true;
     }
     k_reduce_centered<<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, d, mu, A, B);
     cudaError_t e = cudaGetLastError();

@@ -45,21 +45,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 }
 
 // Bounded wait.  Returns false if the limit ran out or another thread of the block already gave up
-// (*abort_flag != 0); the caller then leaves its loop and the block tears down.  After `fast_polls` failed polls
-// the thread sleeps `sleep_ns` between polls: every poll is a shared-memory transaction, and a block full of
-// spinning threads slows down the shared-memory pipe for the threads that do the work.
+// (abort_flag[0] != 0); the caller then leaves its loop and the block tears down.  abort_flag points at two ints in
+// shared memory: [0] the block's abort flag, [1] the poll limit of this launch (kPollLimitDefault unless the host set
+// a shorter one), read only once the fast polls are used up.  After `fast_polls` failed polls the thread sleeps
+// `sleep_ns` between polls: every poll is a shared-memory transaction, and a block full of spinning threads slows
+// down the shared-memory pipe for the threads that do the work.
+constexpr uint32_t kPollLimitDefault = 1u << 22;
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
                                           uint32_t fast_polls = 1u << 14, uint32_t sleep_ns = 64)
 {
-    constexpr uint32_t kPollMax = 1u << 22;
-    for (uint32_t i = 0; i < kPollMax; ++i) {
+    for (uint32_t i = 0; i < fast_polls; ++i)
         if (mbar_try_wait(bar, parity)) return true;
-        if (i >= fast_polls) {
-            if ((i & 63) == 0 && *abort_flag) return false;
-            __nanosleep(sleep_ns);
-        }
+    const uint32_t limit = (uint32_t)abort_flag[1];
+    for (uint32_t i = fast_polls; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63) == 0 && abort_flag[0]) return false;
+        __nanosleep(sleep_ns);
     }
-    *abort_flag = 1;
+    abort_flag[0] = 1;
     return false;
 }
 

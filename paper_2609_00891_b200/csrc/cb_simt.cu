@@ -176,11 +176,10 @@ __global__ void __launch_bounds__(1024) k_reduce(const float *__restrict__ slots
 cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, float *G, float *C, cudaStream_t st)
 {
     const size_t smem = sizeof(float) * ((size_t)d * (2 * d + 1) + 2 * d + 4);
-    static bool attr = false;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_reduce, cudaFuncAttributeMaxDynamicSharedMemorySize, 140 * 1024);
+    static bool attr[MAX_DEVICES] = {};
+    {
+        cudaError_t e = opt_in_smem(k_reduce, (size_t)(140 * 1024), attr);
         if (e != cudaSuccess) return e;
-        attr = true;
     }
     k_reduce<<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, d, G, C);
     cudaError_t e = cudaGetLastError();
@@ -495,11 +494,10 @@ static cudaError_t launch_solve_any(const float *G, const float *C, const float 
     for (int i = 0; i < 16; ++i) a.lambdas[i] = i < n_lambda ? lambdas[i] : 0.f;
     const int p = d + 1;
     const size_t smem = sizeof(double) * ((size_t)tri_row_start(p) + (size_t)p * d);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_ridge_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+    static bool attr[MAX_DEVICES] = {};
+    {
+        cudaError_t e = opt_in_smem(k_ridge_solve, (size_t)(220 * 1024), attr);
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     k_ridge_solve<<<n_maps * n_lambda, SOLVE_THREADS, smem, st>>>(a);
     cudaError_t e = cudaGetLastError();

@@ -310,11 +310,10 @@ template <int MODE, int NT>
 static cudaError_t launch_tile(const LgArgs &a, int J, dim3 grid, cudaStream_t st)
 {
     constexpr size_t smem = sizeof(double) * (LNB * LPAD + LNB * (NT + 2));
-    static bool attr = false;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(k_lg_tile<MODE, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static bool attr[MAX_DEVICES] = {};
+    {
+        cudaError_t e = opt_in_smem(k_lg_tile<MODE, NT>, (size_t)((int)smem), attr);
         if (e != cudaSuccess) return e;
-        attr = true;
     }
     k_lg_tile<MODE, NT><<<grid, 256, smem, st>>>(a, J);
     return cudaSuccess;
@@ -330,11 +329,8 @@ template <bool FWD>
 static void launch_diag(const LgArgs &a, int J, cudaStream_t st)
 {
     const size_t smem = sizeof(double) * LNB * (size_t)a.d;
-    static bool attr = false;
-    if (!attr) {
-        cudaFuncSetAttribute(k_lg_diag<FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(double) * LNB * 128));
-        attr = true;
-    }
+    static bool attr[MAX_DEVICES] = {};
+    opt_in_smem(k_lg_diag<FWD>, sizeof(double) * LNB * 128, attr);
     k_lg_diag<FWD><<<a.nsys, 128, smem, st>>>(a, J);
 }
 

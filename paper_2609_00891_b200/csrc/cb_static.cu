@@ -6,12 +6,11 @@
 
 namespace cb {
 
-// Built-in scratch: partial slots, the head-match tables and a status word.  Every GPU that loads the library
+// Built-in scratch: partial slots and the head-match tables.  Every GPU that loads the library
 // holds this array until the process exits.
 static constexpr size_t STATIC_SCRATCH_BYTES = (size_t)CB_STATIC_SCRATCH_MAX_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
 
-static constexpr int MAX_DEVICES = 64;
 static std::mutex g_static_mutex;
 static unsigned char *g_static_ptr[MAX_DEVICES];   // device address of the array, per device, filled on first use
 
@@ -43,39 +42,33 @@ extern "C" cb_status cb_stats_build_static(const cb_problem *prob, const cb_kv_v
                                            int64_t w_stride_layer, int64_t w_stride_head,
                                            float *G, float *C, void *stream)
 {
-    if (!prob || !prob->src_layer || !prob->src_head || !src || !tgt || !G || !C) return CB_ERR_INVALID_ARG;
-    if (prob->Ls <= 0 || prob->Hs <= 0 || prob->Lt <= 0 || prob->Ht <= 0) return CB_ERR_INVALID_ARG;
-    if (prob->ds != prob->dt || (prob->ds != 64 && prob->ds != 128)) return CB_ERR_UNSUPPORTED;
-    if (prob->n_splits < 0 || prob->n_splits > 64) return CB_ERR_INVALID_ARG;
-    for (int l = 0; l < prob->Lt; ++l)
-        if (prob->src_layer[l] < 0 || prob->src_layer[l] >= prob->Ls) return CB_ERR_INVALID_ARG;
-    for (int h = 0; h < prob->Ht; ++h)
-        if (prob->src_head[h] < 0 || prob->src_head[h] >= prob->Hs) return CB_ERR_INVALID_ARG;
+    // the same host-side checks as cb_create + cb_stats_accumulate
+    cb_status cs = check_problem(prob);
+    if (cs != CB_OK) return cs;
+    if (!G || !C) return CB_ERR_INVALID_ARG;
     const int d = prob->ds;
-    if (src->n_layers != prob->Ls || src->n_heads != prob->Hs || src->head_dim != d) return CB_ERR_INVALID_ARG;
-    if (tgt->n_layers != prob->Lt || tgt->n_heads != prob->Ht || tgt->head_dim != d) return CB_ERR_INVALID_ARG;
+    cs = check_view(src, prob->Ls, prob->Hs, d);
+    if (cs != CB_OK) return cs;
+    cs = check_view(tgt, prob->Lt, prob->Ht, d);
+    if (cs != CB_OK) return cs;
     const int64_t T = src->n_tokens;
-    if (T <= 0 || T != tgt->n_tokens || T >= (1ll << 31)) return CB_ERR_INVALID_ARG;
-    if (!src->k || !src->v || !tgt->k || !tgt->v || !w_k || !w_v) return CB_ERR_INVALID_ARG;
-    if (((uintptr_t)src->k | (uintptr_t)src->v | (uintptr_t)tgt->k | (uintptr_t)tgt->v) & 15) return CB_ERR_INVALID_ARG;
-    if ((src->stride_layer | src->stride_token | src->stride_head | tgt->stride_layer | tgt->stride_token | tgt->stride_head) & 7)
-        return CB_ERR_INVALID_ARG;
-    if (src->stride_token <= 0 || tgt->stride_token <= 0 || w_stride_layer < 0 || w_stride_head < 0) return CB_ERR_INVALID_ARG;
+    if (T <= 0 || T != tgt->n_tokens) return CB_ERR_INVALID_ARG;
+    if (!w_k || !w_v || w_stride_layer < 0 || w_stride_head < 0) return CB_ERR_INVALID_ARG;
+    if (((uintptr_t)w_k | (uintptr_t)w_v) & 3) return CB_ERR_INVALID_ARG;
 
-    // layout inside the built-in array: [slots][tables][status]
+    // layout inside the built-in array: [slots][tables]
     const int n_splits = prob->n_splits > 0 ? prob->n_splits : 1;
     const size_t n_maps = 2 * (size_t)prob->Lt * prob->Ht;
     const size_t slots_bytes = (size_t)n_splits * n_maps * slot_floats(d) * sizeof(float);
     const size_t tab_off = (slots_bytes + 255) / 256 * 256;
-    const size_t status_off = (tab_off + sizeof(int) * ((size_t)prob->Lt + prob->Ht) + 255) / 256 * 256;
-    if (status_off + 256 > STATIC_SCRATCH_BYTES) return CB_ERR_STATIC_LIMIT;
+    const size_t end_off = (tab_off + sizeof(int) * ((size_t)prob->Lt + prob->Ht) + 255) / 256 * 256;
+    if (end_off + 256 > STATIC_SCRATCH_BYTES) return CB_ERR_STATIC_LIMIT;
 
     unsigned char *base = nullptr;
     if (static_scratch_address(&base) != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the array keeps whatever the previous call left: everything that must start at zero is cleared here
     cudaError_t e = cudaMemsetAsync(base, 0, slots_bytes, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(base + status_off, 0, 256, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(base + tab_off, prob->src_layer, sizeof(int) * (size_t)prob->Lt, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(base + tab_off + sizeof(int) * (size_t)prob->Lt, prob->src_head, sizeof(int) * (size_t)prob->Ht,
@@ -93,7 +86,9 @@ extern "C" cb_status cb_stats_build_static(const cb_problem *prob, const cb_kv_v
     a.src_layer = reinterpret_cast<const int *>(base + tab_off);
     a.src_head = a.src_layer + prob->Lt;
     a.slots = reinterpret_cast<float *>(base);
-    a.status = reinterpret_cast<int *>(base + status_off);
+    a.status = library_status_word();     // a device-side time-out shows in cb_last_device_status
+    const TestHooks hk = test_hooks();
+    a.poll_limit = hk.poll_limit; a.starve = hk.starve;
     a.compensated = (prob->flags & CB_FLAG_COMPENSATED) ? 1 : 0;
     e = (prob->flags & CB_FLAG_SIMT) ? launch_accum_simt(a, d, st) : launch_accum_tc(a, d, src, tgt, st);
     if (e == cudaSuccess) e = launch_reduce(a.slots, n_splits, (int)n_maps, d, G, C, st);

@@ -43,6 +43,14 @@ def test_apply_argument_errors_are_reported_before_any_launch():
     assert _apply(prob, _view(4, 2, 128, 64), out=0x3008) == cb.CB_ERR_INVALID_ARG   # misaligned output
     assert _apply(prob, _view(4, 2, 128, 64), dtype=7) == cb.CB_ERR_INVALID_ARG      # unknown output type
     assert _apply(prob, _view(4, 2, 128, 1 << 31)) == cb.CB_ERR_UNSUPPORTED          # too many rows for one call
+    # a broadcast view (stride 0 over several heads or layers, e.g. an expanded one-head cache) cannot be tiled
+    assert _apply(prob, _view(4, 2, 128, 64, sh=0)) == cb.CB_ERR_UNSUPPORTED
+    assert _apply(prob, _view(4, 2, 128, 64, sl=0)) == cb.CB_ERR_UNSUPPORTED
+    assert _apply(prob, _view(4, 2, 128, 64), strides=(64 * 2 * 128, 2 * 128, 0)) == cb.CB_ERR_UNSUPPORTED   # output too
+    assert _apply(prob, _view(4, 2, 128, 64), strides=(0, 2 * 128, 128)) == cb.CB_ERR_UNSUPPORTED
+    sl1, sh1 = cb.cb_head_map_nearest(1, 1, 6, 2)
+    one = cb.Problem(1, 1, 128, 6, 2, 128, sl1, sh1)
+    assert _apply(one, _view(1, 1, 128, 64, sh=0, sl=0)) == cb.CB_ERR_CUDA           # size-1 dimensions: any stride; passes the checks
     assert cb.cb_launch_count() == before
 
 
@@ -73,6 +81,28 @@ def test_without_a_device_the_path_fails_loudly():
     assert "CUDA" in cb.status_string(cb.CB_ERR_CUDA)
     with pytest.raises(cb.CbError):
         cb.cb_create(prob, workspace=torch.zeros(16, dtype=torch.uint8))              # workspace too small
+
+
+def test_static_entry_point_shares_the_argument_checks():
+    sl, sh = cb.cb_head_map_nearest(4, 2, 6, 2)
+    prob = cb.Problem(4, 2, 128, 6, 2, 128, sl, sh)
+
+    def call(vs, vt, wk=0x100, wv=0x100):
+        return cb.lib().cb_stats_build_static(ctypes.byref(prob.c), ctypes.byref(vs), ctypes.byref(vt), ctypes.c_void_p(wk),
+                                              ctypes.c_void_p(wv), ctypes.c_int64(2 * 64), ctypes.c_int64(64),
+                                              ctypes.c_void_p(0x200), ctypes.c_void_p(0x300), ctypes.c_void_p(0))
+    ok_s, ok_t = _view(4, 2, 128, 64), _view(6, 2, 128, 64)
+    assert call(ok_s, ok_t, wk=0x102) == cb.CB_ERR_INVALID_ARG                         # weights must be 4-byte aligned
+    assert call(_view(4, 2, 128, 64, sh=-128), ok_t) == cb.CB_ERR_INVALID_ARG          # negative stride
+    assert call(_view(4, 2, 128, 64, sh=0), ok_t) == cb.CB_ERR_UNSUPPORTED             # broadcast over two heads
+    assert call(ok_s, _view(6, 2, 128, 32)) == cb.CB_ERR_INVALID_ARG                   # token counts differ
+    assert call(ok_s, ok_t) == cb.CB_ERR_CUDA                                          # passes the checks; no device here
+
+
+def test_status_calls_without_a_device():
+    assert cb.lib().cb_last_device_status(ctypes.c_void_p(0)) == cb.CB_ERR_CUDA
+    assert cb.lib().cb_test_hooks(ctypes.c_uint32(1 << 12), 1) == cb.CB_OK             # host state only
+    assert cb.lib().cb_test_hooks(ctypes.c_uint32(0), 0) == cb.CB_OK
 
 
 def test_workspace_and_static_limits():

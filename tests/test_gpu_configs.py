@@ -14,38 +14,34 @@ DEV = "cuda"
 TOL = 1e-3
 
 
-def _sampled_oracle(wl, sl, sh, layers, chunks_host):
-    """Oracle statistics of all heads, K and V, of the sampled target layers: a reduced problem with only those layers."""
+def _sampled_oracle_chunk(sl, sh, layers, ch):
+    """Oracle statistics of one chunk for all heads, K and V, of the sampled target layers: a reduced problem that
+    holds only those layers (and the source layers they read)."""
     src_layers = sorted(set(int(sl[l]) for l in layers))
     remap = np.array([src_layers.index(int(sl[l])) for l in layers], np.int32)
-    G = C = None
-    for ch in chunks_host:
-        g, c = oracle.stats_traces(bits(ch["src_k"][src_layers]), bits(ch["src_v"][src_layers]),
-                                   bits(ch["tgt_k"][layers]), bits(ch["tgt_v"][layers]),
-                                   ch["w_k"][layers].numpy(), ch["w_v"][layers].numpy(), remap, sh)
-        G, C = (g, c) if G is None else (G + g, C + c)
-    idx = [(comp * wl.Lt + l) * wl.Ht + h for comp in range(2) for l in layers for h in range(wl.Ht)]
-    return G, C, idx
+    return oracle.stats_traces(bits(ch["src_k"][src_layers].cpu()), bits(ch["src_v"][src_layers].cpu()),
+                               bits(ch["tgt_k"][layers].cpu()), bits(ch["tgt_v"][layers].cpu()),
+                               ch["w_k"][layers].cpu().numpy(), ch["w_v"][layers].cpu().numpy(), remap, sh)
 
 
-def _run_config(name, layers, max_chunks=None):
+def _run_config(name, layers, chunks=None):
+    """Streams the given chunks (all by default) of a workload through one context; the oracle's statistics of the
+    sampled layers are summed chunk by chunk beside it (statistics are additive), so that no chunk is kept."""
     wl = synth.workload(name)
     sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh)
     ctx = cb.cb_create(prob, device=DEV)
     law = synth.map_law(wl, DEV)
-    src_layers = sorted(set(int(sl[l]) for l in layers))
-    n_chunks = wl.n_chunks if max_chunks is None else min(max_chunks, wl.n_chunks)
-    host, n_tok = [], 0
-    for c in range(n_chunks):
+    chunks = list(range(wl.n_chunks)) if chunks is None else list(chunks)
+    Go = Co = None
+    n_tok, sizes = 0, []
+    for c in chunks:
         ch = synth.make_chunk(wl, c, sl, sh, device=DEV, law=law)
         cb.cb_stats_accumulate(ctx, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], ch["w_k"], ch["w_v"])
-        # host copy of the sampled layers only
-        host.append({
-            "src_k": _dense_layers(ch["src_k"], src_layers, wl.Ls), "src_v": _dense_layers(ch["src_v"], src_layers, wl.Ls),
-            "tgt_k": _dense_layers(ch["tgt_k"], layers, wl.Lt), "tgt_v": _dense_layers(ch["tgt_v"], layers, wl.Lt),
-            "w_k": _dense_layers(ch["w_k"], layers, wl.Lt), "w_v": _dense_layers(ch["w_v"], layers, wl.Lt)})
+        g, co = _sampled_oracle_chunk(sl, sh, layers, ch)
+        Go, Co = (g, co) if Go is None else (Go + g, Co + co)
         n_tok += ch["n_tokens"]
+        sizes.append(ch["n_tokens"])
         del ch
     p, d = wl.d + 1, wl.d
     G = torch.empty(wl.n_maps, p, p, device=DEV)
@@ -53,34 +49,22 @@ def _run_config(name, layers, max_chunks=None):
     n = cb.cb_stats_reduce(ctx, G, C)
     cb.cb_device_status(ctx)
     assert n == n_tok
-    return wl, sl, sh, prob, G, C, n, host
+    idx = [(comp * wl.Lt + l) * wl.Ht + h for comp in range(2) for l in layers for h in range(wl.Ht)]
+    return wl, sl, sh, prob, G, C, n, (Go, Co, idx), sizes
 
 
-def _dense_layers(t, keep, L):
-    """Host copy of the kept layers only, still addressable by the original layer index."""
-    return _Compact(t, keep)
-
-
-class _Compact:
-    """Only the kept layers, addressable by their original layer index (for tensors too large to hold densely)."""
-
-    def __init__(self, t, keep):
-        self.keep = list(keep)
-        self.data = torch.stack([t[j].cpu() for j in self.keep])
-
-    def __getitem__(self, layers):
-        return self.data[[self.keep.index(int(j)) for j in layers]]
-
-
-@pytest.mark.parametrize("name,layers,max_chunks", [
+@pytest.mark.parametrize("name,layers,chunks", [
     ("qwen8b_14b", [0, 4, 5, 39], None),               # config 1 in full: 36 -> 40 layers, 64 x 1024 tokens; layers 4, 5 share a source layer
-    ("ragged_long", [0, 1, 2, 63], 2),                 # config 4, first two ragged chunks of 12 sequences
+    # config 4: the first two ragged chunks of 12 sequences and the LAST one (8 sequences: the short tail); none of
+    # the three ends on a multiple of the 128-token tile, so every chunk boundary falls inside a tile
+    ("ragged_long", [0, 1, 2, 63], [0, 1, 41]),
 ])
-def test_config_statistics_and_fit_on_sampled_maps(name, layers, max_chunks):
-    wl, sl, sh, prob, G, C, n, host = _run_config(name, layers, max_chunks)
+def test_config_statistics_and_fit_on_sampled_maps(name, layers, chunks):
+    wl, sl, sh, prob, G, C, n, (Go, Co, idx), sizes = _run_config(name, layers, chunks)
     if name == "qwen8b_14b":
         assert sl[4] == sl[5]
-    Go, Co, idx = _sampled_oracle(wl, sl, sh, layers, host)
+    else:
+        assert wl.n_chunks == 42 and len(wl.chunk_seq_lens(41)) == 8 and all(t % 128 for t in sizes)
     Gs, Cs = G.cpu().numpy()[idx], C.cpu().numpy()[idx]
     eg, ec = max_rel_fro_per_map(Gs, Go), max_rel_fro_per_map(Cs, Co)
     print("%s (%d tokens): %d sampled maps, max rel err G %.2e C %.2e" % (name, n, len(idx), eg, ec))
@@ -117,15 +101,48 @@ def test_config_statistics_and_fit_on_sampled_maps(name, layers, max_chunks):
         assert rel_fro(gk, ok) <= 3e-3                               # vs unrounded fp64: the bf16 floor (~1.7e-3)
 
 
+def test_config2_full_build_on_sampled_maps():
+    """Config 2 as the benchmark runs it: all ten 51,200-token calls into one context, one reduce, the solve at the three
+    lambdas; 64 sampled maps (target layers 0, 1, 2, 63: first, last, and a pair sharing one source layer; all heads;
+    K and V) against the oracle on all 512,000 tokens."""
+    layers = [0, 1, 2, 63]
+    wl, sl, sh, prob, G, C, n, (Go, Co, idx), sizes = _run_config("qwen14b_32b_500", layers)
+    assert n == 512000 and sizes == [51200] * 10 and sl[1] == sl[2]
+    Gs, Cs = G.cpu().numpy()[idx], C.cpu().numpy()[idx]
+    eg, ec = max_rel_fro_per_map(Gs, Go), max_rel_fro_per_map(Cs, Co)
+    d = wl.d
+    # the tensor cores' fp32 accumulation truncates: on the all-positive diagonal of G the result is systematically
+    # low, in proportion to the tokens summed in tensor memory between drains (at most 16,384)
+    dg = np.einsum("mii->mi", Gs)[:, :d].astype(np.float64)
+    do = np.einsum("mii->mi", Go)[:, :d]
+    bias = float(np.mean((dg - do) / do))
+    print("config 2, 512,000 tokens, 64 sampled maps: max rel err G %.2e C %.2e; signed mean rel err of diag(G) %.2e"
+          % (eg, ec, bias))
+    assert eg <= TOL and ec <= TOL
+    assert -2.0e-4 < bias < 0.0
+    p = d + 1
+    lams = list(wl.lambdas)
+    Wb = torch.empty(len(lams), wl.n_maps, p, d, device=DEV)
+    info = torch.empty(len(lams), wl.n_maps, dtype=torch.int32, device=DEV)
+    cb.cb_ridge_solve(G, C, n, lams, 0, Wb, info)
+    cb.cb_check_info(info)
+    for li, lam in enumerate(lams):
+        To, io = oracle.ridge_solve(Go, Co, n, lam)
+        ew = max_rel_fro_per_map(Wb[li].cpu().numpy()[idx], To)
+        print("lambda %g: max rel err of fitted maps %.2e" % (lam, ew))
+        assert not io.any() and ew <= TOL
+
+
 def test_config3_fullhead_sampled_group():
-    """Config 3 shapes (4 source layers x 8 heads -> 4097-wide regressor), first 2,048 tokens, one (comp, layer) group
-    against the oracle (the full group costs the oracle 70 GFLOP of plain fp64)."""
+    """Config 3 shapes (4 source layers x 8 heads -> 4097-wide regressor), 8,192 tokens, one (comp, layer) group
+    against the oracle (the group costs the oracle 0.35 TFLOP of plain fp64) at the stated 1e-3, pooled over the
+    group and for its worst 128 x 128 block."""
     wl = synth.workload("qwen14b_32b_500")
     sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     sets = cb.cb_fullhead_layer_sets(wl.Ls, wl.Lt, 4)
     assert np.array_equal(sets, oracle.fullhead_layer_sets(wl.Ls, wl.Lt, 4))
     import dataclasses
-    small = dataclasses.replace(wl, seq_lens=(1024, 1024), seqs_per_chunk=2)
+    small = dataclasses.replace(wl, seq_lens=(1024,) * 8, seqs_per_chunk=8)
     ch = synth.make_chunk(small, 0, sl, sh, device=DEV)
     prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
     pf, d = prob.pf, wl.d
@@ -134,12 +151,24 @@ def test_config3_fullhead_sampled_group():
     C = torch.zeros(2, wl.Lt, wl.Ht, pf, d, device=DEV)
     wk, wv = ch["w_k"][:, 0].contiguous(), ch["w_v"][:, 0].contiguous()
     cb.cb_fullhead_stats_accumulate(prob, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], wk, wv, G, C)
-    torch.cuda.synchronize()
+    cb.cb_last_device_status()
     comp, l = 1, 17
     Go, Co = oracle.fullhead_stats(bits(ch["src_v"].cpu()), bits(ch["tgt_v"].cpu()), wv[l].cpu().numpy(), l, sets[l])
-    eg, ec = rel_fro(G[comp, l].cpu().numpy(), Go), rel_fro(C[comp, l].cpu().numpy(), Co)
-    print("config 3, (V, layer 17), 2048 tokens: rel err G %.2e C %.2e" % (eg, ec))
-    assert eg <= 2e-3 and ec <= 2e-3                                   # 2,048 tokens per entry: the plain bf16 fold averages out like 1/sqrt(tokens)
+    Gg, Cg = G[comp, l].cpu().numpy(), C[comp, l].cpu().numpy()
+    eg, ec = rel_fro(Gg, Go), rel_fro(Cg, Co)
+    F = (pf - 1) // d
+    blk_g = max(rel_fro(Gg[i * d:(i + 1) * d, j * d:(j + 1) * d], Go[i * d:(i + 1) * d, j * d:(j + 1) * d])
+                for i in range(F) for j in range(F))
+    blk_c = max(rel_fro(Cg[h, i * d:(i + 1) * d], Co[h, i * d:(i + 1) * d]) for h in range(wl.Ht) for i in range(F))
+    print("config 3, (V, layer 17), 8192 tokens: rel err G %.2e C %.2e; worst 128 x 128 block G %.2e C %.2e"
+          % (eg, ec, blk_g, blk_c))
+    assert eg <= TOL and ec <= TOL
+    assert max(rel_fro(Cg[h], Co[h]) for h in range(wl.Ht)) <= TOL        # every map's own C
+    # A block between two unrelated heads is a sum of terms of random sign: its value and the rounding error of the
+    # bf16 weighted operand (rms 1.1e-3 per term) both grow like sqrt(tokens), so that block's relative error stays
+    # near 1.1e-3 at any size; the blocks that carry signal (diagonal blocks, C of the matched head) fall like
+    # 1/sqrt(tokens) and set the matrix norm.
+    assert blk_g <= 2.5e-3 and blk_c <= 2.5e-3
     assert torch.isfinite(G).all() and torch.isfinite(C).all()
     # every other group must have been filled too (property check): the weight totals
     sw = torch.stack([wk.double().sum(-1), wv.double().sum(-1)]).cpu().numpy()

@@ -62,6 +62,50 @@ def test_multilayer_statistics_and_fit(name, k, flags):
         #  the solver itself is checked on the GPU's own statistics above)
 
 
+def test_k8_fit_against_the_oracle_fit():
+    """The paper's operating point k = 8 (Section 4.1) with enough rows per regressor column (21,504 rows for width
+    1025, n > 20 P): the FITTED map from the GPU's statistics and solver against the oracle's fit from the oracle's own
+    statistics."""
+    wl = synth.workload("deep_fit")
+    k = 8
+    sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    sets = oracle.fullhead_layer_sets(wl.Ls, wl.Lt, k)
+    ch = synth.make_chunk(wl, 0, sl, sh)
+    n_tok = ch["n_tokens"]
+    d = wl.d
+    P = k * d + 1
+    assert n_tok >= 20 * P
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, d, wl.Lt, wl.Ht, d, sets)
+    G = torch.zeros(wl.n_maps, P, P, device=DEV)
+    C = torch.zeros(wl.n_maps, P, d, device=DEV)
+    t = {k_: v.to(DEV) for k_, v in ch.items() if torch.is_tensor(v)}
+    cb.cb_multilayer_stats_accumulate(prob, sh, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], t["w_k"], t["w_v"], G, C)
+    cb.cb_last_device_status()
+    lam = 1e-2
+    ws = torch.empty(cb.cb_ridge_solve_large_workspace_bytes(P, d, wl.n_maps), dtype=torch.uint8, device=DEV)
+    Wb = torch.full((1, wl.n_maps, P, d), float("nan"), device=DEV)
+    info = torch.full((1, wl.n_maps), -1, dtype=torch.int32, device=DEV)
+    cb.cb_ridge_solve_large(G, C, n_tok, [lam], 0, Wb, info, ws)
+    cb.cb_check_info(info)
+    Gc, Cc, Wc = G.cpu().numpy(), C.cpu().numpy(), Wb[0].cpu().numpy()
+    for m in (1, wl.n_maps - 2):
+        comp, l, h = m // (wl.Lt * wl.Ht), (m // wl.Ht) % wl.Lt, m % wl.Ht
+        Go, Co = oracle.multilayer_stats(bits(ch["src_v" if comp else "src_k"]), bits(ch["tgt_v" if comp else "tgt_k"]),
+                                         (ch["w_v"] if comp else ch["w_k"])[l, h].contiguous().numpy(), l, h, int(sh[h]), sets[l])
+        To, io = oracle.ridge_solve_general(Go, Co, n_tok, lam)
+        eg, ec, ew = rel_fro(Gc[m], Go), rel_fro(Cc[m], Co), rel_fro(Wc[m], To)
+        # conditioning of the system after Jacobi scaling (the rounding errors of the statistics are relative per
+        # entry, so the scaled system is the one that amplifies them)
+        Gl = Go.copy()
+        Gl[np.arange(P - 1), np.arange(P - 1)] += lam * Go[P - 1, P - 1] / n_tok
+        s = 1.0 / np.sqrt(np.diag(Gl))
+        ev = np.linalg.eigvalsh(Gl * s[:, None] * s[None, :])
+        kappa = ev[-1] / ev[0]
+        print("k=8 fit, map %d: rel err G %.2e C %.2e fitted map %.2e; scaled condition number %.1f" % (m, eg, ec, ew, kappa))
+        assert io == 0 and eg <= 1e-3 and ec <= 1e-3
+        assert ew <= 1e-3
+
+
 def test_large_solver_agrees_with_the_single_head_solver():
     g = torch.Generator(device=DEV).manual_seed(1)
     n_maps, d = 7, 128

@@ -6,8 +6,10 @@ whose pool owns all device memory, a plug-in hook that must not call cudaMalloc,
 import pytest
 import torch
 
+import oracle
 from paper_2609_00891_b200 import binding as cb
 from paper_2609_00891_b200 import synth
+from util import bits, rel_fro
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -47,6 +49,11 @@ def test_static_scratch_entry_matches_regular_path_twice(name, flags):
         # same kernels, same split order: agreement far inside the 1e-3 the parity tests use
         assert ((G - G_ref).norm() / G_ref.norm()).item() <= 1e-6
         assert ((C - C_ref).norm() / C_ref.norm()).item() <= 1e-6
+        cb.cb_last_device_status()                     # no bounded wait ran out inside the call
+    # and against the oracle itself (second batch), at the tolerance of the parity tests
+    Go, Co = oracle.stats_traces(bits(b["src_k"]), bits(b["src_v"]), bits(b["tgt_k"]), bits(b["tgt_v"]),
+                                 b["w_k"].contiguous().numpy(), b["w_v"].contiguous().numpy(), sl, sh)
+    assert rel_fro(G.cpu().numpy(), Go) <= 1e-3 and rel_fro(C.cpu().numpy(), Co) <= 1e-3
 
 
 def test_static_scratch_entry_rejects_oversized_problems():
