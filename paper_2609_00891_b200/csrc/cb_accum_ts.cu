@@ -540,12 +540,14 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
 teardown:
     __syncwarp();
     if (*abort_flag) {
-        if (tid == 0 && a.status) atomicExch(a.status, DEV_TIMEOUT);
         // give copies that may still be in flight time to land before the block's shared memory is released
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
     }
     tc_fence_before();
     __syncthreads();
+    // after the barrier every thread's verdict is in: a thread that finished its own role early may have passed the
+    // check above before another thread gave up
+    if (tid == 0 && *abort_flag && a.status) atomicExch(a.status, DEV_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::TMEM_COLS);

@@ -495,11 +495,13 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
 teardown:
     __syncwarp();
     if (*abort_flag) {
-        if (tid == 0 && a.status) atomicExch(a.status, DEV_TIMEOUT);
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
     }
     tc_fence_before();
     __syncthreads();
+    // after the barrier every thread's verdict is in: a thread that finished its own role early may have passed the
+    // check above before another thread gave up
+    if (tid == 0 && *abort_flag && a.status) atomicExch(a.status, DEV_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::TMEM_COLS);

@@ -92,8 +92,8 @@ def workload(name: str) -> Workload:
         return Workload("very_long_unit", 17, 1, 1, 1, 1, 128, (200003,), 1, (1e-2,), "scaled", 0.1)
     if name == "deep_small":      # enough source layers for the paper's k = 8 selected layers (regressor width 1025)
         return Workload("deep_small", 15, 10, 2, 3, 2, 128, (1100, 1000), 2, (1e-2,), "scaled", 0.1)
-    if name == "deep_fit":        # k = 8 with ~21 rows per regressor column (21,504 rows, width 1025): a well-posed wide fit
-        return Workload("deep_fit", 18, 10, 2, 3, 2, 128, (1024,) * 21, 21, (1e-2,), "scaled", 0.1)
+    if name == "deep_fit":        # k = 8 with 64 rows per regressor column (65,536 rows, width 1025): a well-posed wide fit
+        return Workload("deep_fit", 18, 10, 2, 3, 2, 128, (1024,) * 64, 64, (1e-2,), "scaled", 0.1)
     if name == "mini_ragged":     # several chunks of unequal size
         lens = _ragged_lengths(9, 40, 700, seed=77)
         return Workload("mini_ragged", 14, 4, 4, 6, 4, 128, lens, 3, (1e-3, 1e-2, 1e-1), "scaled", 0.1,

@@ -134,15 +134,17 @@ def test_config2_full_build_on_sampled_maps():
 
 
 def test_config3_fullhead_sampled_group():
-    """Config 3 shapes (4 source layers x 8 heads -> 4097-wide regressor), 8,192 tokens, one (comp, layer) group
-    against the oracle (the group costs the oracle 0.35 TFLOP of plain fp64) at the stated 1e-3, pooled over the
-    group and for its worst 128 x 128 block."""
+    """Config 3 shapes (4 source layers x 8 heads -> 4097-wide regressor), 32,768 tokens, one (comp, layer) group
+    against the oracle (the group costs the oracle 1.4 TFLOP of plain fp64) at the stated 1e-3, pooled over the
+    group, per map, and for its worst 128 x 128 block.  31 of the 32 feature heads are unrelated to a given target
+    head, so C is mostly noise blocks at small sizes (measured 1.4e-3 at 8,192 tokens, falling like 1/sqrt(tokens);
+    the configuration itself has 204,800)."""
     wl = synth.workload("qwen14b_32b_500")
     sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     sets = cb.cb_fullhead_layer_sets(wl.Ls, wl.Lt, 4)
     assert np.array_equal(sets, oracle.fullhead_layer_sets(wl.Ls, wl.Lt, 4))
     import dataclasses
-    small = dataclasses.replace(wl, seq_lens=(1024,) * 8, seqs_per_chunk=8)
+    small = dataclasses.replace(wl, seq_lens=(1024,) * 32, seqs_per_chunk=32)
     ch = synth.make_chunk(small, 0, sl, sh, device=DEV)
     prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
     pf, d = prob.pf, wl.d
@@ -160,7 +162,7 @@ def test_config3_fullhead_sampled_group():
     blk_g = max(rel_fro(Gg[i * d:(i + 1) * d, j * d:(j + 1) * d], Go[i * d:(i + 1) * d, j * d:(j + 1) * d])
                 for i in range(F) for j in range(F))
     blk_c = max(rel_fro(Cg[h, i * d:(i + 1) * d], Co[h, i * d:(i + 1) * d]) for h in range(wl.Ht) for i in range(F))
-    print("config 3, (V, layer 17), 8192 tokens: rel err G %.2e C %.2e; worst 128 x 128 block G %.2e C %.2e"
+    print("config 3, (V, layer 17), 32768 tokens: rel err G %.2e C %.2e; worst 128 x 128 block G %.2e C %.2e"
           % (eg, ec, blk_g, blk_c))
     assert eg <= TOL and ec <= TOL
     assert max(rel_fro(Cg[h], Co[h]) for h in range(wl.Ht)) <= TOL        # every map's own C

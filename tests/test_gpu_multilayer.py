@@ -63,9 +63,12 @@ def test_multilayer_statistics_and_fit(name, k, flags):
 
 
 def test_k8_fit_against_the_oracle_fit():
-    """The paper's operating point k = 8 (Section 4.1) with enough rows per regressor column (21,504 rows for width
-    1025, n > 20 P): the FITTED map from the GPU's statistics and solver against the oracle's fit from the oracle's own
-    statistics."""
+    """The paper's operating point k = 8 (Section 4.1) with enough rows per regressor column (65,536 rows for width
+    1025; the paper fits on 128,000 positions): the FITTED map from the GPU's statistics and solver against the oracle's
+    fit from the oracle's own statistics.  Seven of the eight feature blocks are unrelated to the target here, so most
+    of C is a sum of terms of random sign whose rounding error does not average out relative to its value; the error
+    of C, and with it the fit's, falls like 1/sqrt(rows) only through the block that carries the signal (measured:
+    C 8.5e-4, fit 1.2e-3 at 21,504 rows)."""
     wl = synth.workload("deep_fit")
     k = 8
     sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
@@ -104,6 +107,7 @@ def test_k8_fit_against_the_oracle_fit():
         print("k=8 fit, map %d: rel err G %.2e C %.2e fitted map %.2e; scaled condition number %.1f" % (m, eg, ec, ew, kappa))
         assert io == 0 and eg <= 1e-3 and ec <= 1e-3
         assert ew <= 1e-3
+        assert ew <= kappa * (eg + ec)          # first-order perturbation bound of the scaled normal equations
 
 
 def test_large_solver_agrees_with_the_single_head_solver():
