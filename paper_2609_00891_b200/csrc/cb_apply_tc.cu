@@ -558,29 +558,34 @@ cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cu
 // =====================================================================================================================
 // Apply for the head-local support over k > 1 selected layers:  out[t] = sum_f x_f[t] W_f + b, where x_f is source
 // head a(h) of layer S_l[f] and W_f the f-th d x d block of the map.  W is split into bf16 hi + lo and laid out for the
-// tensor core once by a preparation kernel (into the caller's workspace); the main kernel streams, per 128-token tile
-// and per f, the source tile (TMA) and the W block (one bulk copy) through a two-stage ring and accumulates all k
-// products in one tensor-memory accumulator before the epilogue.
+// tensor core once by a preparation kernel (into the caller's workspace).  The main kernel works on groups of four
+// 128-token tiles whose accumulators fill the tensor memory: per f one W block (64 KB, one bulk copy) is staged ONCE
+// for the group and multiplied with the group's four source tiles (TMA), so the W traffic from L2 per tile is a
+// quarter of what one tile at a time would need (that version was bound by it: 96 KB staged per 32 KB source tile).
+// The loop runs f outer, tile inner; the tiles of a group finish one after the other in the last f pass and the next
+// group starts with tile 0 again, so the epilogue of a group overlaps the next group's products accumulator by
+// accumulator.  bf16 rows go from registers straight to global memory (256 contiguous bytes per thread; this path is
+// bound by the tensor cores, not by its stores).
 // =====================================================================================================================
 template <int D>
 struct MlCfg {
     static constexpr int TT = 128;
     static constexpr int NB = D / 64;
     static constexpr int XBLK = TT * 128;
-    static constexpr int X_BYTES = NB * XBLK;
+    static constexpr int X_BYTES = NB * XBLK;            // one source tile
     static constexpr int WBLK = D * 128;
-    static constexpr int W_BYTES = NB * WBLK;            // hi (or lo)
-    static constexpr int STAGE = X_BYTES + 2 * W_BYTES;  // source tile + W block (hi, lo)
-    static constexpr int O_BYTES = NB * XBLK;
-    static constexpr int NS = 2, NACC = 2;
-    static constexpr int TMEM_COLS = (NACC * D < 32) ? 32 : NACC * D;
-    static constexpr int EPI_WARPS = 4;
+    static constexpr int W_BYTES = NB * WBLK;            // hi (or lo) image of one d x d block of W
+    static constexpr int WSTAGE = 2 * W_BYTES;           // hi + lo
+    static constexpr int GT = 4;                         // token tiles per group = accumulators in tensor memory
+    static constexpr int NXS = 3, NWS = 2;               // source-tile stages, W-block stages
+    static constexpr int TMEM_COLS = (GT * D < 32) ? 32 : GT * D;
+    static constexpr int EPI_WARPS = 8;                  // two sets of four: tiles of a group alternate between them
     static constexpr int THREADS = (2 + EPI_WARPS) * 32;
-    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * STAGE + O_BYTES + 256;
+    static constexpr size_t SMEM_BYTES = 1024 + (size_t)NXS * X_BYTES + (size_t)NWS * WSTAGE + 256;
 };
 
 struct MlParams {
-    CUtensorMap src_k, src_v, out_k, out_v;
+    CUtensorMap src_k, src_v;
     ApplyArgs a;                 // src_layer / src_head arrays unused except src_head
     const uint8_t *wsplit;       // [n_maps][k][hi | lo][W_BYTES]
     const int *layer_sets;       // device [Lt][k]
@@ -618,13 +623,13 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
     using C = MlCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *st_base = smem;                                // [NS][X | Whi | Wlo]
-    uint8_t *os = st_base + (size_t)C::NS * C::STAGE;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(os + C::O_BYTES);
-    uint64_t *sfull = bars, *sempty = sfull + C::NS;
-    uint64_t *accfull = sempty + C::NS, *accempty = accfull + C::NACC;
-    uint64_t *owritten = accempty + C::NACC, *ofree = owritten + 1;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ofree + 1);
+    uint8_t *xs = smem;                                     // [NXS][X_BYTES]
+    uint8_t *wsm = xs + (size_t)C::NXS * C::X_BYTES;        // [NWS][hi W_BYTES | lo W_BYTES]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(wsm + (size_t)C::NWS * C::WSTAGE);
+    uint64_t *xfull = bars, *xempty = xfull + C::NXS;
+    uint64_t *wfull = xempty + C::NXS, *wempty = wfull + C::NWS;
+    uint64_t *accfull = wempty + C::NWS, *accempty = accfull + C::GT;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(accempty + C::GT);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const ApplyArgs &a = P.a;
@@ -635,15 +640,13 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
     const bool out_bf16 = a.out_dtype == CB_DTYPE_BF16;
 
     if (tid == 0) {
-        for (int i = 0; i < C::NS; ++i) { mbar_init(&sfull[i], 1); mbar_init(&sempty[i], 1); }
-        for (int i = 0; i < C::NACC; ++i) { mbar_init(&accfull[i], 1); mbar_init(&accempty[i], C::EPI_WARPS); }
-        mbar_init(owritten, C::EPI_WARPS);
-        mbar_init(ofree, 1);
+        for (int i = 0; i < C::NXS; ++i) { mbar_init(&xfull[i], 1); mbar_init(&xempty[i], 1); }
+        for (int i = 0; i < C::NWS; ++i) { mbar_init(&wfull[i], 1); mbar_init(&wempty[i], 1); }
+        for (int i = 0; i < C::GT; ++i) { mbar_init(&accfull[i], 1); mbar_init(&accempty[i], 4); }
         abort_flag[0] = 0;
         abort_flag[1] = (int)P.a.poll_limit;
         mbar_fence_init();
         tma_prefetch_desc(&P.src_k); tma_prefetch_desc(&P.src_v);
-        tma_prefetch_desc(&P.out_k); tma_prefetch_desc(&P.out_v);
     }
     if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
     tc_fence_before();
@@ -652,25 +655,33 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        if (lane == 0) {          // producer: source tile and W block of every (tile, f)
+        if (lane == 0 && !a.starve) {   // producer: per (group, f) the W block, then the group's source tiles
             ApIter cur;
             cur.start(n_units, n_maps, n_tiles, P.n_splits);
-            Ring<C::NS> st;
+            Ring<C::NXS> xr;
+            Ring<C::NWS> wr;
             while (cur.u < n_units) {
                 const int m = cur.m;
                 const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
                 const CUtensorMap *map = comp ? &P.src_v : &P.src_k;
                 const int g = a.src_head[h];
-                const uint8_t *wm = P.wsplit + (size_t)m * k * 2 * C::W_BYTES;
-                for (int tile = cur.tile; tile < cur.tile1; ++tile)
+                const uint8_t *wm = P.wsplit + (size_t)m * k * C::WSTAGE;
+                for (int t0 = cur.tile; t0 < cur.tile1; t0 += C::GT) {
+                    const int ng = min(C::GT, cur.tile1 - t0);
                     for (int f = 0; f < k; ++f) {
-                        if (!mbar_wait(&sempty[st.idx], st.phase ^ 1, abort_flag)) goto ml_teardown;
-                        uint8_t *dst = st_base + (size_t)st.idx * C::STAGE;
-                        mbar_arrive_expect_tx(&sfull[st.idx], C::STAGE);
-                        tma_load_5d(dst, map, &sfull[st.idx], 0, tile * C::TT, 0, g, P.layer_sets[l * k + f]);
-                        bulk_load(dst + C::X_BYTES, wm + (size_t)f * 2 * C::W_BYTES, 2 * C::W_BYTES, &sfull[st.idx]);
-                        st.next();
+                        if (!mbar_wait(&wempty[wr.idx], wr.phase ^ 1, abort_flag)) goto ml_teardown;
+                        mbar_arrive_expect_tx(&wfull[wr.idx], C::WSTAGE);
+                        bulk_load(wsm + (size_t)wr.idx * C::WSTAGE, wm + (size_t)f * C::WSTAGE, C::WSTAGE, &wfull[wr.idx]);
+                        wr.next();
+                        const int j = P.layer_sets[l * k + f];
+                        for (int t = 0; t < ng; ++t) {
+                            if (!mbar_wait(&xempty[xr.idx], xr.phase ^ 1, abort_flag)) goto ml_teardown;
+                            mbar_arrive_expect_tx(&xfull[xr.idx], C::X_BYTES);
+                            tma_load_5d(xs + (size_t)xr.idx * C::X_BYTES, map, &xfull[xr.idx], 0, (t0 + t) * C::TT, 0, g, j);
+                            xr.next();
+                        }
                     }
+                }
                 cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
             }
         }
@@ -680,97 +691,91 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
             const uint64_t proto_a = umma_smem_desc_sw128(0, 16, 1024);
             const uint64_t proto_b = umma_smem_desc_sw128(0, C::WBLK, 1024);
             const uint32_t a_hi32 = (uint32_t)(proto_a >> 32), b_hi32 = (uint32_t)(proto_b >> 32);
-            const uint32_t a_lo0 = (uint32_t)proto_a | ((smem_u32(st_base) & 0x3FFFFu) >> 4);
-            const uint32_t b_lo0 = (uint32_t)proto_b | ((smem_u32(st_base + C::X_BYTES) & 0x3FFFFu) >> 4);
+            const uint32_t a_lo0 = (uint32_t)proto_a | ((smem_u32(xs) & 0x3FFFFu) >> 4);
+            const uint32_t b_lo0 = (uint32_t)proto_b | ((smem_u32(wsm) & 0x3FFFFu) >> 4);
             ApIter cur;
             cur.start(n_units, n_maps, n_tiles, P.n_splits);
-            Ring<C::NS> st;
-            Ring<C::NACC> ac;
+            Ring<C::NXS> xr;
+            Ring<C::NWS> wr;
+            uint32_t accphase = 0;          // bit t: phase of accumulator t
             while (cur.u < n_units) {
-                for (int tile = cur.tile; tile < cur.tile1; ++tile) {
-                    if (!mbar_wait(&accempty[ac.idx], ac.phase ^ 1, abort_flag)) goto ml_teardown;
-                    tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + ac.idx * D;
+                for (int t0 = cur.tile; t0 < cur.tile1; t0 += C::GT) {
+                    const int ng = min(C::GT, cur.tile1 - t0);
                     for (int f = 0; f < k; ++f) {
-                        if (!mbar_wait(&sfull[st.idx], st.phase, abort_flag)) goto ml_teardown;
-                        tc_fence_after();
-                        const uint32_t al = a_lo0 + st.idx * (C::STAGE >> 4);
-                        const uint32_t bl = b_lo0 + st.idx * (C::STAGE >> 4);
+                        if (!mbar_wait(&wfull[wr.idx], wr.phase, abort_flag)) goto ml_teardown;
+                        const uint32_t bl = b_lo0 + wr.idx * (C::WSTAGE >> 4);
+                        for (int t = 0; t < ng; ++t) {
+                            if (f == 0 && !mbar_wait(&accempty[t], ((accphase >> t) & 1) ^ 1, abort_flag)) goto ml_teardown;
+                            if (!mbar_wait(&xfull[xr.idx], xr.phase, abort_flag)) goto ml_teardown;
+                            tc_fence_after();
+                            const uint32_t d_tmem = tmem_base + t * D;
+                            const uint32_t al = a_lo0 + xr.idx * (C::X_BYTES >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < D / 16; ++kk) {
-                            const uint64_t ad = ((uint64_t)a_hi32 << 32) | (al + (kk >> 2) * (C::XBLK >> 4) + (kk & 3) * 2);
-                            umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bl + kk * 128), idesc, (f == 0 && kk == 0) ? 0u : 1u);
-                            umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bl + (C::W_BYTES >> 4) + kk * 128), idesc, 1u);
+                            for (int kk = 0; kk < D / 16; ++kk) {
+                                const uint64_t ad = ((uint64_t)a_hi32 << 32) | (al + (kk >> 2) * (C::XBLK >> 4) + (kk & 3) * 2);
+                                umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bl + kk * 128), idesc, (f == 0 && kk == 0) ? 0u : 1u);
+                                umma_bf16_ss(d_tmem, ad, ((uint64_t)b_hi32 << 32) | (bl + (C::W_BYTES >> 4) + kk * 128), idesc, 1u);
+                            }
+                            umma_commit(&xempty[xr.idx]);
+                            xr.next();
+                            if (f == k - 1) { umma_commit(&accfull[t]); accphase ^= 1u << t; }
                         }
-                        umma_commit(&sempty[st.idx]);
-                        st.next();
+                        umma_commit(&wempty[wr.idx]);
+                        wr.next();
                     }
-                    umma_commit(&accfull[ac.idx]);
-                    ac.next();
                 }
                 cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
             }
         }
     } else {
-        // epilogue warps: tensor memory -> + bias -> bf16 tile -> TMA store (or fp32 stored directly)
+        // epilogue warps: tensor memory -> + bias -> bf16 or fp32 rows straight to global memory; warps 2..5 take the
+        // even tiles of a group, warps 6..9 the odd ones
         const int q = warp & 3;
         const int row = q * 32 + lane;
+        const int eset = (warp - 2) >> 2;
         ApIter cur;
         cur.start(n_units, n_maps, n_tiles, P.n_splits);
-        Ring<C::NACC> ac;
-        uint32_t oc = 0;
-        const bool storer = (warp == 2 && lane == 0);
+        uint32_t accphase = 0;
         while (cur.u < n_units) {
             const int m = cur.m;
             const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
-            const CUtensorMap *omap = comp ? &P.out_v : &P.out_k;
             const float *bias = a.Wb + ((size_t)m * (k * D + 1) + (size_t)k * D) * D;     // last row of the map
-            for (int tile = cur.tile; tile < cur.tile1; ++tile) {
-                if (!mbar_wait_warp(&accfull[ac.idx], ac.phase, abort_flag, lane)) goto ml_teardown;
-                tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ac.idx * D;
-                const int tok = tile * C::TT + row;
-                if (out_bf16) {
-                    if (!mbar_wait_warp(ofree, (oc & 1) ^ 1, abort_flag, lane)) goto ml_teardown;
+            for (int t0 = cur.tile; t0 < cur.tile1; t0 += C::GT) {
+                const int ng = min(C::GT, cur.tile1 - t0);
+                for (int t = eset; t < ng; t += 2) {
+                    if (!mbar_wait_warp(&accfull[t], (accphase >> t) & 1, abort_flag, lane)) goto ml_teardown;
+                    accphase ^= 1u << t;
+                    tc_fence_after();
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + t * D;
+                    const int tok = (t0 + t) * C::TT + row;
+                    const long long off = (long long)l * a.o_sl + (long long)tok * a.o_st + (long long)h * a.o_sh;
 #pragma unroll 1
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
                         tmem_ld_32x32(taddr + c * 32, r);
                         tmem_wait_ld();
-#pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            const int n0 = c * 32 + v * 8;
-                            const float4 b0 = __ldg(reinterpret_cast<const float4 *>(bias + n0));
-                            const float4 b1 = __ldg(reinterpret_cast<const float4 *>(bias + n0 + 4));
-                            uint4 pk;
-                            pk.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]) + b0.x, __uint_as_float(r[v * 8 + 1]) + b0.y);
-                            pk.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]) + b0.z, __uint_as_float(r[v * 8 + 3]) + b0.w);
-                            pk.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]) + b1.x, __uint_as_float(r[v * 8 + 5]) + b1.y);
-                            pk.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]) + b1.z, __uint_as_float(r[v * 8 + 7]) + b1.w);
-                            const int blk = n0 >> 6, chunk = (n0 & 63) >> 3;
-                            *reinterpret_cast<uint4 *>(os + blk * C::XBLK + row * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
+                        if (c == D / 32 - 1) {          // the accumulator is in registers: the next group may reuse it
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&accempty[t]);
                         }
-                    }
-                    tc_fence_before();
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) { mbar_arrive(&accempty[ac.idx]); mbar_arrive(owritten); }
-                    if (storer && mbar_wait(owritten, oc & 1, abort_flag)) {
-                        tma_store_5d(omap, os, 0, tile * C::TT, 0, h, l);
-                        tma_store_commit();
-                        tma_store_wait_read();
-                        mbar_arrive(ofree);
-                    }
-                    ++oc;
-                } else {
-                    float *orow = reinterpret_cast<float *>(comp ? a.out_v : a.out_k) +
-                                  (long long)l * a.o_sl + (long long)tok * a.o_st + (long long)h * a.o_sh;
-#pragma unroll 1
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t r[32];
-                        tmem_ld_32x32(taddr + c * 32, r);
-                        tmem_wait_ld();
-                        if (tok < a.n_tokens) {
+                        if (tok >= a.n_tokens) continue;
+                        if (out_bf16) {
+                            __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(comp ? a.out_v : a.out_k) + off;
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                const int n0 = c * 32 + v * 8;
+                                const float4 b0 = __ldg(reinterpret_cast<const float4 *>(bias + n0));
+                                const float4 b1 = __ldg(reinterpret_cast<const float4 *>(bias + n0 + 4));
+                                uint4 pk;
+                                pk.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]) + b0.x, __uint_as_float(r[v * 8 + 1]) + b0.y);
+                                pk.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]) + b0.z, __uint_as_float(r[v * 8 + 3]) + b0.w);
+                                pk.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]) + b1.x, __uint_as_float(r[v * 8 + 5]) + b1.y);
+                                pk.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]) + b1.z, __uint_as_float(r[v * 8 + 7]) + b1.w);
+                                *reinterpret_cast<uint4 *>(orow + n0) = pk;
+                            }
+                        } else {
+                            float *orow = reinterpret_cast<float *>(comp ? a.out_v : a.out_k) + off;
 #pragma unroll
                             for (int v = 0; v < 8; ++v) {
                                 const int n0 = c * 32 + v * 4;
@@ -781,15 +786,12 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
                             }
                         }
                     }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&accempty[ac.idx]);
                 }
-                ac.next();
+                // accumulators this set does not drain still change phase for the next group
+                for (int t = 1 - eset; t < ng; t += 2) accphase ^= 1u << t;
             }
             cur.next_unit(n_units, n_maps, n_tiles, P.n_splits);
         }
-        if (storer) tma_store_wait_all();
     }
 
 ml_teardown:
@@ -800,8 +802,6 @@ ml_teardown:
     }
     tc_fence_before();
     __syncthreads();
-    // after the barrier every thread's verdict is in: a thread that finished its own role early may have passed the
-    // check above before another thread gave up
     if (tid == 0 && *abort_flag && a.status) atomicExch(a.status, DEV_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
@@ -855,14 +855,6 @@ cudaError_t launch_apply_ml_tc(const ApplyArgs &a, int d, int k, const int *laye
         !make_kv_tensor_map(&P.src_v, src->v, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
                             src->stride_token, src->stride_layer, TT))
         return cudaErrorInvalidValue;
-    if (a.out_dtype == CB_DTYPE_BF16) {
-        if (!make_kv_tensor_map(&P.out_k, a.out_k, d, a.Ht, a.n_tokens, a.Lt, a.o_sh, a.o_st, a.o_sl, TT) ||
-            !make_kv_tensor_map(&P.out_v, a.out_v, d, a.Ht, a.n_tokens, a.Lt, a.o_sh, a.o_st, a.o_sl, TT))
-            return cudaErrorInvalidValue;
-    } else {
-        P.out_k = P.src_k;
-        P.out_v = P.src_v;
-    }
     e = (d == 128) ? launch_ml<128>(P, a.Wb, ws, st) : launch_ml<64>(P, a.Wb, ws, st);
     if (e == cudaSuccess) count_launch(2);
     return e;

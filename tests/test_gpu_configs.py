@@ -164,14 +164,69 @@ def test_config3_fullhead_sampled_group():
     blk_c = max(rel_fro(Cg[h, i * d:(i + 1) * d], Co[h, i * d:(i + 1) * d]) for h in range(wl.Ht) for i in range(F))
     print("config 3, (V, layer 17), 32768 tokens: rel err G %.2e C %.2e; worst 128 x 128 block G %.2e C %.2e"
           % (eg, ec, blk_g, blk_c))
-    assert eg <= TOL and ec <= TOL
-    assert max(rel_fro(Cg[h], Co[h]) for h in range(wl.Ht)) <= TOL        # every map's own C
     # A block between two unrelated heads is a sum of terms of random sign: its value and the rounding error of the
-    # bf16 weighted operand (rms 1.1e-3 per term) both grow like sqrt(tokens), so that block's relative error stays
-    # near 1.1e-3 at any size; the blocks that carry signal (diagonal blocks, C of the matched head) fall like
-    # 1/sqrt(tokens) and set the matrix norm.
-    assert blk_g <= 2.5e-3 and blk_c <= 2.5e-3
+    # bf16 weighted operand (relative 2^-9 .. 2^-8 per term) both grow like sqrt(tokens), so that block's relative
+    # error stays at a few 1e-3 at any size; only the blocks that carry signal (diagonal blocks of G, C of the matched
+    # head) improve like 1/sqrt(tokens).  31 of the 32 blocks of a target head's C are of the first kind in these
+    # traces, so C reaches 1e-3 later than G: 1.4e-3 at 8,192 tokens, 1.1e-3 here, below 1e-3 at the configuration's
+    # 204,800 tokens (next test).
+    assert eg <= TOL and ec <= 1.5e-3
+    assert max(rel_fro(Cg[h], Co[h]) for h in range(wl.Ht)) <= 1.5e-3     # every map's own C
+    assert blk_g <= 5e-3 and blk_c <= 5e-3
     assert torch.isfinite(G).all() and torch.isfinite(C).all()
     # every other group must have been filled too (property check): the weight totals
     sw = torch.stack([wk.double().sum(-1), wv.double().sum(-1)]).cpu().numpy()
     np.testing.assert_allclose(G[:, :, pf - 1, pf - 1].cpu().numpy(), sw, rtol=1e-5)
+
+
+def test_config3_full_size_sampled_outputs():
+    """Config 3 itself: 200 sequences x 1,024 tokens in four 51,200-token calls, all 128 (comp, layer) groups on the
+    GPU.  The oracle cannot finish a 4097-wide group at this size in minutes, so sampled outputs are compared: for one
+    group (V, layer 17) and one target head, the whole C (4097 x 128), and the blocks of G that couple one source head
+    across the four selected layers (eight 513 x 513 pieces), each from the oracle's k = 4 head-local statistics of
+    that source head, which are by definition those entries of the full-head statistics."""
+    wl = synth.workload("qwen14b_32b_500")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    sets = cb.cb_fullhead_layer_sets(wl.Ls, wl.Lt, 4)
+    prob = cb.FullHeadProblem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sets)
+    pf, d, k = prob.pf, wl.d, 4
+    G = torch.zeros(2, wl.Lt, pf, pf, device=DEV)
+    C = torch.zeros(2, wl.Lt, wl.Ht, pf, d, device=DEV)
+    law = synth.map_law(wl, DEV)
+    comp, l, h = 1, 17, 5
+    keep = [int(j) for j in sets[l]]
+    Gp = [None] * wl.Hs
+    Cp = [None] * wl.Hs
+    n_tok = 0
+    for c in range(4):                                            # 4 x 50 sequences = the configuration's 200
+        ch = synth.make_chunk(wl, c, sl, sh, device=DEV, law=law)
+        wk, wv = ch["w_k"][:, 0].contiguous(), ch["w_v"][:, 0].contiguous()      # weights per (comp, layer, token)
+        cb.cb_fullhead_stats_accumulate(prob, ch["src_k"], ch["src_v"], ch["tgt_k"], ch["tgt_v"], wk, wv, G, C)
+        src = bits(ch["src_v"][keep].cpu())                       # the four selected layers, re-indexed 0..3
+        tgt = bits(ch["tgt_v"][l:l + 1].cpu())
+        w = wv[l].cpu().numpy()
+        for g in range(wl.Hs):
+            gg, cc = oracle.multilayer_stats(src, tgt, w, 0, h, g, [0, 1, 2, 3])
+            Gp[g] = gg if Gp[g] is None else Gp[g] + gg
+            Cp[g] = cc if Cp[g] is None else Cp[g] + cc
+        n_tok += ch["n_tokens"]
+        del ch
+    cb.cb_last_device_status()
+    assert n_tok == 204800
+    Gg, Cg = G[comp, l].cpu().numpy(), C[comp, l, h].cpu().numpy()
+    Co = np.zeros((pf, d))
+    num = den = 0.0
+    worst = 0.0
+    for g in range(wl.Hs):
+        rows = np.array([(f * wl.Hs + g) * d + c_ for f in range(k) for c_ in range(d)] + [pf - 1])
+        Co[rows[:-1]] = Cp[g][:-1]
+        Co[pf - 1] = Cp[g][-1]
+        sub = Gg[np.ix_(rows, rows)]
+        num += np.linalg.norm(sub - Gp[g]) ** 2
+        den += np.linalg.norm(Gp[g]) ** 2
+        worst = max(worst, rel_fro(sub, Gp[g]))
+    eg, ec = float(np.sqrt(num / den)), rel_fro(Cg, Co)
+    print("config 3 at full size (204,800 tokens), (V, layer 17, head 5): rel err C %.2e; G pieces pooled %.2e, worst %.2e"
+          % (ec, eg, worst))
+    assert ec <= TOL and eg <= TOL and worst <= TOL
+    assert torch.isfinite(G).all() and torch.isfinite(C).all()
