@@ -630,6 +630,23 @@ def multilayer_case(args, cb, synth, torch, wl, sl, sh, dev):
         e1.synchronize()
         ms.append(e0.elapsed_time(e1))
     del ch
+    if args.profile_tokens > 0:
+        # profiling case: no solve (random maps of the right scale), the apply on the same number of tokens
+        Wr = torch.randn(wl.n_maps, P, d, device=dev) / (P ** 0.5)
+        src = synth.make_source_cache(wl, T, dev, synth.map_law(wl, dev))
+        out_k = torch.empty(wl.Lt, T, wl.Ht, d, dtype=torch.bfloat16, device=dev)
+        out_v = torch.empty_like(out_k)
+        tt = []
+        for i in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            cb.cb_apply_multilayer(prob, sh, Wr, src[0], src[1], out_k, out_v)
+            e1.record()
+            e1.synchronize()
+            tt.append(e0.elapsed_time(e1))
+        cb.cb_last_device_status()
+        print("profile case k=%d, %d tokens: statistics ms %s, apply ms %s" % (k, T, ms, tt), file=sys.stderr)
+        return
     lams = list(wl.lambdas)
     nsys = len(lams) * wl.n_maps
     ws = torch.empty(cb.cb_ridge_solve_large_workspace_bytes(P, d, min(nsys, 3072)), dtype=torch.uint8, device=dev)

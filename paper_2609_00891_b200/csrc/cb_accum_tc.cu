@@ -19,15 +19,6 @@
 // Every wait is bounded: if one runs out the block sets the context's status word and tears down.
 #include <cudaTypedefs.h>
 
-#ifndef CB_NS
-#define CB_NS 4          // measured: 3 stages 3 % slower, 5 stages 1 % slower than 4
-#endif
-#ifndef CB_NA
-#define CB_NA 2
-#endif
-#ifndef CB_FOLD_WARPS
-#define CB_FOLD_WARPS 8  // measured: 16 warps 1.5 % slower (more warps polling), 4 warps 6 % slower
-#endif
 
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
@@ -48,14 +39,14 @@ struct TcCfg {
     static constexpr int STAGE_BYTES = (FH ? 3 : 2) * NBX * BLK;
     static constexpr int AS_OFF = FH ? 2 * NBX * BLK : 0;   // where the rows to be weighted start inside a stage
     static constexpr int A_BYTES = 2 * BLK;           // M = 128 always: two blocks (second stays zero for d = 64)
-    static constexpr int NS = FH ? 3 : (COMP ? 4 : CB_NS);   // stages
-    static constexpr int NA = COMP ? 2 : CB_NA;                    // weighted-operand buffers (hi, and lo when compensated)
+    static constexpr int NS = FH ? 3 : 4;   // stages (measured: 3 stages 3 % slower, 5 stages 1 % slower than 4)
+    static constexpr int NA = 2;                    // weighted-operand buffers (hi, and lo when compensated)
     static constexpr int A_PARTS = COMP ? 2 : 1;
     static constexpr int N = 2 * D;                   // accumulator columns
     static constexpr int TMEM_COLS = 2 * N;           // two accumulators
     // ROPE: at most 8 fold warps, so that each fold thread may hold the rotation state of its rows in registers
     // (the block's register file divided by its threads caps a thread at 80 registers with 16 fold warps)
-    static constexpr int FOLD_WARPS = (ROPE && CB_FOLD_WARPS > 8) ? 8 : CB_FOLD_WARPS, DRAIN_WARPS = 4;
+    static constexpr int FOLD_WARPS = 8, DRAIN_WARPS = 4;   // measured: 16 fold warps 1.5 % slower, 4 warps 6 % slower
     static constexpr int YPROD_WARP = 2 + FOLD_WARPS + DRAIN_WARPS;   // second producer: target tiles + weights
     static constexpr int FOLD_THREADS = FOLD_WARPS * 32;
     static constexpr int THREADS = (3 + FOLD_WARPS + DRAIN_WARPS) * 32;
@@ -187,15 +178,6 @@ struct TileIterT {
     }
 };
 
-#ifdef CB_TRACE
-// Tuning aid: block 0 records clock64() of every role for tiles [CB_TRACE_T0, CB_TRACE_T0 + 64).
-#define CB_TRACE_T0 1000
-__device__ long long g_trace[64][40];
-#define CB_TR(itv, slot) do { if (blockIdx.x == 0 && lane == 0 && (itv) >= CB_TRACE_T0 && (itv) < CB_TRACE_T0 + 64) g_trace[(itv) - CB_TRACE_T0][slot] = clock64(); } while (0)
-extern "C" int cb_debug_trace(long long *host) { return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(g_trace)); }
-#else
-#define CB_TR(itv, slot) do {} while (0)
-#endif
 
 // ROPE: key maps (comp = 0) are fitted in content coordinates (Section 3.1): the fold warps rotate every source and
 // target key row back by its position's angles IN PLACE in the staged tile (so the tensor cores read the de-rotated
@@ -273,11 +255,9 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                 const int g = cur.b1_head, j = cur.b1_layer, ag = cur.a_head, aj = cur.a_layer, u = cur.u;
                 do {   // tiles of one unit
                     if (!mbar_wait(&empty[st.idx], st.phase ^ 1, abort_flag)) goto teardown;
-                    CB_TR(it, 0);
                     mbar_arrive_expect_tx(&full[st.idx], (FH ? 2 : 1) * C::NBX * C::BLK);
                     tma_load_5d(xy + st.idx * C::STAGE_BYTES, map, &full[st.idx], 0, cur.tile * C::TT, 0, g, j);
                     if (FH) tma_load_5d(xy + st.idx * C::STAGE_BYTES + C::AS_OFF, map, &full[st.idx], 0, cur.tile * C::TT, 0, ag, aj);
-                    CB_TR(it, 1);
                     st.next();
                     ++it;
                     cur.advance(P, n_units, n_maps, n_tiles);
@@ -298,7 +278,6 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
             const float *w = cur.weights(a);
             do {
                 if (!mbar_wait_warp(&empty[st.idx], st.phase ^ 1, abort_flag, lane)) goto teardown;
-                CB_TR(it, 38);
                 const int tok0 = cur.tile * C::TT;
                 if (lane == 0) {
                     mbar_arrive_expect_tx(&full[st.idx], C::NBX * C::BLK);
@@ -312,7 +291,6 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                     if (ROPE) cp_async_4(&pst[st.idx * C::TT + r], P.rope.pos + (in ? tok0 + r : 0), in ? 4u : 0u);
                 }
                 cp_async_arrive_noinc(&full[st.idx]);
-                CB_TR(it, 39);
                 st.next();
                 ++it;
                 cur.advance(P, n_units, n_maps, n_tiles);
@@ -345,7 +323,6 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                     for (int t = 0; t < n_sub; ++t) {
                         // afull implies full: every fold warp saw the tile land before it wrote the weighted operand
                         if (!mbar_wait(&afull[ar.idx], ar.phase, abort_flag)) goto teardown;
-                        CB_TR(it, 3);
                         tc_fence_after();
                         const uint32_t bl = b_lo0 + st.idx * (C::STAGE_BYTES >> 4);
                         const uint32_t al = a_lo0 + ar.idx * ((C::A_PARTS * C::A_BYTES) >> 4);
@@ -357,7 +334,6 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                         }
                         accum = 1;
                         umma_commit(&empty[st.idx]);     // frees the stage and (through it) the weighted-operand buffer
-                        CB_TR(it, 4);
                         st.next();
                         ar.next();
                         ++it;
@@ -432,7 +408,6 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                     if (!mbar_wait_warp(&empty[old.idx], old.phase, abort_flag, lane)) goto teardown;
                     old.next();
                 }
-                CB_TR(it, 5 + 2 * (warp - 2));
                 const float *wsm = wst + st.idx * C::TT + rg;
                 const uint8_t *xs = xy + st.idx * C::STAGE_BYTES + C::AS_OFF + off0;          // rows to be weighted
                 const uint8_t *ys = xy + st.idx * C::STAGE_BYTES + C::NBX * C::BLK + off0;    // B2: summed with the weights
@@ -573,7 +548,6 @@ __global__ void __launch_bounds__(TcCfg<D, COMP, FH, ROPE>::THREADS, 1) k_accum_
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&afull[ar.idx]); mbar_arrive(&empty[st.idx]); }
-                CB_TR(it, 6 + 2 * (warp - 2));
                 st.next();
                 ar.next();
                 ++it;
@@ -761,8 +735,9 @@ static PFN_cuTensorMapEncodeTiled_v12000 encode_fn()
 
 // 5-D map over (64 channels, token, 64-channel block, head, layer).  One box = box_tokens tokens of one head of
 // one layer, laid out in shared memory as [channel block][token][64 channels] with the 128-byte swizzle.
+// box_cblocks: 64-channel blocks per box (0: all d / 64 of them; 1: one block, selected by the copy's third coordinate).
 bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long long T, int L,
-                        long long sh, long long st, long long sl, int box_tokens)
+                        long long sh, long long st, long long sl, int box_tokens, int box_cblocks)
 {
     PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
     if (!enc) return false;
@@ -771,7 +746,7 @@ bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long l
     };
     cuuint64_t gdim[5] = {64, (cuuint64_t)T, (cuuint64_t)(d / 64), (cuuint64_t)H, (cuuint64_t)L};
     cuuint64_t gstr[4] = {stride(st, T), 128, stride(sh, H), stride(sl, L)};
-    cuuint32_t box[5] = {64, (cuuint32_t)box_tokens, (cuuint32_t)(d / 64), 1, 1}, estr[5] = {1, 1, 1, 1, 1};
+    cuuint32_t box[5] = {64, (cuuint32_t)box_tokens, (cuuint32_t)(box_cblocks > 0 ? box_cblocks : d / 64), 1, 1}, estr[5] = {1, 1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), gdim, gstr, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

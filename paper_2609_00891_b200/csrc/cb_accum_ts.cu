@@ -32,10 +32,6 @@
 // Every wait is bounded: if one runs out the block sets the context's status word and tears down.
 #include <cudaTypedefs.h>
 
-#ifndef CB_TS_TT
-#define CB_TS_TT 128
-#endif
-
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
 #include "cb_math.cuh"
@@ -45,15 +41,12 @@ namespace cb {
 
 using namespace ptx;
 
-bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long long T, int L,
-                        long long sh, long long st, long long sl, int box_tokens);
-
 namespace {
 
 template <bool COMP>
 struct TsCfg {
     static constexpr int D = 128;
-    static constexpr int TT = COMP ? 64 : CB_TS_TT;   // tokens per tile (compensated: two operand images per tile)
+    static constexpr int TT = COMP ? 64 : 128;   // tokens per tile (compensated: two operand images per tile)
     static constexpr int BLK = TT * 128;              // one 64-channel block of a tile: TT rows of 128 bytes
     static constexpr int STAGE_BYTES = 4 * BLK;       // [X blocks 0, 1 | Y blocks 0, 1]
     static constexpr int WB_BYTES = (TT / 64) * 2048; // per 64 tokens: 16 rows of 128 bytes (K-major, 128-byte swizzle)

@@ -19,27 +19,17 @@
 
 #include <cuda_fp16.h>
 
+#include <algorithm>
+#include <vector>
+
 #include "cb_internal.cuh"
 #include "cb_ptx.cuh"
 #include "cb_math.cuh"
 #include "cb_rope.cuh"
 
-#ifndef CB_AP_NS
-#define CB_AP_NS 3
-#endif
-#ifndef CB_AP_NO
-#define CB_AP_NO 2
-#endif
-#ifndef CB_AP_NACC
-#define CB_AP_NACC 4
-#endif
-
 namespace cb {
 
 using namespace ptx;
-
-bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long long T, int L,
-                        long long sh, long long st, long long sl, int box_tokens);
 
 template <int D>
 struct ApCfg {
@@ -50,9 +40,9 @@ struct ApCfg {
     static constexpr int WBLK = D * 128;                // bytes of one W block: D rows (input channels) of 128 bytes
     static constexpr int W_BYTES = NB * WBLK;           // hi (or lo) part of W
     static constexpr int O_BYTES = NB * XBLK;           // bf16 output tile
-    static constexpr int NS = CB_AP_NS;
-    static constexpr int NO = CB_AP_NO;                 // output tiles in shared memory
-    static constexpr int NACC = CB_AP_NACC;
+    static constexpr int NS = 3;
+    static constexpr int NO = 2;                 // output tiles in shared memory
+    static constexpr int NACC = 4;
     static constexpr int AW = D;                        // accumulator columns per tile: X W_hi + X W_lo
     static constexpr int TMEM_COLS = (NACC * AW < 32) ? 32 : NACC * AW;
     static constexpr int EPI_WARPS = 4, CONV_WARPS = 4;
@@ -564,7 +554,11 @@ cudaError_t launch_apply_tc(const ApplyArgs &a, int d, const cb_kv_view *src, cu
 // quarter of what one tile at a time would need (that version was bound by it: 96 KB staged per 32 KB source tile).
 // The loop runs f outer, tile inner; the tiles of a group finish one after the other in the last f pass and the next
 // group starts with tile 0 again, so the epilogue of a group overlaps the next group's products accumulator by
-// accumulator.  bf16 rows go from registers straight to global memory (256 contiguous bytes per thread; this path is
+// accumulator.  What bounds it: shared-memory bandwidth.  Every product reads both operands from shared memory (4 KB
+// of the source tile and 4 KB of W per 128 x 128 x 16 product, i.e. 128 bytes per clock at the tensor cores' full
+// rate) beside the copies that fill the stages; measured: half the tensor cores' rate.  Staging 64-channel pieces
+// instead of whole tiles (deeper rings, twice the barrier traffic per product) measured 15 % slower.
+// bf16 rows go from registers straight to global memory (256 contiguous bytes per thread; this path is
 // bound by the tensor cores, not by its stores).
 // =====================================================================================================================
 template <int D>
@@ -589,6 +583,7 @@ struct MlParams {
     ApplyArgs a;                 // src_layer / src_head arrays unused except src_head
     const uint8_t *wsplit;       // [n_maps][k][hi | lo][W_BYTES]
     const int *layer_sets;       // device [Lt][k]
+    const int *f_order;          // device [Lt][k]: the order in which a map of target layer l walks its k blocks
     int k, n_splits;
 };
 
@@ -671,9 +666,10 @@ __global__ void __launch_bounds__(MlCfg<D>::THREADS, 1) k_apply_ml_tc(const __gr
                     for (int f = 0; f < k; ++f) {
                         if (!mbar_wait(&wempty[wr.idx], wr.phase ^ 1, abort_flag)) goto ml_teardown;
                         mbar_arrive_expect_tx(&wfull[wr.idx], C::WSTAGE);
-                        bulk_load(wsm + (size_t)wr.idx * C::WSTAGE, wm + (size_t)f * C::WSTAGE, C::WSTAGE, &wfull[wr.idx]);
+                        const int fb = P.f_order[l * k + f];          // block of this step (see launch_apply_ml_tc)
+                        bulk_load(wsm + (size_t)wr.idx * C::WSTAGE, wm + (size_t)fb * C::WSTAGE, C::WSTAGE, &wfull[wr.idx]);
                         wr.next();
-                        const int j = P.layer_sets[l * k + f];
+                        const int j = P.layer_sets[l * k + fb];
                         for (int t = 0; t < ng; ++t) {
                             if (!mbar_wait(&xempty[xr.idx], xr.phase ^ 1, abort_flag)) goto ml_teardown;
                             mbar_arrive_expect_tx(&xfull[xr.idx], C::X_BYTES);
@@ -811,7 +807,7 @@ ml_teardown:
 
 size_t apply_ml_workspace_bytes(int n_maps, int k, int d, int Lt)
 {
-    return (size_t)n_maps * k * 2 * (size_t)d * d * 2 + ((sizeof(int) * (size_t)Lt * k + 255) / 256) * 256;
+    return (size_t)n_maps * k * 2 * (size_t)d * d * 2 + ((sizeof(int) * 2 * (size_t)Lt * k + 255) / 256) * 256;
 }
 
 template <int D>
@@ -848,7 +844,21 @@ cudaError_t launch_apply_ml_tc(const ApplyArgs &a, int d, int k, const int *laye
     const size_t wbytes = (size_t)n_maps * k * 2 * (size_t)d * d * 2;
     P.wsplit = ws;
     P.layer_sets = reinterpret_cast<const int *>(ws + wbytes);
-    cudaError_t e = cudaMemcpyAsync(ws + wbytes, layer_sets_host, sizeof(int) * (size_t)a.Lt * k, cudaMemcpyHostToDevice, st);
+    P.f_order = P.layer_sets + (size_t)a.Lt * k;
+    // Order of the k blocks of a map: by (source layer mod k).  The persistent blocks walk their units in step, and
+    // maps of neighbouring target layers select overlapping source layers; with this order every map that reads
+    // layer j reads it in the same step, so that one fetch from device memory serves all of them through L2 (for k
+    // consecutive layers the order is a rotation of the set).  The sum over blocks does not depend on the order
+    // beyond fp32 rounding, and the order is fixed by the problem.
+    std::vector<int> tab(layer_sets_host, layer_sets_host + (size_t)a.Lt * k);
+    tab.resize(2 * (size_t)a.Lt * k);
+    for (int l = 0; l < a.Lt; ++l) {
+        int *ord = tab.data() + (size_t)a.Lt * k + (size_t)l * k;
+        for (int f = 0; f < k; ++f) ord[f] = f;
+        const int *set = layer_sets_host + (size_t)l * k;
+        std::stable_sort(ord, ord + k, [&](int x, int y) { return set[x] % k < set[y] % k; });
+    }
+    cudaError_t e = cudaMemcpyAsync(ws + wbytes, tab.data(), sizeof(int) * tab.size(), cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return e;
     if (!make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
                             src->stride_token, src->stride_layer, TT) ||

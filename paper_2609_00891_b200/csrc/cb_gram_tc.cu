@@ -32,9 +32,6 @@ namespace cb {
 
 using namespace ptx;
 
-bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long long T, int L,
-                        long long sh, long long st, long long sl, int box_tokens);
-
 template <int D>
 struct GrCfg {
     static_assert(D == 128, "two 64-channel blocks per head make the M = 128 operand");
@@ -153,15 +150,6 @@ struct GrUnit {
     }
 };
 
-#ifdef CB_GTRACE
-// Tuning aid: block 0 records clock64() of its roles for its tiles [CB_GTRACE_T0, CB_GTRACE_T0 + 64).
-#define CB_GTRACE_T0 2000
-__device__ long long g_gtrace[64][16];
-#define GTR(itv, slot) do { if (blockIdx.x == 0 && (itv) >= CB_GTRACE_T0 && (itv) < CB_GTRACE_T0 + 64) g_gtrace[(itv) - CB_GTRACE_T0][slot] = clock64(); } while (0)
-extern "C" int cb_debug_gtrace(long long *host) { return (int)cudaMemcpyFromSymbol(host, g_gtrace, sizeof(g_gtrace)); }
-#else
-#define GTR(itv, slot) do {} while (0)
-#endif
 
 template <int D>
 __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_constant__ GrParams P)
@@ -220,9 +208,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                 const CUtensorMap *map = un.comp ? &P.src_v : &P.src_k;
                 const int nrow = 1 + un.va[1];
                 for (int tile = 0; tile < n_tiles; ++tile, ++itc) {
-                    GTR(itc, 0);
                     if (!mbar_wait(&empty[st.idx], st.phase ^ 1, abort_flag)) goto teardown;
-                    GTR(itc, 1);
                     uint8_t *dst = stg + st.idx * C::STAGE_BYTES + 2 * C::HEAD;
                     if (un.diag) {
                         mbar_arrive(&full[st.idx]);              // the fold warps weight the column heads' tiles
@@ -286,9 +272,7 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                     tc_fence_after();
                     uint32_t accum = 0;
                     for (int t = 0; t < n_sub; ++t, ++itm) {
-                        GTR(itm, 2);
                         if (!mbar_wait(&afull[st.idx], st.phase, abort_flag)) goto teardown;
-                        GTR(itm, 3);
                         tc_fence_after();
                         const uint32_t bl = b_lo0 + st.idx * (C::STAGE_BYTES >> 4);
                         const uint32_t al = bl + ((2 * C::HEAD) >> 4);                 // weighted row heads
@@ -302,7 +286,6 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                         }
                         accum = 1;
                         umma_commit(&empty[st.idx]);
-                        GTR(itm, 4);
                         st.next();
                     }
                     umma_commit(accfull);
@@ -319,7 +302,6 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
         const int off0 = blk * C::BLK + rg * 128 + ((lc ^ (rg & 7)) << 4);
         Ring<C::NS> st;
         uint32_t uc = 0;
-        int itf = 0;
         GrUnit un;
         for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++uc) {
             un.decode(P, u);
@@ -330,10 +312,8 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
 #pragma unroll
             for (int e = 0; e < 4; ++e) sa2[e] = sb2[e] = 0ull;
             float sw = 0.f;
-            for (int t = 0; t < n_tiles; ++t, ++itf) {
-                if (lane == 0 && (fw == 0 || fw == 8)) GTR(itf, 5 + (fw >> 3) * 3);
+            for (int t = 0; t < n_tiles; ++t) {
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
-                if (lane == 0 && (fw == 0 || fw == 8)) GTR(itf, 6 + (fw >> 3) * 3);
                 const float *wsm = wst + st.idx * C::TT + rg;
                 uint8_t *ah = stg + st.idx * C::STAGE_BYTES + (2 + g) * C::HEAD + off0;           // weighted row head g
                 const uint8_t *cs = stg + st.idx * C::STAGE_BYTES + g * C::HEAD + off0;           // column head g
@@ -376,12 +356,9 @@ __global__ void __launch_bounds__(GrCfg<D>::THREADS, 1) k_gram2_tc(const __grid_
                         for (int e = 0; e < 4; ++e) sb2[e] = f2_fma(w2, f2_from_bf16x2(yu[e]), sb2[e]);
                     }
                 }
-                if (lane == 0 && fw == 0) GTR(itf, 11);
                 fence_async_smem();
-                if (lane == 0 && fw == 0) GTR(itf, 12);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&afull[st.idx]);
-                if (lane == 0 && (fw == 0 || fw == 8)) GTR(itf, 7 + (fw >> 3) * 3);
                 st.next();
             }
             // ---- bias entries (C units only): lanes holding the same channels add up, fixed-order sum over the

@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of the library (not part of the C ABI).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -128,6 +129,13 @@ cudaError_t launch_rope_rotate(void *k, int L, int H, int d, long long T, long l
                                const int *pos, double base, int inverse, cudaStream_t stream);
 
 void count_launch(int n = 1);
+
+// 5-D tensor map over (64 channels, token, 64-channel block, head, layer) of a strided bf16 K or V tensor.  One box =
+// box_tokens tokens of one head of one layer, laid out in shared memory as [channel block][token][64 channels] with
+// the 128-byte swizzle; box_cblocks = 64-channel blocks per box (0: all d / 64 of them; 1: one block, selected by the
+// copy's third coordinate).
+bool make_kv_tensor_map(CUtensorMap *map, const void *base, int d, int H, long long T, int L,
+                        long long sh, long long st, long long sl, int box_tokens, int box_cblocks = 0);
 
 // Host-side argument checks shared by the entry points (status codes of the C ABI).
 cb_status check_problem(const cb_problem *p);
