@@ -188,336 +188,6 @@ cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, f
 }
 
 // ======================================================================================================
-// Batched ridge solve, fp64, one block per (map, lambda).
-//   A = G + lambda_eff * diag(1,..,1,0);  A = L L^T (packed lower triangle, rows padded to even length);
-//   L Z = C, L^T Theta = Z.
-// ======================================================================================================
-struct SolveArgs {
-    const float *G, *C;    // augmented: G [p][p], C [p][d];  centred: A [d][d], B [d][d]
-    const float *mu;       // centred form only: [n_maps][2d + 1] = mu_x, mu_y, s_w; null for the augmented form
-    float *Wb;
-    int *info;
-    int n_maps, d;
-    double inv_n;
-    unsigned flags;
-    int n_lambda;
-    float lambdas[16];
-};
-
-__host__ __device__ inline int tri_row_start(int i)
-{
-    // sum_{r<i} roundup2(r+1):  rows 0..i-1 have lengths 1..i, each padded to even
-    const int h = i / 2;            // pairs (1,2),(3,4),.. padded to (2,2),(4,4),..
-    return 2 * h * (h + 1) + ((i & 1) ? (i + 1) : 0);
-}
-
-// shuffle of a double between lane pairs
-__device__ __forceinline__ double shfl_xor_f64(double v, int mask)
-{
-    int lo = __double2loint(v), hi = __double2hiint(v);
-    lo = __shfl_xor_sync(0xffffffffu, lo, mask);
-    hi = __shfl_xor_sync(0xffffffffu, hi, mask);
-    return __hiloint2double(hi, lo);
-}
-
-// Cholesky by block columns of 8 (left-looking): thread i owns row i of L; thread n + c owns right-hand-side column c,
-// whose forward substitution obeys the same recurrence as a row of L below the diagonal block and rides along.  For
-// a block column a thread pulls its 8 entries into registers, subtracts the contributions of all finished columns
-// (its own row times the 8 rows of the diagonal block, read as broadcasts), the 8 diagonal-block rows publish theirs,
-// one otherwise idle thread factors that 8 x 8 block in registers while the others already work on the next block
-// column, and every thread solves its own row against the block.  Three block barriers per block column.
-// The backward substitution gives every right-hand-side column to a pair of lanes that split the inner sums; eight
-// rows are kept in registers at a time, so each loaded L entry feeds one FMA and each loaded Z entry feeds eight.
-#ifdef CB_SOLVE_TIMING
-__device__ long long g_solve_t[8];
-extern "C" int cb_debug_solve_t(long long *h) { return (int)cudaMemcpyFromSymbol(h, g_solve_t, sizeof(g_solve_t)); }
-#define ST(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_solve_t[i] = clock64(); } while (0)
-#else
-#define ST(i) do {} while (0)
-#endif
-constexpr int SOLVE_THREADS = 320;     // 129 rows of L + 128 right-hand-side columns, and a warp for the thread that
-constexpr int SOLVE_FACTOR_THREAD = 288;   // factors the diagonal blocks
-#ifndef CB_SOLVE_AHEAD
-#define CB_SOLVE_AHEAD 148
-#endif
-__global__ void __launch_bounds__(SOLVE_THREADS, 1) k_ridge_solve(const SolveArgs a)
-{
-    ST(0);
-    extern __shared__ __align__(16) double sm[];
-    constexpr int NB = 8;
-    const int d = a.d, p = d + 1;
-    const bool centred = a.mu != nullptr;
-    const int n = centred ? d : p;                     // order of the system: the centred form has no bias row
-    // blocks of one map's lambdas are neighbours in launch order: the second and third read G and C from L2
-    const int m = blockIdx.x / a.n_lambda, li = blockIdx.x % a.n_lambda;
-    double *Lp = sm;                                   // packed lower triangle, rows padded to even length
-    double *Z = sm + tri_row_start(n);                 // [n][d]
-    __shared__ double diag[NB][NB];
-    __shared__ double rdiag[136];                      // reciprocals of the diagonal of L
-    __shared__ int s_fail;
-    const int tid = threadIdx.x;
-
-    const float *Gm = a.G + (size_t)m * n * n;
-    const float *Cm = a.C + (size_t)m * n * d;
-    const double s_w = centred ? (double)a.mu[(size_t)m * (2 * d + 1) + 2 * d] : (double)Gm[(size_t)d * p + d];
-    const double lam = (a.flags & CB_FLAG_RAW_LAMBDA) ? (double)a.lambdas[li] : (double)a.lambdas[li] * s_w * a.inv_n;
-    if (tid == 0) s_fail = 0;
-    {
-        // The block that will follow this one on the SM is, to a good guess, gridDim-resident blocks further on (one
-        // block per SM): ask L2 for its statistics now, so that its load phase does not wait for DRAM.
-        const int nb = blockIdx.x + CB_SOLVE_AHEAD;
-        if (nb < (int)gridDim.x && nb / a.n_lambda != m) {
-            const int m2 = nb / a.n_lambda;
-            const char *g2 = reinterpret_cast<const char *>(a.G + (size_t)m2 * n * n);
-            const char *c2 = reinterpret_cast<const char *>(a.C + (size_t)m2 * n * d);
-            for (int o = tid * 128; o < n * n * 4; o += blockDim.x * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(g2 + o));
-            for (int o = tid * 128; o < n * d * 4; o += blockDim.x * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(c2 + o));
-        }
-    }
-    {
-        const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-        // one warp per row (coalesced, no divisions); the global loads of a row are issued together before any
-        // shared-memory store so that they overlap
-        constexpr int MAXV = 5;                            // ceil(129 / 32)
-        // four rows in flight per warp (36 loads per lane): the phase is bound by load latency, L2 or DRAM
-#pragma unroll 4
-        for (int i = warp; i < n; i += nwarps) {
-            const int rsi = tri_row_start(i);
-            float gv[MAXV], cv[MAXV];
-#pragma unroll
-            for (int v = 0; v < MAXV; ++v) {
-                const int k = lane + 32 * v;
-                gv[v] = (k <= i) ? __ldg(Gm + (size_t)i * n + k) : 0.f;
-                cv[v] = (k < d) ? __ldg(Cm + (size_t)i * d + k) : 0.f;
-            }
-#pragma unroll
-            for (int v = 0; v < MAXV; ++v) {
-                const int k = lane + 32 * v;
-                if (k <= i) Lp[rsi + k] = (double)gv[v] + ((i == k && i < d) ? lam : 0.0);
-                if (k < d) Z[(size_t)i * d + k] = (double)cv[v];
-            }
-        }
-    }
-    __syncthreads();
-
-    ST(1);
-    // ---------------- Cholesky, with the forward substitution riding along ----------------
-    // Z^T = (L^-1 C)^T obeys the same recurrence as the rows of L below the diagonal block:
-    //     Z[j][c] = (C[j][c] - sum_{k<j} Z[k][c] L[j][k]) / L[j][j],
-    // so thread n + c treats right-hand-side column c as one more row of the matrix being factored (it never
-    // contributes to a diagonal block).  All 257 threads work through the block columns together and no separate
-    // forward pass is needed.
-    // While one otherwise idle thread factors the 8 x 8 diagonal block of block column j0 (a serial chain of eight
-    // reciprocal square roots), the row threads already subtract the finished columns k < j0 from their entries of
-    // block column j0 + 8; the eight columns of block j0 itself are subtracted at the top of the next iteration.
-    const int row = tid;
-    const bool is_rhs = tid >= n && tid < n + d;
-    const int col = tid - n;                           // right-hand-side column of an extra row
-    const int rs = tri_row_start(row < n ? row : 0);
-    // entries of block column jb owned by this thread, before any subtraction
-    auto init_block = [&](double (&ac)[NB], int jb) {
-        const int nbb = min(NB, n - jb);
-        if (is_rhs) {
-#pragma unroll
-            for (int c = 0; c < NB; ++c) ac[c] = (c < nbb) ? Z[(size_t)(jb + c) * d + col] : 0.0;
-        } else {
-#pragma unroll
-            for (int c = 0; c < NB; ++c) ac[c] = (c < nbb && jb + c <= row) ? Lp[rs + jb + c] : 0.0;
-        }
-    };
-    // ac[c] -= sum_{k0 <= k < k1} (own row)[k] * L[jb + c][k]; k0, k1 multiples of 8: aligned pairs
-    auto subtract_columns = [&](double (&ac)[NB], int jb, int k0, int k1) {
-        int drs[NB];
-#pragma unroll
-        for (int c = 0; c < NB; ++c) drs[c] = tri_row_start(min(jb + c, n - 1));
-        for (int k = k0; k < k1; k += 2) {
-            double2 mine;
-            if (is_rhs) mine = make_double2(Z[(size_t)k * d + col], Z[(size_t)(k + 1) * d + col]);
-            else mine = *reinterpret_cast<const double2 *>(&Lp[rs + k]);
-#pragma unroll
-            for (int c = 0; c < NB; ++c) {
-                const double2 o = *reinterpret_cast<const double2 *>(&Lp[drs[c] + k]);
-                ac[c] -= mine.x * o.x;
-                ac[c] -= mine.y * o.y;
-            }
-        }
-    };
-    double acc[NB];
-#pragma unroll
-    for (int c = 0; c < NB; ++c) acc[c] = 0.0;
-    if (row < n || is_rhs) init_block(acc, 0);
-    for (int j0 = 0; j0 < n; j0 += NB) {
-        const int nb = min(NB, n - j0);
-        const bool active = (row < n && row >= j0) || is_rhs;
-        if (active) {
-            if (j0 > 0) subtract_columns(acc, j0, j0 - NB, j0);
-            if (!is_rhs && row < j0 + nb) {
-#pragma unroll
-                for (int c = 0; c < NB; ++c) diag[row - j0][c] = acc[c];
-            }
-        }
-        __syncthreads();
-        double accn[NB];
-#pragma unroll
-        for (int c = 0; c < NB; ++c) accn[c] = 0.0;
-        if (tid == SOLVE_FACTOR_THREAD) {
-            // one thread factors the nb x nb diagonal block (sqrt and reciprocal are long fp64 sequences: doing
-            // them once and broadcasting beats doing them in every thread); the block is held in registers
-            double Ld[NB][NB];
-#pragma unroll
-            for (int r = 0; r < NB; ++r)
-#pragma unroll
-                for (int c = 0; c < NB; ++c)
-                    if (c <= r) Ld[r][c] = (r < nb) ? diag[r][c] : (r == c ? 1.0 : 0.0);
-            int fail = 0;
-#pragma unroll
-            for (int c = 0; c < NB; ++c) {
-                double v = Ld[c][c];
-#pragma unroll
-                for (int q = 0; q < NB; ++q)
-                    if (q < c) v -= Ld[c][q] * Ld[c][q];
-                if (!(v > 0.0)) { if (!fail) fail = j0 + c + 1; v = 1.0; }
-                const double ri = rsqrt(v);
-                Ld[c][c] = v * ri;
-                if (c < nb) rdiag[j0 + c] = ri;
-#pragma unroll
-                for (int r = 0; r < NB; ++r)
-                    if (r > c) {
-                        double u = Ld[r][c];
-#pragma unroll
-                        for (int q = 0; q < NB; ++q)
-                            if (q < c) u -= Ld[r][q] * Ld[c][q];
-                        Ld[r][c] = u * ri;
-                    }
-            }
-            if (fail) s_fail = fail;
-#pragma unroll
-            for (int r = 0; r < NB; ++r)
-#pragma unroll
-                for (int c = 0; c < NB; ++c)
-                    if (c <= r) diag[r][c] = Ld[r][c];
-        } else if (j0 + NB < n && ((row < n && row >= j0 + NB) || is_rhs)) {
-            init_block(accn, j0 + NB);
-            subtract_columns(accn, j0 + NB, 0, j0);
-        }
-        __syncthreads();
-        if (active) {
-            if (is_rhs || row >= j0 + nb) {
-                // own row against the block: x_c = (acc_c - sum_{q<c} x_q L[c][q]) / L[c][c]
-#pragma unroll
-                for (int c = 0; c < NB; ++c)
-                    if (c < nb) {
-                        double v = acc[c];
-#pragma unroll
-                        for (int q = 0; q < NB; ++q)
-                            if (q < c) v -= acc[q] * diag[c][q];
-                        acc[c] = v * rdiag[j0 + c];
-                        if (is_rhs) Z[(size_t)(j0 + c) * d + col] = acc[c];
-                        else Lp[rs + j0 + c] = acc[c];
-                    }
-            } else {
-                for (int c = 0; c <= row - j0; ++c) Lp[rs + j0 + c] = diag[row - j0][c];
-            }
-        }
-        __syncthreads();
-        if (s_fail) break;
-#pragma unroll
-        for (int c = 0; c < NB; ++c) acc[c] = accn[c];
-    }
-
-    float *Wm = a.Wb + ((size_t)li * a.n_maps + m) * p * d;
-    if (s_fail) {
-        for (int e = tid; e < p * d; e += blockDim.x) Wm[e] = 0.f;
-        if (tid == 0) a.info[(size_t)li * a.n_maps + m] = s_fail;
-        return;
-    }
-
-    ST(2);
-    // ---------------- backward substitution: column c = tid / 2, the two lanes of a pair split the inner sums ----------------
-    constexpr int RB = 8;
-    if (tid < 2 * d) {
-        const int c = tid >> 1, half = tid & 1;
-        ST(3);
-        // backward: L^T Theta = Z, row blocks bottom-up
-        const int last = ((n - 1) / RB) * RB;
-        for (int i0 = last; i0 >= 0; i0 -= RB) {
-            double acc[RB];
-#pragma unroll
-            for (int r = 0; r < RB; ++r) acc[r] = (half == 0 && i0 + r < n) ? Z[(size_t)(i0 + r) * d + c] : 0.0;
-            for (int k = i0 + RB + half; k < n; k += 2) {
-                const double xk = Z[(size_t)k * d + c];
-                const int rsk = tri_row_start(k) + i0;   // even offset: aligned pairs
-#pragma unroll
-                for (int r = 0; r < RB; r += 2) {
-                    const double2 lv = *reinterpret_cast<const double2 *>(&Lp[rsk + r]);
-                    acc[r] -= lv.x * xk;
-                    acc[r + 1] -= lv.y * xk;
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < RB; ++r) acc[r] += shfl_xor_f64(acc[r], 1);
-#pragma unroll
-            for (int r = RB - 1; r >= 0; --r)
-                if (i0 + r < n) {
-                    double v = acc[r];
-#pragma unroll
-                    for (int q = RB - 1; q >= 0; --q)
-                        if (q > r && i0 + q < n) v -= Lp[tri_row_start(i0 + q) + i0 + r] * acc[q];
-                    v *= rdiag[i0 + r];
-                    acc[r] = v;
-                    if (half == 0) Z[(size_t)(i0 + r) * d + c] = v;
-                }
-            __syncwarp();
-        }
-    }
-    __syncthreads();
-    ST(4);
-    for (int e = tid; e < n * d; e += blockDim.x) Wm[e] = (float)Z[e];
-    if (centred && tid < d) {
-        // b = mu_y - mu_x W (Section 3.4, last display)
-        const float *mup = a.mu + (size_t)m * (2 * d + 1);
-        double v = (double)mup[d + tid];
-        for (int i = 0; i < d; ++i) v -= (double)mup[i] * Z[(size_t)i * d + tid];
-        Wm[(size_t)d * d + tid] = (float)v;
-    }
-    if (tid == 0) a.info[(size_t)li * a.n_maps + m] = 0;
-    ST(5);
-}
-
-static cudaError_t launch_solve_any(const float *G, const float *C, const float *mu, int n_maps, int d, long long n_tokens,
-                                    const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st)
-{
-    SolveArgs a;
-    a.G = G; a.C = C; a.mu = mu; a.Wb = Wb; a.info = info; a.n_maps = n_maps; a.d = d;
-    a.inv_n = n_tokens > 0 ? 1.0 / (double)n_tokens : 0.0;
-    a.flags = flags; a.n_lambda = n_lambda;
-    for (int i = 0; i < 16; ++i) a.lambdas[i] = i < n_lambda ? lambdas[i] : 0.f;
-    const int p = d + 1;
-    const size_t smem = sizeof(double) * ((size_t)tri_row_start(p) + (size_t)p * d);
-    static bool attr[MAX_DEVICES] = {};
-    {
-        cudaError_t e = opt_in_smem(k_ridge_solve, (size_t)(220 * 1024), attr);
-        if (e != cudaSuccess) return e;
-    }
-    k_ridge_solve<<<n_maps * n_lambda, SOLVE_THREADS, smem, st>>>(a);
-    cudaError_t e = cudaGetLastError();
-    if (e == cudaSuccess) count_launch();
-    return e;
-}
-
-cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long long n_tokens,
-                         const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st)
-{
-    return launch_solve_any(G, C, nullptr, n_maps, d, n_tokens, lambdas, n_lambda, flags, Wb, info, st);
-}
-
-cudaError_t launch_solve_centered(const float *A, const float *B, const float *mu, int n_maps, int d, long long n_tokens,
-                                  const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st)
-{
-    return launch_solve_any(A, B, mu, n_maps, d, n_tokens, lambdas, n_lambda, flags, Wb, info, st);
-}
-
-// ======================================================================================================
 // Affine apply, CUDA cores.  Grid (n_maps, token splits), 256 threads; W (fp32) stays in shared memory while
 // the block walks its token tiles of 32.
 // ======================================================================================================
