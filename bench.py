@@ -221,6 +221,9 @@ def main():
     ap.add_argument("--two-pass", action="store_true",
                     help="time the two-pass centred construction (means pass, centred accumulation, reduce, centred solve) "
                          "on the selected workload and print its own JSON line")
+    ap.add_argument("--solve-case", action="store_true",
+                    help="stand-alone ridge solve: 1024 synthetic systems of 129 x 129 with 128 right-hand sides at the three "
+                         "lambdas (no traces resident); prints timings, no JSON line (profiling case)")
     ap.add_argument("--profile-tokens", type=int, default=0,
                     help="profiling case: run only the accumulate kernel (3 launches) and the apply kernel on this many "
                          "tokens of the same shapes, print timings, no JSON line")
@@ -245,6 +248,9 @@ def main():
     alg_bytes, alg_flops = algorithmic_work(wl)
     n_chunks = args.chunks if args.chunks > 0 else wl.n_chunks
     sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    if args.solve_case:
+        solve_case(cb, torch, wl, dev)
+        return
     if args.profile_tokens > 0 and (args.fullhead > 0 or args.multilayer > 0):
         import dataclasses                      # small case of the wide-regressor kernels for ncu
         T = args.profile_tokens
@@ -690,6 +696,30 @@ def multilayer_case(args, cb, synth, torch, wl, sl, sh, dev):
                       "solve_ms_%d_systems" % nsys: ts,
                       "solve_fp64_tflops": nsys * (P ** 3 / 3.0 + 2.0 * P * P * d) * 2 / (min(ts) / 1e3) / 1e12,
                       "s_per_128000_positions": 2.5 * min(ms) / 1e3 + min(ts) / 1e3}))
+
+
+def solve_case(cb, torch, wl, dev):
+    """The batched ridge solve alone on synthetic positive definite systems of the benchmark's shape."""
+    g = torch.Generator(device=dev).manual_seed(7)
+    p, d, n = wl.d + 1, wl.d, 4096
+    X = torch.randn(wl.n_maps, 512, p, device=dev, generator=g)
+    X[:, :, d] = 1.0
+    G = (X.transpose(1, 2) @ X).contiguous()
+    C = torch.randn(wl.n_maps, p, d, device=dev, generator=g)
+    lams = list(wl.lambdas)
+    Wb = torch.empty(len(lams), wl.n_maps, p, d, device=dev)
+    info = torch.empty(len(lams), wl.n_maps, dtype=torch.int32, device=dev)
+    ts = []
+    for _ in range(6):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        cb.cb_ridge_solve(G, C, n, lams, 0, Wb, info)
+        e1.record()
+        e1.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    cb.cb_check_info(info)
+    print("solve case: %d systems of order %d, %d right-hand sides: ms %s" % (len(lams) * wl.n_maps, p, d, ["%.3f" % t for t in ts]),
+          file=sys.stderr)
 
 
 def profile_case(args, cb, synth, torch, wl, sl, sh, dev):
