@@ -354,6 +354,25 @@ cb_status cb_rope_rotate(void *k, int32_t n_layers, int32_t n_heads, int32_t hea
                          int64_t stride_layer, int64_t stride_token, int64_t stride_head,
                          const int32_t *positions, double rope_base, int32_t inverse, void *stream);
 /*
+ * The two-pass centred construction (Section 3.4) with the rotary boundary (Section 3.1): both passes see the key rows
+ * in content coordinates.  cb_means_accumulate_rope is cb_means_accumulate with the embedding removed from source and
+ * target keys before they are summed (the means are those of the de-rotated rows, rounded to bf16 as the second pass
+ * will see them); cb_stats_accumulate_centered_rope is cb_stats_accumulate_centered with the staged key tiles rotated
+ * on chip as in cb_stats_accumulate_rope AND centred there (source and target), so that their rounding to bf16 is
+ * relative to the spread of a channel, not to its mean.  Same call order as the plain two-pass path, same positions and
+ * bases in both passes; between two resets either every chunk goes through the _rope call or none does (the context
+ * remembers which, and cb_stats_reduce_centered skips the key maps' mean correction accordingly).  d = 128 only
+ * (CB_ERR_UNSUPPORTED otherwise); the means pass supports both head widths.
+ */
+cb_status cb_means_accumulate_rope(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                   const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                                   void *means_ws, size_t means_ws_bytes,
+                                   const int32_t *positions, double rope_base_src, double rope_base_tgt, void *stream);
+cb_status cb_stats_accumulate_centered_rope(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                            const float *w_k, const float *w_v,
+                                            int64_t w_stride_layer, int64_t w_stride_head, const float *mu,
+                                            const int32_t *positions, double rope_base_src, double rope_base_tgt, void *stream);
+/*
  * cb_apply_rope: as cb_apply, for a source cache whose keys carry the source model's rotary embedding and a target
  * cache that must carry the target model's:  K_out[l][t][h] = R_tgt(pos_t) ( R_src(-pos_t) x_t W + b ),  values as in
  * cb_apply.  Both rotations run inside the apply kernel (the staged source tile is rotated on chip, the mapped rows in

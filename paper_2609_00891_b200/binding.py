@@ -31,6 +31,7 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_means_workspace_bytes", "cb_means_reset", "cb_means_accumulate", "cb_means_finalize",
            "cb_stats_accumulate_centered", "cb_stats_reduce_centered", "cb_ridge_solve_centered",
            "cb_stats_accumulate_rope", "cb_rope_rotate", "cb_apply_rope",
+           "cb_means_accumulate_rope", "cb_stats_accumulate_centered_rope",
            "cb_means_energy", "cb_probe_r2", "cb_probe_scores", "cb_rank_layers",
            "cb_last_device_status", "cb_test_hooks",
            "cb_launch_count")
@@ -339,6 +340,24 @@ def cb_means_accumulate(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k: torch.Ten
                                      _stream_ptr(stream)), "cb_means_accumulate")
 
 
+def cb_means_accumulate_rope(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor, w_v: torch.Tensor,
+                             means_ws: torch.Tensor, positions: torch.Tensor, rope_base_src: float, rope_base_tgt: float,
+                             stream=None) -> None:
+    """As cb_means_accumulate, keys taken in content coordinates; `positions` is a device int32 tensor [T]."""
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    assert w_k.dtype == torch.float32 and w_v.dtype == torch.float32 and w_k.dim() == 3
+    assert w_k.stride() == w_v.stride() and (w_k.stride(2) == 1 or w_k.shape[2] <= 1)
+    assert means_ws.is_cuda and means_ws.dtype == torch.uint8
+    assert positions.dtype == torch.int32 and positions.is_cuda and positions.is_contiguous()
+    assert positions.numel() == src_k.shape[1]
+    _check(lib().cb_means_accumulate_rope(ctx.handle, ctypes.byref(sv), ctypes.byref(tv),
+                                          ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                          ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
+                                          ctypes.c_void_p(means_ws.data_ptr()), ctypes.c_size_t(means_ws.numel()),
+                                          ctypes.c_void_p(positions.data_ptr()), ctypes.c_double(rope_base_src),
+                                          ctypes.c_double(rope_base_tgt), _stream_ptr(stream)), "cb_means_accumulate_rope")
+
+
 def cb_means_finalize(ctx: Context, means_ws: torch.Tensor, mu: torch.Tensor, stream=None) -> None:
     """mu: fp32 device [n_maps][2 d + 1] = mu_x, mu_y, s_w."""
     assert mu.dtype == torch.float32 and mu.is_contiguous() and mu.numel() == ctx.prob.n_maps * (2 * ctx.prob.ds + 1)
@@ -357,6 +376,23 @@ def cb_stats_accumulate_centered(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k: 
                                               ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
                                               ctypes.c_void_p(mu.data_ptr()), _stream_ptr(stream)),
            "cb_stats_accumulate_centered")
+
+
+def cb_stats_accumulate_centered_rope(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k: torch.Tensor, w_v: torch.Tensor,
+                                      mu: torch.Tensor, positions: torch.Tensor, rope_base_src: float, rope_base_tgt: float,
+                                      stream=None) -> None:
+    sv, tv = _kv_view(src_k, src_v), _kv_view(tgt_k, tgt_v)
+    assert w_k.dtype == torch.float32 and w_v.dtype == torch.float32 and w_k.dim() == 3
+    assert w_k.stride() == w_v.stride() and (w_k.stride(2) == 1 or w_k.shape[2] <= 1)
+    assert mu.dtype == torch.float32 and mu.is_contiguous() and mu.numel() == ctx.prob.n_maps * (2 * ctx.prob.ds + 1)
+    assert positions.dtype == torch.int32 and positions.is_cuda and positions.is_contiguous()
+    assert positions.numel() == src_k.shape[1]
+    _check(lib().cb_stats_accumulate_centered_rope(ctx.handle, ctypes.byref(sv), ctypes.byref(tv),
+                                                   ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
+                                                   ctypes.c_int64(w_k.stride(0)), ctypes.c_int64(w_k.stride(1)),
+                                                   ctypes.c_void_p(mu.data_ptr()), ctypes.c_void_p(positions.data_ptr()),
+                                                   ctypes.c_double(rope_base_src), ctypes.c_double(rope_base_tgt),
+                                                   _stream_ptr(stream)), "cb_stats_accumulate_centered_rope")
 
 
 def cb_stats_reduce_centered(ctx: Context, mu: torch.Tensor, A: torch.Tensor, B: torch.Tensor, stream=None) -> int:

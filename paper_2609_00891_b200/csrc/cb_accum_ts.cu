@@ -321,11 +321,27 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                 for (int c = 0; c < 2; ++c) {
                     sx2[g][c] = 0ull;
                     nmu2[g][c] = 0ull;
-                    if (CEN) {
+                    if (CEN && !rope_unit) {
                         const float mu = __ldg(a.mu + (size_t)m * (2 * D + 1) + q * 32 + 16 * g + 8 * c + (lane >> 2));
                         nmu2[g][c] = f2_pack(-mu, -mu);
                     }
                 }
+            // CEN && ROPE, key maps: the rotation phase stores the de-rotated rows ALREADY CENTRED (source and target), so
+            // that their rounding to bf16 is relative to the spread, not to the mean; the fold then has nothing to
+            // subtract and the reduction nothing to correct.  Negated means of this thread's channels in the rotation's
+            // layout: [source | target][pair pp] for the low and the high half of the head.
+            uint64_t rmlo[2][2] = {{0ull, 0ull}, {0ull, 0ull}}, rmhi[2][2] = {{0ull, 0ull}, {0ull, 0ull}};
+            if (CEN && rope_unit) {
+                const float *mup = a.mu + (size_t)m * (2 * D + 1);
+#pragma unroll
+                for (int xyi = 0; xyi < 2; ++xyi)
+#pragma unroll
+                    for (int pp = 0; pp < 2; ++pp) {
+                        const float *b = mup + xyi * D + rc * 4 + 2 * pp;
+                        rmlo[xyi][pp] = f2_pack(-__ldg(b), -__ldg(b + 1));
+                        rmhi[xyi][pp] = f2_pack(-__ldg(b + D / 2), -__ldg(b + D / 2 + 1));
+                    }
+            }
             for (int t = 0; t < n_t; ++t) {
                 if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, lane)) goto teardown;
                 // the operand buffer was last read by the MMAs of tile it - NA, which also release that tile's stage
@@ -387,8 +403,9 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                             for (int pp = 0; pp < 2; ++pp) {          // rotation by -phi
                                 const uint64_t c2 = xyi ? yc2[pp] : cc2[pp], s2 = xyi ? ys2[pp] : ss2[pp];
                                 const uint64_t l2 = f2_from_bf16x2(ul[pp]), h2 = f2_from_bf16x2(uh[pp]);
-                                const uint64_t nl = f2_fma(l2, c2, f2_mul(h2, s2));
-                                const uint64_t nh = f2_fma(h2, c2, f2_mul(f2_mul(l2, s2), neg1));
+                                uint64_t nl = f2_fma(l2, c2, f2_mul(h2, s2));
+                                uint64_t nh = f2_fma(h2, c2, f2_mul(f2_mul(l2, s2), neg1));
+                                if (CEN) { nl = f2_add(nl, rmlo[xyi][pp]); nh = f2_add(nh, rmhi[xyi][pp]); }
                                 float a0, a1;
                                 f2_unpack(nl, a0, a1); ol[pp] = pack_bf16x2(a0, a1);
                                 f2_unpack(nh, a0, a1); oh[pp] = pack_bf16x2(a0, a1);
@@ -590,7 +607,8 @@ cudaError_t launch_accum_ts(const AccumArgs &a, bool comp, const cb_kv_view *src
         rope_frequencies(a.rope_base_src, d, P.rope.f_src);
         rope_frequencies(a.rope_base_tgt, d, P.rope.f_tgt);
         P.rope.same = (a.rope_base_src == a.rope_base_tgt) ? 1 : 0;
-        e = comp ? launch_ts<true, false, true>(P, st) : launch_ts<false, false, true>(P, st);
+        if (a.mu) e = comp ? launch_ts<true, true, true>(P, st) : launch_ts<false, true, true>(P, st);
+        else e = comp ? launch_ts<true, false, true>(P, st) : launch_ts<false, false, true>(P, st);
     } else if (a.mu) e = comp ? launch_ts<true, true>(P, st) : launch_ts<false, true>(P, st);
     else e = comp ? launch_ts<true, false>(P, st) : launch_ts<false, false>(P, st);
     if (e == cudaSuccess) count_launch();

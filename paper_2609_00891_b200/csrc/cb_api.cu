@@ -114,6 +114,7 @@ struct cb_ctx {
     char *ws;
     Layout lay;
     long long n_tokens;
+    bool k_operands_centred;   // centred accumulation with the rotary boundary since the last reset (see cb_stats_reduce_centered)
 };
 
 extern "C" {
@@ -224,6 +225,7 @@ cb_status cb_create(const cb_problem *prob, void *workspace, size_t workspace_by
     c->ws = static_cast<char *>(workspace);
     c->lay = lay;
     c->n_tokens = 0;
+    c->k_operands_centred = false;
 
     std::vector<int32_t> tab(c->src_layer);
     tab.insert(tab.end(), c->src_head.begin(), c->src_head.end());
@@ -255,6 +257,7 @@ cb_status cb_stats_reset(cb_ctx *ctx, void *stream)
     if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + ctx->lay.status_off, 0, 256, st);
     if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     ctx->n_tokens = 0;
+    ctx->k_operands_centred = false;
     return CB_OK;
 }
 
@@ -276,6 +279,7 @@ static cb_status accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const cb_kv
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
     if (centred && !mu) return CB_ERR_INVALID_ARG;
     if (centred && (ctx->prob.flags & CB_FLAG_SIMT)) return CB_ERR_UNSUPPORTED;
+    if (centred && rope && ctx->d != 128) return CB_ERR_UNSUPPORTED;      // the combination exists for d = 128 only
     const cb_problem &P = ctx->prob;
     cb_status s = check_view(src, P.Ls, P.Hs, P.ds);
     if (s != CB_OK) return s;
@@ -307,6 +311,7 @@ static cb_status accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const cb_kv
                                              : launch_accum_tc(a, ctx->d, src, tgt, st);
     if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     ctx->n_tokens += src->n_tokens;
+    if (centred && rope) ctx->k_operands_centred = true;
     return CB_OK;
 }
 
@@ -372,11 +377,15 @@ cb_status cb_means_reset(cb_ctx *ctx, void *means_ws, size_t means_ws_bytes, voi
     return CB_OK;
 }
 
-cb_status cb_means_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
-                              const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
-                              void *means_ws, size_t means_ws_bytes, void *stream)
+static cb_status means_accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                       const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                                       void *means_ws, size_t means_ws_bytes, void *stream, const RopeOpt *rope)
 {
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (rope) {
+        if (!rope_base_ok(rope->base_src) || !rope_base_ok(rope->base_tgt)) return CB_ERR_INVALID_ARG;
+        if (src && src->n_tokens > 0 && (!rope->pos || ((uintptr_t)rope->pos & 3))) return CB_ERR_INVALID_ARG;
+    }
     const cb_problem &P = ctx->prob;
     cb_status s = check_view(src, P.Ls, P.Hs, P.ds);
     if (s != CB_OK) return s;
@@ -398,9 +407,26 @@ cb_status cb_means_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_vi
     a.src_layer = reinterpret_cast<const int *>(ctx->ws + ctx->lay.tab_off);
     a.src_head = a.src_layer + P.Lt;
     a.msum = static_cast<double *>(means_ws);
+    if (rope) { a.rope_pos = rope->pos; a.rope_base_src = rope->base_src; a.rope_base_tgt = rope->base_tgt; }
     cudaError_t e = launch_means(a, ctx->d, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     return CB_OK;
+}
+
+cb_status cb_means_accumulate(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                              const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                              void *means_ws, size_t means_ws_bytes, void *stream)
+{
+    return means_accumulate_impl(ctx, src, tgt, w_k, w_v, w_stride_layer, w_stride_head, means_ws, means_ws_bytes, stream, nullptr);
+}
+
+cb_status cb_means_accumulate_rope(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                   const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,
+                                   void *means_ws, size_t means_ws_bytes,
+                                   const int32_t *positions, double rope_base_src, double rope_base_tgt, void *stream)
+{
+    const RopeOpt r{positions, rope_base_src, rope_base_tgt};
+    return means_accumulate_impl(ctx, src, tgt, w_k, w_v, w_stride_layer, w_stride_head, means_ws, means_ws_bytes, stream, &r);
 }
 
 cb_status cb_means_finalize(cb_ctx *ctx, const void *means_ws, size_t means_ws_bytes, float *mu, void *stream)
@@ -479,12 +505,22 @@ cb_status cb_stats_accumulate_centered(cb_ctx *ctx, const cb_kv_view *src, const
     return accumulate_impl(ctx, src, tgt, w_k, w_v, w_stride_layer, w_stride_head, mu, true, stream);
 }
 
+cb_status cb_stats_accumulate_centered_rope(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
+                                            const float *w_k, const float *w_v,
+                                            int64_t w_stride_layer, int64_t w_stride_head, const float *mu,
+                                            const int32_t *positions, double rope_base_src, double rope_base_tgt, void *stream)
+{
+    const RopeOpt r{positions, rope_base_src, rope_base_tgt};
+    return accumulate_impl(ctx, src, tgt, w_k, w_v, w_stride_layer, w_stride_head, mu, true, stream, &r);
+}
+
 cb_status cb_stats_reduce_centered(cb_ctx *ctx, const float *mu, float *A, float *B, int64_t *n_tokens_out, void *stream)
 {
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
     if (!mu || !A || !B) return CB_ERR_INVALID_ARG;
     cudaError_t e = launch_reduce_centered(reinterpret_cast<const float *>(ctx->ws + ctx->lay.slots_off), ctx->n_splits,
-                                           ctx->n_maps, ctx->d, mu, A, B, static_cast<cudaStream_t>(stream));
+                                           ctx->n_maps, ctx->d, mu, A, B, ctx->k_operands_centred ? 1 : 0,
+                                           static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
     if (n_tokens_out) *n_tokens_out = ctx->n_tokens;
     return CB_OK;

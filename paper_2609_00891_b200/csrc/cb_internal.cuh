@@ -65,6 +65,10 @@ struct MeansArgs {
     const int *src_layer;  // device [Lt]
     const int *src_head;   // device [Ht]
     double *msum;          // device [MEANS_SPLITS][n_maps][means_stride(d)]
+    // Rotary embedding at the boundary: device [n_tokens] positions (null: keys as stored) and the models' bases; the
+    // key maps' sums are then those of the de-rotated rows.
+    const int *rope_pos = nullptr;
+    double rope_base_src = 0.0, rope_base_tgt = 0.0;
 };
 
 struct ApplyArgs {
@@ -109,7 +113,7 @@ cudaError_t launch_probe_r2(const float *G, const float *C, const float *Wb, con
                             double lambda, double inv_n, int raw_lambda, float *r2, cudaStream_t st);
 cudaError_t launch_probe_scores(const float *r2, int Lt, int Ht, const int *src_layer_host, int Ls, float *scores, cudaStream_t st);
 cudaError_t launch_reduce_centered(const float *slots, int n_splits, int n_maps, int d, const float *mu, float *A, float *B,
-                                   cudaStream_t st);
+                                   int k_operands_centred, cudaStream_t st);
 cudaError_t launch_solve_centered(const float *A, const float *B, const float *mu, int n_maps, int d, long long n_tokens,
                                   const float *lambdas, int n_lambda, unsigned flags, float *Wb, int *info, cudaStream_t st);
 cudaError_t launch_solve(const float *G, const float *C, int n_maps, int d, long long n_tokens,

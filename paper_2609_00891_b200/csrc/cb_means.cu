@@ -11,11 +11,16 @@
 //                      slot's s_x entries) the centred statistics are exactly
 //                          A = sum_t a_t (x_t - mu_x)^T = D_xx - r mu_x^T,   B = D_xy - r mu_y^T.
 #include "cb_internal.cuh"
+#include "cb_rope.cuh"
+#include "cb_math.cuh"
 
 namespace cb {
 
-template <int D>
-__global__ void __launch_bounds__(256) k_means(const MeansArgs a)
+// ROPE: key maps (comp = 0) sum the rows with the rotary embedding removed (Section 3.1): a thread also loads the
+// partner chunk of its eight channels (channel i pairs with i + D/2) and turns its own channels back by the row's angles
+// (in fp32; nothing is rounded before it is summed).
+template <int D, bool ROPE>
+__global__ void __launch_bounds__(256) k_means(const MeansArgs a, const RopeDev rope)
 {
     constexpr int CC = D / 8;            // 16-byte chunks per head row
     constexpr int RG = 256 / CC;         // row groups of the block
@@ -35,8 +40,9 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a)
 #pragma unroll
     for (int e = 0; e < 8; ++e) sx[e] = sy[e] = sq[e] = 0.f;
     for (int r0 = t0 + rg; r0 < t1; r0 += UN * RG) {
-        uint4 xv[UN], yv[UN];
+        uint4 xv[UN], yv[UN], xpv[UN], ypv[UN];
         float wt[UN];
+        int pv[UN];
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
             const int r = r0 + u * RG;
@@ -45,21 +51,46 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a)
             xv[u] = __ldg(reinterpret_cast<const uint4 *>(xs + (long long)rr * a.src.st));
             yv[u] = __ldg(reinterpret_cast<const uint4 *>(ys + (long long)rr * a.tgt.st));
             wt[u] = in ? __ldg(ws + rr) : 0.f;
+            if (ROPE && comp == 0) {
+                // partner chunk: + D/2 channels for the lower half of the head, - D/2 for the upper half
+                const int po = (cc < CC / 2) ? D / 2 : -(D / 2);
+                xpv[u] = __ldg(reinterpret_cast<const uint4 *>(xs + (long long)rr * a.src.st + po));
+                ypv[u] = __ldg(reinterpret_cast<const uint4 *>(ys + (long long)rr * a.tgt.st + po));
+                pv[u] = __ldg(rope.pos + rr);
+            }
         }
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
             const unsigned xu[4] = {xv[u].x, xv[u].y, xv[u].z, xv[u].w};
             const unsigned yu[4] = {yv[u].x, yv[u].y, yv[u].z, yv[u].w};
+            float fx[8], fy[8];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                sx[2 * e] = fmaf(wt[u], __uint_as_float(xu[e] << 16), sx[2 * e]);
-                sx[2 * e + 1] = fmaf(wt[u], __uint_as_float(xu[e] & 0xffff0000u), sx[2 * e + 1]);
-                const float y0 = __uint_as_float(yu[e] << 16), y1 = __uint_as_float(yu[e] & 0xffff0000u);
-                const float wy0 = wt[u] * y0, wy1 = wt[u] * y1;
-                sy[2 * e] += wy0;
-                sy[2 * e + 1] += wy1;
-                sq[2 * e] = fmaf(wy0, y0, sq[2 * e]);
-                sq[2 * e + 1] = fmaf(wy1, y1, sq[2 * e + 1]);
+                fx[2 * e] = __uint_as_float(xu[e] << 16); fx[2 * e + 1] = __uint_as_float(xu[e] & 0xffff0000u);
+                fy[2 * e] = __uint_as_float(yu[e] << 16); fy[2 * e + 1] = __uint_as_float(yu[e] & 0xffff0000u);
+            }
+            if (ROPE && comp == 0) {
+                // x~_i = x_i c + x_{i+h} s;  x~_{i+h} = x_{i+h} c - x_i s   (the embedding turned back, kept in fp32)
+                const float sgn = (cc < CC / 2) ? 1.f : -1.f;
+                const unsigned xq[4] = {xpv[u].x, xpv[u].y, xpv[u].z, xpv[u].w}, yq[4] = {ypv[u].x, ypv[u].y, ypv[u].z, ypv[u].w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int fi = (cc % (CC / 2)) * 8 + e;
+                    float cs, sn, ct, st;
+                    rope_cs(rope.f_src[fi], pv[u], cs, sn);
+                    if (rope.same) { ct = cs; st = sn; } else rope_cs(rope.f_tgt[fi], pv[u], ct, st);
+                    const float xb = (e & 1) ? __uint_as_float(xq[e >> 1] & 0xffff0000u) : __uint_as_float(xq[e >> 1] << 16);
+                    const float yb = (e & 1) ? __uint_as_float(yq[e >> 1] & 0xffff0000u) : __uint_as_float(yq[e >> 1] << 16);
+                    fx[e] = fmaf(fx[e], cs, sgn * xb * sn);
+                    fy[e] = fmaf(fy[e], ct, sgn * yb * st);
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                sx[e] = fmaf(wt[u], fx[e], sx[e]);
+                const float wy = wt[u] * fy[e];
+                sy[e] += wy;
+                sq[e] = fmaf(wy, fy[e], sq[e]);
             }
             sw += wt[u];
         }
@@ -80,8 +111,16 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a)
 cudaError_t launch_means(const MeansArgs &a, int d, cudaStream_t st)
 {
     dim3 grid(2 * a.Lt * a.Ht, MEANS_SPLITS);
-    if (d == 128) k_means<128><<<grid, 256, 0, st>>>(a);
-    else k_means<64><<<grid, 256, 0, st>>>(a);
+    RopeDev rope = RopeDev{};
+    if (a.rope_pos) {
+        rope.pos = a.rope_pos;
+        rope_frequencies(a.rope_base_src, d, rope.f_src);
+        rope_frequencies(a.rope_base_tgt, d, rope.f_tgt);
+        rope.same = (a.rope_base_src == a.rope_base_tgt) ? 1 : 0;
+        if (d == 128) k_means<128, true><<<grid, 256, 0, st>>>(a, rope);
+        else k_means<64, true><<<grid, 256, 0, st>>>(a, rope);
+    } else if (d == 128) k_means<128, false><<<grid, 256, 0, st>>>(a, rope);
+    else k_means<64, false><<<grid, 256, 0, st>>>(a, rope);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;
@@ -130,7 +169,7 @@ cudaError_t launch_means_finalize(const double *msum, int n_maps, int d, float *
 // Same split summation as the one-pass reduction, then the rank-one corrections and the symmetrisation of A.
 __global__ void __launch_bounds__(1024) k_reduce_centered(const float *__restrict__ slots, int n_splits, int n_maps, int d,
                                                          const float *__restrict__ mu, float *__restrict__ A,
-                                                         float *__restrict__ B)
+                                                         float *__restrict__ B, int k_operands_centred)
 {
     extern __shared__ __align__(16) float rs[];       // [d][2d + 1] sums of D, then [2d + 4] sums of r, -, s_w; then mu_x, mu_y
     const int m = blockIdx.x, n2 = 2 * d, pitch = 2 * d + 1;
@@ -138,7 +177,9 @@ __global__ void __launch_bounds__(1024) k_reduce_centered(const float *__restric
     const float *base = slots + (size_t)m * sf;
     const size_t sstride = (size_t)n_maps * sf;
     float *mus = rs + (size_t)d * pitch + 2 * d + 4;
-    for (int v = threadIdx.x; v < 2 * d; v += blockDim.x) mus[v] = mu[(size_t)m * (2 * d + 1) + v];
+    // key maps accumulated with the rotary boundary have both operands centred already: nothing to correct
+    const bool no_corr = k_operands_centred && m < n_maps / 2;
+    for (int v = threadIdx.x; v < 2 * d; v += blockDim.x) mus[v] = no_corr ? 0.f : mu[(size_t)m * (2 * d + 1) + v];
     for (int e4 = threadIdx.x; e4 < sf / 4; e4 += blockDim.x) {
         double v[4] = {0.0, 0.0, 0.0, 0.0};
         for (int s = 0; s < n_splits; ++s) {
@@ -166,7 +207,7 @@ __global__ void __launch_bounds__(1024) k_reduce_centered(const float *__restric
 }
 
 cudaError_t launch_reduce_centered(const float *slots, int n_splits, int n_maps, int d, const float *mu, float *A, float *B,
-                                   cudaStream_t st)
+                                   int k_operands_centred, cudaStream_t st)
 {
     const size_t smem = sizeof(float) * ((size_t)d * (2 * d + 1) + 2 * d + 4 + 2 * d);
     static bool attr[MAX_DEVICES] = {};
@@ -174,7 +215,7 @@ cudaError_t launch_reduce_centered(const float *slots, int n_splits, int n_maps,
         cudaError_t e = opt_in_smem(k_reduce_centered, (size_t)(140 * 1024), attr);
         if (e != cudaSuccess) return e;
     }
-    k_reduce_centered<<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, d, mu, A, B);
+    k_reduce_centered<<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, d, mu, A, B, k_operands_centred);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;

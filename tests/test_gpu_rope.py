@@ -307,3 +307,72 @@ def test_fused_statistics_few_rows_and_position_breaks(T):
     assert np.isfinite(Gc).all() and np.isfinite(Cc).all()
     # few rows: the bf16 rounding of the de-rotated second operand does not average out; bound it by its size
     assert max_rel_fro_per_map(Gc, Go) <= 4e-3 and max_rel_fro_per_map(Cc, Co) <= 4e-3
+
+
+@pytest.mark.parametrize("name,flags,bases", [("mid_scaled", 0, (1e6, 1e6)), ("mini_scaled", cb.CB_FLAG_COMPENSATED, (1e6, 1e4)),
+                                               ("mini_ragged", 0, (1e6, 1e6))])
+def test_two_pass_construction_in_content_coordinates(name, flags, bases):
+    """The paper's own construction path (Section 3.4: weighted means, centred statistics, centred solve) with the
+    rotary boundary (Section 3.1): both passes see the keys with the embedding removed.  The keys get a channel mean
+    far from zero in CONTENT coordinates (the case the two-pass path exists for) before they are stored rotated.
+    Expected values: the oracle's literal centred route on the de-rotated fp64 rows."""
+    wl = synth.workload(name)
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    law = synth.map_law(wl)
+    chunks = []
+    for c in range(wl.n_chunks):
+        ch = dict(synth.make_chunk(wl, c, sl, sh, law=law))
+        T = ch["n_tokens"]
+        pos = ((np.arange(T) + 11 * c) % 1024 + (20000 if c == 0 else 0)).astype(np.int32)
+        for k_, shift, base in (("src_k", 6.0, bases[0]), ("tgt_k", -3.0, bases[1])):
+            ch[k_] = _embed((ch[k_].float() + shift).to(torch.bfloat16), pos, base)
+        for k_, shift in (("src_v", 6.0), ("tgt_v", -3.0)):
+            ch[k_] = (ch[k_].float() + shift).to(torch.bfloat16)
+        ch["pos"] = pos
+        chunks.append(ch)
+    prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, flags=flags)
+    ctx = cb.cb_create(prob, device=DEV)
+    dev = [{k: (v.to(DEV) if torch.is_tensor(v) else torch.from_numpy(v).to(DEV)) for k, v in ch.items()
+            if torch.is_tensor(v) or isinstance(v, np.ndarray)} for ch in chunks]
+    ws = torch.empty(cb.cb_means_workspace_bytes(prob), dtype=torch.uint8, device=DEV)
+    cb.cb_means_reset(ctx, ws)
+    for t in dev:
+        cb.cb_means_accumulate_rope(ctx, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], t["w_k"], t["w_v"], ws, t["pos"], *bases)
+    d = wl.d
+    mu = torch.full((wl.n_maps, 2 * d + 1), float("nan"), device=DEV)
+    cb.cb_means_finalize(ctx, ws, mu)
+    cb.cb_stats_reset(ctx)
+    for t in dev:
+        cb.cb_stats_accumulate_centered_rope(ctx, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], t["w_k"], t["w_v"], mu,
+                                             t["pos"], *bases)
+    A = torch.full((wl.n_maps, d, d), float("nan"), device=DEV)
+    B = torch.full((wl.n_maps, d, d), float("nan"), device=DEV)
+    n = cb.cb_stats_reduce_centered(ctx, mu, A, B)
+    cb.cb_device_status(ctx)
+    assert n == wl.n_tokens
+    lam = 1e-2
+    Wb = torch.full((1, wl.n_maps, d + 1, d), float("nan"), device=DEV)
+    info = torch.full((1, wl.n_maps), -1, dtype=torch.int32, device=DEV)
+    cb.cb_ridge_solve_centered(A, B, mu, n, [lam], 0, Wb, info)
+    cb.cb_check_info(info)
+    muc, Wc = mu.cpu().numpy(), Wb[0].cpu().numpy()
+    n_maps = wl.n_maps
+    maps = sorted(set([0, 1, n_maps // 2 - 1, n_maps // 2, n_maps - 1]))
+    worst_mu = worst_w = 0.0
+    for m in maps:
+        comp, l, h = m // (wl.Lt * wl.Ht), (m // wl.Ht) % wl.Lt, m % wl.Ht
+        X = np.concatenate([oracle.bf16_decode(bits(ch["src_v" if comp else "src_k"][sl[l], :, sh[h], :])) for ch in chunks])
+        Y = np.concatenate([oracle.bf16_decode(bits(ch["tgt_v" if comp else "tgt_k"][l, :, h, :])) for ch in chunks])
+        w = np.concatenate([(ch["w_v"] if comp else ch["w_k"])[l, h].numpy().astype(np.float64) for ch in chunks])
+        if comp == 0:
+            pos = np.concatenate([ch["pos"] for ch in chunks])
+            X = oracle.rope_rotate(X, pos, bases[0], inverse=True)
+            Y = oracle.rope_rotate(Y, pos, bases[1], inverse=True)
+        To, io = oracle.ridge_centered(X, Y, w, lam)
+        mx, my = (w[:, None] * X).sum(0) / w.sum(), (w[:, None] * Y).sum(0) / w.sum()
+        worst_mu = max(worst_mu, rel_fro(muc[m, :d], mx), rel_fro(muc[m, d:2 * d], my))
+        worst_w = max(worst_w, rel_fro(Wc[m], To))
+        assert io == 0
+    print("%s two-pass + rotary boundary: means %.2e, fitted maps %.2e (worst of %d maps)" % (name, worst_mu, worst_w, len(maps)))
+    assert worst_mu <= 2e-5                  # fp32 sums of exactly de-rotated rows
+    assert worst_w <= (1e-3 if wl.n_tokens >= 4096 else 2.5e-3)
