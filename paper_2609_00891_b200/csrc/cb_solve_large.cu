@@ -109,9 +109,10 @@ __global__ void __launch_bounds__(128) k_lg_factor(LgArgs a, int J)
         const double ri = rinv[j];
         for (int i = j + 1 + tid; i < LNB; i += 128) Ld[i][j] *= ri;
         __syncthreads();
-        for (int e = tid; e < (LNB - j - 1) * (LNB - j - 1); e += 128) {
-            const int i = j + 1 + e / (LNB - j - 1), k = j + 1 + e % (LNB - j - 1);
-            if (k <= i) Ld[i][k] -= Ld[i][j] * Ld[k][j];
+        // trailing update, thread (ti, tk) of a 16 x 8 grid over (row, column): no index divisions in the loop
+        for (int i = j + 1 + (tid >> 3); i < LNB; i += 16) {
+            const double lij = Ld[i][j];
+            for (int k = j + 1 + (tid & 7); k <= i; k += 8) Ld[i][k] -= lij * Ld[k][j];
         }
         __syncthreads();
     }
