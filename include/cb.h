@@ -175,6 +175,19 @@ cb_status cb_stats_accumulate_host(cb_ctx *ctx, const cb_kv_view *src_host, cons
 cb_status cb_stats_reduce(cb_ctx *ctx, float *G, float *C, int64_t *n_tokens_out, void *stream);
 
 /*
+ * Checkpoint and resume of a streamed build (Section 3.4: statistics are sums over bounded blocks of observations, so
+ * the partial statistics ARE the state of the build).  cb_stats_export copies the partial slots of the context
+ * (cb_stats_state_bytes() bytes, fp32) to `dst`, device or host memory, on the stream and returns the number of rows
+ * accumulated so far; cb_stats_import replaces the context's state by such a copy (same problem shapes and the same
+ * number of token splits: the byte count must match, CB_ERR_INVALID_ARG otherwise) and sets the row count.
+ * Accumulation continues bit-identically after an import.  For the one-pass statistics; a two-pass build checkpoints
+ * its means workspace and mu the same way (they are plain caller-owned buffers).
+ */
+cb_status cb_stats_state_bytes(cb_ctx *ctx, size_t *bytes);
+cb_status cb_stats_export(cb_ctx *ctx, void *dst, size_t dst_bytes, int64_t *n_tokens_out, void *stream);
+cb_status cb_stats_import(cb_ctx *ctx, const void *src, size_t src_bytes, int64_t n_tokens, void *stream);
+
+/*
  * Batched closed-form ridge solve (Section 3.1, Eq. "closedform", written for the bias-column statistics):
  * for every lambda and map,  (G_m + lambda_eff J) Theta = C_m,  J = diag(1,..,1,0) (bias not penalised),
  * by Cholesky factorisation in fp64.  lambda_eff = lambda * s_w / n_tokens with s_w = G_m[d][d] (the paper

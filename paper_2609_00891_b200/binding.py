@@ -33,7 +33,7 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_stats_accumulate_rope", "cb_rope_rotate", "cb_apply_rope",
            "cb_means_accumulate_rope", "cb_stats_accumulate_centered_rope",
            "cb_means_energy", "cb_probe_r2", "cb_probe_scores", "cb_rank_layers",
-           "cb_last_device_status", "cb_test_hooks",
+           "cb_last_device_status", "cb_test_hooks", "cb_stats_state_bytes", "cb_stats_export", "cb_stats_import",
            "cb_launch_count")
 
 
@@ -224,6 +224,27 @@ def cb_stats_accumulate_host(ctx: Context, src_k, src_v, tgt_k, tgt_v, w_k, w_v,
                                           ctypes.c_void_p(w_k.data_ptr()), ctypes.c_void_p(w_v.data_ptr()),
                                           ctypes.c_void_p(staging.data_ptr()), ctypes.c_size_t(staging.numel()),
                                           _stream_ptr(stream)), "cb_stats_accumulate_host")
+
+
+def cb_stats_state_bytes(ctx: Context) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().cb_stats_state_bytes(ctx.handle, ctypes.byref(n)), "cb_stats_state_bytes")
+    return n.value
+
+
+def cb_stats_export(ctx: Context, dst: torch.Tensor, stream=None) -> int:
+    """Copies the partial statistics into `dst` (uint8 tensor, device or pinned/pageable host); returns the row count."""
+    assert dst.dtype == torch.uint8 and dst.is_contiguous()
+    n = ctypes.c_int64(0)
+    _check(lib().cb_stats_export(ctx.handle, ctypes.c_void_p(dst.data_ptr()), ctypes.c_size_t(dst.numel()), ctypes.byref(n),
+                                 _stream_ptr(stream)), "cb_stats_export")
+    return int(n.value)
+
+
+def cb_stats_import(ctx: Context, src: torch.Tensor, n_tokens: int, stream=None) -> None:
+    assert src.dtype == torch.uint8 and src.is_contiguous()
+    _check(lib().cb_stats_import(ctx.handle, ctypes.c_void_p(src.data_ptr()), ctypes.c_size_t(src.numel()),
+                                 ctypes.c_int64(n_tokens), _stream_ptr(stream)), "cb_stats_import")
 
 
 def cb_stats_reduce(ctx: Context, G: torch.Tensor, C: torch.Tensor, stream=None) -> int:

@@ -611,6 +611,40 @@ cb_status cb_stats_accumulate_host(cb_ctx *ctx, const cb_kv_view *src_host, cons
     return cb_stats_accumulate(ctx, &s, &t, wk, wv, (int64_t)P.Ht * T, T, stream);
 }
 
+cb_status cb_stats_state_bytes(cb_ctx *ctx, size_t *bytes)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (!bytes) return CB_ERR_INVALID_ARG;
+    *bytes = ctx->lay.slots_bytes;
+    return CB_OK;
+}
+
+cb_status cb_stats_export(cb_ctx *ctx, void *dst, size_t dst_bytes, int64_t *n_tokens_out, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (!dst || !n_tokens_out) return CB_ERR_INVALID_ARG;
+    if (dst_bytes < ctx->lay.slots_bytes) return CB_ERR_WORKSPACE;
+    cudaError_t e = cudaMemcpyAsync(dst, ctx->ws + ctx->lay.slots_off, ctx->lay.slots_bytes, cudaMemcpyDefault,
+                                    static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    *n_tokens_out = ctx->n_tokens;
+    return CB_OK;
+}
+
+cb_status cb_stats_import(cb_ctx *ctx, const void *src, size_t src_bytes, int64_t n_tokens, void *stream)
+{
+    if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
+    if (!src || n_tokens < 0) return CB_ERR_INVALID_ARG;
+    if (src_bytes != ctx->lay.slots_bytes) return CB_ERR_INVALID_ARG;      // a state of another problem or split count
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(ctx->ws + ctx->lay.slots_off, src, ctx->lay.slots_bytes, cudaMemcpyDefault, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + ctx->lay.status_off, 0, 256, st);
+    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    ctx->n_tokens = n_tokens;
+    ctx->k_operands_centred = false;
+    return CB_OK;
+}
+
 cb_status cb_stats_reduce(cb_ctx *ctx, float *G, float *C, int64_t *n_tokens_out, void *stream)
 {
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;

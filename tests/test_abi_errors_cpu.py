@@ -99,6 +99,15 @@ def test_static_entry_point_shares_the_argument_checks():
     assert call(ok_s, ok_t) == cb.CB_ERR_CUDA                                          # passes the checks; no device here
 
 
+def test_checkpoint_calls_reject_a_missing_context():
+    null = ctypes.c_void_p(0)
+    n = ctypes.c_size_t(0)
+    t = ctypes.c_int64(0)
+    assert cb.lib().cb_stats_state_bytes(null, ctypes.byref(n)) == cb.CB_ERR_STATE
+    assert cb.lib().cb_stats_export(null, ctypes.c_void_p(0x100), ctypes.c_size_t(64), ctypes.byref(t), null) == cb.CB_ERR_STATE
+    assert cb.lib().cb_stats_import(null, ctypes.c_void_p(0x100), ctypes.c_size_t(64), ctypes.c_int64(0), null) == cb.CB_ERR_STATE
+
+
 def test_status_calls_without_a_device():
     assert cb.lib().cb_last_device_status(ctypes.c_void_p(0)) == cb.CB_ERR_CUDA
     assert cb.lib().cb_test_hooks(ctypes.c_uint32(1 << 12), 1) == cb.CB_OK             # host state only

@@ -289,3 +289,47 @@ def test_token_subsampling_through_the_token_stride():
     cb.cb_device_status(ctx)
     assert n == dense["src_k"].shape[1]
     _check_stats(G, C, Go, Co)
+
+
+def test_checkpoint_and_resume_of_a_streamed_build():
+    """Export after the first chunk, import into a FRESH context (through host memory), continue: bitwise the statistics
+    of the uninterrupted build, and the same row count."""
+    wl = synth.workload("mini_ragged")
+    sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
+    law = synth.map_law(wl)
+    chunks = [{k: v.to(DEV) for k, v in synth.make_chunk(wl, c, sl, sh, law=law).items() if torch.is_tensor(v)}
+              for c in range(wl.n_chunks)]
+    prob = cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, n_splits=3)
+    p, d = wl.d + 1, wl.d
+
+    def acc(ctx, t):
+        cb.cb_stats_accumulate(ctx, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], t["w_k"], t["w_v"])
+
+    def reduce(ctx):
+        G = torch.empty(wl.n_maps, p, p, device=DEV)
+        C = torch.empty(wl.n_maps, p, d, device=DEV)
+        n = cb.cb_stats_reduce(ctx, G, C)
+        cb.cb_device_status(ctx)
+        return G, C, n
+
+    ref = cb.cb_create(prob, device=DEV)
+    for t in chunks:
+        acc(ref, t)
+    G0, C0, n0 = reduce(ref)
+    first = cb.cb_create(prob, device=DEV)
+    acc(first, chunks[0])
+    state = torch.empty(cb.cb_stats_state_bytes(first), dtype=torch.uint8)           # host memory
+    n1 = cb.cb_stats_export(first, state)
+    torch.cuda.synchronize()
+    assert n1 == chunks[0]["src_k"].shape[1]
+    second = cb.cb_create(prob, device=DEV)
+    cb.cb_stats_import(second, state, n1)
+    for t in chunks[1:]:
+        acc(second, t)
+    G1, C1, n2 = reduce(second)
+    assert n2 == n0 == wl.n_tokens
+    assert torch.equal(G0, G1) and torch.equal(C0, C1)
+    other = cb.cb_create(cb.Problem(wl.Ls, wl.Hs, wl.d, wl.Lt, wl.Ht, wl.d, sl, sh, n_splits=2), device=DEV)
+    with pytest.raises(cb.CbError) as e:
+        cb.cb_stats_import(other, state, n1)                                          # another split count: refused
+    assert e.value.status == cb.CB_ERR_INVALID_ARG
