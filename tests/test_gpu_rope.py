@@ -225,10 +225,12 @@ def test_apply_identity_map_turns_source_embedding_into_target_embedding():
             assert rel_fro(out_k[l, :, h, :].cpu().numpy(), src_k[sl[l], :, sh[h], :].float().numpy()) < 5e-4
 
 
-def test_rotary_boundary_for_k_selected_layers_by_composition():
+@pytest.mark.parametrize("name", ["mini_ragged", "mid_scaled"])
+def test_rotary_boundary_for_k_selected_layers_by_composition(name):
     """The paper's operating point (k > 1 selected layers, RoPE-aware interface) with the stand-alone rotation around
-    the wide-regressor calls: keys de-rotated in place, statistics over k layers, apply, target embedding restored."""
-    wl = synth.workload("mini_ragged")
+    the wide-regressor calls: keys de-rotated in place, statistics over k layers, apply, target embedding restored.
+    mid_scaled: 5,120 rows per map, where the stated 1e-3 holds for the statistics."""
+    wl = synth.workload(name)
     k, base_s, base_t = 2, 1e6, 1e4
     sl, sh = oracle.head_map(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
     sets = oracle.fullhead_layer_sets(wl.Ls, wl.Lt, k)
@@ -264,7 +266,8 @@ def test_rotary_boundary_for_k_selected_layers_by_composition():
         Go, Co = oracle.multilayer_stats(src_c, tgt_c, ch["w_k"][l, h].contiguous().numpy(), l, h, int(sh[h]), sets[l])
         eg, ec = rel_fro(G[m].cpu().numpy(), Go), rel_fro(C[m].cpu().numpy(), Co)
         print("k=%d with rope, map %d: G %.2e C %.2e" % (k, m, eg, ec))
-        assert eg <= 2.5e-3 and ec <= 2.5e-3                      # ~1,000 tokens per map: plain bf16 fold
+        tol = 1e-3 if T >= 4096 else 2.5e-3                       # ~1,000 tokens per map: the plain bf16 fold has not averaged out
+        assert eg <= tol and ec <= tol
     # apply: de-rotate the source cache, map, restore the target embedding
     rng = np.random.default_rng(3)
     Th = (rng.standard_normal((wl.n_maps, P, d)) / np.sqrt(k * d)).astype(np.float32)
