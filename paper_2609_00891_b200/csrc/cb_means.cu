@@ -5,6 +5,7 @@
 //                      Pure streaming (every source/target element and weight is read once per map that uses it),
 //                      bound by HBM; the reduction order is fixed: a thread sums its rows in token order, the row
 //                      groups of a block are combined in index order, the block adds to its own (split, map) entry.
+//   k_means_rope_keys  the same for key maps whose rows are first turned back by the rotary angles of their positions.
 //   k_means_finalize   sums the splits in index order (fp64) and divides by s_w.
 //   k_reduce_centered  second-pass reduction: the accumulate kernel multiplies the ROUNDED centred operand
 //                      a_t = bf16(w_t (x_t - mu_x)) with the uncentred [x_t | y_t]; with r = sum_t a_t (kept in the
@@ -16,18 +17,15 @@
 
 namespace cb {
 
-// ROPE: key maps (comp = 0) sum the rows with the rotary embedding removed (Section 3.1): a thread also loads the
-// partner chunk of its eight channels (channel i pairs with i + D/2) and turns its own channels back by the row's angles
-// (in fp32; nothing is rounded before it is summed).
-template <int D, bool ROPE>
-__global__ void __launch_bounds__(256) k_means(const MeansArgs a, const RopeDev rope)
+template <int D>
+__global__ void __launch_bounds__(256) k_means(const MeansArgs a, const int map_base)
 {
     constexpr int CC = D / 8;            // 16-byte chunks per head row
     constexpr int RG = 256 / CC;         // row groups of the block
     constexpr int UN = 4;                // rows in flight per thread
     __shared__ float red[RG][3 * D + 1];
     const int n_maps = 2 * a.Lt * a.Ht;
-    const int m = blockIdx.x, split = blockIdx.y;
+    const int m = map_base + blockIdx.x, split = blockIdx.y;
     const int comp = m / (a.Lt * a.Ht), l = (m / a.Ht) % a.Lt, h = m % a.Ht;
     const int t0 = (int)(((long long)a.n_tokens * split) / gridDim.y);
     const int t1 = (int)(((long long)a.n_tokens * (split + 1)) / gridDim.y);
@@ -40,9 +38,8 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a, const RopeDev 
 #pragma unroll
     for (int e = 0; e < 8; ++e) sx[e] = sy[e] = sq[e] = 0.f;
     for (int r0 = t0 + rg; r0 < t1; r0 += UN * RG) {
-        uint4 xv[UN], yv[UN], xpv[UN], ypv[UN];
+        uint4 xv[UN], yv[UN];
         float wt[UN];
-        int pv[UN];
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
             const int r = r0 + u * RG;
@@ -51,13 +48,6 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a, const RopeDev 
             xv[u] = __ldg(reinterpret_cast<const uint4 *>(xs + (long long)rr * a.src.st));
             yv[u] = __ldg(reinterpret_cast<const uint4 *>(ys + (long long)rr * a.tgt.st));
             wt[u] = in ? __ldg(ws + rr) : 0.f;
-            if (ROPE && comp == 0) {
-                // partner chunk: + D/2 channels for the lower half of the head, - D/2 for the upper half
-                const int po = (cc < CC / 2) ? D / 2 : -(D / 2);
-                xpv[u] = __ldg(reinterpret_cast<const uint4 *>(xs + (long long)rr * a.src.st + po));
-                ypv[u] = __ldg(reinterpret_cast<const uint4 *>(ys + (long long)rr * a.tgt.st + po));
-                pv[u] = __ldg(rope.pos + rr);
-            }
         }
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
@@ -68,22 +58,6 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a, const RopeDev 
             for (int e = 0; e < 4; ++e) {
                 fx[2 * e] = __uint_as_float(xu[e] << 16); fx[2 * e + 1] = __uint_as_float(xu[e] & 0xffff0000u);
                 fy[2 * e] = __uint_as_float(yu[e] << 16); fy[2 * e + 1] = __uint_as_float(yu[e] & 0xffff0000u);
-            }
-            if (ROPE && comp == 0) {
-                // x~_i = x_i c + x_{i+h} s;  x~_{i+h} = x_{i+h} c - x_i s   (the embedding turned back, kept in fp32)
-                const float sgn = (cc < CC / 2) ? 1.f : -1.f;
-                const unsigned xq[4] = {xpv[u].x, xpv[u].y, xpv[u].z, xpv[u].w}, yq[4] = {ypv[u].x, ypv[u].y, ypv[u].z, ypv[u].w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int fi = (cc % (CC / 2)) * 8 + e;
-                    float cs, sn, ct, st;
-                    rope_cs(rope.f_src[fi], pv[u], cs, sn);
-                    if (rope.same) { ct = cs; st = sn; } else rope_cs(rope.f_tgt[fi], pv[u], ct, st);
-                    const float xb = (e & 1) ? __uint_as_float(xq[e >> 1] & 0xffff0000u) : __uint_as_float(xq[e >> 1] << 16);
-                    const float yb = (e & 1) ? __uint_as_float(yq[e >> 1] & 0xffff0000u) : __uint_as_float(yq[e >> 1] << 16);
-                    fx[e] = fmaf(fx[e], cs, sgn * xb * sn);
-                    fy[e] = fmaf(fy[e], ct, sgn * yb * st);
-                }
             }
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -108,19 +82,126 @@ __global__ void __launch_bounds__(256) k_means(const MeansArgs a, const RopeDev 
     }
 }
 
+__device__ __forceinline__ void bf16x8_to_f32(const uint4 v, float (&f)[8])
+{
+    const unsigned u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { f[2 * e] = __uint_as_float(u[e] << 16); f[2 * e + 1] = __uint_as_float(u[e] & 0xffff0000u); }
+}
+
+// Key maps with the rotary embedding removed (Section 3.1): the sums are those of the de-rotated rows, turned back in
+// fp32 (nothing is rounded before it is summed).  Channel i pairs with i + D/2, so a thread takes chunk j of the lower
+// half AND chunk j + CC/2 of the upper half of its rows: the eight angles are evaluated once for the sixteen channels
+// they turn.  The two threads that share a chunk pair take alternate rows; their sums are added (lane exchange) before
+// the block's row groups are combined as in k_means.
+template <int D>
+__global__ void __launch_bounds__(256, 2) k_means_rope_keys(const MeansArgs a, const RopeDev rope)
+{
+    constexpr int CC = D / 8, HC = CC / 2;
+    constexpr int RG = 256 / CC;         // row groups of the block; each covers two rows per step
+    constexpr int UN = 2;                // rows in flight per thread
+    __shared__ float red[RG][3 * D + 1];
+    const int n_maps = 2 * a.Lt * a.Ht;
+    const int m = blockIdx.x, split = blockIdx.y;            // key maps are maps 0 .. Lt * Ht - 1
+    const int l = m / a.Ht, h = m % a.Ht;
+    const int t0 = (int)(((long long)a.n_tokens * split) / gridDim.y);
+    const int t1 = (int)(((long long)a.n_tokens * (split + 1)) / gridDim.y);
+    const int cc = threadIdx.x % CC, rg = threadIdx.x / CC, j = cc % HC, odd = cc / HC;
+    const __nv_bfloat16 *xs = a.src.k + (long long)a.src_layer[l] * a.src.sl + (long long)a.src_head[h] * a.src.sh + j * 8;
+    const __nv_bfloat16 *ys = a.tgt.k + (long long)l * a.tgt.sl + (long long)h * a.tgt.sh + j * 8;
+    const float *ws = a.w_k + (long long)l * a.w_sl + (long long)h * a.w_sh;
+    uint32_t fs[8], ft[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { fs[e] = rope.f_src[j * 8 + e]; ft[e] = rope.f_tgt[j * 8 + e]; }
+
+    float sxl[8], sxu[8], syl[8], syu[8], sql[8], squ[8], sw = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) sxl[e] = sxu[e] = syl[e] = syu[e] = sql[e] = squ[e] = 0.f;
+    // the trip count is the same for every thread of the block
+    for (int rb = t0; rb < t1; rb += UN * 2 * RG) {
+        uint4 xl[UN], xu[UN], yl[UN], yu[UN];
+        float wt[UN];
+        int pv[UN];
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const int r = rb + 2 * rg + odd + u * 2 * RG;
+            const bool in = r < t1;
+            const int rr = in ? r : t0;
+            xl[u] = __ldg(reinterpret_cast<const uint4 *>(xs + (long long)rr * a.src.st));
+            xu[u] = __ldg(reinterpret_cast<const uint4 *>(xs + (long long)rr * a.src.st + D / 2));
+            yl[u] = __ldg(reinterpret_cast<const uint4 *>(ys + (long long)rr * a.tgt.st));
+            yu[u] = __ldg(reinterpret_cast<const uint4 *>(ys + (long long)rr * a.tgt.st + D / 2));
+            wt[u] = in ? __ldg(ws + rr) : 0.f;
+            pv[u] = __ldg(rope.pos + rr);
+        }
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            float a0[8], a1[8], b0[8], b1[8];
+            bf16x8_to_f32(xl[u], a0); bf16x8_to_f32(xu[u], a1);
+            bf16x8_to_f32(yl[u], b0); bf16x8_to_f32(yu[u], b1);
+            const float w = wt[u];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                // x~_i = x_i c + x_{i+D/2} s;  x~_{i+D/2} = x_{i+D/2} c - x_i s
+                float c, s, ct, st;
+                rope_cs_poly(fs[e], pv[u], c, s);
+                if (rope.same) { ct = c; st = s; } else rope_cs_poly(ft[e], pv[u], ct, st);
+                const float x0 = fmaf(a0[e], c, a1[e] * s), x1 = fmaf(a1[e], c, -a0[e] * s);
+                const float y0 = fmaf(b0[e], ct, b1[e] * st), y1 = fmaf(b1[e], ct, -b0[e] * st);
+                sxl[e] = fmaf(w, x0, sxl[e]); sxu[e] = fmaf(w, x1, sxu[e]);
+                const float wy0 = w * y0, wy1 = w * y1;
+                syl[e] += wy0; syu[e] += wy1;
+                sql[e] = fmaf(wy0, y0, sql[e]); squ[e] = fmaf(wy1, y1, squ[e]);
+            }
+            sw += w;
+        }
+    }
+    // even rows + odd rows of the row group (the sum of two floats does not depend on which lane forms it)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        sxl[e] += __shfl_xor_sync(0xffffffffu, sxl[e], HC); sxu[e] += __shfl_xor_sync(0xffffffffu, sxu[e], HC);
+        syl[e] += __shfl_xor_sync(0xffffffffu, syl[e], HC); syu[e] += __shfl_xor_sync(0xffffffffu, syu[e], HC);
+        sql[e] += __shfl_xor_sync(0xffffffffu, sql[e], HC); squ[e] += __shfl_xor_sync(0xffffffffu, squ[e], HC);
+    }
+    sw += __shfl_xor_sync(0xffffffffu, sw, HC);
+    const int c0 = odd ? D / 2 + j * 8 : j * 8;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        red[rg][c0 + e] = odd ? sxu[e] : sxl[e];
+        red[rg][D + c0 + e] = odd ? syu[e] : syl[e];
+        red[rg][2 * D + 1 + c0 + e] = odd ? squ[e] : sql[e];
+    }
+    if (cc == 0) red[rg][2 * D] = sw;
+    __syncthreads();
+    double *dst = a.msum + ((size_t)split * n_maps + m) * means_stride(D);
+    for (int v = threadIdx.x; v < 3 * D + 1; v += 256) {
+        double sum = 0.0;
+#pragma unroll 4
+        for (int g = 0; g < RG; ++g) sum += (double)red[g][v];
+        dst[v] += sum;
+    }
+}
+
 cudaError_t launch_means(const MeansArgs &a, int d, cudaStream_t st)
 {
-    dim3 grid(2 * a.Lt * a.Ht, MEANS_SPLITS);
-    RopeDev rope = RopeDev{};
+    const int half = a.Lt * a.Ht;
     if (a.rope_pos) {
+        // key maps through the de-rotating kernel, value maps through the plain one
+        RopeDev rope = RopeDev{};
         rope.pos = a.rope_pos;
         rope_frequencies(a.rope_base_src, d, rope.f_src);
         rope_frequencies(a.rope_base_tgt, d, rope.f_tgt);
         rope.same = (a.rope_base_src == a.rope_base_tgt) ? 1 : 0;
-        if (d == 128) k_means<128, true><<<grid, 256, 0, st>>>(a, rope);
-        else k_means<64, true><<<grid, 256, 0, st>>>(a, rope);
-    } else if (d == 128) k_means<128, false><<<grid, 256, 0, st>>>(a, rope);
-    else k_means<64, false><<<grid, 256, 0, st>>>(a, rope);
+        dim3 grid(half, MEANS_SPLITS);
+        if (d == 128) { k_means_rope_keys<128><<<grid, 256, 0, st>>>(a, rope); k_means<128><<<grid, 256, 0, st>>>(a, half); }
+        else { k_means_rope_keys<64><<<grid, 256, 0, st>>>(a, rope); k_means<64><<<grid, 256, 0, st>>>(a, half); }
+        cudaError_t e = cudaGetLastError();
+        if (e == cudaSuccess) { count_launch(); count_launch(); }
+        return e;
+    }
+    dim3 grid(2 * half, MEANS_SPLITS);
+    if (d == 128) k_means<128><<<grid, 256, 0, st>>>(a, 0);
+    else k_means<64><<<grid, 256, 0, st>>>(a, 0);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;
