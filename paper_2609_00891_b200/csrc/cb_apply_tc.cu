@@ -31,7 +31,16 @@ namespace cb {
 
 using namespace ptx;
 
-template <int D>
+// Rotary kernels: eight epilogue warps (two sets of four, a set takes every other column group of a tile).  Measured on
+// the 32,768-token cache of the 14B -> 32B shapes, interleaved runs: 4 epilogue + 4 conversion warps 4.00 ms, 8 + 4
+// 3.79 ms, 4 + 8 4.80 ms, 8 + 8 4.02 ms (more conversion threads means shorter row blocks, so more first rows that
+// need the special-function unit); sending 4 or 8 of every 16 epilogue angles through the FMA-pipe polynomial
+// instead of the special-function unit: 4.0 / 4.4 ms.  With the epilogue's angles or the source rotation left out the
+// time falls by 0.3 - 0.5 ms each, with both left out to 3.0 ms (2.77 ms without the rotary boundary): the key maps'
+// tiles are bound by the sum of the two roles' instructions, not by one of them.
+constexpr int ROPE_EPI_WARPS = 8;
+
+template <int D, int EW = 4>
 struct ApCfg {
     static constexpr int TT = 128;                      // tokens per tile = MMA M
     static constexpr int NB = D / 64;                   // 64-channel blocks
@@ -45,7 +54,7 @@ struct ApCfg {
     static constexpr int NACC = 4;
     static constexpr int AW = D;                        // accumulator columns per tile: X W_hi + X W_lo
     static constexpr int TMEM_COLS = (NACC * AW < 32) ? 32 : NACC * AW;
-    static constexpr int EPI_WARPS = 4, CONV_WARPS = 4;
+    static constexpr int EPI_WARPS = EW, CONV_WARPS = 4;  // EW = 8: two sets of four, each takes every other column group
     static constexpr int THREADS = (2 + EPI_WARPS + CONV_WARPS) * 32;
     static constexpr size_t SMEM_BYTES = 1024 + (size_t)NS * X_BYTES + 2 * (size_t)W_BYTES + (size_t)NO * O_BYTES + D * 4 + 256;
 };
@@ -91,9 +100,9 @@ __device__ __forceinline__ unsigned ap_pack_f16x2(float lo, float hi)
 // tensor cores run with fp16 operands, and the epilogue rotates the mapped rows forward by the target model's angles.
 // Value maps take the ordinary bf16 path through the same barriers.
 template <int D, bool ROPE>
-__global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_constant__ ApParams P)
+__global__ void __launch_bounds__(ApCfg<D, ROPE ? ROPE_EPI_WARPS : 4>::THREADS, 1) k_apply_tc(const __grid_constant__ ApParams P)
 {
-    using C = ApCfg<D>;
+    using C = ApCfg<D, ROPE ? ROPE_EPI_WARPS : 4>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *xs = smem;                                   // [NS][X_BYTES]
@@ -211,6 +220,8 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         // ================================ epilogue warps ================================
         const int q = warp & 3;                 // tensor-memory lane quarter of this warp
         const int row = q * 32 + lane;          // token row inside the tile
+        constexpr int NSET = C::EPI_WARPS / 4;  // sets of four warps; a set takes the column groups c = set, set + NSET, ..
+        const int set = (warp - 2) >> 2;
         ApIter cur;
         cur.start(n_units, n_maps, n_tiles, P.n_splits);
         Ring<C::NACC> ac;
@@ -225,19 +236,21 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
             const CUtensorMap *omap = comp ? &P.out_v : &P.out_k;
             if (!mbar_wait_warp(wready, uc & 1, abort_flag, lane)) goto teardown;      // bias is in shared memory
             for (int tile = cur.tile; tile < cur.tile1; ++tile) {
+                const int tok = tile * C::TT + row;
+                const bool rope_unit = ROPE && comp == 0;
+                // the row's position is requested before the wait for the accumulator
+                int pos = 0;
+                if (rope_unit && tok < a.n_tokens) pos = __ldg(P.rope.pos + tok);
                 if (!mbar_wait_warp(&accfull[ac.idx], ac.phase, abort_flag, lane)) goto teardown;
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ac.idx * C::AW;
-                const int tok = tile * C::TT + row;
-                const bool rope_unit = ROPE && comp == 0;
                 if (rope_unit) {
                     // forward rotation by the target model's angles: columns i and i + D/2 are a pair
-                    const int pos = (tok < a.n_tokens) ? __ldg(P.rope.pos + tok) : 0;
                     uint8_t *ot = os + (size_t)ob.idx * C::O_BYTES;
                     float *orow = reinterpret_cast<float *>(a.out_k) + (long long)l * a.o_sl + (long long)tok * a.o_st + (long long)h * a.o_sh;
                     if (out_bf16 && !mbar_wait_warp(&ofree[ob.idx], ob.phase ^ 1, abort_flag, lane)) goto teardown;
 #pragma unroll 1
-                    for (int c = 0; c < D / 64; ++c) {
+                    for (int c = set; c < D / 64; c += NSET) {
                         uint32_t rl[32], rh[32];
                         {
                             tmem_ld_32x32(taddr + c * 32, rl);
@@ -297,7 +310,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                     uint8_t *ot = os + (size_t)ob.idx * C::O_BYTES;
                     if (!mbar_wait_warp(&ofree[ob.idx], ob.phase ^ 1, abort_flag, lane)) goto teardown;
 #pragma unroll 1
-                    for (int c = 0; c < D / 32; ++c) {
+                    for (int c = set; c < D / 32; c += NSET) {
                         uint32_t r[32];
                         {
                             tmem_ld_32x32(taddr + c * 32, r);
@@ -338,7 +351,7 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                     float *orow = reinterpret_cast<float *>(comp ? a.out_v : a.out_k) +
                                   (long long)l * a.o_sl + (long long)tok * a.o_st + (long long)h * a.o_sh;
 #pragma unroll 1
-                    for (int c = 0; c < D / 32; ++c) {
+                    for (int c = set; c < D / 32; c += NSET) {
                         uint32_t r[32];
                         {
                             tmem_ld_32x32(taddr + c * 32, r);
@@ -377,16 +390,21 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
         // ROPE: this thread rotates the pair of 16-byte chunks (lc, lc + half a row) of RB consecutive rows.  Along
         // consecutive positions the angle of a frequency advances by a fixed step, so (cos, sin) of the next row follow
         // from the current ones by one rotation with the thread's constants (cos, sin)(theta_i); the special-function
-        // unit is only needed at the first row and where the positions do not advance by one.
+        // unit is only needed at the first row and where the positions do not advance by one.  Packed fp32 pairs.
         constexpr int HC = D / 16, RB = C::TT / (CT / HC);
         const int lc = ct % HC, r0 = (ct / HC) * RB;
         uint32_t fsrc[8];
-        float stc[8], sts[8];
+        uint64_t stc2[4] = {0ull, 0ull, 0ull, 0ull}, sts2[4] = {0ull, 0ull, 0ull, 0ull}, nsts2[4] = {0ull, 0ull, 0ull, 0ull};
         if (ROPE) {
+            static_assert(RB <= HC, "the lanes that share a row block trade its positions");
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                fsrc[e] = P.rope.f_src[lc * 8 + e];
-                rope_cs(fsrc[e], 1, stc[e], sts[e]);
+            for (int e = 0; e < 8; ++e) fsrc[e] = P.rope.f_src[lc * 8 + e];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float c0, s0, c1, s1;
+                rope_cs(fsrc[2 * e], 1, c0, s0);
+                rope_cs(fsrc[2 * e + 1], 1, c1, s1);
+                stc2[e] = f2_pack(c0, c1); sts2[e] = f2_pack(s0, s1); nsts2[e] = f2_pack(-s0, -s1);
             }
         }
         while (cur.u < n_units) {
@@ -424,25 +442,36 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
             ++uc;
             if (ROPE) {
                 for (int tile = cur.tile; tile < cur.tile1; ++tile) {
+                    // the rows' positions are requested before the wait for the tile (their latency hides behind it):
+                    // the HC lanes that share the rows r0 .. r0 + RB - 1 load one position each and trade them below
+                    int mypos = 0;
+                    if (rope_unit) {
+                        const int tok = tile * C::TT + r0 + (lc < RB ? lc : 0);
+                        mypos = (tok < a.n_tokens) ? __ldg(P.rope.pos + tok) : 0;
+                    }
                     if (!mbar_wait_warp(&xfull[st.idx], st.phase, abort_flag, lane)) goto teardown;
                     if (rope_unit) {
                         uint8_t *xt = xs + st.idx * C::X_BYTES;
-                        float cs[8], sn[8];
+                        uint64_t cs2[4], sn2[4];           // packed pairs of frequencies (2 e, 2 e + 1)
                         int prev = 0;
 #pragma unroll 1
                         for (int i = 0; i < RB; ++i) {
                             const int r = r0 + i;
-                            const int tok = tile * C::TT + r;
-                            const int pos = (tok < a.n_tokens) ? __ldg(P.rope.pos + tok) : 0;
+                            const int pos = __shfl_sync(0xffffffffu, mypos, (lane & ~(HC - 1)) + i);
                             if (i == 0 || pos != prev + 1) {
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) rope_cs(fsrc[e], pos, cs[e], sn[e]);
+                                for (int e = 0; e < 4; ++e) {
+                                    float c0, s0, c1, s1;
+                                    rope_cs(fsrc[2 * e], pos, c0, s0);
+                                    rope_cs(fsrc[2 * e + 1], pos, c1, s1);
+                                    cs2[e] = f2_pack(c0, c1); sn2[e] = f2_pack(s0, s1);
+                                }
                             } else {
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    const float c1 = fmaf(cs[e], stc[e], -sn[e] * sts[e]);
-                                    sn[e] = fmaf(sn[e], stc[e], cs[e] * sts[e]);
-                                    cs[e] = c1;
+                                for (int e = 0; e < 4; ++e) {
+                                    const uint64_t c1 = f2_fma(cs2[e], stc2[e], f2_mul(sn2[e], nsts2[e]));
+                                    sn2[e] = f2_fma(sn2[e], stc2[e], f2_mul(cs2[e], sts2[e]));
+                                    cs2[e] = c1;
                                 }
                             }
                             prev = pos;
@@ -452,13 +481,16 @@ __global__ void __launch_bounds__(ApCfg<D>::THREADS, 1) k_apply_tc(const __grid_
                             const uint4 vh = *reinterpret_cast<const uint4 *>(xt + ohi);
                             const unsigned ul[4] = {vl.x, vl.y, vl.z, vl.w}, uh[4] = {vh.x, vh.y, vh.z, vh.w};
                             unsigned wl[4], wh[4];
+                            const uint64_t neg1 = f2_pack(-1.f, -1.f);
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                const float l0 = __uint_as_float(ul[e] << 16), l1 = __uint_as_float(ul[e] & 0xffff0000u);
-                                const float h0 = __uint_as_float(uh[e] << 16), h1 = __uint_as_float(uh[e] & 0xffff0000u);
-                                // rotation by -phi
-                                wl[e] = ap_pack_f16x2(fmaf(l0, cs[2 * e], h0 * sn[2 * e]), fmaf(l1, cs[2 * e + 1], h1 * sn[2 * e + 1]));
-                                wh[e] = ap_pack_f16x2(fmaf(h0, cs[2 * e], -l0 * sn[2 * e]), fmaf(h1, cs[2 * e + 1], -l1 * sn[2 * e + 1]));
+                                // rotation by -phi:  x~_i = x_i c + x_{i+D/2} s,  x~_{i+D/2} = x_{i+D/2} c - x_i s
+                                const uint64_t l2 = f2_from_bf16x2(ul[e]), h2 = f2_from_bf16x2(uh[e]);
+                                const uint64_t nl = f2_fma(l2, cs2[e], f2_mul(h2, sn2[e]));
+                                const uint64_t nh = f2_fma(h2, cs2[e], f2_mul(f2_mul(l2, sn2[e]), neg1));
+                                float a0, a1;
+                                f2_unpack(nl, a0, a1); wl[e] = ap_pack_f16x2(a0, a1);
+                                f2_unpack(nh, a0, a1); wh[e] = ap_pack_f16x2(a0, a1);
                             }
                             *reinterpret_cast<uint4 *>(xt + olo) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
                             *reinterpret_cast<uint4 *>(xt + ohi) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
@@ -494,7 +526,7 @@ teardown:
 template <int D, bool ROPE>
 static cudaError_t launch_ap(const ApParams &P, cudaStream_t st)
 {
-    using C = ApCfg<D>;
+    using C = ApCfg<D, ROPE ? ROPE_EPI_WARPS : 4>;
     static bool attr[MAX_DEVICES] = {};
     {
         cudaError_t e = opt_in_smem(k_apply_tc<D, ROPE>, (size_t)((int)C::SMEM_BYTES), attr);

@@ -31,14 +31,14 @@ inline void rope_frequencies(double base, int d, uint32_t *f)
 }
 
 #ifdef __CUDACC__
-// cos and sin of pos * f turns.  The top 23 bits of the wrapped product become the mantissa of a float in [1, 2):
-// subtracting 1.5 gives the angle minus half a turn, in [-0.5, 0.5) turns, without an integer-to-float conversion
-// (which would share the special-function unit with the sine and cosine); the half turn is undone by the signs.
+// cos and sin of pos * f turns.  The top 23 bits of the wrapped product become the mantissa of a float u in [1, 2):
+// (u - 1.5) 2 pi, in one fused multiply-add, is the angle minus half a turn, in [-pi, pi), without an integer-to-float
+// conversion (which would share the special-function unit with the sine and cosine); the half turn is undone by the
+// signs.
 __device__ __forceinline__ void rope_cs(uint32_t f, int pos, float &c, float &s)
 {
     const uint32_t wrapped = (uint32_t)pos * f;
-    const float t = __uint_as_float(0x3f800000u | (wrapped >> 9)) - 1.5f;
-    const float ang = t * 6.283185307179586f;
+    const float ang = fmaf(__uint_as_float(0x3f800000u | (wrapped >> 9)), 6.283185307179586f, -9.42477796076938f);
     c = -__cosf(ang);
     s = -__sinf(ang);
 }
