@@ -356,52 +356,44 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                     uint8_t *xt = xy + st.idx * C::STAGE_BYTES + rp_off;      // this thread's place in row rr of block 0
                     const int *pt = pst + st.idx * C::TT + rr;
                     const uint64_t neg1 = f2_pack(-1.f, -1.f);
+                    constexpr int NI = C::TT / 16;
+                    // positions of this thread's rows; `contig`: they advance by 16 from row to row (the common case:
+                    // no sequence boundary inside the tile), decided once so that the row loop has no branches
+                    int posv[NI];
+#pragma unroll
+                    for (int i = 0; i < NI; ++i) posv[i] = pt[16 * i];
+                    bool contig = true;
+#pragma unroll
+                    for (int i = 1; i < NI; ++i) contig = contig && (posv[i] == posv[0] + 16 * i);
                     uint64_t cc2[2], ss2[2];
-                    int curpos = 0;
+                    if ((t == 0) || (posv[0] != seedpos + C::TT) || ((t & 15) == 0)) {
 #pragma unroll
-                    for (int i = 0; i < C::TT / 16; ++i) {
-                        const int pos = pt[16 * i];
-                        bool fresh;
-                        if (i == 0) fresh = (t == 0) || (pos != seedpos + C::TT) || ((t & 15) == 0);
-                        else fresh = (pos != curpos + 16);
-                        if (fresh) {
-#pragma unroll
-                            for (int pp = 0; pp < 2; ++pp) {
-                                float c0, s0, c1, s1;
-                                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp], pos, c0, s0);
-                                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp + 1], pos, c1, s1);
-                                cc2[pp] = f2_pack(c0, c1); ss2[pp] = f2_pack(s0, s1);
-                            }
-                        } else {
-#pragma unroll
-                            for (int pp = 0; pp < 2; ++pp) {        // angle += (TT or 16) theta
-                                const uint64_t pc = (i == 0) ? seedc[pp] : cc2[pp], ps = (i == 0) ? seeds[pp] : ss2[pp];
-                                const uint64_t kc = (i == 0) ? rsTc[pp] : rs16c[pp], ks = (i == 0) ? rsTs[pp] : rs16s[pp];
-                                cc2[pp] = f2_fma(pc, kc, f2_mul(f2_mul(ps, ks), neg1));
-                                ss2[pp] = f2_fma(ps, kc, f2_mul(pc, ks));
-                            }
+                        for (int pp = 0; pp < 2; ++pp) {
+                            float c0, s0, c1, s1;
+                            rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp], posv[0], c0, s0);
+                            rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp + 1], posv[0], c1, s1);
+                            cc2[pp] = f2_pack(c0, c1); ss2[pp] = f2_pack(s0, s1);
                         }
-                        if (i == 0) { seedc[0] = cc2[0]; seedc[1] = cc2[1]; seeds[0] = ss2[0]; seeds[1] = ss2[1]; seedpos = pos; }
-                        curpos = pos;
-                        uint64_t yc2[2] = {cc2[0], cc2[1]}, ys2[2] = {ss2[0], ss2[1]};
-                        if (!P.rope.same) {
+                    } else {
 #pragma unroll
-                            for (int pp = 0; pp < 2; ++pp) {
-                                float c0, s0, c1, s1;
-                                rope_cs_poly(P.rope.f_tgt[rc * 4 + 2 * pp], pos, c0, s0);
-                                rope_cs_poly(P.rope.f_tgt[rc * 4 + 2 * pp + 1], pos, c1, s1);
-                                yc2[pp] = f2_pack(c0, c1); ys2[pp] = f2_pack(s0, s1);
-                            }
+                        for (int pp = 0; pp < 2; ++pp) {            // angle += TT theta
+                            cc2[pp] = f2_fma(seedc[pp], rsTc[pp], f2_mul(f2_mul(seeds[pp], rsTs[pp]), neg1));
+                            ss2[pp] = f2_fma(seeds[pp], rsTc[pp], f2_mul(seedc[pp], rsTs[pp]));
                         }
+                    }
+                    seedc[0] = cc2[0]; seedc[1] = cc2[1]; seeds[0] = ss2[0]; seeds[1] = ss2[1]; seedpos = posv[0];
+                    // rows rr + 16 i of the source tile, then of the target tile, turned back by (cc2, ss2) / (yc2, ys2)
+                    auto rotate_rows = [&](int i, const uint64_t (&xc)[2], const uint64_t (&xs)[2], const uint64_t (&yc)[2],
+                                           const uint64_t (&ys)[2]) {
 #pragma unroll
-                        for (int xyi = 0; xyi < 2; ++xyi) {           // source tile, then target tile
+                        for (int xyi = 0; xyi < 2; ++xyi) {
                             uint8_t *lo = xt + xyi * 2 * C::BLK + i * (16 * 128), *hi = lo + C::BLK;
                             const uint2 vl = *reinterpret_cast<const uint2 *>(lo), vh = *reinterpret_cast<const uint2 *>(hi);
                             const unsigned ul[2] = {vl.x, vl.y}, uh[2] = {vh.x, vh.y};
                             unsigned ol[2], oh[2];
 #pragma unroll
                             for (int pp = 0; pp < 2; ++pp) {          // rotation by -phi
-                                const uint64_t c2 = xyi ? yc2[pp] : cc2[pp], s2 = xyi ? ys2[pp] : ss2[pp];
+                                const uint64_t c2 = xyi ? yc[pp] : xc[pp], s2 = xyi ? ys[pp] : xs[pp];
                                 const uint64_t l2 = f2_from_bf16x2(ul[pp]), h2 = f2_from_bf16x2(uh[pp]);
                                 uint64_t nl = f2_fma(l2, c2, f2_mul(h2, s2));
                                 uint64_t nh = f2_fma(h2, c2, f2_mul(f2_mul(l2, s2), neg1));
@@ -412,6 +404,55 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                             }
                             *reinterpret_cast<uint2 *>(lo) = make_uint2(ol[0], ol[1]);
                             *reinterpret_cast<uint2 *>(hi) = make_uint2(oh[0], oh[1]);
+                        }
+                    };
+                    auto target_angles = [&](int pos, uint64_t (&yc)[2], uint64_t (&ys)[2]) {
+#pragma unroll
+                        for (int pp = 0; pp < 2; ++pp) {
+                            float c0, s0, c1, s1;
+                            rope_cs_poly(P.rope.f_tgt[rc * 4 + 2 * pp], pos, c0, s0);
+                            rope_cs_poly(P.rope.f_tgt[rc * 4 + 2 * pp + 1], pos, c1, s1);
+                            yc[pp] = f2_pack(c0, c1); ys[pp] = f2_pack(s0, s1);
+                        }
+                    };
+                    if (contig && P.rope.same) {
+#pragma unroll
+                        for (int i = 0; i < NI; ++i) {
+                            if (i > 0) {
+#pragma unroll
+                                for (int pp = 0; pp < 2; ++pp) {    // angle += 16 theta
+                                    const uint64_t pc = cc2[pp], ps = ss2[pp];
+                                    cc2[pp] = f2_fma(pc, rs16c[pp], f2_mul(f2_mul(ps, rs16s[pp]), neg1));
+                                    ss2[pp] = f2_fma(ps, rs16c[pp], f2_mul(pc, rs16s[pp]));
+                                }
+                            }
+                            rotate_rows(i, cc2, ss2, cc2, ss2);
+                        }
+                    } else {
+#pragma unroll 1
+                        for (int i = 0; i < NI; ++i) {
+                            const int pos = pt[16 * i];
+                            if (i > 0) {
+                                if (pos == pt[16 * (i - 1)] + 16) {
+#pragma unroll
+                                    for (int pp = 0; pp < 2; ++pp) {
+                                        const uint64_t pc = cc2[pp], ps = ss2[pp];
+                                        cc2[pp] = f2_fma(pc, rs16c[pp], f2_mul(f2_mul(ps, rs16s[pp]), neg1));
+                                        ss2[pp] = f2_fma(ps, rs16c[pp], f2_mul(pc, rs16s[pp]));
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int pp = 0; pp < 2; ++pp) {
+                                        float c0, s0, c1, s1;
+                                        rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp], pos, c0, s0);
+                                        rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp + 1], pos, c1, s1);
+                                        cc2[pp] = f2_pack(c0, c1); ss2[pp] = f2_pack(s0, s1);
+                                    }
+                                }
+                            }
+                            uint64_t yc2[2] = {cc2[0], cc2[1]}, ys2[2] = {ss2[0], ss2[1]};
+                            if (!P.rope.same) target_angles(pos, yc2, ys2);
+                            rotate_rows(i, cc2, ss2, yc2, ys2);
                         }
                     }
                     // every fold warp reads rows that other fold warps have just rewritten
