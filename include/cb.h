@@ -439,6 +439,13 @@ cb_status cb_device_status(cb_ctx *ctx, void *stream);
 cb_status cb_last_device_status(void *stream);
 
 /*
+ * The CUDA runtime's error code behind the most recent CB_ERR_CUDA that any call of this library returned (0 if none
+ * since the last call of this function), and, if `text` is not NULL, the runtime's description of it (a static
+ * string owned by the runtime).  Reading clears it.  The paper has no counterpart: error reporting only.
+ */
+int32_t cb_last_cuda_error(const char **text);
+
+/*
  * TEST HOOK, not for production use (the paper has no counterpart).  Affects every later launch of this process:
  * poll_limit > 0 shortens the number of polls after which a bounded device-side wait gives up (0 restores the
  * default of 2^22); starve_producer != 0 makes the source-tile producer of the statistics kernel (d = 128) and of

@@ -34,13 +34,17 @@ EXPORTS = ("cb_status_string", "cb_head_map_nearest", "cb_work_list", "cb_worksp
            "cb_means_accumulate_rope", "cb_stats_accumulate_centered_rope",
            "cb_means_energy", "cb_probe_r2", "cb_probe_scores", "cb_rank_layers",
            "cb_last_device_status", "cb_test_hooks", "cb_stats_state_bytes", "cb_stats_export", "cb_stats_import",
-           "cb_launch_count")
+           "cb_last_cuda_error", "cb_launch_count")
 
 
 class CbError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+        detail = ""
+        if status == CB_ERR_CUDA:
+            self.cuda_error, text = cb_last_cuda_error()
+            detail = ": CUDA error %d, %s" % (self.cuda_error, text)
+        super().__init__("%s: %s (status %d)%s" % (where, status_string(status), status, detail))
 
 
 class _KvView(ctypes.Structure):
@@ -76,6 +80,13 @@ def lib() -> ctypes.CDLL:
         L.cb_destroy.restype = None
         _lib = L
     return _lib
+
+
+def cb_last_cuda_error() -> Tuple[int, str]:
+    """(CUDA runtime error code, its description) behind the most recent CB_ERR_CUDA; (0, "no error") if none.  Clears it."""
+    text = ctypes.c_char_p()
+    code = lib().cb_last_cuda_error(ctypes.byref(text))
+    return int(code), (text.value or b"").decode()
 
 
 def status_string(status: int) -> str:

@@ -209,7 +209,7 @@ cb_status cb_create(const cb_problem *prob, void *workspace, size_t workspace_by
     const Layout lay = workspace_layout(prob->Lt, prob->Ht, prob->ds, n_splits);
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < lay.total) return CB_ERR_WORKSPACE;
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (cudaGetDevice(&dev) != cudaSuccess) { return cuda_failed(); }
 
     cb_ctx *c = new (std::nothrow) cb_ctx();
     if (!c) return CB_ERR_INVALID_ARG;
@@ -234,9 +234,9 @@ cb_status cb_create(const cb_problem *prob, void *workspace, size_t workspace_by
     if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + lay.status_off, 0, 256, 0);
     if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     if (e != cudaSuccess) {
-        cudaGetLastError();
+        const cb_status cf = cuda_failed(e);
         delete c;
-        return CB_ERR_CUDA;
+        return cf;
     }
     *out = c;
     return CB_OK;
@@ -255,7 +255,7 @@ cb_status cb_stats_reset(cb_ctx *ctx, void *stream)
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.slots_off, 0, ctx->lay.slots_bytes, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + ctx->lay.status_off, 0, 256, st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     ctx->n_tokens = 0;
     ctx->k_operands_centred = false;
     return CB_OK;
@@ -309,7 +309,7 @@ static cb_status accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const cb_kv
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = (P.flags & CB_FLAG_SIMT) ? launch_accum_simt(a, ctx->d, st)
                                              : launch_accum_tc(a, ctx->d, src, tgt, st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     ctx->n_tokens += src->n_tokens;
     if (centred && rope) ctx->k_operands_centred = true;
     return CB_OK;
@@ -347,7 +347,7 @@ cb_status cb_rope_rotate(void *k, int32_t n_layers, int32_t n_heads, int32_t hea
     if ((stride_layer | stride_token | stride_head) & 7) return CB_ERR_INVALID_ARG;
     cudaError_t e = launch_rope_rotate(k, n_layers, n_heads, head_dim, n_tokens, stride_layer, stride_token, stride_head,
                                        positions, rope_base, inverse ? 1 : 0, static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -373,7 +373,7 @@ cb_status cb_means_reset(cb_ctx *ctx, void *means_ws, size_t means_ws_bytes, voi
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
     if (!means_ws || ((uintptr_t)means_ws & 255) || means_ws_bytes < means_bytes(ctx)) return CB_ERR_WORKSPACE;
     cudaError_t e = cudaMemsetAsync(means_ws, 0, means_bytes(ctx), static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -409,7 +409,7 @@ static cb_status means_accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const
     a.msum = static_cast<double *>(means_ws);
     if (rope) { a.rope_pos = rope->pos; a.rope_base_src = rope->base_src; a.rope_base_tgt = rope->base_tgt; }
     cudaError_t e = launch_means(a, ctx->d, static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -436,7 +436,7 @@ cb_status cb_means_finalize(cb_ctx *ctx, const void *means_ws, size_t means_ws_b
     if (!mu) return CB_ERR_INVALID_ARG;
     cudaError_t e = launch_means_finalize(static_cast<const double *>(means_ws), ctx->n_maps, ctx->d, mu,
                                           static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -447,7 +447,7 @@ cb_status cb_means_energy(cb_ctx *ctx, const void *means_ws, size_t means_ws_byt
     if (!syy) return CB_ERR_INVALID_ARG;
     cudaError_t e = launch_means_energy(static_cast<const double *>(means_ws), ctx->n_maps, ctx->d, syy,
                                         static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -463,7 +463,7 @@ cb_status cb_probe_r2(const float *G, const float *C, const float *Wb, const flo
     if (n_maps == 0) return CB_OK;
     cudaError_t e = launch_probe_r2(G, C, Wb, syy, n_maps, d, (double)lambda, n_tokens > 0 ? 1.0 / (double)n_tokens : 0.0,
                                     (flags & CB_FLAG_RAW_LAMBDA) ? 1 : 0, r2, static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -475,7 +475,7 @@ cb_status cb_probe_scores(const float *r2, int32_t Lt, int32_t Ht, const int32_t
     for (int l = 0; l < Lt; ++l)
         if (src_layer[l] < 0 || src_layer[l] >= Ls) return CB_ERR_INVALID_ARG;
     cudaError_t e = launch_probe_scores(r2, Lt, Ht, src_layer, Ls, scores, static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -521,7 +521,7 @@ cb_status cb_stats_reduce_centered(cb_ctx *ctx, const float *mu, float *A, float
     cudaError_t e = launch_reduce_centered(reinterpret_cast<const float *>(ctx->ws + ctx->lay.slots_off), ctx->n_splits,
                                            ctx->n_maps, ctx->d, mu, A, B, ctx->k_operands_centred ? 1 : 0,
                                            static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     if (n_tokens_out) *n_tokens_out = ctx->n_tokens;
     return CB_OK;
 }
@@ -539,7 +539,7 @@ cb_status cb_ridge_solve_centered(const float *A, const float *B, const float *m
     if (n_maps == 0) return CB_OK;
     cudaError_t e = launch_solve_centered(A, B, mu, n_maps, d, n_tokens, lambdas, n_lambda, flags, Wb, info,
                                           static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -602,7 +602,7 @@ cb_status cb_stats_accumulate_host(cb_ctx *ctx, const cb_kv_view *src_host, cons
     if (e == cudaSuccess) e = cudaMemcpyAsync(dv + L.tgt_v, tgt_host->v, tb, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(dv + L.w_k, w_k_host, wb, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess && w_v_host != w_k_host) e = cudaMemcpyAsync(dv + L.w_v, w_v_host, wb, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     cb_kv_view s = *src_host, t = *tgt_host;
     s.k = dv + L.src_k; s.v = dv + L.src_v;
     t.k = dv + L.tgt_k; t.v = dv + L.tgt_v;
@@ -626,7 +626,7 @@ cb_status cb_stats_export(cb_ctx *ctx, void *dst, size_t dst_bytes, int64_t *n_t
     if (dst_bytes < ctx->lay.slots_bytes) return CB_ERR_WORKSPACE;
     cudaError_t e = cudaMemcpyAsync(dst, ctx->ws + ctx->lay.slots_off, ctx->lay.slots_bytes, cudaMemcpyDefault,
                                     static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     *n_tokens_out = ctx->n_tokens;
     return CB_OK;
 }
@@ -639,7 +639,7 @@ cb_status cb_stats_import(cb_ctx *ctx, const void *src, size_t src_bytes, int64_
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(ctx->ws + ctx->lay.slots_off, src, ctx->lay.slots_bytes, cudaMemcpyDefault, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + ctx->lay.status_off, 0, 256, st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     ctx->n_tokens = n_tokens;
     ctx->k_operands_centred = false;
     return CB_OK;
@@ -651,7 +651,7 @@ cb_status cb_stats_reduce(cb_ctx *ctx, float *G, float *C, int64_t *n_tokens_out
     if (!G || !C) return CB_ERR_INVALID_ARG;
     cudaError_t e = launch_reduce(reinterpret_cast<const float *>(ctx->ws + ctx->lay.slots_off), ctx->n_splits,
                                   ctx->n_maps, ctx->d, G, C, static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     if (n_tokens_out) *n_tokens_out = ctx->n_tokens;
     return CB_OK;
 }
@@ -669,7 +669,7 @@ cb_status cb_ridge_solve(const float *G, const float *C, int32_t n_maps, int32_t
     if (n_maps == 0) return CB_OK;
     cudaError_t e = launch_solve(G, C, n_maps, d, n_tokens, lambdas, n_lambda, flags, Wb, info,
                                  static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -694,7 +694,7 @@ cb_status cb_ridge_solve_large(const float *G, const float *C, int32_t n_maps, i
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < solve_large_bytes_per_system(P, d)) return CB_ERR_WORKSPACE;
     cudaError_t e = launch_solve_large(G, C, n_maps, P, d, n_tokens, lambdas, n_lambda, flags, Wb, info, workspace,
                                        workspace_bytes, static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -705,7 +705,7 @@ cb_status cb_check_info(const int32_t *info, int64_t n, void *stream, int64_t *f
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(h.data(), info, sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     for (int64_t i = 0; i < n; ++i)
         if (h[(size_t)i] != 0) {
             if (first_bad) *first_bad = i;
@@ -752,7 +752,7 @@ static cb_status apply_impl(const cb_problem *prob, const float *Wb, const cb_kv
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = (prob->flags & CB_FLAG_SIMT) ? launch_apply_simt(a, prob->ds, st)
                                                  : launch_apply_tc(a, prob->ds, src_cache, st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -836,10 +836,7 @@ cb_status cb_fullhead_stats_accumulate(const cb_fullhead_problem *prob, const cb
     tab.insert(tab.end(), gi.begin(), gi.end());
     tab.insert(tab.end(), gq.begin(), gq.end());
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(workspace, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
-        cudaGetLastError();
-        return CB_ERR_CUDA;
-    }
+    if (const cudaError_t ce = cudaMemcpyAsync(workspace, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st); ce != cudaSuccess) return cuda_failed(ce);
     AccumArgs a;
     a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src->k), static_cast<const __nv_bfloat16 *>(src->v),
                   src->stride_layer, src->stride_token, src->stride_head};
@@ -859,7 +856,7 @@ cb_status cb_fullhead_stats_accumulate(const cb_fullhead_problem *prob, const cb
     f.F = F; f.k = prob->k; f.Hs = prob->Hs; f.PF = F * prob->ds + 1; f.NG = NG; f.NC = F * prob->Ht;
     const cudaError_t e = ((prob->flags & CB_FLAG_ONE_ROW_HEAD) || prob->ds != 128) ? launch_fullhead_tc(a, f, prob->ds, src, tgt, st)
                                                                : launch_gram2_tc(a, f, prob->ds, src, tgt, st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -901,10 +898,7 @@ cb_status cb_multilayer_stats_accumulate(const cb_fullhead_problem *prob, const 
         for (int q = 0; 2 * q <= i; ++q) tab.push_back(q);
     tab.insert(tab.end(), src_head, src_head + prob->Ht);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(workspace, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
-        cudaGetLastError();
-        return CB_ERR_CUDA;
-    }
+    if (const cudaError_t ce = cudaMemcpyAsync(workspace, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st); ce != cudaSuccess) return cuda_failed(ce);
     AccumArgs a;
     a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src->k), static_cast<const __nv_bfloat16 *>(src->v),
                   src->stride_layer, src->stride_token, src->stride_head};
@@ -925,7 +919,7 @@ cb_status cb_multilayer_stats_accumulate(const cb_fullhead_problem *prob, const 
     f.F = F; f.k = prob->k; f.Hs = prob->Hs; f.PF = F * prob->ds + 1; f.NG = NG; f.NC = F;
     const cudaError_t e = ((prob->flags & CB_FLAG_ONE_ROW_HEAD) || prob->ds != 128) ? launch_fullhead_tc(a, f, prob->ds, src, tgt, st)
                                                                : launch_gram2_tc(a, f, prob->ds, src, tgt, st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }
 
@@ -972,10 +966,7 @@ cb_status cb_apply_multilayer(const cb_fullhead_problem *prob, const int32_t *sr
     std::memset(a.src_head, 0, sizeof a.src_head);
     for (int h = 0; h < prob->Ht; ++h) a.src_head[h] = src_head[h];
     fill_launch_state(a);
-    if (launch_apply_ml_tc(a, prob->ds, prob->k, prob->layer_sets, src_cache, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
-        cudaGetLastError();
-        return CB_ERR_CUDA;
-    }
+    if (const cudaError_t ce = launch_apply_ml_tc(a, prob->ds, prob->k, prob->layer_sets, src_cache, workspace, static_cast<cudaStream_t>(stream)); ce != cudaSuccess) return cuda_failed(ce);
     return CB_OK;
 }
 
@@ -986,7 +977,7 @@ cb_status cb_device_status(cb_ctx *ctx, void *stream)
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(&h, ctx->ws + ctx->lay.status_off, sizeof h, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return h == DEV_OK ? CB_OK : CB_ERR_TIMEOUT;
 }
 

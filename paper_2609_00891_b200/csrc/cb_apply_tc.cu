@@ -453,35 +453,39 @@ __global__ void __launch_bounds__(ApCfg<D, ROPE ? ROPE_EPI_WARPS : 4>::THREADS, 
                     if (rope_unit) {
                         uint8_t *xt = xs + st.idx * C::X_BYTES;
                         uint64_t cs2[4], sn2[4];           // packed pairs of frequencies (2 e, 2 e + 1)
-                        int prev = 0;
-#pragma unroll 1
-                        for (int i = 0; i < RB; ++i) {
-                            const int r = r0 + i;
-                            const int pos = __shfl_sync(0xffffffffu, mypos, (lane & ~(HC - 1)) + i);
-                            if (i == 0 || pos != prev + 1) {
+                        const uint64_t neg1 = f2_pack(-1.f, -1.f);
+                        int posv[RB];
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    float c0, s0, c1, s1;
-                                    rope_cs(fsrc[2 * e], pos, c0, s0);
-                                    rope_cs(fsrc[2 * e + 1], pos, c1, s1);
-                                    cs2[e] = f2_pack(c0, c1); sn2[e] = f2_pack(s0, s1);
-                                }
-                            } else {
+                        for (int i = 0; i < RB; ++i) posv[i] = __shfl_sync(0xffffffffu, mypos, (lane & ~(HC - 1)) + i);
+                        // decided once per tile, so that the row loop of the common case is straight-line code
+                        bool contig = true;
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const uint64_t c1 = f2_fma(cs2[e], stc2[e], f2_mul(sn2[e], nsts2[e]));
-                                    sn2[e] = f2_fma(sn2[e], stc2[e], f2_mul(cs2[e], sts2[e]));
-                                    cs2[e] = c1;
-                                }
+                        for (int i = 1; i < RB; ++i) contig = contig && (posv[i] == posv[0] + i);
+                        contig = __all_sync(0xffffffffu, contig);      // one path per warp: the general one trades lanes
+                        auto first_angles = [&](int pos) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                float c0, s0, c1, s1;
+                                rope_cs(fsrc[2 * e], pos, c0, s0);
+                                rope_cs(fsrc[2 * e + 1], pos, c1, s1);
+                                cs2[e] = f2_pack(c0, c1); sn2[e] = f2_pack(s0, s1);
                             }
-                            prev = pos;
+                        };
+                        auto next_angles = [&]() {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const uint64_t c1 = f2_fma(cs2[e], stc2[e], f2_mul(sn2[e], nsts2[e]));
+                                sn2[e] = f2_fma(sn2[e], stc2[e], f2_mul(cs2[e], sts2[e]));
+                                cs2[e] = c1;
+                            }
+                        };
+                        auto rotate_row = [&](int r) {
                             const int olo = r * 128 + ((lc ^ (r & 7)) << 4);
                             const int ohi = (D == 128) ? C::XBLK + olo : r * 128 + (((lc + 4) ^ (r & 7)) << 4);
                             const uint4 vl = *reinterpret_cast<const uint4 *>(xt + olo);
                             const uint4 vh = *reinterpret_cast<const uint4 *>(xt + ohi);
                             const unsigned ul[4] = {vl.x, vl.y, vl.z, vl.w}, uh[4] = {vh.x, vh.y, vh.z, vh.w};
                             unsigned wl[4], wh[4];
-                            const uint64_t neg1 = f2_pack(-1.f, -1.f);
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 // rotation by -phi:  x~_i = x_i c + x_{i+D/2} s,  x~_{i+D/2} = x_{i+D/2} c - x_i s
@@ -494,6 +498,24 @@ __global__ void __launch_bounds__(ApCfg<D, ROPE ? ROPE_EPI_WARPS : 4>::THREADS, 
                             }
                             *reinterpret_cast<uint4 *>(xt + olo) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
                             *reinterpret_cast<uint4 *>(xt + ohi) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                        };
+                        first_angles(posv[0]);
+                        if (contig) {
+#pragma unroll
+                            for (int i = 0; i < RB; ++i) {
+                                if (i > 0) next_angles();
+                                rotate_row(r0 + i);
+                            }
+                        } else {
+                            rotate_row(r0);
+#pragma unroll 1
+                            for (int i = 1; i < RB; ++i) {
+                                const int pos = __shfl_sync(0xffffffffu, mypos, (lane & ~(HC - 1)) + i);
+                                const int prev = __shfl_sync(0xffffffffu, mypos, (lane & ~(HC - 1)) + i - 1);
+                                if (pos == prev + 1) next_angles();
+                                else first_angles(pos);
+                                rotate_row(r0 + i);
+                            }
                         }
                         fence_async_smem();
                     }

@@ -77,10 +77,7 @@ extern "C" cb_status cb_ess_weights(const float *r_raw, int32_t n_rows, int64_t 
     if (!r_raw || !w || n_rows < 0 || n_tokens <= 0 || p_width <= 0) return CB_ERR_INVALID_ARG;
     if (r_row_stride < n_tokens || w_row_stride < n_tokens) return CB_ERR_INVALID_ARG;
     if (n_rows == 0) return CB_OK;
-    if (cb::launch_ess(r_raw, n_rows, n_tokens, r_row_stride, p_width, w, w_row_stride, alpha_out,
-                       static_cast<cudaStream_t>(stream)) != cudaSuccess) {
-        cudaGetLastError();
-        return CB_ERR_CUDA;
-    }
+    if (const cudaError_t ce = cb::launch_ess(r_raw, n_rows, n_tokens, r_row_stride, p_width, w, w_row_stride, alpha_out,
+                       static_cast<cudaStream_t>(stream)); ce != cudaSuccess) return cb::cuda_failed(ce);
     return CB_OK;
 }

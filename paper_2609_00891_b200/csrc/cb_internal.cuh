@@ -152,6 +152,10 @@ int device_sm_count();
 // Device address, on the current device, of the library's own status word: kernels launched without a context
 // record a device-side time-out there and cb_last_device_status reads it.  Null if the lookup failed.
 int *library_status_word();
+// A CUDA runtime call failed: remembers its error code for cb_last_cuda_error (`e`, or the runtime's last error when
+// the caller has none), clears the runtime's last-error state and returns CB_ERR_CUDA.
+cb_status cuda_failed(cudaError_t e = cudaSuccess);
+
 // Test hooks (cb_test_hooks): poll limit of the bounded waits and the starved-producer switch for later launches.
 struct TestHooks { unsigned poll_limit; int starve; };
 TestHooks test_hooks();

@@ -65,7 +65,7 @@ extern "C" cb_status cb_stats_build_static(const cb_problem *prob, const cb_kv_v
     if (end_off + 256 > STATIC_SCRATCH_BYTES) return CB_ERR_STATIC_LIMIT;
 
     unsigned char *base = nullptr;
-    if (static_scratch_address(&base) != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (static_scratch_address(&base) != cudaSuccess) { return cuda_failed(); }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the array keeps whatever the previous call left: everything that must start at zero is cleared here
     cudaError_t e = cudaMemsetAsync(base, 0, slots_bytes, st);
@@ -73,7 +73,7 @@ extern "C" cb_status cb_stats_build_static(const cb_problem *prob, const cb_kv_v
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(base + tab_off + sizeof(int) * (size_t)prob->Lt, prob->src_head, sizeof(int) * (size_t)prob->Ht,
                             cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
 
     AccumArgs a;
     a.src = KVPtr{static_cast<const __nv_bfloat16 *>(src->k), static_cast<const __nv_bfloat16 *>(src->v),
@@ -92,6 +92,6 @@ extern "C" cb_status cb_stats_build_static(const cb_problem *prob, const cb_kv_v
     a.compensated = (prob->flags & CB_FLAG_COMPENSATED) ? 1 : 0;
     e = (prob->flags & CB_FLAG_SIMT) ? launch_accum_simt(a, d, st) : launch_accum_tc(a, d, src, tgt, st);
     if (e == cudaSuccess) e = launch_reduce(a.slots, n_splits, (int)n_maps, d, G, C, st);
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return CB_OK;
 }

@@ -53,6 +53,17 @@ int *library_status_word()
 
 TestHooks test_hooks() { return TestHooks{g_poll_limit.load(), g_starve.load()}; }
 
+static std::atomic<int> g_last_cuda_error{0};
+
+cb_status cuda_failed(cudaError_t e)
+{
+    const cudaError_t last = cudaGetLastError();     // also clears the runtime's (non-sticky) last-error state
+    if (e == cudaSuccess) e = last;
+    if (e == cudaSuccess) e = cudaErrorUnknown;
+    g_last_cuda_error.store((int)e);
+    return CB_ERR_CUDA;
+}
+
 }  // namespace cb
 
 using namespace cb;
@@ -60,7 +71,7 @@ using namespace cb;
 extern "C" cb_status cb_last_device_status(void *stream)
 {
     int *w = library_status_word();
-    if (!w) return CB_ERR_CUDA;
+    if (!w) return cuda_failed(cudaErrorNoDevice);      // no current device, or its symbol address was refused
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int h = 0;
     cudaError_t e = cudaMemcpyAsync(&h, w, sizeof h, cudaMemcpyDeviceToHost, st);
@@ -68,7 +79,7 @@ extern "C" cb_status cb_last_device_status(void *stream)
         e = cudaMemsetAsync(w, 0, sizeof h, st);
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     }
-    if (e != cudaSuccess) { cudaGetLastError(); return CB_ERR_CUDA; }
+    if (e != cudaSuccess) return cuda_failed(e);
     return h == DEV_OK ? CB_OK : CB_ERR_TIMEOUT;
 }
 
@@ -77,4 +88,11 @@ extern "C" cb_status cb_test_hooks(uint32_t poll_limit, int32_t starve_producer)
     g_poll_limit.store(poll_limit ? poll_limit : (1u << 22));
     g_starve.store(starve_producer ? 1 : 0);
     return CB_OK;
+}
+
+extern "C" int32_t cb_last_cuda_error(const char **text)
+{
+    const int e = g_last_cuda_error.exchange(0);
+    if (text) *text = e ? cudaGetErrorString(static_cast<cudaError_t>(e)) : "no error";
+    return e;
 }

@@ -108,6 +108,20 @@ def test_checkpoint_calls_reject_a_missing_context():
     assert cb.lib().cb_stats_import(null, ctypes.c_void_p(0x100), ctypes.c_size_t(64), ctypes.c_int64(0), null) == cb.CB_ERR_STATE
 
 
+def test_cuda_failures_carry_the_runtime_error_code():
+    cb.cb_last_cuda_error()                                                           # clear whatever earlier tests left
+    assert cb.cb_last_cuda_error() == (0, "no error")
+    sl, sh = cb.cb_head_map_nearest(2, 2, 2, 2)
+    prob = cb.Problem(2, 2, 64, 2, 2, 64, sl, sh)
+    assert _apply(prob, _view(2, 2, 64, 64)) == cb.CB_ERR_CUDA                        # no device on this machine
+    code, text = cb.cb_last_cuda_error()
+    assert code != 0 and text and text != "no error"
+    assert cb.cb_last_cuda_error() == (0, "no error")                                 # reading cleared it
+    with pytest.raises(cb.CbError) as e:
+        cb._check(cb.lib().cb_last_device_status(ctypes.c_void_p(0)), "cb_last_device_status")
+    assert e.value.status == cb.CB_ERR_CUDA and e.value.cuda_error != 0 and "CUDA error" in str(e.value)
+
+
 def test_status_calls_without_a_device():
     assert cb.lib().cb_last_device_status(ctypes.c_void_p(0)) == cb.CB_ERR_CUDA
     assert cb.lib().cb_test_hooks(ctypes.c_uint32(1 << 12), 1) == cb.CB_OK             # host state only
