@@ -374,8 +374,7 @@ cb_status cb_rope_rotate(void *k, int32_t n_layers, int32_t n_heads, int32_t hea
  * on chip as in cb_stats_accumulate_rope AND centred there (source and target), so that their rounding to bf16 is
  * relative to the spread of a channel, not to its mean.  Same call order as the plain two-pass path, same positions and
  * bases in both passes; between two resets either every chunk goes through the _rope call or none does (the context
- * remembers which, and cb_stats_reduce_centered skips the key maps' mean correction accordingly).  d = 128 only
- * (CB_ERR_UNSUPPORTED otherwise); the means pass supports both head widths.
+ * remembers which, and cb_stats_reduce_centered skips the key maps' mean correction accordingly).  Both head widths.
  */
 cb_status cb_means_accumulate_rope(cb_ctx *ctx, const cb_kv_view *src, const cb_kv_view *tgt,
                                    const float *w_k, const float *w_v, int64_t w_stride_layer, int64_t w_stride_head,

@@ -1,5 +1,7 @@
-// Head-local weighted statistics (d = 128) with the weighted operand in TENSOR MEMORY and the bias sum s_y on the
-// tensor cores; plain, compensated, centred (two-pass) and rotary-boundary variants.
+// Head-local weighted statistics with the weighted operand in TENSOR MEMORY and the bias sum s_y on the tensor
+// cores; plain, compensated, centred (two-pass) and rotary-boundary variants.  Written for 128-wide heads; a 64-wide
+// head runs as a 128-wide one whose upper 64-channel block lies outside the tensor (the tile copies deliver it as
+// zeros), and only the results of the real channels are written out.
 //
 // Same contraction as the shared-memory kernel (D[d][2d] = (w .* X)^T [X | Y] over tokens plus the bias sums), same
 // units, slots and summation order of the splits.  What differs is where the first MMA operand lives: the fold warps
@@ -73,6 +75,9 @@ struct TsParams {
     CUtensorMap src_k, src_v, tgt_k, tgt_v;   // 5-D tiled maps: (64 channels, token, channel block, head, layer)
     AccumArgs a;
     int drain_tiles;                          // tiles accumulated in tensor memory between drains
+    int d;                                    // the heads' real width, 128 or 64.  A 64-wide head runs as a 128-wide one
+                                              // whose upper channel block lies outside the tensor (the tile copies fill
+                                              // it with zeros); only the results of the real channels leave the kernel.
     RopeDev rope;                             // ROPE kernels only
 };
 
@@ -115,7 +120,8 @@ struct UnitIter {
 // ROPE: key maps (comp = 0) are fitted in content coordinates (Section 3.1): before the fold proper, the fold warps
 // rotate every source and target key row of the staged tile back by its position's angles IN PLACE (the tensor cores
 // read the de-rotated rows as the second operand and for s_y); value maps take the ordinary path.
-template <bool COMP, bool CEN, bool ROPE>
+// NARROW (ROPE kernels, 64-wide heads): the rotation pairs channel i with i + 32 inside the first 64-channel block.
+template <bool COMP, bool CEN, bool ROPE, bool NARROW = false>
 __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __grid_constant__ TsParams P)
 {
     using C = TsCfg<COMP>;
@@ -140,6 +146,7 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const AccumArgs &a = P.a;
+    const int dr = P.d;                    // real head width: channels dr .. D - 1 are zero padding
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_maps = 2 * a.Lt * a.Ht;
     const int n_units = n_maps * a.n_splits;
@@ -287,17 +294,23 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
         // tile to tile by TT, so (cos, sin) follow from the previous ones by one rotation with the thread's constants;
         // the polynomial is needed at the first tile of a unit, where positions break, and every 16th tile (drift).
         // Packed fp32 pairs: frequencies (4 rc, 4 rc + 1) and (4 rc + 2, 4 rc + 3).
-        const int rc = (tid - 64) & 15, rr = (tid - 64) >> 4;
+        // A 64-wide head pairs channel i with i + 32, both in the tile's first 64-channel block (the second one is zero
+        // padding): eight threads per row instead of sixteen, so a pass covers 32 rows and there are half as many
+        // passes; in the swizzled row the partner chunk is the own one with address bit 6 flipped.
+        static_assert(ROPE || !NARROW, "NARROW selects the rotation's pairing");
+        constexpr bool narrow = NARROW;
+        const int rc = narrow ? (tid - 64) & 7 : (tid - 64) & 15, rr = narrow ? (tid - 64) >> 3 : (tid - 64) >> 4;
+        constexpr int rstep = narrow ? 32 : 16;                     // rows (and positions) between a thread's passes
         const int rp_off = rr * 128 + (((rc >> 1) ^ (rr & 7)) << 4) + (rc & 1) * 8;
-        uint64_t rs16c[2] = {0ull, 0ull}, rs16s[2] = {0ull, 0ull}, rsTc[2] = {0ull, 0ull}, rsTs[2] = {0ull, 0ull};   // cos, sin of 16 theta, TT theta
+        uint64_t rs16c[2] = {0ull, 0ull}, rs16s[2] = {0ull, 0ull}, rsTc[2] = {0ull, 0ull}, rsTs[2] = {0ull, 0ull};   // cos, sin of rstep theta, TT theta
         uint64_t seedc[2] = {0ull, 0ull}, seeds[2] = {0ull, 0ull};
         int seedpos = 0;
         if (ROPE) {
 #pragma unroll
             for (int pp = 0; pp < 2; ++pp) {
                 float c0, s0, c1, s1;
-                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp], 16, c0, s0);
-                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp + 1], 16, c1, s1);
+                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp], rstep, c0, s0);
+                rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp + 1], rstep, c1, s1);
                 rs16c[pp] = f2_pack(c0, c1); rs16s[pp] = f2_pack(s0, s1);
                 rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp], C::TT, c0, s0);
                 rope_cs_poly(P.rope.f_src[rc * 4 + 2 * pp + 1], C::TT, c1, s1);
@@ -322,7 +335,8 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                     sx2[g][c] = 0ull;
                     nmu2[g][c] = 0ull;
                     if (CEN && !rope_unit) {
-                        const float mu = __ldg(a.mu + (size_t)m * (2 * D + 1) + q * 32 + 16 * g + 8 * c + (lane >> 2));
+                        const int ch = q * 32 + 16 * g + 8 * c + (lane >> 2);
+                        const float mu = ch < dr ? __ldg(a.mu + (size_t)m * (2 * dr + 1) + ch) : 0.f;
                         nmu2[g][c] = f2_pack(-mu, -mu);
                     }
                 }
@@ -332,14 +346,14 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
             // layout: [source | target][pair pp] for the low and the high half of the head.
             uint64_t rmlo[2][2] = {{0ull, 0ull}, {0ull, 0ull}}, rmhi[2][2] = {{0ull, 0ull}, {0ull, 0ull}};
             if (CEN && rope_unit) {
-                const float *mup = a.mu + (size_t)m * (2 * D + 1);
+                const float *mup = a.mu + (size_t)m * (2 * dr + 1);
 #pragma unroll
                 for (int xyi = 0; xyi < 2; ++xyi)
 #pragma unroll
                     for (int pp = 0; pp < 2; ++pp) {
-                        const float *b = mup + xyi * D + rc * 4 + 2 * pp;
+                        const float *b = mup + xyi * dr + rc * 4 + 2 * pp;
                         rmlo[xyi][pp] = f2_pack(-__ldg(b), -__ldg(b + 1));
-                        rmhi[xyi][pp] = f2_pack(-__ldg(b + D / 2), -__ldg(b + D / 2 + 1));
+                        rmhi[xyi][pp] = f2_pack(-__ldg(b + dr / 2), -__ldg(b + dr / 2 + 1));
                     }
             }
             for (int t = 0; t < n_t; ++t) {
@@ -359,12 +373,13 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                     constexpr int NI = C::TT / 16;
                     // positions of this thread's rows; `contig`: they advance by 16 from row to row (the common case:
                     // no sequence boundary inside the tile), decided once so that the row loop has no branches
+                    constexpr int ni = narrow ? NI / 2 : NI;  // passes of this thread
                     int posv[NI];
 #pragma unroll
-                    for (int i = 0; i < NI; ++i) posv[i] = pt[16 * i];
+                    for (int i = 0; i < NI; ++i) posv[i] = (i < ni) ? pt[rstep * i] : 0;
                     bool contig = true;
 #pragma unroll
-                    for (int i = 1; i < NI; ++i) contig = contig && (posv[i] == posv[0] + 16 * i);
+                    for (int i = 1; i < NI; ++i) contig = contig && (i >= ni || posv[i] == posv[0] + rstep * i);
                     uint64_t cc2[2], ss2[2];
                     if ((t == 0) || (posv[0] != seedpos + C::TT) || ((t & 15) == 0)) {
 #pragma unroll
@@ -387,7 +402,8 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                                            const uint64_t (&ys)[2]) {
 #pragma unroll
                         for (int xyi = 0; xyi < 2; ++xyi) {
-                            uint8_t *lo = xt + xyi * 2 * C::BLK + i * (16 * 128), *hi = lo + C::BLK;
+                            uint8_t *lo = xt + xyi * 2 * C::BLK + i * (rstep * 128);
+                            uint8_t *hi = narrow ? reinterpret_cast<uint8_t *>(reinterpret_cast<uintptr_t>(lo) ^ 64) : lo + C::BLK;
                             const uint2 vl = *reinterpret_cast<const uint2 *>(lo), vh = *reinterpret_cast<const uint2 *>(hi);
                             const unsigned ul[2] = {vl.x, vl.y}, uh[2] = {vh.x, vh.y};
                             unsigned ol[2], oh[2];
@@ -418,6 +434,7 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                     if (contig && P.rope.same) {
 #pragma unroll
                         for (int i = 0; i < NI; ++i) {
+                            if (i >= ni) break;
                             if (i > 0) {
 #pragma unroll
                                 for (int pp = 0; pp < 2; ++pp) {    // angle += 16 theta
@@ -430,10 +447,10 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                         }
                     } else {
 #pragma unroll 1
-                        for (int i = 0; i < NI; ++i) {
-                            const int pos = pt[16 * i];
+                        for (int i = 0; i < ni; ++i) {
+                            const int pos = pt[rstep * i];
                             if (i > 0) {
-                                if (pos == pt[16 * (i - 1)] + 16) {
+                                if (pos == pt[rstep * (i - 1)] + rstep) {
 #pragma unroll
                                     for (int pp = 0; pp < 2; ++pp) {
                                         const uint64_t pc = cc2[pp], ps = ss2[pp];
@@ -535,14 +552,14 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
             if (lane == 0) mbar_arrive(redfull);
             if (fw < 4) {
                 if (!mbar_wait_warp(redfull, uc & 1, abort_flag, lane)) goto teardown;
-                float *slot = a.slots + ((size_t)split * n_maps + m) * slot_floats(D);
+                float *slot = a.slots + ((size_t)split * n_maps + m) * slot_floats(dr);
                 const int v = fw * 32 + lane;
-                slot[slot_sx(D) + v] += redx[v] + redx[D + v];
+                if (v < dr) slot[slot_sx(dr) + v] += redx[v] + redx[D + v];
                 if (v == 0) {
                     float sum = 0.f;
 #pragma unroll
                     for (int k = 0; k < C::FOLD_WARPS; ++k) sum += red[k];
-                    slot[slot_sw(D)] += sum;
+                    slot[slot_sw(dr)] += sum;
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(reddone);
@@ -559,8 +576,8 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
         UnitIter cur;
         cur.start(a, n_units, n_maps, n_tiles);
         while (cur.valid(n_units)) {
-            float *slot = a.slots + ((size_t)cur.split * n_maps + cur.m) * slot_floats(D);
-            float *grow = slot + (size_t)row * C::N;
+            float *slot = a.slots + ((size_t)cur.split * n_maps + cur.m) * slot_floats(dr);
+            float *grow = slot + (size_t)row * (2 * dr);             // row of the slot's [dr][2 dr] block
             for (int sr0 = cur.tile; sr0 < cur.tile1; sr0 += P.drain_tiles, ++sr) {
                 if (!mbar_wait_warp(accfull, sr & 1, abort_flag, lane)) goto teardown;
                 tc_fence_after();
@@ -576,13 +593,18 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
                         __syncwarp();
                         if (lane == 0) mbar_arrive(accempty);
                     }
+                    // accumulator columns [0, D) are the source channels, [D, 2 D) the target channels; of each half
+                    // the first dr columns are real, and so are the first dr rows
+                    const int col = c * 32, half = col / D, cin = col % D;
+                    if (row < dr && cin < dr) {
 #pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        red_add_f32x4(grow + c * 32 + v * 4, __uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                      __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                        for (int v = 0; v < 8; ++v)
+                            red_add_f32x4(grow + half * dr + cin + v * 4, __uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                          __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                    }
                 }
                 // D_sy columns 0 and 1: the w_hi and w_lo columns of wb
-                if (!CEN) atomicAdd(slot + slot_sy(D) + row, __uint_as_float(b[0]) + __uint_as_float(b[1]));
+                if (!CEN && row < dr) atomicAdd(slot + slot_sy(dr) + row, __uint_as_float(b[0]) + __uint_as_float(b[1]));
             }
             cur.next_unit(a, n_units, n_maps, n_tiles);
         }
@@ -605,37 +627,39 @@ teardown:
     }
 }
 
-template <bool COMP, bool CEN, bool ROPE = false>
+template <bool COMP, bool CEN, bool ROPE = false, bool NARROW = false>
 cudaError_t launch_ts(const TsParams &P, cudaStream_t st)
 {
     using C = TsCfg<COMP>;
     static bool attr[MAX_DEVICES] = {};
     {
-        cudaError_t e = opt_in_smem(k_accum_ts<COMP, CEN, ROPE>, (size_t)((int)C::SMEM_BYTES), attr);
+        cudaError_t e = opt_in_smem(k_accum_ts<COMP, CEN, ROPE, NARROW>, (size_t)((int)C::SMEM_BYTES), attr);
         if (e != cudaSuccess) return e;
     }
     const int n_units = 2 * P.a.Lt * P.a.Ht * P.a.n_splits;
     const int grid = n_units < device_sm_count() ? n_units : device_sm_count();
-    k_accum_ts<COMP, CEN, ROPE><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
+    k_accum_ts<COMP, CEN, ROPE, NARROW><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(P);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-// d = 128.  `comp`: hi + lo weighted operand.
-cudaError_t launch_accum_ts(const AccumArgs &a, bool comp, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st)
+// d = 128 or 64.  `comp`: hi + lo weighted operand.
+cudaError_t launch_accum_ts(const AccumArgs &a, int d, bool comp, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st)
 {
     TsParams P;
     P.a = a;
-    const int d = 128, TT = comp ? TsCfg<true>::TT : TsCfg<false>::TT;
+    P.d = d;
+    const int TT = comp ? TsCfg<true>::TT : TsCfg<false>::TT;
+    // the copy box always spans two 64-channel blocks: for d = 64 the second one is outside the tensor and arrives as zeros
     if (!make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
-                            src->stride_token, src->stride_layer, TT) ||
+                            src->stride_token, src->stride_layer, TT, 2) ||
         !make_kv_tensor_map(&P.src_v, src->v, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
-                            src->stride_token, src->stride_layer, TT) ||
+                            src->stride_token, src->stride_layer, TT, 2) ||
         !make_kv_tensor_map(&P.tgt_k, tgt->k, d, tgt->n_heads, tgt->n_tokens, tgt->n_layers, tgt->stride_head,
-                            tgt->stride_token, tgt->stride_layer, TT) ||
+                            tgt->stride_token, tgt->stride_layer, TT, 2) ||
         !make_kv_tensor_map(&P.tgt_v, tgt->v, d, tgt->n_heads, tgt->n_tokens, tgt->n_layers, tgt->stride_head,
-                            tgt->stride_token, tgt->stride_layer, TT))
+                            tgt->stride_token, tgt->stride_layer, TT, 2))
         return cudaErrorInvalidValue;
     // Tokens summed in tensor memory before a drain.  The tensor cores' fp32 accumulation loses about 1e-4 (relative,
     // on the all-positive sums of G) over 16,384 tokens; the compensated fold drains eight times as often, so that
@@ -648,7 +672,10 @@ cudaError_t launch_accum_ts(const AccumArgs &a, bool comp, const cb_kv_view *src
         rope_frequencies(a.rope_base_src, d, P.rope.f_src);
         rope_frequencies(a.rope_base_tgt, d, P.rope.f_tgt);
         P.rope.same = (a.rope_base_src == a.rope_base_tgt) ? 1 : 0;
-        if (a.mu) e = comp ? launch_ts<true, true, true>(P, st) : launch_ts<false, true, true>(P, st);
+        if (d == 64) {
+            if (a.mu) e = comp ? launch_ts<true, true, true, true>(P, st) : launch_ts<false, true, true, true>(P, st);
+            else e = comp ? launch_ts<true, false, true, true>(P, st) : launch_ts<false, false, true, true>(P, st);
+        } else if (a.mu) e = comp ? launch_ts<true, true, true>(P, st) : launch_ts<false, true, true>(P, st);
         else e = comp ? launch_ts<true, false, true>(P, st) : launch_ts<false, false, true>(P, st);
     } else if (a.mu) e = comp ? launch_ts<true, true>(P, st) : launch_ts<false, true>(P, st);
     else e = comp ? launch_ts<true, false>(P, st) : launch_ts<false, false>(P, st);

@@ -279,7 +279,6 @@ static cb_status accumulate_impl(cb_ctx *ctx, const cb_kv_view *src, const cb_kv
     if (!ctx || ctx->magic != CTX_MAGIC) return CB_ERR_STATE;
     if (centred && !mu) return CB_ERR_INVALID_ARG;
     if (centred && (ctx->prob.flags & CB_FLAG_SIMT)) return CB_ERR_UNSUPPORTED;
-    if (centred && rope && ctx->d != 128) return CB_ERR_UNSUPPORTED;      // the combination exists for d = 128 only
     const cb_problem &P = ctx->prob;
     cb_status s = check_view(src, P.Ls, P.Hs, P.ds);
     if (s != CB_OK) return s;

@@ -100,7 +100,7 @@ struct FullHeadArgs {
 // Launchers (each returns the cudaError_t of its launch and bumps the launch counter on success).
 cudaError_t launch_accum_simt(const AccumArgs &a, int d, cudaStream_t st);
 cudaError_t launch_accum_tc(const AccumArgs &a, int d, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st);
-cudaError_t launch_accum_ts(const AccumArgs &a, bool comp, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st);
+cudaError_t launch_accum_ts(const AccumArgs &a, int d, bool comp, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st);
 cudaError_t launch_fullhead_tc(const AccumArgs &a, const FullHeadArgs &f, int d, const cb_kv_view *src, const cb_kv_view *tgt,
                                cudaStream_t st);
 cudaError_t launch_gram2_tc(const AccumArgs &a, const FullHeadArgs &f, int d, const cb_kv_view *src, const cb_kv_view *tgt,

@@ -73,7 +73,8 @@ def _oracle_rope_stats(ch, pos, sl, sh, wl, maps, base_s, base_t):
 
 
 @pytest.mark.parametrize("name,flags,bases", [("mid_scaled", 0, (1e6, 1e6)), ("mid_scaled", 0, (1e6, 1e4)),
-                                               ("mini_scaled", cb.CB_FLAG_COMPENSATED, (1e6, 5e5)), ("tiny", 0, (1e4, 1e4))])
+                                               ("mini_scaled", cb.CB_FLAG_COMPENSATED, (1e6, 5e5)), ("tiny", 0, (1e4, 1e4)),
+                                               ("tiny", 0, (1e4, 5e5)), ("tiny", cb.CB_FLAG_COMPENSATED, (1e4, 1e4))])
 def test_fused_statistics_in_content_coordinates(name, flags, bases):
     wl = synth.workload(name)
     sl, sh = cb.cb_head_map_nearest(wl.Ls, wl.Hs, wl.Lt, wl.Ht)
@@ -313,7 +314,7 @@ def test_fused_statistics_few_rows_and_position_breaks(T):
 
 
 @pytest.mark.parametrize("name,flags,bases", [("mid_scaled", 0, (1e6, 1e6)), ("mini_scaled", cb.CB_FLAG_COMPENSATED, (1e6, 1e4)),
-                                               ("mini_ragged", 0, (1e6, 1e6))])
+                                               ("mini_ragged", 0, (1e6, 1e6)), ("tiny", 0, (1e4, 1e4))])
 def test_two_pass_construction_in_content_coordinates(name, flags, bases):
     """The paper's own construction path (Section 3.4: weighted means, centred statistics, centred solve) with the
     rotary boundary (Section 3.1): both passes see the keys with the embedding removed.  The keys get a channel mean
