@@ -75,9 +75,6 @@ struct TsParams {
     CUtensorMap src_k, src_v, tgt_k, tgt_v;   // 5-D tiled maps: (64 channels, token, channel block, head, layer)
     AccumArgs a;
     int drain_tiles;                          // tiles accumulated in tensor memory between drains
-    int d;                                    // the heads' real width, 128 or 64.  A 64-wide head runs as a 128-wide one
-                                              // whose upper channel block lies outside the tensor (the tile copies fill
-                                              // it with zeros); only the results of the real channels leave the kernel.
     RopeDev rope;                             // ROPE kernels only
 };
 
@@ -120,7 +117,8 @@ struct UnitIter {
 // ROPE: key maps (comp = 0) are fitted in content coordinates (Section 3.1): before the fold proper, the fold warps
 // rotate every source and target key row of the staged tile back by its position's angles IN PLACE (the tensor cores
 // read the de-rotated rows as the second operand and for s_y); value maps take the ordinary path.
-// NARROW (ROPE kernels, 64-wide heads): the rotation pairs channel i with i + 32 inside the first 64-channel block.
+// NARROW: 64-wide heads (the upper 64-channel block of every tile is zero padding); the rotation then pairs channel i
+// with i + 32 inside the first block.
 template <bool COMP, bool CEN, bool ROPE, bool NARROW = false>
 __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __grid_constant__ TsParams P)
 {
@@ -146,7 +144,7 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const AccumArgs &a = P.a;
-    const int dr = P.d;                    // real head width: channels dr .. D - 1 are zero padding
+    constexpr int dr = NARROW ? 64 : D;    // real head width: channels dr .. D - 1 are zero padding
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_maps = 2 * a.Lt * a.Ht;
     const int n_units = n_maps * a.n_splits;
@@ -297,7 +295,6 @@ __global__ void __launch_bounds__(TsCfg<COMP>::THREADS, 1) k_accum_ts(const __gr
         // A 64-wide head pairs channel i with i + 32, both in the tile's first 64-channel block (the second one is zero
         // padding): eight threads per row instead of sixteen, so a pass covers 32 rows and there are half as many
         // passes; in the swizzled row the partner chunk is the own one with address bit 6 flipped.
-        static_assert(ROPE || !NARROW, "NARROW selects the rotation's pairing");
         constexpr bool narrow = NARROW;
         const int rc = narrow ? (tid - 64) & 7 : (tid - 64) & 15, rr = narrow ? (tid - 64) >> 3 : (tid - 64) >> 4;
         constexpr int rstep = narrow ? 32 : 16;                     // rows (and positions) between a thread's passes
@@ -644,12 +641,22 @@ cudaError_t launch_ts(const TsParams &P, cudaStream_t st)
 
 }  // namespace
 
+template <bool NARROW>
+static cudaError_t launch_variant(const TsParams &P, bool comp, bool cen, bool rope, cudaStream_t st)
+{
+    if (rope) {
+        if (cen) return comp ? launch_ts<true, true, true, NARROW>(P, st) : launch_ts<false, true, true, NARROW>(P, st);
+        return comp ? launch_ts<true, false, true, NARROW>(P, st) : launch_ts<false, false, true, NARROW>(P, st);
+    }
+    if (cen) return comp ? launch_ts<true, true, false, NARROW>(P, st) : launch_ts<false, true, false, NARROW>(P, st);
+    return comp ? launch_ts<true, false, false, NARROW>(P, st) : launch_ts<false, false, false, NARROW>(P, st);
+}
+
 // d = 128 or 64.  `comp`: hi + lo weighted operand.
 cudaError_t launch_accum_ts(const AccumArgs &a, int d, bool comp, const cb_kv_view *src, const cb_kv_view *tgt, cudaStream_t st)
 {
     TsParams P;
     P.a = a;
-    P.d = d;
     const int TT = comp ? TsCfg<true>::TT : TsCfg<false>::TT;
     // the copy box always spans two 64-channel blocks: for d = 64 the second one is outside the tensor and arrives as zeros
     if (!make_kv_tensor_map(&P.src_k, src->k, d, src->n_heads, src->n_tokens, src->n_layers, src->stride_head,
@@ -672,13 +679,10 @@ cudaError_t launch_accum_ts(const AccumArgs &a, int d, bool comp, const cb_kv_vi
         rope_frequencies(a.rope_base_src, d, P.rope.f_src);
         rope_frequencies(a.rope_base_tgt, d, P.rope.f_tgt);
         P.rope.same = (a.rope_base_src == a.rope_base_tgt) ? 1 : 0;
-        if (d == 64) {
-            if (a.mu) e = comp ? launch_ts<true, true, true, true>(P, st) : launch_ts<false, true, true, true>(P, st);
-            else e = comp ? launch_ts<true, false, true, true>(P, st) : launch_ts<false, false, true, true>(P, st);
-        } else if (a.mu) e = comp ? launch_ts<true, true, true>(P, st) : launch_ts<false, true, true>(P, st);
-        else e = comp ? launch_ts<true, false, true>(P, st) : launch_ts<false, false, true>(P, st);
-    } else if (a.mu) e = comp ? launch_ts<true, true>(P, st) : launch_ts<false, true>(P, st);
-    else e = comp ? launch_ts<true, false>(P, st) : launch_ts<false, false>(P, st);
+    }
+    const bool rope = a.rope_pos != nullptr, cen = a.mu != nullptr;
+    if (d == 64) e = launch_variant<true>(P, comp, cen, rope, st);
+    else e = launch_variant<false>(P, comp, cen, rope, st);
     if (e == cudaSuccess) count_launch();
     return e;
 }
