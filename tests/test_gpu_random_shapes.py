@@ -143,3 +143,82 @@ def test_random_shape_against_the_oracle(seed):
     # the de-rotated rows are rounded to bf16 on chip: 1e-3 needs a few thousand rows per map, below that 2.5e-3
     tol = 1e-3 if T >= 4096 else 2.5e-3
     assert worst_g <= tol and worst_c <= tol
+
+
+@pytest.mark.parametrize("seed", list(range(6)))
+def test_random_shape_wide_regressor_paths(seed):
+    """Head-local support over k layers (statistics, wide solve, apply) and the full-head statistics on random shapes:
+    odd k, more or fewer source than target heads, both head widths (64-wide heads take the one-row-head kernel),
+    token counts that end inside a tile."""
+    rng = np.random.default_rng(3000 + seed)
+    d = int(rng.choice([64, 128]))
+    Ls, Lt = int(rng.integers(2, 7)), int(rng.integers(1, 4))
+    Hs, Ht = int(rng.choice([1, 2, 3])), int(rng.choice([1, 2, 3, 4]))
+    k = int(rng.integers(1, min(Ls, 5) + 1))
+    lens = tuple(int(x) for x in rng.integers(40, 900, size=int(rng.integers(1, 4))))
+    wl = synth.Workload("randomwide%d" % seed, 200 + seed, Ls, Hs, Lt, Ht, d, lens, len(lens), (1e-2,), "scaled", 0.1, seed=seed)
+    sl, sh = oracle.head_map(Ls, Hs, Lt, Ht)
+    sets = cb.cb_fullhead_layer_sets(Ls, Lt, k)
+    assert np.array_equal(sets, oracle.fullhead_layer_sets(Ls, Lt, k))
+    ch = synth.make_chunk(wl, 0, sl, sh)
+    T, nm = ch["n_tokens"], wl.n_maps
+    t = {k_: v.to(DEV) for k_, v in ch.items() if torch.is_tensor(v)}
+    flags = cb.CB_FLAG_ONE_ROW_HEAD if seed % 3 == 2 else 0
+    prob = cb.FullHeadProblem(Ls, Hs, d, Lt, Ht, d, sets, flags=flags)
+    P = k * d + 1
+    G = torch.zeros(nm, P, P, device=DEV)
+    C = torch.zeros(nm, P, d, device=DEV)
+    cb.cb_multilayer_stats_accumulate(prob, sh, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], t["w_k"], t["w_v"], G, C)
+    cb.cb_last_device_status()
+    Gc, Cc = G.cpu().numpy(), C.cpu().numpy()
+    assert np.isfinite(Gc).all() and np.isfinite(Cc).all()
+    lam = 1e-1
+    ws = torch.empty(cb.cb_ridge_solve_large_workspace_bytes(P, d, 3), dtype=torch.uint8, device=DEV)
+    Wb = torch.full((1, nm, P, d), float("nan"), device=DEV)
+    info = torch.full((1, nm), -1, dtype=torch.int32, device=DEV)
+    cb.cb_ridge_solve_large(G, C, T, [lam], 0, Wb, info, ws)
+    cb.cb_check_info(info)
+    Wc = Wb.cpu().numpy()[0]
+    worst = [0.0, 0.0, 0.0]
+    for m in sorted(set([0, nm // 2, nm - 1, int(rng.integers(0, nm))])):
+        comp, l, h = m // (Lt * Ht), (m // Ht) % Lt, m % Ht
+        g, c = oracle.multilayer_stats(bits(ch["src_v" if comp else "src_k"]), bits(ch["tgt_v" if comp else "tgt_k"]),
+                                       (ch["w_v"] if comp else ch["w_k"])[l, h].contiguous().numpy(), l, h, int(sh[h]), sets[l])
+        Ts, i0 = oracle.ridge_solve_general(Gc[m].astype(np.float64), Cc[m].astype(np.float64), T, lam)
+        worst = [max(worst[0], rel_fro(Gc[m], g)), max(worst[1], rel_fro(Cc[m], c)), max(worst[2], rel_fro(Wc[m], Ts))]
+        assert i0 == 0
+    print("seed %d: Ls %d Hs %d Lt %d Ht %d d %d k %d T %d flags %d: G %.2e C %.2e solver %.2e" % (
+        seed, Ls, Hs, Lt, Ht, d, k, T, flags, *worst))
+    assert worst[0] <= 2e-3 and worst[1] <= 2e-3 and worst[2] <= 1e-5       # plain bf16 fold below 4,096 rows: 2e-3
+    # apply with maps of the right scale, fp32 out
+    Wr = torch.from_numpy((rng.standard_normal((nm, P, d)) / np.sqrt(P)).astype(np.float32)).to(DEV)
+    ok = torch.full((Lt, T, Ht, d), float("nan"), device=DEV)
+    ov = torch.full_like(ok, float("nan"))
+    cb.cb_apply_multilayer(prob, sh, Wr, t["src_k"], t["src_v"], ok, ov)
+    cb.cb_last_device_status()
+    okc, ovc = ok.cpu().numpy(), ov.cpu().numpy()
+    Wn = Wr.cpu().numpy().astype(np.float64)
+    for m in (0, nm - 1):
+        comp, l, h = m // (Lt * Ht), (m // Ht) % Lt, m % Ht
+        ref, _ = oracle.apply_multilayer(bits(ch["src_v" if comp else "src_k"]), Wn[m], sets[l], int(sh[h]))
+        got = (ovc if comp else okc)[l, :, h, :]
+        assert rel_fro(got, ref) <= 1e-5
+    # full-head statistics of the same traces: weights per (layer, token)
+    fprob = cb.FullHeadProblem(Ls, Hs, d, Lt, Ht, d, sets, flags=flags)
+    if (k * Hs) % 2:                       # the full-head entry point takes an even number of feature heads (stated in the header)
+        with pytest.raises(cb.CbError) as err:
+            cb.cb_fullhead_workspace_bytes(fprob)
+        assert err.value.status == cb.CB_ERR_UNSUPPORTED
+        return
+    pf = fprob.pf
+    Gf = torch.zeros(2, Lt, pf, pf, device=DEV)
+    Cf = torch.zeros(2, Lt, Ht, pf, d, device=DEV)
+    wk, wv = t["w_k"][:, 0].contiguous(), t["w_v"][:, 0].contiguous()
+    cb.cb_fullhead_stats_accumulate(fprob, t["src_k"], t["src_v"], t["tgt_k"], t["tgt_v"], wk, wv, Gf, Cf)
+    cb.cb_last_device_status()
+    for comp, l in ((0, 0), (1, Lt - 1)):
+        g, c = oracle.fullhead_stats(bits(ch["src_v" if comp else "src_k"]), bits(ch["tgt_v" if comp else "tgt_k"]),
+                                     (ch["w_v"] if comp else ch["w_k"])[l, 0].contiguous().numpy(), l, sets[l])
+        eg, ec = rel_fro(Gf[comp, l].cpu().numpy(), g), rel_fro(Cf[comp, l].cpu().numpy(), c)
+        print("   full-head (comp %d, layer %d), width %d: G %.2e C %.2e" % (comp, l, pf, eg, ec))
+        assert eg <= 2e-3 and ec <= 2e-3
