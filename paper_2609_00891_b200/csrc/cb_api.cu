@@ -792,7 +792,7 @@ static cb_status check_fullhead(const cb_fullhead_problem *p)
     if (p->Ls <= 0 || p->Hs <= 0 || p->Lt <= 0 || p->Ht <= 0 || p->k <= 0 || p->k > p->Ls) return CB_ERR_INVALID_ARG;
     if (p->ds != p->dt || (p->ds != 64 && p->ds != 128)) return CB_ERR_UNSUPPORTED;
     const int F = p->k * p->Hs;
-    if ((F & 1) || F > 64) return CB_ERR_UNSUPPORTED;
+    if (F > 64) return CB_ERR_UNSUPPORTED;
     for (int i = 0; i < p->Lt * p->k; ++i)
         if (p->layer_sets[i] < 0 || p->layer_sets[i] >= p->Ls) return CB_ERR_INVALID_ARG;
     return CB_OK;
