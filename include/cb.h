@@ -255,8 +255,8 @@ cb_status cb_ess_weights(const float *r_raw, int32_t n_rows, int64_t n_tokens, i
  * lower triangle over the upper one; with CB_FLAG_ONE_ROW_HEAD the d x d diagonal blocks are left as computed).
  * w_k / w_v: device fp32 [Lt][n_tokens] at w + l*w_stride_layer + t.  layer_sets: HOST [Lt][k], ascending layers in
  * [0, Ls-1]; k*Hs <= 64 (an odd number of feature heads is fine).  workspace: device, 256-byte aligned,
- * cb_fullhead_workspace_bytes() (small
- * index tables, copied inside the call).  Same stream/ownership/error rules as cb_stats_accumulate; no context.
+ * cb_fullhead_workspace_bytes() (small index tables, copied inside the call).  Same stream/ownership/error rules as
+ * cb_stats_accumulate; no context.
  */
 typedef struct cb_fullhead_problem {
     int32_t Ls, Hs, ds;
