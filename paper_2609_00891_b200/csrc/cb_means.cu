@@ -248,7 +248,8 @@ cudaError_t launch_means_finalize(const double *msum, int n_maps, int d, float *
 }
 
 // Same split summation as the one-pass reduction, then the rank-one corrections and the symmetrisation of A.
-__global__ void __launch_bounds__(1024) k_reduce_centered(const float *__restrict__ slots, int n_splits, int n_maps, int d,
+template <int d>
+__global__ void __launch_bounds__(1024) k_reduce_centered(const float *__restrict__ slots, int n_splits, int n_maps,
                                                          const float *__restrict__ mu, float *__restrict__ A,
                                                          float *__restrict__ B, int k_operands_centred)
 {
@@ -292,11 +293,16 @@ cudaError_t launch_reduce_centered(const float *slots, int n_splits, int n_maps,
 {
     const size_t smem = sizeof(float) * ((size_t)d * (2 * d + 1) + 2 * d + 4 + 2 * d);
     static bool attr[MAX_DEVICES] = {};
-    {
-        cudaError_t e = opt_in_smem(k_reduce_centered, (size_t)(140 * 1024), attr);
+    static bool attr64[MAX_DEVICES] = {};
+    if (d == 128) {
+        cudaError_t e = opt_in_smem(k_reduce_centered<128>, (size_t)(140 * 1024), attr);
         if (e != cudaSuccess) return e;
+        k_reduce_centered<128><<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, mu, A, B, k_operands_centred);
+    } else {
+        cudaError_t e = opt_in_smem(k_reduce_centered<64>, (size_t)(140 * 1024), attr64);
+        if (e != cudaSuccess) return e;
+        k_reduce_centered<64><<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, mu, A, B, k_operands_centred);
     }
-    k_reduce_centered<<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, d, mu, A, B, k_operands_centred);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;

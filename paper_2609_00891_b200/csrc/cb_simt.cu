@@ -132,12 +132,16 @@ cudaError_t launch_accum_simt(const AccumArgs &a, int d, cudaStream_t st)
 // (fp32, padded rows); G and C are then written from that image, the transpose needed for the
 // symmetrisation being a shared-memory access.
 // ======================================================================================================
-__global__ void __launch_bounds__(1024) k_reduce(const float *__restrict__ slots, int n_splits, int n_maps, int d,
+// The head width is a template parameter: every index of the two output loops is a division by d, 2 d or d + 1, and
+// with run-time divisors those divisions were most of the kernel's instructions.
+template <int d>
+__global__ void __launch_bounds__(1024) k_reduce(const float *__restrict__ slots, int n_splits, int n_maps,
                                                 float *__restrict__ G, float *__restrict__ C)
 {
     extern __shared__ __align__(16) float rs[];       // [d][2d + 1] sums of D, then [2d + 1] sums of s_x, s_y, s_w
-    const int m = blockIdx.x, p = d + 1, n2 = 2 * d, pitch = 2 * d + 1;
-    const int sf = slot_floats(d);
+    constexpr int p = d + 1, n2 = 2 * d, pitch = 2 * d + 1;
+    const int m = blockIdx.x;
+    constexpr int sf = slot_floats(d);
     const float *base = slots + (size_t)m * sf;
     const size_t sstride = (size_t)n_maps * sf;
     // sum the splits four floats at a time (slots are 16-byte aligned and sf is a multiple of 4); the slot's last
@@ -177,11 +181,16 @@ cudaError_t launch_reduce(const float *slots, int n_splits, int n_maps, int d, f
 {
     const size_t smem = sizeof(float) * ((size_t)d * (2 * d + 1) + 2 * d + 4);
     static bool attr[MAX_DEVICES] = {};
-    {
-        cudaError_t e = opt_in_smem(k_reduce, (size_t)(140 * 1024), attr);
+    static bool attr64[MAX_DEVICES] = {};
+    if (d == 128) {
+        cudaError_t e = opt_in_smem(k_reduce<128>, (size_t)(140 * 1024), attr);
         if (e != cudaSuccess) return e;
+        k_reduce<128><<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, G, C);
+    } else {
+        cudaError_t e = opt_in_smem(k_reduce<64>, (size_t)(140 * 1024), attr64);
+        if (e != cudaSuccess) return e;
+        k_reduce<64><<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, G, C);
     }
-    k_reduce<<<n_maps, 1024, smem, st>>>(slots, n_splits, n_maps, d, G, C);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;
