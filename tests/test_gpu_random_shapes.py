@@ -140,6 +140,20 @@ def test_random_shape_against_the_oracle(seed):
         g, c = oracle.stats_f64(X, Y, wk[l, h].astype(np.float64))
         worst_g, worst_c = max(worst_g, rel_fro(Gc[m], g)), max(worst_c, rel_fro(Cc[m], c))
     print("   rotary boundary (bases %g, %g): key maps G %.2e C %.2e" % (base_s, base_t, worst_g, worst_c))
+    # apply across the boundary on the stored (rotated) keys, fp32 out: de-rotate, map, re-embed with the target base
+    okr = torch.full((wl.Lt, T, wl.Ht, d), float("nan"), device=DEV)
+    ovr = torch.full_like(okr, float("nan"))
+    cb.cb_apply_rope(prob, Wr, t["src_k"], t["src_v"], okr, ovr, torch.from_numpy(pos).to(DEV), base_s, base_t)
+    cb.cb_last_device_status()
+    assert torch.equal(ovr, ov)                                           # value maps: the ordinary apply
+    Wn = Wr.cpu().numpy().astype(np.float64)
+    worst_a = 0.0
+    for m in range(half):
+        l, h = m // wl.Ht, m % wl.Ht
+        want = oracle.apply_rope_rows(np.ascontiguousarray(B[0][sl[l], :, sh[h], :]), Wn[m], pos, base_s, base_t)
+        worst_a = max(worst_a, rel_fro(okr[l, :, h, :].cpu().numpy(), want))
+    print("   apply across the boundary: worst key map %.2e" % worst_a)
+    assert worst_a <= 1e-3                                                # fp16 operands on chip (11 significant bits)
     # the de-rotated rows are rounded to bf16 on chip: 1e-3 needs a few thousand rows per map, below that 2.5e-3
     tol = 1e-3 if T >= 4096 else 2.5e-3
     assert worst_g <= tol and worst_c <= tol
